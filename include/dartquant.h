@@ -1,0 +1,137 @@
+/*
+ * dartquant.h -- C ABI of the B200 (sm_100a) rotational-distribution-calibration
+ * library.
+ *
+ * One calibration iteration is the loop body of Algorithm 1 of the DartQuant
+ * paper: R <- Q factor of qr(Z) (QR-Orth, Sec. 4.3 / Algorithm 2), O <- X R,
+ * L <- Whip(O) (Eq. 4), Z <- Z - eta dL/dZ.  Every step runs in CUDA kernels of
+ * this library; there is no CPU fallback.
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.
+ *   - Matrices are row-major.  X is [batch][n_tokens][ldx] (one token per row),
+ *     latents / rotations are [batch][d][d] fp32.
+ *   - Every call returns a dq_status; nothing throws, aborts or traps.  Device
+ *     side problems (rank-deficient latent, non-finite loss, a wait that ran
+ *     out) are recorded in a device status word read by dq_calib_status().
+ *   - All work is enqueued on the stream given at init; calls are asynchronous
+ *     with respect to the host unless stated otherwise.
+ *   - Notation: R is always the rotation (the orthogonal factor of Z = R U),
+ *     U the upper-triangular factor with positive diagonal.
+ */
+#ifndef DARTQUANT_H_
+#define DARTQUANT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dq_calib dq_calib_t; /* opaque, owned by the library */
+
+typedef enum {
+  DQ_OK = 0,
+  DQ_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad enum          */
+  DQ_ERR_UNSUPPORTED = 2, /* shape / dtype / path combination not implemented   */
+  DQ_ERR_ALLOC = 3,       /* device allocation failed                           */
+  DQ_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed                  */
+  DQ_ERR_SINGULAR = 5,    /* latent is (numerically) rank deficient: U^-T undefined */
+  DQ_ERR_NONFINITE = 6,   /* loss became NaN/Inf                                */
+  DQ_ERR_TIMEOUT = 7      /* a bounded in-kernel wait gave up                   */
+} dq_status;
+
+enum { DQ_FP32 = 0, DQ_BF16 = 1 };             /* x_dtype                       */
+enum { DQ_PATH_FP32 = 0, DQ_PATH_BF16_TC = 1 }; /* arithmetic of the X R / X^T G contractions */
+enum { DQ_MEAN_TOKENS = 0, DQ_SUM_TOKENS = 1 }; /* reduction of Eq. 4 over token rows */
+enum { DQ_SGD = 0 };                           /* optimiser (Algorithm 1 line 10) */
+
+typedef struct {
+  int32_t d;         /* channels = size of the rotation; multiple of 32 (fp32 path) or 128 (tensor-core path); <= 8192 */
+  int64_t n_tokens;  /* tokens per problem; multiple of 32 (fp32 path) or 256 (tensor-core path) */
+  int32_t batch;     /* independent problems (e.g. attention heads); >= 1       */
+  int32_t x_dtype;   /* DQ_FP32 | DQ_BF16                                       */
+  int32_t path;      /* DQ_PATH_FP32: fp32 FMA contractions (needs DQ_FP32 X);
+                        DQ_PATH_BF16_TC: bf16 tensor-core contractions with fp32 accumulation (needs DQ_BF16 X) */
+  int32_t reduction; /* DQ_MEAN_TOKENS (default reading of Algorithm 1 line 9) | DQ_SUM_TOKENS */
+  int32_t optimizer; /* DQ_SGD                                                  */
+  float lr;          /* eta                                                     */
+  int64_t ldx;       /* row stride of X in elements (>= d); problems are n_tokens*ldx apart */
+} dq_calib_config;
+
+/* Algorithm 1 lines 3-5 hand-off: bind calibration activations and the initial
+ * latent.  d_X is BORROWED (must outlive the handle, is never written).  d_Z0
+ * ([batch][d][d] fp32) is COPIED.  cuda_stream is a cudaStream_t (NULL = legacy
+ * default stream).  Allocates every workspace the step needs.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALLOC, CUDA.  *out is NULL on error. */
+dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void* d_X,
+                        const float* d_Z0, void* cuda_stream);
+
+/* Algorithm 1 lines 6-11, exactly n_steps iterations.  d_loss_out (nullable) is a
+ * device array [n_steps][batch] fp32; entry k is L(Z_k), the loss BEFORE the
+ * k-th update.  No host synchronisation. */
+dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out);
+
+/* Sec. 4.3: the rotation of the CURRENT latent, i.e. the orthogonal factor of
+ * Z = R U with diag(U) > 0 (recomputed if the latent changed since the last
+ * factorisation).  d_R_out is caller-owned [batch][d][d] fp32. */
+dq_status dq_calib_get_rotation(dq_calib_t* h, float* d_R_out);
+
+/* Sec. 3 (Y = X R): apply a rotation to activations and materialise the result.
+ * x_dtype selects both the storage type of X / Y and the arithmetic (DQ_FP32:
+ * fp32 FMA; DQ_BF16: bf16 tensor cores, fp32 accumulation, bf16 output).
+ * X is [n][ldx], Y is [n][ldy], R is [d][d] fp32, all device, no aliasing. */
+dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d, int64_t ldx,
+                          const float* d_R, void* d_Y, int64_t ldy, void* cuda_stream);
+
+/* Checkpoint / resume of the optimised parameter (Algorithm 1 line 5: Z <- Z0). */
+dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out);
+dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z);
+
+/* Synchronises the stream and returns the device status word
+ * (DQ_OK / DQ_ERR_SINGULAR / DQ_ERR_NONFINITE / DQ_ERR_TIMEOUT) or DQ_ERR_CUDA. */
+dq_status dq_calib_status(dq_calib_t* h);
+
+/* Phase times of the most recent dq_calib_step call, averaged per step, in ms
+ * (synchronises).  Order: DQ_PHASE_*.  Writes min(n, DQ_PHASE_COUNT) entries
+ * of the HOST array ms_by_phase. */
+enum {
+  DQ_PHASE_QR_FORWARD = 0, /* factorisation, forming R, gauge, operand copies   */
+  DQ_PHASE_ROTATE_WHIP = 1, /* O = X R with the fused Eq. 4 epilogue + loss reduce */
+  DQ_PHASE_GRAD_ROTATION = 2, /* Gq = X^T G                                      */
+  DQ_PHASE_QR_BACKWARD = 3,
+  DQ_PHASE_UPDATE = 4,
+  DQ_PHASE_COUNT = 5
+};
+dq_status dq_calib_get_timings(dq_calib_t* h, float* h_ms_by_phase, int32_t n);
+/* Enable (1) / disable (0) per-phase CUDA-event timing inside dq_calib_step. */
+dq_status dq_calib_set_timing(dq_calib_t* h, int32_t enabled);
+
+/* Read-only views of the handle's device workspaces after a step, for tests and
+ * diagnostics.  *d_ptr is valid until the handle is destroyed. */
+enum {
+  DQ_BUF_R = 0,        /* fp32 [batch][d][d]  rotation used by the last step       */
+  DQ_BUF_U = 1,        /* fp32 [batch][d][d]  upper factor, positive diagonal      */
+  DQ_BUF_GQ = 2,       /* fp32 [batch][d][d]  dL/dR                                */
+  DQ_BUF_GZ = 3,       /* fp32 [batch][d][d]  dL/dZ                                */
+  DQ_BUF_G = 4,        /* dL/dO without the 1/N factor: fp32 [batch][N][d] (fp32 path)
+                          or bf16 channel-major [batch][d][N] (tensor-core path)   */
+  DQ_BUF_PARTIALS = 5, /* fp32 per-tile loss partial sums of the last step         */
+  DQ_BUF_Z = 6         /* fp32 [batch][d][d]  current latent                       */
+};
+dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int64_t* n_elems);
+
+/* Number of kernels this library launched through the handle so far. */
+int64_t dq_calib_launch_count(dq_calib_t* h);
+
+const char* dq_status_string(dq_status s);
+void dq_calib_destroy(dq_calib_t* h);
+
+/* Compile-time facts of the loaded library: returns a static string such as
+ * "dartquant-b200 sm_100a". */
+const char* dq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DARTQUANT_H_ */

@@ -1,0 +1,311 @@
+// C ABI: handle management, argument validation and the per-step schedule.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "tc_path.cuh"
+
+using namespace dq;
+
+struct dq_calib {
+  dq_calib_config cfg;
+  Ctx ctx;
+  const void* X = nullptr;
+  float* Z = nullptr;
+  float* R = nullptr;
+  float* U = nullptr;
+  float* Gq = nullptr;
+  float* Gz = nullptr;
+  float* gq_part = nullptr;     // fp32 path: split-K partials of Gq
+  int gq_ks = 1;
+  void* G = nullptr;            // fp32 [b][N][d] (fp32 path) or bf16 [b][d][N] (tensor-core path)
+  int64_t g_elems = 0;
+  float* partials = nullptr;
+  int n_partials = 0;           // per problem
+  float* loss_last = nullptr;   // [batch]
+  QrWorkspace ws;
+  TcState tc;                   // tensor-core path state (operand copies, tensor maps)
+  bool r_stale = true;
+  bool timing = false;
+  cudaEvent_t ev[DQ_PHASE_COUNT + 1] = {};
+  double ms_acc[DQ_PHASE_COUNT] = {};
+  int timed_steps = 0;
+};
+
+namespace {
+
+template <typename T>
+dq_status dev_alloc(T** p, int64_t n) {
+  *p = nullptr;
+  if (n <= 0) return DQ_OK;
+  return cudaMalloc((void**)p, sizeof(T) * (size_t)n) == cudaSuccess ? DQ_OK : DQ_ERR_ALLOC;
+}
+
+void free_all(dq_calib* h) {
+  if (!h) return;
+  tc_destroy(h->tc);
+  cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
+  cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->ctx.d_status);
+  cudaFree(h->ws.A); cudaFree(h->ws.V); cudaFree(h->ws.T); cudaFree(h->ws.W); cudaFree(h->ws.W2);
+  cudaFree(h->ws.Q); cudaFree(h->ws.Winv); cudaFree(h->ws.B); cudaFree(h->ws.S); cudaFree(h->ws.tmp);
+  for (auto& e : h->ev) if (e) cudaEventDestroy(e);
+  delete h;
+}
+
+dq_status validate(const dq_calib_config* c) {
+  if (!c) return DQ_ERR_INVALID_ARG;
+  if (c->d <= 0 || c->n_tokens <= 0 || c->batch <= 0 || c->ldx < c->d) return DQ_ERR_INVALID_ARG;
+  if (c->x_dtype != DQ_FP32 && c->x_dtype != DQ_BF16) return DQ_ERR_INVALID_ARG;
+  if (c->path != DQ_PATH_FP32 && c->path != DQ_PATH_BF16_TC) return DQ_ERR_INVALID_ARG;
+  if (c->reduction != DQ_MEAN_TOKENS && c->reduction != DQ_SUM_TOKENS) return DQ_ERR_INVALID_ARG;
+  if (c->optimizer != DQ_SGD) return DQ_ERR_INVALID_ARG;
+  if (!(c->lr == c->lr)) return DQ_ERR_INVALID_ARG;
+  if (c->d > 8192 || c->d % 64 != 0) return DQ_ERR_UNSUPPORTED;
+  if (c->path == DQ_PATH_FP32) {
+    if (c->x_dtype != DQ_FP32) return DQ_ERR_UNSUPPORTED;
+  } else {
+    if (c->x_dtype != DQ_BF16) return DQ_ERR_UNSUPPORTED;
+    if (c->d % 128 != 0 || c->n_tokens % 256 != 0 || c->ldx != c->d) return DQ_ERR_UNSUPPORTED;
+  }
+  return DQ_OK;
+}
+
+dq_status ensure_rotation(dq_calib* h) {
+  if (!h->r_stale) return DQ_OK;
+  DQ_CHECK(qr_forward(h->ctx, h->ws, h->Z, h->R, h->U, tc_rt_operand(h->tc), h->cfg.d, h->cfg.batch));
+  h->r_stale = false;
+  return DQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dq_version(void) { return "dartquant-b200 sm_100a"; }
+
+const char* dq_status_string(dq_status s) {
+  switch (s) {
+    case DQ_OK: return "ok";
+    case DQ_ERR_INVALID_ARG: return "invalid argument";
+    case DQ_ERR_UNSUPPORTED: return "unsupported shape, dtype or path";
+    case DQ_ERR_ALLOC: return "device allocation failed";
+    case DQ_ERR_CUDA: return "CUDA call failed";
+    case DQ_ERR_SINGULAR: return "latent matrix is rank deficient";
+    case DQ_ERR_NONFINITE: return "non-finite loss or factor";
+    case DQ_ERR_TIMEOUT: return "bounded in-kernel wait gave up";
+  }
+  return "unknown status";
+}
+
+dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void* d_X,
+                        const float* d_Z0, void* cuda_stream) {
+  if (!out) return DQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!d_X || !d_Z0) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK(validate(cfg));
+  int dev = 0, cc_major = 0, sms = 0;
+  DQ_CHECK_CUDA(cudaGetDevice(&dev));
+  DQ_CHECK_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+  DQ_CHECK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  if (cc_major != 10) return DQ_ERR_UNSUPPORTED;   // sm_100a code only
+
+  dq_calib* h = new (std::nothrow) dq_calib();
+  if (!h) return DQ_ERR_ALLOC;
+  h->cfg = *cfg;
+  h->ctx.stream = (cudaStream_t)cuda_stream;
+  h->ctx.sm_count = sms;
+  h->X = d_X;
+  const int d = cfg->d, batch = cfg->batch;
+  const int64_t dd = (int64_t)d * d * batch;
+  dq_status st = DQ_OK;
+  auto A = [&](dq_status s) { if (st == DQ_OK) st = s; };
+  A(dev_alloc(&h->ctx.d_status, 1));
+  A(dev_alloc(&h->Z, dd)); A(dev_alloc(&h->R, dd)); A(dev_alloc(&h->U, dd));
+  A(dev_alloc(&h->Gq, dd)); A(dev_alloc(&h->Gz, dd));
+  A(dev_alloc(&h->ws.A, dd)); A(dev_alloc(&h->ws.V, dd)); A(dev_alloc(&h->ws.Q, dd));
+  A(dev_alloc(&h->ws.Winv, dd)); A(dev_alloc(&h->ws.B, dd)); A(dev_alloc(&h->ws.S, dd));
+  A(dev_alloc(&h->ws.tmp, dd));
+  A(dev_alloc(&h->ws.T, (int64_t)batch * d * 32));
+  A(dev_alloc(&h->ws.W, (int64_t)batch * d * 32)); A(dev_alloc(&h->ws.W2, (int64_t)batch * d * 32));
+  A(dev_alloc(&h->loss_last, batch));
+  if (cfg->path == DQ_PATH_FP32) {
+    h->g_elems = (int64_t)batch * cfg->n_tokens * d;
+    float* g = nullptr;
+    A(dev_alloc(&g, h->g_elems));
+    h->G = g;
+    h->n_partials = whip_forward_f32_tiles(cfg->n_tokens, d);
+    const int tiles = ((d + 63) / 64) * ((d + 63) / 64) * batch;
+    int ks = (2 * sms + tiles - 1) / tiles;
+    if (ks > (int)(cfg->n_tokens / 256)) ks = (int)(cfg->n_tokens / 256);
+    if (ks > 16) ks = 16;
+    h->gq_ks = ks < 1 ? 1 : ks;
+    if (h->gq_ks > 1) A(dev_alloc(&h->gq_part, dd * h->gq_ks));
+  } else {
+    h->g_elems = (int64_t)batch * cfg->n_tokens * d;
+    __nv_bfloat16* g = nullptr;
+    A(dev_alloc(&g, h->g_elems));
+    h->G = g;
+    if (st == DQ_OK) A(tc_init(h->tc, h->ctx, *cfg, d_X, (__nv_bfloat16*)h->G, &h->n_partials));
+  }
+  A(dev_alloc(&h->partials, (int64_t)batch * (h->n_partials > 0 ? h->n_partials : 1)));
+  if (st == DQ_OK) {
+    for (auto& e : h->ev)
+      if (cudaEventCreate(&e) != cudaSuccess) st = DQ_ERR_CUDA;
+  }
+  if (st == DQ_OK && cudaMemsetAsync(h->ctx.d_status, 0, sizeof(int), h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
+  if (st == DQ_OK && cudaMemcpyAsync(h->Z, d_Z0, sizeof(float) * dd, cudaMemcpyDeviceToDevice, h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
+  if (st != DQ_OK) { free_all(h); return st; }
+  *out = h;
+  return DQ_OK;
+}
+
+dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
+  if (!h || n_steps < 0) return DQ_ERR_INVALID_ARG;
+  const dq_calib_config& c = h->cfg;
+  const int d = c.d, batch = c.batch;
+  const int64_t N = c.n_tokens;
+  const float inv_n = (c.reduction == DQ_MEAN_TOKENS) ? (float)(1.0 / (double)N) : 1.f;
+  Ctx& ctx = h->ctx;
+  if (h->timing) { for (auto& m : h->ms_acc) m = 0.0; h->timed_steps = 0; }
+  for (int s = 0; s < n_steps; ++s) {
+    float* loss_slot = d_loss_out ? d_loss_out + (int64_t)s * batch : nullptr;
+    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[0], ctx.stream));
+    // (a1) R <- qr(Z)
+    DQ_CHECK(ensure_rotation(h));
+    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[1], ctx.stream));
+    // (a2-a4) O = X R, Whip epilogue, loss reduction
+    if (c.path == DQ_PATH_FP32) {
+      DQ_CHECK(whip_forward_f32(ctx, (const float*)h->X, c.ldx, N * c.ldx, h->R, (float*)h->G,
+                                h->partials, N, d, batch, nullptr));
+    } else {
+      DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
+    }
+    DQ_CHECK(loss_finalize(ctx, h->partials, h->n_partials, batch, inv_n, loss_slot, h->loss_last));
+    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[2], ctx.stream));
+    // (a5) Gq = (1/N) X^T G
+    if (c.path == DQ_PATH_FP32) {
+      GemmDesc g{};
+      g.A = (const float*)h->X; g.lda = c.ldx; g.transA = 1; g.sA = N * c.ldx;
+      g.B = (const float*)h->G; g.ldb = d; g.transB = 0; g.sB = N * (int64_t)d;
+      g.M = d; g.N = d; g.K = (int)N; g.alpha = inv_n; g.beta = 0.f; g.batch = batch;
+      if (h->gq_ks <= 1) {
+        g.C = h->Gq; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = 1;
+        DQ_CHECK(gemm_f32(ctx, g));
+      } else {   // deterministic split-K over the token dimension
+        g.C = h->gq_part; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = h->gq_ks;
+        DQ_CHECK(gemm_f32(ctx, g));
+        DQ_CHECK(splitk_reduce(ctx, h->gq_part, h->gq_ks, (int64_t)d * d, batch, 1.f, 0.f, h->Gq));
+      }
+    } else {
+      DQ_CHECK(tc_grad_rotation(h->tc, ctx, h->Gq, inv_n));
+    }
+    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[3], ctx.stream));
+    // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
+    DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch));
+    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
+    // (a7) Z <- Z - lr Gz
+    DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, (int64_t)d * d * batch));
+    h->r_stale = true;
+    if (h->timing) {
+      DQ_CHECK_CUDA(cudaEventRecord(h->ev[5], ctx.stream));
+      DQ_CHECK_CUDA(cudaEventSynchronize(h->ev[5]));
+      for (int p = 0; p < DQ_PHASE_COUNT; ++p) {
+        float ms = 0.f;
+        DQ_CHECK_CUDA(cudaEventElapsedTime(&ms, h->ev[p], h->ev[p + 1]));
+        h->ms_acc[p] += ms;
+      }
+      h->timed_steps++;
+    }
+  }
+  return DQ_OK;
+}
+
+dq_status dq_calib_get_rotation(dq_calib_t* h, float* d_R_out) {
+  if (!h || !d_R_out) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK(ensure_rotation(h));
+  DQ_CHECK_CUDA(cudaMemcpyAsync(d_R_out, h->R, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
+                                cudaMemcpyDeviceToDevice, h->ctx.stream));
+  return DQ_OK;
+}
+
+dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out) {
+  if (!h || !d_Z_out) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK_CUDA(cudaMemcpyAsync(d_Z_out, h->Z, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
+                                cudaMemcpyDeviceToDevice, h->ctx.stream));
+  return DQ_OK;
+}
+
+dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z) {
+  if (!h || !d_Z) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK_CUDA(cudaMemcpyAsync(h->Z, d_Z, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
+                                cudaMemcpyDeviceToDevice, h->ctx.stream));
+  h->r_stale = true;
+  return DQ_OK;
+}
+
+dq_status dq_calib_status(dq_calib_t* h) {
+  if (!h) return DQ_ERR_INVALID_ARG;
+  int code = 0;
+  if (cudaMemcpyAsync(&code, h->ctx.d_status, sizeof(int), cudaMemcpyDeviceToHost, h->ctx.stream) != cudaSuccess)
+    return DQ_ERR_CUDA;
+  if (cudaStreamSynchronize(h->ctx.stream) != cudaSuccess) return DQ_ERR_CUDA;
+  if (code < 0 || code > DQ_ERR_TIMEOUT) return DQ_ERR_CUDA;
+  return (dq_status)code;
+}
+
+dq_status dq_calib_set_timing(dq_calib_t* h, int32_t enabled) {
+  if (!h) return DQ_ERR_INVALID_ARG;
+  h->timing = enabled != 0;
+  return DQ_OK;
+}
+
+dq_status dq_calib_get_timings(dq_calib_t* h, float* h_ms_by_phase, int32_t n) {
+  if (!h || !h_ms_by_phase || n < 0) return DQ_ERR_INVALID_ARG;
+  for (int p = 0; p < n && p < DQ_PHASE_COUNT; ++p)
+    h_ms_by_phase[p] = h->timed_steps > 0 ? (float)(h->ms_acc[p] / h->timed_steps) : 0.f;
+  return DQ_OK;
+}
+
+dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int64_t* n_elems) {
+  if (!h || !d_ptr || !n_elems) return DQ_ERR_INVALID_ARG;
+  const int64_t dd = (int64_t)h->cfg.d * h->cfg.d * h->cfg.batch;
+  switch (which) {
+    case DQ_BUF_R: *d_ptr = h->R; *n_elems = dd; break;
+    case DQ_BUF_U: *d_ptr = h->U; *n_elems = dd; break;
+    case DQ_BUF_GQ: *d_ptr = h->Gq; *n_elems = dd; break;
+    case DQ_BUF_GZ: *d_ptr = h->Gz; *n_elems = dd; break;
+    case DQ_BUF_G: *d_ptr = h->G; *n_elems = h->g_elems; break;
+    case DQ_BUF_PARTIALS: *d_ptr = h->partials; *n_elems = (int64_t)h->n_partials * h->cfg.batch; break;
+    case DQ_BUF_Z: *d_ptr = h->Z; *n_elems = dd; break;
+    default: return DQ_ERR_INVALID_ARG;
+  }
+  return DQ_OK;
+}
+
+int64_t dq_calib_launch_count(dq_calib_t* h) { return h ? h->ctx.launches : 0; }
+
+void dq_calib_destroy(dq_calib_t* h) {
+  if (!h) return;
+  cudaStreamSynchronize(h->ctx.stream);
+  free_all(h);
+}
+
+dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d, int64_t ldx,
+                          const float* d_R, void* d_Y, int64_t ldy, void* cuda_stream) {
+  if (!d_X || !d_R || !d_Y || n <= 0 || d <= 0 || ldx < d || ldy < d) return DQ_ERR_INVALID_ARG;
+  Ctx ctx;
+  ctx.stream = (cudaStream_t)cuda_stream;
+  if (x_dtype == DQ_FP32) {
+    GemmDesc g{};
+    g.A = (const float*)d_X; g.lda = ldx; g.transA = 0; g.sA = 0;
+    g.B = d_R; g.ldb = d; g.transB = 0; g.sB = 0;
+    g.C = (float*)d_Y; g.ldc = ldy; g.sC = 0;
+    g.M = (int)n; g.N = d; g.K = d; g.alpha = 1.f; g.beta = 0.f; g.batch = 1;
+    return gemm_f32(ctx, g);
+  }
+  if (x_dtype == DQ_BF16) return tc_rotate_apply(ctx, d_X, n, d, ldx, d_R, d_Y, ldy);
+  return DQ_ERR_INVALID_ARG;
+}
+
+}  // extern "C"

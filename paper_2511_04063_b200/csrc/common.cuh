@@ -1,0 +1,101 @@
+// Shared declarations of the library's translation units (host side + small
+// device helpers).  Nothing here is part of the public ABI.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dartquant.h"
+
+namespace dq {
+
+// Per-handle launch context.  d_status is a device int (0 = ok) that kernels set
+// with atomicCAS(0 -> code) so the first problem wins.
+struct Ctx {
+  cudaStream_t stream = nullptr;
+  int* d_status = nullptr;
+  int64_t launches = 0;
+  int sm_count = 148;
+};
+
+#define DQ_CHECK_CUDA(expr)                          \
+  do {                                               \
+    cudaError_t _e = (expr);                         \
+    if (_e != cudaSuccess) return DQ_ERR_CUDA;       \
+  } while (0)
+
+#define DQ_CHECK(expr)                 \
+  do {                                 \
+    dq_status _s = (expr);             \
+    if (_s != DQ_OK) return _s;        \
+  } while (0)
+
+inline dq_status after_launch(Ctx& ctx) {
+  ctx.launches++;
+  return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
+}
+
+__device__ __forceinline__ void set_status(int* d_status, int code) {
+  if (d_status) atomicCAS(d_status, 0, code);
+}
+
+// ---------------------------------------------------------------------------
+// fp32 FMA GEMM (gemm_ffma.cu):  C = alpha op(A) op(B) + beta C, batched/strided.
+// op(A) is M x K, op(B) is K x N; trans* = 1 means the stored matrix is the
+// transpose (stored K x M / N x K).  Any sizes.
+// ---------------------------------------------------------------------------
+struct GemmDesc {
+  const float* A; int64_t lda; int transA;
+  const float* B; int64_t ldb; int transB;
+  float* C; int64_t ldc;
+  int M, N, K;
+  float alpha, beta;
+  int batch; int64_t sA, sB, sC;
+  // Split-K: with ksplit > 1 slice ks of the reduction writes alpha * partial
+  // product (beta ignored) to C + (b * ksplit + ks) * sC; the caller reduces.
+  int ksplit = 1;
+};
+dq_status gemm_f32(Ctx& ctx, const GemmDesc& g);
+// out[b][i] = alpha * sum_ks part[(b * ksplit + ks)][i] + beta * out[b][i], fixed order.
+dq_status splitk_reduce(Ctx& ctx, const float* part, int ksplit, int64_t n_per_batch, int batch,
+                        float alpha, float beta, float* out);
+
+// O = X R with the Whip epilogue (Eq. 4) in fp32: writes G = -sign(O) exp(-|O|)
+// (token-major [batch][N][d], no 1/N) and one loss partial per 64x64 tile.
+// partials layout: [batch][tiles]; returns tiles per problem in *tiles_per_problem.
+dq_status whip_forward_f32(Ctx& ctx, const float* X, int64_t ldx, int64_t strideX, const float* R,
+                           float* G, float* partials, int64_t n_tokens, int d, int batch,
+                           int* tiles_per_problem);
+int whip_forward_f32_tiles(int64_t n_tokens, int d);
+
+// Sums partials[b][0..n) in a fixed order in fp64, scales, stores fp32 loss[b].
+// Sets DQ_ERR_NONFINITE in the status word if a loss is not finite.
+dq_status loss_finalize(Ctx& ctx, const float* partials, int n_per_problem, int batch, float scale,
+                        float* loss_out /* nullable */, float* loss_last);
+
+// ---------------------------------------------------------------------------
+// QR-Orth (qr_forward.cu / qr_backward.cu), fp32 matrices [batch][d][d].
+// ---------------------------------------------------------------------------
+struct QrWorkspace {
+  float* A = nullptr;     // working copy of Z, ends as the raw upper factor
+  float* V = nullptr;     // Householder vectors (unit lower trapezoid per panel)
+  float* T = nullptr;     // [batch][d/32][32][32] compact-WY T factors
+  float* W = nullptr;     // [batch][32][d] scratch
+  float* W2 = nullptr;    // [batch][32][d] scratch
+  float* Q = nullptr;     // accumulated orthogonal factor (raw gauge)
+  float* Winv = nullptr;  // U^-1
+  float* B = nullptr;     // R^T Gq, then R S
+  float* S = nullptr;     // tril(B - B^T, -1)
+  float* tmp = nullptr;   // [batch][d][d] scratch for the triangular inverse
+};
+// Z -> R (rotation, diag(U) > 0), U.  Optionally also a bf16 copy of R^T.
+dq_status qr_forward(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float* U,
+                     __nv_bfloat16* Rt_bf16 /* nullable */, int d, int batch);
+// Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
+dq_status qr_backward(Ctx& ctx, QrWorkspace& ws, const float* R, const float* U, const float* Gq,
+                      float* Gz, int d, int batch);
+
+// Z <- Z - lr Gz  (n elements)
+dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n);
+
+}  // namespace dq

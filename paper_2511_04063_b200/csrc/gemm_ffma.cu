@@ -1,0 +1,225 @@
+// fp32 FMA contractions: the exact-fp32 path of the calibration step and the
+// general small-matrix helper of QR-Orth.
+#include "common.cuh"
+
+namespace dq {
+namespace {
+
+constexpr int BM = 64, BN = 64, BK = 16, PAD = 4;
+
+enum { EPI_AXPBY = 0, EPI_WHIP = 1 };
+
+// 256 threads; thread (ty, tx) owns a 4x4 block of the 64x64 tile.
+template <int EPI>
+__global__ void __launch_bounds__(256) gemm_ffma_kernel(GemmDesc g, float* __restrict__ partials) {
+  __shared__ __align__(16) float As[BK][BM + PAD];
+  __shared__ __align__(16) float Bs[BK][BN + PAD];
+  __shared__ float warp_sums[8];
+
+  const int b = blockIdx.z / g.ksplit, ks = blockIdx.z % g.ksplit;
+  const float* __restrict__ A = g.A + (int64_t)b * g.sA;
+  const float* __restrict__ B = g.B + (int64_t)b * g.sB;
+  float* __restrict__ C = g.C + (int64_t)blockIdx.z * g.sC;
+  // K range of this slice, in multiples of BK
+  const int kchunk = (((g.K + g.ksplit - 1) / g.ksplit) + BK - 1) / BK * BK;
+  const int kbeg = ks * kchunk;
+  const int kend = min(g.K, kbeg + kchunk);
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = kbeg; k0 < kend; k0 += BK) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int idx = tid + i * 256;
+      int m, k;
+      if (!g.transA) { k = idx & 15; m = idx >> 4; } else { m = idx & 63; k = idx >> 6; }
+      float v = 0.f;
+      if (m0 + m < g.M && k0 + k < kend)
+        v = g.transA ? A[(int64_t)(k0 + k) * g.lda + m0 + m] : A[(int64_t)(m0 + m) * g.lda + k0 + k];
+      As[k][m] = v;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int idx = tid + i * 256;
+      int n, k;
+      if (!g.transB) { n = idx & 63; k = idx >> 6; } else { k = idx & 15; n = idx >> 4; }
+      float v = 0.f;
+      if (n0 + n < g.N && k0 + k < kend)
+        v = g.transB ? B[(int64_t)(n0 + n) * g.ldb + k0 + k] : B[(int64_t)(k0 + k) * g.ldb + n0 + n];
+      Bs[k][n] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < BK; ++k) {
+      const float4 a4 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+      const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+
+  if (EPI == EPI_AXPBY) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int m = m0 + ty * 4 + i;
+      if (m >= g.M) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int n = n0 + tx * 4 + j;
+        if (n >= g.N) continue;
+        float* c = C + (int64_t)m * g.ldc + n;
+        float v = g.alpha * acc[i][j];
+        if (g.beta != 0.f && g.ksplit == 1) v = fmaf(g.beta, *c, v);
+        *c = v;
+      }
+    }
+  } else {
+    // Eq. 4 per element: e = exp(-|o|); dL/do = -sign(o) e (0 at o = 0).
+    float local = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int m = m0 + ty * 4 + i;
+      if (m >= g.M) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int n = n0 + tx * 4 + j;
+        if (n >= g.N) continue;
+        const float o = acc[i][j];
+        const float e = expf(-fabsf(o));
+        local += e;
+        C[(int64_t)m * g.ldc + n] = (o > 0.f) ? -e : ((o < 0.f) ? e : 0.f);
+      }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) local += __shfl_xor_sync(0xffffffffu, local, off);
+    if ((tid & 31) == 0) warp_sums[tid >> 5] = local;
+    __syncthreads();
+    if (tid == 0) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) s += warp_sums[w];
+      partials[((int64_t)b * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x] = s;
+    }
+  }
+}
+
+}  // namespace
+
+dq_status gemm_f32(Ctx& ctx, const GemmDesc& g) {
+  if (g.M <= 0 || g.N <= 0 || g.batch <= 0) return DQ_OK;
+  dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch * g.ksplit);
+  gemm_ffma_kernel<EPI_AXPBY><<<grid, 256, 0, ctx.stream>>>(g, nullptr);
+  return after_launch(ctx);
+}
+
+namespace {
+__global__ void splitk_reduce_kernel(const float* __restrict__ part, int ksplit, int64_t n,
+                                     float alpha, float beta, float* __restrict__ out) {
+  const int b = blockIdx.y;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    float s = 0.f;
+    for (int ks = 0; ks < ksplit; ++ks) s += part[((int64_t)b * ksplit + ks) * n + i];
+    float* o = out + (int64_t)b * n + i;
+    *o = (beta != 0.f) ? fmaf(beta, *o, alpha * s) : alpha * s;
+  }
+}
+}  // namespace
+
+dq_status splitk_reduce(Ctx& ctx, const float* part, int ksplit, int64_t n_per_batch, int batch,
+                        float alpha, float beta, float* out) {
+  int bx = (int)((n_per_batch + 255) / 256);
+  if (bx > 1024) bx = 1024;
+  splitk_reduce_kernel<<<dim3(bx, batch), 256, 0, ctx.stream>>>(part, ksplit, n_per_batch, alpha,
+                                                              beta, out);
+  return after_launch(ctx);
+}
+
+int whip_forward_f32_tiles(int64_t n_tokens, int d) {
+  return (int)(((n_tokens + BM - 1) / BM) * ((d + BN - 1) / BN));
+}
+
+dq_status whip_forward_f32(Ctx& ctx, const float* X, int64_t ldx, int64_t strideX, const float* R,
+                           float* G, float* partials, int64_t n_tokens, int d, int batch,
+                           int* tiles_per_problem) {
+  GemmDesc g{};
+  g.A = X; g.lda = ldx; g.transA = 0; g.sA = strideX;
+  g.B = R; g.ldb = d; g.transB = 0; g.sB = (int64_t)d * d;
+  g.C = G; g.ldc = d; g.sC = n_tokens * (int64_t)d;
+  g.M = (int)n_tokens; g.N = d; g.K = d; g.alpha = 1.f; g.beta = 0.f; g.batch = batch; g.ksplit = 1;
+  dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
+  if (tiles_per_problem) *tiles_per_problem = (int)(grid.x * grid.y);
+  gemm_ffma_kernel<EPI_WHIP><<<grid, 256, 0, ctx.stream>>>(g, partials);
+  return after_launch(ctx);
+}
+
+// ---------------------------------------------------------------------------
+// Loss reduction: one block per problem, fixed summation order, fp64 accumulate.
+// ---------------------------------------------------------------------------
+namespace {
+__global__ void __launch_bounds__(256) loss_finalize_kernel(const float* __restrict__ partials, int n,
+                                                            float scale, float* __restrict__ loss_out,
+                                                            float* __restrict__ loss_last,
+                                                            int* d_status) {
+  __shared__ double sm[256];
+  const int b = blockIdx.x;
+  const float* p = partials + (int64_t)b * n;
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += 256) s += (double)p[i];
+  sm[threadIdx.x] = s;
+  __syncthreads();
+  for (int off = 128; off >= 1; off >>= 1) {
+    if (threadIdx.x < off) sm[threadIdx.x] += sm[threadIdx.x + off];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const float L = (float)(sm[0] * (double)scale);
+    if (loss_out) loss_out[b] = L;
+    loss_last[b] = L;
+    if (!isfinite(L)) set_status(d_status, DQ_ERR_NONFINITE);
+  }
+}
+
+__global__ void sgd_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz, float lr, int64_t n4) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    float4 z = Z[i];
+    const float4 g = Gz[i];
+    z.x = fmaf(-lr, g.x, z.x); z.y = fmaf(-lr, g.y, z.y);
+    z.z = fmaf(-lr, g.z, z.z); z.w = fmaf(-lr, g.w, z.w);
+    Z[i] = z;
+  }
+}
+}  // namespace
+
+dq_status loss_finalize(Ctx& ctx, const float* partials, int n_per_problem, int batch, float scale,
+                        float* loss_out, float* loss_last) {
+  loss_finalize_kernel<<<batch, 256, 0, ctx.stream>>>(partials, n_per_problem, scale, loss_out,
+                                                     loss_last, ctx.d_status);
+  return after_launch(ctx);
+}
+
+// Algorithm 1 line 10.  n is a multiple of 4 (d is a multiple of 32).
+dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n) {
+  const int64_t n4 = n / 4;
+  int blocks = (int)((n4 + 255) / 256);
+  const int cap = ctx.sm_count * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  sgd_kernel<<<blocks, 256, 0, ctx.stream>>>(reinterpret_cast<float4*>(Z),
+                                            reinterpret_cast<const float4*>(Gz), lr, n4);
+  return after_launch(ctx);
+}
+
+}  // namespace dq

@@ -1,0 +1,196 @@
+// Host side of the tensor-core path: tensor maps, operand copies, launches.
+#include <vector>
+
+#include "tc_gemm.cuh"
+#include "tc_path.cuh"
+
+namespace dq {
+namespace {
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode_fn() {
+  static EncodeFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeFn>(p);
+  return fn;
+}
+
+// bf16 tensor [batch][rows][k] (k contiguous, row stride ld elements), box = {64, box_rows, 1},
+// 128-byte swizzle: the shared-memory image is the K-major SW128 layout tcgen05 reads.
+dq_status make_map(CUtensorMap* m, const void* base, int64_t k, int64_t rows, int64_t batch, int64_t ld,
+                   int64_t batch_stride, int box_rows) {
+  EncodeFn fn = get_encode_fn();
+  if (!fn) return DQ_ERR_CUDA;
+  cuuint64_t dims[3] = {(cuuint64_t)k, (cuuint64_t)rows, (cuuint64_t)batch};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)batch_stride * 2};
+  cuuint32_t box[3] = {(cuuint32_t)tc::BLOCK_K, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? DQ_OK : DQ_ERR_CUDA;
+}
+
+// out[b][c][r] = in[b][r][c]   (bf16; rows, cols multiples of 64)
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in,
+                                                             __nv_bfloat16* __restrict__ out, int64_t rows,
+                                                             int64_t cols, int64_t ld_in) {
+  __shared__ __nv_bfloat16 t[64][66];
+  in += (int64_t)blockIdx.z * rows * ld_in;
+  out += (int64_t)blockIdx.z * rows * cols;
+  const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  for (int r = ty; r < 64; r += 4) t[r][tx] = in[(r0 + r) * ld_in + c0 + tx];
+  __syncthreads();
+  for (int c = ty; c < 64; c += 4) out[(c0 + c) * rows + r0 + tx] = t[tx][c];
+}
+
+// out[b][c][r] = bf16(in[b][r][c])  (fp32 in, d x d)
+__global__ void __launch_bounds__(256) transpose_f32_to_bf16_kernel(const float* __restrict__ in,
+                                                                    __nv_bfloat16* __restrict__ out, int d) {
+  __shared__ float t[32][33];
+  in += (int64_t)blockIdx.z * d * d;
+  out += (int64_t)blockIdx.z * d * d;
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int r = ty; r < 32; r += 8) t[r][tx] = in[(int64_t)(r0 + r) * d + c0 + tx];
+  __syncthreads();
+  for (int c = ty; c < 32; c += 8) out[(int64_t)(c0 + c) * d + r0 + tx] = __float2bfloat16_rn(t[tx][c]);
+}
+
+template <int BN, int NT, int EPI>
+dq_status launch_gemm(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& alo,
+                      const CUtensorMap& blo, const tc::Params& p) {
+  using L = tc::SmemLayout<BN, NT>;
+  static bool attr_set = false;
+  auto kern = tc::tc_gemm_kernel<BN, NT, EPI>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
+      return DQ_ERR_CUDA;
+    attr_set = true;
+  }
+  const int units = p.m_blocks * p.n_blocks * p.batch * p.ksplit;
+  int grid = units < ctx.sm_count ? units : ctx.sm_count;
+  if (grid < 1) return DQ_OK;
+  kern<<<grid, tc::NUM_THREADS, L::TOTAL, ctx.stream>>>(a, b, alo, blo, p);
+  return after_launch(ctx);
+}
+
+struct Maps {
+  CUtensorMap rt, x, xt, gt128, gt256;
+};
+
+}  // namespace
+
+dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void* d_X, __nv_bfloat16* Gt,
+                  int* n_partials) {
+  const int d = cfg.d, batch = cfg.batch;
+  const int64_t N = cfg.n_tokens;
+  tc.d = d; tc.batch = batch; tc.n_tokens = N;
+  tc.X = reinterpret_cast<const __nv_bfloat16*>(d_X);
+  tc.Gt = Gt;
+  if (cudaMalloc((void**)&tc.Xt, sizeof(__nv_bfloat16) * (size_t)batch * N * d) != cudaSuccess) return DQ_ERR_ALLOC;
+  if (cudaMalloc((void**)&tc.Rt, sizeof(__nv_bfloat16) * (size_t)batch * d * d) != cudaSuccess) return DQ_ERR_ALLOC;
+  // split-K of Gq = X^T G over the token dimension: fill the machine, keep >= 16 k-blocks per slice
+  const int bn = (d % 256 == 0) ? 256 : 128;
+  const int tiles = (d / tc::BLOCK_M) * (d / bn) * batch;
+  int ks = 1;
+  while (tiles * ks < ctx.sm_count && (N / tc::BLOCK_K) / (ks * 2) >= 16 && ks < 64) ks *= 2;
+  tc.ksplit = ks;
+  if (ks > 1 &&
+      cudaMalloc((void**)&tc.part, sizeof(float) * (size_t)batch * ks * d * d) != cudaSuccess)
+    return DQ_ERR_ALLOC;
+  Maps* m = new (std::nothrow) Maps();
+  if (!m) return DQ_ERR_ALLOC;
+  tc.maps = m;
+  DQ_CHECK(make_map(&m->rt, tc.Rt, d, d, batch, d, (int64_t)d * d, tc::BLOCK_M));
+  DQ_CHECK(make_map(&m->x, tc.X, d, N, batch, d, N * d, 256));
+  DQ_CHECK(make_map(&m->xt, tc.Xt, N, d, batch, N, N * d, tc::BLOCK_M));
+  DQ_CHECK(make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
+  DQ_CHECK(make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
+  // X^T copy (X is fixed for the whole calibration)
+  transpose_bf16_kernel<<<dim3(d / 64, (unsigned)(N / 64), batch), 256, 0, ctx.stream>>>(tc.X, tc.Xt, N, d, d);
+  DQ_CHECK(after_launch(ctx));
+  tc.n_partials = (d / tc::BLOCK_M) * (int)(N / 256) * 4;
+  *n_partials = tc.n_partials;
+  tc.ready = true;
+  return DQ_OK;
+}
+
+void tc_destroy(TcState& tc) {
+  cudaFree(tc.Xt); cudaFree(tc.Rt); cudaFree(tc.part);
+  delete reinterpret_cast<Maps*>(tc.maps);
+  tc = TcState();
+}
+
+// O^T = R^T X^T per 128 x 256 tile (rows = channels, columns = tokens), Whip epilogue:
+// writes G^T (bf16, channel-major) and 4 loss partials per tile.
+dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
+  Maps* m = reinterpret_cast<Maps*>(tc.maps);
+  tc::Params p{};
+  p.m_blocks = tc.d / tc::BLOCK_M; p.n_blocks = (int)(tc.n_tokens / 256); p.batch = tc.batch; p.ksplit = 1;
+  p.k_blocks = tc.d / tc::BLOCK_K;
+  p.out = tc.Gt; p.ld = tc.n_tokens; p.batch_stride = tc.n_tokens * tc.d; p.split_stride = 0;
+  p.alpha = 1.f; p.partials = partials; p.d_status = ctx.d_status;
+  return launch_gemm<256, 1, tc::EPI_WHIP>(ctx, m->rt, m->x, m->rt, m->x, p);
+}
+
+// Gq = scale * X^T G : A = X^T [d][N], B = G^T [d][N], reduction over tokens.
+dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
+  Maps* m = reinterpret_cast<Maps*>(tc.maps);
+  const int d = tc.d;
+  const int bn = (d % 256 == 0) ? 256 : 128;
+  tc::Params p{};
+  p.m_blocks = d / tc::BLOCK_M; p.n_blocks = d / bn; p.batch = tc.batch; p.ksplit = tc.ksplit;
+  p.k_blocks = (int)(tc.n_tokens / tc::BLOCK_K);
+  p.ld = d; p.alpha = scale; p.partials = nullptr; p.d_status = ctx.d_status;
+  if (tc.ksplit == 1) {
+    p.out = Gq; p.batch_stride = (int64_t)d * d; p.split_stride = 0;
+  } else {
+    p.out = tc.part; p.batch_stride = (int64_t)tc.ksplit * d * d; p.split_stride = (int64_t)d * d;
+  }
+  if (bn == 256) DQ_CHECK((launch_gemm<256, 1, tc::EPI_F32>(ctx, m->xt, m->gt256, m->xt, m->gt256, p)));
+  else DQ_CHECK((launch_gemm<128, 1, tc::EPI_F32>(ctx, m->xt, m->gt128, m->xt, m->gt128, p)));
+  if (tc.ksplit > 1) DQ_CHECK(splitk_reduce(ctx, tc.part, tc.ksplit, (int64_t)d * d, tc.batch, 1.f, 0.f, Gq));
+  return DQ_OK;
+}
+
+// Y = X R for bf16 activations: A = X [n][d], B = bf16(R^T) [d][d]; bf16 output, row stride ldy.
+dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t ldx, const float* d_R,
+                          void* d_Y, int64_t ldy) {
+  if (d % 128 != 0 || n % 128 != 0 || ldx % 8 != 0 || ldy % 8 != 0) return DQ_ERR_UNSUPPORTED;
+  int sms = 0, dev = 0;
+  DQ_CHECK_CUDA(cudaGetDevice(&dev));
+  DQ_CHECK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  ctx.sm_count = sms;
+  __nv_bfloat16* rt = nullptr;
+  if (cudaMallocAsync((void**)&rt, sizeof(__nv_bfloat16) * (size_t)d * d, ctx.stream) != cudaSuccess)
+    return DQ_ERR_ALLOC;
+  transpose_f32_to_bf16_kernel<<<dim3(d / 32, d / 32, 1), 256, 0, ctx.stream>>>(d_R, rt, d);
+  dq_status st = after_launch(ctx);
+  const int bn = (d % 256 == 0) ? 256 : 128;
+  CUtensorMap ma, mb;
+  if (st == DQ_OK) st = make_map(&ma, d_X, d, n, 1, ldx, n * ldx, tc::BLOCK_M);
+  if (st == DQ_OK) st = make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, bn);
+  if (st == DQ_OK) {
+    tc::Params p{};
+    p.m_blocks = (int)(n / tc::BLOCK_M); p.n_blocks = d / bn; p.batch = 1; p.ksplit = 1;
+    p.k_blocks = d / tc::BLOCK_K;
+    p.out = d_Y; p.ld = ldy; p.batch_stride = 0; p.split_stride = 0; p.alpha = 1.f;
+    p.partials = nullptr; p.d_status = nullptr;
+    st = (bn == 256) ? launch_gemm<256, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p)
+                     : launch_gemm<128, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p);
+  }
+  cudaFreeAsync(rt, ctx.stream);
+  return st;
+}
+
+}  // namespace dq

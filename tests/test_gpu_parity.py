@@ -1,0 +1,193 @@
+"""GPU parity: the CUDA path (through the C ABI) against the float64 oracle on the
+same seeded inputs.  Tolerances are the contract's: loss relative error <= 1e-4
+(fp32 path) / <= 2e-2 (bf16 tensor-core path); per-step max|R_gpu - R_ref| <= 1e-3;
+max|R^T R - I| <= 1e-4.  Stage-wise tolerances are derived from fp32 / bf16
+rounding and stated next to each check."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2511_04063_b200 as dq
+from paper_2511_04063_b200 import inputs as gen
+from gpu_util import Calib, x_f64
+
+pytestmark = pytest.mark.gpu
+
+LOSS_TOL_FP32, LOSS_TOL_BF16 = 1e-4, 2e-2
+R_TOL, ORTHO_TOL = 1e-3, 1e-4
+
+
+def ortho_err(R):
+    return np.abs(R.T @ R - np.eye(R.shape[0])).max()
+
+
+# --------------------------------------------------------------------- QR-Orth forward
+@pytest.mark.parametrize("d,batch", [(64, 1), (128, 3), (256, 1), (576, 1), (1024, 1)])
+def test_qr_forward_matches_unique_factorisation(d, batch):
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], d=d, n_tokens=64, batch=batch, n_outlier_channels=1)
+    rng = np.random.default_rng(d)
+    Z0 = (rng.standard_normal((batch, d, d)) / np.sqrt(d) + np.eye(d)).astype(np.float32)
+    c = Calib(w, Z0=Z0)
+    R = c.rotation()
+    assert c.status() == dq.DQ_OK
+    U = c.buf(dq.DQ_BUF_U).cpu().numpy().astype(np.float64)
+    for b in range(batch):
+        Rr, Ur = orc.qr_pos_lapack(Z0[b])
+        assert np.abs(R[b] - Rr).max() <= 2e-5          # fp32 Householder vs float64
+        assert np.abs(U[b] - Ur).max() <= 5e-5
+        assert ortho_err(R[b]) <= 2e-5
+        assert np.abs(np.tril(U[b], -1)).max() == 0.0 and (np.diag(U[b]) > 0).all()
+    c.close()
+
+
+def test_qr_of_random_hadamard_is_itself():
+    w = gen.scaled(gen.WORKLOADS["c2_7b"], d=512, n_tokens=256, x_dtype="fp32", path="fp32", dist="normal",
+                   n_outlier_channels=2)
+    c = Calib(w)
+    R = c.rotation()[0]
+    assert np.abs(R - c.Z0_host[0]).max() <= 1e-5
+    c.close()
+
+
+# --------------------------------------------------------------------- fp32 path, every stage
+@pytest.mark.parametrize("d,n,batch", [(128, 512, 1), (192, 416, 2)])
+def test_fp32_path_every_stage(d, n, batch):
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], d=d, n_tokens=n, batch=batch, n_outlier_channels=2)
+    c = Calib(w)
+    Z0 = c.latent()
+    loss = c.step(1)[0]
+    assert c.status() == dq.DQ_OK
+    R = c.buf(dq.DQ_BUF_R).cpu().numpy().astype(np.float64)
+    Gq = c.buf(dq.DQ_BUF_GQ).cpu().numpy().astype(np.float64)
+    Gz = c.buf(dq.DQ_BUF_GZ).cpu().numpy().astype(np.float64)
+    G = c.buf(dq.DQ_BUF_G, shape=(batch, n, d)).cpu().numpy().astype(np.float64)
+    Z1 = c.latent().astype(np.float64)
+    for b in range(batch):
+        ref = orc.calib_step(x_f64(w, c.X_host, b), Z0[b], w.lr)
+        assert abs(loss[b] - ref["loss"]) <= LOSS_TOL_FP32 * ref["loss"]
+        assert np.abs(R[b] - ref["R"]).max() <= 2e-5
+        # G is stored without the 1/N factor; values in [-1, 1]; O differs by ~1e-4 at most
+        Gref = ref["G"] * n
+        far = np.abs(ref["O"]) > 1e-3
+        assert np.abs(G[b] - Gref)[far].max() <= 1e-3
+        scale = np.abs(ref["Gq"]).max()
+        assert np.abs(Gq[b] - ref["Gq"]).max() <= 2e-3 * scale
+        assert np.abs(Gz[b] - ref["Gz"]).max() <= 5e-3 * np.abs(ref["Gz"]).max()
+        assert np.abs(Z1[b] - ref["Z_new"]).max() <= 1e-5
+    c.close()
+
+
+def test_c1_tiny_twenty_steps_teacher_forced_and_free_running():
+    w = gen.WORKLOADS["c1_tiny"]
+    c = Calib(w)
+    X = x_f64(w, c.X_host)
+    golden = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "c1_tiny_trajectory.json")))
+    # free running: 20 steps on the GPU, compare the loss curve with the stored oracle curve
+    losses = c.step(w.steps)[:, 0]
+    assert c.status() == dq.DQ_OK
+    ref_losses = np.array(golden["losses"])
+    assert np.abs(losses - ref_losses).max() <= 5e-3 * ref_losses.max()   # trajectories may drift a little
+    assert losses[-1] < 0.5 * losses[0]
+    Rf = c.rotation()[0]
+    assert ortho_err(Rf) <= ORTHO_TOL
+    # teacher forced: every step starts from the oracle's latent
+    Z = c.Z0_host[0].astype(np.float64)
+    for k in range(w.steps):
+        c.set_latent(Z[None])
+        lk = c.step(1)[0, 0]
+        ref = orc.calib_step(X, Z.astype(np.float32), w.lr)
+        assert abs(lk - ref["loss"]) <= LOSS_TOL_FP32 * ref["loss"], k
+        Rg = c.buf(dq.DQ_BUF_R).cpu().numpy()[0].astype(np.float64)
+        assert np.abs(Rg - ref["R"]).max() <= R_TOL, k
+        assert ortho_err(Rg) <= ORTHO_TOL, k
+        Rnext = c.rotation()[0]
+        Rnext_ref, _ = orc.qr_pos(ref["Z_new"])
+        assert np.abs(Rnext - Rnext_ref).max() <= R_TOL, k
+        Z = ref["Z_new"]
+    c.close()
+
+
+def test_fp32_path_is_bit_reproducible():
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], d=128, n_tokens=512)
+    outs = []
+    for _ in range(2):
+        c = Calib(w)
+        l = c.step(3)
+        outs.append((l.copy(), c.latent().copy()))
+        c.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+def test_sum_reduction_is_n_times_mean():
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], d=128, n_tokens=256)
+    a = Calib(w, lr=0.0)
+    b = Calib(w, lr=0.0, reduction=dq.DQ_SUM_TOKENS)
+    la, lb = a.step(1)[0, 0], b.step(1)[0, 0]
+    assert lb == pytest.approx(la * 256, rel=1e-5)
+    ref = orc.whip_loss(orc.rotate(x_f64(w, a.X_host), orc.qr_pos(a.Z0_host[0])[0]), "sum")
+    assert lb == pytest.approx(ref, rel=1e-4)
+    a.close(); b.close()
+
+
+# --------------------------------------------------------------------- rotate_apply
+def test_rotate_apply_fp32():
+    rng = np.random.default_rng(3)
+    n, d = 300, 96
+    X = rng.standard_normal((n, d)).astype(np.float32)
+    R, _ = orc.qr_pos(rng.standard_normal((d, d)))
+    Xd, Rd = torch.from_numpy(X).cuda(), torch.from_numpy(R.astype(np.float32)).cuda()
+    Y = torch.empty((n, d), dtype=torch.float32, device="cuda")
+    dq.dq_rotate_apply(Xd, Rd, Y)
+    ref = orc.rotate(X, R.astype(np.float32))
+    assert np.abs(Y.cpu().numpy() - ref).max() <= 1e-4
+    # Sec. 3 / norm invariance: rows keep their Euclidean norm
+    assert np.allclose(np.linalg.norm(Y.cpu().numpy().astype(np.float64), axis=1),
+                       np.linalg.norm(X.astype(np.float64), axis=1), rtol=1e-5)
+
+
+# --------------------------------------------------------------------- host-side error behaviour
+def test_invalid_arguments_are_reported_not_raised_by_cuda():
+    import ctypes as C
+    lib = dq.load_library()
+    h = C.c_void_p(0)
+    cfg = dq.dq_calib_config(d=128, n_tokens=256, batch=1, x_dtype=dq.DQ_FP32, path=dq.DQ_PATH_FP32,
+                             reduction=0, optimizer=0, lr=0.1, ldx=128)
+    X = torch.zeros((256, 128), device="cuda")
+    Z = torch.eye(128, device="cuda")
+    p = lambda t: C.c_void_p(t.data_ptr())
+    assert lib.dq_calib_init(C.byref(h), C.byref(cfg), None, p(Z), None) == dq.DQ_ERR_INVALID_ARG
+    assert lib.dq_calib_init(None, C.byref(cfg), p(X), p(Z), None) == dq.DQ_ERR_INVALID_ARG
+    cfg.d = 100
+    cfg.ldx = 100
+    assert lib.dq_calib_init(C.byref(h), C.byref(cfg), p(X), p(Z), None) == dq.DQ_ERR_UNSUPPORTED
+    cfg.d = 128; cfg.ldx = 64
+    assert lib.dq_calib_init(C.byref(h), C.byref(cfg), p(X), p(Z), None) == dq.DQ_ERR_INVALID_ARG
+    cfg.ldx = 128; cfg.path = dq.DQ_PATH_BF16_TC       # fp32 activations on the tensor-core path
+    assert lib.dq_calib_init(C.byref(h), C.byref(cfg), p(X), p(Z), None) == dq.DQ_ERR_UNSUPPORTED
+    assert h.value is None
+    assert lib.dq_calib_step(None, 1, None) == dq.DQ_ERR_INVALID_ARG
+    assert dq.status_string(dq.DQ_ERR_TIMEOUT) != ""
+
+
+def test_rank_deficient_latent_sets_singular_status():
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], d=128, n_tokens=256)
+    Z0 = gen.gen_latent_init(w)
+    Z0[0, :, 5] = 0.0                                   # a zero column: U^-T does not exist
+    c = Calib(w, Z0=Z0)
+    c.rotation()
+    assert c.status() == dq.DQ_ERR_SINGULAR
+    c.close()
+
+
+def test_nonfinite_input_sets_status():
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], d=128, n_tokens=256)
+    X = gen.gen_activations(w)
+    X[0, 3, 7] = np.nan
+    c = Calib(w, X=X)
+    c.step(1)
+    assert c.status() == dq.DQ_ERR_NONFINITE
+    c.close()

@@ -1,0 +1,108 @@
+"""GPU parity of the bf16 tensor-core path (tcgen05 GEMMs with the fused Eq. 4
+epilogue) against the float64 oracle, on small cases that still span several
+tiles, several k-blocks, split-K and more than one problem."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2511_04063_b200 as dq
+from paper_2511_04063_b200 import inputs as gen
+from gpu_util import Calib, x_f64
+
+pytestmark = pytest.mark.gpu
+
+LOSS_TOL_BF16 = 2e-2
+R_TOL, ORTHO_TOL = 1e-3, 1e-4
+
+
+def small(name, **kw):
+    return gen.scaled(gen.WORKLOADS[name], **kw)
+
+
+CASES = [
+    small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3),
+    small("c2_7b", d=384, n_tokens=512, batch=2, n_outlier_channels=4),     # 128-wide N tiles, 2 problems
+    small("c3_heads", d=128, n_tokens=2048, batch=4),                       # per-head rotations
+    small("c5_70b", d=512, n_tokens=4096, n_outlier_channels=2),            # token scales, several waves
+]
+
+
+@pytest.mark.parametrize("w", CASES, ids=lambda w: "%s-d%d-n%d-b%d" % (w.name, w.d, w.n_tokens, w.batch))
+def test_tensor_core_step_every_stage(w):
+    c = Calib(w)
+    Z0 = c.latent()
+    loss = c.step(1)[0]
+    assert c.status() == dq.DQ_OK
+    n, d, batch = w.n_tokens, w.d, w.batch
+    R = c.buf(dq.DQ_BUF_R).cpu().numpy().astype(np.float64)
+    Gq = c.buf(dq.DQ_BUF_GQ).cpu().numpy().astype(np.float64)
+    Gz = c.buf(dq.DQ_BUF_GZ).cpu().numpy().astype(np.float64)
+    Gt = c.buf(dq.DQ_BUF_G, dtype=torch.bfloat16, shape=(batch, d, n)).float().cpu().numpy().astype(np.float64)
+    Z1 = c.latent().astype(np.float64)
+    for b in range(batch):
+        X = x_f64(w, c.X_host, b)
+        ref = orc.calib_step(X, Z0[b], w.lr)
+        assert abs(loss[b] - ref["loss"]) <= LOSS_TOL_BF16 * ref["loss"]
+        assert np.abs(R[b] - ref["R"]).max() <= 2e-5
+        # dL/dO (no 1/N), stored channel-major.  R is rounded to bf16 (2^-9 relative), so
+        # |dO| <~ ||x_t|| 2^-9 / sqrt(d) * few; compare where |O| is clear of the kink at 0.
+        row_norm = np.linalg.norm(X, axis=1)
+        dO = 8.0 * row_norm / np.sqrt(d) * 2.0 ** -9 + 1e-3
+        G_ref = ref["G"] * n
+        clear = np.abs(ref["O"]) > 2.0 * dO[:, None]
+        err = np.abs(Gt[b].T - G_ref)
+        bound = np.exp(-np.abs(ref["O"])) * (np.exp(dO)[:, None] - 1.0) + 2.0 ** -8
+        assert (err[clear] <= bound[clear]).all()
+        assert clear.mean() > 0.5
+        # Gq: random-sign accumulation of those errors; 2e-2 of the largest entry
+        assert np.abs(Gq[b] - ref["Gq"]).max() <= 2e-2 * np.abs(ref["Gq"]).max()
+        rel_f = np.linalg.norm(Gq[b] - ref["Gq"]) / np.linalg.norm(ref["Gq"])
+        assert rel_f <= 2e-2
+        assert np.linalg.norm(Gz[b] - ref["Gz"]) <= 3e-2 * np.linalg.norm(ref["Gz"])
+        # one teacher-forced step: rotation of the updated latent
+        R1, _ = orc.qr_pos_lapack(Z1[b])
+        R1_ref, _ = orc.qr_pos_lapack(ref["Z_new"])
+        assert np.abs(R1 - R1_ref).max() <= R_TOL
+    Rn = c.rotation()
+    for b in range(batch):
+        assert np.abs(Rn[b].T @ Rn[b] - np.eye(d)).max() <= ORTHO_TOL
+    c.close()
+
+
+def test_tensor_core_path_is_bit_reproducible():
+    w = small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3)
+    outs = []
+    for _ in range(2):
+        c = Calib(w)
+        l = c.step(3)
+        outs.append((l.copy(), c.latent().copy()))
+        c.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+def test_loss_decreases_over_steps_on_heavy_tailed_input():
+    w = small("c2_7b", d=256, n_tokens=2048, n_outlier_channels=3, lr=2e-3)
+    c = Calib(w)
+    losses = c.step(10)[:, 0]
+    assert c.status() == dq.DQ_OK
+    assert losses[-1] < losses[0]
+    c.close()
+
+
+@pytest.mark.parametrize("n,d", [(256, 128), (1024, 256), (384, 640)])
+def test_rotate_apply_bf16(n, d):
+    rng = np.random.default_rng(7)
+    Xf = rng.standard_normal((n, d)).astype(np.float32)
+    Xb = gen.f32_to_bf16_bits(Xf)
+    R, _ = orc.qr_pos_lapack(rng.standard_normal((d, d)))
+    Xd = torch.from_numpy(Xb.view(np.int16)).cuda().view(torch.bfloat16)
+    Rd = torch.from_numpy(R.astype(np.float32)).cuda()
+    Y = torch.empty((n, d), dtype=torch.bfloat16, device="cuda")
+    dq.dq_rotate_apply(Xd, Rd, Y)
+    torch.cuda.synchronize()
+    ref = orc.rotate(gen.bf16_bits_to_f32(Xb).reshape(n, d), R)
+    got = Y.float().cpu().numpy().astype(np.float64)
+    # bf16 operands (2^-9) and bf16 output (2^-9): a few 1e-2 absolute on O(1..4) values
+    assert np.abs(got - ref).max() <= 6e-2
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-2
