@@ -1,0 +1,290 @@
+#!/usr/bin/env python
+"""Benchmark of the calibration hot path (one step = qr(Z) -> X R -> Whip ->
+backward -> SGD) on synthetic LLM-shaped activations.
+
+  python bench.py --gpus N --steps K --warmup W [--workload c2_7b] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is calibration steps/s with inputs resident in
+HBM; `e2e` is the same metric through the C ABI with host buffers (a fresh activation
+batch copied host->device and the loss read back every step); `roofline` is the
+forward X R + Whip tensor-core kernel against the measured bf16 peak; `cpu_baseline`
+is the float64 oracle timed on this machine's host cores on a bounded sample.
+With N > 1 every rank calibrates an independent rotation (replicas, no collective
+on the data path): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "calibration steps/sec"
+UNIT = "steps/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM traffic of one launch of the forward kernel on the c2_7b workload, from the ncu
+# capture summarised in profiles/ (bytes read + written); None until captured.
+NCU_TRAFFIC_BYTES = {"c2_7b": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle sampling during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, reasons = [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                out["sm_max_mhz"] = float(r[2])
+            except ValueError:
+                continue
+            for k, nme in enumerate(names):
+                if r[5 + k].strip().lower().startswith("active"):
+                    reasons.add(nme)
+        if sm:
+            # samples under load = upper half of the observed clocks is not meaningful; take the median
+            out["sm_mhz"] = float(np.median(sm))
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        return out
+
+
+def oracle_sample_steps_per_s(w, n_steps: int, shrink: int):
+    """Times the float64 oracle on the workload shrunk by `shrink` in both d and N.
+    Every term of a step scales with N d^2 or d^3, i.e. by shrink^3, so the full-size
+    rate is the sample's rate / shrink^3."""
+    import oracle as orc
+    from paper_2511_04063_b200 import inputs as gen
+    ws = gen.scaled(w, d=w.d // shrink, n_tokens=w.n_tokens // shrink,
+                    n_outlier_channels=max(1, w.n_outlier_channels // shrink))
+    X = gen.activations_as_f32(ws, gen.gen_activations(ws))[0].astype(np.float64)
+    Z = gen.gen_latent_init(ws)[0].astype(np.float64)
+    t0 = time.perf_counter()
+    for _ in range(n_steps):
+        Z = orc.calib_step(X, Z, ws.lr)["Z_new"]
+    dt = (time.perf_counter() - t0) / n_steps
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    sample = ("oracle.calib_step x%d on the same recipe at d=%d, N=%d (1/%d of each dimension); "
+              "rate divided by %d^3" % (n_steps, ws.d, ws.n_tokens, shrink, shrink))
+    return 1.0 / (dt * shrink ** 3), dt, cores, sample
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shrink = 4 if w.d >= 2048 else 1
+    total = max(1, args.steps + args.warmup)
+    v, dt, cores, sample = oracle_sample_steps_per_s(w, min(total, 3), shrink)
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / v, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "d": w.d, "n_tokens": w.n_tokens, "batch": w.batch},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2_7b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2511_04063_b200 import inputs as gen
+    w = gen.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import paper_2511_04063_b200 as dq
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the calibration path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------------------------------------------------------- inputs
+    # every rank gets its own seeded problem (an independent rotation site)
+    wr = gen.scaled(w, seed=w.seed + rank)
+    X_host = gen.gen_activations(wr)
+    Z0_host = gen.gen_latent_init(wr)
+    as_torch = (lambda a: torch.from_numpy(a)) if wr.x_dtype == "fp32" else \
+        (lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16))
+    X_pinned = as_torch(X_host).pin_memory()
+    Xd = X_pinned.cuda(non_blocking=True)
+    Zd = torch.from_numpy(Z0_host).cuda()
+    path = dq.DQ_PATH_FP32 if wr.path == "fp32" else dq.DQ_PATH_BF16_TC
+    h = dq.dq_calib_init(Xd, Zd, lr=wr.lr, path=path)
+    K, W = args.steps, max(args.warmup, 3)
+    loss_dev = torch.empty((max(K, W), wr.batch), dtype=torch.float32, device="cuda")
+
+    # ---------------------------------------------------------------- device-resident timing
+    dq.dq_calib_step(h, W, loss_dev)
+    st = dq.dq_calib_status(h)
+    assert st == dq.DQ_OK, dq.status_string(st)
+    sampler = ClockSampler(local_rank)
+    launches0 = dq.dq_calib_launch_count(h)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    dq.dq_calib_step(h, K, loss_dev)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    launches = dq.dq_calib_launch_count(h) - launches0
+    st = dq.dq_calib_status(h)
+    assert st == dq.DQ_OK, dq.status_string(st)
+    losses = loss_dev[:K].float().cpu().numpy()
+
+    # ---------------------------------------------------------------- per-phase times (events inside the library)
+    dq.dq_calib_set_timing(h, True)
+    n_phase_steps = min(K, 5)
+    dq.dq_calib_step(h, n_phase_steps, loss_dev)
+    phases = dq.dq_calib_get_timings(h)
+    dq.dq_calib_set_timing(h, False)
+
+    # ---------------------------------------------------------------- end to end (host buffers)
+    loss_host = torch.empty((1, wr.batch), dtype=torch.float32).pin_memory()
+    Ke = min(K, 10)
+    barrier()
+    t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0e.record()
+    for _ in range(Ke):
+        Xd.copy_(X_pinned, non_blocking=True)          # this step's activation batch, host -> device
+        dq.dq_calib_refresh_inputs(h)
+        dq.dq_calib_step(h, 1, loss_dev)
+        loss_host.copy_(loss_dev[:1], non_blocking=True)  # the step's result, device -> host
+        torch.cuda.current_stream().synchronize()
+    t1e.record()
+    barrier()
+    ms_e2e = t0e.elapsed_time(t1e)
+    h2d = X_pinned.numel() * X_pinned.element_size()
+    d2h = loss_host.numel() * 4
+
+    # ---------------------------------------------------------------- reduce over ranks
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, ms_e2e = float(t[0]), float(t[1])
+    value = world * K / (ms * 1e-3)
+    e2e_value = world * Ke / (ms_e2e * 1e-3)
+
+    if rank == 0:
+        peaks = load_peaks()
+        d, N, B = wr.d, wr.n_tokens, wr.batch
+        fwd_flops = 2.0 * N * d * d * B
+        t_fwd = phases["rotate_whip"] * 1e-3
+        t_bwd = phases["grad_rotation"] * 1e-3
+        achieved = fwd_flops / t_fwd / 1e12 if t_fwd > 0 else 0.0
+        peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        gemm_tflops = 2 * fwd_flops / (t_fwd + t_bwd) / 1e12 if (t_fwd + t_bwd) > 0 else 0.0
+        total_phase = sum(phases.values())
+        roofline = {"bound": "tensor", "kernel": "tc_gemm_kernel<256,1,WHIP> (O^T = R^T X^T, Eq. 4 epilogue)"
+                    if path == dq.DQ_PATH_BF16_TC else "gemm_ffma_kernel<WHIP>",
+                    "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "peak_source": "%s (sustained; kernel timed inside the step)" % peaks["_source"],
+                    "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                    "frac_of_nominal_2250": achieved / 2250.0,
+                    "traffic": NCU_TRAFFIC_BYTES.get(wr.name),
+                    "algorithmic_flops_per_launch": fwd_flops}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16" if path == dq.DQ_PATH_BF16_TC else "f32", "data": "synthetic",
+                "config": {"workload": wr.name, "d": d, "n_tokens": N, "batch": B, "lr": wr.lr,
+                           "parallelism": "replicas x%d" % world,
+                           "l2": "inputs (%.0f MiB X + G) exceed the 126 MB L2" % (2 * h2d / 2 ** 20)},
+                "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
+                           "reasons": clocks["reasons"], "samples": clocks["samples"]},
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "steps": Ke},
+                "gpu_launches": int(launches),
+                "roofline": roofline,
+                "phases_ms": phases,
+                "gemm_tflops": gemm_tflops,
+                "gemm_frac_of_measured_burst": gemm_tflops / peaks["bf16_tflops"],
+                "gemm_frac_of_nominal_2250": gemm_tflops / 2250.0,
+                "qr_orth_share": (phases["qr_forward"] + phases["qr_backward"]) / total_phase if total_phase else None,
+                "loss_first_last": [float(losses[0].mean()), float(losses[-1].mean())]}
+        if not args.no_cpu_baseline and world == 1:
+            shrink = 4 if d >= 2048 else 1
+            v, dt, cores, sample = oracle_sample_steps_per_s(w, 2 if shrink > 1 else 3, shrink)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+        print(json.dumps(line), flush=True)
+    dq.dq_calib_destroy(h)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -84,6 +84,12 @@ dq_status dq_calib_get_rotation(dq_calib_t* h, float* d_R_out);
 dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d, int64_t ldx,
                           const float* d_R, void* d_Y, int64_t ldy, void* cuda_stream);
 
+/* Mini-batch use (the paper feeds the loop with batches of sampled tokens): the
+ * caller overwrote the borrowed activation buffer d_X in place (same shape) on
+ * the handle's stream; rebuild every operand copy derived from it.  Cheap no-op on
+ * the fp32 path. */
+dq_status dq_calib_refresh_inputs(dq_calib_t* h);
+
 /* Checkpoint / resume of the optimised parameter (Algorithm 1 line 5: Z <- Z0). */
 dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out);
 dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z);

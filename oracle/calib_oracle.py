@@ -54,11 +54,19 @@ def whip_loss(O: np.ndarray, reduction: str = "mean") -> float:
     raise ValueError(reduction)
 
 
-def whip_grad_wrt_output(O: np.ndarray, reduction: str = "mean") -> np.ndarray:
-    """G = dL/dO.  d/do exp(-|o|) = -sign(o) exp(-|o|), sign(0) = 0 (Eq. 4)."""
+def whip_grad_wrt_output(O: np.ndarray, reduction: str = "mean", sign_of_O=None) -> np.ndarray:
+    """G = dL/dO.  d/do exp(-|o|) = -sign(o) exp(-|o|), sign(0) = 0 (Eq. 4).
+
+    Eq. 4 has a kink at o = 0, so sign(o) is a discrete decision taken on a
+    floating-point value.  A caller comparing against an implementation in lower
+    precision may pass sign_of_O (entries in {-1, 0, +1}) to take that decision
+    in the other implementation's precision for outputs that are zero to within
+    its rounding error; everything else is unchanged.
+    """
     O = np.asarray(O, dtype=F64)
     scale = 1.0 / O.shape[0] if reduction == "mean" else 1.0
-    return -np.sign(O) * np.exp(-np.abs(O)) * scale
+    sgn = np.sign(O) if sign_of_O is None else np.asarray(sign_of_O, dtype=F64)
+    return -sgn * np.exp(-np.abs(O)) * scale
 
 
 # ----------------------------------------------------------------------------
@@ -148,16 +156,18 @@ def sgd_step(Z: np.ndarray, Gz: np.ndarray, lr: float) -> np.ndarray:
 
 
 def calib_step(X: np.ndarray, Z: np.ndarray, lr: float, reduction: str = "mean",
-               qr=qr_pos):
+               qr=qr_pos, sign_decider=None):
     """One pass of the loop body of Algorithm 1 (lines 7-10).
 
     Returns a dict with every intermediate so that tests can compare each stage.
-    The loss is L(Z) before the update.
+    The loss is L(Z) before the update.  sign_decider(O) -> sign array lets a
+    test take the sign decision at the kink of Eq. 4 in the precision of the
+    implementation under test (see whip_grad_wrt_output).
     """
     R, U = qr(Z)
     O = rotate(X, R)
     loss = whip_loss(O, reduction)
-    G = whip_grad_wrt_output(O, reduction)
+    G = whip_grad_wrt_output(O, reduction, None if sign_decider is None else sign_decider(O))
     Gq = grad_wrt_rotation(X, G)
     Gz = qr_backward(R, U, Gq)
     Z_new = sgd_step(Z, Gz, lr)

@@ -23,8 +23,8 @@ DQ_BUF_R, DQ_BUF_U, DQ_BUF_GQ, DQ_BUF_GZ, DQ_BUF_G, DQ_BUF_PARTIALS, DQ_BUF_Z = 
 
 EXPORTED_SYMBOLS = (
     "dq_calib_init", "dq_calib_step", "dq_calib_get_rotation", "dq_rotate_apply",
-    "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_status", "dq_calib_get_timings",
-    "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
+    "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
+    "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
     "dq_calib_destroy", "dq_version",
 )
 
@@ -61,6 +61,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_get_latent.argtypes = [vp, vp]
     lib.dq_calib_set_latent.argtypes = [vp, vp]
     lib.dq_calib_status.argtypes = [vp]
+    lib.dq_calib_refresh_inputs.argtypes = [vp]
     lib.dq_calib_get_timings.argtypes = [vp, C.POINTER(C.c_float), i32]
     lib.dq_calib_set_timing.argtypes = [vp, i32]
     lib.dq_calib_debug_buffer.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i64)]
@@ -73,7 +74,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_version.restype = C.c_char_p
     for name in ("dq_calib_init", "dq_calib_step", "dq_calib_get_rotation", "dq_rotate_apply",
                  "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_status", "dq_calib_get_timings",
-                 "dq_calib_set_timing", "dq_calib_debug_buffer"):
+                 "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_refresh_inputs"):
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -133,6 +134,10 @@ def dq_calib_get_latent(h, Z_out):
 
 def dq_calib_set_latent(h, Z):
     _check(load_library().dq_calib_set_latent(h, _ptr(Z)), "dq_calib_set_latent")
+
+
+def dq_calib_refresh_inputs(h):
+    _check(load_library().dq_calib_refresh_inputs(h), "dq_calib_refresh_inputs")
 
 
 def dq_calib_status(h) -> int:

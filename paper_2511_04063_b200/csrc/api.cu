@@ -229,6 +229,12 @@ dq_status dq_calib_get_rotation(dq_calib_t* h, float* d_R_out) {
   return DQ_OK;
 }
 
+dq_status dq_calib_refresh_inputs(dq_calib_t* h) {
+  if (!h) return DQ_ERR_INVALID_ARG;
+  if (h->cfg.path == DQ_PATH_BF16_TC) return tc_refresh_inputs(h->tc, h->ctx);
+  return DQ_OK;
+}
+
 dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out) {
   if (!h || !d_Z_out) return DQ_ERR_INVALID_ARG;
   DQ_CHECK_CUDA(cudaMemcpyAsync(d_Z_out, h->Z, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,

@@ -116,13 +116,18 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   DQ_CHECK(make_map(&m->xt, tc.Xt, N, d, batch, N, N * d, tc::BLOCK_M));
   DQ_CHECK(make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
   DQ_CHECK(make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
-  // X^T copy (X is fixed for the whole calibration)
-  transpose_bf16_kernel<<<dim3(d / 64, (unsigned)(N / 64), batch), 256, 0, ctx.stream>>>(tc.X, tc.Xt, N, d, d);
-  DQ_CHECK(after_launch(ctx));
+  DQ_CHECK(tc_refresh_inputs(tc, ctx));
   tc.n_partials = (d / tc::BLOCK_M) * (int)(N / 256) * 4;
   *n_partials = tc.n_partials;
   tc.ready = true;
   return DQ_OK;
+}
+
+// X^T copy (channel-major) for the K-major A operand of Gq = X^T G.
+dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx) {
+  transpose_bf16_kernel<<<dim3(tc.d / 64, (unsigned)(tc.n_tokens / 64), tc.batch), 256, 0, ctx.stream>>>(
+      tc.X, tc.Xt, tc.n_tokens, tc.d, tc.d);
+  return after_launch(ctx);
 }
 
 void tc_destroy(TcState& tc) {

@@ -21,6 +21,7 @@ struct TcState {
 dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void* d_X,
                   __nv_bfloat16* Gt, int* n_partials);
 void tc_destroy(TcState& tc);
+dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx);   // X changed in place: rebuild X^T
 inline __nv_bfloat16* tc_rt_operand(TcState& tc) { return tc.ready ? tc.Rt : nullptr; }
 dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials);
 dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale);

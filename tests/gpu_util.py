@@ -70,3 +70,19 @@ class Calib:
 
 def x_f64(w, X, b=0):
     return gen.activations_as_f32(w, X)[b].astype(np.float64)
+
+
+def sign_decider_from_gpu(G_gpu_token_major, band):
+    """Eq. 4 has a kink at o = 0: where the oracle's |O| is within `band` (the rounding
+    error of the GPU arithmetic; scalar or per-token column vector) the sign decision is
+    taken in the kernel's precision, i.e. from the stored dL/dO.  Elsewhere the signs must agree."""
+    sg = -np.sign(G_gpu_token_major)
+
+    def decide(O):
+        s = np.sign(O)
+        near = np.abs(O) <= band
+        # beyond |o| ~ 87 exp(-|o|) underflows in fp32 and the stored derivative is an exact 0
+        chk = ~near & (np.abs(O) < 60.0)
+        assert np.array_equal(s[chk], sg[chk]), "sign of dL/dO differs away from the kink"
+        return np.where(near, sg, s)
+    return decide

@@ -13,7 +13,7 @@ import torch
 import oracle as orc
 import paper_2511_04063_b200 as dq
 from paper_2511_04063_b200 import inputs as gen
-from gpu_util import Calib, x_f64
+from gpu_util import Calib, x_f64, sign_decider_from_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -99,7 +99,10 @@ def test_c1_tiny_twenty_steps_teacher_forced_and_free_running():
     for k in range(w.steps):
         c.set_latent(Z[None])
         lk = c.step(1)[0, 0]
-        ref = orc.calib_step(X, Z.astype(np.float32), w.lr)
+        G = c.buf(dq.DQ_BUF_G, shape=(1, w.n_tokens, w.d)).cpu().numpy()[0].astype(np.float64)
+        # fp32 rounding of O = X R is ~1e-6 ||x_t||; the sign at the kink of Eq. 4 is decided there
+        band = 4e-6 * np.linalg.norm(X, axis=1)[:, None]
+        ref = orc.calib_step(X, Z.astype(np.float32), w.lr, sign_decider=sign_decider_from_gpu(G, band))
         assert abs(lk - ref["loss"]) <= LOSS_TOL_FP32 * ref["loss"], k
         Rg = c.buf(dq.DQ_BUF_R).cpu().numpy()[0].astype(np.float64)
         assert np.abs(Rg - ref["R"]).max() <= R_TOL, k

@@ -92,6 +92,18 @@ def test_gradient_wrt_rotation_central_differences():
             assert fd == pytest.approx(Gq[i, j], rel=1e-6, abs=1e-10)
 
 
+def test_sign_override_only_changes_the_overridden_entries():
+    O = np.array([[1e-9, -2.0, 0.5], [-1e-9, 3.0, 0.0]])
+    G0 = orc.whip_grad_wrt_output(O)
+    S = np.sign(O)
+    S[0, 0] = -1.0                      # the other implementation saw a tiny negative value
+    G1 = orc.whip_grad_wrt_output(O, sign_of_O=S)
+    assert G1[0, 0] == -G0[0, 0] and abs(G1[0, 0]) == pytest.approx(0.5, rel=1e-8)
+    mask = np.ones_like(O, bool)
+    mask[0, 0] = False
+    assert np.array_equal(G0[mask], G1[mask])
+
+
 # ------------------------------------------------------------- QR (Algorithm 2)
 @pytest.mark.parametrize("n", [1, 2, 5, 33, 128])
 def test_qr_factorisation_properties(n):
