@@ -1,4 +1,9 @@
 // C ABI: handle management, argument validation and the per-step schedule.
+//
+// All work of a handle runs on an internal stream that is fenced against the
+// caller's stream with events at every entry point, so the caller sees ordinary
+// stream semantics while whole steps can be replayed as a CUDA graph (stream
+// capture is not allowed on the legacy default stream callers often pass).
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -10,7 +15,9 @@ using namespace dq;
 
 struct dq_calib {
   dq_calib_config cfg;
-  Ctx ctx;
+  Ctx ctx;                      // ctx.stream is the internal work stream
+  cudaStream_t user_stream = nullptr;
+  cudaEvent_t ev_in = nullptr, ev_out = nullptr;
   const void* X = nullptr;
   float* Z = nullptr;
   float* R = nullptr;
@@ -25,12 +32,19 @@ struct dq_calib {
   int n_partials = 0;           // per problem
   float* loss_last = nullptr;   // [batch]
   QrWorkspace ws;
-  TcState tc;                   // tensor-core path state (operand copies, tensor maps)
+  TcState tc;                   // tensor-core contractions (operand copies, tensor maps)
+  QrTcState qtc;                // tensor-core QR-Orth operand copies
+  bool fast_qr = false;
   bool r_stale = true;
   bool timing = false;
   cudaEvent_t ev[DQ_PHASE_COUNT + 1] = {};
   double ms_acc[DQ_PHASE_COUNT] = {};
   int timed_steps = 0;
+  // one whole step (QR forward .. update) captured once and replayed
+  cudaGraphExec_t graph = nullptr;
+  int64_t graph_launches = 0;
+  bool graph_failed = false;
+  int eager_steps_done = 0;
 };
 
 namespace {
@@ -44,12 +58,17 @@ dq_status dev_alloc(T** p, int64_t n) {
 
 void free_all(dq_calib* h) {
   if (!h) return;
+  if (h->graph) cudaGraphExecDestroy(h->graph);
   tc_destroy(h->tc);
+  qr_tc_destroy(h->qtc);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
   cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->ctx.d_status);
   cudaFree(h->ws.A); cudaFree(h->ws.V); cudaFree(h->ws.T); cudaFree(h->ws.W); cudaFree(h->ws.W2);
   cudaFree(h->ws.Q); cudaFree(h->ws.Winv); cudaFree(h->ws.B); cudaFree(h->ws.S); cudaFree(h->ws.tmp);
   for (auto& e : h->ev) if (e) cudaEventDestroy(e);
+  if (h->ev_in) cudaEventDestroy(h->ev_in);
+  if (h->ev_out) cudaEventDestroy(h->ev_out);
+  if (h->ctx.stream) cudaStreamDestroy(h->ctx.stream);
   delete h;
 }
 
@@ -71,11 +90,110 @@ dq_status validate(const dq_calib_config* c) {
   return DQ_OK;
 }
 
+// Order the internal stream after everything the caller enqueued so far / the caller's
+// stream after everything this call enqueued.
+dq_status fence_in(dq_calib* h) {
+  DQ_CHECK_CUDA(cudaEventRecord(h->ev_in, h->user_stream));
+  DQ_CHECK_CUDA(cudaStreamWaitEvent(h->ctx.stream, h->ev_in, 0));
+  return DQ_OK;
+}
+dq_status fence_out(dq_calib* h) {
+  DQ_CHECK_CUDA(cudaEventRecord(h->ev_out, h->ctx.stream));
+  DQ_CHECK_CUDA(cudaStreamWaitEvent(h->user_stream, h->ev_out, 0));
+  return DQ_OK;
+}
+
 dq_status ensure_rotation(dq_calib* h) {
   if (!h->r_stale) return DQ_OK;
-  DQ_CHECK(qr_forward(h->ctx, h->ws, h->Z, h->R, h->U, tc_rt_operand(h->tc), h->cfg.d, h->cfg.batch));
+  if (h->fast_qr) {
+    DQ_CHECK(qr_forward_fast(h->ctx, h->ws, h->qtc, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch));
+  } else {
+    DQ_CHECK(qr_forward(h->ctx, h->ws, h->Z, h->R, h->U, tc_rt_operand(h->tc), h->cfg.d, h->cfg.batch));
+  }
   h->r_stale = false;
   return DQ_OK;
+}
+
+// One iteration of Algorithm 1 (lines 7-10) enqueued on the work stream.
+dq_status enqueue_step(dq_calib* h, bool timed) {
+  const dq_calib_config& c = h->cfg;
+  const int d = c.d, batch = c.batch;
+  const int64_t N = c.n_tokens;
+  const float inv_n = (c.reduction == DQ_MEAN_TOKENS) ? (float)(1.0 / (double)N) : 1.f;
+  Ctx& ctx = h->ctx;
+  if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[0], ctx.stream));
+  // (a1) R <- qr(Z)
+  DQ_CHECK(ensure_rotation(h));
+  if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[1], ctx.stream));
+  // (a2-a4) O = X R, Whip epilogue, loss reduction
+  if (c.path == DQ_PATH_FP32) {
+    DQ_CHECK(whip_forward_f32(ctx, (const float*)h->X, c.ldx, N * c.ldx, h->R, (float*)h->G, h->partials, N, d,
+                              batch, nullptr));
+  } else {
+    DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
+  }
+  DQ_CHECK(loss_finalize(ctx, h->partials, h->n_partials, batch, inv_n, nullptr, h->loss_last));
+  if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[2], ctx.stream));
+  // (a5) Gq = (1/N) X^T G
+  if (c.path == DQ_PATH_FP32) {
+    GemmDesc g{};
+    g.A = (const float*)h->X; g.lda = c.ldx; g.transA = 1; g.sA = N * c.ldx;
+    g.B = (const float*)h->G; g.ldb = d; g.transB = 0; g.sB = N * (int64_t)d;
+    g.M = d; g.N = d; g.K = (int)N; g.alpha = inv_n; g.beta = 0.f; g.batch = batch;
+    if (h->gq_ks <= 1) {
+      g.C = h->Gq; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = 1;
+      DQ_CHECK(gemm_f32(ctx, g));
+    } else {   // deterministic split-K over the token dimension
+      g.C = h->gq_part; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = h->gq_ks;
+      DQ_CHECK(gemm_f32(ctx, g));
+      DQ_CHECK(splitk_reduce(ctx, h->gq_part, h->gq_ks, (int64_t)d * d, batch, 1.f, 0.f, h->Gq));
+    }
+  } else {
+    DQ_CHECK(tc_grad_rotation(h->tc, ctx, h->Gq, inv_n));
+  }
+  if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[3], ctx.stream));
+  // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
+  if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch));
+  else DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch));
+  if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
+  // (a7) Z <- Z - lr Gz
+  DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, (int64_t)d * d * batch));
+  h->r_stale = true;
+  if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[5], ctx.stream));
+  return DQ_OK;
+}
+
+// Capture one full step into an executable graph (after one eager step has set every
+// kernel attribute).  Failure is not an error: the handle keeps launching eagerly.
+void try_capture(dq_calib* h) {
+  if (h->graph || h->graph_failed) return;
+  const int64_t before = h->ctx.launches;
+  h->r_stale = true;
+  if (cudaStreamBeginCapture(h->ctx.stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    h->graph_failed = true;
+    return;
+  }
+  const dq_status st = enqueue_step(h, false);
+  cudaGraph_t g = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(h->ctx.stream, &g);
+  if (st != DQ_OK || e != cudaSuccess || !g) {
+    cudaGetLastError();
+    if (g) cudaGraphDestroy(g);
+    h->graph_failed = true;
+    h->ctx.launches = before;
+    h->r_stale = true;
+    return;
+  }
+  if (cudaGraphInstantiate(&h->graph, g, 0) != cudaSuccess) {
+    cudaGetLastError();
+    h->graph = nullptr;
+    h->graph_failed = true;
+  }
+  cudaGraphDestroy(g);
+  h->graph_launches = h->ctx.launches - before;
+  h->ctx.launches = before;      // capture enqueued nothing
+  h->r_stale = true;
 }
 
 }  // namespace
@@ -113,13 +231,16 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
   dq_calib* h = new (std::nothrow) dq_calib();
   if (!h) return DQ_ERR_ALLOC;
   h->cfg = *cfg;
-  h->ctx.stream = (cudaStream_t)cuda_stream;
+  h->user_stream = (cudaStream_t)cuda_stream;
   h->ctx.sm_count = sms;
   h->X = d_X;
   const int d = cfg->d, batch = cfg->batch;
   const int64_t dd = (int64_t)d * d * batch;
   dq_status st = DQ_OK;
   auto A = [&](dq_status s) { if (st == DQ_OK) st = s; };
+  if (cudaStreamCreateWithFlags(&h->ctx.stream, cudaStreamNonBlocking) != cudaSuccess) st = DQ_ERR_CUDA;
+  if (st == DQ_OK && cudaEventCreateWithFlags(&h->ev_in, cudaEventDisableTiming) != cudaSuccess) st = DQ_ERR_CUDA;
+  if (st == DQ_OK && cudaEventCreateWithFlags(&h->ev_out, cudaEventDisableTiming) != cudaSuccess) st = DQ_ERR_CUDA;
   A(dev_alloc(&h->ctx.d_status, 1));
   A(dev_alloc(&h->Z, dd)); A(dev_alloc(&h->R, dd)); A(dev_alloc(&h->U, dd));
   A(dev_alloc(&h->Gq, dd)); A(dev_alloc(&h->Gz, dd));
@@ -129,6 +250,11 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
   A(dev_alloc(&h->ws.T, (int64_t)batch * d * 32));
   A(dev_alloc(&h->ws.W, (int64_t)batch * d * 32)); A(dev_alloc(&h->ws.W2, (int64_t)batch * d * 32));
   A(dev_alloc(&h->loss_last, batch));
+  if (st == DQ_OK) {
+    for (auto& e : h->ev)
+      if (cudaEventCreate(&e) != cudaSuccess) st = DQ_ERR_CUDA;
+  }
+  if (st == DQ_OK) st = fence_in(h);
   if (cfg->path == DQ_PATH_FP32) {
     h->g_elems = (int64_t)batch * cfg->n_tokens * d;
     float* g = nullptr;
@@ -146,15 +272,15 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
     __nv_bfloat16* g = nullptr;
     A(dev_alloc(&g, h->g_elems));
     h->G = g;
-    if (st == DQ_OK) A(tc_init(h->tc, h->ctx, *cfg, d_X, (__nv_bfloat16*)h->G, &h->n_partials));
+    if (st == DQ_OK) A(qr_tc_init(h->qtc, d, batch));
+    h->fast_qr = (st == DQ_OK);
+    if (st == DQ_OK)
+      A(tc_init(h->tc, h->ctx, *cfg, d_X, (__nv_bfloat16*)h->G, h->qtc.rt_hi, &h->n_partials));
   }
   A(dev_alloc(&h->partials, (int64_t)batch * (h->n_partials > 0 ? h->n_partials : 1)));
-  if (st == DQ_OK) {
-    for (auto& e : h->ev)
-      if (cudaEventCreate(&e) != cudaSuccess) st = DQ_ERR_CUDA;
-  }
   if (st == DQ_OK && cudaMemsetAsync(h->ctx.d_status, 0, sizeof(int), h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
   if (st == DQ_OK && cudaMemcpyAsync(h->Z, d_Z0, sizeof(float) * dd, cudaMemcpyDeviceToDevice, h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
+  if (st == DQ_OK) st = fence_out(h);
   if (st != DQ_OK) { free_all(h); return st; }
   *out = h;
   return DQ_OK;
@@ -162,92 +288,69 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
 
 dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
   if (!h || n_steps < 0) return DQ_ERR_INVALID_ARG;
-  const dq_calib_config& c = h->cfg;
-  const int d = c.d, batch = c.batch;
-  const int64_t N = c.n_tokens;
-  const float inv_n = (c.reduction == DQ_MEAN_TOKENS) ? (float)(1.0 / (double)N) : 1.f;
+  const int batch = h->cfg.batch;
   Ctx& ctx = h->ctx;
+  DQ_CHECK(fence_in(h));
   if (h->timing) { for (auto& m : h->ms_acc) m = 0.0; h->timed_steps = 0; }
   for (int s = 0; s < n_steps; ++s) {
-    float* loss_slot = d_loss_out ? d_loss_out + (int64_t)s * batch : nullptr;
-    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[0], ctx.stream));
-    // (a1) R <- qr(Z)
-    DQ_CHECK(ensure_rotation(h));
-    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[1], ctx.stream));
-    // (a2-a4) O = X R, Whip epilogue, loss reduction
-    if (c.path == DQ_PATH_FP32) {
-      DQ_CHECK(whip_forward_f32(ctx, (const float*)h->X, c.ldx, N * c.ldx, h->R, (float*)h->G,
-                                h->partials, N, d, batch, nullptr));
+    const bool use_graph = !h->timing && h->r_stale && h->eager_steps_done >= 1;
+    if (use_graph && !h->graph && !h->graph_failed) try_capture(h);
+    if (use_graph && h->graph) {
+      DQ_CHECK_CUDA(cudaGraphLaunch(h->graph, ctx.stream));
+      ctx.launches += h->graph_launches;
+      h->r_stale = true;
     } else {
-      DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
-    }
-    DQ_CHECK(loss_finalize(ctx, h->partials, h->n_partials, batch, inv_n, loss_slot, h->loss_last));
-    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[2], ctx.stream));
-    // (a5) Gq = (1/N) X^T G
-    if (c.path == DQ_PATH_FP32) {
-      GemmDesc g{};
-      g.A = (const float*)h->X; g.lda = c.ldx; g.transA = 1; g.sA = N * c.ldx;
-      g.B = (const float*)h->G; g.ldb = d; g.transB = 0; g.sB = N * (int64_t)d;
-      g.M = d; g.N = d; g.K = (int)N; g.alpha = inv_n; g.beta = 0.f; g.batch = batch;
-      if (h->gq_ks <= 1) {
-        g.C = h->Gq; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = 1;
-        DQ_CHECK(gemm_f32(ctx, g));
-      } else {   // deterministic split-K over the token dimension
-        g.C = h->gq_part; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = h->gq_ks;
-        DQ_CHECK(gemm_f32(ctx, g));
-        DQ_CHECK(splitk_reduce(ctx, h->gq_part, h->gq_ks, (int64_t)d * d, batch, 1.f, 0.f, h->Gq));
+      DQ_CHECK(enqueue_step(h, h->timing));
+      h->eager_steps_done++;
+      if (h->timing) {
+        DQ_CHECK_CUDA(cudaEventSynchronize(h->ev[DQ_PHASE_COUNT]));
+        for (int p = 0; p < DQ_PHASE_COUNT; ++p) {
+          float ms = 0.f;
+          DQ_CHECK_CUDA(cudaEventElapsedTime(&ms, h->ev[p], h->ev[p + 1]));
+          h->ms_acc[p] += ms;
+        }
+        h->timed_steps++;
       }
-    } else {
-      DQ_CHECK(tc_grad_rotation(h->tc, ctx, h->Gq, inv_n));
     }
-    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[3], ctx.stream));
-    // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
-    DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch));
-    if (h->timing) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
-    // (a7) Z <- Z - lr Gz
-    DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, (int64_t)d * d * batch));
-    h->r_stale = true;
-    if (h->timing) {
-      DQ_CHECK_CUDA(cudaEventRecord(h->ev[5], ctx.stream));
-      DQ_CHECK_CUDA(cudaEventSynchronize(h->ev[5]));
-      for (int p = 0; p < DQ_PHASE_COUNT; ++p) {
-        float ms = 0.f;
-        DQ_CHECK_CUDA(cudaEventElapsedTime(&ms, h->ev[p], h->ev[p + 1]));
-        h->ms_acc[p] += ms;
-      }
-      h->timed_steps++;
-    }
+    if (d_loss_out)
+      DQ_CHECK_CUDA(cudaMemcpyAsync(d_loss_out + (int64_t)s * batch, h->loss_last, sizeof(float) * batch,
+                                    cudaMemcpyDeviceToDevice, ctx.stream));
   }
-  return DQ_OK;
+  return fence_out(h);
 }
 
 dq_status dq_calib_get_rotation(dq_calib_t* h, float* d_R_out) {
   if (!h || !d_R_out) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK(fence_in(h));
   DQ_CHECK(ensure_rotation(h));
   DQ_CHECK_CUDA(cudaMemcpyAsync(d_R_out, h->R, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
                                 cudaMemcpyDeviceToDevice, h->ctx.stream));
-  return DQ_OK;
+  return fence_out(h);
 }
 
 dq_status dq_calib_refresh_inputs(dq_calib_t* h) {
   if (!h) return DQ_ERR_INVALID_ARG;
-  if (h->cfg.path == DQ_PATH_BF16_TC) return tc_refresh_inputs(h->tc, h->ctx);
-  return DQ_OK;
+  if (h->cfg.path != DQ_PATH_BF16_TC) return DQ_OK;
+  DQ_CHECK(fence_in(h));
+  DQ_CHECK(tc_refresh_inputs(h->tc, h->ctx));
+  return fence_out(h);
 }
 
 dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out) {
   if (!h || !d_Z_out) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK(fence_in(h));
   DQ_CHECK_CUDA(cudaMemcpyAsync(d_Z_out, h->Z, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
                                 cudaMemcpyDeviceToDevice, h->ctx.stream));
-  return DQ_OK;
+  return fence_out(h);
 }
 
 dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z) {
   if (!h || !d_Z) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK(fence_in(h));
   DQ_CHECK_CUDA(cudaMemcpyAsync(h->Z, d_Z, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
                                 cudaMemcpyDeviceToDevice, h->ctx.stream));
   h->r_stale = true;
-  return DQ_OK;
+  return fence_out(h);
 }
 
 dq_status dq_calib_status(dq_calib_t* h) {

@@ -88,6 +88,8 @@ struct QrWorkspace {
   float* S = nullptr;     // tril(B - B^T, -1)
   float* tmp = nullptr;   // [batch][d][d] scratch for the triangular inverse
 };
+// Factorisation only: ws.A <- raw upper factor, ws.V / ws.T <- reflectors.
+dq_status qr_factor(Ctx& ctx, QrWorkspace& ws, const float* Z, int d, int batch);
 // Z -> R (rotation, diag(U) > 0), U.  Optionally also a bf16 copy of R^T.
 dq_status qr_forward(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float* U,
                      __nv_bfloat16* Rt_bf16 /* nullable */, int d, int batch);

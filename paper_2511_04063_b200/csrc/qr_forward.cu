@@ -303,8 +303,9 @@ dq_status apply_block_reflector(Ctx& ctx, QrWorkspace& ws, float* C, int d, int 
 
 }  // namespace
 
-dq_status qr_forward(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float* U,
-                     __nv_bfloat16* Rt_bf16, int d, int batch) {
+// Blocked Householder factorisation only: ws.A <- raw upper factor (Algorithm 2 signs),
+// ws.V / ws.T <- compact-WY reflectors.
+dq_status qr_factor(Ctx& ctx, QrWorkspace& ws, const float* Z, int d, int batch) {
   if (d % PB != 0 || d > PC * PT * RPT) return DQ_ERR_UNSUPPORTED;
   const int64_t dd = (int64_t)d * d;
   DQ_CHECK_CUDA(cudaMemcpyAsync(ws.A, Z, sizeof(float) * dd * batch, cudaMemcpyDeviceToDevice, ctx.stream));
@@ -318,7 +319,14 @@ dq_status qr_forward(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float*
     if (nt > 0) DQ_CHECK(apply_block_reflector(ctx, ws, ws.A, d, batch, c0, c0 + PB, nt, /*transT=*/1));
   }
   diag_check_kernel<<<batch, 256, 0, ctx.stream>>>(ws.A, d, ctx.d_status);
-  DQ_CHECK(after_launch(ctx));
+  return after_launch(ctx);
+}
+
+dq_status qr_forward(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float* U,
+                     __nv_bfloat16* Rt_bf16, int d, int batch) {
+  DQ_CHECK(qr_factor(ctx, ws, Z, d, batch));
+  const int64_t dd = (int64_t)d * d;
+  const int np = d / PB;
   // Q = H_1 ... H_n applied to I, last panel first; only Q[c0:, c0:] is touched.
   {
     int bx = (int)((dd + 255) / 256);

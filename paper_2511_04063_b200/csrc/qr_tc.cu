@@ -1,0 +1,269 @@
+// QR-Orth on the tensor cores ("fast" mode used with the tensor-core path).
+//
+// Forward:  blocked Householder factorisation Z = Q U (only U is kept), gauge
+//           diag(U) > 0, W = U^-1 by recursive block inversion, R = Z W.
+//           (R is the same orthogonal factor the reflectors would give; forming it
+//           as Z U^-1 costs one GEMM instead of d/32 dependent block updates.  Its
+//           orthogonality error grows like cond(Z) * 2^-16, which is fine for the
+//           near-orthogonal latents of the calibration loop.)
+// Backward: B = R^T Gq, S = tril(B - B^T, -1), Gz = (R S) W^T.
+// All d x d products run as split-bf16 tcgen05 GEMMs (three bf16 MMAs per product,
+// fp32 accumulation, ~2^-16 relative error).
+#include "tc_host.cuh"
+#include "tc_path.cuh"
+
+namespace dq {
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+__device__ __forceinline__ void split2(float v, bf16& hi, bf16& lo) {
+  hi = __float2bfloat16_rn(v);
+  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+// dst(hi, lo)[b][r][c] = split(src[b][r][c])             (transpose == 0)
+// dst(hi, lo)[b][c][r] = split(src[b][r][c])             (transpose == 1)
+// src is n x n fp32 row-major (n % 32 == 0); dst dense n x n.
+__global__ void __launch_bounds__(256) split_kernel(const float* __restrict__ src, bf16* __restrict__ hi,
+                                                    bf16* __restrict__ lo, int n, int transpose) {
+  __shared__ float t[32][33];
+  const int64_t off = (int64_t)blockIdx.z * n * n;
+  src += off; hi += off; lo += off;
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  if (!transpose) {
+    for (int r = ty; r < 32; r += 8) {
+      const int64_t i = (int64_t)(r0 + r) * n + c0 + tx;
+      split2(src[i], hi[i], lo[i]);
+    }
+  } else {
+    for (int r = ty; r < 32; r += 8) t[r][tx] = src[(int64_t)(r0 + r) * n + c0 + tx];
+    __syncthreads();
+    for (int c = ty; c < 32; c += 8) {
+      const int64_t i = (int64_t)(c0 + c) * n + r0 + tx;
+      split2(t[tx][c], hi[i], lo[i]);
+    }
+  }
+}
+
+// Gauge of the raw factor: U = diag(s) triu(A), s_i = sign(A_ii) (+1 at 0); fp32 + split copy.
+__global__ void __launch_bounds__(256) gauge_u_kernel(const float* __restrict__ A, float* __restrict__ U,
+                                                      bf16* __restrict__ hi, bf16* __restrict__ lo, int d) {
+  const int64_t off = (int64_t)blockIdx.z * d * d;
+  A += off; U += off; hi += off; lo += off;
+  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int r = ty; r < 32; r += 8) {
+    const int i = i0 + r, j = j0 + tx;
+    const float si = (A[(int64_t)i * d + i] < 0.f) ? -1.f : 1.f;
+    const float v = (j >= i) ? si * A[(int64_t)i * d + j] : 0.f;
+    const int64_t idx = (int64_t)i * d + j;
+    U[idx] = v;
+    split2(v, hi[idx], lo[idx]);
+  }
+}
+
+// St(hi, lo)[j][k] = S[k][j] with S = tril(B - B^T, -1):  (k > j) ? B[k][j] - B[j][k] : 0
+__global__ void __launch_bounds__(256) skew_t_split_kernel(const float* __restrict__ B, bf16* __restrict__ hi,
+                                                           bf16* __restrict__ lo, int d) {
+  __shared__ float t[32][33];
+  const int64_t off = (int64_t)blockIdx.z * d * d;
+  B += off; hi += off; lo += off;
+  const int j0 = blockIdx.y * 32, k0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  if (k0 + 31 <= j0) {   // tile entirely on or below the diagonal of St: zeros
+    for (int r = ty; r < 32; r += 8) {
+      const int64_t i = (int64_t)(j0 + r) * d + k0 + tx;
+      hi[i] = __float2bfloat16_rn(0.f); lo[i] = __float2bfloat16_rn(0.f);
+    }
+    return;
+  }
+  for (int r = ty; r < 32; r += 8) t[r][tx] = B[(int64_t)(k0 + r) * d + j0 + tx];   // B[k][j]
+  __syncthreads();
+  for (int r = ty; r < 32; r += 8) {
+    const int j = j0 + r, k = k0 + tx;
+    const float v = (k > j) ? t[tx][r] - B[(int64_t)j * d + k] : 0.f;
+    const int64_t i = (int64_t)j * d + k;
+    split2(v, hi[i], lo[i]);
+  }
+}
+
+// Inverse of each 128 x 128 upper-triangular diagonal block of U; thread j solves U x = e_j
+// by back-substitution.  Writes the split inverse in row-major (WN) and transposed (WT) form.
+constexpr int DB = 128;
+__global__ void __launch_bounds__(DB) tri_inv_diag128_kernel(const float* __restrict__ U, bf16* __restrict__ wn_hi,
+                                                             bf16* __restrict__ wn_lo, bf16* __restrict__ wt_hi,
+                                                             bf16* __restrict__ wt_lo, int d) {
+  extern __shared__ float sm[];
+  float (*Us)[DB + 1] = reinterpret_cast<float (*)[DB + 1]>(sm);
+  float (*Xs)[DB + 1] = reinterpret_cast<float (*)[DB + 1]>(sm + DB * (DB + 1));
+  const int64_t off = (int64_t)blockIdx.y * d * d + (int64_t)blockIdx.x * DB * (d + 1);
+  U += off; wn_hi += off; wn_lo += off; wt_hi += off; wt_lo += off;
+  const int j = threadIdx.x;
+  for (int r = 0; r < DB; ++r) Us[r][j] = U[(int64_t)r * d + j];
+  __syncthreads();
+  for (int i = DB - 1; i > j; --i) Xs[i][j] = 0.f;
+  Xs[j][j] = 1.f / Us[j][j];
+  for (int i = j - 1; i >= 0; --i) {
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    int k = i + 1;
+    for (; k + 3 <= j; k += 4) {
+      s0 = fmaf(Us[i][k], Xs[k][j], s0);
+      s1 = fmaf(Us[i][k + 1], Xs[k + 1][j], s1);
+      s2 = fmaf(Us[i][k + 2], Xs[k + 2][j], s2);
+      s3 = fmaf(Us[i][k + 3], Xs[k + 3][j], s3);
+    }
+    for (; k <= j; ++k) s0 = fmaf(Us[i][k], Xs[k][j], s0);
+    Xs[i][j] = -((s0 + s1) + (s2 + s3)) / Us[i][i];
+  }
+  __syncthreads();
+  for (int r = 0; r < DB; ++r) {
+    bf16 h, l;
+    split2(Xs[r][j], h, l);                       // X[r][j] -> WN[r][j]
+    wn_hi[(int64_t)r * d + j] = h; wn_lo[(int64_t)r * d + j] = l;
+    split2(Xs[j][r], h, l);                       // X[j][r] -> WT[r][j]
+    wt_hi[(int64_t)r * d + j] = h; wt_lo[(int64_t)r * d + j] = l;
+  }
+}
+
+struct Op {   // K-major operand: rows x K, split pair, leading dimension, batch stride (elements)
+  const bf16* hi; const bf16* lo; int64_t ld; int64_t bs;
+};
+struct Out {
+  float* f32 = nullptr; int64_t ld = 0; int64_t bs = 0;
+  bf16* hi = nullptr; bf16* lo = nullptr; int64_t ld_h = 0; int64_t bs_h = 0;
+  float alpha = 1.f, beta = 0.f;
+};
+
+// D[m][n] = alpha sum_k A[m][k] B[n][k] (+ beta D) with split-bf16 operands; M, N % 128 == 0, K % 64 == 0.
+dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, int batch, const Out& o) {
+  if (M % 128 || N % 128 || K % 64) return DQ_ERR_UNSUPPORTED;
+  CUtensorMap ma, mal, mb, mbl;
+  const int64_t bsa = A.bs ? A.bs : (int64_t)M * A.ld, bsb = B.bs ? B.bs : (int64_t)N * B.ld;
+  DQ_CHECK(tch::make_map(&ma, A.hi, K, M, batch, A.ld, bsa, tc::BLOCK_M));
+  DQ_CHECK(tch::make_map(&mal, A.lo, K, M, batch, A.ld, bsa, tc::BLOCK_M));
+  DQ_CHECK(tch::make_map(&mb, B.hi, K, N, batch, B.ld, bsb, 128));
+  DQ_CHECK(tch::make_map(&mbl, B.lo, K, N, batch, B.ld, bsb, 128));
+  tc::Params p{};
+  p.m_blocks = M / 128; p.n_blocks = N / 128; p.batch = batch; p.ksplit = 1; p.k_blocks = K / tc::BLOCK_K;
+  p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = 0;
+  p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
+  p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
+  return tch::launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
+}
+
+// Block column of the inverse:  W[0:k, k:k+s] = -W[0:k,0:k] U[0:k, k:k+s] W[k:k+s, k:k+s]
+// for `count` independent diagonal positions `stride` elements apart (3rd tensor dimension).
+dq_status merge(Ctx& ctx, QrTcState& q, int d, int k, int s, int count, int64_t stride, int64_t base) {
+  // T1t[j][i] = sum_l W22^T[j][l] U12[i][l]        (s x k, dense temporary)
+  Op a{q.wt_hi + base + (int64_t)k * d + k, q.wt_lo + base + (int64_t)k * d + k, d, stride};
+  Op b{q.u_hi + base + k, q.u_lo + base + k, d, stride};
+  Out t1; t1.hi = q.t1_hi; t1.lo = q.t1_lo; t1.ld_h = k; t1.bs_h = (int64_t)s * k;
+  DQ_CHECK(gemm3(ctx, a, b, s, k, s, count, t1));
+  Op w11{q.wn_hi + base, q.wn_lo + base, d, stride};
+  Op t1o{q.t1_hi, q.t1_lo, k, (int64_t)s * k};
+  // W12[i][j] = -sum_l W11[i][l] T1t[j][l]   -> WN block (0, k)
+  Out o12; o12.hi = q.wn_hi + base + k; o12.lo = q.wn_lo + base + k; o12.ld_h = d; o12.bs_h = stride; o12.alpha = -1.f;
+  DQ_CHECK(gemm3(ctx, w11, t1o, k, s, k, count, o12));
+  // W12^T[j][i] = -sum_l T1t[j][l] W11[i][l] -> WT block (k, 0)
+  Out o21; o21.hi = q.wt_hi + base + (int64_t)k * d; o21.lo = q.wt_lo + base + (int64_t)k * d; o21.ld_h = d;
+  o21.bs_h = stride; o21.alpha = -1.f;
+  return gemm3(ctx, t1o, w11, s, k, k, count, o21);
+}
+
+dq_status tri_inverse_tc(Ctx& ctx, QrTcState& q, const float* U, int d, int batch) {
+  const int64_t dd = (int64_t)d * d;
+  const size_t bytes = sizeof(bf16) * (size_t)dd * batch;
+  DQ_CHECK_CUDA(cudaMemsetAsync(q.wn_hi, 0, bytes, ctx.stream));
+  DQ_CHECK_CUDA(cudaMemsetAsync(q.wn_lo, 0, bytes, ctx.stream));
+  DQ_CHECK_CUDA(cudaMemsetAsync(q.wt_hi, 0, bytes, ctx.stream));
+  DQ_CHECK_CUDA(cudaMemsetAsync(q.wt_lo, 0, bytes, ctx.stream));
+  const int smem = 2 * DB * (DB + 1) * (int)sizeof(float);
+  static bool attr = false;
+  if (!attr) {
+    DQ_CHECK_CUDA(cudaFuncSetAttribute(tri_inv_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr = true;
+  }
+  tri_inv_diag128_kernel<<<dim3(d / DB, batch), DB, smem, ctx.stream>>>(U, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, d);
+  DQ_CHECK(after_launch(ctx));
+  int s = DB, count = d / DB;
+  while (count > 1 && count % 2 == 0) {
+    const int pairs = count / 2;
+    const int64_t pair_stride = (int64_t)2 * s * (d + 1);
+    if (batch == 1) {
+      DQ_CHECK(merge(ctx, q, d, s, s, pairs, pair_stride, 0));
+    } else {
+      for (int pidx = 0; pidx < pairs; ++pidx) DQ_CHECK(merge(ctx, q, d, s, s, batch, dd, pidx * pair_stride));
+    }
+    s *= 2; count = pairs;
+  }
+  for (int kb = 1; kb < count; ++kb) DQ_CHECK(merge(ctx, q, d, kb * s, s, batch, dd, 0));
+  return DQ_OK;
+}
+
+template <typename T>
+dq_status alloc(T** p, int64_t n) {
+  return cudaMalloc((void**)p, sizeof(T) * (size_t)n) == cudaSuccess ? DQ_OK : DQ_ERR_ALLOC;
+}
+
+}  // namespace
+
+dq_status qr_tc_init(QrTcState& q, int d, int batch) {
+  const int64_t dd = (int64_t)d * d * batch;
+  bf16** all[] = {&q.z_hi, &q.z_lo, &q.u_hi, &q.u_lo, &q.wn_hi, &q.wn_lo, &q.wt_hi, &q.wt_lo, &q.r_hi, &q.r_lo,
+                  &q.rt_hi, &q.rt_lo, &q.gqt_hi, &q.gqt_lo, &q.st_hi, &q.st_lo, &q.m_hi, &q.m_lo, &q.t1_hi, &q.t1_lo};
+  for (bf16** p : all) DQ_CHECK(alloc(p, dd));
+  q.ready = true;
+  return DQ_OK;
+}
+
+void qr_tc_destroy(QrTcState& q) {
+  bf16* all[] = {q.z_hi, q.z_lo, q.u_hi, q.u_lo, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, q.r_hi, q.r_lo,
+                 q.rt_hi, q.rt_lo, q.gqt_hi, q.gqt_lo, q.st_hi, q.st_lo, q.m_hi, q.m_lo, q.t1_hi, q.t1_lo};
+  for (bf16* p : all) cudaFree(p);
+  q = QrTcState();
+}
+
+dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
+                          int batch) {
+  if (d % 128 != 0) return DQ_ERR_UNSUPPORTED;
+  const int64_t dd = (int64_t)d * d;
+  const dim3 tiles(d / 32, d / 32, batch);
+  DQ_CHECK(qr_factor(ctx, ws, Z, d, batch));
+  gauge_u_kernel<<<tiles, 256, 0, ctx.stream>>>(ws.A, U, q.u_hi, q.u_lo, d);
+  DQ_CHECK(after_launch(ctx));
+  DQ_CHECK(tri_inverse_tc(ctx, q, U, d, batch));
+  split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
+  DQ_CHECK(after_launch(ctx));
+  // R[i][j] = sum_k Z[i][k] W[k][j]:  A = Z (row-major), B = W^T
+  Op a{q.z_hi, q.z_lo, d, dd};
+  Op b{q.wt_hi, q.wt_lo, d, dd};
+  Out o; o.f32 = R; o.ld = d; o.bs = dd; o.hi = q.r_hi; o.lo = q.r_lo; o.ld_h = d; o.bs_h = dd;
+  DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
+  split_kernel<<<tiles, 256, 0, ctx.stream>>>(R, q.rt_hi, q.rt_lo, d, 1);
+  return after_launch(ctx);
+}
+
+dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch) {
+  const int64_t dd = (int64_t)d * d;
+  const dim3 tiles(d / 32, d / 32, batch);
+  split_kernel<<<tiles, 256, 0, ctx.stream>>>(Gq, q.gqt_hi, q.gqt_lo, d, 1);
+  DQ_CHECK(after_launch(ctx));
+  // B[i][j] = sum_k R[k][i] Gq[k][j]:  A = R^T, B-operand = Gq^T
+  Op rt{q.rt_hi, q.rt_lo, d, dd}, gqt{q.gqt_hi, q.gqt_lo, d, dd};
+  Out ob; ob.f32 = ws.B; ob.ld = d; ob.bs = dd;
+  DQ_CHECK(gemm3(ctx, rt, gqt, d, d, d, batch, ob));
+  skew_t_split_kernel<<<tiles, 256, 0, ctx.stream>>>(ws.B, q.st_hi, q.st_lo, d);
+  DQ_CHECK(after_launch(ctx));
+  // M[i][j] = sum_k R[i][k] S[k][j]:  A = R, B-operand = S^T; only the split copy is kept
+  Op r{q.r_hi, q.r_lo, d, dd}, st{q.st_hi, q.st_lo, d, dd};
+  Out om; om.hi = q.m_hi; om.lo = q.m_lo; om.ld_h = d; om.bs_h = dd;
+  DQ_CHECK(gemm3(ctx, r, st, d, d, d, batch, om));
+  // Gz[i][j] = sum_k M[i][k] W[j][k]
+  Op m{q.m_hi, q.m_lo, d, dd}, wn{q.wn_hi, q.wn_lo, d, dd};
+  Out og; og.f32 = Gz; og.ld = d; og.bs = dd;
+  return gemm3(ctx, m, wn, d, d, d, batch, og);
+}
+
+}  // namespace dq

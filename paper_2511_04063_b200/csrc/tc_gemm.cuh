@@ -24,15 +24,19 @@ constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr uint64_t WAIT_LIMIT_NS = 4000000000ull;
 
-enum { EPI_WHIP = 0, EPI_F32 = 1, EPI_BF16 = 2 };
+enum { EPI_WHIP = 0, EPI_GEN = 1, EPI_BF16 = 2 };
 
 struct Params {
   int m_blocks, n_blocks, batch, ksplit;
   int k_blocks;            // K / 64 (whole reduction)
   // output addressing: out + b * batch_stride + split * split_stride + m * ld + n
-  void* out;
+  void* out;               // EPI_WHIP / EPI_BF16: bf16; EPI_GEN: fp32 (nullable)
   int64_t ld, batch_stride, split_stride;
-  float alpha;
+  // EPI_GEN only: v = alpha * acc + beta * out_old; optional split-bf16 copy (hi + lo ~ v)
+  __nv_bfloat16* out_hi;
+  __nv_bfloat16* out_lo;
+  int64_t ld_h, batch_stride_h;
+  float alpha, beta;
   float* partials;         // EPI_WHIP: [unit][4] loss partial sums
   int* d_status;
 };
@@ -306,12 +310,42 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 #pragma unroll
           for (int i = 0; i < 4; ++i)
             dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-        } else if (EPI == EPI_F32) {
-          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_off + c * 32);
+        } else if (EPI == EPI_GEN) {
+          float f[32];
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            dst[i] = make_float4(p.alpha * __uint_as_float(v[4 * i]), p.alpha * __uint_as_float(v[4 * i + 1]),
-                                 p.alpha * __uint_as_float(v[4 * i + 2]), p.alpha * __uint_as_float(v[4 * i + 3]));
+          for (int i = 0; i < 32; ++i) f[i] = p.alpha * __uint_as_float(v[i]);
+          if (p.out) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_off + c * 32);
+            if (p.beta != 0.f) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float4 o = dst[i];
+                f[4 * i] = fmaf(p.beta, o.x, f[4 * i]); f[4 * i + 1] = fmaf(p.beta, o.y, f[4 * i + 1]);
+                f[4 * i + 2] = fmaf(p.beta, o.z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.beta, o.w, f[4 * i + 3]);
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+          }
+          if (p.out_hi) {
+            const int64_t off_h = (int64_t)b * p.batch_stride_h + (int64_t)row * p.ld_h + (int64_t)nb * BLOCK_N + c * 32;
+            uint32_t ph[16], pl[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+              const float2 hf = __bfloat1622float2(h);
+              const __nv_bfloat162 l = __floats2bfloat162_rn(f[2 * i] - hf.x, f[2 * i + 1] - hf.y);
+              ph[i] = *reinterpret_cast<const uint32_t*>(&h);
+              pl[i] = *reinterpret_cast<const uint32_t*>(&l);
+            }
+            uint4* dh = reinterpret_cast<uint4*>(p.out_hi + off_h);
+            uint4* dl = reinterpret_cast<uint4*>(p.out_lo + off_h);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              dh[i] = make_uint4(ph[4 * i], ph[4 * i + 1], ph[4 * i + 2], ph[4 * i + 3]);
+              dl[i] = make_uint4(pl[4 * i], pl[4 * i + 1], pl[4 * i + 2], pl[4 * i + 3]);
+            }
+          }
         } else {
           uint32_t packed[16];
 #pragma unroll

@@ -1,43 +1,11 @@
 // Host side of the tensor-core path: tensor maps, operand copies, launches.
 #include <vector>
 
-#include "tc_gemm.cuh"
+#include "tc_host.cuh"
 #include "tc_path.cuh"
 
 namespace dq {
 namespace {
-
-using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn get_encode_fn() {
-  static EncodeFn fn = nullptr;
-  if (fn) return fn;
-  void* p = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-      qres != cudaDriverEntryPointSuccess)
-    return nullptr;
-  fn = reinterpret_cast<EncodeFn>(p);
-  return fn;
-}
-
-// bf16 tensor [batch][rows][k] (k contiguous, row stride ld elements), box = {64, box_rows, 1},
-// 128-byte swizzle: the shared-memory image is the K-major SW128 layout tcgen05 reads.
-dq_status make_map(CUtensorMap* m, const void* base, int64_t k, int64_t rows, int64_t batch, int64_t ld,
-                   int64_t batch_stride, int box_rows) {
-  EncodeFn fn = get_encode_fn();
-  if (!fn) return DQ_ERR_CUDA;
-  cuuint64_t dims[3] = {(cuuint64_t)k, (cuuint64_t)rows, (cuuint64_t)batch};
-  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)batch_stride * 2};
-  cuuint32_t box[3] = {(cuuint32_t)tc::BLOCK_K, (cuuint32_t)box_rows, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? DQ_OK : DQ_ERR_CUDA;
-}
 
 // out[b][c][r] = in[b][r][c]   (bf16; rows, cols multiples of 64)
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in,
@@ -66,24 +34,6 @@ __global__ void __launch_bounds__(256) transpose_f32_to_bf16_kernel(const float*
   for (int c = ty; c < 32; c += 8) out[(int64_t)(c0 + c) * d + r0 + tx] = __float2bfloat16_rn(t[tx][c]);
 }
 
-template <int BN, int NT, int EPI>
-dq_status launch_gemm(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& alo,
-                      const CUtensorMap& blo, const tc::Params& p) {
-  using L = tc::SmemLayout<BN, NT>;
-  static bool attr_set = false;
-  auto kern = tc::tc_gemm_kernel<BN, NT, EPI>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
-      return DQ_ERR_CUDA;
-    attr_set = true;
-  }
-  const int units = p.m_blocks * p.n_blocks * p.batch * p.ksplit;
-  int grid = units < ctx.sm_count ? units : ctx.sm_count;
-  if (grid < 1) return DQ_OK;
-  kern<<<grid, tc::NUM_THREADS, L::TOTAL, ctx.stream>>>(a, b, alo, blo, p);
-  return after_launch(ctx);
-}
-
 struct Maps {
   CUtensorMap rt, x, xt, gt128, gt256;
 };
@@ -91,14 +41,18 @@ struct Maps {
 }  // namespace
 
 dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void* d_X, __nv_bfloat16* Gt,
-                  int* n_partials) {
+                  __nv_bfloat16* rt_external, int* n_partials) {
   const int d = cfg.d, batch = cfg.batch;
   const int64_t N = cfg.n_tokens;
   tc.d = d; tc.batch = batch; tc.n_tokens = N;
   tc.X = reinterpret_cast<const __nv_bfloat16*>(d_X);
   tc.Gt = Gt;
   if (cudaMalloc((void**)&tc.Xt, sizeof(__nv_bfloat16) * (size_t)batch * N * d) != cudaSuccess) return DQ_ERR_ALLOC;
-  if (cudaMalloc((void**)&tc.Rt, sizeof(__nv_bfloat16) * (size_t)batch * d * d) != cudaSuccess) return DQ_ERR_ALLOC;
+  if (rt_external) {
+    tc.Rt = rt_external; tc.rt_external = true;
+  } else if (cudaMalloc((void**)&tc.Rt, sizeof(__nv_bfloat16) * (size_t)batch * d * d) != cudaSuccess) {
+    return DQ_ERR_ALLOC;
+  }
   // split-K of Gq = X^T G over the token dimension: fill the machine, keep >= 16 k-blocks per slice
   const int bn = (d % 256 == 0) ? 256 : 128;
   const int tiles = (d / tc::BLOCK_M) * (d / bn) * batch;
@@ -111,11 +65,11 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   Maps* m = new (std::nothrow) Maps();
   if (!m) return DQ_ERR_ALLOC;
   tc.maps = m;
-  DQ_CHECK(make_map(&m->rt, tc.Rt, d, d, batch, d, (int64_t)d * d, tc::BLOCK_M));
-  DQ_CHECK(make_map(&m->x, tc.X, d, N, batch, d, N * d, 256));
-  DQ_CHECK(make_map(&m->xt, tc.Xt, N, d, batch, N, N * d, tc::BLOCK_M));
-  DQ_CHECK(make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
-  DQ_CHECK(make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
+  DQ_CHECK(tch::make_map(&m->rt, tc.Rt, d, d, batch, d, (int64_t)d * d, tc::BLOCK_M));
+  DQ_CHECK(tch::make_map(&m->x, tc.X, d, N, batch, d, N * d, 256));
+  DQ_CHECK(tch::make_map(&m->xt, tc.Xt, N, d, batch, N, N * d, tc::BLOCK_M));
+  DQ_CHECK(tch::make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
+  DQ_CHECK(tch::make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
   DQ_CHECK(tc_refresh_inputs(tc, ctx));
   tc.n_partials = (d / tc::BLOCK_M) * (int)(N / 256) * 4;
   *n_partials = tc.n_partials;
@@ -131,7 +85,7 @@ dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx) {
 }
 
 void tc_destroy(TcState& tc) {
-  cudaFree(tc.Xt); cudaFree(tc.Rt); cudaFree(tc.part);
+  cudaFree(tc.Xt); if (!tc.rt_external) cudaFree(tc.Rt); cudaFree(tc.part);
   delete reinterpret_cast<Maps*>(tc.maps);
   tc = TcState();
 }
@@ -145,7 +99,7 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
   p.k_blocks = tc.d / tc::BLOCK_K;
   p.out = tc.Gt; p.ld = tc.n_tokens; p.batch_stride = tc.n_tokens * tc.d; p.split_stride = 0;
   p.alpha = 1.f; p.partials = partials; p.d_status = ctx.d_status;
-  return launch_gemm<256, 1, tc::EPI_WHIP>(ctx, m->rt, m->x, m->rt, m->x, p);
+  return tch::launch_gemm<256, 1, tc::EPI_WHIP>(ctx, m->rt, m->x, m->rt, m->x, p);
 }
 
 // Gq = scale * X^T G : A = X^T [d][N], B = G^T [d][N], reduction over tokens.
@@ -156,14 +110,15 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
   tc::Params p{};
   p.m_blocks = d / tc::BLOCK_M; p.n_blocks = d / bn; p.batch = tc.batch; p.ksplit = tc.ksplit;
   p.k_blocks = (int)(tc.n_tokens / tc::BLOCK_K);
-  p.ld = d; p.alpha = scale; p.partials = nullptr; p.d_status = ctx.d_status;
+  p.ld = d; p.alpha = scale; p.beta = 0.f; p.out_hi = nullptr; p.out_lo = nullptr;
+  p.partials = nullptr; p.d_status = ctx.d_status;
   if (tc.ksplit == 1) {
     p.out = Gq; p.batch_stride = (int64_t)d * d; p.split_stride = 0;
   } else {
     p.out = tc.part; p.batch_stride = (int64_t)tc.ksplit * d * d; p.split_stride = (int64_t)d * d;
   }
-  if (bn == 256) DQ_CHECK((launch_gemm<256, 1, tc::EPI_F32>(ctx, m->xt, m->gt256, m->xt, m->gt256, p)));
-  else DQ_CHECK((launch_gemm<128, 1, tc::EPI_F32>(ctx, m->xt, m->gt128, m->xt, m->gt128, p)));
+  if (bn == 256) DQ_CHECK((tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, m->xt, m->gt256, m->xt, m->gt256, p)));
+  else DQ_CHECK((tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, p)));
   if (tc.ksplit > 1) DQ_CHECK(splitk_reduce(ctx, tc.part, tc.ksplit, (int64_t)d * d, tc.batch, 1.f, 0.f, Gq));
   return DQ_OK;
 }
@@ -183,16 +138,16 @@ dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t l
   dq_status st = after_launch(ctx);
   const int bn = (d % 256 == 0) ? 256 : 128;
   CUtensorMap ma, mb;
-  if (st == DQ_OK) st = make_map(&ma, d_X, d, n, 1, ldx, n * ldx, tc::BLOCK_M);
-  if (st == DQ_OK) st = make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, bn);
+  if (st == DQ_OK) st = tch::make_map(&ma, d_X, d, n, 1, ldx, n * ldx, tc::BLOCK_M);
+  if (st == DQ_OK) st = tch::make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, bn);
   if (st == DQ_OK) {
     tc::Params p{};
     p.m_blocks = (int)(n / tc::BLOCK_M); p.n_blocks = d / bn; p.batch = 1; p.ksplit = 1;
     p.k_blocks = d / tc::BLOCK_K;
     p.out = d_Y; p.ld = ldy; p.batch_stride = 0; p.split_stride = 0; p.alpha = 1.f;
     p.partials = nullptr; p.d_status = nullptr;
-    st = (bn == 256) ? launch_gemm<256, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p)
-                     : launch_gemm<128, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p);
+    st = (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p)
+                     : tch::launch_gemm<128, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p);
   }
   cudaFreeAsync(rt, ctx.stream);
   return st;

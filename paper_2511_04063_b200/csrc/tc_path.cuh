@@ -10,7 +10,8 @@ struct TcState {
   int64_t n_tokens = 0;
   const __nv_bfloat16* X = nullptr;   // [batch][N][d] token-major (borrowed)
   __nv_bfloat16* Xt = nullptr;        // [batch][d][N] channel-major copy (owned)
-  __nv_bfloat16* Rt = nullptr;        // [batch][d][d] bf16(R^T) (owned)
+  __nv_bfloat16* Rt = nullptr;        // [batch][d][d] bf16(R^T) (owned unless rt_external)
+  bool rt_external = false;
   __nv_bfloat16* Gt = nullptr;        // [batch][d][N] dL/dO, channel-major (borrowed from handle)
   float* part = nullptr;              // split-K partials of Gq (owned)
   int ksplit = 1;
@@ -19,7 +20,7 @@ struct TcState {
 };
 
 dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void* d_X,
-                  __nv_bfloat16* Gt, int* n_partials);
+                  __nv_bfloat16* Gt, __nv_bfloat16* rt_external, int* n_partials);
 void tc_destroy(TcState& tc);
 dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx);   // X changed in place: rebuild X^T
 inline __nv_bfloat16* tc_rt_operand(TcState& tc) { return tc.ready ? tc.Rt : nullptr; }
@@ -27,5 +28,26 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials);
 dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale);
 dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t ldx, const float* d_R,
                           void* d_Y, int64_t ldy);
+
+
+// Split-bf16 operand copies used by the tensor-core QR-Orth (all [batch][d][d]).
+struct QrTcState {
+  bool ready = false;
+  __nv_bfloat16 *z_hi = nullptr, *z_lo = nullptr;       // latent Z
+  __nv_bfloat16 *u_hi = nullptr, *u_lo = nullptr;       // upper factor U
+  __nv_bfloat16 *wn_hi = nullptr, *wn_lo = nullptr;     // W = U^-1, row-major
+  __nv_bfloat16 *wt_hi = nullptr, *wt_lo = nullptr;     // W^T
+  __nv_bfloat16 *r_hi = nullptr, *r_lo = nullptr;       // R
+  __nv_bfloat16 *rt_hi = nullptr, *rt_lo = nullptr;     // R^T (rt_hi is also the operand of X R)
+  __nv_bfloat16 *gqt_hi = nullptr, *gqt_lo = nullptr;   // Gq^T
+  __nv_bfloat16 *st_hi = nullptr, *st_lo = nullptr;     // S^T
+  __nv_bfloat16 *m_hi = nullptr, *m_lo = nullptr;       // R S
+  __nv_bfloat16 *t1_hi = nullptr, *t1_lo = nullptr;     // scratch of the block inversion
+};
+dq_status qr_tc_init(QrTcState& q, int d, int batch);
+void qr_tc_destroy(QrTcState& q);
+dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
+                          int batch);
+dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch);
 
 }  // namespace dq
