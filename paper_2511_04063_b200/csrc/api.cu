@@ -272,7 +272,7 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
     __nv_bfloat16* g = nullptr;
     A(dev_alloc(&g, h->g_elems));
     h->G = g;
-    if (st == DQ_OK) A(qr_tc_init(h->qtc, d, batch));
+    if (st == DQ_OK) A(qr_tc_init(h->qtc, d, batch, sms));
     h->fast_qr = (st == DQ_OK);
     if (st == DQ_OK)
       A(tc_init(h->tc, h->ctx, *cfg, d_X, (__nv_bfloat16*)h->G, h->qtc.rt_hi, &h->n_partials));

@@ -322,6 +322,11 @@ dq_status qr_factor(Ctx& ctx, QrWorkspace& ws, const float* Z, int d, int batch)
   return after_launch(ctx);
 }
 
+dq_status qr_diag_check(Ctx& ctx, const float* A, int d, int batch) {
+  diag_check_kernel<<<batch, 256, 0, ctx.stream>>>(A, d, ctx.d_status);
+  return after_launch(ctx);
+}
+
 dq_status qr_forward(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float* U,
                      __nv_bfloat16* Rt_bf16, int d, int batch) {
   DQ_CHECK(qr_factor(ctx, ws, Z, d, batch));

@@ -1,0 +1,622 @@
+// Blocked Householder factorisation (Algorithm 2 in compact-WY form) with the
+// trailing updates on the tensor cores.
+//
+// The working matrix is kept TRANSPOSED (At[c][r] = A[r][c]) so that columns are
+// contiguous: panel loads are coalesced and both tensor-core products of the
+// trailing update contract over a contiguous index.
+//
+// Per outer block of 128 columns [c0, c0 + 128), rows [c0, d) (m rows):
+//   1. qr_panel_cm_kernel   one thread-block cluster; four inner panels of 32
+//                           columns, each held in registers (two rows per thread),
+//                           earlier inner panels applied left-looking; writes U / V
+//                           into At and the split-bf16 reflector block Y (both
+//                           orientations).
+//   2. tensor-core GEMM     [S; W^T] = [Y C]^T Y   (split over the m rows)
+//   3. wy_t_kernel          T = (striu(S) + diag(S)/2)^-1  so that H_1..H_128 = I - Y T Y^T
+//   4. wy_w2_kernel         W2^T = W^T T          (fp32, also reduces the split partials)
+//   5. tensor-core GEMM     C^T -= W2^T Y^T       (fp32 result + split-bf16 copy)
+// Exchanges inside the cluster are pushes into every CTA's shared memory followed
+// by one cluster barrier; all sums run in a fixed order (bit-reproducible).
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+#include "tc_path.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace dq {
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int IB = 32;     // inner panel width
+constexpr int OB = 128;    // outer block width
+constexpr int MAX_CS = 8;  // CTAs per cluster
+
+__device__ __forceinline__ void split2(float v, bf16& hi, bf16& lo) {
+  hi = __float2bfloat16_rn(v);
+  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+__device__ __forceinline__ uint32_t pack2(bf16 a, bf16 b) {
+  return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
+}
+
+// Store a float at the same shared-memory offset in CTA `rank` of this cluster.
+__device__ __forceinline__ void st_dsmem(float* local, int rank, float v) {
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(local);
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(addr), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+// Sum v[c] over the 32 lanes; lane c returns the total of entry c.
+__device__ __forceinline__ float warp_transpose_reduce32(float (&v)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool up = (lane & off) != 0;
+#pragma unroll
+    for (int k = 0; k < off; ++k) {
+      const float send = up ? v[k] : v[k + off];
+      const float keep = up ? v[k + off] : v[k];
+      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+  return v[0];
+}
+
+// At[c][r] = Z[r][c] (fp32) plus its split-bf16 copy; 32 x 32 tiles.
+__global__ void __launch_bounds__(256) transpose_split_kernel(const float* __restrict__ Z, float* __restrict__ At,
+                                                              bf16* __restrict__ hi, bf16* __restrict__ lo, int d) {
+  __shared__ float t[32][33];
+  const int64_t off = (int64_t)blockIdx.z * d * d;
+  Z += off; At += off; hi += off; lo += off;
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int r = ty; r < 32; r += 8) t[r][tx] = Z[(int64_t)(r0 + r) * d + c0 + tx];
+  __syncthreads();
+  for (int c = ty; c < 32; c += 8) {
+    const int64_t i = (int64_t)(c0 + c) * d + r0 + tx;
+    const float v = t[tx][c];
+    At[i] = v;
+    split2(v, hi[i], lo[i]);
+  }
+}
+
+// Shared-memory carve-up of the panel kernel (floats).
+template <int NW>
+struct PanelSmem {
+  static constexpr int RED = 0;                          // [NW][32] warp partials of a column step
+  static constexpr int XCH = RED + NW * 32;              // [2][MAX_CS][32] per-CTA partials (pushed)
+  static constexpr int DIAG = XCH + 2 * MAX_CS * 32;     // [2][32] the diagonal row (pushed)
+  static constexpr int DLOC = DIAG + 64;                 // [32] owner's staging of the diagonal row
+  static constexpr int COEF = DLOC + 32;                 // [NW][32]
+  static constexpr int ZS = COEF + NW * 32;              // [32][33] V^T v_j of the inner panel
+  static constexpr int TAU = ZS + 32 * 33;               // [32]
+  static constexpr int TS = TAU + 32;                    // [4][32][33] T of each inner panel
+  static constexpr int WP = TS + 4 * 32 * 33;            // [NW][32][32] per-warp partials of V_k^T P
+  static constexpr int WX = WP + NW * 1024;              // [MAX_CS][1024] per-CTA partials (pushed)
+  static constexpr int WF = WX + MAX_CS * 1024;          // [32][32] V_k^T P
+  static constexpr int W2 = WF + 1024;                   // [32][32] T_k^T V_k^T P
+  static constexpr int TOTAL = W2 + 1024;
+  static constexpr int BYTES = TOTAL * 4;
+};
+
+
+// Entries of eight consecutive reflectors (columns cp0.. of inner panel k, diagonal rows dg0..)
+// for this thread's two rows: stored value below the diagonal, 1 on it, 0 above.
+__device__ __forceinline__ void load_v8(float (&vv)[8][2], const float* Vk, int d, int dg0, int cp0,
+                                        const int (&rowi)[2], int m) {
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const float* vcol = Vk + (int64_t)(cp0 + u) * d;
+#pragma unroll
+    for (int s = 0; s < 2; ++s)
+      vv[u][s] = (rowi[s] > dg0 + u) ? ((rowi[s] < m) ? vcol[rowi[s]] : 0.f) : ((rowi[s] == dg0 + u) ? 1.f : 0.f);
+  }
+}
+
+struct PanelCtx {
+  float *red, *xch, *diag, *dloc, *coefs, *Zs, *taus;
+  int CS, cta, warp, lane, own_cta, own_warp, NW;
+};
+
+// One Householder column step.  R = register index of the current column (position 0);
+// position p lives in register (R + p) mod 32.  idg = row of the diagonal (relative to the
+// outer block), j = column index inside the inner panel.
+template <int R>
+__device__ __forceinline__ void col_step(float (&a)[2][32], const int (&rowi)[2], int idg, int j,
+                                         const PanelCtx& c) {
+  const int par = j & 1, lane = c.lane, warp = c.warp;
+  float acc[32];
+  {
+    const float x0 = (rowi[0] >= idg) ? a[0][R] : 0.f;
+    const float x1 = (rowi[1] >= idg) ? a[1][R] : 0.f;
+#pragma unroll
+    for (int p = 0; p < 32; ++p) acc[p] = fmaf(x1, a[1][(R + p) & 31], x0 * a[0][(R + p) & 31]);
+  }
+  const float tot = warp_transpose_reduce32(acc, lane);
+  c.red[warp * 32 + lane] = tot;
+  if (c.cta == c.own_cta && warp == c.own_warp && lane == j) {   // this thread holds the diagonal row
+#pragma unroll
+    for (int p = 0; p < 32; ++p) c.dloc[p] = a[0][(R + p) & 31];
+  }
+  __syncthreads();
+  if (warp == 0) {
+    float s = 0.f;
+    for (int w = 0; w < c.NW; ++w) s += c.red[w * 32 + lane];
+    if (c.CS > 1) {
+      for (int rk = 0; rk < c.CS; ++rk) st_dsmem(&c.xch[(par * MAX_CS + c.cta) * 32 + lane], rk, s);
+      if (c.cta == c.own_cta) {
+        const float dv = c.dloc[lane];
+        for (int rk = 0; rk < c.CS; ++rk) st_dsmem(&c.diag[par * 32 + lane], rk, dv);
+      }
+    } else {
+      c.xch[par * MAX_CS * 32 + lane] = s;
+      c.diag[par * 32 + lane] = c.dloc[lane];
+    }
+  }
+  if (c.CS > 1) cg::this_cluster().sync(); else __syncthreads();
+  float g = 0.f;
+  for (int rk = 0; rk < c.CS; ++rk) g += c.xch[(par * MAX_CS + rk) * 32 + lane];
+  const float dr = c.diag[par * 32 + lane];
+  const float alpha = __shfl_sync(0xffffffffu, dr, 0);
+  const float nrm2 = __shfl_sync(0xffffffffu, g, 0);
+  const float sigma = nrm2 - alpha * alpha;          // squared norm below the diagonal
+  const bool skip = !(sigma > 0.f);                  // nothing to annihilate: H_j = I
+  const float beta = skip ? alpha : -copysignf(__fsqrt_rn(nrm2), alpha);
+  const float denom = alpha - beta;
+  const float inv_denom = skip ? 0.f : __frcp_rn(denom);
+  const float tau = skip ? 0.f : -denom * __frcp_rn(beta);
+  const float w = fmaf(g - alpha * dr, inv_denom, dr);   // v_j^T (column at this position)
+  const int npos = 32 - j;                            // positions >= npos hold finished reflectors
+  c.coefs[warp * 32 + lane] = (lane >= 1 && lane < npos) ? tau * w : 0.f;
+  if (warp == 0) {
+    if (lane >= npos) c.Zs[(lane - npos) * 33 + j] = w;   // v_c^T v_j for c < j
+    if (lane == 0) c.taus[j] = tau;
+  }
+  __syncwarp();
+  const float4* cf = reinterpret_cast<const float4*>(c.coefs + warp * 32);
+#pragma unroll
+  for (int s = 0; s < 2; ++s) {
+    const bool on = rowi[s] == idg, below = rowi[s] > idg;
+    const float scaled = a[s][R] * inv_denom;
+    const float v = on ? 1.f : (below ? scaled : 0.f);
+    const float newc = on ? beta : (below ? scaled : a[s][R]);
+#pragma unroll
+    for (int q4 = 0; q4 < 8; ++q4) {
+      const float4 c4 = cf[q4];
+      a[s][(R + 4 * q4 + 0) & 31] = fmaf(-v, c4.x, a[s][(R + 4 * q4 + 0) & 31]);
+      a[s][(R + 4 * q4 + 1) & 31] = fmaf(-v, c4.y, a[s][(R + 4 * q4 + 1) & 31]);
+      a[s][(R + 4 * q4 + 2) & 31] = fmaf(-v, c4.z, a[s][(R + 4 * q4 + 2) & 31]);
+      a[s][(R + 4 * q4 + 3) & 31] = fmaf(-v, c4.w, a[s][(R + 4 * q4 + 3) & 31]);
+    }
+    a[s][R] = newc;   // the finished column stays put: it is position 31 of the next step
+  }
+  __syncwarp();   // coefs[warp] is rewritten in the next step
+}
+
+// Factor columns [c0, c0 + 128) of A (rows c0..d) held transposed in At.
+//   At   <- U on and above the diagonal, Householder vectors (unit diagonal implied) below
+//   yt   <- split-bf16 Y^T: rows c0..c0+127 of (at_hi, at_lo), entries r >= c0
+//   y    <- split-bf16 Y:   [d][128] row-major, rows r >= c0
+// Reflector j: H = I - tau v v^T, v = (x - beta e1) / (x_1 - beta), beta = -sign(x_1) ||x||
+// (Algorithm 2's sign rule), tau = (beta - x_1) / beta.
+template <int NT>
+__global__ void __launch_bounds__(NT, 1)
+qr_panel_cm_kernel(float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, int d, int c0) {
+  constexpr int NW = NT / 32;
+  using L = PanelSmem<NW>;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int CS = (int)cluster.num_blocks();
+  const int cta = (int)cluster.block_rank();
+  {
+    const int64_t dd = (int64_t)d * d, boff = (int64_t)blockIdx.y;
+    At += boff * dd; at_hi += boff * dd; at_lo += boff * dd;
+    y_hi += boff * (int64_t)d * OB; y_lo += boff * (int64_t)d * OB;
+  }
+  extern __shared__ float sm[];
+  float* red = sm + L::RED;
+  float* xch = sm + L::XCH;
+  float* diag = sm + L::DIAG;
+  float* dloc = sm + L::DLOC;
+  float* coefs = sm + L::COEF;
+  float* Zs = sm + L::ZS;
+  float* taus = sm + L::TAU;
+  float* Ts = sm + L::TS;
+  float* Wp = sm + L::WP;
+  float* wx = sm + L::WX;
+  float* Wf = sm + L::WF;
+  float* W2s = sm + L::W2;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int m = d - c0;
+  int rowi[2];
+#pragma unroll
+  for (int s = 0; s < 2; ++s) rowi[s] = ((s * NW + warp) * CS + cta) * 32 + lane;   // 32-row groups dealt round-robin
+  float a[2][32];
+
+#pragma unroll 1
+  for (int ip = 0; ip < OB / IB; ++ip) {
+    const int cb = c0 + ip * IB;
+    // ---- load the 32 columns of this inner panel (all rows c0..d)
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+#pragma unroll
+      for (int c = 0; c < 32; ++c)
+        a[s][c] = (rowi[s] < m) ? At[(int64_t)(cb + c) * d + c0 + rowi[s]] : 0.f;
+    }
+    // ---- left-looking: apply the block reflectors of the earlier inner panels
+#pragma unroll 1
+    for (int k = 0; k < ip; ++k) {
+      const float* Vk = At + (int64_t)(c0 + k * IB) * d + c0;
+#pragma unroll 1
+      for (int cp0 = 0; cp0 < 32; cp0 += 8) {
+        float vv[8][2];
+        load_v8(vv, Vk, d, k * IB + cp0, cp0, rowi, m);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          float acc[32];
+#pragma unroll
+          for (int p = 0; p < 32; ++p) acc[p] = fmaf(vv[u][1], a[1][p], vv[u][0] * a[0][p]);
+          const float t = warp_transpose_reduce32(acc, lane);
+          Wp[(warp * 32 + cp0 + u) * 32 + lane] = t;
+        }
+      }
+      __syncthreads();
+      for (int e = tid; e < 1024; e += NT) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) s += Wp[w * 1024 + e];
+        for (int rk = 0; rk < CS; ++rk) st_dsmem(&wx[cta * 1024 + e], rk, s);
+      }
+      cluster.sync();
+      for (int e = tid; e < 1024; e += NT) {
+        float s = 0.f;
+        for (int rk = 0; rk < CS; ++rk) s += wx[rk * 1024 + e];
+        Wf[e] = s;
+      }
+      cluster.sync();   // wx may be overwritten by the next exchange only after everyone has read it
+      const float* Tk = Ts + k * 32 * 33;
+      for (int e = tid; e < 1024; e += NT) {   // W2 = T_k^T (V_k^T P): apply Q^T
+        const int q = e >> 5, p = e & 31;
+        float s = 0.f;
+        for (int c = 0; c <= q; ++c) s = fmaf(Tk[c * 33 + q], Wf[c * 32 + p], s);
+        W2s[e] = s;
+      }
+      __syncthreads();
+#pragma unroll 1
+      for (int cp0 = 0; cp0 < 32; cp0 += 8) {
+        float vv[8][2];
+        load_v8(vv, Vk, d, k * IB + cp0, cp0, rowi, m);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float4* w2 = reinterpret_cast<const float4*>(W2s + (cp0 + u) * 32);
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4) {
+            const float4 w = w2[q4];
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+              a[s][4 * q4 + 0] = fmaf(-vv[u][s], w.x, a[s][4 * q4 + 0]);
+              a[s][4 * q4 + 1] = fmaf(-vv[u][s], w.y, a[s][4 * q4 + 1]);
+              a[s][4 * q4 + 2] = fmaf(-vv[u][s], w.z, a[s][4 * q4 + 2]);
+              a[s][4 * q4 + 3] = fmaf(-vv[u][s], w.w, a[s][4 * q4 + 3]);
+            }
+          }
+        }
+      }
+    }
+    // ---- factor the inner panel.  Position p of step j is column (j + p) mod 32; inside a group
+    // of four steps the rotation is a compile-time register offset, then the registers move by 4.
+    PanelCtx pc{red, xch, diag, dloc, coefs, Zs, taus, CS, cta, warp, lane, ip % CS, ip / CS, NW};
+#pragma unroll 1
+    for (int j4 = 0; j4 < 32; j4 += 4) {
+      col_step<0>(a, rowi, ip * IB + j4 + 0, j4 + 0, pc);
+      col_step<1>(a, rowi, ip * IB + j4 + 1, j4 + 1, pc);
+      col_step<2>(a, rowi, ip * IB + j4 + 2, j4 + 2, pc);
+      col_step<3>(a, rowi, ip * IB + j4 + 3, j4 + 3, pc);
+#pragma unroll
+      for (int s = 0; s < 2; ++s) {
+        const float t0 = a[s][0], t1 = a[s][1], t2 = a[s][2], t3 = a[s][3];
+#pragma unroll
+        for (int p = 0; p < 28; ++p) a[s][p] = a[s][p + 4];
+        a[s][28] = t0; a[s][29] = t1; a[s][30] = t2; a[s][31] = t3;
+      }
+    }
+    // ---- after 32 rotations the registers are back in natural order: column c at a[.][c]
+    __syncthreads();   // taus[] of the last step is visible to every warp
+    if (warp == 0) {
+      // T[0:j, j] = -tau_j T[0:j, 0:j] (V^T v_j), T[j][j] = tau_j; lane i keeps row i in registers
+      float* T = Ts + ip * 32 * 33;
+      float trow[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float tj = taus[j];
+        float s = 0.f;
+#pragma unroll
+        for (int c = 0; c < j; ++c) s = fmaf(trow[c], Zs[c * 33 + j], s);   // trow[c] = 0 for c < lane
+        trow[j] = (lane < j) ? -tj * s : ((lane == j) ? tj : 0.f);
+      }
+#pragma unroll
+      for (int j = 0; j < 32; ++j) T[lane * 33 + j] = trow[j];
+    }
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      const int i = rowi[s];
+      if (i < m) {
+        uint32_t ph[16], pl[16];
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          bf16 h0, l0, h1, l1;
+          const int dg0 = ip * IB + c, dg1 = dg0 + 1;
+          // a skipped reflector (tau = 0, H = I) contributes a zero column to Y
+          const float v0 = (i > dg0) ? a[s][c] : ((i == dg0 && taus[c] != 0.f) ? 1.f : 0.f);
+          const float v1 = (i > dg1) ? a[s][c + 1] : ((i == dg1 && taus[c + 1] != 0.f) ? 1.f : 0.f);
+          split2(v0, h0, l0);
+          split2(v1, h1, l1);
+          const int64_t t0 = (int64_t)(cb + c) * d + c0 + i, t1 = t0 + d;
+          At[t0] = a[s][c];
+          At[t1] = a[s][c + 1];
+          at_hi[t0] = h0; at_lo[t0] = l0;
+          at_hi[t1] = h1; at_lo[t1] = l1;
+          ph[c >> 1] = pack2(h0, h1);
+          pl[c >> 1] = pack2(l0, l1);
+        }
+        uint4* yh = reinterpret_cast<uint4*>(y_hi + (int64_t)(c0 + i) * OB + ip * IB);
+        uint4* yl = reinterpret_cast<uint4*>(y_lo + (int64_t)(c0 + i) * OB + ip * IB);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          yh[q] = make_uint4(ph[4 * q], ph[4 * q + 1], ph[4 * q + 2], ph[4 * q + 3]);
+          yl[q] = make_uint4(pl[4 * q], pl[4 * q + 1], pl[4 * q + 2], pl[4 * q + 3]);
+        }
+      }
+    }
+    __syncthreads();   // T of this inner panel is complete; At writes are ordered before re-reads
+  }
+  cluster.sync();   // no CTA may exit while others can still push into its shared memory
+}
+
+
+// ----------------------------------------------------------------------------- T of the outer block
+// Dense C[M x N] (+)= alpha A[M x K] B[K x N] on shared-memory matrices (leading dimensions lda, ldb,
+// ldc), 4 x 4 register tiles, 256 threads; M, N multiples of 4.
+__device__ __forceinline__ void smem_mm(const float* A, int lda, const float* B, int ldb, float* C, int ldc,
+                                        int M, int N, int K, float alpha, int tid) {
+  const int tn = N / 4, tiles = (M / 4) * tn;
+  for (int t = tid; t < tiles; t += 256) {
+    const int r0 = (t / tn) * 4, c0 = (t % tn) * 4;
+    float acc[4][4] = {};
+    for (int k = 0; k < K; ++k) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) av[i] = A[(r0 + i) * lda + k];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bv[j] = B[k * ldb + c0 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) C[(r0 + i) * ldc + c0 + j] = alpha * acc[i][j];
+  }
+}
+
+constexpr int TLD = 129;
+constexpr int WY_T_SMEM = (2 * 128 * TLD + 64 * 65) * 4;
+
+// S = sum of the split partials (rows 0..127 of part); T = (striu(S) + diag(S) / 2)^-1, the
+// compact-WY factor of the 128 reflectors (T^-1 + T^-T = Y^T Y).  A zero column of Y (skipped
+// reflector) decouples: its diagonal gets a placeholder.  One CTA per problem.
+__global__ void __launch_bounds__(256) wy_t_kernel(const float* __restrict__ part, int ksplit, int m,
+                                                   int64_t part_batch_stride, float* __restrict__ T) {
+  extern __shared__ float sm[];
+  float* U = sm;                    // [128][TLD]  T^-1 (upper triangular)
+  float* X = sm + 128 * TLD;        // [128][TLD]  its inverse
+  float* Tmp = X + 128 * TLD;       // [64][65]
+  part += (int64_t)blockIdx.y * part_batch_stride;
+  T += (int64_t)blockIdx.y * 128 * 128;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#pragma unroll 4
+  for (int it = 0; it < 16; ++it) {   // independent 16-byte loads: the partials sit in L2 / HBM
+    const int e = (it * 256 + tid) * 4;
+    const int r = e >> 7, c0 = e & 127;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c0 + 3 >= r)
+      for (int sp = 0; sp < ksplit; ++sp) {
+        const float4 t = *reinterpret_cast<const float4*>(part + (int64_t)sp * m * 128 + e);
+        s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+      }
+    const float sv[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int c = c0 + q;
+      float v = (c > r) ? sv[q] : ((c == r) ? 0.5f * sv[q] : 0.f);
+      if (c == r && !(v > 0.f)) v = 1.f;
+      U[r * TLD + c] = v;
+      X[r * TLD + c] = 0.f;
+    }
+  }
+  __syncthreads();
+  if (warp < 4) {   // inverse of the four 32 x 32 diagonal blocks: lane j solves U x = e_j
+    const int o = warp * 32, j = lane;
+    X[(o + j) * TLD + o + j] = 1.f / U[(o + j) * TLD + o + j];
+    for (int i = j - 1; i >= 0; --i) {
+      float s = 0.f;
+      for (int k = i + 1; k <= j; ++k) s = fmaf(U[(o + i) * TLD + o + k], X[(o + k) * TLD + o + j], s);
+      X[(o + i) * TLD + o + j] = -s / U[(o + i) * TLD + o + i];
+    }
+  }
+  __syncthreads();
+  // inv([A B; 0 C]) = [A^-1, -A^-1 B C^-1; 0, C^-1]: 32-blocks -> 64-blocks -> 128
+  for (int pair = 0; pair < 2; ++pair) {
+    const int o = pair * 64;
+    smem_mm(U + o * TLD + o + 32, TLD, X + (o + 32) * TLD + o + 32, TLD, Tmp, 65, 32, 32, 32, 1.f, tid);
+    __syncthreads();
+    smem_mm(X + o * TLD + o, TLD, Tmp, 65, X + o * TLD + o + 32, TLD, 32, 32, 32, -1.f, tid);
+    __syncthreads();
+  }
+  smem_mm(U + 64, TLD, X + 64 * TLD + 64, TLD, Tmp, 65, 64, 64, 64, 1.f, tid);
+  __syncthreads();
+  smem_mm(X, TLD, Tmp, 65, X + 64, TLD, 64, 64, 64, -1.f, tid);
+  __syncthreads();
+  for (int e = tid; e < 128 * 128; e += 256) {
+    const int r = e >> 7, c = e & 127;
+    T[e] = (c >= r) ? X[r * TLD + c] : 0.f;
+  }
+}
+
+// W2^T[row][j] = sum_k W^T[row][k] T[k][j] with W^T = sum of the split partials (rows 128.. of
+// part); written as a split-bf16 pair [n][128].  64 rows per CTA, 4 x 8 outputs per thread.
+constexpr int WY_W2_SMEM = (128 * 128 + 64 * TLD) * 4;
+__global__ void __launch_bounds__(256) wy_w2_kernel(const float* __restrict__ part, int ksplit, int m,
+                                                    int64_t part_batch_stride, const float* __restrict__ T,
+                                                    bf16* __restrict__ w2_hi, bf16* __restrict__ w2_lo,
+                                                    int64_t w2_batch_stride) {
+  extern __shared__ float sm[];
+  float* Ts = sm;                 // [128][128]
+  float* Ws = sm + 128 * 128;     // [64][TLD]
+  part += (int64_t)blockIdx.y * part_batch_stride;
+  T += (int64_t)blockIdx.y * 128 * 128;
+  w2_hi += (int64_t)blockIdx.y * w2_batch_stride;
+  w2_lo += (int64_t)blockIdx.y * w2_batch_stride;
+  const int tid = threadIdx.x;
+  const int row0 = blockIdx.x * 64;
+  for (int e = tid; e < 128 * 128 / 4; e += 256)
+    reinterpret_cast<float4*>(Ts)[e] = reinterpret_cast<const float4*>(T)[e];
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {    // independent 16-byte loads
+    const int e = (it * 256 + tid) * 4;
+    const int r = e >> 7, k = e & 127;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int sp = 0; sp < ksplit; ++sp) {
+      const float4 t = *reinterpret_cast<const float4*>(part + ((int64_t)sp * m + 128 + row0 + r) * 128 + k);
+      s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+    }
+    Ws[r * TLD + k] = s.x; Ws[r * TLD + k + 1] = s.y; Ws[r * TLD + k + 2] = s.z; Ws[r * TLD + k + 3] = s.w;
+  }
+  __syncthreads();
+  const int r0 = (tid >> 4) * 4, c0 = (tid & 15) * 8;
+  float acc[4][8] = {};
+  for (int k = 0; k < c0 + 8; ++k) {   // T is upper triangular: T[k][j] = 0 for k > j
+    float wv[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) wv[i] = Ws[(r0 + i) * TLD + k];
+    const float4 t0 = *reinterpret_cast<const float4*>(Ts + k * 128 + c0);
+    const float4 t1 = *reinterpret_cast<const float4*>(Ts + k * 128 + c0 + 4);
+    const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(wv[i], tv[j], acc[i][j]);
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t ph[4], pl[4];
+#pragma unroll
+    for (int j = 0; j < 8; j += 2) {
+      bf16 h0, l0, h1, l1;
+      split2(acc[i][j], h0, l0);
+      split2(acc[i][j + 1], h1, l1);
+      ph[j >> 1] = pack2(h0, h1);
+      pl[j >> 1] = pack2(l0, l1);
+    }
+    const int64_t o = (int64_t)(row0 + r0 + i) * 128 + c0;
+    *reinterpret_cast<uint4*>(w2_hi + o) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+    *reinterpret_cast<uint4*>(w2_lo + o) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+  }
+}
+
+// Gauge of the raw factor held transposed: U[i][j] = s_i At[j][i] for j >= i, s_i = sign(At[i][i])
+// (+1 at 0); fp32 + split copy.
+__global__ void __launch_bounds__(256) gauge_ut_kernel(const float* __restrict__ At, float* __restrict__ U,
+                                                       bf16* __restrict__ hi, bf16* __restrict__ lo, int d) {
+  __shared__ float t[32][33];
+  const int64_t off = (int64_t)blockIdx.z * d * d;
+  At += off; U += off; hi += off; lo += off;
+  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  if (j0 >= i0)
+    for (int r = ty; r < 32; r += 8) t[r][tx] = At[(int64_t)(j0 + r) * d + i0 + tx];   // At[j][i]
+  __syncthreads();
+  for (int r = ty; r < 32; r += 8) {
+    const int i = i0 + r, j = j0 + tx;
+    const float si = (At[(int64_t)i * d + i] < 0.f) ? -1.f : 1.f;
+    const float v = (j >= i) ? si * t[tx][r] : 0.f;
+    const int64_t idx = (int64_t)i * d + j;
+    U[idx] = v;
+    split2(v, hi[idx], lo[idx]);
+  }
+}
+
+template <int NT>
+dq_status launch_panel(Ctx& ctx, int cs, int batch, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo,
+                       int d, int c0) {
+  using L = PanelSmem<NT / 32>;
+  static bool attr = false;
+  auto kern = qr_panel_cm_kernel<NT>;
+  if (!attr) {
+    DQ_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES));
+    attr = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(cs, batch, 1);
+  cfg.blockDim = dim3(NT, 1, 1);
+  cfg.dynamicSmemBytes = L::BYTES;
+  cfg.stream = ctx.stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  DQ_CHECK_CUDA(cudaLaunchKernelEx(&cfg, kern, At, at_hi, at_lo, y_hi, y_lo, d, c0));
+  return after_launch(ctx);
+}
+
+}  // namespace
+
+dq_status qrp_transpose_split(Ctx& ctx, const float* Z, float* At, bf16* hi, bf16* lo, int d, int batch) {
+  transpose_split_kernel<<<dim3(d / 32, d / 32, batch), 256, 0, ctx.stream>>>(Z, At, hi, lo, d);
+  return after_launch(ctx);
+}
+
+dq_status qrp_panel(Ctx& ctx, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, int d, int c0,
+                    int batch) {
+  const int m = d - c0;
+  if (m <= 0 || m % OB != 0 || m > 8192) return DQ_ERR_UNSUPPORTED;
+  const bool wide = m > 4096;                       // 1024 rows per CTA instead of 512
+  const int rows_per_cta = wide ? 1024 : 512;
+  int cs = 1;
+  while (cs * rows_per_cta < m) cs *= 2;
+  if (cs > MAX_CS) return DQ_ERR_UNSUPPORTED;
+  return wide ? launch_panel<512>(ctx, cs, batch, At, at_hi, at_lo, y_hi, y_lo, d, c0)
+              : launch_panel<256>(ctx, cs, batch, At, at_hi, at_lo, y_hi, y_lo, d, c0);
+}
+
+dq_status qrp_wy_t(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, float* T, int batch) {
+  static bool attr = false;
+  if (!attr) {
+    DQ_CHECK_CUDA(cudaFuncSetAttribute(wy_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WY_T_SMEM));
+    attr = true;
+  }
+  wy_t_kernel<<<dim3(1, batch), 256, WY_T_SMEM, ctx.stream>>>(part, ksplit, m, part_bs, T);
+  return after_launch(ctx);
+}
+
+dq_status qrp_wy_w2(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, const float* T, bf16* w2_hi,
+                    bf16* w2_lo, int64_t w2_bs, int n, int batch) {
+  static bool attr = false;
+  if (!attr) {
+    DQ_CHECK_CUDA(cudaFuncSetAttribute(wy_w2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WY_W2_SMEM));
+    attr = true;
+  }
+  wy_w2_kernel<<<dim3(n / 64, batch), 256, WY_W2_SMEM, ctx.stream>>>(part, ksplit, m, part_bs, T, w2_hi, w2_lo, w2_bs);
+  return after_launch(ctx);
+}
+
+dq_status qrp_gauge_ut(Ctx& ctx, const float* At, float* U, bf16* hi, bf16* lo, int d, int batch) {
+  gauge_ut_kernel<<<dim3(d / 32, d / 32, batch), 256, 0, ctx.stream>>>(At, U, hi, lo, d);
+  return after_launch(ctx);
+}
+
+}  // namespace dq

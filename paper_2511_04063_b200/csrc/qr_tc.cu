@@ -127,31 +127,9 @@ __global__ void __launch_bounds__(DB) tri_inv_diag128_kernel(const float* __rest
   }
 }
 
-struct Op {   // K-major operand: rows x K, split pair, leading dimension, batch stride (elements)
-  const bf16* hi; const bf16* lo; int64_t ld; int64_t bs;
-};
-struct Out {
-  float* f32 = nullptr; int64_t ld = 0; int64_t bs = 0;
-  bf16* hi = nullptr; bf16* lo = nullptr; int64_t ld_h = 0; int64_t bs_h = 0;
-  float alpha = 1.f, beta = 0.f;
-};
-
-// D[m][n] = alpha sum_k A[m][k] B[n][k] (+ beta D) with split-bf16 operands; M, N % 128 == 0, K % 64 == 0.
-dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, int batch, const Out& o) {
-  if (M % 128 || N % 128 || K % 64) return DQ_ERR_UNSUPPORTED;
-  CUtensorMap ma, mal, mb, mbl;
-  const int64_t bsa = A.bs ? A.bs : (int64_t)M * A.ld, bsb = B.bs ? B.bs : (int64_t)N * B.ld;
-  DQ_CHECK(tch::make_map(&ma, A.hi, K, M, batch, A.ld, bsa, tc::BLOCK_M));
-  DQ_CHECK(tch::make_map(&mal, A.lo, K, M, batch, A.ld, bsa, tc::BLOCK_M));
-  DQ_CHECK(tch::make_map(&mb, B.hi, K, N, batch, B.ld, bsb, 128));
-  DQ_CHECK(tch::make_map(&mbl, B.lo, K, N, batch, B.ld, bsb, 128));
-  tc::Params p{};
-  p.m_blocks = M / 128; p.n_blocks = N / 128; p.batch = batch; p.ksplit = 1; p.k_blocks = K / tc::BLOCK_K;
-  p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = 0;
-  p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
-  p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
-  return tch::launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
-}
+using tch::Op;
+using tch::Out;
+using tch::gemm3;
 
 // Block column of the inverse:  W[0:k, k:k+s] = -W[0:k,0:k] U[0:k, k:k+s] W[k:k+s, k:k+s]
 // for `count` independent diagonal positions `stride` elements apart (3rd tensor dimension).
@@ -207,13 +185,32 @@ dq_status alloc(T** p, int64_t n) {
   return cudaMalloc((void**)p, sizeof(T) * (size_t)n) == cudaSuccess ? DQ_OK : DQ_ERR_ALLOC;
 }
 
+// Split-K factor of the [S; W^T] product of an outer block with m active rows: fill the SMs,
+// keep at least two 64-row k-blocks per slice.
+int wy_ksplit(int m, int batch, int sm_count) {
+  const int tiles = (m / 128) * batch;
+  int ks = sm_count / tiles;
+  if (ks > m / 128) ks = m / 128;
+  return ks < 1 ? 1 : ks;
+}
+
 }  // namespace
 
-dq_status qr_tc_init(QrTcState& q, int d, int batch) {
+dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   const int64_t dd = (int64_t)d * d * batch;
   bf16** all[] = {&q.z_hi, &q.z_lo, &q.u_hi, &q.u_lo, &q.wn_hi, &q.wn_lo, &q.wt_hi, &q.wt_lo, &q.r_hi, &q.r_lo,
                   &q.rt_hi, &q.rt_lo, &q.gqt_hi, &q.gqt_lo, &q.st_hi, &q.st_lo, &q.m_hi, &q.m_lo, &q.t1_hi, &q.t1_lo};
   for (bf16** p : all) DQ_CHECK(alloc(p, dd));
+  const int64_t yb = (int64_t)d * 128 * batch;
+  DQ_CHECK(alloc(&q.y_hi, yb)); DQ_CHECK(alloc(&q.y_lo, yb));
+  DQ_CHECK(alloc(&q.w2_hi, yb)); DQ_CHECK(alloc(&q.w2_lo, yb));
+  DQ_CHECK(alloc(&q.T, (int64_t)128 * 128 * batch));
+  q.part_bs = 0;
+  for (int m = d; m > 128; m -= 128) {
+    const int64_t e = (int64_t)wy_ksplit(m, batch, sm_count) * m * 128;
+    if (e > q.part_bs) q.part_bs = e;
+  }
+  if (q.part_bs > 0) DQ_CHECK(alloc(&q.part, q.part_bs * batch));
   q.ready = true;
   return DQ_OK;
 }
@@ -222,7 +219,38 @@ void qr_tc_destroy(QrTcState& q) {
   bf16* all[] = {q.z_hi, q.z_lo, q.u_hi, q.u_lo, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, q.r_hi, q.r_lo,
                  q.rt_hi, q.rt_lo, q.gqt_hi, q.gqt_lo, q.st_hi, q.st_lo, q.m_hi, q.m_lo, q.t1_hi, q.t1_lo};
   for (bf16* p : all) cudaFree(p);
+  cudaFree(q.y_hi); cudaFree(q.y_lo); cudaFree(q.w2_hi); cudaFree(q.w2_lo); cudaFree(q.part); cudaFree(q.T);
   q = QrTcState();
+}
+
+// Blocked Householder factorisation of Z on the transposed working matrix ws.A (= A^T): 128-column
+// outer blocks, panel on the CUDA cores, compact-WY trailing update as split-bf16 tensor-core GEMMs.
+// On return ws.A holds U^T on / below its diagonal (raw signs of Algorithm 2).
+dq_status qr_factor_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, int d, int batch) {
+  const int64_t dd = (int64_t)d * d, yb = (int64_t)d * 128;
+  float* At = ws.A;
+  bf16 *at_hi = q.st_hi, *at_lo = q.st_lo;   // free until the backward pass
+  DQ_CHECK(qrp_transpose_split(ctx, Z, At, at_hi, at_lo, d, batch));
+  for (int c0 = 0; c0 < d; c0 += 128) {
+    const int m = d - c0, n = m - 128;
+    DQ_CHECK(qrp_panel(ctx, At, at_hi, at_lo, q.y_hi, q.y_lo, d, c0, batch));
+    if (n == 0) break;
+    const int64_t o = (int64_t)c0 * d + c0;
+    // [S; W^T][i][j] = sum_r At[c0 + i][r] Y^T[j][r], r in [c0, d): rows 0..127 are Y^T Y, the rest W^T
+    const int ks = wy_ksplit(m, batch, ctx.sm_count);
+    Op a{at_hi + o, at_lo + o, d, dd}, b{at_hi + o, at_lo + o, d, dd};
+    Out sw; sw.f32 = q.part; sw.ld = 128; sw.bs = q.part_bs; sw.ksplit = ks; sw.split_stride = (int64_t)m * 128;
+    DQ_CHECK(gemm3(ctx, a, b, m, 128, m, batch, sw));
+    DQ_CHECK(qrp_wy_t(ctx, q.part, ks, m, q.part_bs, q.T, batch));
+    DQ_CHECK(qrp_wy_w2(ctx, q.part, ks, m, q.part_bs, q.T, q.w2_hi, q.w2_lo, yb, n, batch));
+    // C^T[c][r] -= sum_j W2^T[c][j] Y[r][j]
+    Op w2{q.w2_hi, q.w2_lo, 128, yb}, y{q.y_hi + (int64_t)c0 * 128, q.y_lo + (int64_t)c0 * 128, 128, yb};
+    const int64_t oc = o + (int64_t)128 * d;
+    Out up; up.f32 = At + oc; up.ld = d; up.bs = dd; up.hi = at_hi + oc; up.lo = at_lo + oc; up.ld_h = d; up.bs_h = dd;
+    up.alpha = -1.f; up.beta = 1.f;
+    DQ_CHECK(gemm3(ctx, w2, y, n, m, 128, batch, up));
+  }
+  return qr_diag_check(ctx, At, d, batch);
 }
 
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
@@ -230,9 +258,8 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
   if (d % 128 != 0) return DQ_ERR_UNSUPPORTED;
   const int64_t dd = (int64_t)d * d;
   const dim3 tiles(d / 32, d / 32, batch);
-  DQ_CHECK(qr_factor(ctx, ws, Z, d, batch));
-  gauge_u_kernel<<<tiles, 256, 0, ctx.stream>>>(ws.A, U, q.u_hi, q.u_lo, d);
-  DQ_CHECK(after_launch(ctx));
+  DQ_CHECK(qr_factor_tc(ctx, ws, q, Z, d, batch));
+  DQ_CHECK(qrp_gauge_ut(ctx, ws.A, U, q.u_hi, q.u_lo, d, batch));
   DQ_CHECK(tri_inverse_tc(ctx, q, U, d, batch));
   split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
   DQ_CHECK(after_launch(ctx));

@@ -202,7 +202,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 
   const int tiles_per_batch = p.m_blocks * p.n_blocks;
   const int units = tiles_per_batch * p.batch * p.ksplit;
-  const int kb_per_split = p.k_blocks / p.ksplit;
+  // split s of the reduction covers k-blocks [s * k_blocks / ksplit, (s + 1) * k_blocks / ksplit)
+  auto split_begin = [&](int s) { return (int)(((int64_t)s * p.k_blocks) / p.ksplit); };
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
@@ -216,7 +217,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         const int b = t / tiles_per_batch;
         const int r = t % tiles_per_batch;
         const int mb = r % p.m_blocks, nb = r / p.m_blocks;   // m fastest: neighbours share the B tile
-        const int k0 = split * kb_per_split;
+        const int k0 = split_begin(split);
+        const int kb_per_split = split_begin(split + 1) - k0;
         for (int kb = 0; kb < kb_per_split; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), L::STAGE_BYTES);
@@ -245,6 +247,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BLOCK_N);
+        const int split = u % p.ksplit;
+        const int kb_per_split = split_begin(split + 1) - split_begin(split);
         for (int kb = 0; kb < kb_per_split; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, p.d_status)) { ok = false; break; }
           tc_fence_after();

@@ -57,5 +57,37 @@ dq_status launch_gemm(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, cons
   return after_launch(ctx);
 }
 
+using bf16 = __nv_bfloat16;
+
+struct Op {   // K-major operand: rows x K, split pair, leading dimension, batch stride (elements)
+  const bf16* hi; const bf16* lo; int64_t ld; int64_t bs;
+};
+struct Out {
+  float* f32 = nullptr; int64_t ld = 0; int64_t bs = 0;
+  bf16* hi = nullptr; bf16* lo = nullptr; int64_t ld_h = 0; int64_t bs_h = 0;
+  float alpha = 1.f, beta = 0.f;
+  // split-K: slice s of the reduction writes alpha * partial product (beta must be 0, no
+  // split copy) to f32 + s * split_stride; the caller reduces.
+  int ksplit = 1; int64_t split_stride = 0;
+};
+
+// D[m][n] = alpha sum_k A[m][k] B[n][k] (+ beta D) with split-bf16 operands (three bf16 MMAs per
+// product, fp32 accumulation); M, N % 128 == 0, K % 64 == 0.
+inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, int batch, const Out& o) {
+  if (M % 128 || N % 128 || K % 64 || o.ksplit < 1 || o.ksplit > K / 64) return DQ_ERR_UNSUPPORTED;
+  CUtensorMap ma, mal, mb, mbl;
+  const int64_t bsa = A.bs ? A.bs : (int64_t)M * A.ld, bsb = B.bs ? B.bs : (int64_t)N * B.ld;
+  DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, tc::BLOCK_M));
+  DQ_CHECK(make_map(&mal, A.lo, K, M, batch, A.ld, bsa, tc::BLOCK_M));
+  DQ_CHECK(make_map(&mb, B.hi, K, N, batch, B.ld, bsb, 128));
+  DQ_CHECK(make_map(&mbl, B.lo, K, N, batch, B.ld, bsb, 128));
+  tc::Params p{};
+  p.m_blocks = M / 128; p.n_blocks = N / 128; p.batch = batch; p.ksplit = o.ksplit; p.k_blocks = K / tc::BLOCK_K;
+  p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = o.split_stride;
+  p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
+  p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
+  return launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
+}
+
 }  // namespace tch
 }  // namespace dq

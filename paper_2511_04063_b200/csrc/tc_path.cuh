@@ -43,11 +43,31 @@ struct QrTcState {
   __nv_bfloat16 *st_hi = nullptr, *st_lo = nullptr;     // S^T
   __nv_bfloat16 *m_hi = nullptr, *m_lo = nullptr;       // R S
   __nv_bfloat16 *t1_hi = nullptr, *t1_lo = nullptr;     // scratch of the block inversion
+  // blocked Householder factorisation with tensor-core trailing updates
+  __nv_bfloat16 *y_hi = nullptr, *y_lo = nullptr;       // [batch][d][128] reflector block Y of the outer block
+  __nv_bfloat16 *w2_hi = nullptr, *w2_lo = nullptr;     // [batch][d][128] (T^T Y^T C)^T
+  float* part = nullptr;                                // split partials of [S; W^T]
+  int64_t part_bs = 0;                                  // elements per problem
+  float* T = nullptr;                                   // [batch][128][128] compact-WY factor
 };
-dq_status qr_tc_init(QrTcState& q, int d, int batch);
+dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count);
 void qr_tc_destroy(QrTcState& q);
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
                           int batch);
 dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch);
+
+
+// Kernels of the blocked Householder factorisation on a transposed working matrix
+// (qr_panel_tc.cu); the tensor-core products between them are issued by qr_tc.cu.
+dq_status qrp_transpose_split(Ctx& ctx, const float* Z, float* At, __nv_bfloat16* hi, __nv_bfloat16* lo, int d,
+                              int batch);
+dq_status qrp_panel(Ctx& ctx, float* At, __nv_bfloat16* at_hi, __nv_bfloat16* at_lo, __nv_bfloat16* y_hi,
+                    __nv_bfloat16* y_lo, int d, int c0, int batch);
+dq_status qrp_wy_t(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, float* T, int batch);
+dq_status qrp_wy_w2(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, const float* T,
+                    __nv_bfloat16* w2_hi, __nv_bfloat16* w2_lo, int64_t w2_bs, int n, int batch);
+dq_status qrp_gauge_ut(Ctx& ctx, const float* At, float* U, __nv_bfloat16* hi, __nv_bfloat16* lo, int d, int batch);
+// Rank / finiteness test of diag(U) (qr_forward.cu); works on either orientation.
+dq_status qr_diag_check(Ctx& ctx, const float* A, int d, int batch);
 
 }  // namespace dq

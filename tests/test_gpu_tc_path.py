@@ -72,6 +72,37 @@ def test_tensor_core_step_every_stage(w):
     c.close()
 
 
+@pytest.mark.parametrize("d,batch,kind", [(128, 2, "noisy"), (256, 1, "noisy"), (640, 1, "noisy"), (1024, 1, "noisy"),
+                                          (1152, 1, "hadamard_like"), (256, 1, "identity"), (384, 2, "upper")])
+def test_tensor_core_qr_forward_matches_unique_factorisation(d, batch, kind):
+    """Blocked Householder with tensor-core trailing updates (outer blocks of 128, inner panels of
+    32) against the library QR in float64: several outer blocks, a ragged cluster, skipped
+    reflectors (identity / upper-triangular latents have nothing to annihilate)."""
+    w = small("c2_7b", d=d, n_tokens=256, batch=batch, n_outlier_channels=1)
+    rng = np.random.default_rng(d + batch)
+    Z0 = np.empty((batch, d, d), dtype=np.float32)
+    for b in range(batch):
+        if kind == "identity":
+            Z0[b] = np.eye(d)
+        elif kind == "upper":
+            Z0[b] = np.triu(rng.standard_normal((d, d)) * 0.05) + np.diag(1.0 + rng.random(d))
+        else:
+            Q, _ = np.linalg.qr(rng.standard_normal((d, d)))
+            amp = 0.02 if kind == "noisy" else 0.0
+            Z0[b] = Q + amp * rng.standard_normal((d, d)) / np.sqrt(d) * np.sqrt(d) * 0.05
+    c = Calib(w, Z0=Z0)
+    R = c.rotation()
+    assert c.status() == dq.DQ_OK
+    U = c.buf(dq.DQ_BUF_U).cpu().numpy().astype(np.float64)
+    for b in range(batch):
+        Rr, Ur = orc.qr_pos_lapack(Z0[b])
+        assert np.abs(U[b] - Ur).max() <= 2e-5 * max(1.0, np.abs(Ur).max())
+        assert np.abs(np.tril(U[b], -1)).max() == 0.0 and (np.diag(U[b]) > 0).all()
+        assert np.abs(R[b] - Rr).max() <= 5e-5
+        assert np.abs(R[b].T @ R[b] - np.eye(d)).max() <= 5e-5
+    c.close()
+
+
 def test_tensor_core_path_is_bit_reproducible():
     w = small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3)
     outs = []
