@@ -84,6 +84,25 @@ dq_status dq_calib_get_rotation(dq_calib_t* h, float* d_R_out);
 dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d, int64_t ldx,
                           const float* d_R, void* d_Y, int64_t ldy, void* cuda_stream);
 
+/* (No counterpart in the paper: a packaging variant of dq_rotate_apply for bf16 activations.)
+ * The same Y = X R, for callers that must not allocate device memory: a serving process that
+ * handed all of HBM to its own arena at start-up (a later cudaMalloc would fail or fragment
+ * it), or a latency-critical loop where the implicit device synchronisation of cudaFree is
+ * not acceptable.  dq_rotate_apply allocates and frees a bf16 copy of R^T on every call; this
+ * variant keeps that copy in a fixed device array inside the library (8 MiB, held by every GPU
+ * that loads the library until the process exits) and calls no cudaMalloc / cudaFree or any
+ * other allocating routine.
+ *   - X, Y: bf16 [n][ldx] / [n][ldy]; R: fp32 [d][d]; all device, caller-owned, no aliasing.
+ *   - d <= 2048 (the size of the fixed array), d % 128 == 0, n % 128 == 0, ldx % 8 == ldy % 8 == 0;
+ *     anything else returns DQ_ERR_UNSUPPORTED and launches nothing.
+ *   - The first call on each device also looks up the array's device address; make that call
+ *     once, with that device current, before any stream capture.
+ *   - All calls share the one array.  Each call rewrites the part it uses before reading it, so
+ *     calls on one stream are independent; calls that overlap on the GPU (different streams or
+ *     threads without ordering between them) race on it and must be serialised by the caller. */
+dq_status dq_rotate_apply_static(const void* d_X, int64_t n, int32_t d, int64_t ldx, const float* d_R,
+                                 void* d_Y, int64_t ldy, void* cuda_stream);
+
 /* Mini-batch use (the paper feeds the loop with batches of sampled tokens): the
  * caller overwrote the borrowed activation buffer d_X in place (same shape) on
  * the handle's stream; rebuild every operand copy derived from it.  Cheap no-op on

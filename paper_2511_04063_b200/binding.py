@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_init", "dq_calib_step", "dq_calib_get_rotation", "dq_rotate_apply",
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
-    "dq_calib_destroy", "dq_version",
+    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static",
 )
 
 
@@ -58,6 +58,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_step.argtypes = [vp, i32, vp]
     lib.dq_calib_get_rotation.argtypes = [vp, vp]
     lib.dq_rotate_apply.argtypes = [vp, i32, i64, i32, i64, vp, vp, i64, vp]
+    lib.dq_rotate_apply_static.argtypes = [vp, i64, i32, i64, vp, vp, i64, vp]
+    lib.dq_rotate_apply_static.restype = i32
     lib.dq_calib_get_latent.argtypes = [vp, vp]
     lib.dq_calib_set_latent.argtypes = [vp, vp]
     lib.dq_calib_status.argtypes = [vp]
@@ -193,6 +195,17 @@ def dq_rotate_apply(X, R, Y, stream=None):
     _check(load_library().dq_rotate_apply(_ptr(X), DQ_FP32 if X.dtype == torch.float32 else DQ_BF16, n, d,
                                           X.stride(0), _ptr(R), _ptr(Y), Y.stride(0), _stream_ptr(stream)),
            "dq_rotate_apply")
+
+
+def dq_rotate_apply_static(X, R, Y, stream=None):
+    """Y = X R for bfloat16 X, Y ([n, d]) and float32 R ([d, d]) without any device allocation:
+    for callers whose memory is all spoken for (see include/dartquant.h).  d <= 2048."""
+    import torch
+    assert X.is_cuda and R.is_cuda and Y.is_cuda and R.dtype == torch.float32
+    assert X.dtype == torch.bfloat16 and Y.dtype == torch.bfloat16
+    n, d = X.shape
+    _check(load_library().dq_rotate_apply_static(_ptr(X), n, d, X.stride(0), _ptr(R), _ptr(Y), Y.stride(0),
+                                                 _stream_ptr(stream)), "dq_rotate_apply_static")
 
 
 def dq_version() -> str:

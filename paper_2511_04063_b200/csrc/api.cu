@@ -417,4 +417,12 @@ dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d
   return DQ_ERR_INVALID_ARG;
 }
 
+dq_status dq_rotate_apply_static(const void* d_X, int64_t n, int32_t d, int64_t ldx, const float* d_R,
+                                 void* d_Y, int64_t ldy, void* cuda_stream) {
+  if (!d_X || !d_R || !d_Y || n <= 0 || d <= 0 || ldx < d || ldy < d) return DQ_ERR_INVALID_ARG;
+  Ctx ctx;
+  ctx.stream = (cudaStream_t)cuda_stream;
+  return tc_rotate_apply_static(ctx, d_X, n, d, ldx, d_R, d_Y, ldy);
+}
+
 }  // extern "C"

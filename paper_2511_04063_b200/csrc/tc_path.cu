@@ -153,4 +153,57 @@ dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t l
   return st;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Y = X R without any allocation (dq_rotate_apply_static).
+//
+// The only scratch the bf16 rotation needs is the bf16 copy of R^T that feeds the tensor cores.
+// Here it lives in a file-scope device array, so the call never touches the CUDA allocator.
+// Every device that loads the library carries the array (8 MiB) until the process exits.
+// ---------------------------------------------------------------------------------------------
+constexpr int STATIC_MAX_D = 2048;
+static __device__ __align__(256) __nv_bfloat16 g_static_rt[(size_t)STATIC_MAX_D * STATIC_MAX_D];
+
+namespace {
+constexpr int STATIC_MAX_DEVICES = 64;
+__nv_bfloat16* g_static_rt_ptr[STATIC_MAX_DEVICES] = {};   // device address of g_static_rt, per device
+int g_static_sms[STATIC_MAX_DEVICES] = {};
+}  // namespace
+
+dq_status tc_rotate_apply_static(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t ldx, const float* d_R,
+                                 void* d_Y, int64_t ldy) {
+  if (d > STATIC_MAX_D) return DQ_ERR_UNSUPPORTED;
+  if (d % 128 != 0 || n % 128 != 0 || ldx % 8 != 0 || ldy % 8 != 0) return DQ_ERR_UNSUPPORTED;
+  int dev = 0;
+  DQ_CHECK_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= STATIC_MAX_DEVICES) return DQ_ERR_UNSUPPORTED;
+  if (!g_static_rt_ptr[dev]) {
+    // First call on this device: in host code the array's name is only a handle; the kernels need
+    // its device address.
+    int cc_major = 0;
+    DQ_CHECK_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (cc_major != 10) return DQ_ERR_UNSUPPORTED;
+    DQ_CHECK_CUDA(cudaDeviceGetAttribute(&g_static_sms[dev], cudaDevAttrMultiProcessorCount, dev));
+    __nv_bfloat16* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_static_rt) != cudaSuccess || !p) return DQ_ERR_CUDA;
+    g_static_rt_ptr[dev] = p;
+  }
+  ctx.sm_count = g_static_sms[dev];
+  __nv_bfloat16* rt = g_static_rt_ptr[dev];
+  // Every element of rt[0 : d*d) is overwritten, so nothing of an earlier call survives.
+  transpose_f32_to_bf16_kernel<<<dim3(d / 32, d / 32, 1), 256, 0, ctx.stream>>>(d_R, rt, d);
+  DQ_CHECK(after_launch(ctx));
+  const int bn = (d % 256 == 0) ? 256 : 128;
+  CUtensorMap ma, mb;
+  DQ_CHECK(tch::make_map(&ma, d_X, d, n, 1, ldx, n * ldx, tc::BLOCK_M));
+  DQ_CHECK(tch::make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, bn));
+  tc::Params p{};
+  p.m_blocks = (int)(n / tc::BLOCK_M); p.n_blocks = d / bn; p.batch = 1; p.ksplit = 1;
+  p.k_blocks = d / tc::BLOCK_K;
+  p.out = d_Y; p.ld = ldy; p.batch_stride = 0; p.split_stride = 0; p.alpha = 1.f;
+  p.partials = nullptr; p.d_status = nullptr;
+  return (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p)
+                     : tch::launch_gemm<128, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p);
+}
+
 }  // namespace dq
