@@ -35,6 +35,7 @@ struct dq_calib {
   TcState tc;                   // tensor-core contractions (operand copies, tensor maps)
   QrTcState qtc;                // tensor-core QR-Orth operand copies
   bool fast_qr = false;
+  bool small128 = false;        // d == 128: shared-memory-resident batched QR-Orth
   bool r_stale = true;
   bool timing = false;
   cudaEvent_t ev[DQ_PHASE_COUNT + 1] = {};
@@ -105,7 +106,10 @@ dq_status fence_out(dq_calib* h) {
 
 dq_status ensure_rotation(dq_calib* h) {
   if (!h->r_stale) return DQ_OK;
-  if (h->fast_qr) {
+  if (h->small128) {
+    DQ_CHECK(qr128_forward(h->ctx, h->Z, h->R, h->U, h->ws.Winv,
+                           h->cfg.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr, h->cfg.batch));
+  } else if (h->fast_qr) {
     DQ_CHECK(qr_forward_fast(h->ctx, h->ws, h->qtc, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch));
   } else {
     DQ_CHECK(qr_forward(h->ctx, h->ws, h->Z, h->R, h->U, tc_rt_operand(h->tc), h->cfg.d, h->cfg.batch));
@@ -153,11 +157,16 @@ dq_status enqueue_step(dq_calib* h, bool timed) {
   }
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[3], ctx.stream));
   // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
-  if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch));
-  else DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch));
-  if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
-  // (a7) Z <- Z - lr Gz
-  DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, (int64_t)d * d * batch));
+  // (a7) Z <- Z - lr Gz  (fused into the backward kernel for 128 x 128 latents)
+  if (h->small128) {
+    DQ_CHECK(qr128_backward_sgd(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, c.lr, batch));
+    if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
+  } else {
+    if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch));
+    else DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch));
+    if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
+    DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, (int64_t)d * d * batch));
+  }
   h->r_stale = true;
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[5], ctx.stream));
   return DQ_OK;
@@ -234,6 +243,7 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
   h->user_stream = (cudaStream_t)cuda_stream;
   h->ctx.sm_count = sms;
   h->X = d_X;
+  h->small128 = (cfg->d == 128);
   const int d = cfg->d, batch = cfg->batch;
   const int64_t dd = (int64_t)d * d * batch;
   dq_status st = DQ_OK;

@@ -97,6 +97,12 @@ dq_status qr_forward(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float*
 dq_status qr_backward(Ctx& ctx, QrWorkspace& ws, const float* R, const float* U, const float* Gq,
                       float* Gz, int d, int batch);
 
+// Batched 128 x 128 QR-Orth resident in shared memory (qr128.cu), one CTA per problem.
+// Forward: R, U (diag > 0), W = U^-1, optional bf16(R^T).  Backward: Gz and the SGD update of Z.
+dq_status qr128_forward(Ctx& ctx, const float* Z, float* R, float* U, float* W, __nv_bfloat16* Rt_bf16, int batch);
+dq_status qr128_backward_sgd(Ctx& ctx, const float* R, const float* W, const float* Gq, float* Gz, float* Z, float lr,
+                             int batch);
+
 // Z <- Z - lr Gz  (n elements)
 dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n);
 
