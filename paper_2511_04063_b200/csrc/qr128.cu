@@ -100,37 +100,51 @@ qr128_forward_kernel(const float* __restrict__ Z, float* __restrict__ R, float* 
   }
   __syncthreads();
 
-  // ---- Householder factorisation, one column per step
+  // ---- Householder factorisation, one column per step, two barriers per step.
+  // v_j is never materialised: v_r = x_r / (x_1 - beta) below the diagonal, 1 on it, so
+  // v^T A[:, c] = A[j][c] + (sum_{r > j} x_r A[r][c]) / (x_1 - beta) and the dot products can
+  // start before the scalars are known.  The squared norm of the next column is accumulated
+  // by the threads that update it.
+  float* rowj = vs;                  // [128] row j of A before the update
+  float* nrmpart = sc;               // [4] partial squared norms of the current column
+  if (c == 0) {
+    float s = 0.f;
+    for (int r = q * 32; r < q * 32 + 32; ++r) s = fmaf(A[r * LD], A[r * LD], s);
+    nrmpart[q] = s;
+  }
+  __syncthreads();
+  const int rlo = q * 32, rhi = rlo + 32;
   for (int j = 0; j < N - 1; ++j) {
-    if (warp < 4) {                  // squared norm of A[j:, j]
-      const int r = warp * 32 + lane;
-      const float x = (r >= j) ? A[r * LD + j] : 0.f;
-      const float s = warp_sum(x * x);
-      if (lane == 0) sc[warp] = s;
-    }
-    __syncthreads();
-    const float nrm2 = (sc[0] + sc[1]) + (sc[2] + sc[3]);
+    const float nrm2 = (nrmpart[0] + nrmpart[1]) + (nrmpart[2] + nrmpart[3]);
     const float alpha = A[j * LD + j];
+    const int r_first = (rlo > j + 1) ? rlo : j + 1;   // rows strictly below the diagonal in this quarter
+    float part = 0.f;
+    if (c > j) {
+      for (int r = r_first; r < rhi; ++r) part = fmaf(A[r * LD + j], A[r * LD + c], part);
+      wpart[q * N + c] = part;
+      if (j >= rlo && j < rhi) rowj[c] = A[j * LD + c];
+    }
     const float sigma = nrm2 - alpha * alpha;
     const bool skip = !(sigma > 0.f);
     const float beta = skip ? alpha : -copysignf(sqrtf(nrm2), alpha);
     const float denom = alpha - beta;
     const float inv_denom = skip ? 0.f : 1.f / denom;
     const float tau = skip ? 0.f : -denom / beta;
-    if (tid < N) vs[tid] = (tid == j) ? 1.f : ((tid > j) ? A[tid * LD + j] * inv_denom : 0.f);
     __syncthreads();
-    const int rlo = q * 32, rhi = rlo + 32;
-    float part = 0.f;
-    if (c > j && rhi > j) {
-      for (int r = (rlo > j ? rlo : j); r < rhi; ++r) part = fmaf(vs[r], A[r * LD + c], part);
+    if (c > j) {
+      const float dot = (wpart[c] + wpart[N + c]) + (wpart[2 * N + c] + wpart[3 * N + c]);
+      const float w = tau * fmaf(dot, inv_denom, rowj[c]);
+      const float wv = w * inv_denom;
+      float nn = 0.f;
+      if (j >= rlo && j < rhi) A[j * LD + c] -= w;                 // diagonal row: v = 1 (not part of the next norm)
+      for (int r = r_first; r < rhi; ++r) {
+        const float t = fmaf(-A[r * LD + j], wv, A[r * LD + c]);
+        A[r * LD + c] = t;
+        nn = fmaf(t, t, nn);
+      }
+      if (c == j + 1) nrmpart[q] = nn;
     }
-    wpart[q * N + c] = part;
-    __syncthreads();
-    if (c > j && rhi > j) {
-      const float w = tau * ((wpart[c] + wpart[N + c]) + (wpart[2 * N + c] + wpart[3 * N + c]));
-      for (int r = (rlo > j ? rlo : j); r < rhi; ++r) A[r * LD + c] = fmaf(-vs[r], w, A[r * LD + c]);
-    }
-    if (tid < N && tid >= j) A[tid * LD + j] = (tid == j) ? beta : vs[tid];   // reflector stays below the diagonal
+    if (tid == 0) A[j * LD + j] = beta;
     __syncthreads();
   }
 

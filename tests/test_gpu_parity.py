@@ -37,9 +37,13 @@ def test_qr_forward_matches_unique_factorisation(d, batch):
     U = c.buf(dq.DQ_BUF_U).cpu().numpy().astype(np.float64)
     for b in range(batch):
         Rr, Ur = orc.qr_pos_lapack(Z0[b])
-        assert np.abs(R[b] - Rr).max() <= 2e-5          # fp32 Householder vs float64
+        # fp32 Householder vs float64.  The 128 x 128 kernel forms R = Z U^-1, whose rounding
+        # error grows with cond(Z) (a few hundred for these matrices): 2^-24 cond sqrt(d) / 4.
+        cond = np.linalg.cond(Z0[b].astype(np.float64))
+        tol_r = 2e-5 if d != 128 else max(2e-5, 6e-8 * cond * np.sqrt(d) / 4)
+        assert np.abs(R[b] - Rr).max() <= tol_r
         assert np.abs(U[b] - Ur).max() <= 5e-5
-        assert ortho_err(R[b]) <= 2e-5
+        assert ortho_err(R[b]) <= tol_r
         assert np.abs(np.tril(U[b], -1)).max() == 0.0 and (np.diag(U[b]) > 0).all()
     c.close()
 
