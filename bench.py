@@ -146,6 +146,8 @@ def main():
     ap.add_argument("--workload", default="c2_7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--qr", default="householder", choices=["householder", "iterative"],
+                    help="QR-Orth forward on the tensor-core path (see dq_calib_set_qr_method)")
     args = ap.parse_args()
 
     from paper_2511_04063_b200 import inputs as gen
@@ -174,7 +176,8 @@ def main():
 
     # ---------------------------------------------------------------- inputs
     # every rank gets its own seeded problem (an independent rotation site)
-    wr = gen.scaled(w, seed=w.seed + rank)
+    from paper_2511_04063_b200 import replicas
+    wr = replicas.workload_for_rank(w, rank)
     X_host = gen.gen_activations(wr)
     Z0_host = gen.gen_latent_init(wr)
     as_torch = (lambda a: torch.from_numpy(a)) if wr.x_dtype == "fp32" else \
@@ -184,6 +187,8 @@ def main():
     Zd = torch.from_numpy(Z0_host).cuda()
     path = dq.DQ_PATH_FP32 if wr.path == "fp32" else dq.DQ_PATH_BF16_TC
     h = dq.dq_calib_init(Xd, Zd, lr=wr.lr, path=path)
+    if args.qr == "iterative":
+        dq.dq_calib_set_qr_method(h, dq.DQ_QR_ITERATIVE, 8)
     K, W = args.steps, max(args.warmup, 3)
     loss_dev = torch.empty((max(K, W), wr.batch), dtype=torch.float32, device="cuda")
 
@@ -233,12 +238,9 @@ def main():
     d2h = loss_host.numel() * 4
 
     # ---------------------------------------------------------------- reduce over ranks
-    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, ms_e2e = float(t[0]), float(t[1])
-    value = world * K / (ms * 1e-3)
-    e2e_value = world * Ke / (ms_e2e * 1e-3)
+    ms, ms_e2e = replicas.max_over_ranks([ms, ms_e2e], device="cuda")
+    value = replicas.whole_job_rate(K, world, ms)
+    e2e_value = replicas.whole_job_rate(Ke, world, ms_e2e)
 
     if rank == 0:
         peaks = load_peaks()
@@ -262,7 +264,7 @@ def main():
                 "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16" if path == dq.DQ_PATH_BF16_TC else "f32", "data": "synthetic",
                 "config": {"workload": wr.name, "d": d, "n_tokens": N, "batch": B, "lr": wr.lr,
-                           "parallelism": "replicas x%d" % world,
+                           "parallelism": "replicas x%d" % world, "qr": args.qr,
                            "l2": "inputs (%.0f MiB X + G) exceed the 126 MB L2" % (2 * h2d / 2 ** 20)},
                 "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"],
                            "reasons": clocks["reasons"], "samples": clocks["samples"]},

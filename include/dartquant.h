@@ -38,7 +38,8 @@ typedef enum {
   DQ_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed                  */
   DQ_ERR_SINGULAR = 5,    /* latent is (numerically) rank deficient: U^-T undefined */
   DQ_ERR_NONFINITE = 6,   /* loss became NaN/Inf                                */
-  DQ_ERR_TIMEOUT = 7      /* a bounded in-kernel wait gave up                   */
+  DQ_ERR_TIMEOUT = 7,     /* a bounded in-kernel wait gave up                   */
+  DQ_ERR_NOT_CONVERGED = 8 /* DQ_QR_ITERATIVE: latent too far from orthogonal     */
 } dq_status;
 
 enum { DQ_FP32 = 0, DQ_BF16 = 1 };             /* x_dtype                       */
@@ -108,6 +109,20 @@ dq_status dq_rotate_apply_static(const void* d_X, int64_t n, int32_t d, int64_t 
  * the handle's stream; rebuild every operand copy derived from it.  Cheap no-op on
  * the fp32 path. */
 dq_status dq_calib_refresh_inputs(dq_calib_t* h);
+
+/* How the QR-Orth forward (Sec. 4.3: Z = R U) is computed on the tensor-core path.  Both
+ * give the same unique factors (diag(U) > 0).
+ *   DQ_QR_HOUSEHOLDER (default): blocked Householder QR (Algorithm 2 in compact-WY form), valid
+ *     for any full-rank latent.
+ *   DQ_QR_ITERATIVE: for latents close to an orthogonal matrix (the regime of the calibration
+ *     loop: Z0 orthogonal, small steps).  U = I + T is the Cholesky factor of Z^T Z = I + E,
+ *     found by the fixed-point iteration T <- striu(E - T^T T) + diag(E - T^T T) / 2 (n_iters
+ *     tensor-core GEMMs, no dependent column steps).  The iteration contracts for roughly
+ *     cond(Z) < 1.5; if the last update is still larger than 1e-5 the status word becomes
+ *     DQ_ERR_NOT_CONVERGED.  n_iters <= 0 selects the default (8).
+ * Ignored (DQ_OK) on the fp32 path and for d == 128. */
+enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
+dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 
 /* Checkpoint / resume of the optimised parameter (Algorithm 1 line 5: Z <- Z0). */
 dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out);

@@ -13,7 +13,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libdartquant.so")
 
 DQ_OK, DQ_ERR_INVALID_ARG, DQ_ERR_UNSUPPORTED, DQ_ERR_ALLOC, DQ_ERR_CUDA = 0, 1, 2, 3, 4
-DQ_ERR_SINGULAR, DQ_ERR_NONFINITE, DQ_ERR_TIMEOUT = 5, 6, 7
+DQ_ERR_SINGULAR, DQ_ERR_NONFINITE, DQ_ERR_TIMEOUT, DQ_ERR_NOT_CONVERGED = 5, 6, 7, 8
+DQ_QR_HOUSEHOLDER, DQ_QR_ITERATIVE = 0, 1
 DQ_FP32, DQ_BF16 = 0, 1
 DQ_PATH_FP32, DQ_PATH_BF16_TC = 0, 1
 DQ_MEAN_TOKENS, DQ_SUM_TOKENS = 0, 1
@@ -25,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_init", "dq_calib_step", "dq_calib_get_rotation", "dq_rotate_apply",
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
-    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static",
+    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method",
 )
 
 
@@ -60,6 +61,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_rotate_apply.argtypes = [vp, i32, i64, i32, i64, vp, vp, i64, vp]
     lib.dq_rotate_apply_static.argtypes = [vp, i64, i32, i64, vp, vp, i64, vp]
     lib.dq_rotate_apply_static.restype = i32
+    lib.dq_calib_set_qr_method.argtypes = [vp, i32, i32]
+    lib.dq_calib_set_qr_method.restype = i32
     lib.dq_calib_get_latent.argtypes = [vp, vp]
     lib.dq_calib_set_latent.argtypes = [vp, vp]
     lib.dq_calib_status.argtypes = [vp]
@@ -148,6 +151,10 @@ def dq_calib_status(h) -> int:
 
 def dq_calib_set_timing(h, enabled: bool):
     _check(load_library().dq_calib_set_timing(h, int(enabled)), "dq_calib_set_timing")
+
+
+def dq_calib_set_qr_method(h, method: int, n_iters: int = 0):
+    _check(load_library().dq_calib_set_qr_method(h, method, n_iters), "dq_calib_set_qr_method")
 
 
 def dq_calib_get_timings(h) -> dict:

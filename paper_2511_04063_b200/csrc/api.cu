@@ -35,6 +35,7 @@ struct dq_calib {
   TcState tc;                   // tensor-core contractions (operand copies, tensor maps)
   QrTcState qtc;                // tensor-core QR-Orth operand copies
   bool fast_qr = false;
+  int qr_method = DQ_QR_HOUSEHOLDER, qr_iters = 8;
   bool small128 = false;        // d == 128: shared-memory-resident batched QR-Orth
   bool r_stale = true;
   bool timing = false;
@@ -110,7 +111,8 @@ dq_status ensure_rotation(dq_calib* h) {
     DQ_CHECK(qr128_forward(h->ctx, h->Z, h->R, h->U, h->ws.Winv,
                            h->cfg.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr, h->cfg.batch));
   } else if (h->fast_qr) {
-    DQ_CHECK(qr_forward_fast(h->ctx, h->ws, h->qtc, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch));
+    DQ_CHECK(qr_forward_fast(h->ctx, h->ws, h->qtc, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch,
+                             h->qr_method == DQ_QR_ITERATIVE ? h->qr_iters : 0));
   } else {
     DQ_CHECK(qr_forward(h->ctx, h->ws, h->Z, h->R, h->U, tc_rt_operand(h->tc), h->cfg.d, h->cfg.batch));
   }
@@ -221,6 +223,7 @@ const char* dq_status_string(dq_status s) {
     case DQ_ERR_SINGULAR: return "latent matrix is rank deficient";
     case DQ_ERR_NONFINITE: return "non-finite loss or factor";
     case DQ_ERR_TIMEOUT: return "bounded in-kernel wait gave up";
+    case DQ_ERR_NOT_CONVERGED: return "iterative QR did not converge: latent too far from orthogonal";
   }
   return "unknown status";
 }
@@ -369,8 +372,21 @@ dq_status dq_calib_status(dq_calib_t* h) {
   if (cudaMemcpyAsync(&code, h->ctx.d_status, sizeof(int), cudaMemcpyDeviceToHost, h->ctx.stream) != cudaSuccess)
     return DQ_ERR_CUDA;
   if (cudaStreamSynchronize(h->ctx.stream) != cudaSuccess) return DQ_ERR_CUDA;
-  if (code < 0 || code > DQ_ERR_TIMEOUT) return DQ_ERR_CUDA;
+  if (code < 0 || code > DQ_ERR_NOT_CONVERGED) return DQ_ERR_CUDA;
   return (dq_status)code;
+}
+
+dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters) {
+  if (!h || (method != DQ_QR_HOUSEHOLDER && method != DQ_QR_ITERATIVE) || n_iters > 64) return DQ_ERR_INVALID_ARG;
+  const int iters = n_iters <= 0 ? 8 : n_iters;
+  if (method == h->qr_method && iters == h->qr_iters) return DQ_OK;
+  DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
+  h->qr_method = method;
+  h->qr_iters = iters;
+  h->r_stale = true;
+  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
+  h->graph_failed = false;
+  return DQ_OK;
 }
 
 dq_status dq_calib_set_timing(dq_calib_t* h, int32_t enabled) {

@@ -89,6 +89,51 @@ __global__ void __launch_bounds__(256) skew_t_split_kernel(const float* __restri
   }
 }
 
+// One sweep of the fixed-point iteration for the Cholesky factor U = I + T of G = Z^T Z:
+//   T <- striu(G - I - P) + diag(G - I - P) / 2,   P = T^T T (nullptr on the first sweep: T = 0).
+// G and P are only valid on and above the diagonal.  Writes T (fp32, row-major, zeros below the
+// diagonal), the split-bf16 copy of T^T (operand of the next P = T^T T) and, on the last sweep,
+// U = I + T with its split copy.  check: flag DQ_ERR_NOT_CONVERGED if an entry still moved by
+// more than tol (the iteration contracts, so the remaining error is below the last update).
+__global__ void __launch_bounds__(256) chol_fixpoint_kernel(const float* __restrict__ G, const float* __restrict__ P,
+                                                            float* __restrict__ T, bf16* __restrict__ tt_hi,
+                                                            bf16* __restrict__ tt_lo, float* __restrict__ U,
+                                                            bf16* __restrict__ u_hi, bf16* __restrict__ u_lo, int d,
+                                                            int check, float tol, int* d_status) {
+  __shared__ float t[32][33];
+  const int64_t off = (int64_t)blockIdx.z * d * d;
+  G += off; T += off; tt_hi += off; tt_lo += off;
+  if (P) P += off;
+  if (U) { U += off; u_hi += off; u_lo += off; }
+  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const bool upper = j0 + 31 >= i0;     // tile touches the upper triangle
+  bool moved = false;
+  for (int r = ty; r < 32; r += 8) {
+    const int i = i0 + r, j = j0 + tx;
+    const int64_t idx = (int64_t)i * d + j;
+    float v = 0.f;
+    if (upper && j >= i) {
+      v = G[idx] - ((i == j) ? 1.f : 0.f) - (P ? P[idx] : 0.f);
+      if (i == j) v *= 0.5f;
+      if (check && !(fabsf(v - T[idx]) <= tol)) moved = true;
+    }
+    T[idx] = v;
+    t[r][tx] = v;
+    if (U) {
+      const float u = v + ((i == j) ? 1.f : 0.f);
+      U[idx] = u;
+      split2(u, u_hi[idx], u_lo[idx]);
+    }
+  }
+  if (moved) set_status(d_status, DQ_ERR_NOT_CONVERGED);
+  __syncthreads();
+  for (int c = ty; c < 32; c += 8) {    // T^T[j][i] = T[i][j]
+    const int64_t idx = (int64_t)(j0 + c) * d + i0 + tx;
+    split2(t[tx][c], tt_hi[idx], tt_lo[idx]);
+  }
+}
+
 // Inverse of each 128 x 128 upper-triangular diagonal block of U; thread j solves U x = e_j
 // by back-substitution.  Writes the split inverse in row-major (WN) and transposed (WT) form.
 constexpr int DB = 128;
@@ -253,13 +298,47 @@ dq_status qr_factor_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, 
   return qr_diag_check(ctx, At, d, batch);
 }
 
+// U of a latent close to an orthogonal matrix, without dependent column steps: G = Z^T Z (upper
+// tiles), then n_iters sweeps T <- Phi(G - I - T^T T); every product is a split-bf16 tensor-core
+// GEMM restricted to the non-zero blocks of its triangular operands.
+dq_status qr_upper_factor_iterative(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* U, int d,
+                                    int batch, int n_iters) {
+  const int64_t dd = (int64_t)d * d;
+  const dim3 tiles(d / 32, d / 32, batch);
+  bf16 *zt_hi = q.st_hi, *zt_lo = q.st_lo;     // free until the backward pass
+  float *G = ws.B, *P = ws.S, *T = ws.tmp;
+  DQ_CHECK(qrp_transpose_split(ctx, Z, ws.A, zt_hi, zt_lo, d, batch));
+  {   // G[i][j] = sum_k Z[k][i] Z[k][j], tiles on and above the block diagonal
+    Op a{zt_hi, zt_lo, d, dd};
+    Out o; o.f32 = G; o.ld = d; o.bs = dd; o.tri_skip = 1;
+    DQ_CHECK(gemm3(ctx, a, a, d, d, d, batch, o));
+  }
+  for (int it = 0; it < n_iters; ++it) {
+    const bool last = it == n_iters - 1;
+    if (it > 0) {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
+      Op tt{q.t1_hi, q.t1_lo, d, dd};
+      Out o; o.f32 = P; o.ld = d; o.bs = dd; o.tri_skip = 1; o.k_mode = 2;
+      DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
+    }
+    chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, it > 0 ? P : nullptr, T, q.t1_hi, q.t1_lo,
+                                                        last ? U : nullptr, q.u_hi, q.u_lo, d,
+                                                        (last && it > 0) ? 1 : 0, 1e-5f, ctx.d_status);
+    DQ_CHECK(after_launch(ctx));
+  }
+  return qr_diag_check(ctx, U, d, batch);
+}
+
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
-                          int batch) {
+                          int batch, int iterative_iters) {
   if (d % 128 != 0) return DQ_ERR_UNSUPPORTED;
   const int64_t dd = (int64_t)d * d;
   const dim3 tiles(d / 32, d / 32, batch);
-  DQ_CHECK(qr_factor_tc(ctx, ws, q, Z, d, batch));
-  DQ_CHECK(qrp_gauge_ut(ctx, ws.A, U, q.u_hi, q.u_lo, d, batch));
+  if (iterative_iters > 0) {
+    DQ_CHECK(qr_upper_factor_iterative(ctx, ws, q, Z, U, d, batch, iterative_iters));
+  } else {
+    DQ_CHECK(qr_factor_tc(ctx, ws, q, Z, d, batch));
+    DQ_CHECK(qrp_gauge_ut(ctx, ws.A, U, q.u_hi, q.u_lo, d, batch));
+  }
   DQ_CHECK(tri_inverse_tc(ctx, q, U, d, batch));
   split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
   DQ_CHECK(after_launch(ctx));

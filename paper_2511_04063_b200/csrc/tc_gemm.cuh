@@ -39,6 +39,12 @@ struct Params {
   float alpha, beta;
   float* partials;         // EPI_WHIP: [unit][4] loss partial sums
   int* d_status;
+  // Triangular structure (square tiles, ksplit == 1).  tri_skip: tiles below the block diagonal
+  // (mb > nb) are not computed.  k_mode bits restrict the reduction of tile (mb, nb) to the
+  // k-range where both operands can be non-zero:
+  //   1: A[m][k] = 0 for k <  128 mb        2: A[m][k] = 0 for k >= 128 (mb + 1)
+  //   4: B[n][k] = 0 for k >= 128 (nb + 1)  8: B[n][k] = 0 for k <  128 nb
+  int tri_skip, k_mode;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -202,8 +208,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 
   const int tiles_per_batch = p.m_blocks * p.n_blocks;
   const int units = tiles_per_batch * p.batch * p.ksplit;
-  // split s of the reduction covers k-blocks [s * k_blocks / ksplit, (s + 1) * k_blocks / ksplit)
-  auto split_begin = [&](int s) { return (int)(((int64_t)s * p.k_blocks) / p.ksplit); };
+  // split s of the reduction covers k-blocks [s * k_blocks / ksplit, (s + 1) * k_blocks / ksplit);
+  // with k_mode the range is clipped to the non-zero part of triangular operands.
+  auto k_range = [&](int split, int mb, int nb, int& k0, int& kn) {
+    int lo = (int)(((int64_t)split * p.k_blocks) / p.ksplit);
+    int hi = (int)(((int64_t)(split + 1) * p.k_blocks) / p.ksplit);
+    if (p.k_mode) {
+      constexpr int R = BLOCK_M / BLOCK_K;   // k-blocks per 128 rows
+      if ((p.k_mode & 1) && lo < R * mb) lo = R * mb;
+      if ((p.k_mode & 8) && lo < R * nb) lo = R * nb;
+      if ((p.k_mode & 2) && hi > R * (mb + 1)) hi = R * (mb + 1);
+      if ((p.k_mode & 4) && hi > R * (nb + 1)) hi = R * (nb + 1);
+    }
+    k0 = lo; kn = hi - lo;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
@@ -217,8 +235,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         const int b = t / tiles_per_batch;
         const int r = t % tiles_per_batch;
         const int mb = r % p.m_blocks, nb = r / p.m_blocks;   // m fastest: neighbours share the B tile
-        const int k0 = split_begin(split);
-        const int kb_per_split = split_begin(split + 1) - k0;
+        if (p.tri_skip && mb > nb) continue;
+        int k0, kb_per_split;
+        k_range(split, mb, nb, k0, kb_per_split);
         for (int kb = 0; kb < kb_per_split; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), L::STAGE_BYTES);
@@ -244,11 +263,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        const int split = u % p.ksplit;
+        const int rr = (u / p.ksplit) % tiles_per_batch;
+        const int mb = rr % p.m_blocks, nb = rr / p.m_blocks;
+        if (p.tri_skip && mb > nb) continue;
+        int k0_unused, kb_per_split;
+        k_range(split, mb, nb, k0_unused, kb_per_split);
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BLOCK_N);
-        const int split = u % p.ksplit;
-        const int kb_per_split = split_begin(split + 1) - split_begin(split);
         for (int kb = 0; kb < kb_per_split; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, p.d_status)) { ok = false; break; }
           tc_fence_after();
@@ -286,13 +309,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       const int b = t / tiles_per_batch;
       const int r = t % tiles_per_batch;
       const int mb = r % p.m_blocks, nb = r / p.m_blocks;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
-      tc_fence_after();
+      if (p.tri_skip && mb > nb) continue;
       const int row = mb * BLOCK_M + q * 32 + lane;
       const int64_t out_off = (int64_t)b * p.batch_stride + (int64_t)split * p.split_stride +
                               (int64_t)row * p.ld + (int64_t)nb * BLOCK_N;
+      // Accumulating epilogue (beta != 0): fetch the old output row while the MMAs of this tile
+      // are still running, so the global-load latency is not paid once per 32-column chunk.
+      constexpr bool PREFETCH = (EPI == EPI_GEN && BLOCK_N == 128);
+      float4 old[PREFETCH ? 32 : 1];
+      const bool use_old = PREFETCH && p.out != nullptr && p.beta != 0.f;
+      if (PREFETCH && use_old) {
+        const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.out) + out_off);
+#pragma unroll
+        for (int i = 0; i < (PREFETCH ? 32 : 1); ++i) old[i] = src[i];
+      }
+      if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
+      tc_fence_after();
       float esum = 0.f;
-#pragma unroll 1
+#pragma unroll(PREFETCH ? 4 : 1)
       for (int c = 0; c < BLOCK_N / 32; ++c) {
         uint32_t v[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BLOCK_N + c * 32), v);
@@ -323,7 +357,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             if (p.beta != 0.f) {
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                const float4 o = dst[i];
+                const float4 o = PREFETCH ? old[PREFETCH ? c * 8 + i : 0] : dst[i];
                 f[4 * i] = fmaf(p.beta, o.x, f[4 * i]); f[4 * i + 1] = fmaf(p.beta, o.y, f[4 * i + 1]);
                 f[4 * i + 2] = fmaf(p.beta, o.z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.beta, o.w, f[4 * i + 3]);
               }

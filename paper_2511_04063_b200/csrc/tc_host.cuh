@@ -69,6 +69,7 @@ struct Out {
   // split-K: slice s of the reduction writes alpha * partial product (beta must be 0, no
   // split copy) to f32 + s * split_stride; the caller reduces.
   int ksplit = 1; int64_t split_stride = 0;
+  int tri_skip = 0, k_mode = 0;   // triangular structure, see tc::Params
 };
 
 // D[m][n] = alpha sum_k A[m][k] B[n][k] (+ beta D) with split-bf16 operands (three bf16 MMAs per
@@ -86,6 +87,8 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
   p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = o.split_stride;
   p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
   p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
+  if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
+  p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
   return launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
 }
 

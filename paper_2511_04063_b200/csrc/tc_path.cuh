@@ -55,8 +55,9 @@ struct QrTcState {
 };
 dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count);
 void qr_tc_destroy(QrTcState& q);
+// iterative_iters > 0: U by the near-orthogonal fixed-point iteration instead of Householder.
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
-                          int batch);
+                          int batch, int iterative_iters);
 dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch);
 
 

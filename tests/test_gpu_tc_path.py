@@ -103,6 +103,57 @@ def test_tensor_core_qr_forward_matches_unique_factorisation(d, batch, kind):
     c.close()
 
 
+def _near_orthogonal(d, batch, amp, seed):
+    rng = np.random.default_rng(seed)
+    Z0 = np.empty((batch, d, d), dtype=np.float32)
+    for b in range(batch):
+        Q, _ = np.linalg.qr(rng.standard_normal((d, d)))
+        Z0[b] = Q + amp * rng.standard_normal((d, d)) / np.sqrt(d)
+    return Z0
+
+
+@pytest.mark.parametrize("d,batch,amp", [(256, 2, 0.02), (640, 1, 0.05), (1024, 1, 0.02), (1152, 1, 0.1)])
+def test_iterative_qr_matches_unique_factorisation_near_orthogonal(d, batch, amp):
+    """DQ_QR_ITERATIVE: U = I + T from the fixed-point iteration on Z^T Z equals the Cholesky /
+    QR factor for latents near an orthogonal matrix (cond(Z) about 1.06 .. 1.3 here)."""
+    w = small("c2_7b", d=d, n_tokens=256, batch=batch, n_outlier_channels=1)
+    Z0 = _near_orthogonal(d, batch, amp, d)
+    c = Calib(w, Z0=Z0)
+    dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_ITERATIVE, 10)
+    R = c.rotation()
+    assert c.status() == dq.DQ_OK
+    U = c.buf(dq.DQ_BUF_U).cpu().numpy().astype(np.float64)
+    for b in range(batch):
+        Rr, Ur = orc.qr_pos_lapack(Z0[b])
+        assert np.abs(U[b] - Ur).max() <= 2e-5
+        assert np.abs(np.tril(U[b], -1)).max() == 0.0 and (np.diag(U[b]) > 0).all()
+        assert np.abs(R[b] - Rr).max() <= 5e-5
+        assert np.abs(R[b].T @ R[b] - np.eye(d)).max() <= 5e-5
+    # the two methods agree on a whole step
+    l_it = c.step(1)[0]
+    Z_it = c.latent()
+    c2 = Calib(w, Z0=Z0)
+    l_hh = c2.step(1)[0]
+    Z_hh = c2.latent()
+    assert np.allclose(l_it, l_hh, rtol=1e-4)
+    # R differs in its last bits between the methods, so a few entries of bf16(R) round the other way
+    # and a few dL/dO near the kink of Eq. 4 change sign: the updates agree to a few percent.
+    assert np.linalg.norm(Z_it - Z_hh) <= 5e-2 * np.linalg.norm(Z_hh - Z0)
+    c.close(); c2.close()
+
+
+def test_iterative_qr_flags_latents_far_from_orthogonal():
+    d = 256
+    w = small("c2_7b", d=d, n_tokens=256, n_outlier_channels=1)
+    Z0 = _near_orthogonal(d, 1, 0.02, 5) * np.float32(1.6)          # Z^T Z = 2.56 I + ...: no contraction
+    c = Calib(w, Z0=Z0)
+    dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_ITERATIVE, 8)
+    c.rotation()
+    assert c.status() == dq.DQ_ERR_NOT_CONVERGED
+    assert "converge" in dq.status_string(dq.DQ_ERR_NOT_CONVERGED)
+    c.close()
+
+
 def test_tensor_core_path_is_bit_reproducible():
     w = small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3)
     outs = []

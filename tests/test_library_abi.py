@@ -34,8 +34,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_version_and_status_strings(lib):
     assert "sm_100a" in dq.dq_version()
-    seen = {dq.status_string(s) for s in range(8)}
-    assert len(seen) == 8
+    seen = {dq.status_string(s) for s in range(9)}
+    assert len(seen) == 9
 
 
 def test_null_arguments_fail_before_any_cuda_call(lib):
