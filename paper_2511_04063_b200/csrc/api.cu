@@ -306,7 +306,10 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
   DQ_CHECK(fence_in(h));
   if (h->timing) { for (auto& m : h->ms_acc) m = 0.0; h->timed_steps = 0; }
   for (int s = 0; s < n_steps; ++s) {
-    const bool use_graph = !h->timing && h->r_stale && h->eager_steps_done >= 1;
+    // The captured step of the iterative QR is the warm-started one: replay it only while the
+    // previous step's factor belongs to a nearby latent.
+    const bool iterative = h->fast_qr && !h->small128 && h->qr_method == DQ_QR_ITERATIVE;
+    const bool use_graph = !h->timing && h->r_stale && h->eager_steps_done >= 1 && (!iterative || h->qtc.t_warm);
     if (use_graph && !h->graph && !h->graph_failed) try_capture(h);
     if (use_graph && h->graph) {
       DQ_CHECK_CUDA(cudaGraphLaunch(h->graph, ctx.stream));
@@ -363,6 +366,7 @@ dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z) {
   DQ_CHECK_CUDA(cudaMemcpyAsync(h->Z, d_Z, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
                                 cudaMemcpyDeviceToDevice, h->ctx.stream));
   h->r_stale = true;
+  h->qtc.t_warm = false;   // the new latent may be far from the one the iterative QR last saw
   return fence_out(h);
 }
 
@@ -384,6 +388,7 @@ dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters)
   h->qr_method = method;
   h->qr_iters = iters;
   h->r_stale = true;
+  h->qtc.t_warm = false;
   if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
   h->graph_failed = false;
   return DQ_OK;

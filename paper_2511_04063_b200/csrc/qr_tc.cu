@@ -9,6 +9,9 @@
 // Backward: B = R^T Gq, S = tril(B - B^T, -1), Gz = (R S) W^T.
 // All d x d products run as split-bf16 tcgen05 GEMMs (three bf16 MMAs per product,
 // fp32 accumulation, ~2^-16 relative error).
+#include <algorithm>
+#include <vector>
+
 #include "tc_host.cuh"
 #include "tc_path.cuh"
 
@@ -95,11 +98,12 @@ __global__ void __launch_bounds__(256) skew_t_split_kernel(const float* __restri
 // diagonal), the split-bf16 copy of T^T (operand of the next P = T^T T) and, on the last sweep,
 // U = I + T with its split copy.  check: flag DQ_ERR_NOT_CONVERGED if an entry still moved by
 // more than tol (the iteration contracts, so the remaining error is below the last update).
+// lower_done: tiles strictly below the diagonal already hold their zeros.
 __global__ void __launch_bounds__(256) chol_fixpoint_kernel(const float* __restrict__ G, const float* __restrict__ P,
                                                             float* __restrict__ T, bf16* __restrict__ tt_hi,
                                                             bf16* __restrict__ tt_lo, float* __restrict__ U,
                                                             bf16* __restrict__ u_hi, bf16* __restrict__ u_lo, int d,
-                                                            int check, float tol, int* d_status) {
+                                                            int check, int lower_done, float tol, int* d_status) {
   __shared__ float t[32][33];
   const int64_t off = (int64_t)blockIdx.z * d * d;
   G += off; T += off; tt_hi += off; tt_lo += off;
@@ -108,6 +112,7 @@ __global__ void __launch_bounds__(256) chol_fixpoint_kernel(const float* __restr
   const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const bool upper = j0 + 31 >= i0;     // tile touches the upper triangle
+  if (!upper && lower_done && !U) return;   // zeros written by an earlier sweep stay zeros
   bool moved = false;
   for (int r = ty; r < 32; r += 8) {
     const int i = i0 + r, j = j0 + tx;
@@ -134,41 +139,85 @@ __global__ void __launch_bounds__(256) chol_fixpoint_kernel(const float* __restr
   }
 }
 
-// Inverse of each 128 x 128 upper-triangular diagonal block of U; thread j solves U x = e_j
-// by back-substitution.  Writes the split inverse in row-major (WN) and transposed (WT) form.
+// Inverse of each 128 x 128 upper-triangular diagonal block of U, one CTA per block: the four
+// 32 x 32 diagonal sub-blocks by back-substitution (one warp each, lane j solves U x = e_j), then
+// inv([A B; 0 C]) = [A^-1, -A^-1 B C^-1; 0, C^-1] twice as shared-memory products.  Writes the
+// split inverse in row-major (WN) and transposed (WT) form.
 constexpr int DB = 128;
-__global__ void __launch_bounds__(DB) tri_inv_diag128_kernel(const float* __restrict__ U, bf16* __restrict__ wn_hi,
-                                                             bf16* __restrict__ wn_lo, bf16* __restrict__ wt_hi,
-                                                             bf16* __restrict__ wt_lo, int d) {
+constexpr int DLD = 129;
+constexpr int TRI_INV_THREADS = 256;
+constexpr int TRI_INV_SMEM = (2 * DB * DLD + 64 * 65) * 4;
+
+__device__ __forceinline__ void smem_mm4(const float* A, int lda, const float* B, int ldb, float* C, int ldc, int M,
+                                         int N, int K, float alpha, int tid) {
+  const int tn = N / 4, tiles = (M / 4) * tn;
+  for (int t = tid; t < tiles; t += TRI_INV_THREADS) {
+    const int r0 = (t / tn) * 4, c0 = (t % tn) * 4;
+    float acc[4][4] = {};
+    for (int k = 0; k < K; ++k) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) av[i] = A[(r0 + i) * lda + k];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bv[j] = B[k * ldb + c0 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) C[(r0 + i) * ldc + c0 + j] = alpha * acc[i][j];
+  }
+}
+
+__global__ void __launch_bounds__(TRI_INV_THREADS) tri_inv_diag128_kernel(const float* __restrict__ U,
+                                                                          bf16* __restrict__ wn_hi,
+                                                                          bf16* __restrict__ wn_lo,
+                                                                          bf16* __restrict__ wt_hi,
+                                                                          bf16* __restrict__ wt_lo, int d) {
   extern __shared__ float sm[];
-  float (*Us)[DB + 1] = reinterpret_cast<float (*)[DB + 1]>(sm);
-  float (*Xs)[DB + 1] = reinterpret_cast<float (*)[DB + 1]>(sm + DB * (DB + 1));
+  float* Us = sm;
+  float* Xs = sm + DB * DLD;
+  float* Tmp = Xs + DB * DLD;
   const int64_t off = (int64_t)blockIdx.y * d * d + (int64_t)blockIdx.x * DB * (d + 1);
   U += off; wn_hi += off; wn_lo += off; wt_hi += off; wt_lo += off;
-  const int j = threadIdx.x;
-  for (int r = 0; r < DB; ++r) Us[r][j] = U[(int64_t)r * d + j];
-  __syncthreads();
-  for (int i = DB - 1; i > j; --i) Xs[i][j] = 0.f;
-  Xs[j][j] = 1.f / Us[j][j];
-  for (int i = j - 1; i >= 0; --i) {
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-    int k = i + 1;
-    for (; k + 3 <= j; k += 4) {
-      s0 = fmaf(Us[i][k], Xs[k][j], s0);
-      s1 = fmaf(Us[i][k + 1], Xs[k + 1][j], s1);
-      s2 = fmaf(Us[i][k + 2], Xs[k + 2][j], s2);
-      s3 = fmaf(Us[i][k + 3], Xs[k + 3][j], s3);
-    }
-    for (; k <= j; ++k) s0 = fmaf(Us[i][k], Xs[k][j], s0);
-    Xs[i][j] = -((s0 + s1) + (s2 + s3)) / Us[i][i];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int e = tid; e < DB * DB; e += TRI_INV_THREADS) {
+    const int r = e >> 7, c = e & 127;
+    Us[r * DLD + c] = U[(int64_t)r * d + c];
+    Xs[r * DLD + c] = 0.f;
   }
   __syncthreads();
-  for (int r = 0; r < DB; ++r) {
+  if (warp < 4) {
+    const int o = warp * 32, j = lane;
+    Xs[(o + j) * DLD + o + j] = 1.f / Us[(o + j) * DLD + o + j];
+    for (int i = j - 1; i >= 0; --i) {
+      float s = 0.f;
+      for (int k = i + 1; k <= j; ++k) s = fmaf(Us[(o + i) * DLD + o + k], Xs[(o + k) * DLD + o + j], s);
+      Xs[(o + i) * DLD + o + j] = -s / Us[(o + i) * DLD + o + i];
+    }
+  }
+  __syncthreads();
+  for (int pair = 0; pair < 2; ++pair) {
+    const int o = pair * 64;
+    smem_mm4(Us + o * DLD + o + 32, DLD, Xs + (o + 32) * DLD + o + 32, DLD, Tmp, 65, 32, 32, 32, 1.f, tid);
+    __syncthreads();
+    smem_mm4(Xs + o * DLD + o, DLD, Tmp, 65, Xs + o * DLD + o + 32, DLD, 32, 32, 32, -1.f, tid);
+    __syncthreads();
+  }
+  smem_mm4(Us + 64, DLD, Xs + 64 * DLD + 64, DLD, Tmp, 65, 64, 64, 64, 1.f, tid);
+  __syncthreads();
+  smem_mm4(Xs, DLD, Tmp, 65, Xs + 64, DLD, 64, 64, 64, -1.f, tid);
+  __syncthreads();
+  for (int e = tid; e < DB * DB; e += TRI_INV_THREADS) {
+    const int r = e >> 7, c = e & 127;
     bf16 h, l;
-    split2(Xs[r][j], h, l);                       // X[r][j] -> WN[r][j]
-    wn_hi[(int64_t)r * d + j] = h; wn_lo[(int64_t)r * d + j] = l;
-    split2(Xs[j][r], h, l);                       // X[j][r] -> WT[r][j]
-    wt_hi[(int64_t)r * d + j] = h; wt_lo[(int64_t)r * d + j] = l;
+    split2(Xs[r * DLD + c], h, l);                 // X[r][c] -> WN[r][c]
+    wn_hi[(int64_t)r * d + c] = h; wn_lo[(int64_t)r * d + c] = l;
+    split2(Xs[c * DLD + r], h, l);                 // X[c][r] -> WT[r][c]
+    wt_hi[(int64_t)r * d + c] = h; wt_lo[(int64_t)r * d + c] = l;
   }
 }
 
@@ -202,13 +251,13 @@ dq_status tri_inverse_tc(Ctx& ctx, QrTcState& q, const float* U, int d, int batc
   DQ_CHECK_CUDA(cudaMemsetAsync(q.wn_lo, 0, bytes, ctx.stream));
   DQ_CHECK_CUDA(cudaMemsetAsync(q.wt_hi, 0, bytes, ctx.stream));
   DQ_CHECK_CUDA(cudaMemsetAsync(q.wt_lo, 0, bytes, ctx.stream));
-  const int smem = 2 * DB * (DB + 1) * (int)sizeof(float);
+  const int smem = TRI_INV_SMEM;
   static bool attr = false;
   if (!attr) {
     DQ_CHECK_CUDA(cudaFuncSetAttribute(tri_inv_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr = true;
   }
-  tri_inv_diag128_kernel<<<dim3(d / DB, batch), DB, smem, ctx.stream>>>(U, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, d);
+  tri_inv_diag128_kernel<<<dim3(d / DB, batch), TRI_INV_THREADS, smem, ctx.stream>>>(U, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, d);
   DQ_CHECK(after_launch(ctx));
   int s = DB, count = d / DB;
   while (count > 1 && count % 2 == 0) {
@@ -256,6 +305,25 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
     if (e > q.part_bs) q.part_bs = e;
   }
   if (q.part_bs > 0) DQ_CHECK(alloc(&q.part, q.part_bs * batch));
+  DQ_CHECK(alloc(&q.tw_hi, dd)); DQ_CHECK(alloc(&q.tw_lo, dd));
+  {   // tile orders: most expensive tiles first, dealt round-robin to the persistent CTAs
+    const int nb = d / 128;
+    std::vector<int> upper, desc, asc;
+    for (int j = 0; j < nb; ++j)
+      for (int i = 0; i < nb; ++i) {
+        if (i <= j) upper.push_back(i | (j << 16));
+        desc.push_back(i | (j << 16));
+      }
+    std::stable_sort(upper.begin(), upper.end(), [](int a, int b) { return (a & 0xffff) > (b & 0xffff); });
+    std::stable_sort(desc.begin(), desc.end(), [](int a, int b) { return (a >> 16) > (b >> 16); });
+    asc = desc;
+    std::reverse(asc.begin(), asc.end());
+    q.n_upper = (int)upper.size(); q.n_all = (int)desc.size();
+    DQ_CHECK(alloc(&q.tl_upper, q.n_upper)); DQ_CHECK(alloc(&q.tl_desc_nb, q.n_all)); DQ_CHECK(alloc(&q.tl_asc_nb, q.n_all));
+    DQ_CHECK_CUDA(cudaMemcpy(q.tl_upper, upper.data(), sizeof(int) * upper.size(), cudaMemcpyHostToDevice));
+    DQ_CHECK_CUDA(cudaMemcpy(q.tl_desc_nb, desc.data(), sizeof(int) * desc.size(), cudaMemcpyHostToDevice));
+    DQ_CHECK_CUDA(cudaMemcpy(q.tl_asc_nb, asc.data(), sizeof(int) * asc.size(), cudaMemcpyHostToDevice));
+  }
   q.ready = true;
   return DQ_OK;
 }
@@ -265,6 +333,7 @@ void qr_tc_destroy(QrTcState& q) {
                  q.rt_hi, q.rt_lo, q.gqt_hi, q.gqt_lo, q.st_hi, q.st_lo, q.m_hi, q.m_lo, q.t1_hi, q.t1_lo};
   for (bf16* p : all) cudaFree(p);
   cudaFree(q.y_hi); cudaFree(q.y_lo); cudaFree(q.w2_hi); cudaFree(q.w2_lo); cudaFree(q.part); cudaFree(q.T);
+  cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.tl_upper); cudaFree(q.tl_desc_nb); cudaFree(q.tl_asc_nb);
   q = QrTcState();
 }
 
@@ -310,21 +379,28 @@ dq_status qr_upper_factor_iterative(Ctx& ctx, QrWorkspace& ws, QrTcState& q, con
   DQ_CHECK(qrp_transpose_split(ctx, Z, ws.A, zt_hi, zt_lo, d, batch));
   {   // G[i][j] = sum_k Z[k][i] Z[k][j], tiles on and above the block diagonal
     Op a{zt_hi, zt_lo, d, dd};
-    Out o; o.f32 = G; o.ld = d; o.bs = dd; o.tri_skip = 1;
+    Out o; o.f32 = G; o.ld = d; o.bs = dd; o.tile_list = q.tl_upper; o.n_list = q.n_upper;
     DQ_CHECK(gemm3(ctx, a, a, d, d, d, batch, o));
   }
-  for (int it = 0; it < n_iters; ++it) {
-    const bool last = it == n_iters - 1;
-    if (it > 0) {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
-      Op tt{q.t1_hi, q.t1_lo, d, dd};
-      Out o; o.f32 = P; o.ld = d; o.bs = dd; o.tri_skip = 1; o.k_mode = 2;
+  // From T = 0: n_iters sweeps, the first without the product.  From the previous step's T (the
+  // latent moved by one optimiser step): three sweeps.
+  const bool warm = q.t_warm;
+  const int sweeps = warm ? (n_iters < 3 ? n_iters : 3) : n_iters;
+  for (int it = 0; it < sweeps; ++it) {
+    const bool last = it == sweeps - 1;
+    const bool with_p = warm || it > 0;
+    if (with_p) {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
+      Op tt{q.tw_hi, q.tw_lo, d, dd};
+      Out o; o.f32 = P; o.ld = d; o.bs = dd; o.k_mode = 2; o.tile_list = q.tl_upper; o.n_list = q.n_upper;
       DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
     }
-    chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, it > 0 ? P : nullptr, T, q.t1_hi, q.t1_lo,
+    chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, with_p ? P : nullptr, T, q.tw_hi, q.tw_lo,
                                                         last ? U : nullptr, q.u_hi, q.u_lo, d,
-                                                        (last && it > 0) ? 1 : 0, 1e-5f, ctx.d_status);
+                                                        (last && with_p) ? 1 : 0, (warm || it > 0) ? 1 : 0, 1e-5f,
+                                                        ctx.d_status);
     DQ_CHECK(after_launch(ctx));
   }
+  q.t_warm = true;
   return qr_diag_check(ctx, U, d, batch);
 }
 
@@ -346,6 +422,8 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
   Op a{q.z_hi, q.z_lo, d, dd};
   Op b{q.wt_hi, q.wt_lo, d, dd};
   Out o; o.f32 = R; o.ld = d; o.bs = dd; o.hi = q.r_hi; o.lo = q.r_lo; o.ld_h = d; o.bs_h = dd;
+  o.k_mode = 4;   // W is upper triangular: W^T[j][k] = 0 for k > j
+  o.tile_list = q.tl_desc_nb; o.n_list = q.n_all;
   DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   split_kernel<<<tiles, 256, 0, ctx.stream>>>(R, q.rt_hi, q.rt_lo, d, 1);
   return after_launch(ctx);
@@ -365,10 +443,14 @@ dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* G
   // M[i][j] = sum_k R[i][k] S[k][j]:  A = R, B-operand = S^T; only the split copy is kept
   Op r{q.r_hi, q.r_lo, d, dd}, st{q.st_hi, q.st_lo, d, dd};
   Out om; om.hi = q.m_hi; om.lo = q.m_lo; om.ld_h = d; om.bs_h = dd;
+  om.k_mode = 8;  // S is strictly lower triangular: S^T[j][k] = 0 for k < j
+  om.tile_list = q.tl_asc_nb; om.n_list = q.n_all;
   DQ_CHECK(gemm3(ctx, r, st, d, d, d, batch, om));
   // Gz[i][j] = sum_k M[i][k] W[j][k]
   Op m{q.m_hi, q.m_lo, d, dd}, wn{q.wn_hi, q.wn_lo, d, dd};
   Out og; og.f32 = Gz; og.ld = d; og.bs = dd;
+  og.k_mode = 8;  // W[j][k] = 0 for k < j
+  og.tile_list = q.tl_asc_nb; og.n_list = q.n_all;
   return gemm3(ctx, m, wn, d, d, d, batch, og);
 }
 

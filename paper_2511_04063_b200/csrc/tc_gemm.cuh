@@ -45,6 +45,10 @@ struct Params {
   //   1: A[m][k] = 0 for k <  128 mb        2: A[m][k] = 0 for k >= 128 (mb + 1)
   //   4: B[n][k] = 0 for k >= 128 (nb + 1)  8: B[n][k] = 0 for k <  128 nb
   int tri_skip, k_mode;
+  // Optional explicit tile order (device array of mb | nb << 16, n_list entries per problem), e.g.
+  // most expensive tiles first so that the round-robin deal over the persistent CTAs is balanced.
+  const int* tile_list;
+  int n_list;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -206,7 +210,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
 
-  const int tiles_per_batch = p.m_blocks * p.n_blocks;
+  const int tiles_per_batch = p.tile_list ? p.n_list : p.m_blocks * p.n_blocks;
+  auto tile_of = [&](int r, int& mb, int& nb) {
+    if (p.tile_list) { const int code = p.tile_list[r]; mb = code & 0xffff; nb = code >> 16; }
+    else { mb = r % p.m_blocks; nb = r / p.m_blocks; }   // m fastest: neighbours share the B tile
+  };
   const int units = tiles_per_batch * p.batch * p.ksplit;
   // split s of the reduction covers k-blocks [s * k_blocks / ksplit, (s + 1) * k_blocks / ksplit);
   // with k_mode the range is clipped to the non-zero part of triangular operands.
@@ -234,7 +242,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         const int t = u / p.ksplit;
         const int b = t / tiles_per_batch;
         const int r = t % tiles_per_batch;
-        const int mb = r % p.m_blocks, nb = r / p.m_blocks;   // m fastest: neighbours share the B tile
+        int mb, nb;
+        tile_of(r, mb, nb);
         if (p.tri_skip && mb > nb) continue;
         int k0, kb_per_split;
         k_range(split, mb, nb, k0, kb_per_split);
@@ -265,7 +274,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
         const int split = u % p.ksplit;
         const int rr = (u / p.ksplit) % tiles_per_batch;
-        const int mb = rr % p.m_blocks, nb = rr / p.m_blocks;
+        int mb, nb;
+        tile_of(rr, mb, nb);
         if (p.tri_skip && mb > nb) continue;
         int k0_unused, kb_per_split;
         k_range(split, mb, nb, k0_unused, kb_per_split);
@@ -308,7 +318,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       const int t = u / p.ksplit;
       const int b = t / tiles_per_batch;
       const int r = t % tiles_per_batch;
-      const int mb = r % p.m_blocks, nb = r / p.m_blocks;
+      int mb, nb;
+      tile_of(r, mb, nb);
       if (p.tri_skip && mb > nb) continue;
       const int row = mb * BLOCK_M + q * 32 + lane;
       const int64_t out_off = (int64_t)b * p.batch_stride + (int64_t)split * p.split_stride +

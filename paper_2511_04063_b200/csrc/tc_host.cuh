@@ -50,7 +50,7 @@ dq_status launch_gemm(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, cons
       return DQ_ERR_CUDA;
     attr_set = true;
   }
-  const int units = p.m_blocks * p.n_blocks * p.batch * p.ksplit;
+  const int units = (p.tile_list ? p.n_list : p.m_blocks * p.n_blocks) * p.batch * p.ksplit;
   int grid = units < ctx.sm_count ? units : ctx.sm_count;
   if (grid < 1) return DQ_OK;
   kern<<<grid, tc::NUM_THREADS, L::TOTAL, ctx.stream>>>(a, b, alo, blo, p);
@@ -70,6 +70,7 @@ struct Out {
   // split copy) to f32 + s * split_stride; the caller reduces.
   int ksplit = 1; int64_t split_stride = 0;
   int tri_skip = 0, k_mode = 0;   // triangular structure, see tc::Params
+  const int* tile_list = nullptr; int n_list = 0;   // explicit tile order (device), see tc::Params
 };
 
 // D[m][n] = alpha sum_k A[m][k] B[n][k] (+ beta D) with split-bf16 operands (three bf16 MMAs per
@@ -89,6 +90,7 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
   p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
   if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
   p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
+  p.tile_list = o.tile_list; p.n_list = o.n_list;
   return launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
 }
 

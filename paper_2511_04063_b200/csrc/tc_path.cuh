@@ -52,10 +52,18 @@ struct QrTcState {
   float* part = nullptr;                                // split partials of [S; W^T]
   int64_t part_bs = 0;                                  // elements per problem
   float* T = nullptr;                                   // [batch][128][128] compact-WY factor
+  // near-orthogonal iterative factorisation
+  __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T^T of U = I + T, kept from step to step (warm start)
+  bool t_warm = false;                                  // tw_* / the fp32 T belong to a nearby latent
+  // tile orders for triangular products (device arrays of mb | nb << 16)
+  int* tl_upper = nullptr; int n_upper = 0;             // tiles mb <= nb, largest mb first
+  int* tl_desc_nb = nullptr;                            // all tiles, largest nb first
+  int* tl_asc_nb = nullptr; int n_all = 0;              // all tiles, smallest nb first
 };
 dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count);
 void qr_tc_destroy(QrTcState& q);
-// iterative_iters > 0: U by the near-orthogonal fixed-point iteration instead of Householder.
+// iterative_iters > 0: U by the near-orthogonal fixed-point iteration instead of Householder
+// (iterative_iters sweeps from T = 0, or three sweeps from the previous step's T when q.t_warm).
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
                           int batch, int iterative_iters);
 dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch);
