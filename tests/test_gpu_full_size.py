@@ -25,10 +25,14 @@ def perturbed_latent(w, Z0, seed):
     return (Z0 + np.float32(0.02 / np.sqrt(w.d)) * noise).astype(np.float32)
 
 
-@pytest.mark.parametrize("name", ["c1_tiny", "c2_7b", "c3_heads", "c4_13b", "c5_70b"])
-def test_one_step_at_full_size(name):
+@pytest.mark.parametrize("name,qr", [("c1_tiny", "householder"), ("c2_7b", "householder"), ("c2_7b", "iterative"),
+                                     ("c3_heads", "householder"), ("c4_13b", "householder"), ("c4_13b", "iterative"),
+                                     ("c5_70b", "householder"), ("c5_70b", "iterative")])
+def test_one_step_at_full_size(name, qr):
     w = gen.WORKLOADS[name]
     c = Calib(w)
+    if qr == "iterative":
+        dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_ITERATIVE, 8)
     Z = perturbed_latent(w, c.Z0_host, w.seed)
     c.set_latent(Z)
     loss = c.step(1)[0]
@@ -58,8 +62,8 @@ def test_one_step_at_full_size(name):
         assert np.abs(R_used[b].T @ R_used[b] - np.eye(w.d)).max() <= ORTHO_TOL
         Rn_ref, _ = orc.qr_pos_lapack(ref["Z_new"])
         err_next = np.abs(R_next[b] - Rn_ref).max()
-        print("%s[%d]: loss %.6f ref %.6f, |R-Rref| %.2e, |Rnext-ref| %.2e" %
-              (name, b, loss[b], ref["loss"], np.abs(R_used[b] - ref["R"]).max(), err_next))
+        print("%s/%s[%d]: loss %.6f ref %.6f, |R-Rref| %.2e, |Rnext-ref| %.2e" %
+              (name, qr, b, loss[b], ref["loss"], np.abs(R_used[b] - ref["R"]).max(), err_next))
         assert err_next <= R_TOL
         assert np.abs(R_next[b].T @ R_next[b] - np.eye(w.d)).max() <= ORTHO_TOL
         if w.path == "fp32":
