@@ -34,6 +34,25 @@ __global__ void __launch_bounds__(256) transpose_f32_to_bf16_kernel(const float*
   for (int c = ty; c < 32; c += 8) out[(int64_t)(c0 + c) * d + r0 + tx] = __float2bfloat16_rn(t[tx][c]);
 }
 
+// out tile = sum over slices of part[slice] tile, for the tiles of `list` (mb | nb << 16; tiles
+// are 128 x bn); one CTA per tile, fixed summation order.
+__global__ void __launch_bounds__(256) tile_reduce_kernel(const float* __restrict__ part, int slices,
+                                                          int64_t slice_stride, const int* __restrict__ list, int bn,
+                                                          int d, float* __restrict__ out) {
+  const int code = list[blockIdx.x];
+  const int r0 = (code & 0xffff) * 128, c0 = (code >> 16) * bn;
+  const int per_row = bn / 4;
+  for (int e = threadIdx.x; e < 128 * per_row; e += 256) {
+    const int64_t idx = (int64_t)(r0 + e / per_row) * d + c0 + (e % per_row) * 4;
+    float4 s = *reinterpret_cast<const float4*>(part + idx);
+    for (int k = 1; k < slices; ++k) {
+      const float4 t = *reinterpret_cast<const float4*>(part + (int64_t)k * slice_stride + idx);
+      s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+    }
+    *reinterpret_cast<float4*>(out + idx) = s;
+  }
+}
+
 struct Maps {
   CUtensorMap rt, x, xt, gt128, gt256;
 };
@@ -62,6 +81,24 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   if (ks > 1 &&
       cudaMalloc((void**)&tc.part, sizeof(float) * (size_t)batch * ks * d * d) != cudaSuccess)
     return DQ_ERR_ALLOC;
+  if (ks == 1 && batch == 1 && tiles > ctx.sm_count && tiles % ctx.sm_count != 0) {
+    // a partly filled last wave: split its reduction so that it fills the machine once more
+    const int rem = tiles % ctx.sm_count, full = tiles - rem, mbk = d / tc::BLOCK_M;
+    int sp = ctx.sm_count / rem;
+    if (sp > 4) sp = 4;
+    while (sp > 1 && (N / tc::BLOCK_K) / sp < 16) --sp;
+    if (sp > 1) {
+      std::vector<int> head(full), tail(rem);
+      for (int r = 0; r < tiles; ++r) (r < full ? head[r] : tail[r - full]) = (r % mbk) | ((r / mbk) << 16);
+      tc.n_head = full; tc.n_tail = rem; tc.tail_split = sp;
+      if (cudaMalloc((void**)&tc.tl_head, sizeof(int) * full) != cudaSuccess ||
+          cudaMalloc((void**)&tc.tl_tail, sizeof(int) * rem) != cudaSuccess ||
+          cudaMalloc((void**)&tc.tail_part, sizeof(float) * (size_t)sp * d * d) != cudaSuccess)
+        return DQ_ERR_ALLOC;
+      DQ_CHECK_CUDA(cudaMemcpy(tc.tl_head, head.data(), sizeof(int) * full, cudaMemcpyHostToDevice));
+      DQ_CHECK_CUDA(cudaMemcpy(tc.tl_tail, tail.data(), sizeof(int) * rem, cudaMemcpyHostToDevice));
+    }
+  }
   Maps* m = new (std::nothrow) Maps();
   if (!m) return DQ_ERR_ALLOC;
   tc.maps = m;
@@ -86,6 +123,7 @@ dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx) {
 
 void tc_destroy(TcState& tc) {
   cudaFree(tc.Xt); if (!tc.rt_external) cudaFree(tc.Rt); cudaFree(tc.part);
+  cudaFree(tc.tl_head); cudaFree(tc.tl_tail); cudaFree(tc.tail_part);
   delete reinterpret_cast<Maps*>(tc.maps);
   tc = TcState();
 }
@@ -117,8 +155,23 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
   } else {
     p.out = tc.part; p.batch_stride = (int64_t)tc.ksplit * d * d; p.split_stride = (int64_t)d * d;
   }
-  if (bn == 256) DQ_CHECK((tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, m->xt, m->gt256, m->xt, m->gt256, p)));
-  else DQ_CHECK((tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, p)));
+  auto launch = [&](const tc::Params& pp) {
+    return (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, m->xt, m->gt256, m->xt, m->gt256, pp)
+                       : tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, pp);
+  };
+  if (tc.tail_split > 1) {
+    tc::Params ph = p;      // full waves: whole reduction per tile
+    ph.tile_list = tc.tl_head; ph.n_list = tc.n_head;
+    DQ_CHECK(launch(ph));
+    tc::Params pt = p;      // last wave: reduction in slices, then a fixed-order sum
+    pt.tile_list = tc.tl_tail; pt.n_list = tc.n_tail; pt.ksplit = tc.tail_split;
+    pt.out = tc.tail_part; pt.batch_stride = 0; pt.split_stride = (int64_t)d * d;
+    DQ_CHECK(launch(pt));
+    tile_reduce_kernel<<<tc.n_tail, 256, 0, ctx.stream>>>(tc.tail_part, tc.tail_split, (int64_t)d * d, tc.tl_tail, bn,
+                                                          d, Gq);
+    return after_launch(ctx);
+  }
+  DQ_CHECK(launch(p));
   if (tc.ksplit > 1) DQ_CHECK(splitk_reduce(ctx, tc.part, tc.ksplit, (int64_t)d * d, tc.batch, 1.f, 0.f, Gq));
   return DQ_OK;
 }

@@ -17,6 +17,12 @@ struct TcState {
   int ksplit = 1;
   void* maps = nullptr;               // host array of CUtensorMap
   int n_partials = 0;
+  // Gq = X^T G when the tile count is not a multiple of the SM count: the last, partly filled
+  // wave of tiles is computed with its reduction split in `tail_split` slices instead
+  int* tl_head = nullptr; int n_head = 0;
+  int* tl_tail = nullptr; int n_tail = 0;
+  int tail_split = 1;
+  float* tail_part = nullptr;         // [tail_split][d][d] (only the tail tiles are touched)
 };
 
 dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void* d_X,

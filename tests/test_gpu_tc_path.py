@@ -25,6 +25,7 @@ CASES = [
     small("c4_13b", d=640, n_tokens=512, batch=2, n_outlier_channels=4),    # 128-wide N tiles, 2 problems
     small("c3_heads", d=128, n_tokens=2048, batch=4),                       # per-head rotations
     small("c5_70b", d=512, n_tokens=4096, n_outlier_channels=2),            # token scales, several waves
+    small("c4_13b", d=2560, n_tokens=2048, n_outlier_channels=6),           # 200 Gq tiles on 148 SMs: split tail wave
 ]
 
 
@@ -46,7 +47,8 @@ def test_tensor_core_step_every_stage(w):
         # band of the kink of Eq. 4 the sign decision is the kernel's.
         row_norm = np.linalg.norm(X, axis=1)
         dO = 8.0 * row_norm / np.sqrt(d) * 2.0 ** -9 + 1e-3
-        ref = orc.calib_step(X, Z0[b], w.lr, sign_decider=sign_decider_from_gpu(Gt[b].T, 2.0 * dO[:, None]))
+        ref = orc.calib_step(X, Z0[b], w.lr, sign_decider=sign_decider_from_gpu(Gt[b].T, 2.0 * dO[:, None]),
+                             qr=orc.qr_pos if d <= 1024 else orc.qr_pos_lapack)
         assert abs(loss[b] - ref["loss"]) <= LOSS_TOL_BF16 * ref["loss"]
         assert np.abs(R[b] - ref["R"]).max() <= 2e-5
         # dL/dO (no 1/N), stored channel-major; compare where |O| is clear of the kink at 0.
