@@ -45,7 +45,7 @@ typedef enum {
 enum { DQ_FP32 = 0, DQ_BF16 = 1 };             /* x_dtype                       */
 enum { DQ_PATH_FP32 = 0, DQ_PATH_BF16_TC = 1 }; /* arithmetic of the X R / X^T G contractions */
 enum { DQ_MEAN_TOKENS = 0, DQ_SUM_TOKENS = 1 }; /* reduction of Eq. 4 over token rows */
-enum { DQ_SGD = 0 };                           /* optimiser (Algorithm 1 line 10) */
+enum { DQ_SGD = 0 };                           /* optimiser (Algorithm 1, update step) */
 
 typedef struct {
   int32_t d;         /* channels = size of the rotation; multiple of 32 (fp32 path) or 128 (tensor-core path); <= 8192 */
@@ -54,13 +54,13 @@ typedef struct {
   int32_t x_dtype;   /* DQ_FP32 | DQ_BF16                                       */
   int32_t path;      /* DQ_PATH_FP32: fp32 FMA contractions (needs DQ_FP32 X);
                         DQ_PATH_BF16_TC: bf16 tensor-core contractions with fp32 accumulation (needs DQ_BF16 X) */
-  int32_t reduction; /* DQ_MEAN_TOKENS (default reading of Algorithm 1 line 9) | DQ_SUM_TOKENS */
+  int32_t reduction; /* DQ_MEAN_TOKENS (default reading of Algorithm 1's loss step) | DQ_SUM_TOKENS */
   int32_t optimizer; /* DQ_SGD                                                  */
   float lr;          /* eta                                                     */
   int64_t ldx;       /* row stride of X in elements (>= d); problems are n_tokens*ldx apart */
 } dq_calib_config;
 
-/* Algorithm 1 lines 3-5 hand-off: bind calibration activations and the initial
+/* Algorithm 1, hand-off before the loop: bind calibration activations and the initial
  * latent.  d_X is BORROWED (must outlive the handle, is never written).  d_Z0
  * ([batch][d][d] fp32) is COPIED.  cuda_stream is a cudaStream_t (NULL = legacy
  * default stream).  Allocates every workspace the step needs.
@@ -68,7 +68,7 @@ typedef struct {
 dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void* d_X,
                         const float* d_Z0, void* cuda_stream);
 
-/* Algorithm 1 lines 6-11, exactly n_steps iterations.  d_loss_out (nullable) is a
+/* Algorithm 1's loop, exactly n_steps iterations.  d_loss_out (nullable) is a
  * device array [n_steps][batch] fp32; entry k is L(Z_k), the loss BEFORE the
  * k-th update.  No host synchronisation. */
 dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out);
@@ -124,7 +124,7 @@ dq_status dq_calib_refresh_inputs(dq_calib_t* h);
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 
-/* Checkpoint / resume of the optimised parameter (Algorithm 1 line 5: Z <- Z0). */
+/* Checkpoint / resume of the optimised parameter (Algorithm 1: Z <- Z0). */
 dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out);
 dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z);
 

@@ -6,6 +6,6 @@ It shares no code with the CUDA path.
 """
 from .calib_oracle import (  # noqa: F401
     whip_per_token, whip_loss, whip_grad_wrt_output, householder_qr_alg2,
-    qr_pos, qr_pos_lapack, rotate, grad_wrt_rotation, qr_backward, sgd_step,
+    qr_pos, qr_pos_lapack, rotate, grad_wrt_rotation, qr_backward, sgd_step, momentum_step, adam_step,
     calib_step, calib_run, widen_input,
 )

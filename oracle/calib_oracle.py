@@ -13,13 +13,13 @@ calls them Q and R).  O = X R.  G = dL/dO.  Gq = dL/dR.  Gz = dL/dZ.
 
 Readings taken where the paper is silent (each is also listed in the design
 notes of the repository):
-  * Whip of a matrix (Algorithm 1 line 9) = mean over tokens of Eq. 4 applied
+  * Whip of a matrix (Algorithm 1, the loss of the rotated activations) = mean over tokens of Eq. 4 applied
     to each token row; "sum" keeps the plain sum over tokens.
   * d|o|/do at o = 0 is taken as 0.
   * The rotation reported is the unique factor with diag(U) > 0; Algorithm 2's
     own sign rule yields the same R up to column signs, which change neither
     the loss nor dL/dZ.
-  * Algorithm 2 line 9 as printed touches only Q[k:n, k:n]; the accumulated
+  * Algorithm 2's update of Q as printed touches only Q[k:n, k:n]; the accumulated
     product of reflectors needs the full rows k:n, which is what is done here.
   * Plain SGD: no momentum, no weight decay, constant learning rate.
 """
@@ -45,7 +45,7 @@ def whip_per_token(O: np.ndarray) -> np.ndarray:
 
 
 def whip_loss(O: np.ndarray, reduction: str = "mean") -> float:
-    """Algorithm 1 line 9: Whip of the rotated activation matrix."""
+    """Algorithm 1 (loss step): Whip of the rotated activation matrix."""
     per_tok = whip_per_token(O)
     if reduction == "mean":
         return float(per_tok.sum() / per_tok.shape[0])
@@ -124,7 +124,7 @@ def qr_pos_lapack(Z: np.ndarray):
 # Rotation, back-propagation, optimiser
 # ----------------------------------------------------------------------------
 def rotate(X: np.ndarray, R: np.ndarray) -> np.ndarray:
-    """Algorithm 1 line 8: O = X @ R (tokens are rows)."""
+    """Algorithm 1 (rotation step): O = X @ R (tokens are rows)."""
     return widen_input(X) @ np.asarray(R, dtype=F64)
 
 
@@ -134,7 +134,7 @@ def grad_wrt_rotation(X: np.ndarray, G: np.ndarray) -> np.ndarray:
 
 
 def qr_backward(R: np.ndarray, U: np.ndarray, Gq: np.ndarray) -> np.ndarray:
-    """dL/dZ given dL/dR, for Z = R U (Algorithm 1 line 10 by the chain rule).
+    """dL/dZ given dL/dR, for Z = R U (Algorithm 1, update step, by the chain rule).
 
     dZ = dR U + R dU.  With A = R^T dZ U^-1 = Omega + dU U^-1, Omega = R^T dR
     skew and dU U^-1 upper triangular, Omega is fixed by the strictly lower part
@@ -151,13 +151,34 @@ def qr_backward(R: np.ndarray, U: np.ndarray, Gq: np.ndarray) -> np.ndarray:
 
 
 def sgd_step(Z: np.ndarray, Gz: np.ndarray, lr: float) -> np.ndarray:
-    """Algorithm 1 line 10: Z <- Z - eta dL/dZ."""
+    """Algorithm 1 (update step): Z <- Z - eta dL/dZ."""
     return np.asarray(Z, dtype=F64) - lr * np.asarray(Gz, dtype=F64)
+
+
+def momentum_step(Z: np.ndarray, Gz: np.ndarray, velocity: np.ndarray, lr: float, momentum: float):
+    """SGD with (heavy-ball) momentum on the latent: the paper optimises Z with a standard
+    optimiser (Sec. 4.3, "SGD or Adam").  v <- mu v + g;  Z <- Z - eta v.  Returns (Z, v)."""
+    v = momentum * np.asarray(velocity, dtype=F64) + np.asarray(Gz, dtype=F64)
+    return np.asarray(Z, dtype=F64) - lr * v, v
+
+
+def adam_step(Z: np.ndarray, Gz: np.ndarray, m: np.ndarray, v: np.ndarray, t: int, lr: float,
+              beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8):
+    """Adam on the latent (Sec. 4.3 / the optimiser comparison table use it unchanged), in its
+    published form: m <- b1 m + (1 - b1) g;  v <- b2 v + (1 - b2) g^2;  bias-corrected
+    mhat = m / (1 - b1^t), vhat = v / (1 - b2^t);  Z <- Z - eta mhat / (sqrt(vhat) + eps).
+    t is the 1-based index of this step.  Returns (Z, m, v)."""
+    g = np.asarray(Gz, dtype=F64)
+    m = beta1 * np.asarray(m, dtype=F64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, dtype=F64) + (1.0 - beta2) * g * g
+    mhat = m / (1.0 - beta1 ** t)
+    vhat = v / (1.0 - beta2 ** t)
+    return np.asarray(Z, dtype=F64) - lr * mhat / (np.sqrt(vhat) + eps), m, v
 
 
 def calib_step(X: np.ndarray, Z: np.ndarray, lr: float, reduction: str = "mean",
                qr=qr_pos, sign_decider=None):
-    """One pass of the loop body of Algorithm 1 (lines 7-10).
+    """One pass of the loop body of Algorithm 1.
 
     Returns a dict with every intermediate so that tests can compare each stage.
     The loss is L(Z) before the update.  sign_decider(O) -> sign array lets a
@@ -177,7 +198,7 @@ def calib_step(X: np.ndarray, Z: np.ndarray, lr: float, reduction: str = "mean",
 
 def calib_run(X: np.ndarray, Z0: np.ndarray, lr: float, n_steps: int,
               reduction: str = "mean", qr=qr_pos):
-    """Algorithm 1 lines 5-11 for exactly n_steps iterations.
+    """Algorithm 1's loop for exactly n_steps iterations.
 
     Returns (losses[n_steps], Z_final, R_final) with R_final the rotation of the
     final latent (one more QR, not the rotation used by the last step).

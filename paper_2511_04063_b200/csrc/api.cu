@@ -120,7 +120,7 @@ dq_status ensure_rotation(dq_calib* h) {
   return DQ_OK;
 }
 
-// One iteration of Algorithm 1 (lines 7-10) enqueued on the work stream.
+// One iteration of Algorithm 1's loop body enqueued on the work stream.
 dq_status enqueue_step(dq_calib* h, bool timed) {
   const dq_calib_config& c = h->cfg;
   const int d = c.d, batch = c.batch;

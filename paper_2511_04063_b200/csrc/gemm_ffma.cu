@@ -210,7 +210,7 @@ dq_status loss_finalize(Ctx& ctx, const float* partials, int n_per_problem, int 
   return after_launch(ctx);
 }
 
-// Algorithm 1 line 10.  n is a multiple of 4 (d is a multiple of 32).
+// Algorithm 1 (update step).  n is a multiple of 4 (d is a multiple of 32).
 dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n) {
   const int64_t n4 = n / 4;
   int blocks = (int)((n4 + 255) / 256);

@@ -5,7 +5,7 @@
 //                              W = U^-1 (blocked inversion), R = Z W; also bf16(R^T) for the
 //                              tensor-core contraction.
 //   qr128_backward_sgd_kernel  B = R^T Gq, S = tril(B - B^T, -1), Gz = (R S) W^T,
-//                              Z <- Z - lr Gz  (Algorithm 1 line 10), all in one launch.
+//                              Z <- Z - lr Gz  (Algorithm 1, update step), all in one launch.
 // fp32 FMA arithmetic throughout; sums run in a fixed order (bit-reproducible).
 #include "common.cuh"
 

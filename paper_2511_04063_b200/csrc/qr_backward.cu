@@ -1,5 +1,5 @@
 // QR-Orth backward: Gz = R tril(B - B^T, -1) U^-T with B = R^T Gq, the gradient of
-// the latent for Z = R U (chain rule of Algorithm 1 line 10 through Sec. 4.3).
+// the latent for Z = R U (chain rule of Algorithm 1's update step through Sec. 4.3).
 // U^-1 is formed explicitly: 64 x 64 diagonal blocks by back-substitution, then
 // block merges  inv([U11 U12; 0 U22]) = [W11, -W11 U12 W22; 0, W22]  as GEMMs.
 #include "common.cuh"

@@ -267,3 +267,40 @@ def test_c1_trajectory_matches_stored_fixture():
     Z0 = gen.gen_latent_init(w)[0]
     losses, Z, R = orc.calib_run(X, Z0, w.lr, 3, qr=orc.qr_pos)
     assert np.allclose(losses, ref["losses"][:3], rtol=1e-12)
+
+
+# --------------------------------------------------------------------- optimisers on the latent
+def test_momentum_zero_is_plain_sgd_and_constant_gradient_gives_geometric_series():
+    rng = np.random.default_rng(1)
+    Z, g = rng.standard_normal((5, 5)), rng.standard_normal((5, 5))
+    Z1, v1 = orc.momentum_step(Z, g, np.zeros_like(Z), 0.1, 0.0)
+    assert np.array_equal(Z1, orc.sgd_step(Z, g, 0.1)) and np.array_equal(v1, g)
+    mu, lr, Zk, v = 0.9, 0.05, Z.copy(), np.zeros_like(Z)
+    for k in range(1, 8):
+        Zk, v = orc.momentum_step(Zk, g, v, lr, mu)
+        assert np.allclose(v, g * (1 - mu ** k) / (1 - mu), rtol=1e-13)          # closed form of the velocity
+    total = sum((1 - mu ** k) / (1 - mu) for k in range(1, 8))
+    assert np.allclose(Zk, Z - lr * total * g, rtol=1e-12, atol=1e-14)
+
+
+def test_adam_first_step_is_lr_times_sign_and_is_scale_free():
+    rng = np.random.default_rng(2)
+    Z, g = rng.standard_normal((6, 6)), rng.standard_normal((6, 6))
+    zeros = np.zeros_like(Z)
+    Z1, m1, v1 = orc.adam_step(Z, g, zeros, zeros, 1, 1e-2, eps=0.0)
+    assert np.allclose(Z1, Z - 1e-2 * np.sign(g), rtol=0, atol=1e-15)            # mhat / sqrt(vhat) = g / |g|
+    assert np.allclose(m1, 0.1 * g) and np.allclose(v1, 1e-3 * g * g)
+    Za, _, _ = orc.adam_step(Z, 1000.0 * g, zeros, zeros, 1, 1e-2, eps=0.0)
+    assert np.allclose(Za, Z1, atol=1e-14)                                       # invariant to gradient scale
+    # a constant gradient keeps every step at exactly lr: bias correction cancels the warm-up
+    Zk, m, v = Z.copy(), zeros, zeros
+    for t in range(1, 6):
+        Zn, m, v = orc.adam_step(Zk, g, m, v, t, 1e-2, eps=0.0)
+        assert np.allclose(Zn - Zk, -1e-2 * np.sign(g), atol=1e-14)
+        Zk = Zn
+
+
+def test_adam_epsilon_bounds_the_step_for_tiny_gradients():
+    Z, g = np.zeros((2, 2)), np.full((2, 2), 1e-12)
+    Z1, _, _ = orc.adam_step(Z, g, np.zeros_like(Z), np.zeros_like(Z), 1, 1.0, eps=1e-8)
+    assert np.allclose(Z1, -1e-12 / (1e-12 + 1e-8))                              # |step| = lr g / (|g| + eps)
