@@ -45,7 +45,7 @@ typedef enum {
 enum { DQ_FP32 = 0, DQ_BF16 = 1 };             /* x_dtype                       */
 enum { DQ_PATH_FP32 = 0, DQ_PATH_BF16_TC = 1 }; /* arithmetic of the X R / X^T G contractions */
 enum { DQ_MEAN_TOKENS = 0, DQ_SUM_TOKENS = 1 }; /* reduction of Eq. 4 over token rows */
-enum { DQ_SGD = 0 };                           /* optimiser (Algorithm 1, update step) */
+enum { DQ_SGD = 0, DQ_SGD_MOMENTUM = 1, DQ_ADAM = 2 }; /* optimiser (Algorithm 1, update step; Sec. 4.3: "SGD or Adam") */
 
 typedef struct {
   int32_t d;         /* channels = size of the rotation; multiple of 32 (fp32 path) or 128 (tensor-core path); <= 8192 */
@@ -55,7 +55,7 @@ typedef struct {
   int32_t path;      /* DQ_PATH_FP32: fp32 FMA contractions (needs DQ_FP32 X);
                         DQ_PATH_BF16_TC: bf16 tensor-core contractions with fp32 accumulation (needs DQ_BF16 X) */
   int32_t reduction; /* DQ_MEAN_TOKENS (default reading of Algorithm 1's loss step) | DQ_SUM_TOKENS */
-  int32_t optimizer; /* DQ_SGD                                                  */
+  int32_t optimizer; /* DQ_SGD here; others via dq_calib_set_optimizer          */
   float lr;          /* eta                                                     */
   int64_t ldx;       /* row stride of X in elements (>= d); problems are n_tokens*ldx apart */
 } dq_calib_config;
@@ -110,6 +110,15 @@ dq_status dq_rotate_apply_static(const void* d_X, int64_t n, int32_t d, int64_t 
  * the fp32 path. */
 dq_status dq_calib_refresh_inputs(dq_calib_t* h);
 
+/* Optimiser of the latent (Sec. 4.3: QR-Orth works with any standard optimiser; the paper reports
+ * SGD and Adam).  Resets the optimiser state (moments, step count) and replaces the learning rate.
+ *   DQ_SGD:          Z <- Z - lr g                                   (beta1, beta2, eps ignored)
+ *   DQ_SGD_MOMENTUM: v <- beta1 v + g;  Z <- Z - lr v                 (beta1 = momentum)
+ *   DQ_ADAM:         m <- beta1 m + (1 - beta1) g;  v <- beta2 v + (1 - beta2) g^2;
+ *                    Z <- Z - lr (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps)
+ * Errors: INVALID_ARG (bad enum, betas outside [0, 1), eps < 0), ALLOC, CUDA. */
+dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, float beta1, float beta2, float eps);
+
 /* How the QR-Orth forward (Sec. 4.3: Z = R U) is computed on the tensor-core path.  Both
  * give the same unique factors (diag(U) > 0).
  *   DQ_QR_HOUSEHOLDER (default): blocked Householder QR (Algorithm 2 in compact-WY form), valid
@@ -157,7 +166,9 @@ enum {
   DQ_BUF_G = 4,        /* dL/dO without the 1/N factor: fp32 [batch][N][d] (fp32 path)
                           or bf16 channel-major [batch][d][N] (tensor-core path)   */
   DQ_BUF_PARTIALS = 5, /* fp32 per-tile loss partial sums of the last step         */
-  DQ_BUF_Z = 6         /* fp32 [batch][d][d]  current latent                       */
+  DQ_BUF_Z = 6,        /* fp32 [batch][d][d]  current latent                       */
+  DQ_BUF_OPT_M = 7,    /* fp32 [batch][d][d]  first moment / velocity (NULL for DQ_SGD)  */
+  DQ_BUF_OPT_V = 8     /* fp32 [batch][d][d]  second moment (DQ_ADAM only)         */
 };
 dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int64_t* n_elems);
 

@@ -18,15 +18,15 @@ DQ_QR_HOUSEHOLDER, DQ_QR_ITERATIVE = 0, 1
 DQ_FP32, DQ_BF16 = 0, 1
 DQ_PATH_FP32, DQ_PATH_BF16_TC = 0, 1
 DQ_MEAN_TOKENS, DQ_SUM_TOKENS = 0, 1
-DQ_SGD = 0
+DQ_SGD, DQ_SGD_MOMENTUM, DQ_ADAM = 0, 1, 2
 DQ_PHASE_NAMES = ("qr_forward", "rotate_whip", "grad_rotation", "qr_backward", "update")
-DQ_BUF_R, DQ_BUF_U, DQ_BUF_GQ, DQ_BUF_GZ, DQ_BUF_G, DQ_BUF_PARTIALS, DQ_BUF_Z = range(7)
+DQ_BUF_R, DQ_BUF_U, DQ_BUF_GQ, DQ_BUF_GZ, DQ_BUF_G, DQ_BUF_PARTIALS, DQ_BUF_Z, DQ_BUF_OPT_M, DQ_BUF_OPT_V = range(9)
 
 EXPORTED_SYMBOLS = (
     "dq_calib_init", "dq_calib_step", "dq_calib_get_rotation", "dq_rotate_apply",
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
-    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method",
+    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer",
 )
 
 
@@ -61,6 +61,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_rotate_apply.argtypes = [vp, i32, i64, i32, i64, vp, vp, i64, vp]
     lib.dq_rotate_apply_static.argtypes = [vp, i64, i32, i64, vp, vp, i64, vp]
     lib.dq_rotate_apply_static.restype = i32
+    lib.dq_calib_set_optimizer.argtypes = [vp, i32, C.c_float, C.c_float, C.c_float, C.c_float]
+    lib.dq_calib_set_optimizer.restype = i32
     lib.dq_calib_set_qr_method.argtypes = [vp, i32, i32]
     lib.dq_calib_set_qr_method.restype = i32
     lib.dq_calib_get_latent.argtypes = [vp, vp]
@@ -151,6 +153,10 @@ def dq_calib_status(h) -> int:
 
 def dq_calib_set_timing(h, enabled: bool):
     _check(load_library().dq_calib_set_timing(h, int(enabled)), "dq_calib_set_timing")
+
+
+def dq_calib_set_optimizer(h, optimizer: int, lr: float, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8):
+    _check(load_library().dq_calib_set_optimizer(h, optimizer, lr, beta1, beta2, eps), "dq_calib_set_optimizer")
 
 
 def dq_calib_set_qr_method(h, method: int, n_iters: int = 0):

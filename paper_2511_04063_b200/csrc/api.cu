@@ -36,6 +36,11 @@ struct dq_calib {
   QrTcState qtc;                // tensor-core QR-Orth operand copies
   bool fast_qr = false;
   int qr_method = DQ_QR_HOUSEHOLDER, qr_iters = 8;
+  int optimizer = DQ_SGD;
+  float beta1 = 0.f, beta2 = 0.f, eps = 0.f;
+  float* opt_m = nullptr;       // first moment / velocity
+  float* opt_v = nullptr;       // second moment
+  float* opt_pw = nullptr;      // device float[2]: beta1^t, beta2^t
   bool small128 = false;        // d == 128: shared-memory-resident batched QR-Orth
   bool r_stale = true;
   bool timing = false;
@@ -64,6 +69,7 @@ void free_all(dq_calib* h) {
   tc_destroy(h->tc);
   qr_tc_destroy(h->qtc);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
+  cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw);
   cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->ctx.d_status);
   cudaFree(h->ws.A); cudaFree(h->ws.V); cudaFree(h->ws.T); cudaFree(h->ws.W); cudaFree(h->ws.W2);
   cudaFree(h->ws.Q); cudaFree(h->ws.Winv); cudaFree(h->ws.B); cudaFree(h->ws.S); cudaFree(h->ws.tmp);
@@ -160,15 +166,20 @@ dq_status enqueue_step(dq_calib* h, bool timed) {
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[3], ctx.stream));
   // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
   // (a7) Z <- Z - lr Gz  (fused into the backward kernel for 128 x 128 latents)
-  if (h->small128) {
-    DQ_CHECK(qr128_backward_sgd(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, c.lr, batch));
+  const int64_t n_latent = (int64_t)d * d * batch;
+  if (h->small128) {   // plain SGD is fused into the backward kernel; other optimisers follow it
+    DQ_CHECK(qr128_backward_sgd(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, h->optimizer == DQ_SGD ? c.lr : 0.f, batch));
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
   } else {
     if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch));
     else DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch));
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
-    DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, (int64_t)d * d * batch));
+    if (h->optimizer == DQ_SGD) DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, n_latent));
   }
+  if (h->optimizer == DQ_SGD_MOMENTUM)
+    DQ_CHECK(momentum_update(ctx, h->Z, h->Gz, h->opt_m, c.lr, h->beta1, n_latent));
+  else if (h->optimizer == DQ_ADAM)
+    DQ_CHECK(adam_update(ctx, h->Z, h->Gz, h->opt_m, h->opt_v, h->opt_pw, c.lr, h->beta1, h->beta2, h->eps, n_latent));
   h->r_stale = true;
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[5], ctx.stream));
   return DQ_OK;
@@ -380,6 +391,31 @@ dq_status dq_calib_status(dq_calib_t* h) {
   return (dq_status)code;
 }
 
+dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, float beta1, float beta2, float eps) {
+  if (!h || !(lr == lr)) return DQ_ERR_INVALID_ARG;
+  if (optimizer != DQ_SGD && optimizer != DQ_SGD_MOMENTUM && optimizer != DQ_ADAM) return DQ_ERR_INVALID_ARG;
+  if (optimizer != DQ_SGD && !(beta1 >= 0.f && beta1 < 1.f)) return DQ_ERR_INVALID_ARG;
+  if (optimizer == DQ_ADAM && (!(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f))) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
+  const int64_t dd = (int64_t)h->cfg.d * h->cfg.d * h->cfg.batch;
+  if (optimizer != DQ_SGD && !h->opt_m) DQ_CHECK(dev_alloc(&h->opt_m, dd));
+  if (optimizer == DQ_ADAM && !h->opt_v) DQ_CHECK(dev_alloc(&h->opt_v, dd));
+  if (optimizer == DQ_ADAM && !h->opt_pw) DQ_CHECK(dev_alloc(&h->opt_pw, 2));
+  if (h->opt_m) DQ_CHECK_CUDA(cudaMemsetAsync(h->opt_m, 0, sizeof(float) * dd, h->ctx.stream));
+  if (h->opt_v) DQ_CHECK_CUDA(cudaMemsetAsync(h->opt_v, 0, sizeof(float) * dd, h->ctx.stream));
+  if (h->opt_pw) {
+    const float ones[2] = {1.f, 1.f};
+    DQ_CHECK_CUDA(cudaMemcpyAsync(h->opt_pw, ones, sizeof(ones), cudaMemcpyHostToDevice, h->ctx.stream));
+    DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
+  }
+  h->optimizer = optimizer;
+  h->cfg.lr = lr;
+  h->beta1 = beta1; h->beta2 = beta2; h->eps = eps;
+  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
+  h->graph_failed = false;
+  return DQ_OK;
+}
+
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters) {
   if (!h || (method != DQ_QR_HOUSEHOLDER && method != DQ_QR_ITERATIVE) || n_iters > 64) return DQ_ERR_INVALID_ARG;
   const int iters = n_iters <= 0 ? 8 : n_iters;
@@ -418,6 +454,8 @@ dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int6
     case DQ_BUF_G: *d_ptr = h->G; *n_elems = h->g_elems; break;
     case DQ_BUF_PARTIALS: *d_ptr = h->partials; *n_elems = (int64_t)h->n_partials * h->cfg.batch; break;
     case DQ_BUF_Z: *d_ptr = h->Z; *n_elems = dd; break;
+    case DQ_BUF_OPT_M: *d_ptr = h->opt_m; *n_elems = h->opt_m ? dd : 0; break;
+    case DQ_BUF_OPT_V: *d_ptr = h->opt_v; *n_elems = h->opt_v ? dd : 0; break;
     default: return DQ_ERR_INVALID_ARG;
   }
   return DQ_OK;

@@ -105,5 +105,10 @@ dq_status qr128_backward_sgd(Ctx& ctx, const float* R, const float* W, const flo
 
 // Z <- Z - lr Gz  (n elements)
 dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n);
+// v <- mu v + Gz; Z <- Z - lr v
+dq_status momentum_update(Ctx& ctx, float* Z, const float* Gz, float* V, float lr, float mu, int64_t n);
+// Adam with bias correction; pw = device float[2] {beta1^t, beta2^t}, advanced on the device
+dq_status adam_update(Ctx& ctx, float* Z, const float* Gz, float* M, float* V, float* pw, float lr, float b1,
+                      float b2, float eps, int64_t n);
 
 }  // namespace dq

@@ -201,6 +201,53 @@ __global__ void sgd_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz
     Z[i] = z;
   }
 }
+
+// v <- mu v + g;  Z <- Z - lr v
+__global__ void momentum_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz, float4* __restrict__ V,
+                                float lr, float mu, int64_t n4) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    float4 z = Z[i], v = V[i];
+    const float4 g = Gz[i];
+    v.x = fmaf(mu, v.x, g.x); v.y = fmaf(mu, v.y, g.y); v.z = fmaf(mu, v.z, g.z); v.w = fmaf(mu, v.w, g.w);
+    z.x = fmaf(-lr, v.x, z.x); z.y = fmaf(-lr, v.y, z.y); z.z = fmaf(-lr, v.z, z.z); z.w = fmaf(-lr, v.w, z.w);
+    V[i] = v;
+    Z[i] = z;
+  }
+}
+
+// pw[0] = beta1^t, pw[1] = beta2^t of the step about to be taken (t counted on the device so that a
+// replayed CUDA graph advances it)
+__global__ void adam_advance_kernel(float* pw, float beta1, float beta2) {
+  pw[0] *= beta1;
+  pw[1] *= beta2;
+}
+
+__device__ __forceinline__ float adam_one(float& z, float g, float& m, float& v, float b1, float b2, float c1,
+                                          float c2, float lr, float eps) {
+  m = fmaf(b1, m, (1.f - b1) * g);
+  v = fmaf(b2, v, (1.f - b2) * g * g);
+  const float mhat = m * c1, vhat = v * c2;
+  z -= lr * mhat / (sqrtf(vhat) + eps);
+  return z;
+}
+
+// Adam in its published form with bias correction; c1 = 1 / (1 - beta1^t), c2 = 1 / (1 - beta2^t).
+__global__ void adam_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz, float4* __restrict__ M,
+                            float4* __restrict__ V, const float* __restrict__ pw, float lr, float b1, float b2,
+                            float eps, int64_t n4) {
+  const float c1 = 1.f / (1.f - pw[0]), c2 = 1.f / (1.f - pw[1]);
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    float4 z = Z[i], m = M[i], v = V[i];
+    const float4 g = Gz[i];
+    adam_one(z.x, g.x, m.x, v.x, b1, b2, c1, c2, lr, eps);
+    adam_one(z.y, g.y, m.y, v.y, b1, b2, c1, c2, lr, eps);
+    adam_one(z.z, g.z, m.z, v.z, b1, b2, c1, c2, lr, eps);
+    adam_one(z.w, g.w, m.w, v.w, b1, b2, c1, c2, lr, eps);
+    M[i] = m; V[i] = v; Z[i] = z;
+  }
+}
 }  // namespace
 
 dq_status loss_finalize(Ctx& ctx, const float* partials, int n_per_problem, int batch, float scale,
@@ -219,6 +266,35 @@ dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n) {
   if (blocks < 1) blocks = 1;
   sgd_kernel<<<blocks, 256, 0, ctx.stream>>>(reinterpret_cast<float4*>(Z),
                                             reinterpret_cast<const float4*>(Gz), lr, n4);
+  return after_launch(ctx);
+}
+
+
+static int update_blocks(const Ctx& ctx, int64_t n4) {
+  int blocks = (int)((n4 + 255) / 256);
+  const int cap = ctx.sm_count * 8;
+  if (blocks > cap) blocks = cap;
+  return blocks < 1 ? 1 : blocks;
+}
+
+// SGD with momentum on the latent (Sec. 4.3: Z is optimised with a standard optimiser).
+dq_status momentum_update(Ctx& ctx, float* Z, const float* Gz, float* V, float lr, float mu, int64_t n) {
+  const int64_t n4 = n / 4;
+  momentum_kernel<<<update_blocks(ctx, n4), 256, 0, ctx.stream>>>(
+      reinterpret_cast<float4*>(Z), reinterpret_cast<const float4*>(Gz), reinterpret_cast<float4*>(V), lr, mu, n4);
+  return after_launch(ctx);
+}
+
+// Adam on the latent (Sec. 4.3, optimiser comparison).  pw: device float[2] holding beta1^t, beta2^t of
+// the previous step (1, 1 before the first).
+dq_status adam_update(Ctx& ctx, float* Z, const float* Gz, float* M, float* V, float* pw, float lr, float b1,
+                      float b2, float eps, int64_t n) {
+  const int64_t n4 = n / 4;
+  adam_advance_kernel<<<1, 1, 0, ctx.stream>>>(pw, b1, b2);
+  DQ_CHECK(after_launch(ctx));
+  adam_kernel<<<update_blocks(ctx, n4), 256, 0, ctx.stream>>>(
+      reinterpret_cast<float4*>(Z), reinterpret_cast<const float4*>(Gz), reinterpret_cast<float4*>(M),
+      reinterpret_cast<float4*>(V), pw, lr, b1, b2, eps, n4);
   return after_launch(ctx);
 }
 
