@@ -188,7 +188,7 @@ def main():
     path = dq.DQ_PATH_FP32 if wr.path == "fp32" else dq.DQ_PATH_BF16_TC
     h = dq.dq_calib_init(Xd, Zd, lr=wr.lr, path=path)
     if args.qr == "iterative":
-        dq.dq_calib_set_qr_method(h, dq.DQ_QR_ITERATIVE, 8)
+        dq.dq_calib_set_qr_method(h, dq.DQ_QR_ITERATIVE, 0)
     K, W = args.steps, max(args.warmup, 3)
     loss_dev = torch.empty((max(K, W), wr.batch), dtype=torch.float32, device="cuda")
 
@@ -222,7 +222,7 @@ def main():
     # ---------------------------------------------------------------- same workload, iterative QR-Orth forward
     alt = None
     if path == dq.DQ_PATH_BF16_TC and wr.d != 128 and args.qr == "householder":
-        dq.dq_calib_set_qr_method(h, dq.DQ_QR_ITERATIVE, 8)
+        dq.dq_calib_set_qr_method(h, dq.DQ_QR_ITERATIVE, 0)
         dq.dq_calib_step(h, W, loss_dev)
         barrier()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -39,7 +39,7 @@ typedef enum {
   DQ_ERR_SINGULAR = 5,    /* latent is (numerically) rank deficient: U^-T undefined */
   DQ_ERR_NONFINITE = 6,   /* loss became NaN/Inf                                */
   DQ_ERR_TIMEOUT = 7,     /* a bounded in-kernel wait gave up                   */
-  DQ_ERR_NOT_CONVERGED = 8 /* DQ_QR_ITERATIVE: latent too far from orthogonal     */
+  DQ_ERR_NOT_CONVERGED = 8 /* DQ_QR_ITERATIVE: one step moved the latent too far     */
 } dq_status;
 
 enum { DQ_FP32 = 0, DQ_BF16 = 1 };             /* x_dtype                       */
@@ -121,14 +121,16 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
 
 /* How the QR-Orth forward (Sec. 4.3: Z = R U) is computed on the tensor-core path.  Both
  * give the same unique factors (diag(U) > 0).
- *   DQ_QR_HOUSEHOLDER (default): blocked Householder QR (Algorithm 2 in compact-WY form), valid
- *     for any full-rank latent.
- *   DQ_QR_ITERATIVE: for latents close to an orthogonal matrix (the regime of the calibration
- *     loop: Z0 orthogonal, small steps).  U = I + T is the Cholesky factor of Z^T Z = I + E,
- *     found by the fixed-point iteration T <- striu(E - T^T T) + diag(E - T^T T) / 2 (n_iters
- *     tensor-core GEMMs, no dependent column steps).  The iteration contracts for roughly
- *     cond(Z) < 1.5; if the last update is still larger than 1e-5 the status word becomes
- *     DQ_ERR_NOT_CONVERGED.  n_iters <= 0 selects the default (8).
+ *   DQ_QR_HOUSEHOLDER (default): blocked Householder QR (Algorithm 2 in compact-WY form) at
+ *     every step.
+ *   DQ_QR_ITERATIVE: blocked Householder only when no factors of a nearby latent are known (first
+ *     step, after dq_calib_set_latent); afterwards incremental.  With the previous step's
+ *     U_old, Zh = Z U_old^-1 is close to orthogonal whatever Z is, its upper factor I + T is the
+ *     fixed point of T <- striu(E - T^T T) + diag(E - T^T T) / 2 with E = Zh^T Zh - I, reached from
+ *     T = 0 in n_iters sweeps of triangular tensor-core GEMMs (no dependent column steps), and
+ *     U = (I + T) U_old.  If one optimiser step moved the latent so far that the last sweep still
+ *     changed an entry by more than 1e-5, the status word becomes DQ_ERR_NOT_CONVERGED (raise
+ *     n_iters or lower the learning rate).  n_iters <= 0 selects the default (5).
  * Ignored (DQ_OK) on the fp32 path and for d == 128. */
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);

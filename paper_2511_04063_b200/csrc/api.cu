@@ -35,7 +35,7 @@ struct dq_calib {
   TcState tc;                   // tensor-core contractions (operand copies, tensor maps)
   QrTcState qtc;                // tensor-core QR-Orth operand copies
   bool fast_qr = false;
-  int qr_method = DQ_QR_HOUSEHOLDER, qr_iters = 8;
+  int qr_method = DQ_QR_HOUSEHOLDER, qr_iters = 5;
   int optimizer = DQ_SGD;
   float beta1 = 0.f, beta2 = 0.f, eps = 0.f;
   float* opt_m = nullptr;       // first moment / velocity
@@ -234,7 +234,7 @@ const char* dq_status_string(dq_status s) {
     case DQ_ERR_SINGULAR: return "latent matrix is rank deficient";
     case DQ_ERR_NONFINITE: return "non-finite loss or factor";
     case DQ_ERR_TIMEOUT: return "bounded in-kernel wait gave up";
-    case DQ_ERR_NOT_CONVERGED: return "iterative QR did not converge: latent too far from orthogonal";
+    case DQ_ERR_NOT_CONVERGED: return "iterative QR did not converge: the latent moved too far in one step";
   }
   return "unknown status";
 }
@@ -317,8 +317,8 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
   DQ_CHECK(fence_in(h));
   if (h->timing) { for (auto& m : h->ms_acc) m = 0.0; h->timed_steps = 0; }
   for (int s = 0; s < n_steps; ++s) {
-    // The captured step of the iterative QR is the warm-started one: replay it only while the
-    // previous step's factor belongs to a nearby latent.
+    // The captured step of the iterative QR is the incremental one: replay it only while the
+    // previous step's factors belong to the latent one optimiser step back.
     const bool iterative = h->fast_qr && !h->small128 && h->qr_method == DQ_QR_ITERATIVE;
     const bool use_graph = !h->timing && h->r_stale && h->eager_steps_done >= 1 && (!iterative || h->qtc.t_warm);
     if (use_graph && !h->graph && !h->graph_failed) try_capture(h);
@@ -418,7 +418,7 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
 
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters) {
   if (!h || (method != DQ_QR_HOUSEHOLDER && method != DQ_QR_ITERATIVE) || n_iters > 64) return DQ_ERR_INVALID_ARG;
-  const int iters = n_iters <= 0 ? 8 : n_iters;
+  const int iters = n_iters <= 0 ? 5 : n_iters;
   if (method == h->qr_method && iters == h->qr_iters) return DQ_OK;
   DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
   h->qr_method = method;

@@ -306,6 +306,7 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   }
   if (q.part_bs > 0) DQ_CHECK(alloc(&q.part, q.part_bs * batch));
   DQ_CHECK(alloc(&q.tw_hi, dd)); DQ_CHECK(alloc(&q.tw_lo, dd));
+  DQ_CHECK(alloc(&q.uot_hi, dd)); DQ_CHECK(alloc(&q.uot_lo, dd));
   {   // tile orders: most expensive tiles first, dealt round-robin to the persistent CTAs
     const int nb = d / 128;
     std::vector<int> upper, desc, asc;
@@ -333,7 +334,7 @@ void qr_tc_destroy(QrTcState& q) {
                  q.rt_hi, q.rt_lo, q.gqt_hi, q.gqt_lo, q.st_hi, q.st_lo, q.m_hi, q.m_lo, q.t1_hi, q.t1_lo};
   for (bf16* p : all) cudaFree(p);
   cudaFree(q.y_hi); cudaFree(q.y_lo); cudaFree(q.w2_hi); cudaFree(q.w2_lo); cudaFree(q.part); cudaFree(q.T);
-  cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.tl_upper); cudaFree(q.tl_desc_nb); cudaFree(q.tl_asc_nb);
+  cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.uot_hi); cudaFree(q.uot_lo); cudaFree(q.tl_upper); cudaFree(q.tl_desc_nb); cudaFree(q.tl_asc_nb);
   q = QrTcState();
 }
 
@@ -367,40 +368,50 @@ dq_status qr_factor_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, 
   return qr_diag_check(ctx, At, d, batch);
 }
 
-// U of a latent close to an orthogonal matrix, without dependent column steps: G = Z^T Z (upper
-// tiles), then n_iters sweeps T <- Phi(G - I - T^T T); every product is a split-bf16 tensor-core
-// GEMM restricted to the non-zero blocks of its triangular operands.
-dq_status qr_upper_factor_iterative(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* U, int d,
-                                    int batch, int n_iters) {
+// U of the latent one optimiser step after a latent whose factors (U_old, W_old = U_old^-1) are
+// known, without dependent column steps.  Zh = Z W_old is close to orthogonal however far Z itself
+// has drifted (Zh = R_old + (Z - Z_old) W_old), so its upper factor Uh = I + T is the fixed point of
+//   T <- Phi(Zh^T Zh - I - T^T T),  Phi(S) = striu(S) + diag(S) / 2,
+// reached from T = 0 in a few sweeps; then U = Uh U_old.  Every product is a split-bf16
+// tensor-core GEMM restricted to the non-zero blocks of its triangular operands.
+dq_status qr_upper_factor_incremental(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* U, int d,
+                                      int batch, int n_sweeps) {
   const int64_t dd = (int64_t)d * d;
   const dim3 tiles(d / 32, d / 32, batch);
-  bf16 *zt_hi = q.st_hi, *zt_lo = q.st_lo;     // free until the backward pass
-  float *G = ws.B, *P = ws.S, *T = ws.tmp;
-  DQ_CHECK(qrp_transpose_split(ctx, Z, ws.A, zt_hi, zt_lo, d, batch));
-  {   // G[i][j] = sum_k Z[k][i] Z[k][j], tiles on and above the block diagonal
-    Op a{zt_hi, zt_lo, d, dd};
+  bf16 *zht_hi = q.st_hi, *zht_lo = q.st_lo;   // free until the backward pass
+  bf16 *uh_hi = q.gqt_hi, *uh_lo = q.gqt_lo;   // likewise
+  float *Zh = ws.A, *G = ws.B, *P = ws.S, *T = ws.tmp, *scratch = ws.Q;
+  split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
+  DQ_CHECK(after_launch(ctx));
+  {   // Zh[i][j] = sum_k Z[i][k] W_old[k][j]
+    Op a{q.z_hi, q.z_lo, d, dd}, b{q.wt_hi, q.wt_lo, d, dd};
+    Out o; o.f32 = Zh; o.ld = d; o.bs = dd; o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all;
+    DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
+  }
+  DQ_CHECK(qrp_transpose_split(ctx, Zh, scratch, zht_hi, zht_lo, d, batch));
+  {   // G[i][j] = sum_k Zh[k][i] Zh[k][j], tiles on and above the block diagonal
+    Op a{zht_hi, zht_lo, d, dd};
     Out o; o.f32 = G; o.ld = d; o.bs = dd; o.tile_list = q.tl_upper; o.n_list = q.n_upper;
     DQ_CHECK(gemm3(ctx, a, a, d, d, d, batch, o));
   }
-  // From T = 0: n_iters sweeps, the first without the product.  From the previous step's T (the
-  // latent moved by one optimiser step): three sweeps.
-  const bool warm = q.t_warm;
-  const int sweeps = warm ? (n_iters < 3 ? n_iters : 3) : n_iters;
-  for (int it = 0; it < sweeps; ++it) {
-    const bool last = it == sweeps - 1;
-    const bool with_p = warm || it > 0;
-    if (with_p) {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
+  for (int it = 0; it < n_sweeps; ++it) {
+    const bool last = it == n_sweeps - 1;
+    if (it > 0) {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
       Op tt{q.tw_hi, q.tw_lo, d, dd};
       Out o; o.f32 = P; o.ld = d; o.bs = dd; o.k_mode = 2; o.tile_list = q.tl_upper; o.n_list = q.n_upper;
       DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
     }
-    chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, with_p ? P : nullptr, T, q.tw_hi, q.tw_lo,
-                                                        last ? U : nullptr, q.u_hi, q.u_lo, d,
-                                                        (last && with_p) ? 1 : 0, (warm || it > 0) ? 1 : 0, 1e-5f,
-                                                        ctx.d_status);
+    chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, it > 0 ? P : nullptr, T, q.tw_hi, q.tw_lo,
+                                                        last ? scratch : nullptr, uh_hi, uh_lo, d,
+                                                        (last && it > 0) ? 1 : 0, it > 0 ? 1 : 0, 1e-5f, ctx.d_status);
     DQ_CHECK(after_launch(ctx));
   }
-  q.t_warm = true;
+  {   // U[i][j] = sum_k Uh[i][k] U_old[k][j]: both upper triangular, k in [128 mb, 128 (nb + 1))
+    Op a{uh_hi, uh_lo, d, dd}, b{q.uot_hi, q.uot_lo, d, dd};
+    Out o; o.f32 = U; o.ld = d; o.bs = dd; o.hi = q.u_hi; o.lo = q.u_lo; o.ld_h = d; o.bs_h = dd;
+    o.k_mode = 1 | 4; o.tile_list = q.tl_upper; o.n_list = q.n_upper;
+    DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
+  }
   return qr_diag_check(ctx, U, d, batch);
 }
 
@@ -409,15 +420,23 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
   if (d % 128 != 0) return DQ_ERR_UNSUPPORTED;
   const int64_t dd = (int64_t)d * d;
   const dim3 tiles(d / 32, d / 32, batch);
-  if (iterative_iters > 0) {
-    DQ_CHECK(qr_upper_factor_iterative(ctx, ws, q, Z, U, d, batch, iterative_iters));
-  } else {
+  const bool incremental = iterative_iters > 0 && q.t_warm;
+  if (incremental) {
+    DQ_CHECK(qr_upper_factor_incremental(ctx, ws, q, Z, U, d, batch, iterative_iters));
+  } else {   // no factors of a nearby latent yet (first call, latent replaced): Householder
     DQ_CHECK(qr_factor_tc(ctx, ws, q, Z, d, batch));
     DQ_CHECK(qrp_gauge_ut(ctx, ws.A, U, q.u_hi, q.u_lo, d, batch));
   }
   DQ_CHECK(tri_inverse_tc(ctx, q, U, d, batch));
-  split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
-  DQ_CHECK(after_launch(ctx));
+  if (iterative_iters > 0) {   // U^T for the next step's U = Uh U_old
+    split_kernel<<<tiles, 256, 0, ctx.stream>>>(U, q.uot_hi, q.uot_lo, d, 1);
+    DQ_CHECK(after_launch(ctx));
+    q.t_warm = true;
+  }
+  if (!incremental) {
+    split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
+    DQ_CHECK(after_launch(ctx));
+  }
   // R[i][j] = sum_k Z[i][k] W[k][j]:  A = Z (row-major), B = W^T
   Op a{q.z_hi, q.z_lo, d, dd};
   Op b{q.wt_hi, q.wt_lo, d, dd};

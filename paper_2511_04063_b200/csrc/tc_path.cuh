@@ -59,8 +59,9 @@ struct QrTcState {
   int64_t part_bs = 0;                                  // elements per problem
   float* T = nullptr;                                   // [batch][128][128] compact-WY factor
   // near-orthogonal iterative factorisation
-  __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T^T of U = I + T, kept from step to step (warm start)
-  bool t_warm = false;                                  // tw_* / the fp32 T belong to a nearby latent
+  __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T^T of the sweeps
+  __nv_bfloat16 *uot_hi = nullptr, *uot_lo = nullptr;   // U^T of the previous step
+  bool t_warm = false;                                  // wt_* / uot_* hold the factors of the previous step's latent
   // tile orders for triangular products (device arrays of mb | nb << 16)
   int* tl_upper = nullptr; int n_upper = 0;             // tiles mb <= nb, largest mb first
   int* tl_desc_nb = nullptr;                            // all tiles, largest nb first
@@ -68,8 +69,8 @@ struct QrTcState {
 };
 dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count);
 void qr_tc_destroy(QrTcState& q);
-// iterative_iters > 0: U by the near-orthogonal fixed-point iteration instead of Householder
-// (iterative_iters sweeps from T = 0, or three sweeps from the previous step's T when q.t_warm).
+// iterative_iters > 0 and q.t_warm: U from the previous step's factors by iterative_iters fixed-point
+// sweeps (no dependent column steps); otherwise blocked Householder.
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
                           int batch, int iterative_iters);
 dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch);

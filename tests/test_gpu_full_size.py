@@ -32,9 +32,15 @@ def test_one_step_at_full_size(name, qr):
     w = gen.WORKLOADS[name]
     c = Calib(w)
     if qr == "iterative":
-        dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_ITERATIVE, 8)
+        dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_ITERATIVE, 0)
     Z = perturbed_latent(w, c.Z0_host, w.seed)
     c.set_latent(Z)
+    if qr == "iterative":
+        # the first step after set_latent factors with Householder; the step under test is the next
+        # one, which uses the incremental factorisation
+        c.step(1)
+        assert c.status() == dq.DQ_OK
+        Z = c.latent()
     loss = c.step(1)[0]
     assert c.status() == dq.DQ_OK
     R_used = c.buf(dq.DQ_BUF_R).cpu().numpy().astype(np.float64)
