@@ -302,6 +302,13 @@ def main():
                 "gemm_frac_of_nominal_2250": gemm_tflops / 2250.0,
                 "qr_orth_share": (phases["qr_forward"] + phases["qr_backward"]) / total_phase if total_phase else None,
                 "loss_first_last": [float(losses[0].mean()), float(losses[-1].mean())]}
+        # the optimiser update is the HBM-bound kernel of the path: 12 bytes per latent entry (SGD)
+        upd_bytes = 12.0 * d * d * B
+        if phases["update"] > 0 and d != 128:      # for d = 128 the update is fused into the backward kernel
+            gbs = upd_bytes / (phases["update"] * 1e-3) / 1e9
+            line["update_hbm"] = {"kernel": "sgd_kernel", "bytes_per_launch": upd_bytes, "achieved_gbs": gbs,
+                                  "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
+                                  "note": "event-timed phase (includes launch latency; meaningful for d >= 2048)"}
         if alt is not None:
             # same metric with dq_calib_set_qr_method(DQ_QR_ITERATIVE): the QR-Orth forward as triangular
             # tensor-core GEMMs (valid for latents near an orthogonal matrix, as in this workload)
