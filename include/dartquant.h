@@ -104,6 +104,17 @@ dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d
 dq_status dq_rotate_apply_static(const void* d_X, int64_t n, int32_t d, int64_t ldx, const float* d_R,
                                  void* d_Y, int64_t ldy, void* cuda_stream);
 
+/* Algorithm 1, X <- token_sampling(X), and the mini-batches of the hyper-parameter appendix:
+ * d_out[i] = d_X[pi(first + i)] for 0 <= i < count, where pi is a pseudo-random permutation of the
+ * token rows [0, n_total) fixed by `seed` (uniform sampling without replacement: a Feistel network
+ * with cycle walking over the Philox4x32-10 generator).  A sample of k tokens is first = 0,
+ * count = k; mini-batches are consecutive windows; use another seed for another epoch.
+ * X is [n_total][ldx], out is [count][ldo], both device, x_dtype DQ_FP32 or DQ_BF16, rows and row
+ * strides multiples of 16 bytes (else DQ_ERR_UNSUPPORTED).  To calibrate on the batch, gather into
+ * the buffer bound at dq_calib_init and call dq_calib_refresh_inputs. */
+dq_status dq_gather_tokens(const void* d_X, int32_t x_dtype, int64_t n_total, int32_t d, int64_t ldx, uint64_t seed,
+                           int64_t first, int64_t count, void* d_out, int64_t ldo, void* cuda_stream);
+
 /* Mini-batch use (the paper feeds the loop with batches of sampled tokens): the
  * caller overwrote the borrowed activation buffer d_X in place (same shape) on
  * the handle's stream; rebuild every operand copy derived from it.  Cheap no-op on

@@ -9,3 +9,4 @@ from .calib_oracle import (  # noqa: F401
     qr_pos, qr_pos_lapack, rotate, grad_wrt_rotation, qr_backward, sgd_step, momentum_step, adam_step,
     calib_step, calib_run, widen_input,
 )
+from .token_sampling import philox4x32_10, permute_index, gather_tokens  # noqa: F401,E402

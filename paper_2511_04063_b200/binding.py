@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_init", "dq_calib_step", "dq_calib_get_rotation", "dq_rotate_apply",
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
-    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer",
+    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens",
 )
 
 
@@ -65,6 +65,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_set_optimizer.restype = i32
     lib.dq_calib_set_qr_method.argtypes = [vp, i32, i32]
     lib.dq_calib_set_qr_method.restype = i32
+    lib.dq_gather_tokens.argtypes = [vp, i32, i64, i32, i64, C.c_uint64, i64, i64, vp, i64, vp]
+    lib.dq_gather_tokens.restype = i32
     lib.dq_calib_get_latent.argtypes = [vp, vp]
     lib.dq_calib_set_latent.argtypes = [vp, vp]
     lib.dq_calib_status.argtypes = [vp]
@@ -219,6 +221,17 @@ def dq_rotate_apply_static(X, R, Y, stream=None):
     n, d = X.shape
     _check(load_library().dq_rotate_apply_static(_ptr(X), n, d, X.stride(0), _ptr(R), _ptr(Y), Y.stride(0),
                                                  _stream_ptr(stream)), "dq_rotate_apply_static")
+
+
+def dq_gather_tokens(X, seed: int, first: int, count: int, out, stream=None):
+    """out[i] = X[pi_seed(first + i)]: seeded sampling of token rows without replacement.
+    X: CUDA [n, d] float32 or bfloat16; out: CUDA [count, d] of the same dtype."""
+    import torch
+    assert X.is_cuda and out.is_cuda and X.dtype == out.dtype and X.dim() == 2 and out.dim() == 2
+    n, d = X.shape
+    _check(load_library().dq_gather_tokens(_ptr(X), DQ_FP32 if X.dtype == torch.float32 else DQ_BF16, n, d,
+                                           X.stride(0), seed, first, count, _ptr(out), out.stride(0),
+                                           _stream_ptr(stream)), "dq_gather_tokens")
 
 
 def dq_version() -> str:

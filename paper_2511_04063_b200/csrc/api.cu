@@ -486,6 +486,17 @@ dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d
   return DQ_ERR_INVALID_ARG;
 }
 
+dq_status dq_gather_tokens(const void* d_X, int32_t x_dtype, int64_t n_total, int32_t d, int64_t ldx, uint64_t seed,
+                           int64_t first, int64_t count, void* d_out, int64_t ldo, void* cuda_stream) {
+  if (!d_X || !d_out || n_total <= 0 || d <= 0 || ldx < d || ldo < d || first < 0 || count < 0 ||
+      first + count > n_total)
+    return DQ_ERR_INVALID_ARG;
+  if (x_dtype != DQ_FP32 && x_dtype != DQ_BF16) return DQ_ERR_INVALID_ARG;
+  Ctx ctx;
+  ctx.stream = (cudaStream_t)cuda_stream;
+  return gather_tokens(ctx, d_X, x_dtype == DQ_FP32 ? 4 : 2, n_total, d, ldx, seed, first, count, d_out, ldo);
+}
+
 dq_status dq_rotate_apply_static(const void* d_X, int64_t n, int32_t d, int64_t ldx, const float* d_R,
                                  void* d_Y, int64_t ldy, void* cuda_stream) {
   if (!d_X || !d_R || !d_Y || n <= 0 || d <= 0 || ldx < d || ldy < d) return DQ_ERR_INVALID_ARG;

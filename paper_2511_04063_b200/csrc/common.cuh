@@ -103,6 +103,11 @@ dq_status qr128_forward(Ctx& ctx, const float* Z, float* R, float* U, float* W, 
 dq_status qr128_backward_sgd(Ctx& ctx, const float* R, const float* W, const float* Gq, float* Gz, float* Z, float lr,
                              int batch);
 
+// out[i] = X[pi_seed(first + i)] for i < count: seeded sampling of token rows without replacement
+// (token_sampling.cu).  elem_bytes = 2 (bf16) or 4 (fp32); rows must be multiples of 16 bytes.
+dq_status gather_tokens(Ctx& ctx, const void* X, int elem_bytes, int64_t n, int d, int64_t ldx, uint64_t seed,
+                        int64_t first, int64_t count, void* out, int64_t ldo);
+
 // Z <- Z - lr Gz  (n elements)
 dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n);
 // v <- mu v + Gz; Z <- Z - lr v
