@@ -104,6 +104,18 @@ dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d
 dq_status dq_rotate_apply_static(const void* d_X, int64_t n, int32_t d, int64_t ldx, const float* d_R,
                                  void* d_Y, int64_t ldy, void* cuda_stream);
 
+/* What the paper measures a rotation by (Sec. 4.1, Eq. 1; appendix on outliers and quantisation
+ * errors), for O = X R with X [n][ldx] (DQ_FP32 or DQ_BF16) and R fp32 [d][d], all device:
+ *   d_out[0] = number of entries with |o| > tau                                  (Eq. 1 over all tokens)
+ *   d_out[1] = mean squared error of per-token asymmetric uniform quantisation of O to `bits` bits:
+ *              scale = (max - min) / (2^bits - 1), zero = round(-min / scale),
+ *              q = clamp(round(o / scale) + zero, 0, 2^bits - 1), dequantised = scale (q - zero)
+ * d_out is a device double[2], written on the stream.  O is computed with bf16 tensor cores for
+ * DQ_BF16 (d % 128 == 0, n % 128 == 0) and fp32 FMA for DQ_FP32.  Allocates stream-ordered scratch.
+ * Errors: INVALID_ARG (null, bits outside 1..16, tau < 0), UNSUPPORTED, ALLOC, CUDA. */
+dq_status dq_eval_rotation(const void* d_X, int32_t x_dtype, int64_t n, int32_t d, int64_t ldx, const float* d_R,
+                           float tau, int32_t bits, double* d_out, void* cuda_stream);
+
 /* Algorithm 1, X <- token_sampling(X), and the mini-batches of the hyper-parameter appendix:
  * d_out[i] = d_X[pi(first + i)] for 0 <= i < count, where pi is a pseudo-random permutation of the
  * token rows [0, n_total) fixed by `seed` (uniform sampling without replacement: a Feistel network

@@ -10,3 +10,4 @@ from .calib_oracle import (  # noqa: F401
     calib_step, calib_run, widen_input,
 )
 from .token_sampling import philox4x32_10, permute_index, gather_tokens  # noqa: F401,E402
+from .eval_metrics import outlier_count, quantize_per_token_asymmetric, quantization_mse  # noqa: F401,E402

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_init", "dq_calib_step", "dq_calib_get_rotation", "dq_rotate_apply",
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
-    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens",
+    "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens", "dq_eval_rotation",
 )
 
 
@@ -67,6 +67,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_set_qr_method.restype = i32
     lib.dq_gather_tokens.argtypes = [vp, i32, i64, i32, i64, C.c_uint64, i64, i64, vp, i64, vp]
     lib.dq_gather_tokens.restype = i32
+    lib.dq_eval_rotation.argtypes = [vp, i32, i64, i32, i64, vp, C.c_float, i32, vp, vp]
+    lib.dq_eval_rotation.restype = i32
     lib.dq_calib_get_latent.argtypes = [vp, vp]
     lib.dq_calib_set_latent.argtypes = [vp, vp]
     lib.dq_calib_status.argtypes = [vp]
@@ -232,6 +234,20 @@ def dq_gather_tokens(X, seed: int, first: int, count: int, out, stream=None):
     _check(load_library().dq_gather_tokens(_ptr(X), DQ_FP32 if X.dtype == torch.float32 else DQ_BF16, n, d,
                                            X.stride(0), seed, first, count, _ptr(out), out.stride(0),
                                            _stream_ptr(stream)), "dq_gather_tokens")
+
+
+def dq_eval_rotation(X, R, tau: float, bits: int, stream=None):
+    """(number of outliers |o| > tau, mean squared per-token asymmetric quantisation error) of O = X R.
+    X: CUDA [n, d] float32 or bfloat16; R: CUDA float32 [d, d].  Synchronises to read the result."""
+    import torch
+    assert X.is_cuda and R.is_cuda and R.dtype == torch.float32 and X.dim() == 2
+    n, d = X.shape
+    out = torch.zeros(2, dtype=torch.float64, device=X.device)
+    _check(load_library().dq_eval_rotation(_ptr(X), DQ_FP32 if X.dtype == torch.float32 else DQ_BF16, n, d,
+                                           X.stride(0), _ptr(R), tau, bits, _ptr(out), _stream_ptr(stream)),
+           "dq_eval_rotation")
+    res = out.cpu()
+    return int(round(float(res[0]))), float(res[1])
 
 
 def dq_version() -> str:

@@ -486,6 +486,15 @@ dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d
   return DQ_ERR_INVALID_ARG;
 }
 
+dq_status dq_eval_rotation(const void* d_X, int32_t x_dtype, int64_t n, int32_t d, int64_t ldx, const float* d_R,
+                           float tau, int32_t bits, double* d_out, void* cuda_stream) {
+  if (!d_X || !d_R || !d_out || n <= 0 || d <= 0 || ldx < d) return DQ_ERR_INVALID_ARG;
+  if (x_dtype != DQ_FP32 && x_dtype != DQ_BF16) return DQ_ERR_INVALID_ARG;
+  Ctx ctx;
+  ctx.stream = (cudaStream_t)cuda_stream;
+  return eval_rotation(ctx, d_X, x_dtype, n, d, ldx, d_R, tau, bits, d_out);
+}
+
 dq_status dq_gather_tokens(const void* d_X, int32_t x_dtype, int64_t n_total, int32_t d, int64_t ldx, uint64_t seed,
                            int64_t first, int64_t count, void* d_out, int64_t ldo, void* cuda_stream) {
   if (!d_X || !d_out || n_total <= 0 || d <= 0 || ldx < d || ldo < d || first < 0 || count < 0 ||

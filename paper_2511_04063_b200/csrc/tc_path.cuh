@@ -34,6 +34,9 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials);
 dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale);
 dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t ldx, const float* d_R,
                           void* d_Y, int64_t ldy);
+// Outliers (Eq. 1) and per-token asymmetric quantisation error of O = X R (eval_metrics.cu).
+dq_status eval_rotation(Ctx& ctx, const void* d_X, int x_dtype, int64_t n, int d, int64_t ldx, const float* d_R,
+                        float tau, int bits, double* d_out);
 // Same product with its scratch in a file-scope device array: no allocation of any kind.
 dq_status tc_rotate_apply_static(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t ldx, const float* d_R,
                                  void* d_Y, int64_t ldy);

@@ -304,3 +304,38 @@ def test_adam_epsilon_bounds_the_step_for_tiny_gradients():
     Z, g = np.zeros((2, 2)), np.full((2, 2), 1e-12)
     Z1, _, _ = orc.adam_step(Z, g, np.zeros_like(Z), np.zeros_like(Z), 1, 1.0, eps=1e-8)
     assert np.allclose(Z1, -1e-12 / (1e-12 + 1e-8))                              # |step| = lr g / (|g| + eps)
+
+
+# --------------------------------------------------------------------- evaluation metrics (Eq. 1, quantisation error)
+def test_outlier_count_matches_brute_force_and_is_rotation_sensitive():
+    rng = np.random.default_rng(4)
+    O = rng.standard_normal((7, 9)) * 3
+    brute = sum(1 for t in range(7) for j in range(9) if abs(O[t, j]) > 2.5)
+    assert orc.outlier_count(O, 2.5) == brute
+    # one massive channel: d outliers-free values after a Hadamard rotation spreads it (norm invariance)
+    d = 16
+    x = np.zeros((1, d)); x[0, 3] = 8.0
+    H = np.array([[(-1) ** bin(i & j).count("1") for j in range(d)] for i in range(d)]) / np.sqrt(d)
+    assert orc.outlier_count(x, 4.0) == 1 and orc.outlier_count(x @ H, 4.0) == 0
+
+
+def test_asymmetric_quantiser_closed_forms():
+    # values already on the grid of the row are reproduced exactly
+    row = np.array([[-1.0, -0.5, 0.0, 0.5, 1.0, 6.5]])            # range 7.5, 4 bits: step 0.5
+    assert np.allclose(orc.quantize_per_token_asymmetric(row, 4), row, atol=1e-12)
+    assert orc.quantization_mse(row, 4) < 1e-24
+    # the error of any entry is at most half a step (plus the shift of the rounded zero point)
+    rng = np.random.default_rng(5)
+    O = rng.standard_normal((50, 33)) * rng.uniform(0.1, 20, size=(50, 1))
+    for bits in (2, 4, 8):
+        Q = orc.quantize_per_token_asymmetric(O, bits)
+        step = (O.max(1) - O.min(1)) / (2 ** bits - 1)
+        assert (np.abs(Q - O).max(axis=1) <= step * (1.0 + 1e-9)).all()
+        assert len(np.unique(np.round(Q[0] / step[0], 6))) <= 2 ** bits
+    # uniform data on [0, 1): mean squared error of a uniform quantiser is step^2 / 12
+    U = rng.uniform(0, 1, size=(20, 20000))
+    mse = orc.quantization_mse(U, 4)
+    assert abs(mse - (1.0 / 15) ** 2 / 12) < 0.05 * (1.0 / 15) ** 2 / 12
+    # constant rows carry no error; per-token scaling makes the relative error scale-free
+    assert orc.quantization_mse(np.full((3, 5), 2.5), 4) == 0.0
+    assert np.isclose(orc.quantization_mse(O * 8.0, 4), 64.0 * orc.quantization_mse(O, 4), rtol=1e-12)
