@@ -12,9 +12,9 @@
 //                           into At and the split-bf16 reflector block Y (both
 //                           orientations).
 //   2. tensor-core GEMM     [S; W^T] = [Y C]^T Y   (split over the m rows)
-//   3. wy_t_kernel          T = (striu(S) + diag(S)/2)^-1  so that H_1..H_128 = I - Y T Y^T
-//   4. wy_w2_kernel         W2^T = W^T T          (fp32, also reduces the split partials)
-//   5. tensor-core GEMM     C^T -= W2^T Y^T       (fp32 result + split-bf16 copy)
+//   3. wy_w2_kernel         W2 with Q^T C = C - Y W2: block forward substitution over the four
+//                           inner block reflectors (T_k from the panel, S_kl = V_k^T V_l), fp32
+//   4. tensor-core GEMM     C^T -= W2^T Y^T       (fp32 result + split-bf16 copy)
 // Exchanges inside the cluster are pushes into every CTA's shared memory followed
 // by one cluster barrier; all sums run in a fixed order (bit-reproducible).
 #include <cooperative_groups.h>
@@ -203,7 +203,7 @@ __device__ __forceinline__ void col_step(float (&a)[2][32], const int (&rowi)[2]
 // (Algorithm 2's sign rule), tau = (beta - x_1) / beta.
 template <int NT>
 __global__ void __launch_bounds__(NT, 1)
-qr_panel_cm_kernel(float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, int d, int c0) {
+qr_panel_cm_kernel(float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, float* Tk, int d, int c0) {
   constexpr int NW = NT / 32;
   using L = PanelSmem<NW>;
   cg::cluster_group cluster = cg::this_cluster();
@@ -213,6 +213,7 @@ qr_panel_cm_kernel(float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, 
     const int64_t dd = (int64_t)d * d, boff = (int64_t)blockIdx.y;
     At += boff * dd; at_hi += boff * dd; at_lo += boff * dd;
     y_hi += boff * (int64_t)d * OB; y_lo += boff * (int64_t)d * OB;
+    Tk += boff * OB * IB;
   }
   extern __shared__ float sm[];
   float* red = sm + L::RED;
@@ -372,121 +373,52 @@ qr_panel_cm_kernel(float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, 
     }
     __syncthreads();   // T of this inner panel is complete; At writes are ordered before re-reads
   }
+  if (cta == 0) {   // compact-WY factors of the four inner panels: Tk[k][i][j]
+    for (int e = tid; e < (OB / IB) * IB * IB; e += NT) Tk[e] = Ts[(e >> 10) * 32 * 33 + ((e >> 5) & 31) * 33 + (e & 31)];
+  }
   cluster.sync();   // no CTA may exit while others can still push into its shared memory
 }
 
 
-// ----------------------------------------------------------------------------- T of the outer block
-// Dense C[M x N] (+)= alpha A[M x K] B[K x N] on shared-memory matrices (leading dimensions lda, ldb,
-// ldc), 4 x 4 register tiles, 256 threads; M, N multiples of 4.
-__device__ __forceinline__ void smem_mm(const float* A, int lda, const float* B, int ldb, float* C, int ldc,
-                                        int M, int N, int K, float alpha, int tid) {
-  const int tn = N / 4, tiles = (M / 4) * tn;
-  for (int t = tid; t < tiles; t += 256) {
-    const int r0 = (t / tn) * 4, c0 = (t % tn) * 4;
-    float acc[4][4] = {};
-    for (int k = 0; k < K; ++k) {
-      float av[4], bv[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) av[i] = A[(r0 + i) * lda + k];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) bv[j] = B[k * ldb + c0 + j];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) C[(r0 + i) * ldc + c0 + j] = alpha * acc[i][j];
-  }
-}
-
-constexpr int TLD = 129;
-constexpr int WY_T_SMEM = (2 * 128 * TLD + 64 * 65) * 4;
-
-// S = sum of the split partials (rows 0..127 of part); T = (striu(S) + diag(S) / 2)^-1, the
-// compact-WY factor of the 128 reflectors (T^-1 + T^-T = Y^T Y).  A zero column of Y (skipped
-// reflector) decouples: its diagonal gets a placeholder.  One CTA per problem.
-__global__ void __launch_bounds__(256) wy_t_kernel(const float* __restrict__ part, int ksplit, int m,
-                                                   int64_t part_batch_stride, float* __restrict__ T) {
-  extern __shared__ float sm[];
-  float* U = sm;                    // [128][TLD]  T^-1 (upper triangular)
-  float* X = sm + 128 * TLD;        // [128][TLD]  its inverse
-  float* Tmp = X + 128 * TLD;       // [64][65]
-  part += (int64_t)blockIdx.y * part_batch_stride;
-  T += (int64_t)blockIdx.y * 128 * 128;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-#pragma unroll 4
-  for (int it = 0; it < 16; ++it) {   // independent 16-byte loads: the partials sit in L2 / HBM
-    const int e = (it * 256 + tid) * 4;
-    const int r = e >> 7, c0 = e & 127;
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (c0 + 3 >= r)
-      for (int sp = 0; sp < ksplit; ++sp) {
-        const float4 t = *reinterpret_cast<const float4*>(part + (int64_t)sp * m * 128 + e);
-        s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
-      }
-    const float sv[4] = {s.x, s.y, s.z, s.w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int c = c0 + q;
-      float v = (c > r) ? sv[q] : ((c == r) ? 0.5f * sv[q] : 0.f);
-      if (c == r && !(v > 0.f)) v = 1.f;
-      U[r * TLD + c] = v;
-      X[r * TLD + c] = 0.f;
-    }
-  }
-  __syncthreads();
-  if (warp < 4) {   // inverse of the four 32 x 32 diagonal blocks: lane j solves U x = e_j
-    const int o = warp * 32, j = lane;
-    X[(o + j) * TLD + o + j] = 1.f / U[(o + j) * TLD + o + j];
-    for (int i = j - 1; i >= 0; --i) {
-      float s = 0.f;
-      for (int k = i + 1; k <= j; ++k) s = fmaf(U[(o + i) * TLD + o + k], X[(o + k) * TLD + o + j], s);
-      X[(o + i) * TLD + o + j] = -s / U[(o + i) * TLD + o + i];
-    }
-  }
-  __syncthreads();
-  // inv([A B; 0 C]) = [A^-1, -A^-1 B C^-1; 0, C^-1]: 32-blocks -> 64-blocks -> 128
-  for (int pair = 0; pair < 2; ++pair) {
-    const int o = pair * 64;
-    smem_mm(U + o * TLD + o + 32, TLD, X + (o + 32) * TLD + o + 32, TLD, Tmp, 65, 32, 32, 32, 1.f, tid);
-    __syncthreads();
-    smem_mm(X + o * TLD + o, TLD, Tmp, 65, X + o * TLD + o + 32, TLD, 32, 32, 32, -1.f, tid);
-    __syncthreads();
-  }
-  smem_mm(U + 64, TLD, X + 64 * TLD + 64, TLD, Tmp, 65, 64, 64, 64, 1.f, tid);
-  __syncthreads();
-  smem_mm(X, TLD, Tmp, 65, X + 64, TLD, 64, 64, 64, -1.f, tid);
-  __syncthreads();
-  for (int e = tid; e < 128 * 128; e += 256) {
-    const int r = e >> 7, c = e & 127;
-    T[e] = (c >= r) ? X[r * TLD + c] : 0.f;
-  }
-}
-
-// W2^T[row][j] = sum_k W^T[row][k] T[k][j] with W^T = sum of the split partials (rows 128.. of
-// part); written as a split-bf16 pair [n][128].  64 rows per CTA, 4 x 8 outputs per thread.
-constexpr int WY_W2_SMEM = (128 * 128 + 64 * TLD) * 4;
+// ----------------------------------------------------------------------------- W2 of the outer block
+// The outer block's 128 reflectors are four block reflectors H_k = I - V_k T_k V_k^T (T_k from the
+// panel kernel).  Q^T C = H_3^T H_2^T H_1^T H_0^T C = C - Y W2 with, per column of C (= row of W^T),
+//   W2_k = T_k^T (W_k - sum_{l < k} S_kl W2_l),   W = Y^T C,  S = Y^T Y  (S_kl = V_k^T V_l),
+// a block forward substitution with 32 x 32 blocks.  W^T and S are the sums of the split partials
+// of the [S; W^T] product (S = rows 0..127).
+constexpr int SLD = 129;
+constexpr int W2_ROWS_PER_CTA = 64;
+constexpr int WY_W2_SMEM = (128 * SLD + 4 * 32 * 32 + W2_ROWS_PER_CTA * SLD) * 4;
+// 64 rows of W^T per CTA, staged in shared memory and turned into W2^T block by block; every
+// product is a (64 x K) x (K x 32) shared-memory matmul, 2 x 4 outputs per thread.
 __global__ void __launch_bounds__(256) wy_w2_kernel(const float* __restrict__ part, int ksplit, int m,
-                                                    int64_t part_batch_stride, const float* __restrict__ T,
+                                                    int64_t part_batch_stride, const float* __restrict__ Tk,
                                                     bf16* __restrict__ w2_hi, bf16* __restrict__ w2_lo,
                                                     int64_t w2_batch_stride) {
   extern __shared__ float sm[];
-  float* Ts = sm;                 // [128][128]
-  float* Ws = sm + 128 * 128;     // [64][TLD]
+  float* Ss = sm;                  // [128][SLD]  Y^T Y (only the blocks below the block diagonal are used)
+  float* Ts = sm + 128 * SLD;      // [4][32][32]
+  float* Ws = Ts + 4 * 32 * 32;    // [64][SLD]   W^T rows, overwritten block by block with W2^T
   part += (int64_t)blockIdx.y * part_batch_stride;
-  T += (int64_t)blockIdx.y * 128 * 128;
+  Tk += (int64_t)blockIdx.y * 4 * 32 * 32;
   w2_hi += (int64_t)blockIdx.y * w2_batch_stride;
   w2_lo += (int64_t)blockIdx.y * w2_batch_stride;
   const int tid = threadIdx.x;
-  const int row0 = blockIdx.x * 64;
-  for (int e = tid; e < 128 * 128 / 4; e += 256)
-    reinterpret_cast<float4*>(Ts)[e] = reinterpret_cast<const float4*>(T)[e];
+  const int row0 = blockIdx.x * W2_ROWS_PER_CTA;
+#pragma unroll 4
+  for (int it = 0; it < 12; ++it) {   // rows 32..127 of S, independent 16-byte loads
+    const int e = (it * 256 + tid) * 4;
+    const int r = 32 + (e >> 7), c = e & 127;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < (r & ~31))
+      for (int sp = 0; sp < ksplit; ++sp) {
+        const float4 t = *reinterpret_cast<const float4*>(part + (int64_t)sp * m * 128 + r * 128 + c);
+        s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
+      }
+    Ss[r * SLD + c] = s.x; Ss[r * SLD + c + 1] = s.y; Ss[r * SLD + c + 2] = s.z; Ss[r * SLD + c + 3] = s.w;
+  }
 #pragma unroll
-  for (int it = 0; it < 8; ++it) {    // independent 16-byte loads
+  for (int it = 0; it < 8; ++it) {    // the 64 x 128 tile of W^T
     const int e = (it * 256 + tid) * 4;
     const int r = e >> 7, k = e & 127;
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -494,37 +426,59 @@ __global__ void __launch_bounds__(256) wy_w2_kernel(const float* __restrict__ pa
       const float4 t = *reinterpret_cast<const float4*>(part + ((int64_t)sp * m + 128 + row0 + r) * 128 + k);
       s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
     }
-    Ws[r * TLD + k] = s.x; Ws[r * TLD + k + 1] = s.y; Ws[r * TLD + k + 2] = s.z; Ws[r * TLD + k + 3] = s.w;
+    Ws[r * SLD + k] = s.x; Ws[r * SLD + k + 1] = s.y; Ws[r * SLD + k + 2] = s.z; Ws[r * SLD + k + 3] = s.w;
   }
+  for (int e = tid; e < 4 * 32 * 32; e += 256) Ts[e] = Tk[e];
   __syncthreads();
-  const int r0 = (tid >> 4) * 4, c0 = (tid & 15) * 8;
-  float acc[4][8] = {};
-  for (int k = 0; k < c0 + 8; ++k) {   // T is upper triangular: T[k][j] = 0 for k > j
-    float wv[4];
+  const int r0 = (tid >> 3) * 2, c0 = (tid & 7) * 4;   // rows r0, r0 + 1; columns c0 .. c0 + 3 of the current block
+#pragma unroll 1
+  for (int k = 0; k < 4; ++k) {
+    // X_k = W_k - [W2_0 .. W2_{k-1}] S_k,0:k^T
+    float x[2][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) wv[i] = Ws[(r0 + i) * TLD + k];
-    const float4 t0 = *reinterpret_cast<const float4*>(Ts + k * 128 + c0);
-    const float4 t1 = *reinterpret_cast<const float4*>(Ts + k * 128 + c0 + 4);
-    const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+    for (int a = 0; a < 2; ++a)
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+      for (int j = 0; j < 4; ++j) x[a][j] = Ws[(r0 + a) * SLD + 32 * k + c0 + j];
+    for (int i = 0; i < 32 * k; ++i) {
+      const float a0 = Ws[r0 * SLD + i], a1 = Ws[(r0 + 1) * SLD + i];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(wv[i], tv[j], acc[i][j]);
-  }
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint32_t ph[4], pl[4];
-#pragma unroll
-    for (int j = 0; j < 8; j += 2) {
-      bf16 h0, l0, h1, l1;
-      split2(acc[i][j], h0, l0);
-      split2(acc[i][j + 1], h1, l1);
-      ph[j >> 1] = pack2(h0, h1);
-      pl[j >> 1] = pack2(l0, l1);
+      for (int j = 0; j < 4; ++j) {
+        const float sv = Ss[(32 * k + c0 + j) * SLD + i];
+        x[0][j] = fmaf(-a0, sv, x[0][j]);
+        x[1][j] = fmaf(-a1, sv, x[1][j]);
+      }
     }
-    const int64_t o = (int64_t)(row0 + r0 + i) * 128 + c0;
-    *reinterpret_cast<uint4*>(w2_hi + o) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
-    *reinterpret_cast<uint4*>(w2_lo + o) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+    __syncthreads();                 // everyone has read the old block k
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) Ws[(r0 + a) * SLD + 32 * k + c0 + j] = x[a][j];
+    __syncthreads();
+    // W2_k = X_k T_k  (T_k upper triangular: i <= column)
+    float o[2][4] = {};
+    const float* T = Ts + k * 1024;
+    for (int i = 0; i < c0 + 4; ++i) {
+      const float a0 = Ws[r0 * SLD + 32 * k + i], a1 = Ws[(r0 + 1) * SLD + 32 * k + i];
+      const float4 t = *reinterpret_cast<const float4*>(T + i * 32 + c0);
+      o[0][0] = fmaf(a0, t.x, o[0][0]); o[0][1] = fmaf(a0, t.y, o[0][1]);
+      o[0][2] = fmaf(a0, t.z, o[0][2]); o[0][3] = fmaf(a0, t.w, o[0][3]);
+      o[1][0] = fmaf(a1, t.x, o[1][0]); o[1][1] = fmaf(a1, t.y, o[1][1]);
+      o[1][2] = fmaf(a1, t.z, o[1][2]); o[1][3] = fmaf(a1, t.w, o[1][3]);
+    }
+    __syncthreads();                 // everyone has read X_k
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      bf16 h[4], l[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        Ws[(r0 + a) * SLD + 32 * k + c0 + j] = o[a][j];
+        split2(o[a][j], h[j], l[j]);
+      }
+      const int64_t off = (int64_t)(row0 + r0 + a) * 128 + 32 * k + c0;
+      *reinterpret_cast<uint2*>(w2_hi + off) = make_uint2(pack2(h[0], h[1]), pack2(h[2], h[3]));
+      *reinterpret_cast<uint2*>(w2_lo + off) = make_uint2(pack2(l[0], l[1]), pack2(l[2], l[3]));
+    }
+    __syncthreads();
   }
 }
 
@@ -552,7 +506,7 @@ __global__ void __launch_bounds__(256) gauge_ut_kernel(const float* __restrict__
 
 template <int NT>
 dq_status launch_panel(Ctx& ctx, int cs, int batch, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo,
-                       int d, int c0) {
+                       float* Tk, int d, int c0) {
   using L = PanelSmem<NT / 32>;
   static bool attr = false;
   auto kern = qr_panel_cm_kernel<NT>;
@@ -569,7 +523,7 @@ dq_status launch_panel(Ctx& ctx, int cs, int batch, float* At, bf16* at_hi, bf16
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  DQ_CHECK_CUDA(cudaLaunchKernelEx(&cfg, kern, At, at_hi, at_lo, y_hi, y_lo, d, c0));
+  DQ_CHECK_CUDA(cudaLaunchKernelEx(&cfg, kern, At, at_hi, at_lo, y_hi, y_lo, Tk, d, c0));
   return after_launch(ctx);
 }
 
@@ -580,8 +534,8 @@ dq_status qrp_transpose_split(Ctx& ctx, const float* Z, float* At, bf16* hi, bf1
   return after_launch(ctx);
 }
 
-dq_status qrp_panel(Ctx& ctx, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, int d, int c0,
-                    int batch) {
+dq_status qrp_panel(Ctx& ctx, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, float* Tk, int d,
+                    int c0, int batch) {
   const int m = d - c0;
   if (m <= 0 || m % OB != 0 || m > 8192) return DQ_ERR_UNSUPPORTED;
   const bool wide = m > 4096;                       // 1024 rows per CTA instead of 512
@@ -589,28 +543,19 @@ dq_status qrp_panel(Ctx& ctx, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, b
   int cs = 1;
   while (cs * rows_per_cta < m) cs *= 2;
   if (cs > MAX_CS) return DQ_ERR_UNSUPPORTED;
-  return wide ? launch_panel<512>(ctx, cs, batch, At, at_hi, at_lo, y_hi, y_lo, d, c0)
-              : launch_panel<256>(ctx, cs, batch, At, at_hi, at_lo, y_hi, y_lo, d, c0);
+  return wide ? launch_panel<512>(ctx, cs, batch, At, at_hi, at_lo, y_hi, y_lo, Tk, d, c0)
+              : launch_panel<256>(ctx, cs, batch, At, at_hi, at_lo, y_hi, y_lo, Tk, d, c0);
 }
 
-dq_status qrp_wy_t(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, float* T, int batch) {
-  static bool attr = false;
-  if (!attr) {
-    DQ_CHECK_CUDA(cudaFuncSetAttribute(wy_t_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WY_T_SMEM));
-    attr = true;
-  }
-  wy_t_kernel<<<dim3(1, batch), 256, WY_T_SMEM, ctx.stream>>>(part, ksplit, m, part_bs, T);
-  return after_launch(ctx);
-}
-
-dq_status qrp_wy_w2(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, const float* T, bf16* w2_hi,
+dq_status qrp_wy_w2(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, const float* Tk, bf16* w2_hi,
                     bf16* w2_lo, int64_t w2_bs, int n, int batch) {
   static bool attr = false;
   if (!attr) {
     DQ_CHECK_CUDA(cudaFuncSetAttribute(wy_w2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WY_W2_SMEM));
     attr = true;
   }
-  wy_w2_kernel<<<dim3(n / 64, batch), 256, WY_W2_SMEM, ctx.stream>>>(part, ksplit, m, part_bs, T, w2_hi, w2_lo, w2_bs);
+  wy_w2_kernel<<<dim3(n / W2_ROWS_PER_CTA, batch), 256, WY_W2_SMEM, ctx.stream>>>(part, ksplit, m, part_bs, Tk, w2_hi,
+                                                                                 w2_lo, w2_bs);
   return after_launch(ctx);
 }
 

@@ -348,7 +348,7 @@ dq_status qr_factor_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, 
   DQ_CHECK(qrp_transpose_split(ctx, Z, At, at_hi, at_lo, d, batch));
   for (int c0 = 0; c0 < d; c0 += 128) {
     const int m = d - c0, n = m - 128;
-    DQ_CHECK(qrp_panel(ctx, At, at_hi, at_lo, q.y_hi, q.y_lo, d, c0, batch));
+    DQ_CHECK(qrp_panel(ctx, At, at_hi, at_lo, q.y_hi, q.y_lo, q.T, d, c0, batch));
     if (n == 0) break;
     const int64_t o = (int64_t)c0 * d + c0;
     // [S; W^T][i][j] = sum_r At[c0 + i][r] Y^T[j][r], r in [c0, d): rows 0..127 are Y^T Y, the rest W^T
@@ -356,7 +356,6 @@ dq_status qr_factor_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, 
     Op a{at_hi + o, at_lo + o, d, dd}, b{at_hi + o, at_lo + o, d, dd};
     Out sw; sw.f32 = q.part; sw.ld = 128; sw.bs = q.part_bs; sw.ksplit = ks; sw.split_stride = (int64_t)m * 128;
     DQ_CHECK(gemm3(ctx, a, b, m, 128, m, batch, sw));
-    DQ_CHECK(qrp_wy_t(ctx, q.part, ks, m, q.part_bs, q.T, batch));
     DQ_CHECK(qrp_wy_w2(ctx, q.part, ks, m, q.part_bs, q.T, q.w2_hi, q.w2_lo, yb, n, batch));
     // C^T[c][r] -= sum_j W2^T[c][j] Y[r][j]
     Op w2{q.w2_hi, q.w2_lo, 128, yb}, y{q.y_hi + (int64_t)c0 * 128, q.y_lo + (int64_t)c0 * 128, 128, yb};

@@ -60,7 +60,7 @@ struct QrTcState {
   __nv_bfloat16 *w2_hi = nullptr, *w2_lo = nullptr;     // [batch][d][128] (T^T Y^T C)^T
   float* part = nullptr;                                // split partials of [S; W^T]
   int64_t part_bs = 0;                                  // elements per problem
-  float* T = nullptr;                                   // [batch][128][128] compact-WY factor
+  float* T = nullptr;                                   // [batch][4][32][32] compact-WY factors of the inner panels
   // near-orthogonal iterative factorisation
   __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T^T of the sweeps
   __nv_bfloat16 *uot_hi = nullptr, *uot_lo = nullptr;   // U^T of the previous step
@@ -84,9 +84,8 @@ dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* G
 dq_status qrp_transpose_split(Ctx& ctx, const float* Z, float* At, __nv_bfloat16* hi, __nv_bfloat16* lo, int d,
                               int batch);
 dq_status qrp_panel(Ctx& ctx, float* At, __nv_bfloat16* at_hi, __nv_bfloat16* at_lo, __nv_bfloat16* y_hi,
-                    __nv_bfloat16* y_lo, int d, int c0, int batch);
-dq_status qrp_wy_t(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, float* T, int batch);
-dq_status qrp_wy_w2(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, const float* T,
+                    __nv_bfloat16* y_lo, float* Tk, int d, int c0, int batch);
+dq_status qrp_wy_w2(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, const float* Tk,
                     __nv_bfloat16* w2_hi, __nv_bfloat16* w2_lo, int64_t w2_bs, int n, int batch);
 dq_status qrp_gauge_ut(Ctx& ctx, const float* At, float* U, __nv_bfloat16* hi, __nv_bfloat16* lo, int d, int batch);
 // Rank / finiteness test of diag(U) (qr_forward.cu); works on either orientation.
