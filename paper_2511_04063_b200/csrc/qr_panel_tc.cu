@@ -97,7 +97,8 @@ struct PanelSmem {
   static constexpr int WX = WP + NW * 1024;              // [MAX_CS][1024] per-CTA partials (pushed)
   static constexpr int WF = WX + MAX_CS * 1024;          // [32][32] V_k^T P
   static constexpr int W2 = WF + 1024;                   // [32][32] T_k^T V_k^T P
-  static constexpr int TOTAL = W2 + 1024;
+  static constexpr int STG = W2 + 1024;                  // [NW][2][32][STG_LD] staging of V_k / P rows for the warp MMAs
+  static constexpr int TOTAL = STG + (NW == 8 ? NW * 2 * 32 * 40 : 0);
   static constexpr int BYTES = TOTAL * 4;
 };
 
@@ -113,6 +114,87 @@ __device__ __forceinline__ void load_v8(float (&vv)[8][2], const float* Vk, int 
     for (int s = 0; s < 2; ++s)
       vv[u][s] = (rowi[s] > dg0 + u) ? ((rowi[s] < m) ? vcol[rowi[s]] : 0.f) : ((rowi[s] == dg0 + u) ? 1.f : 0.f);
   }
+}
+
+constexpr int STG_LD = 40;   // row stride of the staging tiles: fragment loads hit 32 distinct banks
+
+// x = hi + lo with hi, lo representable in tf32 (about 2^-22 relative): three tensor-core products
+// hi*hi + hi*lo + lo*hi recover fp32-like accuracy.
+__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
+  const float r = x - __uint_as_float(hi);
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(r));
+}
+// D += A B for one 16 x 8 x 8 tile (A row-major M x K, B column-major K x N), tf32 inputs, fp32 accumulate.
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// Warp partial of W = V_k^T P over this warp's 64 rows (two 32-row groups, lane = row) on the
+// tensor cores: rows are staged in shared memory, fragments of A = V_k^T (M = reflector, K = row) and
+// B = P (K = row, N = panel column) are read back in the warp-MMA layout, products in 3 x tf32.
+// Result: Wp[cp][p] for this warp.
+__device__ __forceinline__ void warp_vtp_mma(const float (&a)[2][32], const float* Vk, int d, int dg0,
+                                             const int (&rowi)[2], int m, float* Vs, float* Ps, float* Wp_warp,
+                                             int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  float acc[2][4][4];
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
+#pragma unroll
+  for (int s = 0; s < 2; ++s) {   // unrolled: a[s][.] must stay in registers
+    float v[32];
+#pragma unroll
+    for (int cp = 0; cp < 32; ++cp)
+      v[cp] = (rowi[s] > dg0 + cp) ? ((rowi[s] < m) ? Vk[(int64_t)cp * d + rowi[s]] : 0.f)
+                                   : ((rowi[s] == dg0 + cp) ? 1.f : 0.f);
+    __syncwarp();
+#pragma unroll
+    for (int cp = 0; cp < 32; ++cp) {
+      Vs[lane * STG_LD + cp] = v[cp];
+      Ps[lane * STG_LD + cp] = a[s][cp];
+    }
+    __syncwarp();
+#pragma unroll 1
+    for (int kt = 0; kt < 4; ++kt) {
+      uint32_t bh[4][2], bl[4][2];
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        split_tf32(Ps[(8 * kt + t) * STG_LD + 8 * nt + g], bh[nt][0], bl[nt][0]);
+        split_tf32(Ps[(8 * kt + t + 4) * STG_LD + 8 * nt + g], bh[nt][1], bl[nt][1]);
+      }
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        uint32_t ah[4], al[4];
+        split_tf32(Vs[(8 * kt + t) * STG_LD + 16 * mt + g], ah[0], al[0]);
+        split_tf32(Vs[(8 * kt + t) * STG_LD + 16 * mt + g + 8], ah[1], al[1]);
+        split_tf32(Vs[(8 * kt + t + 4) * STG_LD + 16 * mt + g], ah[2], al[2]);
+        split_tf32(Vs[(8 * kt + t + 4) * STG_LD + 16 * mt + g + 8], ah[3], al[3]);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          mma_tf32(acc[mt][nt], al, bh[nt]);
+          mma_tf32(acc[mt][nt], ah, bl[nt]);
+          mma_tf32(acc[mt][nt], ah, bh[nt]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      float* o = Wp_warp + (16 * mt + g) * 32 + 8 * nt + 2 * t;
+      o[0] = acc[mt][nt][0]; o[1] = acc[mt][nt][1];
+      o[8 * 32] = acc[mt][nt][2]; o[8 * 32 + 1] = acc[mt][nt][3];
+    }
 }
 
 struct PanelCtx {
@@ -250,17 +332,22 @@ qr_panel_cm_kernel(float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo, 
 #pragma unroll 1
     for (int k = 0; k < ip; ++k) {
       const float* Vk = At + (int64_t)(c0 + k * IB) * d + c0;
+      if constexpr (NW == 8) {   // 255 registers per thread: room for the MMA fragments
+        float* stg = sm + L::STG + warp * (2 * 32 * STG_LD);
+        warp_vtp_mma(a, Vk, d, k * IB, rowi, m, stg, stg + 32 * STG_LD, Wp + warp * 1024, lane);
+      } else {
 #pragma unroll 1
-      for (int cp0 = 0; cp0 < 32; cp0 += 8) {
-        float vv[8][2];
-        load_v8(vv, Vk, d, k * IB + cp0, cp0, rowi, m);
+        for (int cp0 = 0; cp0 < 32; cp0 += 8) {
+          float vv[8][2];
+          load_v8(vv, Vk, d, k * IB + cp0, cp0, rowi, m);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          float acc[32];
+          for (int u = 0; u < 8; ++u) {
+            float acc[32];
 #pragma unroll
-          for (int p = 0; p < 32; ++p) acc[p] = fmaf(vv[u][1], a[1][p], vv[u][0] * a[0][p]);
-          const float t = warp_transpose_reduce32(acc, lane);
-          Wp[(warp * 32 + cp0 + u) * 32 + lane] = t;
+            for (int p = 0; p < 32; ++p) acc[p] = fmaf(vv[u][1], a[1][p], vv[u][0] * a[0][p]);
+            const float t = warp_transpose_reduce32(acc, lane);
+            Wp[(warp * 32 + cp0 + u) * 32 + lane] = t;
+          }
         }
       }
       __syncthreads();
