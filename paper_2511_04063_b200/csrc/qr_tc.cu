@@ -1,14 +1,14 @@
-// QR-Orth on the tensor cores ("fast" mode used with the tensor-core path).
+// QR-Orth on the tensor cores (used with the tensor-core path).
 //
-// Forward:  blocked Householder factorisation Z = Q U (only U is kept), gauge
-//           diag(U) > 0, W = U^-1 by recursive block inversion, R = Z W.
-//           (R is the same orthogonal factor the reflectors would give; forming it
-//           as Z U^-1 costs one GEMM instead of d/32 dependent block updates.  Its
-//           orthogonality error grows like cond(Z) * 2^-16, which is fine for the
-//           near-orthogonal latents of the calibration loop.)
+// Forward:  U of Z = R U either by the blocked Householder factorisation (qr_panel_tc.cu kernels
+//           with the compact-WY products issued here) or, from the second step on, incrementally:
+//           U = (I + T) U_old with T from fixed-point sweeps on (Z U_old^-1)^T (Z U_old^-1).
+//           Then W = U^-1 by recursive block inversion and R = Z W.  (R is the same orthogonal
+//           factor the reflectors would give; forming it as Z U^-1 costs one GEMM instead of
+//           d / 128 dependent block updates.  Its orthogonality error grows like cond(Z) * 2^-17.)
 // Backward: B = R^T Gq, S = tril(B - B^T, -1), Gz = (R S) W^T.
-// All d x d products run as split-bf16 tcgen05 GEMMs (three bf16 MMAs per product,
-// fp32 accumulation, ~2^-16 relative error).
+// All d x d products run as split-bf16 tcgen05 GEMMs (three bf16 MMAs per product, fp32
+// accumulation, ~2^-17 relative error), clipped to the non-zero blocks of triangular operands.
 #include <algorithm>
 #include <vector>
 
@@ -47,23 +47,6 @@ __global__ void __launch_bounds__(256) split_kernel(const float* __restrict__ sr
       const int64_t i = (int64_t)(c0 + c) * n + r0 + tx;
       split2(t[tx][c], hi[i], lo[i]);
     }
-  }
-}
-
-// Gauge of the raw factor: U = diag(s) triu(A), s_i = sign(A_ii) (+1 at 0); fp32 + split copy.
-__global__ void __launch_bounds__(256) gauge_u_kernel(const float* __restrict__ A, float* __restrict__ U,
-                                                      bf16* __restrict__ hi, bf16* __restrict__ lo, int d) {
-  const int64_t off = (int64_t)blockIdx.z * d * d;
-  A += off; U += off; hi += off; lo += off;
-  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int r = ty; r < 32; r += 8) {
-    const int i = i0 + r, j = j0 + tx;
-    const float si = (A[(int64_t)i * d + i] < 0.f) ? -1.f : 1.f;
-    const float v = (j >= i) ? si * A[(int64_t)i * d + j] : 0.f;
-    const int64_t idx = (int64_t)i * d + j;
-    U[idx] = v;
-    split2(v, hi[idx], lo[idx]);
   }
 }
 
