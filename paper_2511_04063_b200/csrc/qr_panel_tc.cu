@@ -31,7 +31,7 @@ using bf16 = __nv_bfloat16;
 
 constexpr int IB = 32;     // inner panel width
 constexpr int OB = 128;    // outer block width
-constexpr int MAX_CS = 8;  // CTAs per cluster
+constexpr int MAX_CS = 16; // CTAs per cluster (8 is the portable limit; 16 where the device allows it)
 
 __device__ __forceinline__ void split2(float v, bf16& hi, bf16& lo) {
   hi = __float2bfloat16_rn(v);
@@ -625,7 +625,27 @@ dq_status qrp_panel(Ctx& ctx, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, b
                     int c0, int batch) {
   const int m = d - c0;
   if (m <= 0 || m % OB != 0 || m > 8192) return DQ_ERR_UNSUPPORTED;
-  const bool wide = m > 4096;                       // 1024 rows per CTA instead of 512
+  // 512 rows per CTA (two rows per thread, 255 registers) in clusters of up to 8; beyond 4096 rows
+  // either a cluster of 16 (non-portable size, if the device can co-schedule it) or 1024 rows per CTA.
+  static int can16 = -1;
+  if (m > 4096 && can16 < 0) {
+    can16 = 0;
+    auto kern = qr_panel_cm_kernel<256>;
+    using L = PanelSmem<8>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(16, 1, 1); cfg.blockDim = dim3(256, 1, 1); cfg.dynamicSmemBytes = L::BYTES;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 16; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      cfg.attrs = at; cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n >= 1) can16 = 1;
+    }
+    cudaGetLastError();
+  }
+  const bool wide = m > 4096 && can16 != 1;
   const int rows_per_cta = wide ? 1024 : 512;
   int cs = 1;
   while (cs * rows_per_cta < m) cs *= 2;
