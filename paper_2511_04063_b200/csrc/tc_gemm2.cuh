@@ -1,0 +1,259 @@
+// Two-CTA variant of the tcgen05 GEMM building block: a pair of CTAs on neighbouring SMs (a
+// cluster of two) computes one 256 x 256 output tile with `tcgen05.mma.cta_group::2`.
+//
+//   D[m][n] = sum_k A[m][k] * B[n][k]       (both operands K-major bf16, fp32 accumulate)
+//
+// Each CTA stages only its own half of the operands (128 rows of A, 128 rows of B: 32 KB per
+// 64-wide k-block instead of 48 KB) and owns the 128 x 256 accumulator rows of its half in its own
+// TMEM; the MMAs of both halves are issued by the even-ranked CTA ("leader"), which reads the
+// peer's operands from the same shared-memory offsets.  Protocol per CTA (192 threads as in the
+// one-CTA kernel):
+//   warp 0   TMA producer: waits on its own empty barrier (armed for both CTAs by the leader's
+//            multicast commit); both CTAs' loads complete on the LEADER's full barrier
+//   warp 1   leader only: MMA issue; commits multicast to both CTAs' empty / accumulator-full barriers
+//   warps 2..5  epilogue from the CTA's own TMEM; both CTAs arrive on the leader's accumulator-empty
+//            barrier
+// No TMA multicast is used.  Every wait is bounded (DQ_ERR_TIMEOUT in the status word on expiry).
+#pragma once
+#include "tc_gemm.cuh"
+
+namespace dq {
+namespace tc2 {
+
+using namespace tc;
+
+constexpr int PAIR_M = 256, PAIR_N = 256;
+constexpr int HALF = 128;
+constexpr int A_BYTES = HALF * BLOCK_K * 2;
+constexpr int B_BYTES = HALF * BLOCK_K * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // per CTA
+constexpr int STAGES = 6;
+constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + 1024 + 1024;
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;             // clears the bit that separates the two CTAs of a pair
+constexpr uint32_t TMEM_COLS = 512;                     // two 256-column accumulators
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Load a tile into this CTA's shared memory; the bytes are counted on the leader's barrier.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                                 int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_dst), "l"((uint64_t)map), "r"(bar & PEER_MASK), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  const uint32_t z = 0u;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8, %9, %10, %11, %12}, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(z), "r"(z), "r"(z), "r"(z), "r"(z), "r"(z),
+        "r"(z), "r"(z)
+      : "memory");
+}
+// One arrival on the barrier at this offset in BOTH CTAs once every MMA issued so far has completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+// Arrive on the leader's copy of a barrier (from either CTA of the pair).
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_MASK) : "memory");
+}
+// kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both K-major, M = 256 over the pair, N = 256.
+__host__ __device__ constexpr uint32_t make_idesc_bf16_pair() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(PAIR_N >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
+}
+
+// Params as in the one-CTA kernel; m_blocks / n_blocks count 256 x 256 pair tiles, tile_list entries
+// are mb | nb << 16 in those units, partials get eight values per tile (CTA rank, lane quarter).
+template <int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const Params p) {
+  constexpr uint32_t IDESC = make_idesc_bf16_pair();
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+  const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
+  uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader
+  const bool leader = rank == 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    prefetch_tensormap(&mapA);
+    prefetch_tensormap(&mapB);
+  }
+  if (warp == 1) tmem_alloc_pair(tmem_slot, TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                               // both CTAs' barriers exist before any remote arrival
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  const int tiles_per_batch = p.tile_list ? p.n_list : p.m_blocks * p.n_blocks;
+  auto tile_of = [&](int r, int& mb, int& nb) {
+    if (p.tile_list) { const int code = p.tile_list[r]; mb = code & 0xffff; nb = code >> 16; }
+    else { mb = r % p.m_blocks; nb = r / p.m_blocks; }
+  };
+  auto k_range = [&](int split, int& k0, int& kn) {
+    const int lo = (int)(((int64_t)split * p.k_blocks) / p.ksplit);
+    const int hi = (int)(((int64_t)(split + 1) * p.k_blocks) / p.ksplit);
+    k0 = lo; kn = hi - lo;
+  };
+  const int units = tiles_per_batch * p.batch * p.ksplit;
+  const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int u = pair; u < units && ok; u += pairs) {
+        const int split = u % p.ksplit;
+        const int t = u / p.ksplit;
+        const int b = t / tiles_per_batch;
+        int mb, nb;
+        tile_of(t % tiles_per_batch, mb, nb);
+        int k0, kn;
+        k_range(split, k0, kn);
+        for (int kb = 0; kb < kn; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
+          if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+          const int kc = (k0 + kb) * BLOCK_K;
+          tma_load_3d_pair(sa, &mapA, full_bar(stage), kc, mb * PAIR_M + (int)rank * HALF, b);
+          tma_load_3d_pair(sb, &mapB, full_bar(stage), kc, nb * PAIR_N + (int)rank * HALF, b);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------- MMA issuer (leader CTA only)
+    if (leader && lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int u = pair; u < units && ok; u += pairs) {
+        int k0, kn;
+        k_range(u % p.ksplit, k0, kn);
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * PAIR_N);
+        for (int kb = 0; kb < kn; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, p.d_status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+            umma_bf16_pair(tmem_d, make_kmajor_sw128_desc(sa + k * UMMA_K * 2), make_kmajor_sw128_desc(sb + k * UMMA_K * 2),
+                           IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit_pair(empty_bar(stage));      // both CTAs may refill this slot once the MMAs retire
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(tfull_bar(acc));          // accumulator complete in both CTAs
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------- epilogue (warps 2..5, both CTAs)
+    const int q = warp & 3;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int u = pair; u < units && ok; u += pairs) {
+      const int split = u % p.ksplit;
+      const int t = u / p.ksplit;
+      const int b = t / tiles_per_batch;
+      int mb, nb;
+      tile_of(t % tiles_per_batch, mb, nb);
+      if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
+      tc_fence_after();
+      const int row = mb * PAIR_M + (int)rank * HALF + q * 32 + lane;
+      const int64_t out_off = (int64_t)b * p.batch_stride + (int64_t)split * p.split_stride + (int64_t)row * p.ld +
+                              (int64_t)nb * PAIR_N;
+      float esum = 0.f;
+#pragma unroll 1
+      for (int c = 0; c < PAIR_N / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * PAIR_N + c * 32), v);
+        tmem_ld_wait();
+        if (EPI == EPI_WHIP) {
+          // Eq. 4: e = exp(-|o|); dL/do = -sign(o) e, zero at o = 0; 1/N is applied later.
+          uint32_t packed[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
+            const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
+            esum += e0 + e1;
+            const float g0 = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
+            const float g1 = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
+            const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
+            packed[i] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_off + c * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+        } else {   // EPI_GEN: fp32 store of alpha * acc
+          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_off + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            dst[i] = make_float4(p.alpha * __uint_as_float(v[4 * i]), p.alpha * __uint_as_float(v[4 * i + 1]),
+                                 p.alpha * __uint_as_float(v[4 * i + 2]), p.alpha * __uint_as_float(v[4 * i + 3]));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(tempty_bar(acc));   // eight arrivals (four warps of each CTA) free the accumulator
+      if (EPI == EPI_WHIP) {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) esum += __shfl_xor_sync(0xffffffffu, esum, off);
+        if (lane == 0) p.partials[((int64_t)u * 2 + rank) * 4 + q] = esum;
+      }
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                               // the peer has finished with its TMEM and barriers too
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace tc2
+}  // namespace dq

@@ -3,6 +3,7 @@
 // the launch wrapper of tc_gemm_kernel.
 #pragma once
 #include "tc_gemm.cuh"
+#include "tc_gemm2.cuh"
 
 namespace dq {
 namespace tch {
@@ -54,6 +55,33 @@ dq_status launch_gemm(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, cons
   int grid = units < ctx.sm_count ? units : ctx.sm_count;
   if (grid < 1) return DQ_OK;
   kern<<<grid, tc::NUM_THREADS, L::TOTAL, ctx.stream>>>(a, b, alo, blo, p);
+  return after_launch(ctx);
+}
+
+// Two-CTA kernel (tc_gemm2.cuh): p.m_blocks / p.n_blocks count 256 x 256 tiles; one cluster of two
+// CTAs per tile, at most one pair per two SMs.
+template <int EPI>
+dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, const tc::Params& p) {
+  static bool attr_set = false;
+  auto kern = tc2::tc_gemm2_kernel<EPI>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::SMEM_TOTAL) != cudaSuccess)
+      return DQ_ERR_CUDA;
+    attr_set = true;
+  }
+  const int units = (p.tile_list ? p.n_list : p.m_blocks * p.n_blocks) * p.batch * p.ksplit;
+  int pairs = units < ctx.sm_count / 2 ? units : ctx.sm_count / 2;
+  if (pairs < 1) return DQ_OK;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(tc::NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = tc2::SMEM_TOTAL;
+  cfg.stream = ctx.stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, a, b, p) != cudaSuccess) return DQ_ERR_CUDA;
   return after_launch(ctx);
 }
 

@@ -35,14 +35,14 @@ __global__ void __launch_bounds__(256) transpose_f32_to_bf16_kernel(const float*
 }
 
 // out tile = sum over slices of part[slice] tile, for the tiles of `list` (mb | nb << 16; tiles
-// are 128 x bn); one CTA per tile, fixed summation order.
+// are bm x bn); one CTA per tile, fixed summation order.
 __global__ void __launch_bounds__(256) tile_reduce_kernel(const float* __restrict__ part, int slices,
-                                                          int64_t slice_stride, const int* __restrict__ list, int bn,
-                                                          int d, float* __restrict__ out) {
+                                                          int64_t slice_stride, const int* __restrict__ list, int bm,
+                                                          int bn, int d, float* __restrict__ out) {
   const int code = list[blockIdx.x];
-  const int r0 = (code & 0xffff) * 128, c0 = (code >> 16) * bn;
+  const int r0 = (code & 0xffff) * bm, c0 = (code >> 16) * bn;
   const int per_row = bn / 4;
-  for (int e = threadIdx.x; e < 128 * per_row; e += 256) {
+  for (int e = threadIdx.x; e < bm * per_row; e += 256) {
     const int64_t idx = (int64_t)(r0 + e / per_row) * d + c0 + (e % per_row) * 4;
     float4 s = *reinterpret_cast<const float4*>(part + idx);
     for (int k = 1; k < slices; ++k) {
@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(256) tile_reduce_kernel(const float* __restric
 }
 
 struct Maps {
-  CUtensorMap rt, x, xt, gt128, gt256;
+  CUtensorMap rt, x, x128, xt, gt128, gt256;
 };
 
 }  // namespace
@@ -74,17 +74,20 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   }
   // split-K of Gq = X^T G over the token dimension: fill the machine, keep >= 16 k-blocks per slice
   const int bn = (d % 256 == 0) ? 256 : 128;
-  const int tiles = (d / tc::BLOCK_M) * (d / bn) * batch;
+  tc.pair = (d % 256 == 0) && ctx.sm_count >= 2;
+  const int bm = tc.pair ? 256 : tc::BLOCK_M;
+  const int n_cta_units = tc.pair ? ctx.sm_count / 2 : ctx.sm_count;   // tiles computed at a time
+  const int tiles = (d / bm) * (d / bn) * batch;
   int ks = 1;
-  while (tiles * ks < ctx.sm_count && (N / tc::BLOCK_K) / (ks * 2) >= 16 && ks < 64) ks *= 2;
+  while (tiles * ks < n_cta_units && (N / tc::BLOCK_K) / (ks * 2) >= 16 && ks < 64) ks *= 2;
   tc.ksplit = ks;
   if (ks > 1 &&
       cudaMalloc((void**)&tc.part, sizeof(float) * (size_t)batch * ks * d * d) != cudaSuccess)
     return DQ_ERR_ALLOC;
-  if (ks == 1 && batch == 1 && tiles > ctx.sm_count && tiles % ctx.sm_count != 0) {
+  if (ks == 1 && batch == 1 && tiles > n_cta_units && tiles % n_cta_units != 0) {
     // a partly filled last wave: split its reduction so that it fills the machine once more
-    const int rem = tiles % ctx.sm_count, full = tiles - rem, mbk = d / tc::BLOCK_M;
-    int sp = ctx.sm_count / rem;
+    const int rem = tiles % n_cta_units, full = tiles - rem, mbk = d / bm;
+    int sp = n_cta_units / rem;
     if (sp > 4) sp = 4;
     while (sp > 1 && (N / tc::BLOCK_K) / sp < 16) --sp;
     if (sp > 1) {
@@ -104,6 +107,7 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   tc.maps = m;
   DQ_CHECK(tch::make_map(&m->rt, tc.Rt, d, d, batch, d, (int64_t)d * d, tc::BLOCK_M));
   DQ_CHECK(tch::make_map(&m->x, tc.X, d, N, batch, d, N * d, 256));
+  DQ_CHECK(tch::make_map(&m->x128, tc.X, d, N, batch, d, N * d, 128));
   DQ_CHECK(tch::make_map(&m->xt, tc.Xt, N, d, batch, N, N * d, tc::BLOCK_M));
   DQ_CHECK(tch::make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
   DQ_CHECK(tch::make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
@@ -137,6 +141,10 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
   p.k_blocks = tc.d / tc::BLOCK_K;
   p.out = tc.Gt; p.ld = tc.n_tokens; p.batch_stride = tc.n_tokens * tc.d; p.split_stride = 0;
   p.alpha = 1.f; p.partials = partials; p.d_status = ctx.d_status;
+  if (tc.pair) {   // 256 channels x 256 tokens per CTA pair
+    p.m_blocks = tc.d / 256;
+    return tch::launch_gemm2<tc::EPI_WHIP>(ctx, m->rt, m->x128, p);
+  }
   return tch::launch_gemm<256, 1, tc::EPI_WHIP>(ctx, m->rt, m->x, m->rt, m->x, p);
 }
 
@@ -155,7 +163,9 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
   } else {
     p.out = tc.part; p.batch_stride = (int64_t)tc.ksplit * d * d; p.split_stride = (int64_t)d * d;
   }
+  if (tc.pair) p.m_blocks = d / 256;
   auto launch = [&](const tc::Params& pp) {
+    if (tc.pair) return tch::launch_gemm2<tc::EPI_GEN>(ctx, m->xt, m->gt128, pp);
     return (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, m->xt, m->gt256, m->xt, m->gt256, pp)
                        : tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, pp);
   };
@@ -167,8 +177,8 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
     pt.tile_list = tc.tl_tail; pt.n_list = tc.n_tail; pt.ksplit = tc.tail_split;
     pt.out = tc.tail_part; pt.batch_stride = 0; pt.split_stride = (int64_t)d * d;
     DQ_CHECK(launch(pt));
-    tile_reduce_kernel<<<tc.n_tail, 256, 0, ctx.stream>>>(tc.tail_part, tc.tail_split, (int64_t)d * d, tc.tl_tail, bn,
-                                                          d, Gq);
+    tile_reduce_kernel<<<tc.n_tail, 256, 0, ctx.stream>>>(tc.tail_part, tc.tail_split, (int64_t)d * d, tc.tl_tail,
+                                                          tc.pair ? 256 : 128, bn, d, Gq);
     return after_launch(ctx);
   }
   DQ_CHECK(launch(p));

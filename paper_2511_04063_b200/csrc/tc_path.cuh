@@ -17,6 +17,7 @@ struct TcState {
   int ksplit = 1;
   void* maps = nullptr;               // host array of CUtensorMap
   int n_partials = 0;
+  bool pair = false;                  // 256 x 256 tiles on CTA pairs (tcgen05 cta_group::2) for both contractions
   // Gq = X^T G when the tile count is not a multiple of the SM count: the last, partly filled
   // wave of tiles is computed with its reduction split in `tail_split` slices instead
   int* tl_head = nullptr; int n_head = 0;
