@@ -32,7 +32,7 @@ UNIT = "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic of one launch of the forward kernel on the c2_7b workload, from the ncu
 # capture summarised in profiles/ (bytes read + written); None until captured.
-NCU_TRAFFIC_BYTES = {"c2_7b": 293.0e6}   # profiles/tc_gemm_whip_forward_c2_7b.md
+NCU_TRAFFIC_BYTES = {"c2_7b": 313.0e6}   # profiles/tc_gemm_whip_forward_c2_7b.md
 
 
 def load_peaks():
@@ -276,7 +276,7 @@ def main():
         peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) if capped else peaks["bf16_tflops"]
         gemm_tflops = 2 * fwd_flops / (t_fwd + t_bwd) / 1e12 if (t_fwd + t_bwd) > 0 else 0.0
         total_phase = sum(phases.values())
-        roofline = {"bound": "tensor", "kernel": "tc_gemm_kernel<256,1,WHIP> (O^T = R^T X^T, Eq. 4 epilogue)"
+        roofline = {"bound": "tensor", "kernel": ("tc_gemm2_kernel<WHIP>" if d % 256 == 0 else "tc_gemm_kernel<256,1,WHIP>") + " (O^T = R^T X^T, Eq. 4 epilogue)"
                     if path == dq.DQ_PATH_BF16_TC else "gemm_ffma_kernel<WHIP>",
                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                     "peak_source": "%s (%s bf16 matmul peak)" % (peaks["_source"], "sustained" if capped else "burst"),
