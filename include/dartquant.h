@@ -158,6 +158,26 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 
+/* Which orthogonal optimiser updates the rotation.
+ *   DQ_ORTH_QR (default): QR-Orth (Sec. 4.3): a free latent Z with R = the orthogonal factor of Z.
+ *   DQ_ORTH_CAYLEY: Cayley SGD with momentum (Algorithm 3), the optimiser Sec. 5.3 and Table 4
+ *     compare QR-Orth with.  The iterate is the rotation itself (X_1 = the orthogonal factor of the
+ *     current latent, computed once); each dq_calib_step iteration computes the same loss and
+ *     dL/dR as QR-Orth and then
+ *       M <- beta M - dL/dR;  What = M R^T - R (R^T M R^T) / 2;  W = What - What^T;  M <- W R;
+ *       a = min(lr, 2 q / (|W|_F + 1e-8));  Y^0 = R + a M;  Y^i = R + a/2 W (R + Y^(i-1)), i = 1..s;
+ *       R <- Y^s
+ *     with lr the handle's learning rate, six d x d tensor-core products per iteration.  The
+ *     skew-symmetrisation is read as What - What^T and the norm as the Frobenius norm (Algorithm 3
+ *     prints W on both sides of that step and does not name the norm).  q <= 0 selects 0.5, s <= 0 selects 2.
+ *     The latent Z, the QR method and dq_calib_set_optimizer's choice are not used in this mode;
+ *     dq_calib_get_rotation returns the iterate.  Selecting a method resets the momentum, and the
+ *     next step starts again from the orthogonal factor of the latent.
+ * Errors: INVALID_ARG (bad enum, beta outside [0, 1), q > 1, s > 16), UNSUPPORTED (fp32 path or
+ * d == 128: only the tensor-core path with d >= 256 implements it), ALLOC, CUDA. */
+enum { DQ_ORTH_QR = 0, DQ_ORTH_CAYLEY = 1 };
+dq_status dq_calib_set_orth_method(dq_calib_t* h, int32_t method, float beta, float q, int32_t s);
+
 /* Checkpoint / resume of the optimised parameter (Algorithm 1: Z <- Z0). */
 dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out);
 dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z);
@@ -193,7 +213,9 @@ enum {
   DQ_BUF_PARTIALS = 5, /* fp32 per-tile loss partial sums of the last step         */
   DQ_BUF_Z = 6,        /* fp32 [batch][d][d]  current latent                       */
   DQ_BUF_OPT_M = 7,    /* fp32 [batch][d][d]  first moment / velocity (NULL for DQ_SGD)  */
-  DQ_BUF_OPT_V = 8     /* fp32 [batch][d][d]  second moment (DQ_ADAM only)         */
+  DQ_BUF_OPT_V = 8,    /* fp32 [batch][d][d]  second moment (DQ_ADAM only)         */
+  DQ_BUF_CAYLEY_M = 9, /* fp32 [batch][d][d]  momentum of DQ_ORTH_CAYLEY            */
+  DQ_BUF_CAYLEY_ALPHA = 10 /* fp32 [batch]    step size of the last Cayley iteration */
 };
 dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int64_t* n_elems);
 

@@ -15,18 +15,21 @@ LIB_PATH = os.path.join(HERE, "libdartquant.so")
 DQ_OK, DQ_ERR_INVALID_ARG, DQ_ERR_UNSUPPORTED, DQ_ERR_ALLOC, DQ_ERR_CUDA = 0, 1, 2, 3, 4
 DQ_ERR_SINGULAR, DQ_ERR_NONFINITE, DQ_ERR_TIMEOUT, DQ_ERR_NOT_CONVERGED = 5, 6, 7, 8
 DQ_QR_HOUSEHOLDER, DQ_QR_ITERATIVE = 0, 1
+DQ_ORTH_QR, DQ_ORTH_CAYLEY = 0, 1
 DQ_FP32, DQ_BF16 = 0, 1
 DQ_PATH_FP32, DQ_PATH_BF16_TC = 0, 1
 DQ_MEAN_TOKENS, DQ_SUM_TOKENS = 0, 1
 DQ_SGD, DQ_SGD_MOMENTUM, DQ_ADAM = 0, 1, 2
 DQ_PHASE_NAMES = ("qr_forward", "rotate_whip", "grad_rotation", "qr_backward", "update")
 DQ_BUF_R, DQ_BUF_U, DQ_BUF_GQ, DQ_BUF_GZ, DQ_BUF_G, DQ_BUF_PARTIALS, DQ_BUF_Z, DQ_BUF_OPT_M, DQ_BUF_OPT_V = range(9)
+DQ_BUF_CAYLEY_M, DQ_BUF_CAYLEY_ALPHA = 9, 10
 
 EXPORTED_SYMBOLS = (
     "dq_calib_init", "dq_calib_step", "dq_calib_get_rotation", "dq_rotate_apply",
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
     "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens", "dq_eval_rotation",
+    "dq_calib_set_orth_method",
 )
 
 
@@ -65,6 +68,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_set_optimizer.restype = i32
     lib.dq_calib_set_qr_method.argtypes = [vp, i32, i32]
     lib.dq_calib_set_qr_method.restype = i32
+    lib.dq_calib_set_orth_method.argtypes = [vp, i32, C.c_float, C.c_float, i32]
+    lib.dq_calib_set_orth_method.restype = i32
     lib.dq_gather_tokens.argtypes = [vp, i32, i64, i32, i64, C.c_uint64, i64, i64, vp, i64, vp]
     lib.dq_gather_tokens.restype = i32
     lib.dq_eval_rotation.argtypes = [vp, i32, i64, i32, i64, vp, C.c_float, i32, vp, vp]
@@ -165,6 +170,10 @@ def dq_calib_set_optimizer(h, optimizer: int, lr: float, beta1: float = 0.9, bet
 
 def dq_calib_set_qr_method(h, method: int, n_iters: int = 0):
     _check(load_library().dq_calib_set_qr_method(h, method, n_iters), "dq_calib_set_qr_method")
+
+
+def dq_calib_set_orth_method(h, method: int, beta: float = 0.0, q: float = 0.0, s: int = 0):
+    _check(load_library().dq_calib_set_orth_method(h, method, beta, q, s), "dq_calib_set_orth_method")
 
 
 def dq_calib_get_timings(h) -> dict:

@@ -41,6 +41,9 @@ struct dq_calib {
   float* opt_m = nullptr;       // first moment / velocity
   float* opt_v = nullptr;       // second moment
   float* opt_pw = nullptr;      // device float[2]: beta1^t, beta2^t
+  int orth_method = DQ_ORTH_QR;
+  CayleyState cay;              // DQ_ORTH_CAYLEY: momentum and step size
+  bool cay_started = false;     // R and its split copies hold the Cayley iterate
   bool small128 = false;        // d == 128: shared-memory-resident batched QR-Orth
   bool r_stale = true;
   bool timing = false;
@@ -68,6 +71,7 @@ void free_all(dq_calib* h) {
   if (h->graph) cudaGraphExecDestroy(h->graph);
   tc_destroy(h->tc);
   qr_tc_destroy(h->qtc);
+  cayley_destroy(h->cay);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
   cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw);
   cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->ctx.d_status);
@@ -112,6 +116,7 @@ dq_status fence_out(dq_calib* h) {
 }
 
 dq_status ensure_rotation(dq_calib* h) {
+  if (h->orth_method == DQ_ORTH_CAYLEY && h->cay_started) return DQ_OK;   // R is the iterate itself
   if (!h->r_stale) return DQ_OK;
   if (h->small128) {
     DQ_CHECK(qr128_forward(h->ctx, h->Z, h->R, h->U, h->ws.Winv,
@@ -134,8 +139,9 @@ dq_status enqueue_step(dq_calib* h, bool timed) {
   const float inv_n = (c.reduction == DQ_MEAN_TOKENS) ? (float)(1.0 / (double)N) : 1.f;
   Ctx& ctx = h->ctx;
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[0], ctx.stream));
-  // (a1) R <- qr(Z)
-  DQ_CHECK(ensure_rotation(h));
+  const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
+  // (a1) R <- qr(Z)   (Cayley SGD: only to obtain the first iterate)
+  if (!cayley || !h->cay_started) DQ_CHECK(ensure_rotation(h));
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[1], ctx.stream));
   // (a2-a4) O = X R, Whip epilogue, loss reduction
   if (c.path == DQ_PATH_FP32) {
@@ -167,6 +173,16 @@ dq_status enqueue_step(dq_calib* h, bool timed) {
   // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
   // (a7) Z <- Z - lr Gz  (fused into the backward kernel for 128 x 128 latents)
   const int64_t n_latent = (int64_t)d * d * batch;
+  if (cayley) {   // Algorithm 3 updates the rotation itself; there is no latent
+    DQ_CHECK(cayley_step_tc(ctx, h->ws, h->qtc, h->cay, h->R, h->Gq, c.lr, d, batch));
+    h->cay_started = true;
+    h->r_stale = false;
+    if (timed) {
+      DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
+      DQ_CHECK_CUDA(cudaEventRecord(h->ev[5], ctx.stream));
+    }
+    return DQ_OK;
+  }
   if (h->small128) {   // plain SGD is fused into the backward kernel; other optimisers follow it
     DQ_CHECK(qr128_backward_sgd(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, h->optimizer == DQ_SGD ? c.lr : 0.f, batch));
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
@@ -320,12 +336,15 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
     // The captured step of the iterative QR is the incremental one: replay it only while the
     // previous step's factors belong to the latent one optimiser step back.
     const bool iterative = h->fast_qr && !h->small128 && h->qr_method == DQ_QR_ITERATIVE;
-    const bool use_graph = !h->timing && h->r_stale && h->eager_steps_done >= 1 && (!iterative || h->qtc.t_warm);
+    const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
+    const bool use_graph = cayley ? (!h->timing && h->cay_started && h->eager_steps_done >= 1)
+                                  : (!h->timing && h->r_stale && h->eager_steps_done >= 1 &&
+                                     (!iterative || h->qtc.t_warm));
     if (use_graph && !h->graph && !h->graph_failed) try_capture(h);
     if (use_graph && h->graph) {
       DQ_CHECK_CUDA(cudaGraphLaunch(h->graph, ctx.stream));
       ctx.launches += h->graph_launches;
-      h->r_stale = true;
+      h->r_stale = !cayley;
     } else {
       DQ_CHECK(enqueue_step(h, h->timing));
       h->eager_steps_done++;
@@ -378,6 +397,7 @@ dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z) {
                                 cudaMemcpyDeviceToDevice, h->ctx.stream));
   h->r_stale = true;
   h->qtc.t_warm = false;   // the new latent may be far from the one the iterative QR last saw
+  h->cay_started = false;  // Cayley SGD restarts from the orthogonal factor of the new latent
   return fence_out(h);
 }
 
@@ -430,6 +450,34 @@ dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters)
   return DQ_OK;
 }
 
+dq_status dq_calib_set_orth_method(dq_calib_t* h, int32_t method, float beta, float q, int32_t s) {
+  if (!h || (method != DQ_ORTH_QR && method != DQ_ORTH_CAYLEY)) return DQ_ERR_INVALID_ARG;
+  if (method == DQ_ORTH_CAYLEY) {
+    if (!(beta >= 0.f && beta < 1.f) || q > 1.f || s > 16) return DQ_ERR_INVALID_ARG;
+    if (!h->fast_qr || h->small128) return DQ_ERR_UNSUPPORTED;
+  }
+  DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
+  if (method == DQ_ORTH_CAYLEY) {
+    if (!h->cay.ready) {
+      const dq_status st = cayley_init(h->cay, h->cfg.d, h->cfg.batch);
+      if (st != DQ_OK) { cayley_destroy(h->cay); return st; }
+    }
+    h->cay.beta = beta;
+    h->cay.q = q > 0.f ? q : 0.5f;
+    h->cay.s = s > 0 ? s : 2;
+    DQ_CHECK_CUDA(cudaMemsetAsync(h->cay.M, 0, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
+                                  h->ctx.stream));
+    DQ_CHECK_CUDA(cudaMemsetAsync(h->cay.alpha, 0, sizeof(float) * h->cfg.batch, h->ctx.stream));
+  }
+  h->orth_method = method;
+  h->cay_started = false;
+  h->r_stale = true;
+  h->qtc.t_warm = false;
+  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
+  h->graph_failed = false;
+  return DQ_OK;
+}
+
 dq_status dq_calib_set_timing(dq_calib_t* h, int32_t enabled) {
   if (!h) return DQ_ERR_INVALID_ARG;
   h->timing = enabled != 0;
@@ -456,6 +504,8 @@ dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int6
     case DQ_BUF_Z: *d_ptr = h->Z; *n_elems = dd; break;
     case DQ_BUF_OPT_M: *d_ptr = h->opt_m; *n_elems = h->opt_m ? dd : 0; break;
     case DQ_BUF_OPT_V: *d_ptr = h->opt_v; *n_elems = h->opt_v ? dd : 0; break;
+    case DQ_BUF_CAYLEY_M: *d_ptr = h->cay.M; *n_elems = h->cay.M ? dd : 0; break;
+    case DQ_BUF_CAYLEY_ALPHA: *d_ptr = h->cay.alpha; *n_elems = h->cay.alpha ? h->cfg.batch : 0; break;
     default: return DQ_ERR_INVALID_ARG;
   }
   return DQ_OK;

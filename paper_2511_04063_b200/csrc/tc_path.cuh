@@ -79,6 +79,23 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
                           int batch, int iterative_iters);
 dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch);
 
+// Cayley SGD with momentum (Algorithm 3) on the rotation itself (cayley_tc.cu).
+struct CayleyState {
+  bool ready = false;
+  float* M = nullptr;        // [batch][d][d] momentum
+  float* part = nullptr;     // [batch][n_part] partial sums of |W|_F^2
+  float* alpha = nullptr;    // [batch] step size of the current iteration
+  int n_part = 0;
+  float beta = 0.f, q = 0.5f, eps = 1e-8f;
+  int s = 2;
+};
+dq_status cayley_init(CayleyState& cs, int d, int batch);
+void cayley_destroy(CayleyState& cs);
+// One update R <- Cayley step of (R, M, Gq); needs q.r_* / q.rt_* to hold the split copies of R and
+// leaves them holding those of the new R.  Uses ws.B, ws.S, ws.tmp and the split scratch of q.
+dq_status cayley_step_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, CayleyState& cs, float* R, const float* Gq,
+                         float lr, int d, int batch);
+
 
 // Kernels of the blocked Householder factorisation on a transposed working matrix
 // (qr_panel_tc.cu); the tensor-core products between them are issued by qr_tc.cu.
