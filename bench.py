@@ -240,6 +240,27 @@ def main():
         alt = {"ms_per_step": ms_alt / K, "phases_ms": phases_alt}
         dq.dq_calib_set_qr_method(h, dq.DQ_QR_HOUSEHOLDER, 0)
 
+    # ---------------------------------------------------------------- same contractions, Cayley SGD (Algorithm 3)
+    cay = None
+    if path == dq.DQ_PATH_BF16_TC and wr.d != 128:
+        dq.dq_calib_set_orth_method(h, dq.DQ_ORTH_CAYLEY, 0.9)
+        dq.dq_calib_step(h, W, loss_dev)
+        barrier()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        dq.dq_calib_step(h, K, loss_dev)
+        c1.record()
+        barrier()
+        ms_cay = c0.elapsed_time(c1)
+        dq.dq_calib_set_timing(h, True)
+        dq.dq_calib_step(h, n_phase_steps, loss_dev)
+        phases_cay = dq.dq_calib_get_timings(h)
+        dq.dq_calib_set_timing(h, False)
+        st = dq.dq_calib_status(h)
+        assert st == dq.DQ_OK, dq.status_string(st)
+        cay = {"ms_per_step": ms_cay / K, "update_ms": phases_cay["qr_backward"]}
+        dq.dq_calib_set_orth_method(h, dq.DQ_ORTH_QR)
+
     # ---------------------------------------------------------------- end to end (host buffers)
     loss_host = torch.empty((1, wr.batch), dtype=torch.float32).pin_memory()
     Ke = min(K, 10)
@@ -316,6 +337,13 @@ def main():
             line["qr_iterative"] = {"value": world * 1e3 / alt["ms_per_step"], "unit": UNIT,
                                     "ms_per_step": alt["ms_per_step"], "phases_ms": alt["phases_ms"],
                                     "qr_orth_share": (alt["phases_ms"]["qr_forward"] + alt["phases_ms"]["qr_backward"]) / ta}
+        if cay is not None:
+            # Table 4's comparison on this GPU: the same loss and dL/dR, rotation updated by Cayley SGD with
+            # momentum (six d x d split-bf16 products, 12 d^3 flops, three bf16 MMAs per product)
+            line["cayley_sgd"] = {"value": world * 1e3 / cay["ms_per_step"], "unit": UNIT,
+                                  "ms_per_step": cay["ms_per_step"], "update_ms": cay["update_ms"],
+                                  "update_mma_tflops": 3 * 12.0 * d ** 3 * B / (cay["update_ms"] * 1e-3) / 1e12
+                                  if cay["update_ms"] > 0 else None}
         if not args.no_cpu_baseline and world == 1:
             shrink = 4 if d >= 2048 else 1
             v, dt, cores, sample = oracle_sample_steps_per_s(w, 2 if shrink > 1 else 3, shrink)
