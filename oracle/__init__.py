@@ -12,3 +12,4 @@ from .calib_oracle import (  # noqa: F401
 from .token_sampling import philox4x32_10, permute_index, gather_tokens  # noqa: F401,E402
 from .eval_metrics import outlier_count, quantize_per_token_asymmetric, quantization_mse  # noqa: F401,E402
 from .cayley_oracle import cayley_sgd_step, cayley_calib_step, cayley_calib_run  # noqa: F401,E402
+from . import objectives  # noqa: F401,E402
