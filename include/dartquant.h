@@ -158,6 +158,24 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 
+/* The calibration objective.  DQ_OBJ_WHIP (default) is Eq. 4.  The other three are the objectives the
+ * ablation of Sec. 5.3 compares it with; the paper names them without formulas, so they are read as
+ * per-token statistics over the d channels of the rotated token o = x R (as Eq. 4 is per token),
+ * averaged over tokens like the Whip loss (or summed, with DQ_SUM_TOKENS):
+ *   DQ_OBJ_VARIANCE: (1/d) sum_j (o_j - mean(o))^2
+ *   DQ_OBJ_KURTOSIS: m4 / m2^2 - 3 with m_p = (1/d) sum_j (o_j - mean(o))^p   (excess kurtosis)
+ *   DQ_OBJ_QUANT:    (1/d) sum_j (o_j - Q(o)_j)^2, Q = per-token asymmetric uniform quantiser to `bits`
+ *                    bits (the one of dq_eval_rotation); derivative with the grid held fixed and rounding
+ *                    piecewise constant: (2/d) (o_j - Q(o)_j)
+ * These need statistics of the whole token before any entry of dL/dO, so the rotated activations are
+ * materialised chunk by chunk in fp32 instead of staying in tensor memory; everything after dL/dO
+ * (contraction with X, QR backward or Cayley update, optimiser) is unchanged.  bits: 1..16, <= 0 selects
+ * 4; ignored unless DQ_OBJ_QUANT.  A token whose rotated entries are all equal makes the kurtosis
+ * undefined: the loss becomes non-finite and the status word DQ_ERR_NONFINITE.
+ * Errors: INVALID_ARG (bad enum, bits > 16), ALLOC, CUDA. */
+enum { DQ_OBJ_WHIP = 0, DQ_OBJ_VARIANCE = 1, DQ_OBJ_KURTOSIS = 2, DQ_OBJ_QUANT = 3 };
+dq_status dq_calib_set_objective(dq_calib_t* h, int32_t objective, int32_t bits);
+
 /* Which orthogonal optimiser updates the rotation.
  *   DQ_ORTH_QR (default): QR-Orth (Sec. 4.3): a free latent Z with R = the orthogonal factor of Z.
  *   DQ_ORTH_CAYLEY: Cayley SGD with momentum (Algorithm 3), the optimiser Sec. 5.3 and Table 4

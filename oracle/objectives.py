@@ -60,8 +60,29 @@ def loss(O: np.ndarray, objective: str, reduction: str = "mean", bits: int = 4) 
     raise ValueError(reduction)
 
 
-def grad_wrt_output(O: np.ndarray, objective: str, reduction: str = "mean", bits: int = 4) -> np.ndarray:
-    """G = dL/dO (N x d)."""
+def quant_grid(O: np.ndarray, bits: int):
+    """Per-token grid of the asymmetric uniform quantiser: (scale, zero, codes), scale = 0 on a
+    constant row (which is reproduced exactly)."""
+    O = np.asarray(O, dtype=F64)
+    maxq = float(2 ** bits - 1)
+    lo = O.min(axis=1, keepdims=True)
+    hi = O.max(axis=1, keepdims=True)
+    scale = (hi - lo) / maxq
+    safe = np.where(scale == 0.0, 1.0, scale)
+    zero = np.rint(-lo / safe)
+    codes = np.clip(np.rint(O / safe) + zero, 0.0, maxq)
+    return scale, zero, codes
+
+
+def grad_wrt_output(O: np.ndarray, objective: str, reduction: str = "mean", bits: int = 4,
+                    code_decider=None) -> np.ndarray:
+    """G = dL/dO (N x d).
+
+    The quantiser's code rint(o / scale) + zero is a discrete decision taken on a floating-point
+    value: an implementation in lower precision may legitimately take the neighbouring code for an
+    entry that sits on a rounding boundary.  code_decider(O, scale, zero, codes) -> codes lets a test
+    take that decision in the precision of the implementation under test (as sign_decider does for
+    the kink of Eq. 4); the derivative formula itself is unchanged."""
     O = np.asarray(O, dtype=F64)
     n, d = O.shape
     if objective == "variance":
@@ -75,19 +96,24 @@ def grad_wrt_output(O: np.ndarray, objective: str, reduction: str = "mean", bits
         # dm4/do_j = (4/d)(c_j^3 - m3), dm2/do_j = (2/d) c_j
         G = (4.0 / d) * ((C ** 3 - m3) / m2 ** 2 - m4 * C / m2 ** 3)
     elif objective == "quant":
-        G = 2.0 * (O - quantize_per_token_asymmetric(O, bits)) / d
+        if code_decider is None:
+            G = 2.0 * (O - quantize_per_token_asymmetric(O, bits)) / d
+        else:
+            scale, zero, codes = quant_grid(O, bits)
+            codes = code_decider(O, scale, zero, codes)
+            G = np.where(scale == 0.0, 0.0, 2.0 * (O - scale * (codes - zero)) / d)
     else:
         raise ValueError(objective)
     return G / n if reduction == "mean" else G
 
 
 def objective_step(X: np.ndarray, Z: np.ndarray, lr: float, objective: str, reduction: str = "mean",
-                   bits: int = 4, qr=co.qr_pos):
+                   bits: int = 4, qr=co.qr_pos, code_decider=None):
     """One pass of the loop body of Algorithm 1 with the Whip loss replaced by `objective`."""
     R, U = qr(Z)
     O = co.rotate(X, R)
     L = loss(O, objective, reduction, bits)
-    G = grad_wrt_output(O, objective, reduction, bits)
+    G = grad_wrt_output(O, objective, reduction, bits, code_decider)
     Gq = co.grad_wrt_rotation(X, G)
     Gz = co.qr_backward(R, U, Gq)
     return {"R": R, "U": U, "O": O, "loss": L, "G": G, "Gq": Gq, "Gz": Gz, "Z_new": co.sgd_step(Z, Gz, lr)}

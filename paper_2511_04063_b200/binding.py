@@ -16,6 +16,7 @@ DQ_OK, DQ_ERR_INVALID_ARG, DQ_ERR_UNSUPPORTED, DQ_ERR_ALLOC, DQ_ERR_CUDA = 0, 1,
 DQ_ERR_SINGULAR, DQ_ERR_NONFINITE, DQ_ERR_TIMEOUT, DQ_ERR_NOT_CONVERGED = 5, 6, 7, 8
 DQ_QR_HOUSEHOLDER, DQ_QR_ITERATIVE = 0, 1
 DQ_ORTH_QR, DQ_ORTH_CAYLEY = 0, 1
+DQ_OBJ_WHIP, DQ_OBJ_VARIANCE, DQ_OBJ_KURTOSIS, DQ_OBJ_QUANT = 0, 1, 2, 3
 DQ_FP32, DQ_BF16 = 0, 1
 DQ_PATH_FP32, DQ_PATH_BF16_TC = 0, 1
 DQ_MEAN_TOKENS, DQ_SUM_TOKENS = 0, 1
@@ -29,7 +30,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
     "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens", "dq_eval_rotation",
-    "dq_calib_set_orth_method",
+    "dq_calib_set_orth_method", "dq_calib_set_objective",
 )
 
 
@@ -68,6 +69,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_set_optimizer.restype = i32
     lib.dq_calib_set_qr_method.argtypes = [vp, i32, i32]
     lib.dq_calib_set_qr_method.restype = i32
+    lib.dq_calib_set_objective.argtypes = [vp, i32, i32]
+    lib.dq_calib_set_objective.restype = i32
     lib.dq_calib_set_orth_method.argtypes = [vp, i32, C.c_float, C.c_float, i32]
     lib.dq_calib_set_orth_method.restype = i32
     lib.dq_gather_tokens.argtypes = [vp, i32, i64, i32, i64, C.c_uint64, i64, i64, vp, i64, vp]
@@ -170,6 +173,10 @@ def dq_calib_set_optimizer(h, optimizer: int, lr: float, beta1: float = 0.9, bet
 
 def dq_calib_set_qr_method(h, method: int, n_iters: int = 0):
     _check(load_library().dq_calib_set_qr_method(h, method, n_iters), "dq_calib_set_qr_method")
+
+
+def dq_calib_set_objective(h, objective: int, bits: int = 0):
+    _check(load_library().dq_calib_set_objective(h, objective, bits), "dq_calib_set_objective")
 
 
 def dq_calib_set_orth_method(h, method: int, beta: float = 0.0, q: float = 0.0, s: int = 0):

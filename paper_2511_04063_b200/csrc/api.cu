@@ -41,6 +41,7 @@ struct dq_calib {
   float* opt_m = nullptr;       // first moment / velocity
   float* opt_v = nullptr;       // second moment
   float* opt_pw = nullptr;      // device float[2]: beta1^t, beta2^t
+  ObjectiveState obj;           // objectives other than Eq. 4
   int orth_method = DQ_ORTH_QR;
   CayleyState cay;              // DQ_ORTH_CAYLEY: momentum and step size
   bool cay_started = false;     // R and its split copies hold the Cayley iterate
@@ -72,6 +73,7 @@ void free_all(dq_calib* h) {
   tc_destroy(h->tc);
   qr_tc_destroy(h->qtc);
   cayley_destroy(h->cay);
+  objective_destroy(h->obj);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
   cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw);
   cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->ctx.d_status);
@@ -144,13 +146,18 @@ dq_status enqueue_step(dq_calib* h, bool timed) {
   if (!cayley || !h->cay_started) DQ_CHECK(ensure_rotation(h));
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[1], ctx.stream));
   // (a2-a4) O = X R, Whip epilogue, loss reduction
-  if (c.path == DQ_PATH_FP32) {
-    DQ_CHECK(whip_forward_f32(ctx, (const float*)h->X, c.ldx, N * c.ldx, h->R, (float*)h->G, h->partials, N, d,
-                              batch, nullptr));
+  if (h->obj.objective != DQ_OBJ_WHIP) {   // ablation objectives: per-token statistics, materialised O
+    DQ_CHECK(objective_forward(ctx, h->obj, c, h->X, h->R, c.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr, h->G,
+                               inv_n, h->loss_last));
   } else {
-    DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
+    if (c.path == DQ_PATH_FP32) {
+      DQ_CHECK(whip_forward_f32(ctx, (const float*)h->X, c.ldx, N * c.ldx, h->R, (float*)h->G, h->partials, N, d,
+                                batch, nullptr));
+    } else {
+      DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
+    }
+    DQ_CHECK(loss_finalize(ctx, h->partials, h->n_partials, batch, inv_n, nullptr, h->loss_last));
   }
-  DQ_CHECK(loss_finalize(ctx, h->partials, h->n_partials, batch, inv_n, nullptr, h->loss_last));
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[2], ctx.stream));
   // (a5) Gq = (1/N) X^T G
   if (c.path == DQ_PATH_FP32) {
@@ -445,6 +452,20 @@ dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters)
   h->qr_iters = iters;
   h->r_stale = true;
   h->qtc.t_warm = false;
+  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
+  h->graph_failed = false;
+  return DQ_OK;
+}
+
+dq_status dq_calib_set_objective(dq_calib_t* h, int32_t objective, int32_t bits) {
+  if (!h || objective < DQ_OBJ_WHIP || objective > DQ_OBJ_QUANT || bits > 16) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
+  if (objective != DQ_OBJ_WHIP && !h->obj.ready) {
+    const dq_status st = objective_init(h->obj, h->cfg.d, h->cfg.n_tokens, h->cfg.batch);
+    if (st != DQ_OK) { objective_destroy(h->obj); return st; }
+  }
+  h->obj.objective = objective;
+  h->obj.bits = bits > 0 ? bits : 4;
   if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
   h->graph_failed = false;
   return DQ_OK;

@@ -79,6 +79,20 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
                           int batch, int iterative_iters);
 dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch);
 
+// Alternative objectives of the ablation in Sec. 5.3 (objectives.cu).
+struct ObjectiveState {
+  bool ready = false;
+  int objective = DQ_OBJ_WHIP, bits = 4;
+  float* O = nullptr;          // [chunk][d] fp32 rotated activations of one chunk of tokens
+  int64_t chunk = 0;
+  double* tok_loss = nullptr;  // [chunk] per-token objective
+  double* acc = nullptr;       // [batch] sum over tokens
+};
+dq_status objective_init(ObjectiveState& os, int d, int64_t n_tokens, int batch);
+void objective_destroy(ObjectiveState& os);
+dq_status objective_forward(Ctx& ctx, ObjectiveState& os, const dq_calib_config& cfg, const void* X, const float* R,
+                            const __nv_bfloat16* rt, void* G, float loss_scale, float* loss_last);
+
 // Cayley SGD with momentum (Algorithm 3) on the rotation itself (cayley_tc.cu).
 struct CayleyState {
   bool ready = false;

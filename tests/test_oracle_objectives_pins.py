@@ -122,3 +122,22 @@ def test_objective_step_gradient_through_rotation_and_qr(name):
         fd = (obj.objective_step(X, P, 0.1, name)["loss"] - obj.objective_step(X, M, 0.1, name)["loss"]) / (2 * h)
         assert out["Gz"][i, j] == pytest.approx(fd, rel=1e-5, abs=1e-9)
     assert np.allclose(out["Z_new"], Z - 0.1 * out["Gz"])
+
+
+def test_quant_grid_reproduces_the_quantiser_and_a_decider_changes_only_what_it_decides():
+    O = RNG.laplace(size=(6, 30))
+    O[2, :] = 1.25                                               # constant row
+    scale, zero, codes = obj.quant_grid(O, 4)
+    deq = np.where(scale == 0.0, O, scale * (codes - zero))
+    assert np.array_equal(deq, orc.quantize_per_token_asymmetric(O, 4))
+    same = obj.grad_wrt_output(O, "quant", "sum", 4, code_decider=lambda O_, s_, z_, c_: c_)
+    assert np.array_equal(same, obj.grad_wrt_output(O, "quant", "sum", 4))
+    # bumping one code by one moves that entry's derivative by exactly -(2/d) scale
+    def bump(O_, s_, z_, c_):
+        c = c_.copy()
+        c[0, 3] += 1.0
+        return c
+    moved = obj.grad_wrt_output(O, "quant", "sum", 4, code_decider=bump) - same
+    assert moved[0, 3] == pytest.approx(-2.0 / 30 * scale[0, 0], rel=1e-12)
+    moved[0, 3] = 0.0
+    assert np.abs(moved).max() == 0.0
