@@ -158,6 +158,27 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 
+/* Algorithm 1's loop around the step: token sampling and mini-batches (hyper-parameter appendix: a
+ * fraction of the captured tokens per epoch, fixed batch size, several epochs).
+ * d_pool: device, [n_pool][ld_pool] token rows of the handle's x_dtype, borrowed, never written.
+ * Epoch e draws the seeded permutation pi of dq_gather_tokens with seed + e and uses its first
+ * floor(sample_ratio * n_pool) rows (sampling without replacement), cut into optimiser steps of
+ * accum micro-batches of the handle's n_tokens rows each; an incomplete last step is dropped.
+ * Every micro-batch is gathered into the activation buffer given to dq_calib_init, WHICH THIS CALL
+ * OVERWRITES (it must be writable device memory of n_tokens rows); dL/dR and the loss of a step are
+ * the mean over all accum * n_tokens tokens of the step (gradient accumulation: the sum with
+ * DQ_SUM_TOKENS), then one QR backward / optimiser update follows.  The paper does not say how tokens
+ * are drawn or batched; this is the reading.  d_loss_out: nullable, device
+ * [n_epochs * steps_per_epoch] with steps_per_epoch = floor(floor(sample_ratio * n_pool) /
+ * (accum * n_tokens)); the product runs in double precision on the float sample_ratio.
+ * h_steps_out: nullable HOST pointer, receives the number of optimiser steps enqueued.
+ * Asynchronous like dq_calib_step; steps are not replayed from a graph (the gather changes).
+ * Errors: INVALID_ARG (null, sizes, ratio outside (0, 1], no complete step), UNSUPPORTED (batch > 1),
+ * CUDA. */
+dq_status dq_calib_run_epochs(dq_calib_t* h, const void* d_pool, int64_t n_pool, int64_t ld_pool,
+                              float sample_ratio, int32_t accum, int32_t n_epochs, uint64_t seed,
+                              float* d_loss_out, int64_t* h_steps_out);
+
 /* The calibration objective.  DQ_OBJ_WHIP (default) is Eq. 4.  The other three are the objectives the
  * ablation of Sec. 5.3 compares it with; the paper names them without formulas, so they are read as
  * per-token statistics over the d channels of the rotated token o = x R (as Eq. 4 is per token),

@@ -13,3 +13,4 @@ from .token_sampling import philox4x32_10, permute_index, gather_tokens  # noqa:
 from .eval_metrics import outlier_count, quantize_per_token_asymmetric, quantization_mse  # noqa: F401,E402
 from .cayley_oracle import cayley_sgd_step, cayley_calib_step, cayley_calib_run  # noqa: F401,E402
 from . import objectives  # noqa: F401,E402
+from . import epochs  # noqa: F401,E402

@@ -30,7 +30,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
     "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens", "dq_eval_rotation",
-    "dq_calib_set_orth_method", "dq_calib_set_objective",
+    "dq_calib_set_orth_method", "dq_calib_set_objective", "dq_calib_run_epochs",
 )
 
 
@@ -69,6 +69,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_set_optimizer.restype = i32
     lib.dq_calib_set_qr_method.argtypes = [vp, i32, i32]
     lib.dq_calib_set_qr_method.restype = i32
+    lib.dq_calib_run_epochs.argtypes = [vp, vp, i64, i64, C.c_float, i32, i32, C.c_uint64, vp, C.POINTER(i64)]
+    lib.dq_calib_run_epochs.restype = i32
     lib.dq_calib_set_objective.argtypes = [vp, i32, i32]
     lib.dq_calib_set_objective.restype = i32
     lib.dq_calib_set_orth_method.argtypes = [vp, i32, C.c_float, C.c_float, i32]
@@ -173,6 +175,15 @@ def dq_calib_set_optimizer(h, optimizer: int, lr: float, beta1: float = 0.9, bet
 
 def dq_calib_set_qr_method(h, method: int, n_iters: int = 0):
     _check(load_library().dq_calib_set_qr_method(h, method, n_iters), "dq_calib_set_qr_method")
+
+
+def dq_calib_run_epochs(h, pool, sample_ratio: float, accum: int, n_epochs: int, seed: int, loss_out=None) -> int:
+    """pool: CUDA tensor [n_pool, d] (row stride = pool.stride(0)).  Returns the number of optimiser steps."""
+    steps = C.c_int64(0)
+    _check(load_library().dq_calib_run_epochs(h, pool.data_ptr(), pool.shape[0], pool.stride(0), sample_ratio, accum,
+                                              n_epochs, seed, loss_out.data_ptr() if loss_out is not None else None,
+                                              C.byref(steps)), "dq_calib_run_epochs")
+    return int(steps.value)
 
 
 def dq_calib_set_objective(h, objective: int, bits: int = 0):

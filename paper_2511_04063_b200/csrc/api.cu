@@ -31,6 +31,7 @@ struct dq_calib {
   float* partials = nullptr;
   int n_partials = 0;           // per problem
   float* loss_last = nullptr;   // [batch]
+  float* loss_tmp = nullptr;    // [batch] loss of a later micro-batch before it is accumulated
   QrWorkspace ws;
   TcState tc;                   // tensor-core contractions (operand copies, tensor maps)
   QrTcState qtc;                // tensor-core QR-Orth operand copies
@@ -76,7 +77,7 @@ void free_all(dq_calib* h) {
   objective_destroy(h->obj);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
   cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw);
-  cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->ctx.d_status);
+  cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->loss_tmp); cudaFree(h->ctx.d_status);
   cudaFree(h->ws.A); cudaFree(h->ws.V); cudaFree(h->ws.T); cudaFree(h->ws.W); cudaFree(h->ws.W2);
   cudaFree(h->ws.Q); cudaFree(h->ws.Winv); cudaFree(h->ws.B); cudaFree(h->ws.S); cudaFree(h->ws.tmp);
   for (auto& e : h->ev) if (e) cudaEventDestroy(e);
@@ -133,48 +134,69 @@ dq_status ensure_rotation(dq_calib* h) {
   return DQ_OK;
 }
 
+// Mini-batches of one optimiser step drawn from a pool of token rows (Algorithm 1's token sampling):
+// micro-batch a is rows pi_seed(first + a * n_tokens ...) of the pool, gathered into the handle's
+// activation buffer; dL/dR and the loss are averaged (summed with DQ_SUM_TOKENS) over the micro-batches.
+struct MiniBatch {
+  const void* pool; int64_t n_pool, ld_pool; uint64_t seed; int64_t first; int n_micro;
+};
+
 // One iteration of Algorithm 1's loop body enqueued on the work stream.
-dq_status enqueue_step(dq_calib* h, bool timed) {
+dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
   const dq_calib_config& c = h->cfg;
   const int d = c.d, batch = c.batch;
   const int64_t N = c.n_tokens;
-  const float inv_n = (c.reduction == DQ_MEAN_TOKENS) ? (float)(1.0 / (double)N) : 1.f;
+  const int n_micro = mb ? mb->n_micro : 1;
+  const float inv_n = (c.reduction == DQ_MEAN_TOKENS) ? (float)(1.0 / ((double)N * n_micro)) : 1.f;
   Ctx& ctx = h->ctx;
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[0], ctx.stream));
   const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
   // (a1) R <- qr(Z)   (Cayley SGD: only to obtain the first iterate)
   if (!cayley || !h->cay_started) DQ_CHECK(ensure_rotation(h));
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[1], ctx.stream));
-  // (a2-a4) O = X R, Whip epilogue, loss reduction
-  if (h->obj.objective != DQ_OBJ_WHIP) {   // ablation objectives: per-token statistics, materialised O
-    DQ_CHECK(objective_forward(ctx, h->obj, c, h->X, h->R, c.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr, h->G,
-                               inv_n, h->loss_last));
-  } else {
-    if (c.path == DQ_PATH_FP32) {
-      DQ_CHECK(whip_forward_f32(ctx, (const float*)h->X, c.ldx, N * c.ldx, h->R, (float*)h->G, h->partials, N, d,
-                                batch, nullptr));
+  for (int a = 0; a < n_micro; ++a) {
+    float* loss_dst = (a == 0) ? h->loss_last : h->loss_tmp;
+    float* gq_dst = (a == 0) ? h->Gq : h->ws.tmp;
+    if (mb) {
+      DQ_CHECK(gather_tokens(ctx, mb->pool, c.x_dtype == DQ_FP32 ? 4 : 2, mb->n_pool, d, mb->ld_pool, mb->seed,
+                             mb->first + (int64_t)a * N, N, const_cast<void*>(h->X), c.ldx));
+      if (c.path == DQ_PATH_BF16_TC) DQ_CHECK(tc_refresh_inputs(h->tc, ctx));
+    }
+    // (a2-a4) O = X R, Whip epilogue, loss reduction
+    if (h->obj.objective != DQ_OBJ_WHIP) {   // ablation objectives: per-token statistics, materialised O
+      DQ_CHECK(objective_forward(ctx, h->obj, c, h->X, h->R, c.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr,
+                                 h->G, inv_n, loss_dst));
     } else {
-      DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
+      if (c.path == DQ_PATH_FP32) {
+        DQ_CHECK(whip_forward_f32(ctx, (const float*)h->X, c.ldx, N * c.ldx, h->R, (float*)h->G, h->partials, N, d,
+                                  batch, nullptr));
+      } else {
+        DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
+      }
+      DQ_CHECK(loss_finalize(ctx, h->partials, h->n_partials, batch, inv_n, nullptr, loss_dst));
     }
-    DQ_CHECK(loss_finalize(ctx, h->partials, h->n_partials, batch, inv_n, nullptr, h->loss_last));
-  }
-  if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[2], ctx.stream));
-  // (a5) Gq = (1/N) X^T G
-  if (c.path == DQ_PATH_FP32) {
-    GemmDesc g{};
-    g.A = (const float*)h->X; g.lda = c.ldx; g.transA = 1; g.sA = N * c.ldx;
-    g.B = (const float*)h->G; g.ldb = d; g.transB = 0; g.sB = N * (int64_t)d;
-    g.M = d; g.N = d; g.K = (int)N; g.alpha = inv_n; g.beta = 0.f; g.batch = batch;
-    if (h->gq_ks <= 1) {
-      g.C = h->Gq; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = 1;
-      DQ_CHECK(gemm_f32(ctx, g));
-    } else {   // deterministic split-K over the token dimension
-      g.C = h->gq_part; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = h->gq_ks;
-      DQ_CHECK(gemm_f32(ctx, g));
-      DQ_CHECK(splitk_reduce(ctx, h->gq_part, h->gq_ks, (int64_t)d * d, batch, 1.f, 0.f, h->Gq));
+    if (timed && a == n_micro - 1) DQ_CHECK_CUDA(cudaEventRecord(h->ev[2], ctx.stream));
+    // (a5) Gq = (1/N) X^T G
+    if (c.path == DQ_PATH_FP32) {
+      GemmDesc g{};
+      g.A = (const float*)h->X; g.lda = c.ldx; g.transA = 1; g.sA = N * c.ldx;
+      g.B = (const float*)h->G; g.ldb = d; g.transB = 0; g.sB = N * (int64_t)d;
+      g.M = d; g.N = d; g.K = (int)N; g.alpha = inv_n; g.beta = 0.f; g.batch = batch;
+      if (h->gq_ks <= 1) {
+        g.C = gq_dst; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = 1;
+        DQ_CHECK(gemm_f32(ctx, g));
+      } else {   // deterministic split-K over the token dimension
+        g.C = h->gq_part; g.ldc = d; g.sC = (int64_t)d * d; g.ksplit = h->gq_ks;
+        DQ_CHECK(gemm_f32(ctx, g));
+        DQ_CHECK(splitk_reduce(ctx, h->gq_part, h->gq_ks, (int64_t)d * d, batch, 1.f, 0.f, gq_dst));
+      }
+    } else {
+      DQ_CHECK(tc_grad_rotation(h->tc, ctx, gq_dst, inv_n));
     }
-  } else {
-    DQ_CHECK(tc_grad_rotation(h->tc, ctx, h->Gq, inv_n));
+    if (a > 0) {
+      DQ_CHECK(accumulate(ctx, h->Gq, gq_dst, (int64_t)d * d * batch));
+      DQ_CHECK(accumulate(ctx, h->loss_last, loss_dst, batch));
+    }
   }
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[3], ctx.stream));
   // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
@@ -296,7 +318,7 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
   A(dev_alloc(&h->ws.tmp, dd));
   A(dev_alloc(&h->ws.T, (int64_t)batch * d * 32));
   A(dev_alloc(&h->ws.W, (int64_t)batch * d * 32)); A(dev_alloc(&h->ws.W2, (int64_t)batch * d * 32));
-  A(dev_alloc(&h->loss_last, batch));
+  A(dev_alloc(&h->loss_last, batch)); A(dev_alloc(&h->loss_tmp, batch));
   if (st == DQ_OK) {
     for (auto& e : h->ev)
       if (cudaEventCreate(&e) != cudaSuccess) st = DQ_ERR_CUDA;
@@ -369,6 +391,34 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
       DQ_CHECK_CUDA(cudaMemcpyAsync(d_loss_out + (int64_t)s * batch, h->loss_last, sizeof(float) * batch,
                                     cudaMemcpyDeviceToDevice, ctx.stream));
   }
+  return fence_out(h);
+}
+
+dq_status dq_calib_run_epochs(dq_calib_t* h, const void* d_pool, int64_t n_pool, int64_t ld_pool, float sample_ratio,
+                              int32_t accum, int32_t n_epochs, uint64_t seed, float* d_loss_out,
+                              int64_t* h_steps_out) {
+  if (h_steps_out) *h_steps_out = 0;
+  if (!h || !d_pool || n_pool <= 0 || ld_pool < h->cfg.d || accum < 1 || n_epochs < 0 ||
+      !(sample_ratio > 0.f && sample_ratio <= 1.f))
+    return DQ_ERR_INVALID_ARG;
+  if (h->cfg.batch != 1) return DQ_ERR_UNSUPPORTED;
+  const int64_t N = h->cfg.n_tokens;
+  const int64_t n_sampled = (int64_t)((double)sample_ratio * (double)n_pool);
+  const int64_t steps_per_epoch = n_sampled / (N * accum);
+  if (steps_per_epoch < 1) return DQ_ERR_INVALID_ARG;
+  DQ_CHECK(fence_in(h));
+  int64_t k = 0;
+  for (int e = 0; e < n_epochs; ++e) {
+    for (int64_t s = 0; s < steps_per_epoch; ++s, ++k) {
+      MiniBatch mb{d_pool, n_pool, ld_pool, seed + (uint64_t)e, s * accum * N, accum};
+      DQ_CHECK(enqueue_step(h, false, &mb));
+      h->eager_steps_done++;
+      if (d_loss_out)
+        DQ_CHECK_CUDA(cudaMemcpyAsync(d_loss_out + k, h->loss_last, sizeof(float), cudaMemcpyDeviceToDevice,
+                                      h->ctx.stream));
+    }
+  }
+  if (h_steps_out) *h_steps_out = k;
   return fence_out(h);
 }
 

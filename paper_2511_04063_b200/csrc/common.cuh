@@ -108,6 +108,8 @@ dq_status qr128_backward_sgd(Ctx& ctx, const float* R, const float* W, const flo
 dq_status gather_tokens(Ctx& ctx, const void* X, int elem_bytes, int64_t n, int d, int64_t ldx, uint64_t seed,
                         int64_t first, int64_t count, void* out, int64_t ldo);
 
+// dst += src (n elements)
+dq_status accumulate(Ctx& ctx, float* dst, const float* src, int64_t n);
 // Z <- Z - lr Gz  (n elements)
 dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n);
 // v <- mu v + Gz; Z <- Z - lr v

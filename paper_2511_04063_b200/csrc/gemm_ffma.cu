@@ -257,6 +257,24 @@ dq_status loss_finalize(Ctx& ctx, const float* partials, int n_per_problem, int 
   return after_launch(ctx);
 }
 
+namespace {
+__global__ void __launch_bounds__(256) accumulate_kernel(float* __restrict__ dst, const float* __restrict__ src,
+                                                         int64_t n) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] += src[i];
+}
+}  // namespace
+
+// dst += src (gradient accumulation over micro-batches)
+dq_status accumulate(Ctx& ctx, float* dst, const float* src, int64_t n) {
+  int blocks = (int)((n + 255) / 256);
+  const int cap = ctx.sm_count * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  accumulate_kernel<<<blocks, 256, 0, ctx.stream>>>(dst, src, n);
+  return after_launch(ctx);
+}
+
 // Algorithm 1 (update step).  n is a multiple of 4 (d is a multiple of 32).
 dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n) {
   const int64_t n4 = n / 4;
