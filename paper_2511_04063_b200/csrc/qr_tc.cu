@@ -290,8 +290,9 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   if (q.part_bs > 0) DQ_CHECK(alloc(&q.part, q.part_bs * batch));
   DQ_CHECK(alloc(&q.tw_hi, dd)); DQ_CHECK(alloc(&q.tw_lo, dd));
   DQ_CHECK(alloc(&q.uot_hi, dd)); DQ_CHECK(alloc(&q.uot_lo, dd));
-  {   // tile orders: most expensive tiles first, dealt round-robin to the persistent CTAs
-    const int nb = d / 128;
+  for (int unit = 128; unit <= 256; unit *= 2) {   // tile orders: most expensive tiles first, dealt round-robin to the persistent CTAs
+    if (d % unit != 0) break;
+    const int nb = d / unit;
     std::vector<int> upper, desc, asc;
     for (int j = 0; j < nb; ++j)
       for (int i = 0; i < nb; ++i) {
@@ -302,11 +303,15 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
     std::stable_sort(desc.begin(), desc.end(), [](int a, int b) { return (a >> 16) > (b >> 16); });
     asc = desc;
     std::reverse(asc.begin(), asc.end());
-    q.n_upper = (int)upper.size(); q.n_all = (int)desc.size();
-    DQ_CHECK(alloc(&q.tl_upper, q.n_upper)); DQ_CHECK(alloc(&q.tl_desc_nb, q.n_all)); DQ_CHECK(alloc(&q.tl_asc_nb, q.n_all));
-    DQ_CHECK_CUDA(cudaMemcpy(q.tl_upper, upper.data(), sizeof(int) * upper.size(), cudaMemcpyHostToDevice));
-    DQ_CHECK_CUDA(cudaMemcpy(q.tl_desc_nb, desc.data(), sizeof(int) * desc.size(), cudaMemcpyHostToDevice));
-    DQ_CHECK_CUDA(cudaMemcpy(q.tl_asc_nb, asc.data(), sizeof(int) * asc.size(), cudaMemcpyHostToDevice));
+    int*& tu = (unit == 128) ? q.tl_upper : q.tl2_upper;
+    int*& td = (unit == 128) ? q.tl_desc_nb : q.tl2_desc_nb;
+    int*& ta = (unit == 128) ? q.tl_asc_nb : q.tl2_asc_nb;
+    ((unit == 128) ? q.n_upper : q.n2_upper) = (int)upper.size();
+    ((unit == 128) ? q.n_all : q.n2_all) = (int)desc.size();
+    DQ_CHECK(alloc(&tu, (int64_t)upper.size())); DQ_CHECK(alloc(&td, (int64_t)desc.size())); DQ_CHECK(alloc(&ta, (int64_t)desc.size()));
+    DQ_CHECK_CUDA(cudaMemcpy(tu, upper.data(), sizeof(int) * upper.size(), cudaMemcpyHostToDevice));
+    DQ_CHECK_CUDA(cudaMemcpy(td, desc.data(), sizeof(int) * desc.size(), cudaMemcpyHostToDevice));
+    DQ_CHECK_CUDA(cudaMemcpy(ta, asc.data(), sizeof(int) * asc.size(), cudaMemcpyHostToDevice));
   }
   q.ready = true;
   return DQ_OK;
@@ -318,6 +323,7 @@ void qr_tc_destroy(QrTcState& q) {
   for (bf16* p : all) cudaFree(p);
   cudaFree(q.y_hi); cudaFree(q.y_lo); cudaFree(q.w2_hi); cudaFree(q.w2_lo); cudaFree(q.part); cudaFree(q.T);
   cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.uot_hi); cudaFree(q.uot_lo); cudaFree(q.tl_upper); cudaFree(q.tl_desc_nb); cudaFree(q.tl_asc_nb);
+  cudaFree(q.tl2_upper); cudaFree(q.tl2_desc_nb); cudaFree(q.tl2_asc_nb);
   q = QrTcState();
 }
 
@@ -367,20 +373,20 @@ dq_status qr_upper_factor_incremental(Ctx& ctx, QrWorkspace& ws, QrTcState& q, c
   DQ_CHECK(after_launch(ctx));
   {   // Zh[i][j] = sum_k Z[i][k] W_old[k][j]
     Op a{q.z_hi, q.z_lo, d, dd}, b{q.wt_hi, q.wt_lo, d, dd};
-    Out o; o.f32 = Zh; o.ld = d; o.bs = dd; o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all;
+    Out o; o.f32 = Zh; o.ld = d; o.bs = dd; o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
     DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   }
   DQ_CHECK(qrp_transpose_split(ctx, Zh, scratch, zht_hi, zht_lo, d, batch));
   {   // G[i][j] = sum_k Zh[k][i] Zh[k][j], tiles on and above the block diagonal
     Op a{zht_hi, zht_lo, d, dd};
-    Out o; o.f32 = G; o.ld = d; o.bs = dd; o.tile_list = q.tl_upper; o.n_list = q.n_upper;
+    Out o; o.f32 = G; o.ld = d; o.bs = dd; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
     DQ_CHECK(gemm3(ctx, a, a, d, d, d, batch, o));
   }
   for (int it = 0; it < n_sweeps; ++it) {
     const bool last = it == n_sweeps - 1;
     if (it > 0) {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
       Op tt{q.tw_hi, q.tw_lo, d, dd};
-      Out o; o.f32 = P; o.ld = d; o.bs = dd; o.k_mode = 2; o.tile_list = q.tl_upper; o.n_list = q.n_upper;
+      Out o; o.f32 = P; o.ld = d; o.bs = dd; o.k_mode = 2; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
       DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
     }
     chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, it > 0 ? P : nullptr, T, q.tw_hi, q.tw_lo,
@@ -391,7 +397,7 @@ dq_status qr_upper_factor_incremental(Ctx& ctx, QrWorkspace& ws, QrTcState& q, c
   {   // U[i][j] = sum_k Uh[i][k] U_old[k][j]: both upper triangular, k in [128 mb, 128 (nb + 1))
     Op a{uh_hi, uh_lo, d, dd}, b{q.uot_hi, q.uot_lo, d, dd};
     Out o; o.f32 = U; o.ld = d; o.bs = dd; o.hi = q.u_hi; o.lo = q.u_lo; o.ld_h = d; o.bs_h = dd;
-    o.k_mode = 1 | 4; o.tile_list = q.tl_upper; o.n_list = q.n_upper;
+    o.k_mode = 1 | 4; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
     DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   }
   return qr_diag_check(ctx, U, d, batch);
@@ -424,7 +430,7 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
   Op b{q.wt_hi, q.wt_lo, d, dd};
   Out o; o.f32 = R; o.ld = d; o.bs = dd; o.hi = q.r_hi; o.lo = q.r_lo; o.ld_h = d; o.bs_h = dd;
   o.k_mode = 4;   // W is upper triangular: W^T[j][k] = 0 for k > j
-  o.tile_list = q.tl_desc_nb; o.n_list = q.n_all;
+  o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
   DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   split_kernel<<<tiles, 256, 0, ctx.stream>>>(R, q.rt_hi, q.rt_lo, d, 1);
   return after_launch(ctx);
@@ -445,13 +451,13 @@ dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* G
   Op r{q.r_hi, q.r_lo, d, dd}, st{q.st_hi, q.st_lo, d, dd};
   Out om; om.hi = q.m_hi; om.lo = q.m_lo; om.ld_h = d; om.bs_h = dd;
   om.k_mode = 8;  // S is strictly lower triangular: S^T[j][k] = 0 for k < j
-  om.tile_list = q.tl_asc_nb; om.n_list = q.n_all;
+  om.tile_list = q.tl_asc_nb; om.n_list = q.n_all; om.tile_list2 = q.tl2_asc_nb; om.n_list2 = q.n2_all;
   DQ_CHECK(gemm3(ctx, r, st, d, d, d, batch, om));
   // Gz[i][j] = sum_k M[i][k] W[j][k]
   Op m{q.m_hi, q.m_lo, d, dd}, wn{q.wn_hi, q.wn_lo, d, dd};
   Out og; og.f32 = Gz; og.ld = d; og.bs = dd;
   og.k_mode = 8;  // W[j][k] = 0 for k < j
-  og.tile_list = q.tl_asc_nb; og.n_list = q.n_all;
+  og.tile_list = q.tl_asc_nb; og.n_list = q.n_all; og.tile_list2 = q.tl2_asc_nb; og.n_list2 = q.n2_all;
   return gemm3(ctx, m, wn, d, d, d, batch, og);
 }
 

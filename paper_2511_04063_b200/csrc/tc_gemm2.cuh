@@ -26,9 +26,15 @@ constexpr int PAIR_M = 256, PAIR_N = 256;
 constexpr int HALF = 128;
 constexpr int A_BYTES = HALF * BLOCK_K * 2;
 constexpr int B_BYTES = HALF * BLOCK_K * 2;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // per CTA
-constexpr int STAGES = 6;
-constexpr int SMEM_TOTAL = STAGES * STAGE_BYTES + 1024 + 1024;
+// NTERMS = 1: plain bf16 product.  NTERMS = 3: split-bf16 operands (hi, lo), three MMAs per product
+// (hi hi + hi lo + lo hi), about 2^-17 relative.
+template <int NTERMS>
+struct PairSmem {
+  static constexpr int NOPS = (NTERMS == 1) ? 1 : 2;
+  static constexpr int STAGE_BYTES = NOPS * (A_BYTES + B_BYTES);     // per CTA: 32 KB or 64 KB
+  static constexpr int STAGES = (NTERMS == 1) ? 6 : 3;
+  static constexpr int TOTAL = STAGES * STAGE_BYTES + 1024 + 1024;
+};
 constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;             // clears the bit that separates the two CTAs of a pair
 constexpr uint32_t TMEM_COLS = 512;                     // two 256-column accumulators
 
@@ -82,10 +88,16 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16_pair() {
 }
 
 // Params as in the one-CTA kernel; m_blocks / n_blocks count 256 x 256 pair tiles, tile_list entries
-// are mb | nb << 16 in those units, partials get eight values per tile (CTA rank, lane quarter).
-template <int EPI>
+// are mb | nb << 16 in those units (tri_skip and k_mode refer to them too), partials get eight values
+// per tile (CTA rank, lane quarter).
+template <int NTERMS, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, const Params p) {
+tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapB_lo,
+                const Params p) {
+  using L = PairSmem<NTERMS>;
+  constexpr int STAGES = L::STAGES;
+  constexpr int STAGE_BYTES = L::STAGE_BYTES;
   constexpr uint32_t IDESC = make_idesc_bf16_pair();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -107,6 +119,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tensormap(&mapA);
     prefetch_tensormap(&mapB);
+    if (NTERMS > 1) { prefetch_tensormap(&mapA_lo); prefetch_tensormap(&mapB_lo); }
   }
   if (warp == 1) tmem_alloc_pair(tmem_slot, TMEM_COLS);
   tc_fence_before();
@@ -120,9 +133,17 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     if (p.tile_list) { const int code = p.tile_list[r]; mb = code & 0xffff; nb = code >> 16; }
     else { mb = r % p.m_blocks; nb = r / p.m_blocks; }
   };
-  auto k_range = [&](int split, int& k0, int& kn) {
-    const int lo = (int)(((int64_t)split * p.k_blocks) / p.ksplit);
-    const int hi = (int)(((int64_t)(split + 1) * p.k_blocks) / p.ksplit);
+  // as in the one-CTA kernel; k_mode clips the range to the non-zero part of triangular operands
+  auto k_range = [&](int split, int mb, int nb, int& k0, int& kn) {
+    int lo = (int)(((int64_t)split * p.k_blocks) / p.ksplit);
+    int hi = (int)(((int64_t)(split + 1) * p.k_blocks) / p.ksplit);
+    if (p.k_mode) {
+      constexpr int R = PAIR_M / BLOCK_K;   // k-blocks per 256 rows
+      if ((p.k_mode & 1) && lo < R * mb) lo = R * mb;
+      if ((p.k_mode & 8) && lo < R * nb) lo = R * nb;
+      if ((p.k_mode & 2) && hi > R * (mb + 1)) hi = R * (mb + 1);
+      if ((p.k_mode & 4) && hi > R * (nb + 1)) hi = R * (nb + 1);
+    }
     k0 = lo; kn = hi - lo;
   };
   const int units = tiles_per_batch * p.batch * p.ksplit;
@@ -140,16 +161,21 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const int b = t / tiles_per_batch;
         int mb, nb;
         tile_of(t % tiles_per_batch, mb, nb);
+        if (p.tri_skip && mb > nb) continue;
         int k0, kn;
-        k_range(split, k0, kn);
+        k_range(split, mb, nb, k0, kn);
         for (int kb = 0; kb < kn; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
           if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          const uint32_t sb = sa + A_BYTES;
+          const uint32_t sb = sa + L::NOPS * A_BYTES;
           const int kc = (k0 + kb) * BLOCK_K;
           tma_load_3d_pair(sa, &mapA, full_bar(stage), kc, mb * PAIR_M + (int)rank * HALF, b);
           tma_load_3d_pair(sb, &mapB, full_bar(stage), kc, nb * PAIR_N + (int)rank * HALF, b);
+          if (NTERMS > 1) {
+            tma_load_3d_pair(sa + A_BYTES, &mapA_lo, full_bar(stage), kc, mb * PAIR_M + (int)rank * HALF, b);
+            tma_load_3d_pair(sb + B_BYTES, &mapB_lo, full_bar(stage), kc, nb * PAIR_N + (int)rank * HALF, b);
+          }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -163,8 +189,11 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int u = pair; u < units && ok; u += pairs) {
+        int mb, nb;
+        tile_of((u / p.ksplit) % tiles_per_batch, mb, nb);
+        if (p.tri_skip && mb > nb) continue;
         int k0, kn;
-        k_range(u % p.ksplit, k0, kn);
+        k_range(u % p.ksplit, mb, nb, k0, kn);
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * PAIR_N);
@@ -172,11 +201,19 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
           if (!mbar_wait(full_bar(stage), phase, p.d_status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          const uint32_t sb = sa + A_BYTES;
+          const uint32_t sb = sa + L::NOPS * A_BYTES;
 #pragma unroll
-          for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-            umma_bf16_pair(tmem_d, make_kmajor_sw128_desc(sa + k * UMMA_K * 2), make_kmajor_sw128_desc(sb + k * UMMA_K * 2),
-                           IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+            const uint64_t a_hi = make_kmajor_sw128_desc(sa + k * UMMA_K * 2);
+            const uint64_t b_hi = make_kmajor_sw128_desc(sb + k * UMMA_K * 2);
+            umma_bf16_pair(tmem_d, a_hi, b_hi, IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+            if (NTERMS > 1) {
+              const uint64_t a_lo = make_kmajor_sw128_desc(sa + A_BYTES + k * UMMA_K * 2);
+              const uint64_t b_lo = make_kmajor_sw128_desc(sb + B_BYTES + k * UMMA_K * 2);
+              umma_bf16_pair(tmem_d, a_hi, b_lo, IDESC, 1u);
+              umma_bf16_pair(tmem_d, a_lo, b_hi, IDESC, 1u);
+            }
+          }
           umma_commit_pair(empty_bar(stage));      // both CTAs may refill this slot once the MMAs retire
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -197,6 +234,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       const int b = t / tiles_per_batch;
       int mb, nb;
       tile_of(t % tiles_per_batch, mb, nb);
+      if (p.tri_skip && mb > nb) continue;
       if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
       tc_fence_after();
       const int row = mb * PAIR_M + (int)rank * HALF + q * 32 + lane;
@@ -225,12 +263,42 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 4; ++i)
             dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-        } else {   // EPI_GEN: fp32 store of alpha * acc
-          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_off + c * 32);
+        } else {   // EPI_GEN: alpha * acc (+ beta * old) as fp32 and / or as a split-bf16 copy
+          float f[32];
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            dst[i] = make_float4(p.alpha * __uint_as_float(v[4 * i]), p.alpha * __uint_as_float(v[4 * i + 1]),
-                                 p.alpha * __uint_as_float(v[4 * i + 2]), p.alpha * __uint_as_float(v[4 * i + 3]));
+          for (int i = 0; i < 32; ++i) f[i] = p.alpha * __uint_as_float(v[i]);
+          if (p.out) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_off + c * 32);
+            if (p.beta != 0.f) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float4 o = dst[i];
+                f[4 * i] = fmaf(p.beta, o.x, f[4 * i]); f[4 * i + 1] = fmaf(p.beta, o.y, f[4 * i + 1]);
+                f[4 * i + 2] = fmaf(p.beta, o.z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.beta, o.w, f[4 * i + 3]);
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+          }
+          if (p.out_hi) {
+            const int64_t off_h = (int64_t)b * p.batch_stride_h + (int64_t)row * p.ld_h + (int64_t)nb * PAIR_N + c * 32;
+            uint32_t ph[16], pl[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+              const float2 hf = __bfloat1622float2(h);
+              const __nv_bfloat162 l = __floats2bfloat162_rn(f[2 * i] - hf.x, f[2 * i + 1] - hf.y);
+              ph[i] = *reinterpret_cast<const uint32_t*>(&h);
+              pl[i] = *reinterpret_cast<const uint32_t*>(&l);
+            }
+            uint4* dh = reinterpret_cast<uint4*>(p.out_hi + off_h);
+            uint4* dl = reinterpret_cast<uint4*>(p.out_lo + off_h);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              dh[i] = make_uint4(ph[4 * i], ph[4 * i + 1], ph[4 * i + 2], ph[4 * i + 3]);
+              dl[i] = make_uint4(pl[4 * i], pl[4 * i + 1], pl[4 * i + 2], pl[4 * i + 3]);
+            }
+          }
         }
       }
       tc_fence_before();

@@ -60,12 +60,14 @@ dq_status launch_gemm(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, cons
 
 // Two-CTA kernel (tc_gemm2.cuh): p.m_blocks / p.n_blocks count 256 x 256 tiles; one cluster of two
 // CTAs per tile, at most one pair per two SMs.
-template <int EPI>
-dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, const tc::Params& p) {
+template <int NT, int EPI>
+dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& alo,
+                       const CUtensorMap& blo, const tc::Params& p) {
   static bool attr_set = false;
-  auto kern = tc2::tc_gemm2_kernel<EPI>;
+  auto kern = tc2::tc_gemm2_kernel<NT, EPI>;
+  constexpr int SMEM = tc2::PairSmem<NT>::TOTAL;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::SMEM_TOTAL) != cudaSuccess)
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
       return DQ_ERR_CUDA;
     attr_set = true;
   }
@@ -75,13 +77,13 @@ dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, con
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   cfg.blockDim = dim3(tc::NUM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = tc2::SMEM_TOTAL;
+  cfg.dynamicSmemBytes = SMEM;
   cfg.stream = ctx.stream;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kern, a, b, p) != cudaSuccess) return DQ_ERR_CUDA;
+  if (cudaLaunchKernelEx(&cfg, kern, a, b, alo, blo, p) != cudaSuccess) return DQ_ERR_CUDA;
   return after_launch(ctx);
 }
 
@@ -99,6 +101,7 @@ struct Out {
   int ksplit = 1; int64_t split_stride = 0;
   int tri_skip = 0, k_mode = 0;   // triangular structure, see tc::Params
   const int* tile_list = nullptr; int n_list = 0;   // explicit tile order (device), see tc::Params
+  const int* tile_list2 = nullptr; int n_list2 = 0; // the same order in 256 x 256 tiles (two-CTA kernel)
 };
 
 // D[m][n] = alpha sum_k A[m][k] B[n][k] (+ beta D) with split-bf16 operands (three bf16 MMAs per
@@ -107,6 +110,25 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
   if (M % 128 || N % 128 || K % 64 || o.ksplit < 1 || o.ksplit > K / 64) return DQ_ERR_UNSUPPORTED;
   CUtensorMap ma, mal, mb, mbl;
   const int64_t bsa = A.bs ? A.bs : (int64_t)M * A.ld, bsb = B.bs ? B.bs : (int64_t)N * B.ld;
+  // Large products run on CTA pairs (256 x 256 tiles, half the operand traffic per MMA); a caller that
+  // orders its tiles must also give the order in pair tiles.
+  const bool pair_ok = M % 256 == 0 && N % 256 == 0 && (!o.tile_list || o.tile_list2) &&
+                       (int64_t)(M / 256) * (N / 256) * batch * o.ksplit >= 32;
+  if (pair_ok) {
+    if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
+    DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, tc2::HALF));
+    DQ_CHECK(make_map(&mal, A.lo, K, M, batch, A.ld, bsa, tc2::HALF));
+    DQ_CHECK(make_map(&mb, B.hi, K, N, batch, B.ld, bsb, tc2::HALF));
+    DQ_CHECK(make_map(&mbl, B.lo, K, N, batch, B.ld, bsb, tc2::HALF));
+    tc::Params p{};
+    p.m_blocks = M / 256; p.n_blocks = N / 256; p.batch = batch; p.ksplit = o.ksplit; p.k_blocks = K / tc::BLOCK_K;
+    p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = o.split_stride;
+    p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
+    p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
+    p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
+    p.tile_list = o.tile_list2; p.n_list = o.n_list2;
+    return launch_gemm2<3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
+  }
   DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, tc::BLOCK_M));
   DQ_CHECK(make_map(&mal, A.lo, K, M, batch, A.ld, bsa, tc::BLOCK_M));
   DQ_CHECK(make_map(&mb, B.hi, K, N, batch, B.ld, bsb, 128));

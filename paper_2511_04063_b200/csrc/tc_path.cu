@@ -143,7 +143,7 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
   p.alpha = 1.f; p.partials = partials; p.d_status = ctx.d_status;
   if (tc.pair) {   // 256 channels x 256 tokens per CTA pair
     p.m_blocks = tc.d / 256;
-    return tch::launch_gemm2<tc::EPI_WHIP>(ctx, m->rt, m->x128, p);
+    return tch::launch_gemm2<1, tc::EPI_WHIP>(ctx, m->rt, m->x128, m->rt, m->x128, p);
   }
   return tch::launch_gemm<256, 1, tc::EPI_WHIP>(ctx, m->rt, m->x, m->rt, m->x, p);
 }
@@ -165,7 +165,7 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
   }
   if (tc.pair) p.m_blocks = d / 256;
   auto launch = [&](const tc::Params& pp) {
-    if (tc.pair) return tch::launch_gemm2<tc::EPI_GEN>(ctx, m->xt, m->gt128, pp);
+    if (tc.pair) return tch::launch_gemm2<1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, pp);
     return (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, m->xt, m->gt256, m->xt, m->gt256, pp)
                        : tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, pp);
   };

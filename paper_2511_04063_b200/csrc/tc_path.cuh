@@ -70,6 +70,10 @@ struct QrTcState {
   int* tl_upper = nullptr; int n_upper = 0;             // tiles mb <= nb, largest mb first
   int* tl_desc_nb = nullptr;                            // all tiles, largest nb first
   int* tl_asc_nb = nullptr; int n_all = 0;              // all tiles, smallest nb first
+  // the same orders in 256 x 256 tiles for the two-CTA kernel (d % 256 == 0 only)
+  int* tl2_upper = nullptr; int n2_upper = 0;
+  int* tl2_desc_nb = nullptr;
+  int* tl2_asc_nb = nullptr; int n2_all = 0;
 };
 dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count);
 void qr_tc_destroy(QrTcState& q);
