@@ -261,6 +261,24 @@ def main():
         cay = {"ms_per_step": ms_cay / K, "update_ms": phases_cay["qr_backward"]}
         dq.dq_calib_set_orth_method(h, dq.DQ_ORTH_QR)
 
+    # ---------------------------------------------------------------- Y = X R materialised (dq_rotate_apply)
+    rot = None
+    if path == dq.DQ_PATH_BF16_TC and wr.batch == 1:
+        Rdev = torch.empty((wr.d, wr.d), dtype=torch.float32, device="cuda")
+        dq.dq_calib_get_rotation(h, Rdev)
+        Y = torch.empty((wr.n_tokens, wr.d), dtype=torch.bfloat16, device="cuda")
+        for _ in range(3):
+            dq.dq_rotate_apply(Xd[0], Rdev, Y)
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        r0.record()
+        for _ in range(10):
+            dq.dq_rotate_apply(Xd[0], Rdev, Y)
+        r1.record()
+        torch.cuda.synchronize()
+        rot = r0.elapsed_time(r1) / 10
+        del Y
+
     # ---------------------------------------------------------------- end to end (host buffers)
     loss_host = torch.empty((1, wr.batch), dtype=torch.float32).pin_memory()
     Ke = min(K, 10)
@@ -337,6 +355,10 @@ def main():
             line["qr_iterative"] = {"value": world * 1e3 / alt["ms_per_step"], "unit": UNIT,
                                     "ms_per_step": alt["ms_per_step"], "phases_ms": alt["phases_ms"],
                                     "qr_orth_share": (alt["phases_ms"]["qr_forward"] + alt["phases_ms"]["qr_backward"]) / ta}
+        if rot is not None:
+            # includes the fp32 -> bf16 transpose of R (d^2 entries) in front of the contraction
+            line["rotate_apply"] = {"ms": rot, "tflops": 2.0 * N * d * d / (rot * 1e-3) / 1e12,
+                                    "hbm_bytes": 4.0 * N * d + 6.0 * d * d}
         if cay is not None:
             # Table 4's comparison on this GPU: the same loss and dL/dR, rotation updated by Cayley SGD with
             # momentum (six d x d split-bf16 products, 12 d^3 flops, three bf16 MMAs per product)

@@ -113,18 +113,8 @@ dq_status eval_rotation(Ctx& ctx, const void* d_X, int x_dtype, int64_t n, int d
   for (int64_t r0 = 0; r0 < n && st == DQ_OK; r0 += chunk) {
     const int64_t rows = (n - r0 < chunk) ? n - r0 : chunk;
     if (tcp) {   // O[token][channel] = sum_k X[token][k] R^T[channel][k]
-      const int bn = (d % 256 == 0) ? 256 : 128;
-      CUtensorMap ma, mb;
       const __nv_bfloat16* xc = reinterpret_cast<const __nv_bfloat16*>(d_X) + r0 * ldx;
-      st = tch::make_map(&ma, xc, d, rows, 1, ldx, rows * ldx, tc::BLOCK_M);
-      if (st == DQ_OK) st = tch::make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, bn);
-      if (st != DQ_OK) break;
-      tc::Params p{};
-      p.m_blocks = (int)(rows / tc::BLOCK_M); p.n_blocks = d / bn; p.batch = 1; p.ksplit = 1;
-      p.k_blocks = d / tc::BLOCK_K;
-      p.out = O; p.ld = d; p.alpha = 1.f; p.beta = 0.f; p.d_status = nullptr;
-      st = (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
-                       : tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p);
+      st = tch::rotate_tokens<tc::EPI_GEN>(ctx, xc, rows, d, ldx, rt, O, d, nullptr);
     } else {
       GemmDesc g{};
       g.A = reinterpret_cast<const float*>(d_X) + r0 * ldx; g.lda = ldx; g.transA = 0;

@@ -196,17 +196,9 @@ dq_status objective_forward(Ctx& ctx, ObjectiveState& os, const dq_calib_config&
     for (int64_t r0 = 0; r0 < N; r0 += os.chunk) {
       const int64_t rows = (N - r0 < os.chunk) ? N - r0 : os.chunk;
       if (tcp) {   // O[token][channel] = sum_k X[token][k] R^T[channel][k]
-        const int bn = (d % 256 == 0) ? 256 : 128;
-        CUtensorMap ma, mb;
         const bf16* xc = reinterpret_cast<const bf16*>(X) + ((int64_t)b * N + r0) * cfg.ldx;
-        DQ_CHECK(tch::make_map(&ma, xc, d, rows, 1, cfg.ldx, rows * cfg.ldx, tc::BLOCK_M));
-        DQ_CHECK(tch::make_map(&mb, rt + (int64_t)b * d * d, d, d, 1, d, (int64_t)d * d, bn));
-        tc::Params p{};
-        p.m_blocks = (int)(rows / tc::BLOCK_M); p.n_blocks = d / bn; p.batch = 1; p.ksplit = 1;
-        p.k_blocks = d / tc::BLOCK_K;
-        p.out = os.O; p.ld = d; p.alpha = 1.f; p.beta = 0.f; p.d_status = ctx.d_status;
-        DQ_CHECK((bn == 256) ? (tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p))
-                             : (tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)));
+        DQ_CHECK(tch::rotate_tokens<tc::EPI_GEN>(ctx, xc, rows, d, cfg.ldx, rt + (int64_t)b * d * d, os.O, d,
+                                                 ctx.d_status));
         objective_grad_kernel<true><<<(unsigned)((rows + TOK - 1) / TOK), 256, 0, ctx.stream>>>(
             os.O, rows, d, os.objective, maxq, reinterpret_cast<bf16*>(G) + (int64_t)b * d * N, N, r0, os.tok_loss);
       } else {

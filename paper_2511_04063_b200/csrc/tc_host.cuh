@@ -89,6 +89,29 @@ dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, con
 
 using bf16 = __nv_bfloat16;
 
+// O[token][channel] = sum_k X[token][k] Rt[channel][k] for n token rows (bf16, row stride ldx) and a
+// d x d bf16 R^T; EPI = EPI_BF16 (bf16 rows, stride ldo) or EPI_GEN (fp32 rows).  CTA pairs with
+// 256 x 256 tiles when the shape allows, else the one-CTA kernel.  n % 128 == 0, d % 128 == 0.
+template <int EPI>
+inline dq_status rotate_tokens(Ctx& ctx, const void* X, int64_t n, int d, int64_t ldx, const bf16* rt, void* out,
+                               int64_t ldo, int* d_status) {
+  CUtensorMap ma, mb;
+  tc::Params p{};
+  p.batch = 1; p.ksplit = 1; p.k_blocks = d / tc::BLOCK_K;
+  p.out = out; p.ld = ldo; p.alpha = 1.f; p.beta = 0.f; p.d_status = d_status;
+  if (d % 256 == 0 && n % 256 == 0 && ctx.sm_count >= 2) {
+    DQ_CHECK(make_map(&ma, X, d, n, 1, ldx, n * ldx, tc2::HALF));
+    DQ_CHECK(make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, tc2::HALF));
+    p.m_blocks = (int)(n / 256); p.n_blocks = d / 256;
+    return launch_gemm2<1, EPI>(ctx, ma, mb, ma, mb, p);
+  }
+  const int bn = (d % 256 == 0) ? 256 : 128;
+  DQ_CHECK(make_map(&ma, X, d, n, 1, ldx, n * ldx, tc::BLOCK_M));
+  DQ_CHECK(make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, bn));
+  p.m_blocks = (int)(n / tc::BLOCK_M); p.n_blocks = d / bn;
+  return (bn == 256) ? launch_gemm<256, 1, EPI>(ctx, ma, mb, ma, mb, p) : launch_gemm<128, 1, EPI>(ctx, ma, mb, ma, mb, p);
+}
+
 struct Op {   // K-major operand: rows x K, split pair, leading dimension, batch stride (elements)
   const bf16* hi; const bf16* lo; int64_t ld; int64_t bs;
 };

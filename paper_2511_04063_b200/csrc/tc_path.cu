@@ -199,19 +199,7 @@ dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t l
     return DQ_ERR_ALLOC;
   transpose_f32_to_bf16_kernel<<<dim3(d / 32, d / 32, 1), 256, 0, ctx.stream>>>(d_R, rt, d);
   dq_status st = after_launch(ctx);
-  const int bn = (d % 256 == 0) ? 256 : 128;
-  CUtensorMap ma, mb;
-  if (st == DQ_OK) st = tch::make_map(&ma, d_X, d, n, 1, ldx, n * ldx, tc::BLOCK_M);
-  if (st == DQ_OK) st = tch::make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, bn);
-  if (st == DQ_OK) {
-    tc::Params p{};
-    p.m_blocks = (int)(n / tc::BLOCK_M); p.n_blocks = d / bn; p.batch = 1; p.ksplit = 1;
-    p.k_blocks = d / tc::BLOCK_K;
-    p.out = d_Y; p.ld = ldy; p.batch_stride = 0; p.split_stride = 0; p.alpha = 1.f;
-    p.partials = nullptr; p.d_status = nullptr;
-    st = (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p)
-                     : tch::launch_gemm<128, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p);
-  }
+  if (st == DQ_OK) st = tch::rotate_tokens<tc::EPI_BF16>(ctx, d_X, n, d, ldx, rt, d_Y, ldy, nullptr);
   cudaFreeAsync(rt, ctx.stream);
   return st;
 }
@@ -256,17 +244,7 @@ dq_status tc_rotate_apply_static(Ctx& ctx, const void* d_X, int64_t n, int d, in
   // Every element of rt[0 : d*d) is overwritten, so nothing of an earlier call survives.
   transpose_f32_to_bf16_kernel<<<dim3(d / 32, d / 32, 1), 256, 0, ctx.stream>>>(d_R, rt, d);
   DQ_CHECK(after_launch(ctx));
-  const int bn = (d % 256 == 0) ? 256 : 128;
-  CUtensorMap ma, mb;
-  DQ_CHECK(tch::make_map(&ma, d_X, d, n, 1, ldx, n * ldx, tc::BLOCK_M));
-  DQ_CHECK(tch::make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, bn));
-  tc::Params p{};
-  p.m_blocks = (int)(n / tc::BLOCK_M); p.n_blocks = d / bn; p.batch = 1; p.ksplit = 1;
-  p.k_blocks = d / tc::BLOCK_K;
-  p.out = d_Y; p.ld = ldy; p.batch_stride = 0; p.split_stride = 0; p.alpha = 1.f;
-  p.partials = nullptr; p.d_status = nullptr;
-  return (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p)
-                     : tch::launch_gemm<128, 1, tc::EPI_BF16>(ctx, ma, mb, ma, mb, p);
+  return tch::rotate_tokens<tc::EPI_BF16>(ctx, d_X, n, d, ldx, rt, d_Y, ldy, nullptr);
 }
 
 }  // namespace dq

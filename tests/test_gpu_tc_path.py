@@ -180,7 +180,7 @@ def test_loss_decreases_over_steps_on_heavy_tailed_input():
     c.close()
 
 
-@pytest.mark.parametrize("n,d", [(256, 128), (1024, 256), (384, 640)])
+@pytest.mark.parametrize("n,d", [(256, 128), (1024, 256), (384, 640), (2048, 1024)])   # one-CTA tiles and CTA pairs
 def test_rotate_apply_bf16(n, d):
     rng = np.random.default_rng(7)
     Xf = rng.standard_normal((n, d)).astype(np.float32)
