@@ -13,7 +13,11 @@
  *     latents / rotations are [batch][d][d] fp32.
  *   - Every call returns a dq_status; nothing throws, aborts or traps.  Device
  *     side problems (rank-deficient latent, non-finite loss, a wait that ran
- *     out) are recorded in a device status word read by dq_calib_status().
+ *     out) are recorded in a device status word read by dq_calib_status().  The
+ *     first error wins and stays until dq_calib_set_latent or one of the
+ *     dq_calib_set_* configuration calls clears it; while it is set, the kernels
+ *     that update the latent (or the Cayley iterate) and the optimiser state
+ *     change nothing, so the parameter stays at the last good iterate.
  *   - All work is enqueued on the stream given at init; calls are asynchronous
  *     with respect to the host unless stated otherwise.
  *   - Notation: R is always the rotation (the orthogonal factor of Z = R U),
@@ -144,17 +148,20 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
 
 /* How the QR-Orth forward (Sec. 4.3: Z = R U) is computed on the tensor-core path.  Both
  * give the same unique factors (diag(U) > 0).
- *   DQ_QR_HOUSEHOLDER (default): blocked Householder QR (Algorithm 2 in compact-WY form) at
- *     every step.
- *   DQ_QR_ITERATIVE: blocked Householder only when no factors of a nearby latent are known (first
- *     step, after dq_calib_set_latent); afterwards incremental.  With the previous step's
- *     U_old, Zh = Z U_old^-1 is close to orthogonal whatever Z is, its upper factor I + T is the
- *     fixed point of T <- striu(E - T^T T) + diag(E - T^T T) / 2 with E = Zh^T Zh - I, reached from
- *     T = 0 in n_iters sweeps of triangular tensor-core GEMMs (no dependent column steps), and
+ *   DQ_QR_ITERATIVE (default): incremental.  Blocked Householder QR (Algorithm 2 in compact-WY
+ *     form) only when no factors of a nearby latent are known (first step, after
+ *     dq_calib_set_latent or a change of method).  Afterwards, with the previous step's U_old,
+ *     Zh = Z U_old^-1 is close to orthogonal whatever Z is, its upper factor I + T is the fixed point
+ *     of T <- striu(E - T^T T) + diag(E - T^T T) / 2 with E = Zh^T Zh - I, reached from T = 0 in
+ *     n_iters sweeps of triangular tensor-core GEMMs (no dependent column steps), and
  *     U = (I + T) U_old.  If one optimiser step moved the latent so far that the last sweep still
- *     changed an entry by more than 1e-5, the status word becomes DQ_ERR_NOT_CONVERGED (raise
- *     n_iters or lower the learning rate).  n_iters <= 0 selects the default (5).
- * Ignored (DQ_OK) on the fp32 path and for d == 128. */
+ *     changed an entry by more than 1e-5, the status word becomes DQ_ERR_NOT_CONVERGED and, as after
+ *     every device-side error, the update kernels leave the latent and the optimiser state untouched
+ *     from then on: the latent stays at the last good iterate.  Recover with
+ *     dq_calib_set_qr_method(h, DQ_QR_HOUSEHOLDER, 0) (or more sweeps, or a lower learning rate) and
+ *     step again.  n_iters <= 0 selects the default (5).
+ *   DQ_QR_HOUSEHOLDER: blocked Householder QR at every step; no assumption on the step size.
+ * The call clears the status word.  Ignored (DQ_OK) on the fp32 path and for d == 128. */
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 
@@ -217,12 +224,13 @@ dq_status dq_calib_set_objective(dq_calib_t* h, int32_t objective, int32_t bits)
 enum { DQ_ORTH_QR = 0, DQ_ORTH_CAYLEY = 1 };
 dq_status dq_calib_set_orth_method(dq_calib_t* h, int32_t method, float beta, float q, int32_t s);
 
-/* Checkpoint / resume of the optimised parameter (Algorithm 1: Z <- Z0). */
+/* Checkpoint / resume of the optimised parameter (Algorithm 1: Z <- Z0).  dq_calib_set_latent clears
+ * the status word. */
 dq_status dq_calib_get_latent(dq_calib_t* h, float* d_Z_out);
 dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z);
 
 /* Synchronises the stream and returns the device status word
- * (DQ_OK / DQ_ERR_SINGULAR / DQ_ERR_NONFINITE / DQ_ERR_TIMEOUT) or DQ_ERR_CUDA. */
+ * (DQ_OK / DQ_ERR_SINGULAR / DQ_ERR_NONFINITE / DQ_ERR_TIMEOUT / DQ_ERR_NOT_CONVERGED) or DQ_ERR_CUDA. */
 dq_status dq_calib_status(dq_calib_t* h);
 
 /* Phase times of the most recent dq_calib_step call, averaged per step, in ms

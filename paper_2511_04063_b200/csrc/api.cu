@@ -36,7 +36,7 @@ struct dq_calib {
   TcState tc;                   // tensor-core contractions (operand copies, tensor maps)
   QrTcState qtc;                // tensor-core QR-Orth operand copies
   bool fast_qr = false;
-  int qr_method = DQ_QR_HOUSEHOLDER, qr_iters = 5;
+  int qr_method = DQ_QR_ITERATIVE, qr_iters = 5;
   int optimizer = DQ_SGD;
   float beta1 = 0.f, beta2 = 0.f, eps = 0.f;
   float* opt_m = nullptr;       // first moment / velocity
@@ -115,6 +115,12 @@ dq_status fence_in(dq_calib* h) {
 dq_status fence_out(dq_calib* h) {
   DQ_CHECK_CUDA(cudaEventRecord(h->ev_out, h->ctx.stream));
   DQ_CHECK_CUDA(cudaStreamWaitEvent(h->user_stream, h->ev_out, 0));
+  return DQ_OK;
+}
+
+// A configuration change or a new latent acknowledges an earlier device-side error.
+dq_status clear_status(dq_calib* h) {
+  DQ_CHECK_CUDA(cudaMemsetAsync(h->ctx.d_status, 0, sizeof(int), h->ctx.stream));
   return DQ_OK;
 }
 
@@ -452,6 +458,7 @@ dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z) {
   DQ_CHECK(fence_in(h));
   DQ_CHECK_CUDA(cudaMemcpyAsync(h->Z, d_Z, sizeof(float) * (size_t)h->cfg.d * h->cfg.d * h->cfg.batch,
                                 cudaMemcpyDeviceToDevice, h->ctx.stream));
+  DQ_CHECK(clear_status(h));
   h->r_stale = true;
   h->qtc.t_warm = false;   // the new latent may be far from the one the iterative QR last saw
   h->cay_started = false;  // Cayley SGD restarts from the orthogonal factor of the new latent
@@ -485,6 +492,7 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
     DQ_CHECK_CUDA(cudaMemcpyAsync(h->opt_pw, ones, sizeof(ones), cudaMemcpyHostToDevice, h->ctx.stream));
     DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
   }
+  DQ_CHECK(clear_status(h));
   h->optimizer = optimizer;
   h->cfg.lr = lr;
   h->beta1 = beta1; h->beta2 = beta2; h->eps = eps;
@@ -498,6 +506,7 @@ dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters)
   const int iters = n_iters <= 0 ? 5 : n_iters;
   if (method == h->qr_method && iters == h->qr_iters) return DQ_OK;
   DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
+  DQ_CHECK(clear_status(h));
   h->qr_method = method;
   h->qr_iters = iters;
   h->r_stale = true;
@@ -514,6 +523,7 @@ dq_status dq_calib_set_objective(dq_calib_t* h, int32_t objective, int32_t bits)
     const dq_status st = objective_init(h->obj, h->cfg.d, h->cfg.n_tokens, h->cfg.batch);
     if (st != DQ_OK) { objective_destroy(h->obj); return st; }
   }
+  DQ_CHECK(clear_status(h));
   h->obj.objective = objective;
   h->obj.bits = bits > 0 ? bits : 4;
   if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
@@ -540,6 +550,7 @@ dq_status dq_calib_set_orth_method(dq_calib_t* h, int32_t method, float beta, fl
                                   h->ctx.stream));
     DQ_CHECK_CUDA(cudaMemsetAsync(h->cay.alpha, 0, sizeof(float) * h->cfg.batch, h->ctx.stream));
   }
+  DQ_CHECK(clear_status(h));
   h->orth_method = method;
   h->cay_started = false;
   h->r_stale = true;

@@ -31,8 +31,10 @@ __device__ __forceinline__ void split2(float v, bf16& hi, bf16& lo) {
 __global__ void __launch_bounds__(256) combine_split_kernel(const float* A, const float* __restrict__ B, float ca,
                                                             float cb, const float* __restrict__ alpha, int use_alpha,
                                                             float* out, bf16* __restrict__ hi, bf16* __restrict__ lo,
-                                                            bf16* __restrict__ thi, bf16* __restrict__ tlo, int n) {
+                                                            bf16* __restrict__ thi, bf16* __restrict__ tlo, int n,
+                                                            const int* __restrict__ d_status) {
   __shared__ float t[32][33];
+  if (d_status && *d_status != 0) return;   // commit nothing once the status word holds an error
   const int64_t off = (int64_t)blockIdx.z * n * n;
   const float s = use_alpha ? alpha[blockIdx.z] : 1.f;
   const float cbs = cb * s;
@@ -134,7 +136,7 @@ dq_status cayley_step_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, CayleyState& c
   const Op r{q.r_hi, q.r_lo, d, dd}, rt{q.rt_hi, q.rt_lo, d, dd};
   // M1 = beta M - G: only its split copy is needed (B operand of T1^T = X M1^T)
   combine_split_kernel<<<tiles, 256, 0, ctx.stream>>>(cs.M, Gq, cs.beta, -1.f, nullptr, 0, nullptr, q.gqt_hi, q.gqt_lo,
-                                                      nullptr, nullptr, d);
+                                                      nullptr, nullptr, d, nullptr);
   DQ_CHECK(after_launch(ctx));
   // T1^T[m][n] = sum_k X[m][k] M1[n][k]
   {
@@ -167,7 +169,7 @@ dq_status cayley_step_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, CayleyState& c
   }
   // X + Y^0 = 2 X + a M, transposed split copy (B operand of W (X + Y))
   combine_split_kernel<<<tiles, 256, 0, ctx.stream>>>(R, cs.M, 2.f, 1.f, cs.alpha, 1, nullptr, nullptr, nullptr,
-                                                      q.z_hi, q.z_lo, d);
+                                                      q.z_hi, q.z_lo, d, nullptr);
   DQ_CHECK(after_launch(ctx));
   const Op st{q.z_hi, q.z_lo, d, dd};
   for (int i = 1; i <= cs.s; ++i) {
@@ -175,10 +177,10 @@ dq_status cayley_step_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, CayleyState& c
     DQ_CHECK(gemm3(ctx, w, st, d, d, d, batch, o));   // P = W (X + Y^(i-1))
     if (i < cs.s) {   // X + Y^i = 2 X + a/2 P
       combine_split_kernel<<<tiles, 256, 0, ctx.stream>>>(R, ws.tmp, 2.f, 0.5f, cs.alpha, 1, nullptr, nullptr, nullptr,
-                                                          q.z_hi, q.z_lo, d);
+                                                          q.z_hi, q.z_lo, d, nullptr);
     } else {          // X <- Y^s = X + a/2 P, with both operand copies of the new rotation
       combine_split_kernel<<<tiles, 256, 0, ctx.stream>>>(R, ws.tmp, 1.f, 0.5f, cs.alpha, 1, R, q.r_hi, q.r_lo,
-                                                          q.rt_hi, q.rt_lo, d);
+                                                          q.rt_hi, q.rt_lo, d, ctx.d_status);
     }
     DQ_CHECK(after_launch(ctx));
   }

@@ -191,7 +191,11 @@ __global__ void __launch_bounds__(256) loss_finalize_kernel(const float* __restr
   }
 }
 
-__global__ void sgd_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz, float lr, int64_t n4) {
+// Every update kernel leaves the parameter (and the optimiser state) untouched once the status word holds
+// an error: a step whose factorisation failed or whose loss was not finite never reaches the latent.
+__global__ void sgd_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz, float lr, int64_t n4,
+                           const int* __restrict__ d_status) {
+  if (d_status && *d_status != 0) return;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
     float4 z = Z[i];
@@ -204,7 +208,8 @@ __global__ void sgd_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz
 
 // v <- mu v + g;  Z <- Z - lr v
 __global__ void momentum_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz, float4* __restrict__ V,
-                                float lr, float mu, int64_t n4) {
+                                float lr, float mu, int64_t n4, const int* __restrict__ d_status) {
+  if (d_status && *d_status != 0) return;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
     float4 z = Z[i], v = V[i];
@@ -218,7 +223,8 @@ __global__ void momentum_kernel(float4* __restrict__ Z, const float4* __restrict
 
 // pw[0] = beta1^t, pw[1] = beta2^t of the step about to be taken (t counted on the device so that a
 // replayed CUDA graph advances it)
-__global__ void adam_advance_kernel(float* pw, float beta1, float beta2) {
+__global__ void adam_advance_kernel(float* pw, float beta1, float beta2, const int* d_status) {
+  if (d_status && *d_status != 0) return;
   pw[0] *= beta1;
   pw[1] *= beta2;
 }
@@ -235,7 +241,8 @@ __device__ __forceinline__ float adam_one(float& z, float g, float& m, float& v,
 // Adam in its published form with bias correction; c1 = 1 / (1 - beta1^t), c2 = 1 / (1 - beta2^t).
 __global__ void adam_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz, float4* __restrict__ M,
                             float4* __restrict__ V, const float* __restrict__ pw, float lr, float b1, float b2,
-                            float eps, int64_t n4) {
+                            float eps, int64_t n4, const int* __restrict__ d_status) {
+  if (d_status && *d_status != 0) return;
   const float c1 = 1.f / (1.f - pw[0]), c2 = 1.f / (1.f - pw[1]);
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
@@ -283,7 +290,7 @@ dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n) {
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   sgd_kernel<<<blocks, 256, 0, ctx.stream>>>(reinterpret_cast<float4*>(Z),
-                                            reinterpret_cast<const float4*>(Gz), lr, n4);
+                                            reinterpret_cast<const float4*>(Gz), lr, n4, ctx.d_status);
   return after_launch(ctx);
 }
 
@@ -299,7 +306,7 @@ static int update_blocks(const Ctx& ctx, int64_t n4) {
 dq_status momentum_update(Ctx& ctx, float* Z, const float* Gz, float* V, float lr, float mu, int64_t n) {
   const int64_t n4 = n / 4;
   momentum_kernel<<<update_blocks(ctx, n4), 256, 0, ctx.stream>>>(
-      reinterpret_cast<float4*>(Z), reinterpret_cast<const float4*>(Gz), reinterpret_cast<float4*>(V), lr, mu, n4);
+      reinterpret_cast<float4*>(Z), reinterpret_cast<const float4*>(Gz), reinterpret_cast<float4*>(V), lr, mu, n4, ctx.d_status);
   return after_launch(ctx);
 }
 
@@ -308,11 +315,11 @@ dq_status momentum_update(Ctx& ctx, float* Z, const float* Gz, float* V, float l
 dq_status adam_update(Ctx& ctx, float* Z, const float* Gz, float* M, float* V, float* pw, float lr, float b1,
                       float b2, float eps, int64_t n) {
   const int64_t n4 = n / 4;
-  adam_advance_kernel<<<1, 1, 0, ctx.stream>>>(pw, b1, b2);
+  adam_advance_kernel<<<1, 1, 0, ctx.stream>>>(pw, b1, b2, ctx.d_status);
   DQ_CHECK(after_launch(ctx));
   adam_kernel<<<update_blocks(ctx, n4), 256, 0, ctx.stream>>>(
       reinterpret_cast<float4*>(Z), reinterpret_cast<const float4*>(Gz), reinterpret_cast<float4*>(M),
-      reinterpret_cast<float4*>(V), pw, lr, b1, b2, eps, n4);
+      reinterpret_cast<float4*>(V), pw, lr, b1, b2, eps, n4, ctx.d_status);
   return after_launch(ctx);
 }
 

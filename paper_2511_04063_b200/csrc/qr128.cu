@@ -223,8 +223,9 @@ constexpr int BWD_SMEM = 3 * N * LD * 4;
 
 __global__ void __launch_bounds__(NT, 1)
 qr128_backward_sgd_kernel(const float* __restrict__ R, const float* __restrict__ W, const float* __restrict__ Gq,
-                          float* __restrict__ Gz, float* __restrict__ Z, float lr) {
+                          float* __restrict__ Gz, float* __restrict__ Z, float lr, const int* __restrict__ d_status) {
   extern __shared__ float sm[];
+  if (d_status && *d_status != 0) lr = 0.f;   // an earlier error freezes the latent
   float* P0 = sm;                    // R
   float* P1 = P0 + N * LD;           // Gq, then S, then W
   float* P2 = P1 + N * LD;           // B, then M = R S
@@ -264,7 +265,7 @@ qr128_backward_sgd_kernel(const float* __restrict__ R, const float* __restrict__
     for (int j = 0; j < 8; ++j) {
       const int e = (r0 + i) * N + cl + 16 * j;
       Gz[e] = acc[i][j];
-      Z[e] = fmaf(-lr, acc[i][j], Z[e]);
+      if (lr != 0.f) Z[e] = fmaf(-lr, acc[i][j], Z[e]);
     }
 }
 
@@ -287,7 +288,7 @@ dq_status qr128_backward_sgd(Ctx& ctx, const float* R, const float* W, const flo
     DQ_CHECK_CUDA(cudaFuncSetAttribute(qr128_backward_sgd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD_SMEM));
     attr = true;
   }
-  qr128_backward_sgd_kernel<<<batch, NT, BWD_SMEM, ctx.stream>>>(R, W, Gq, Gz, Z, lr);
+  qr128_backward_sgd_kernel<<<batch, NT, BWD_SMEM, ctx.stream>>>(R, W, Gq, Gz, Z, lr, ctx.d_status);
   return after_launch(ctx);
 }
 

@@ -31,8 +31,7 @@ def perturbed_latent(w, Z0, seed):
 def test_one_step_at_full_size(name, qr):
     w = gen.WORKLOADS[name]
     c = Calib(w)
-    if qr == "iterative":
-        dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_ITERATIVE, 0)
+    dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_ITERATIVE if qr == "iterative" else dq.DQ_QR_HOUSEHOLDER, 0)
     Z = perturbed_latent(w, c.Z0_host, w.seed)
     c.set_latent(Z)
     if qr == "iterative":

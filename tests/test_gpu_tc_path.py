@@ -160,6 +160,45 @@ def test_incremental_qr_flags_a_step_that_moves_the_latent_too_far():
     c.close()
 
 
+def test_a_failed_step_freezes_the_latent_until_the_method_is_changed():
+    d = 256
+    w = small("c2_7b", d=d, n_tokens=256, n_outlier_channels=1)
+    c = Calib(w, Z0=_near_orthogonal(d, 1, 0.02, 5), lr=20.0)
+    c.step(1)                                                       # Householder start, absurd step
+    assert c.status() == dq.DQ_OK
+    Z1 = c.latent()
+    c.step(3)                                                       # incremental (the default): too far
+    assert c.status() != dq.DQ_OK
+    assert np.array_equal(c.latent(), Z1)                           # no update reached the latent
+    dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_HOUSEHOLDER, 0)         # clears the status word
+    assert c.status() == dq.DQ_OK
+    R = c.rotation()[0]
+    Rr, _ = orc.qr_pos_lapack(Z1[0])
+    # the absurd step left an ill-conditioned latent: R = Z U^-1 loses cond(Z) * 2^-17
+    cond = np.linalg.cond(Z1[0].astype(np.float64))
+    assert np.abs(R - Rr).max() <= 2e-5 * max(1.0, cond)
+    c.close()
+
+
+def test_incremental_qr_does_not_accumulate_error_over_many_steps():
+    """Forty steps of the default (incremental) factorisation, replayed from a CUDA graph: the rotation
+    reported at the end is the unique factor of the latent the handle holds, to the same accuracy as a
+    fresh Householder factorisation."""
+    w = small("c2_7b", d=512, n_tokens=1024, n_outlier_channels=3)
+    c = Calib(w)
+    c.step(40)
+    assert c.status() == dq.DQ_OK
+    Z = c.latent()[0].astype(np.float64)
+    R = c.rotation()[0]                     # incremental: the latent moved since the last factorisation
+    assert c.status() == dq.DQ_OK
+    Rr, _ = orc.qr_pos_lapack(Z)
+    assert np.abs(R - Rr).max() <= 5e-5
+    assert np.abs(R.T @ R - np.eye(w.d)).max() <= 5e-5
+    dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_HOUSEHOLDER, 0)
+    assert np.abs(c.rotation()[0] - Rr).max() <= 5e-5
+    c.close()
+
+
 def test_tensor_core_path_is_bit_reproducible():
     w = small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3)
     outs = []
