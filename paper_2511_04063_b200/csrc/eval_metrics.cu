@@ -93,6 +93,7 @@ dq_status eval_rotation(Ctx& ctx, const void* d_X, int x_dtype, int64_t n, int d
   DQ_CHECK_CUDA(cudaGetDevice(&dev));
   DQ_CHECK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ctx.sm_count = sms;
+  tch::keep_pool_memory(dev);
   int64_t chunk = (int64_t)(((int64_t)1 << 25) / d);            // 128 MiB of fp32 outputs at a time
   chunk = (chunk / 128) * 128;
   if (chunk < 128) chunk = 128;

@@ -89,6 +89,22 @@ dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, con
 
 using bf16 = __nv_bfloat16;
 
+// The stand-alone entry points take their scratch from the device's stream-ordered pool.  By default the
+// pool hands freed memory back to the driver at every synchronisation, which turns each later call into a
+// fresh device allocation; keep up to 1 GiB cached in this process's pool instead (set once per device).
+inline void keep_pool_memory(int dev) {
+  static bool done[64] = {};
+  if (dev < 0 || dev >= 64 || done[dev]) return;
+  cudaMemPool_t pool = nullptr;
+  if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess && pool) {
+    uint64_t cur = 0, want = (uint64_t)1 << 30;
+    if (cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &cur) == cudaSuccess && cur < want)
+      cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &want);
+  }
+  cudaGetLastError();
+  done[dev] = true;
+}
+
 // O[token][channel] = sum_k X[token][k] Rt[channel][k] for n token rows (bf16, row stride ldx) and a
 // d x d bf16 R^T; EPI = EPI_BF16 (bf16 rows, stride ldo) or EPI_GEN (fp32 rows).  CTA pairs with
 // 256 x 256 tiles when the shape allows, else the one-CTA kernel.  n % 128 == 0, d % 128 == 0.

@@ -194,6 +194,7 @@ dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t l
   DQ_CHECK_CUDA(cudaGetDevice(&dev));
   DQ_CHECK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   ctx.sm_count = sms;
+  tch::keep_pool_memory(dev);
   __nv_bfloat16* rt = nullptr;
   if (cudaMallocAsync((void**)&rt, sizeof(__nv_bfloat16) * (size_t)d * d, ctx.stream) != cudaSuccess)
     return DQ_ERR_ALLOC;
