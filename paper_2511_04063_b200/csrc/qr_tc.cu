@@ -387,6 +387,10 @@ dq_status qr_upper_factor_incremental(Ctx& ctx, QrWorkspace& ws, QrTcState& q, c
     if (it > 0) {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
       Op tt{q.tw_hi, q.tw_lo, d, dd};
       Out o; o.f32 = P; o.ld = d; o.bs = dd; o.k_mode = 2; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
+      // Only the last sweep's product enters the returned factor at full weight: the fixed point
+      // T* = Phi(E - T*^T T*) forgives an error e in an earlier product by a factor ||T|| per later sweep,
+      // so the earlier sweeps use plain bf16 operands (relative error 2^-9 on a term of size ||T||^2).
+      if (!last) o.nterms = 1;
       DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
     }
     chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, it > 0 ? P : nullptr, T, q.tw_hi, q.tw_lo,

@@ -141,6 +141,7 @@ struct Out {
   int tri_skip = 0, k_mode = 0;   // triangular structure, see tc::Params
   const int* tile_list = nullptr; int n_list = 0;   // explicit tile order (device), see tc::Params
   const int* tile_list2 = nullptr; int n_list2 = 0; // the same order in 256 x 256 tiles (two-CTA kernel)
+  int nterms = 3;   // 1: plain bf16 product of the hi parts only (2^-9 relative), a third of the MMAs
 };
 
 // D[m][n] = alpha sum_k A[m][k] B[n][k] (+ beta D) with split-bf16 operands (three bf16 MMAs per
@@ -166,7 +167,8 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
     p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
     p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
     p.tile_list = o.tile_list2; p.n_list = o.n_list2;
-    return launch_gemm2<3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
+    return o.nterms == 1 ? launch_gemm2<1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
+                         : launch_gemm2<3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
   }
   DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, tc::BLOCK_M));
   DQ_CHECK(make_map(&mal, A.lo, K, M, batch, A.ld, bsa, tc::BLOCK_M));
@@ -180,7 +182,8 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
   if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
   p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
   p.tile_list = o.tile_list; p.n_list = o.n_list;
-  return launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
+  return o.nterms == 1 ? launch_gemm<128, 1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
+                       : launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
 }
 
 }  // namespace tch
