@@ -217,7 +217,9 @@ def main():
     # ---------------------------------------------------------------- per-phase times (events inside the library)
     dq.dq_calib_set_timing(h, True)
     n_phase_steps = min(K, 5)
+    flops0 = dq.dq_calib_mma_flops(h)
     dq.dq_calib_step(h, n_phase_steps, loss_dev)
+    mma_flops_per_step = (dq.dq_calib_mma_flops(h) - flops0) / n_phase_steps
     phases = dq.dq_calib_get_timings(h)
     dq.dq_calib_set_timing(h, False)
 
@@ -382,6 +384,18 @@ def main():
             line["qr_" + other_qr] = {"value": world * 1e3 / alt["ms_per_step"], "unit": UNIT,
                                     "ms_per_step": alt["ms_per_step"], "phases_ms": alt["phases_ms"],
                                     "qr_orth_share": (alt["phases_ms"]["qr_forward"] + alt["phases_ms"]["qr_backward"]) / ta}
+        if path == dq.DQ_PATH_BF16_TC and d != 128:
+            # issued bf16 MMA flops (counted by the library at launch: three products per split-bf16 term, k clipped
+            # to the non-zero blocks of triangular operands) over the event-timed phases that issue them
+            qr_flops = mma_flops_per_step - 2 * fwd_flops
+            t_qr = (phases["qr_forward"] + phases["qr_backward"]) * 1e-3
+            t_all = t_qr + (phases["rotate_whip"] + phases["grad_rotation"]) * 1e-3
+            line["mma_issued"] = {"flops_per_step": mma_flops_per_step,
+                                  "step_tflops": mma_flops_per_step / t_all / 1e12,
+                                  "qr_orth_flops_per_step": qr_flops,
+                                  "qr_orth_tflops": qr_flops / t_qr / 1e12 if t_qr > 0 else None,
+                                  "qr_orth_frac_of_measured_burst": qr_flops / t_qr / 1e12 / peaks["bf16_tflops"],
+                                  "note": "QR-Orth phases also hold their HBM-bound element-wise kernels"}
         if rot is not None:
             # includes the fp32 -> bf16 transpose of R (d^2 entries) in front of the contraction
             line["rotate_apply"] = {"ms": rot, "tflops": 2.0 * N * d * d / (rot * 1e-3) / 1e12,

@@ -161,7 +161,9 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
  *     dq_calib_set_qr_method(h, DQ_QR_HOUSEHOLDER, 0) (or more sweeps, or a lower learning rate) and
  *     step again.  n_iters <= 0 selects the default (5).
  *   DQ_QR_HOUSEHOLDER: blocked Householder QR at every step; no assumption on the step size.
- * The call clears the status word.  Ignored (DQ_OK) on the fp32 path and for d == 128. */
+ * The call clears the status word.  For d == 128 (any path) the same two methods exist as kernels that
+ * keep a whole latent in shared memory; there the sweeps stop as soon as no entry moves (one more is
+ * taken) and n_iters only bounds them (8 n_iters).  Otherwise ignored (DQ_OK) on the fp32 path. */
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 
@@ -268,6 +270,12 @@ dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int6
 
 /* Number of kernels this library launched through the handle so far. */
 int64_t dq_calib_launch_count(dq_calib_t* h);
+
+/* bf16 tensor-core flops the handle's tcgen05 kernels were asked to issue so far (2 m n k per MMA
+ * product, three products per split-bf16 term, k clipped to the non-zero blocks of triangular
+ * operands exactly as the kernels clip it; counted on the host at launch).  For measurement:
+ * the difference across a timed region divided by its duration is the issued MMA rate. */
+double dq_calib_mma_flops(dq_calib_t* h);
 
 const char* dq_status_string(dq_status s);
 void dq_calib_destroy(dq_calib_t* h);

@@ -46,6 +46,7 @@ struct dq_calib {
   int orth_method = DQ_ORTH_QR;
   CayleyState cay;              // DQ_ORTH_CAYLEY: momentum and step size
   bool cay_started = false;     // R and its split copies hold the Cayley iterate
+  bool small_warm = false;      // d == 128: U and U^-1 hold the factors of the previous step's latent
   bool small128 = false;        // d == 128: shared-memory-resident batched QR-Orth
   bool r_stale = true;
   bool timing = false;
@@ -55,6 +56,7 @@ struct dq_calib {
   // one whole step (QR forward .. update) captured once and replayed
   cudaGraphExec_t graph = nullptr;
   int64_t graph_launches = 0;
+  double graph_flops = 0.0;
   bool graph_failed = false;
   int eager_steps_done = 0;
 };
@@ -128,8 +130,13 @@ dq_status ensure_rotation(dq_calib* h) {
   if (h->orth_method == DQ_ORTH_CAYLEY && h->cay_started) return DQ_OK;   // R is the iterate itself
   if (!h->r_stale) return DQ_OK;
   if (h->small128) {
-    DQ_CHECK(qr128_forward(h->ctx, h->Z, h->R, h->U, h->ws.Winv,
-                           h->cfg.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr, h->cfg.batch));
+    __nv_bfloat16* rt = h->cfg.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr;
+    if (h->qr_method == DQ_QR_ITERATIVE && h->small_warm) {
+      DQ_CHECK(qr128_forward_incremental(h->ctx, h->Z, h->R, h->U, h->ws.Winv, rt, h->qr_iters, h->cfg.batch));
+    } else {
+      DQ_CHECK(qr128_forward(h->ctx, h->Z, h->R, h->U, h->ws.Winv, rt, h->cfg.batch));
+      h->small_warm = true;
+    }
   } else if (h->fast_qr) {
     DQ_CHECK(qr_forward_fast(h->ctx, h->ws, h->qtc, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch,
                              h->qr_method == DQ_QR_ITERATIVE ? h->qr_iters : 0));
@@ -219,7 +226,7 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
     return DQ_OK;
   }
   if (h->small128) {   // plain SGD is fused into the backward kernel; other optimisers follow it
-    DQ_CHECK(qr128_backward_sgd(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, h->optimizer == DQ_SGD ? c.lr : 0.f, batch));
+    DQ_CHECK(qr128_backward_sgd_tc(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, h->optimizer == DQ_SGD ? c.lr : 0.f, batch));
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
   } else {
     if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch));
@@ -241,6 +248,7 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
 void try_capture(dq_calib* h) {
   if (h->graph || h->graph_failed) return;
   const int64_t before = h->ctx.launches;
+  const double flops_before = h->ctx.mma_flops;
   h->r_stale = true;
   if (cudaStreamBeginCapture(h->ctx.stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();
@@ -255,6 +263,7 @@ void try_capture(dq_calib* h) {
     if (g) cudaGraphDestroy(g);
     h->graph_failed = true;
     h->ctx.launches = before;
+    h->ctx.mma_flops = flops_before;
     h->r_stale = true;
     return;
   }
@@ -265,7 +274,9 @@ void try_capture(dq_calib* h) {
   }
   cudaGraphDestroy(g);
   h->graph_launches = h->ctx.launches - before;
+  h->graph_flops = h->ctx.mma_flops - flops_before;
   h->ctx.launches = before;      // capture enqueued nothing
+  h->ctx.mma_flops = flops_before;
   h->r_stale = true;
 }
 
@@ -370,15 +381,17 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
   for (int s = 0; s < n_steps; ++s) {
     // The captured step of the iterative QR is the incremental one: replay it only while the
     // previous step's factors belong to the latent one optimiser step back.
-    const bool iterative = h->fast_qr && !h->small128 && h->qr_method == DQ_QR_ITERATIVE;
+    const bool iterative = h->qr_method == DQ_QR_ITERATIVE && (h->small128 || h->fast_qr);
+    const bool warm = h->small128 ? h->small_warm : h->qtc.t_warm;
     const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
     const bool use_graph = cayley ? (!h->timing && h->cay_started && h->eager_steps_done >= 1)
                                   : (!h->timing && h->r_stale && h->eager_steps_done >= 1 &&
-                                     (!iterative || h->qtc.t_warm));
+                                     (!iterative || warm));
     if (use_graph && !h->graph && !h->graph_failed) try_capture(h);
     if (use_graph && h->graph) {
       DQ_CHECK_CUDA(cudaGraphLaunch(h->graph, ctx.stream));
       ctx.launches += h->graph_launches;
+      ctx.mma_flops += h->graph_flops;
       h->r_stale = !cayley;
     } else {
       DQ_CHECK(enqueue_step(h, h->timing));
@@ -461,6 +474,7 @@ dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z) {
   DQ_CHECK(clear_status(h));
   h->r_stale = true;
   h->qtc.t_warm = false;   // the new latent may be far from the one the iterative QR last saw
+  h->small_warm = false;
   h->cay_started = false;  // Cayley SGD restarts from the orthogonal factor of the new latent
   return fence_out(h);
 }
@@ -511,6 +525,7 @@ dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters)
   h->qr_iters = iters;
   h->r_stale = true;
   h->qtc.t_warm = false;
+  h->small_warm = false;
   if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
   h->graph_failed = false;
   return DQ_OK;
@@ -594,6 +609,8 @@ dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int6
 }
 
 int64_t dq_calib_launch_count(dq_calib_t* h) { return h ? h->ctx.launches : 0; }
+
+double dq_calib_mma_flops(dq_calib_t* h) { return h ? h->ctx.mma_flops : 0.0; }
 
 void dq_calib_destroy(dq_calib_t* h) {
   if (!h) return;

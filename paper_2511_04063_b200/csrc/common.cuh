@@ -15,6 +15,7 @@ struct Ctx {
   cudaStream_t stream = nullptr;
   int* d_status = nullptr;
   int64_t launches = 0;
+  double mma_flops = 0.0;   // bf16 tensor-core flops issued by the tcgen05 kernels (counted on the host)
   int sm_count = 148;
 };
 
@@ -102,6 +103,13 @@ dq_status qr_backward(Ctx& ctx, QrWorkspace& ws, const float* R, const float* U,
 dq_status qr128_forward(Ctx& ctx, const float* Z, float* R, float* U, float* W, __nv_bfloat16* Rt_bf16, int batch);
 dq_status qr128_backward_sgd(Ctx& ctx, const float* R, const float* W, const float* Gq, float* Gz, float* Z, float lr,
                              int batch);
+
+// Tensor-core variants (qr128_inc.cu): incremental forward from the previous step's U and W (both updated
+// in place) and the backward with warp-level MMAs.
+dq_status qr128_forward_incremental(Ctx& ctx, const float* Z, float* R, float* U, float* W, __nv_bfloat16* Rt_bf16,
+                                    int n_sweeps, int batch);
+dq_status qr128_backward_sgd_tc(Ctx& ctx, const float* R, const float* W, const float* Gq, float* Gz, float* Z,
+                                float lr, int batch);
 
 // out[i] = X[pi_seed(first + i)] for i < count: seeded sampling of token rows without replacement
 // (token_sampling.cu).  elem_bytes = 2 (bf16) or 4 (fp32); rows must be multiples of 16 bytes.

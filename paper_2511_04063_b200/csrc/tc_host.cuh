@@ -144,6 +144,24 @@ struct Out {
   int nterms = 3;   // 1: plain bf16 product of the hi parts only (2^-9 relative), a third of the MMAs
 };
 
+// 64-wide k-blocks the kernels run for a product: the same clipping as their k_range, over all tiles or
+// (upper) over the tiles with mb <= nb.  unit = tile edge (128 or 256).
+inline int64_t count_kblocks(int m_tiles, int n_tiles, int k_blocks, int k_mode, bool upper, int unit) {
+  const int R = unit / tc::BLOCK_K;
+  int64_t total = 0;
+  for (int nb = 0; nb < n_tiles; ++nb)
+    for (int mb = 0; mb < m_tiles; ++mb) {
+      if (upper && mb > nb) continue;
+      int lo = 0, hi = k_blocks;
+      if ((k_mode & 1) && lo < R * mb) lo = R * mb;
+      if ((k_mode & 8) && lo < R * nb) lo = R * nb;
+      if ((k_mode & 2) && hi > R * (mb + 1)) hi = R * (mb + 1);
+      if ((k_mode & 4) && hi > R * (nb + 1)) hi = R * (nb + 1);
+      if (hi > lo) total += hi - lo;
+    }
+  return total;
+}
+
 // D[m][n] = alpha sum_k A[m][k] B[n][k] (+ beta D) with split-bf16 operands (three bf16 MMAs per
 // product, fp32 accumulation); M, N % 128 == 0, K % 64 == 0.
 inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, int batch, const Out& o) {
@@ -167,6 +185,11 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
     p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
     p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
     p.tile_list = o.tile_list2; p.n_list = o.n_list2;
+    {
+      const bool upper = o.tri_skip || (o.tile_list2 && o.n_list2 < p.m_blocks * p.n_blocks);
+      ctx.mma_flops += (double)count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode, upper, 256) *
+                       (2.0 * 256 * 256 * tc::BLOCK_K) * (o.nterms == 1 ? 1 : 3) * batch;
+    }
     return o.nterms == 1 ? launch_gemm2<1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
                          : launch_gemm2<3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
   }
@@ -182,6 +205,11 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
   if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
   p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
   p.tile_list = o.tile_list; p.n_list = o.n_list;
+  {
+    const bool upper = o.tri_skip || (o.tile_list && o.n_list < p.m_blocks * p.n_blocks);
+    ctx.mma_flops += (double)count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode, upper, 128) *
+                     (2.0 * 128 * 128 * tc::BLOCK_K) * (o.nterms == 1 ? 1 : 3) * batch;
+  }
   return o.nterms == 1 ? launch_gemm<128, 1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
                        : launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
 }

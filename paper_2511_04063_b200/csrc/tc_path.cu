@@ -135,6 +135,7 @@ void tc_destroy(TcState& tc) {
 // O^T = R^T X^T per 128 x 256 tile (rows = channels, columns = tokens), Whip epilogue:
 // writes G^T (bf16, channel-major) and 4 loss partials per tile.
 dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
+  ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;
   Maps* m = reinterpret_cast<Maps*>(tc.maps);
   tc::Params p{};
   p.m_blocks = tc.d / tc::BLOCK_M; p.n_blocks = (int)(tc.n_tokens / 256); p.batch = tc.batch; p.ksplit = 1;
@@ -150,6 +151,7 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
 
 // Gq = scale * X^T G : A = X^T [d][N], B = G^T [d][N], reduction over tokens.
 dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
+  ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;
   Maps* m = reinterpret_cast<Maps*>(tc.maps);
   const int d = tc.d;
   const int bn = (d % 256 == 0) ? 256 : 128;
