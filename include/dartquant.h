@@ -268,6 +268,12 @@ enum {
 };
 dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int64_t* n_elems);
 
+/* For d == 128 on the tensor-core path both contractions and the Eq. 4 epilogue run in one kernel and
+ * dL/dO never leaves the chip, so DQ_BUF_G is not written.  keep != 0 makes that kernel store dL/dO to
+ * DQ_BUF_G as well (for inspection and tests; the results of a step do not change).  No effect on
+ * other shapes, where DQ_BUF_G is always written. */
+dq_status dq_calib_set_keep_gradient(dq_calib_t* h, int32_t keep);
+
 /* Number of kernels this library launched through the handle so far. */
 int64_t dq_calib_launch_count(dq_calib_t* h);
 

@@ -30,7 +30,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_get_latent", "dq_calib_set_latent", "dq_calib_refresh_inputs", "dq_calib_status",
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
     "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens", "dq_eval_rotation",
-    "dq_calib_set_orth_method", "dq_calib_set_objective", "dq_calib_run_epochs", "dq_calib_mma_flops",
+    "dq_calib_set_orth_method", "dq_calib_set_objective", "dq_calib_run_epochs", "dq_calib_mma_flops", "dq_calib_set_keep_gradient",
 )
 
 
@@ -86,6 +86,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_get_timings.argtypes = [vp, C.POINTER(C.c_float), i32]
     lib.dq_calib_set_timing.argtypes = [vp, i32]
     lib.dq_calib_debug_buffer.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i64)]
+    lib.dq_calib_set_keep_gradient.argtypes = [vp, i32]
+    lib.dq_calib_set_keep_gradient.restype = i32
     lib.dq_calib_launch_count.argtypes = [vp]
     lib.dq_calib_mma_flops.argtypes = [vp]
     lib.dq_calib_mma_flops.restype = C.c_double
@@ -186,6 +188,10 @@ def dq_calib_run_epochs(h, pool, sample_ratio: float, accum: int, n_epochs: int,
                                               n_epochs, seed, loss_out.data_ptr() if loss_out is not None else None,
                                               C.byref(steps)), "dq_calib_run_epochs")
     return int(steps.value)
+
+
+def dq_calib_set_keep_gradient(h, keep: bool = True):
+    _check(load_library().dq_calib_set_keep_gradient(h, 1 if keep else 0), "dq_calib_set_keep_gradient")
 
 
 def dq_calib_mma_flops(h) -> float:

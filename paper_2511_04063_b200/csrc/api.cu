@@ -186,7 +186,8 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
       } else {
         DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
       }
-      DQ_CHECK(loss_finalize(ctx, h->partials, h->n_partials, batch, inv_n, nullptr, loss_dst));
+      DQ_CHECK(loss_finalize(ctx, h->partials, c.path == DQ_PATH_BF16_TC ? h->tc.n_partials_live : h->n_partials, batch,
+                             inv_n, nullptr, loss_dst));
     }
     if (timed && a == n_micro - 1) DQ_CHECK_CUDA(cudaEventRecord(h->ev[2], ctx.stream));
     // (a5) Gq = (1/N) X^T G
@@ -571,6 +572,17 @@ dq_status dq_calib_set_orth_method(dq_calib_t* h, int32_t method, float beta, fl
   h->r_stale = true;
   h->qtc.t_warm = false;
   if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
+  h->graph_failed = false;
+  return DQ_OK;
+}
+
+dq_status dq_calib_set_keep_gradient(dq_calib_t* h, int32_t keep) {
+  if (!h) return DQ_ERR_INVALID_ARG;
+  const bool k = keep != 0;
+  if (k == h->tc.keep_g) return DQ_OK;
+  DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
+  h->tc.keep_g = k;
+  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the kernel arguments changed: capture again
   h->graph_failed = false;
   return DQ_OK;
 }

@@ -1,0 +1,267 @@
+// Fused Whip step for many 128 x 128 rotations (per-head rotations): one kernel computes, per head h
+// and per tile of 128 tokens,
+//   O^T = R_h^T X_t^T   (tcgen05, accumulator in tensor memory)
+//   e = exp(-|o|), loss partials, G = -sign(o) e   (Eq. 4; epilogue from tensor memory)
+//   Gq_h += X_t^T G_t    (second tcgen05 product: G_t goes from the epilogue's registers into shared
+//                         memory as the K-major operand, the accumulator stays in tensor memory
+//                         for all tiles of the unit)
+// so the rotated activations and dL/dO never reach HBM; X is read once in each orientation.
+// R_h^T stays resident in shared memory for a unit (head, range of token tiles); every unit writes
+// one 128 x 128 fp32 partial of Gq and four loss partials, summed afterwards in a fixed order.
+//
+// 192 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue.  Two operand stages,
+// two O accumulators, two G buffers.  Every wait is bounded (DQ_ERR_TIMEOUT on expiry).
+#pragma once
+#include "tc_gemm.cuh"
+
+namespace dq {
+namespace heads {
+
+using namespace tc;
+
+constexpr int KB_BYTES = 128 * BLOCK_K * 2;        // one [128 rows][64 bf16] K-major block: 16 KB
+constexpr int RT_BYTES = 2 * KB_BYTES;             // R_h^T: rows = output channel, K = input channel (128)
+constexpr int XA_BYTES = 2 * KB_BYTES;             // X_t:   rows = token, K = input channel
+constexpr int XT_BYTES = 2 * KB_BYTES;             // X_t^T: rows = input channel, K = token
+constexpr int STAGE_BYTES = XA_BYTES + XT_BYTES;
+constexpr int G_BYTES = 2 * KB_BYTES;              // G_t^T: rows = output channel, K = token
+constexpr int STAGES = 2;
+constexpr int SMEM_TOTAL = RT_BYTES + STAGES * STAGE_BYTES + 2 * G_BYTES + 1024 + 1024;
+constexpr uint32_t TMEM_COLS = 512;                // O (2 x 128 columns) + Gq (128 columns)
+
+struct Params {
+  int batch, tiles_per_head, splits;   // units = batch * splits; unit u = head u / splits, slice u % splits
+  int64_t n_tokens;
+  float* part;                         // [units][128][128] partial Gq (row = input channel)
+  float* partials;                     // [units][4] loss partials
+  __nv_bfloat16* Gt;                   // nullable: also store dL/dO, [batch][128][n_tokens] channel-major
+  int* d_status;
+};
+
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_constant__ CUtensorMap mapX,
+                  const __grid_constant__ CUtensorMap mapXt, const Params p) {
+  constexpr uint32_t IDESC = make_idesc_bf16(128);
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t rt_smem = smem_base;
+  const uint32_t stage_base = rt_smem + RT_BYTES;
+  const uint32_t g_base = stage_base + STAGES * STAGE_BYTES;
+  const uint32_t bar_base = g_base + 2 * G_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (2 + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (4 + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (6 + a); };
+  auto gfull_bar = [&](int g) { return bar_base + 8u * (8 + g); };
+  auto gempty_bar = [&](int g) { return bar_base + 8u * (10 + g); };
+  const uint32_t rtfull_bar = bar_base + 8u * 12, rtempty_bar = bar_base + 8u * 13;
+  const uint32_t qfull_bar = bar_base + 8u * 14, qempty_bar = bar_base + 8u * 15;
+  const uint32_t tmem_slot = bar_base + 8u * 16;
+  uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+  uint8_t* g_ptr = smem_raw + (g_base - smem_u32(smem_raw));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1);
+      mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), 4);
+      mbar_init(gfull_bar(s), 4); mbar_init(gempty_bar(s), 1);
+    }
+    mbar_init(rtfull_bar, 1); mbar_init(rtempty_bar, 1);
+    mbar_init(qfull_bar, 1); mbar_init(qempty_bar, 4);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    prefetch_tensormap(&mapRt); prefetch_tensormap(&mapX); prefetch_tensormap(&mapXt);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  const uint32_t tmem_q = tmem_base + 256u;
+
+  const int units = p.batch * p.splits;
+  auto unit_range = [&](int u, int& b, int& t0, int& t1) {
+    b = u / p.splits;
+    const int s = u % p.splits;
+    t0 = (int)(((int64_t)s * p.tiles_per_head) / p.splits);
+    t1 = (int)(((int64_t)(s + 1) * p.tiles_per_head) / p.splits);
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0, rt_phase = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        int b, t0, t1;
+        unit_range(u, b, t0, t1);
+        if (!mbar_wait(rtempty_bar, rt_phase ^ 1u, p.d_status)) break;
+        rt_phase ^= 1u;
+        mbar_expect_tx(rtfull_bar, RT_BYTES);
+        tma_load_3d(rt_smem, &mapRt, rtfull_bar, 0, 0, b);
+        tma_load_3d(rt_smem + KB_BYTES, &mapRt, rtfull_bar, BLOCK_K, 0, b);
+        for (int t = t0; t < t1; ++t) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
+          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          const uint32_t xa = stage_base + stage * STAGE_BYTES, xt = xa + XA_BYTES;
+          tma_load_3d(xa, &mapX, full_bar(stage), 0, t * 128, b);
+          tma_load_3d(xa + KB_BYTES, &mapX, full_bar(stage), BLOCK_K, t * 128, b);
+          tma_load_3d(xt, &mapXt, full_bar(stage), t * 128, 0, b);
+          tma_load_3d(xt + KB_BYTES, &mapXt, full_bar(stage), t * 128 + BLOCK_K, 0, b);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      int st1 = 0, st2 = 0, acc = 0, g = 0;
+      uint32_t ph1 = 0, acc_phase = 0, g_phase = 0, rt_phase = 0, q_phase = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        int b, t0, t1;
+        unit_range(u, b, t0, t1);
+        const int nt = t1 - t0;
+        if (!mbar_wait(rtfull_bar, rt_phase, p.d_status)) break;
+        rt_phase ^= 1u;
+        tc_fence_after();
+        for (int i = 0; i <= nt && ok; ++i) {
+          if (i < nt) {   // O^T of tile i
+            if (!mbar_wait(full_bar(st1), ph1, p.d_status)) { ok = false; break; }
+            if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t xa = stage_base + st1 * STAGE_BYTES;
+            const uint32_t tmem_o = tmem_base + (uint32_t)(acc * 128);
+#pragma unroll
+            for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+              for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                umma_bf16(tmem_o, make_kmajor_sw128_desc(rt_smem + kb * KB_BYTES + k * UMMA_K * 2),
+                          make_kmajor_sw128_desc(xa + kb * KB_BYTES + k * UMMA_K * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+            umma_commit(tfull_bar(acc));
+            if (i == nt - 1) umma_commit(rtempty_bar);   // R_h^T may be replaced once these products retire
+            if (++st1 == STAGES) { st1 = 0; ph1 ^= 1u; }
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+          }
+          if (i > 0) {    // Gq += X_t^T G_t of tile i - 1
+            const int j = i - 1;
+            if (j == 0) {   // the accumulator of the previous unit has been read out
+              if (!mbar_wait(qempty_bar, q_phase ^ 1u, p.d_status)) { ok = false; break; }
+              q_phase ^= 1u;
+            }
+            if (!mbar_wait(gfull_bar(g), g_phase, p.d_status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t xt = stage_base + st2 * STAGE_BYTES + XA_BYTES;
+            const uint32_t gb = g_base + g * G_BYTES;
+#pragma unroll
+            for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+              for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                umma_bf16(tmem_q, make_kmajor_sw128_desc(xt + kb * KB_BYTES + k * UMMA_K * 2),
+                          make_kmajor_sw128_desc(gb + kb * KB_BYTES + k * UMMA_K * 2), IDESC,
+                          (j > 0 || kb > 0 || k > 0) ? 1u : 0u);
+            umma_commit(empty_bar(st2));    // both operand tiles of the stage are consumed
+            umma_commit(gempty_bar(g));
+            if (j == nt - 1) umma_commit(qfull_bar);
+            if (++st2 == STAGES) st2 = 0;
+            if (++g == 2) { g = 0; g_phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------- epilogue (warps 2..5)
+    const int q = warp & 3;
+    const int row = q * 32 + lane;             // output channel (O^T, G^T) / input channel (Gq)
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    int acc = 0, g = 0;
+    uint32_t acc_phase = 0, g_phase = 0, q_phase = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      int b, t0, t1;
+      unit_range(u, b, t0, t1);
+      float esum = 0.f;
+      for (int t = t0; t < t1; ++t) {
+        if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
+        if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }
+        tc_fence_after();
+        uint8_t* gbuf = g_ptr + g * G_BYTES;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * 128 + c * 32), v);
+          tmem_ld_wait();
+          uint32_t packed[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
+            const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
+            esum += e0 + e1;
+            const float g0 = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
+            const float g1 = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
+            const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
+            packed[i] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+          // tokens 32 c .. 32 c + 31 of row `row`: k-block c >> 1, 16-byte chunks 4 (c & 1) .. + 3,
+          // stored where the 128-byte swizzle of a K-major tile expects them
+          uint8_t* rowp = gbuf + (c >> 1) * KB_BYTES + row * 128;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int chunk = ((c & 1) * 4 + i) ^ (row & 7);
+            *reinterpret_cast<uint4*>(rowp + chunk * 16) =
+                make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+          }
+          if (p.Gt) {
+            uint4* dst = reinterpret_cast<uint4*>(p.Gt + ((int64_t)b * 128 + row) * p.n_tokens + (int64_t)t * 128 + c * 32);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+          }
+        }
+        tc_fence_before();
+        fence_async_smem();                    // the tensor core reads G through the async proxy
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(tempty_bar(acc)); mbar_arrive(gfull_bar(g)); }
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (++g == 2) { g = 0; g_phase ^= 1u; }
+      }
+      if (!ok) break;
+      // partial Gq of the unit
+      if (!mbar_wait(qfull_bar, q_phase, p.d_status)) { ok = false; break; }
+      q_phase ^= 1u;
+      tc_fence_after();
+      float* dst_row = p.part + ((int64_t)u * 128 + row) * 128;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tmem_q + lane_addr + (uint32_t)(c * 32), v);
+        tmem_ld_wait();
+        float4* dst = reinterpret_cast<float4*>(dst_row + c * 32);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                               __uint_as_float(v[4 * i + 3]));
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(qempty_bar);
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) esum += __shfl_xor_sync(0xffffffffu, esum, off);
+      if (lane == 0) p.partials[(int64_t)u * 4 + q] = esum;
+    }
+  }
+
+  // ------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace heads
+}  // namespace dq

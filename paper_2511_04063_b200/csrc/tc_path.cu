@@ -1,6 +1,7 @@
 // Host side of the tensor-core path: tensor maps, operand copies, launches.
 #include <vector>
 
+#include "tc_heads.cuh"
 #include "tc_host.cuh"
 #include "tc_path.cuh"
 
@@ -112,6 +113,20 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   DQ_CHECK(tch::make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
   DQ_CHECK(tch::make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
   DQ_CHECK(tc_refresh_inputs(tc, ctx));
+  if (d == 128) {   // per-head rotations: fused kernel, units = (head, range of 128-token tiles)
+    const int tiles_per_head = (int)(N / 128);
+    int sp = ctx.sm_count / batch;
+    if (sp > (int)(N / 256)) sp = (int)(N / 256);   // the loss-partial buffer holds N / 256 x 4 values per head
+    if (sp > tiles_per_head) sp = tiles_per_head;
+    if (sp < 1) sp = 1;
+    tc.splits = sp;
+    if (cudaMalloc((void**)&tc.heads_part, sizeof(float) * (size_t)batch * sp * 128 * 128) != cudaSuccess)
+      return DQ_ERR_ALLOC;
+    if (cudaFuncSetAttribute(heads::heads_whip_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             heads::SMEM_TOTAL) != cudaSuccess)
+      return DQ_ERR_CUDA;
+    tc.fused = true;
+  }
   tc.n_partials = (d / tc::BLOCK_M) * (int)(N / 256) * 4;
   *n_partials = tc.n_partials;
   tc.ready = true;
@@ -127,7 +142,7 @@ dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx) {
 
 void tc_destroy(TcState& tc) {
   cudaFree(tc.Xt); if (!tc.rt_external) cudaFree(tc.Rt); cudaFree(tc.part);
-  cudaFree(tc.tl_head); cudaFree(tc.tl_tail); cudaFree(tc.tail_part);
+  cudaFree(tc.tl_head); cudaFree(tc.tl_tail); cudaFree(tc.tail_part); cudaFree(tc.heads_part);
   delete reinterpret_cast<Maps*>(tc.maps);
   tc = TcState();
 }
@@ -136,6 +151,22 @@ void tc_destroy(TcState& tc) {
 // writes G^T (bf16, channel-major) and 4 loss partials per tile.
 dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
   ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;
+  tc.n_partials_live = tc.n_partials;
+  tc.fused_valid = false;
+  if (tc.fused) {
+    Maps* mm = reinterpret_cast<Maps*>(tc.maps);
+    heads::Params hp{};
+    hp.batch = tc.batch; hp.tiles_per_head = (int)(tc.n_tokens / 128); hp.splits = tc.splits;
+    hp.n_tokens = tc.n_tokens; hp.part = tc.heads_part; hp.partials = partials;
+    hp.Gt = tc.keep_g ? tc.Gt : nullptr; hp.d_status = ctx.d_status;
+    const int units = tc.batch * tc.splits;
+    const int grid = units < ctx.sm_count ? units : ctx.sm_count;
+    heads::heads_whip_kernel<<<grid, tc::NUM_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x128, mm->xt, hp);
+    tc.n_partials_live = tc.splits * 4;
+    tc.fused_valid = true;
+    ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;   // the second product runs here too
+    return after_launch(ctx);
+  }
   Maps* m = reinterpret_cast<Maps*>(tc.maps);
   tc::Params p{};
   p.m_blocks = tc.d / tc::BLOCK_M; p.n_blocks = (int)(tc.n_tokens / 256); p.batch = tc.batch; p.ksplit = 1;
@@ -151,6 +182,8 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
 
 // Gq = scale * X^T G : A = X^T [d][N], B = G^T [d][N], reduction over tokens.
 dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
+  if (tc.fused && tc.fused_valid)   // the fused kernel left one partial per unit: sum them in a fixed order
+    return splitk_reduce(ctx, tc.heads_part, tc.splits, (int64_t)tc.d * tc.d, tc.batch, scale, 0.f, Gq);
   ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;
   Maps* m = reinterpret_cast<Maps*>(tc.maps);
   const int d = tc.d;

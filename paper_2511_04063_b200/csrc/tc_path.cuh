@@ -24,6 +24,13 @@ struct TcState {
   int* tl_tail = nullptr; int n_tail = 0;
   int tail_split = 1;
   float* tail_part = nullptr;         // [tail_split][d][d] (only the tail tiles are touched)
+  // d == 128: both contractions and the Eq. 4 epilogue in one kernel (tc_heads.cuh); dL/dO stays on chip
+  bool fused = false;
+  int splits = 1;                     // units per head (each covers a range of token tiles)
+  float* heads_part = nullptr;        // [batch * splits][128][128] partial Gq
+  bool keep_g = false;                // also store dL/dO to Gt (inspection / tests)
+  bool fused_valid = false;           // heads_part holds the partials of the current step
+  int n_partials_live = 0;            // loss partials per problem written by the last forward
 };
 
 dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void* d_X,

@@ -30,6 +30,7 @@ class Calib:
         self.h = dq.dq_calib_init(self.X, self.Z0, lr=w.lr if lr is None else lr, path=path_of(w),
                                   reduction=reduction)
         self.dd = (w.batch, w.d, w.d)
+        dq.dq_calib_set_keep_gradient(self.h, True)    # the tests read dL/dO (DQ_BUF_G) at every shape
 
     def step(self, n=1):
         loss = torch.empty((n, self.w.batch), dtype=torch.float32, device="cuda")

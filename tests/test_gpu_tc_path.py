@@ -235,3 +235,37 @@ def test_rotate_apply_bf16(n, d):
     # bf16 operands (2^-9) and bf16 output (2^-9): a few 1e-2 absolute on O(1..4) values
     assert np.abs(got - ref).max() <= 6e-2
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-2
+
+
+@pytest.mark.parametrize("batch,n", [(4, 2048), (160, 256), (3, 768)])
+def test_fused_per_head_kernel_with_and_without_stored_gradient(batch, n):
+    """d = 128: one kernel computes O, Eq. 4, dL/dO and X^T dL/dO with dL/dO kept on chip.  Storing dL/dO
+    as well (what the other tests switch on to read it) must not change any result; more heads than SMs
+    makes every CTA run several units back to back, 768 tokens gives an uneven split of the token tiles."""
+    w = small("c3_heads", d=128, n_tokens=n, batch=batch)
+    outs = []
+    for keep in (True, False):
+        c = Calib(w)
+        dq.dq_calib_set_keep_gradient(c.h, keep)
+        loss = c.step(2)
+        assert c.status() == dq.DQ_OK
+        outs.append((loss, c.buf(dq.DQ_BUF_GQ).cpu().numpy().copy(), c.latent()))
+        if keep:
+            Z0 = c.Z0_host
+            Gq = outs[0][1]
+        c.close()
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(a, b)
+    # against the oracle, first step, a few heads (the second step's dL/dR is what Gq holds: recompute it)
+    c = Calib(w)
+    loss0 = c.step(1)[0]
+    Gq0 = c.buf(dq.DQ_BUF_GQ).cpu().numpy().astype(np.float64)
+    Gt = c.buf(dq.DQ_BUF_G, dtype=torch.bfloat16, shape=(batch, 128, n)).float().cpu().numpy().astype(np.float64)
+    for b in sorted({0, batch // 2, batch - 1}):
+        X = x_f64(w, c.X_host, b)
+        dO = 8.0 * np.linalg.norm(X, axis=1) / np.sqrt(128) * 2.0 ** -9 + 1e-3
+        ref = orc.calib_step(X, c.Z0_host[b], w.lr, sign_decider=sign_decider_from_gpu(Gt[b].T, 2.0 * dO[:, None]),
+                             qr=orc.qr_pos_lapack)
+        assert abs(loss0[b] - ref["loss"]) <= LOSS_TOL_BF16 * ref["loss"]
+        assert np.linalg.norm(Gq0[b] - ref["Gq"]) <= 5e-2 * np.linalg.norm(ref["Gq"])
+    c.close()
