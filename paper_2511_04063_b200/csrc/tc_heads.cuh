@@ -9,8 +9,10 @@
 // R_h^T stays resident in shared memory for a unit (head, range of token tiles); every unit writes
 // one 128 x 128 fp32 partial of Gq and four loss partials, summed afterwards in a fixed order.
 //
-// 192 threads: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue.  Two operand stages,
-// two O accumulators, two G buffers.  Every wait is bounded (DQ_ERR_TIMEOUT on expiry).
+// 320 threads: warp 0 TMA producers (lane 0: R_h^T and the X_t ring, lane 1: the X_t^T ring), warp 1 MMA
+// issuer, warps 2..9 epilogue (two warps per quarter of the tensor-memory lanes, 64 columns each).  Two stages per operand ring (X_t is released as soon as the first product
+// has retired, X_t^T after the second), two O accumulators, two G buffers.  Every wait is bounded
+// (DQ_ERR_TIMEOUT on expiry).
 #pragma once
 #include "tc_gemm.cuh"
 
@@ -28,19 +30,21 @@ constexpr int G_BYTES = 2 * KB_BYTES;              // G_t^T: rows = output chann
 constexpr int STAGES = 2;
 constexpr int SMEM_TOTAL = RT_BYTES + STAGES * STAGE_BYTES + 2 * G_BYTES + 1024 + 1024;
 constexpr uint32_t TMEM_COLS = 512;                // O (2 x 128 columns) + Gq (128 columns)
+constexpr int HEADS_THREADS = 320;
+constexpr int EPI_WARPS = 8;
 
 struct Params {
   int batch, tiles_per_head, splits;   // units = batch * splits; unit u = head u / splits, slice u % splits
   int64_t n_tokens;
   float* part;                         // [units][128][128] partial Gq (row = input channel)
-  float* partials;                     // [units][4] loss partials
+  float* partials;                     // [units][8] loss partials
   __nv_bfloat16* Gt;                   // nullable: also store dL/dO, [batch][128][n_tokens] channel-major
   int* d_status;
 };
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(HEADS_THREADS, 1)
 heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_constant__ CUtensorMap mapX,
                   const __grid_constant__ CUtensorMap mapXt, const Params p) {
   constexpr uint32_t IDESC = make_idesc_bf16(128);
@@ -50,27 +54,30 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
   const uint32_t stage_base = rt_smem + RT_BYTES;
   const uint32_t g_base = stage_base + STAGES * STAGE_BYTES;
   const uint32_t bar_base = g_base + 2 * G_BYTES;
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (2 + s); };
+  auto xa_full = [&](int s) { return bar_base + 8u * s; };
+  auto xa_empty = [&](int s) { return bar_base + 8u * (2 + s); };
+  auto xt_full = [&](int s) { return bar_base + 8u * (17 + s); };
+  auto xt_empty = [&](int s) { return bar_base + 8u * (19 + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (4 + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (6 + a); };
   auto gfull_bar = [&](int g) { return bar_base + 8u * (8 + g); };
   auto gempty_bar = [&](int g) { return bar_base + 8u * (10 + g); };
   const uint32_t rtfull_bar = bar_base + 8u * 12, rtempty_bar = bar_base + 8u * 13;
   const uint32_t qfull_bar = bar_base + 8u * 14, qempty_bar = bar_base + 8u * 15;
-  const uint32_t tmem_slot = bar_base + 8u * 16;
+  const uint32_t tmem_slot = bar_base + 8u * 16;   // barriers 17..20: the X_t^T ring
   uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
   uint8_t* g_ptr = smem_raw + (g_base - smem_u32(smem_raw));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
-      mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1);
-      mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), 4);
-      mbar_init(gfull_bar(s), 4); mbar_init(gempty_bar(s), 1);
+      mbar_init(xa_full(s), 1); mbar_init(xa_empty(s), 1);
+      mbar_init(xt_full(s), 1); mbar_init(xt_empty(s), 1);
+      mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EPI_WARPS);
+      mbar_init(gfull_bar(s), EPI_WARPS); mbar_init(gempty_bar(s), 1);
     }
     mbar_init(rtfull_bar, 1); mbar_init(rtempty_bar, 1);
-    mbar_init(qfull_bar, 1); mbar_init(qempty_bar, 4);
+    mbar_init(qfull_bar, 1); mbar_init(qempty_bar, EPI_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tensormap(&mapRt); prefetch_tensormap(&mapX); prefetch_tensormap(&mapXt);
   }
@@ -90,8 +97,8 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
   };
 
   if (warp == 0) {
-    // ------------------------------------------------------------- TMA producer
-    if (lane == 0) {
+    // ------------------------------------------------------------- TMA producers
+    if (lane == 0) {          // R_h^T per unit and the X_t ring
       int stage = 0;
       uint32_t phase = 0, rt_phase = 0;
       bool ok = true;
@@ -104,13 +111,27 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         tma_load_3d(rt_smem, &mapRt, rtfull_bar, 0, 0, b);
         tma_load_3d(rt_smem + KB_BYTES, &mapRt, rtfull_bar, BLOCK_K, 0, b);
         for (int t = t0; t < t1; ++t) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
-          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
-          const uint32_t xa = stage_base + stage * STAGE_BYTES, xt = xa + XA_BYTES;
-          tma_load_3d(xa, &mapX, full_bar(stage), 0, t * 128, b);
-          tma_load_3d(xa + KB_BYTES, &mapX, full_bar(stage), BLOCK_K, t * 128, b);
-          tma_load_3d(xt, &mapXt, full_bar(stage), t * 128, 0, b);
-          tma_load_3d(xt + KB_BYTES, &mapXt, full_bar(stage), t * 128 + BLOCK_K, 0, b);
+          if (!mbar_wait(xa_empty(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
+          mbar_expect_tx(xa_full(stage), XA_BYTES);
+          const uint32_t xa = stage_base + stage * STAGE_BYTES;
+          tma_load_3d(xa, &mapX, xa_full(stage), 0, t * 128, b);
+          tma_load_3d(xa + KB_BYTES, &mapX, xa_full(stage), BLOCK_K, t * 128, b);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    } else if (lane == 1) {   // the X_t^T ring
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        int b, t0, t1;
+        unit_range(u, b, t0, t1);
+        for (int t = t0; t < t1; ++t) {
+          if (!mbar_wait(xt_empty(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
+          mbar_expect_tx(xt_full(stage), XT_BYTES);
+          const uint32_t xt = stage_base + stage * STAGE_BYTES + XA_BYTES;
+          tma_load_3d(xt, &mapXt, xt_full(stage), t * 128, 0, b);
+          tma_load_3d(xt + KB_BYTES, &mapXt, xt_full(stage), t * 128 + BLOCK_K, 0, b);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -119,7 +140,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
     // ------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       int st1 = 0, st2 = 0, acc = 0, g = 0;
-      uint32_t ph1 = 0, acc_phase = 0, g_phase = 0, rt_phase = 0, q_phase = 0;
+      uint32_t ph1 = 0, ph2 = 0, acc_phase = 0, g_phase = 0, rt_phase = 0, q_phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
         int b, t0, t1;
@@ -130,7 +151,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         tc_fence_after();
         for (int i = 0; i <= nt && ok; ++i) {
           if (i < nt) {   // O^T of tile i
-            if (!mbar_wait(full_bar(st1), ph1, p.d_status)) { ok = false; break; }
+            if (!mbar_wait(xa_full(st1), ph1, p.d_status)) { ok = false; break; }
             if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t xa = stage_base + st1 * STAGE_BYTES;
@@ -142,6 +163,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
                 umma_bf16(tmem_o, make_kmajor_sw128_desc(rt_smem + kb * KB_BYTES + k * UMMA_K * 2),
                           make_kmajor_sw128_desc(xa + kb * KB_BYTES + k * UMMA_K * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
             umma_commit(tfull_bar(acc));
+            umma_commit(xa_empty(st1));                  // X_t can be replaced once this product has retired
             if (i == nt - 1) umma_commit(rtempty_bar);   // R_h^T may be replaced once these products retire
             if (++st1 == STAGES) { st1 = 0; ph1 ^= 1u; }
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -152,6 +174,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
               if (!mbar_wait(qempty_bar, q_phase ^ 1u, p.d_status)) { ok = false; break; }
               q_phase ^= 1u;
             }
+            if (!mbar_wait(xt_full(st2), ph2, p.d_status)) { ok = false; break; }
             if (!mbar_wait(gfull_bar(g), g_phase, p.d_status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t xt = stage_base + st2 * STAGE_BYTES + XA_BYTES;
@@ -163,18 +186,19 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
                 umma_bf16(tmem_q, make_kmajor_sw128_desc(xt + kb * KB_BYTES + k * UMMA_K * 2),
                           make_kmajor_sw128_desc(gb + kb * KB_BYTES + k * UMMA_K * 2), IDESC,
                           (j > 0 || kb > 0 || k > 0) ? 1u : 0u);
-            umma_commit(empty_bar(st2));    // both operand tiles of the stage are consumed
+            umma_commit(xt_empty(st2));
             umma_commit(gempty_bar(g));
             if (j == nt - 1) umma_commit(qfull_bar);
-            if (++st2 == STAGES) st2 = 0;
+            if (++st2 == STAGES) { st2 = 0; ph2 ^= 1u; }
             if (++g == 2) { g = 0; g_phase ^= 1u; }
           }
         }
       }
     }
   } else {
-    // ------------------------------------------------------------- epilogue (warps 2..5)
-    const int q = warp & 3;
+    // ------------------------------------------------------------- epilogue (warps 2..9)
+    const int q = warp & 3;                    // quarter of the tensor-memory lanes this warp may read
+    const int half = (warp - 2) >> 2;          // which 64 of the 128 columns
     const int row = q * 32 + lane;             // output channel (O^T, G^T) / input channel (Gq)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     int acc = 0, g = 0;
@@ -190,7 +214,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         tc_fence_after();
         uint8_t* gbuf = g_ptr + g * G_BYTES;
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 2 * half; c < 2 * half + 2; ++c) {
           uint32_t v[32];
           tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * 128 + c * 32), v);
           tmem_ld_wait();
@@ -235,7 +259,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
       tc_fence_after();
       float* dst_row = p.part + ((int64_t)u * 128 + row) * 128;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 2 * half; c < 2 * half + 2; ++c) {
         uint32_t v[32];
         tmem_ld32(tmem_q + lane_addr + (uint32_t)(c * 32), v);
         tmem_ld_wait();
@@ -250,7 +274,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
       if (lane == 0) mbar_arrive(qempty_bar);
 #pragma unroll
       for (int off = 16; off >= 1; off >>= 1) esum += __shfl_xor_sync(0xffffffffu, esum, off);
-      if (lane == 0) p.partials[(int64_t)u * 4 + q] = esum;
+      if (lane == 0) p.partials[(int64_t)u * EPI_WARPS + (warp - 2)] = esum;
     }
   }
 

@@ -116,7 +116,6 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   if (d == 128) {   // per-head rotations: fused kernel, units = (head, range of 128-token tiles)
     const int tiles_per_head = (int)(N / 128);
     int sp = ctx.sm_count / batch;
-    if (sp > (int)(N / 256)) sp = (int)(N / 256);   // the loss-partial buffer holds N / 256 x 4 values per head
     if (sp > tiles_per_head) sp = tiles_per_head;
     if (sp < 1) sp = 1;
     tc.splits = sp;
@@ -128,6 +127,7 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
     tc.fused = true;
   }
   tc.n_partials = (d / tc::BLOCK_M) * (int)(N / 256) * 4;
+  if (tc.fused && tc.n_partials < tc.splits * heads::EPI_WARPS) tc.n_partials = tc.splits * heads::EPI_WARPS;
   *n_partials = tc.n_partials;
   tc.ready = true;
   return DQ_OK;
@@ -161,8 +161,8 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
     hp.Gt = tc.keep_g ? tc.Gt : nullptr; hp.d_status = ctx.d_status;
     const int units = tc.batch * tc.splits;
     const int grid = units < ctx.sm_count ? units : ctx.sm_count;
-    heads::heads_whip_kernel<<<grid, tc::NUM_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x128, mm->xt, hp);
-    tc.n_partials_live = tc.splits * 4;
+    heads::heads_whip_kernel<<<grid, heads::HEADS_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x128, mm->xt, hp);
+    tc.n_partials_live = tc.splits * heads::EPI_WARPS;
     tc.fused_valid = true;
     ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;   // the second product runs here too
     return after_launch(ctx);
