@@ -152,18 +152,21 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
  *     form) only when no factors of a nearby latent are known (first step, after
  *     dq_calib_set_latent or a change of method).  Afterwards, with the previous step's U_old,
  *     Zh = Z U_old^-1 is close to orthogonal whatever Z is, its upper factor I + T is the fixed point
- *     of T <- striu(E - T^T T) + diag(E - T^T T) / 2 with E = Zh^T Zh - I, reached from T = 0 in
- *     n_iters sweeps of triangular tensor-core GEMMs (no dependent column steps), and
- *     U = (I + T) U_old.  If one optimiser step moved the latent so far that the last sweep still
- *     changed an entry by more than 1e-5, the status word becomes DQ_ERR_NOT_CONVERGED and, as after
- *     every device-side error, the update kernels leave the latent and the optimiser state untouched
- *     from then on: the latent stays at the last good iterate.  Recover with
- *     dq_calib_set_qr_method(h, DQ_QR_HOUSEHOLDER, 0) (or more sweeps, or a lower learning rate) and
- *     step again.  n_iters <= 0 selects the default (5).
+ *     of T <- striu(E - T^T T) + diag(E - T^T T) / 2 with E = Zh^T Zh - I, reached from T = 0 by
+ *     sweeps of triangular tensor-core GEMMs (no dependent column steps), and U = (I + T) U_old.
+ *     The sweeps stop by themselves: up to n_iters sweeps with a plain bf16 product, each skipped (by
+ *     a device-side flag, so the launch sequence and a captured graph stay fixed) once the sweep
+ *     before it moved no entry by more than 1e-5, then up to three sweeps with the split-bf16
+ *     product.  If the last of those still moved an entry, one optimiser step has moved the latent
+ *     too far: the status word becomes DQ_ERR_NOT_CONVERGED and, as after every device-side error,
+ *     the update kernels leave the latent and the optimiser state untouched from then on: the
+ *     latent stays at the last good iterate.  Recover with
+ *     dq_calib_set_qr_method(h, DQ_QR_HOUSEHOLDER, 0) (or a lower learning rate) and step again.
+ *     n_iters <= 0 selects the default (12); at most 64.
  *   DQ_QR_HOUSEHOLDER: blocked Householder QR at every step; no assumption on the step size.
  * The call clears the status word.  For d == 128 (any path) the same two methods exist as kernels that
  * keep a whole latent in shared memory; there the sweeps stop as soon as no entry moves (one more is
- * taken) and n_iters only bounds them (8 n_iters).  Otherwise ignored (DQ_OK) on the fp32 path. */
+ * taken) and n_iters only bounds them (4 n_iters).  Otherwise ignored (DQ_OK) on the fp32 path. */
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 

@@ -36,7 +36,7 @@ struct dq_calib {
   TcState tc;                   // tensor-core contractions (operand copies, tensor maps)
   QrTcState qtc;                // tensor-core QR-Orth operand copies
   bool fast_qr = false;
-  int qr_method = DQ_QR_ITERATIVE, qr_iters = 5;
+  int qr_method = DQ_QR_ITERATIVE, qr_iters = 12;
   int optimizer = DQ_SGD;
   float beta1 = 0.f, beta2 = 0.f, eps = 0.f;
   float* opt_m = nullptr;       // first moment / velocity
@@ -518,7 +518,7 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
 
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters) {
   if (!h || (method != DQ_QR_HOUSEHOLDER && method != DQ_QR_ITERATIVE) || n_iters > 64) return DQ_ERR_INVALID_ARG;
-  const int iters = n_iters <= 0 ? 5 : n_iters;
+  const int iters = n_iters <= 0 ? 12 : n_iters;
   if (method == h->qr_method && iters == h->qr_iters) return DQ_OK;
   DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
   DQ_CHECK(clear_status(h));

@@ -5,7 +5,7 @@
 //   qr128_forward_inc_kernel    incremental factorisation from the previous step's factors
 //                               (U_old, W_old = U_old^-1): Zh = Z W_old, E = Zh^T Zh - I,
 //                               T <- Phi(E - T^T T) (Phi(S) = striu(S) + diag(S) / 2) from T = 0 until no
-//                               entry moves (at most 8 x the configured sweep count),
+//                               entry moves (at most 4 x the configured sweep count),
 //                               U = (I + T) U_old, W = U^-1, R = Z W.  Same unique factors as the
 //                               Householder kernel; no dependent column steps.
 //   qr128_backward_sgd_tc_kernel B = R^T Gq, S = tril(B - B^T, -1), Gz = (R S) W^T, Z <- Z - lr Gz.
@@ -261,7 +261,7 @@ dq_status qr128_forward_incremental(Ctx& ctx, const float* Z, float* R, float* U
     DQ_CHECK_CUDA(cudaFuncSetAttribute(qr128_forward_inc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM));
     attr = true;
   }
-  qr128_forward_inc_kernel<<<batch, NT, FWD_SMEM, ctx.stream>>>(Z, R, U, W, Rt_bf16, 8 * (n_sweeps < 1 ? 1 : n_sweeps), 1e-5f,
+  qr128_forward_inc_kernel<<<batch, NT, FWD_SMEM, ctx.stream>>>(Z, R, U, W, Rt_bf16, 4 * (n_sweeps < 1 ? 1 : n_sweeps), 1e-5f,
                                                                 ctx.d_status);
   return after_launch(ctx);
 }

@@ -78,16 +78,21 @@ __global__ void __launch_bounds__(256) skew_t_split_kernel(const float* __restri
 // One sweep of the fixed-point iteration for the Cholesky factor U = I + T of G = Z^T Z:
 //   T <- striu(G - I - P) + diag(G - I - P) / 2,   P = T^T T (nullptr on the first sweep: T = 0).
 // G and P are only valid on and above the diagonal.  Writes T (fp32, row-major, zeros below the
-// diagonal), the split-bf16 copy of T^T (operand of the next P = T^T T) and, on the last sweep,
-// U = I + T with its split copy.  check: flag DQ_ERR_NOT_CONVERGED if an entry still moved by
-// more than tol (the iteration contracts, so the remaining error is below the last update).
+// diagonal), the split-bf16 copy of T^T (operand of the next P = T^T T) and, if U is given,
+// U = I + T with its split copy.
+// run_if (nullable): the sweep is skipped when *run_if == 0 (the previous sweep moved nothing).
+// moved_out (nullable): set to 1 if an entry moved by more than tol (0 otherwise: the caller clears it).
+// fail_if_moved: that case also sets DQ_ERR_NOT_CONVERGED (last sweep the schedule allows).
 // lower_done: tiles strictly below the diagonal already hold their zeros.
 __global__ void __launch_bounds__(256) chol_fixpoint_kernel(const float* __restrict__ G, const float* __restrict__ P,
                                                             float* __restrict__ T, bf16* __restrict__ tt_hi,
                                                             bf16* __restrict__ tt_lo, float* __restrict__ U,
                                                             bf16* __restrict__ u_hi, bf16* __restrict__ u_lo, int d,
-                                                            int check, int lower_done, float tol, int* d_status) {
+                                                            const int* __restrict__ run_if, int* __restrict__ moved_out,
+                                                            int fail_if_moved, int lower_done, float tol,
+                                                            int* d_status) {
   __shared__ float t[32][33];
+  if (run_if && *run_if == 0) return;
   const int64_t off = (int64_t)blockIdx.z * d * d;
   G += off; T += off; tt_hi += off; tt_lo += off;
   if (P) P += off;
@@ -104,7 +109,7 @@ __global__ void __launch_bounds__(256) chol_fixpoint_kernel(const float* __restr
     if (upper && j >= i) {
       v = G[idx] - ((i == j) ? 1.f : 0.f) - (P ? P[idx] : 0.f);
       if (i == j) v *= 0.5f;
-      if (check && !(fabsf(v - T[idx]) <= tol)) moved = true;
+      if (P && !(fabsf(v - T[idx]) <= tol)) moved = true;
     }
     T[idx] = v;
     t[r][tx] = v;
@@ -114,7 +119,10 @@ __global__ void __launch_bounds__(256) chol_fixpoint_kernel(const float* __restr
       split2(u, u_hi[idx], u_lo[idx]);
     }
   }
-  if (moved) set_status(d_status, DQ_ERR_NOT_CONVERGED);
+  if (moved) {
+    if (moved_out) *moved_out = 1;
+    if (fail_if_moved) set_status(d_status, DQ_ERR_NOT_CONVERGED);
+  }
   __syncthreads();
   for (int c = ty; c < 32; c += 8) {    // T^T[j][i] = T[i][j]
     const int64_t idx = (int64_t)(j0 + c) * d + i0 + tx;
@@ -289,6 +297,7 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   }
   if (q.part_bs > 0) DQ_CHECK(alloc(&q.part, q.part_bs * batch));
   DQ_CHECK(alloc(&q.tw_hi, dd)); DQ_CHECK(alloc(&q.tw_lo, dd));
+  DQ_CHECK(alloc(&q.sweep_flags, 80));
   DQ_CHECK(alloc(&q.uot_hi, dd)); DQ_CHECK(alloc(&q.uot_lo, dd));
   for (int unit = 128; unit <= 256; unit *= 2) {   // tile orders: most expensive tiles first, dealt round-robin to the persistent CTAs
     if (d % unit != 0) break;
@@ -323,7 +332,7 @@ void qr_tc_destroy(QrTcState& q) {
   for (bf16* p : all) cudaFree(p);
   cudaFree(q.y_hi); cudaFree(q.y_lo); cudaFree(q.w2_hi); cudaFree(q.w2_lo); cudaFree(q.part); cudaFree(q.T);
   cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.uot_hi); cudaFree(q.uot_lo); cudaFree(q.tl_upper); cudaFree(q.tl_desc_nb); cudaFree(q.tl_asc_nb);
-  cudaFree(q.tl2_upper); cudaFree(q.tl2_desc_nb); cudaFree(q.tl2_asc_nb);
+  cudaFree(q.tl2_upper); cudaFree(q.tl2_desc_nb); cudaFree(q.tl2_asc_nb); cudaFree(q.sweep_flags);
   q = QrTcState();
 }
 
@@ -382,20 +391,34 @@ dq_status qr_upper_factor_incremental(Ctx& ctx, QrWorkspace& ws, QrTcState& q, c
     Out o; o.f32 = G; o.ld = d; o.bs = dd; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
     DQ_CHECK(gemm3(ctx, a, a, d, d, d, batch, o));
   }
-  for (int it = 0; it < n_sweeps; ++it) {
-    const bool last = it == n_sweeps - 1;
-    if (it > 0) {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
+  // Sweep 0 sets T = Phi(E).  Then up to n_sweeps cheap sweeps (plain bf16 product: its relative error 2^-9
+  // acts on a term of size ||T||^2 and later sweeps forgive it by a factor ||T|| each), each skipped once
+  // the sweep before it moved no entry by more than the tolerance, and finally up to three accurate sweeps
+  // (split-bf16 product), the first always taken, the others only while entries still move.  flags[k] = 1
+  // if sweep k moved something; the launch sequence is fixed, so a captured graph replays it unchanged.
+  constexpr int ACCURATE = 3;
+  int* flags = q.sweep_flags;
+  DQ_CHECK_CUDA(cudaMemsetAsync(flags, 0, sizeof(int) * (n_sweeps + ACCURATE + 2), ctx.stream));
+  chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, nullptr, T, q.tw_hi, q.tw_lo, nullptr, nullptr, nullptr, d,
+                                                      nullptr, nullptr, 0, 0, 1e-5f, ctx.d_status);
+  DQ_CHECK(after_launch(ctx));
+  for (int it = 1; it <= n_sweeps + ACCURATE; ++it) {
+    const bool accurate = it > n_sweeps;
+    const bool first_accurate = it == n_sweeps + 1;
+    const bool last = it == n_sweeps + ACCURATE;
+    // cheap sweep 1 always runs; a later cheap sweep runs if the one before moved; the first accurate sweep
+    // always runs; a later accurate sweep runs if the accurate sweep before it moved
+    const int* run_if = (it == 1 || first_accurate) ? nullptr : flags + it - 1;
+    {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
       Op tt{q.tw_hi, q.tw_lo, d, dd};
       Out o; o.f32 = P; o.ld = d; o.bs = dd; o.k_mode = 2; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
-      // Only the last sweep's product enters the returned factor at full weight: the fixed point
-      // T* = Phi(E - T*^T T*) forgives an error e in an earlier product by a factor ||T|| per later sweep,
-      // so the earlier sweeps use plain bf16 operands (relative error 2^-9 on a term of size ||T||^2).
-      if (!last) o.nterms = 1;
+      o.nterms = accurate ? 3 : 1;
+      o.run_if = run_if;
       DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
     }
-    chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, it > 0 ? P : nullptr, T, q.tw_hi, q.tw_lo,
-                                                        last ? scratch : nullptr, uh_hi, uh_lo, d,
-                                                        (last && it > 0) ? 1 : 0, it > 0 ? 1 : 0, 1e-5f, ctx.d_status);
+    chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, P, T, q.tw_hi, q.tw_lo, accurate ? scratch : nullptr, uh_hi,
+                                                        uh_lo, d, run_if, flags + it, last ? 1 : 0, 1, 1e-5f,
+                                                        ctx.d_status);
     DQ_CHECK(after_launch(ctx));
   }
   {   // U[i][j] = sum_k Uh[i][k] U_old[k][j]: both upper triangular, k in [128 mb, 128 (nb + 1))

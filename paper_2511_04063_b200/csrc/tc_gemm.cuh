@@ -49,6 +49,9 @@ struct Params {
   // most expensive tiles first so that the round-robin deal over the persistent CTAs is balanced.
   const int* tile_list;
   int n_list;
+  // Optional device flag: the kernel does nothing when *run_if == 0 (lets a fixed launch sequence, e.g. a
+  // captured graph, stop a data-dependent iteration early).  nullptr: always run.
+  const int* run_if;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -179,6 +182,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapB_lo,
                const Params p) {
+  if (p.run_if && *p.run_if == 0) return;                     // uniform over the grid: nothing is allocated yet
   using L = SmemLayout<BLOCK_N, NTERMS>;
   constexpr int STAGES = L::STAGES;
   constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;                 // 256 or 512: power of two

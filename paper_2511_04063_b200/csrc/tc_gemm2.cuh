@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapB_lo,
                 const Params p) {
+  if (p.run_if && *p.run_if == 0) return;           // uniform over the grid (both CTAs of every pair)
   using L = PairSmem<NTERMS>;
   constexpr int STAGES = L::STAGES;
   constexpr int STAGE_BYTES = L::STAGE_BYTES;

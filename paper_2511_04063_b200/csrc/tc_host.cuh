@@ -142,6 +142,7 @@ struct Out {
   const int* tile_list = nullptr; int n_list = 0;   // explicit tile order (device), see tc::Params
   const int* tile_list2 = nullptr; int n_list2 = 0; // the same order in 256 x 256 tiles (two-CTA kernel)
   int nterms = 3;   // 1: plain bf16 product of the hi parts only (2^-9 relative), a third of the MMAs
+  const int* run_if = nullptr;   // device flag: skip the product when it is 0 (see tc::Params)
 };
 
 // 64-wide k-blocks the kernels run for a product: the same clipping as their k_range, over all tiles or
@@ -184,11 +185,12 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
     p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
     p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
     p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
-    p.tile_list = o.tile_list2; p.n_list = o.n_list2;
+    p.tile_list = o.tile_list2; p.n_list = o.n_list2; p.run_if = o.run_if;
     {
       const bool upper = o.tri_skip || (o.tile_list2 && o.n_list2 < p.m_blocks * p.n_blocks);
-      ctx.mma_flops += (double)count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode, upper, 256) *
-                       (2.0 * 256 * 256 * tc::BLOCK_K) * (o.nterms == 1 ? 1 : 3) * batch;
+      if (!o.run_if)   // products that a device flag may skip are left out of the count
+        ctx.mma_flops += (double)count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode, upper, 256) *
+                         (2.0 * 256 * 256 * tc::BLOCK_K) * (o.nterms == 1 ? 1 : 3) * batch;
     }
     return o.nterms == 1 ? launch_gemm2<1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
                          : launch_gemm2<3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
@@ -204,11 +206,12 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
   p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
   if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
   p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
-  p.tile_list = o.tile_list; p.n_list = o.n_list;
+  p.tile_list = o.tile_list; p.n_list = o.n_list; p.run_if = o.run_if;
   {
     const bool upper = o.tri_skip || (o.tile_list && o.n_list < p.m_blocks * p.n_blocks);
-    ctx.mma_flops += (double)count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode, upper, 128) *
-                     (2.0 * 128 * 128 * tc::BLOCK_K) * (o.nterms == 1 ? 1 : 3) * batch;
+    if (!o.run_if)
+      ctx.mma_flops += (double)count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode, upper, 128) *
+                       (2.0 * 128 * 128 * tc::BLOCK_K) * (o.nterms == 1 ? 1 : 3) * batch;
   }
   return o.nterms == 1 ? launch_gemm<128, 1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
                        : launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);

@@ -73,6 +73,7 @@ struct QrTcState {
   __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T^T of the sweeps
   __nv_bfloat16 *uot_hi = nullptr, *uot_lo = nullptr;   // U^T of the previous step
   bool t_warm = false;                                  // wt_* / uot_* hold the factors of the previous step's latent
+  int* sweep_flags = nullptr;                           // [80] device flags: sweep k moved an entry
   // tile orders for triangular products (device arrays of mb | nb << 16)
   int* tl_upper = nullptr; int n_upper = 0;             // tiles mb <= nb, largest mb first
   int* tl_desc_nb = nullptr;                            // all tiles, largest nb first
