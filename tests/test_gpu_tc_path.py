@@ -269,3 +269,23 @@ def test_fused_per_head_kernel_with_and_without_stored_gradient(batch, n):
         assert abs(loss0[b] - ref["loss"]) <= LOSS_TOL_BF16 * ref["loss"]
         assert np.linalg.norm(Gq0[b] - ref["Gq"]) <= 5e-2 * np.linalg.norm(ref["Gq"])
     c.close()
+
+
+def test_incremental_qr_takes_as_many_sweeps_as_a_large_step_needs():
+    """Adam moves every entry of the latent by about lr per step: a sign-like update of spectral norm
+    ~ 2 lr sqrt(d), far larger than an SGD step.  The sweep schedule (device flags) must carry the
+    incremental factorisation through it without a host round trip, replayed from a graph."""
+    w = small("c2_7b", d=512, n_tokens=1024, n_outlier_channels=3)
+    c = Calib(w)
+    dq.dq_calib_set_optimizer(c.h, dq.DQ_ADAM, 5e-3, 0.9, 0.999, 1e-8)
+    c.step(6)
+    assert c.status() == dq.DQ_OK
+    Z = c.latent()[0].astype(np.float64)
+    assert np.abs(Z - c.Z0_host[0]).max() > 1e-2                    # the latent really moved that far
+    R = c.rotation()[0]
+    assert c.status() == dq.DQ_OK
+    Rr, _ = orc.qr_pos_lapack(Z)
+    cond = np.linalg.cond(Z)
+    assert np.abs(R - Rr).max() <= 5e-5 * max(1.0, cond)
+    assert np.abs(R.T @ R - np.eye(w.d)).max() <= 1e-4
+    c.close()
