@@ -99,13 +99,11 @@ dq_status qr_backward(Ctx& ctx, QrWorkspace& ws, const float* R, const float* U,
                       float* Gz, int d, int batch);
 
 // Batched 128 x 128 QR-Orth resident in shared memory (qr128.cu), one CTA per problem.
-// Forward: R, U (diag > 0), W = U^-1, optional bf16(R^T).  Backward: Gz and the SGD update of Z.
+// Forward (Householder): R, U (diag > 0), W = U^-1, optional bf16(R^T).
 dq_status qr128_forward(Ctx& ctx, const float* Z, float* R, float* U, float* W, __nv_bfloat16* Rt_bf16, int batch);
-dq_status qr128_backward_sgd(Ctx& ctx, const float* R, const float* W, const float* Gq, float* Gz, float* Z, float lr,
-                             int batch);
 
-// Tensor-core variants (qr128_inc.cu): incremental forward from the previous step's U and W (both updated
-// in place) and the backward with warp-level MMAs.
+// Tensor-core kernels (qr128_inc.cu): incremental forward from the previous step's U and W (both updated
+// in place); backward Gz = R tril(R^T Gq - Gq^T R, -1) W^T with the SGD update of Z fused (lr = 0: none).
 dq_status qr128_forward_incremental(Ctx& ctx, const float* Z, float* R, float* U, float* W, __nv_bfloat16* Rt_bf16,
                                     int n_sweeps, int batch);
 dq_status qr128_backward_sgd_tc(Ctx& ctx, const float* R, const float* W, const float* Gq, float* Gz, float* Z,

@@ -4,9 +4,9 @@
 //   qr128_forward_kernel       Z -> U (Householder, Algorithm 2, in place), gauge diag(U) > 0,
 //                              W = U^-1 (blocked inversion), R = Z W; also bf16(R^T) for the
 //                              tensor-core contraction.
-//   qr128_backward_sgd_kernel  B = R^T Gq, S = tril(B - B^T, -1), Gz = (R S) W^T,
-//                              Z <- Z - lr Gz  (Algorithm 1, update step), all in one launch.
-// fp32 FMA arithmetic throughout; sums run in a fixed order (bit-reproducible).
+// fp32 FMA arithmetic throughout; sums run in a fixed order (bit-reproducible).  Used for the first
+// factorisation of a handle and with DQ_QR_HOUSEHOLDER; the incremental forward and the backward are
+// in qr128_inc.cu.
 #include "common.cuh"
 
 namespace dq {
@@ -219,56 +219,6 @@ qr128_forward_kernel(const float* __restrict__ Z, float* __restrict__ R, float* 
   }
 }
 
-constexpr int BWD_SMEM = 3 * N * LD * 4;
-
-__global__ void __launch_bounds__(NT, 1)
-qr128_backward_sgd_kernel(const float* __restrict__ R, const float* __restrict__ W, const float* __restrict__ Gq,
-                          float* __restrict__ Gz, float* __restrict__ Z, float lr, const int* __restrict__ d_status) {
-  extern __shared__ float sm[];
-  if (d_status && *d_status != 0) lr = 0.f;   // an earlier error freezes the latent
-  float* P0 = sm;                    // R
-  float* P1 = P0 + N * LD;           // Gq, then S, then W
-  float* P2 = P1 + N * LD;           // B, then M = R S
-  const int64_t off = (int64_t)blockIdx.x * N * N;
-  R += off; W += off; Gq += off; Gz += off; Z += off;
-  const int tid = threadIdx.x;
-  const int r0 = (tid >> 4) * 4, cl = tid & 15;
-  for (int e = tid; e < N * N; e += NT) {
-    P0[(e >> 7) * LD + (e & 127)] = R[e];
-    P1[(e >> 7) * LD + (e & 127)] = Gq[e];
-  }
-  __syncthreads();
-  float acc[4][8];
-  mm128<true, false>(P0, P1, acc, r0, cl);                // B = R^T Gq
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) P2[(r0 + i) * LD + cl + 16 * j] = acc[i][j];
-  __syncthreads();
-  for (int e = tid; e < N * N; e += NT) {                 // S = tril(B - B^T, -1)
-    const int i = e >> 7, j = e & 127;
-    P1[i * LD + j] = (i > j) ? P2[i * LD + j] - P2[j * LD + i] : 0.f;
-  }
-  __syncthreads();
-  mm128<false, false>(P0, P1, acc, r0, cl);               // M = R S
-  __syncthreads();
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) P2[(r0 + i) * LD + cl + 16 * j] = acc[i][j];
-  for (int e = tid; e < N * N; e += NT) P1[(e >> 7) * LD + (e & 127)] = W[e];
-  __syncthreads();
-  mm128<false, true>(P2, P1, acc, r0, cl);                // Gz = M W^T
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int e = (r0 + i) * N + cl + 16 * j;
-      Gz[e] = acc[i][j];
-      if (lr != 0.f) Z[e] = fmaf(-lr, acc[i][j], Z[e]);
-    }
-}
-
 }  // namespace
 
 dq_status qr128_forward(Ctx& ctx, const float* Z, float* R, float* U, float* W, __nv_bfloat16* Rt_bf16, int batch) {
@@ -278,17 +228,6 @@ dq_status qr128_forward(Ctx& ctx, const float* Z, float* R, float* U, float* W, 
     attr = true;
   }
   qr128_forward_kernel<<<batch, NT, FWD_SMEM, ctx.stream>>>(Z, R, U, W, Rt_bf16, ctx.d_status);
-  return after_launch(ctx);
-}
-
-dq_status qr128_backward_sgd(Ctx& ctx, const float* R, const float* W, const float* Gq, float* Gz, float* Z, float lr,
-                             int batch) {
-  static bool attr = false;
-  if (!attr) {
-    DQ_CHECK_CUDA(cudaFuncSetAttribute(qr128_backward_sgd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD_SMEM));
-    attr = true;
-  }
-  qr128_backward_sgd_kernel<<<batch, NT, BWD_SMEM, ctx.stream>>>(R, W, Gq, Gz, Z, lr, ctx.d_status);
   return after_launch(ctx);
 }
 

@@ -20,6 +20,7 @@
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "mma_tf32.cuh"
 #include "tc_path.cuh"
 
 namespace cg = cooperative_groups;
@@ -118,21 +119,8 @@ __device__ __forceinline__ void load_v8(float (&vv)[8][2], const float* Vk, int 
 
 constexpr int STG_LD = 40;   // row stride of the staging tiles: fragment loads hit 32 distinct banks
 
-// x = hi + lo with hi, lo representable in tf32 (about 2^-22 relative): three tensor-core products
-// hi*hi + hi*lo + lo*hi recover fp32-like accuracy.
-__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
-  const float r = x - __uint_as_float(hi);
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(r));
-}
-// D += A B for one 16 x 8 x 8 tile (A row-major M x K, B column-major K x N), tf32 inputs, fp32 accumulate.
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-      "{%0, %1, %2, %3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
-}
+using mma::split_tf32;
+using mma::mma_tf32;
 
 // Warp partial of W = V_k^T P over this warp's 64 rows (two 32-row groups, lane = row) on the
 // tensor cores: rows are staged in shared memory, fragments of A = V_k^T (M = reflector, K = row) and
