@@ -6,7 +6,7 @@
 //           Then W = U^-1 by recursive block inversion and R = Z W.  (R is the same orthogonal
 //           factor the reflectors would give; forming it as Z U^-1 costs one GEMM instead of
 //           d / 128 dependent block updates.  Its orthogonality error grows like cond(Z) * 2^-17.)
-// Backward: B = R^T Gq, S = tril(B - B^T, -1), Gz = (R S) W^T.
+// Backward: B = R^T Gq, S = tril(B - B^T, -1), Gz = R (S W^T).
 // All d x d products run as split-bf16 tcgen05 GEMMs (three bf16 MMAs per product, fp32
 // accumulation, ~2^-17 relative error), clipped to the non-zero blocks of triangular operands.
 #include <algorithm>
@@ -50,28 +50,28 @@ __global__ void __launch_bounds__(256) split_kernel(const float* __restrict__ sr
   }
 }
 
-// St(hi, lo)[j][k] = S[k][j] with S = tril(B - B^T, -1):  (k > j) ? B[k][j] - B[j][k] : 0
-__global__ void __launch_bounds__(256) skew_t_split_kernel(const float* __restrict__ B, bf16* __restrict__ hi,
-                                                           bf16* __restrict__ lo, int d) {
+// S(hi, lo) = split of S = tril(B - B^T, -1), row-major:  S[i][j] = (i > j) ? B[i][j] - B[j][i] : 0
+__global__ void __launch_bounds__(256) skew_split_kernel(const float* __restrict__ B, bf16* __restrict__ hi,
+                                                         bf16* __restrict__ lo, int d) {
   __shared__ float t[32][33];
   const int64_t off = (int64_t)blockIdx.z * d * d;
   B += off; hi += off; lo += off;
-  const int j0 = blockIdx.y * 32, k0 = blockIdx.x * 32;
+  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  if (k0 + 31 <= j0) {   // tile entirely on or below the diagonal of St: zeros
+  if (j0 >= i0 + 31) {   // tile entirely on or above the diagonal: zeros
     for (int r = ty; r < 32; r += 8) {
-      const int64_t i = (int64_t)(j0 + r) * d + k0 + tx;
+      const int64_t i = (int64_t)(i0 + r) * d + j0 + tx;
       hi[i] = __float2bfloat16_rn(0.f); lo[i] = __float2bfloat16_rn(0.f);
     }
     return;
   }
-  for (int r = ty; r < 32; r += 8) t[r][tx] = B[(int64_t)(k0 + r) * d + j0 + tx];   // B[k][j]
+  for (int r = ty; r < 32; r += 8) t[r][tx] = B[(int64_t)(j0 + r) * d + i0 + tx];   // B[j][i]
   __syncthreads();
   for (int r = ty; r < 32; r += 8) {
-    const int j = j0 + r, k = k0 + tx;
-    const float v = (k > j) ? t[tx][r] - B[(int64_t)j * d + k] : 0.f;
-    const int64_t i = (int64_t)j * d + k;
-    split2(v, hi[i], lo[i]);
+    const int i = i0 + r, j = j0 + tx;
+    const int64_t idx = (int64_t)i * d + j;
+    const float v = (i > j) ? B[idx] - t[tx][r] : 0.f;
+    split2(v, hi[idx], lo[idx]);
   }
 }
 
@@ -472,20 +472,24 @@ dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* G
   Op rt{q.rt_hi, q.rt_lo, d, dd}, gqt{q.gqt_hi, q.gqt_lo, d, dd};
   Out ob; ob.f32 = ws.B; ob.ld = d; ob.bs = dd;
   DQ_CHECK(gemm3(ctx, rt, gqt, d, d, d, batch, ob));
-  skew_t_split_kernel<<<tiles, 256, 0, ctx.stream>>>(ws.B, q.st_hi, q.st_lo, d);
+  skew_split_kernel<<<tiles, 256, 0, ctx.stream>>>(ws.B, q.st_hi, q.st_lo, d);
   DQ_CHECK(after_launch(ctx));
-  // M[i][j] = sum_k R[i][k] S[k][j]:  A = R, B-operand = S^T; only the split copy is kept
-  Op r{q.r_hi, q.r_lo, d, dd}, st{q.st_hi, q.st_lo, d, dd};
-  Out om; om.hi = q.m_hi; om.lo = q.m_lo; om.ld_h = d; om.bs_h = dd;
-  om.k_mode = 8;  // S is strictly lower triangular: S^T[j][k] = 0 for k < j
-  om.tile_list = q.tl_asc_nb; om.n_list = q.n_all; om.tile_list2 = q.tl2_asc_nb; om.n_list2 = q.n2_all;
-  DQ_CHECK(gemm3(ctx, r, st, d, d, d, batch, om));
-  // Gz[i][j] = sum_k M[i][k] W[j][k]
-  Op m{q.m_hi, q.m_lo, d, dd}, wn{q.wn_hi, q.wn_lo, d, dd};
+  // Gz = R S W^T = R D with D = S W^T lower triangular.  D^T[m][n] = sum_k W[m][k] S[n][k]: W[m][k] = 0 for
+  // k < m and S[n][k] = 0 for k >= n, so only tiles mb <= nb with k in [128 mb, 128 (nb + 1)): a sixth of a
+  // dense product (R S first would cost half of one).  Only the split copy of D^T is kept.
+  Op wn{q.wn_hi, q.wn_lo, d, dd}, sr{q.st_hi, q.st_lo, d, dd};
+  Out od; od.hi = q.m_hi; od.lo = q.m_lo; od.ld_h = d; od.bs_h = dd;
+  od.k_mode = 1 | 4;
+  od.tile_list = q.tl_upper; od.n_list = q.n_upper; od.tile_list2 = q.tl2_upper; od.n_list2 = q.n2_upper;
+  DQ_CHECK(gemm3(ctx, wn, sr, d, d, d, batch, od));
+  // (tiles below the block diagonal of D^T are neither written here nor read by the next product; the entries
+  // below the diagonal inside the diagonal tiles come out as exact zeros)
+  // Gz[i][j] = sum_k R[i][k] D^T[j][k]; D^T[j][k] = 0 for k < j
+  Op r{q.r_hi, q.r_lo, d, dd}, dt{q.m_hi, q.m_lo, d, dd};
   Out og; og.f32 = Gz; og.ld = d; og.bs = dd;
-  og.k_mode = 8;  // W[j][k] = 0 for k < j
+  og.k_mode = 8;
   og.tile_list = q.tl_asc_nb; og.n_list = q.n_all; og.tile_list2 = q.tl2_asc_nb; og.n_list2 = q.n2_all;
-  return gemm3(ctx, m, wn, d, d, d, batch, og);
+  return gemm3(ctx, r, dt, d, d, d, batch, og);
 }
 
 }  // namespace dq
