@@ -166,7 +166,9 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
  *   DQ_QR_HOUSEHOLDER: blocked Householder QR at every step; no assumption on the step size.
  * The call clears the status word.  For d == 128 (any path) the same two methods exist as kernels that
  * keep a whole latent in shared memory; there the sweeps stop as soon as no entry moves (one more is
- * taken) and n_iters only bounds them (4 n_iters).  Otherwise ignored (DQ_OK) on the fp32 path. */
+ * taken) and n_iters only bounds them (4 n_iters).  On the fp32 path with d <= 1024 the incremental
+ * factorisation runs on fp32 FMA products (up to n_iters + 3 sweeps, switched off the same way); larger fp32
+ * latents are always factored with Householder. */
 enum { DQ_QR_HOUSEHOLDER = 0, DQ_QR_ITERATIVE = 1 };
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters);
 

@@ -46,6 +46,8 @@ struct dq_calib {
   int orth_method = DQ_ORTH_QR;
   CayleyState cay;              // DQ_ORTH_CAYLEY: momentum and step size
   bool cay_started = false;     // R and its split copies hold the Cayley iterate
+  bool f32_winv_valid = false;  // fp32 path: ws.Winv is the inverse of the U currently stored
+  int* f32_flags = nullptr;     // fp32 path: sweep flags of the incremental factorisation
   bool small_warm = false;      // d == 128: U and U^-1 hold the factors of the previous step's latent
   bool small128 = false;        // d == 128: shared-memory-resident batched QR-Orth
   bool r_stale = true;
@@ -79,7 +81,7 @@ void free_all(dq_calib* h) {
   objective_destroy(h->obj);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
   cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw);
-  cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->loss_tmp); cudaFree(h->ctx.d_status);
+  cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->loss_tmp); cudaFree(h->f32_flags); cudaFree(h->ctx.d_status);
   cudaFree(h->ws.A); cudaFree(h->ws.V); cudaFree(h->ws.T); cudaFree(h->ws.W); cudaFree(h->ws.W2);
   cudaFree(h->ws.Q); cudaFree(h->ws.Winv); cudaFree(h->ws.B); cudaFree(h->ws.S); cudaFree(h->ws.tmp);
   for (auto& e : h->ev) if (e) cudaEventDestroy(e);
@@ -140,8 +142,13 @@ dq_status ensure_rotation(dq_calib* h) {
   } else if (h->fast_qr) {
     DQ_CHECK(qr_forward_fast(h->ctx, h->ws, h->qtc, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch,
                              h->qr_method == DQ_QR_ITERATIVE ? h->qr_iters : 0));
+  } else if (h->qr_method == DQ_QR_ITERATIVE && h->f32_winv_valid && h->f32_flags && h->cfg.d <= 1024) {
+    // fp32 path: the same incremental factorisation on fp32 FMA products (U and U^-1 of the previous step)
+    DQ_CHECK(qr_forward_incremental_f32(h->ctx, h->ws, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch, h->qr_iters,
+                                        h->f32_flags));
   } else {
     DQ_CHECK(qr_forward(h->ctx, h->ws, h->Z, h->R, h->U, tc_rt_operand(h->tc), h->cfg.d, h->cfg.batch));
+    h->f32_winv_valid = false;
   }
   h->r_stale = false;
   return DQ_OK;
@@ -231,7 +238,10 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
   } else {
     if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch));
-    else DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch));
+    else {
+      DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch, h->f32_winv_valid));
+      h->f32_winv_valid = true;
+    }
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
     if (h->optimizer == DQ_SGD) DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, n_latent));
   }
@@ -337,6 +347,7 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
   A(dev_alloc(&h->ws.T, (int64_t)batch * d * 32));
   A(dev_alloc(&h->ws.W, (int64_t)batch * d * 32)); A(dev_alloc(&h->ws.W2, (int64_t)batch * d * 32));
   A(dev_alloc(&h->loss_last, batch)); A(dev_alloc(&h->loss_tmp, batch));
+  if (cfg->path == DQ_PATH_FP32) A(dev_alloc(&h->f32_flags, 80));
   if (st == DQ_OK) {
     for (auto& e : h->ev)
       if (cudaEventCreate(&e) != cudaSuccess) st = DQ_ERR_CUDA;
@@ -382,8 +393,9 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
   for (int s = 0; s < n_steps; ++s) {
     // The captured step of the iterative QR is the incremental one: replay it only while the
     // previous step's factors belong to the latent one optimiser step back.
-    const bool iterative = h->qr_method == DQ_QR_ITERATIVE && (h->small128 || h->fast_qr);
-    const bool warm = h->small128 ? h->small_warm : h->qtc.t_warm;
+    const bool f32_inc = !h->small128 && !h->fast_qr && h->f32_flags && h->cfg.d <= 1024;
+    const bool iterative = h->qr_method == DQ_QR_ITERATIVE && (h->small128 || h->fast_qr || f32_inc);
+    const bool warm = h->small128 ? h->small_warm : (h->fast_qr ? h->qtc.t_warm : h->f32_winv_valid);
     const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
     const bool use_graph = cayley ? (!h->timing && h->cay_started && h->eager_steps_done >= 1)
                                   : (!h->timing && h->r_stale && h->eager_steps_done >= 1 &&
@@ -476,6 +488,7 @@ dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z) {
   h->r_stale = true;
   h->qtc.t_warm = false;   // the new latent may be far from the one the iterative QR last saw
   h->small_warm = false;
+  h->f32_winv_valid = false;
   h->cay_started = false;  // Cayley SGD restarts from the orthogonal factor of the new latent
   return fence_out(h);
 }
@@ -527,6 +540,7 @@ dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters)
   h->r_stale = true;
   h->qtc.t_warm = false;
   h->small_warm = false;
+  h->f32_winv_valid = false;
   if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
   h->graph_failed = false;
   return DQ_OK;

@@ -55,6 +55,8 @@ struct GemmDesc {
   // Split-K: with ksplit > 1 slice ks of the reduction writes alpha * partial
   // product (beta ignored) to C + (b * ksplit + ks) * sC; the caller reduces.
   int ksplit = 1;
+  // Optional device flag: the kernel does nothing when *run_if == 0.
+  const int* run_if = nullptr;
 };
 dq_status gemm_f32(Ctx& ctx, const GemmDesc& g);
 // out[b][i] = alpha * sum_ks part[(b * ksplit + ks)][i] + beta * out[b][i], fixed order.
@@ -94,9 +96,16 @@ dq_status qr_factor(Ctx& ctx, QrWorkspace& ws, const float* Z, int d, int batch)
 // Z -> R (rotation, diag(U) > 0), U.  Optionally also a bf16 copy of R^T.
 dq_status qr_forward(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float* U,
                      __nv_bfloat16* Rt_bf16 /* nullable */, int d, int batch);
-// Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
+// Rank / finiteness test of diag(U) (qr_forward.cu); works on either orientation.
+dq_status qr_diag_check(Ctx& ctx, const float* A, int d, int batch);
+// Gz = R tril(R^T Gq - Gq^T R, -1) U^-T.  winv_fresh: ws.Winv already holds U^-1.
 dq_status qr_backward(Ctx& ctx, QrWorkspace& ws, const float* R, const float* U, const float* Gq,
-                      float* Gz, int d, int batch);
+                      float* Gz, int d, int batch, bool winv_fresh);
+// Incremental factorisation in fp32 from the previous factors (U holds U_old, ws.Winv its inverse; both are
+// replaced): Zh = Z W_old, E = Zh^T Zh - I, T <- Phi(E - T^T T) until nothing moves (device flags, at most
+// n_sweeps + 3 sweeps), U = (I + T) U_old, W = U^-1, R = Z W.  flags: device int[n_sweeps + 5].
+dq_status qr_forward_incremental_f32(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float* U, int d, int batch,
+                                     int n_sweeps, int* flags);
 
 // Batched 128 x 128 QR-Orth resident in shared memory (qr128.cu), one CTA per problem.
 // Forward (Householder): R, U (diag > 0), W = U^-1, optional bf16(R^T).

@@ -15,6 +15,7 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(GemmDesc g, float* __res
   __shared__ __align__(16) float As[BK][BM + PAD];
   __shared__ __align__(16) float Bs[BK][BN + PAD];
   __shared__ float warp_sums[8];
+  if (g.run_if && *g.run_if == 0) return;
 
   const int b = blockIdx.z / g.ksplit, ks = blockIdx.z % g.ksplit;
   const float* __restrict__ A = g.A + (int64_t)b * g.sA;

@@ -95,10 +95,71 @@ dq_status tri_inverse(Ctx& ctx, QrWorkspace& ws, const float* U, int d, int batc
   return DQ_OK;
 }
 
+// T = Phi(G - I - P), Phi(S) = striu(S) + diag(S) / 2 (P == nullptr: T = Phi(G - I)); see
+// qr_forward_incremental_f32.  One launch covers all problems (blockIdx.y).
+__global__ void __launch_bounds__(256) fixpoint_f32_kernel(const float* __restrict__ G, const float* __restrict__ P,
+                                                           float* __restrict__ T, int d, const int* __restrict__ run_if,
+                                                           int* __restrict__ moved_out, int fail_if_moved, float tol,
+                                                           int* d_status) {
+  if (run_if && *run_if == 0) return;
+  const int64_t dd = (int64_t)d * d, off = (int64_t)blockIdx.y * dd;
+  bool moved = false;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < dd; e += (int64_t)gridDim.x * blockDim.x) {
+    const int i = (int)(e / d), j = (int)(e % d);
+    float v = 0.f;
+    if (j >= i) {
+      v = G[off + e] - ((i == j) ? 1.f : 0.f) - (P ? P[off + e] : 0.f);
+      if (i == j) v *= 0.5f;
+      if (P && !(fabsf(v - T[off + e]) <= tol)) moved = true;
+    }
+    T[off + e] = v;
+  }
+  if (moved) {
+    if (moved_out) *moved_out = 1;
+    if (fail_if_moved) set_status(d_status, DQ_ERR_NOT_CONVERGED);
+  }
+}
+
 }  // namespace
 
+dq_status qr_forward_incremental_f32(Ctx& ctx, QrWorkspace& ws, const float* Z, float* R, float* U, int d, int batch,
+                                     int n_sweeps, int* flags) {
+  const int64_t dd = (int64_t)d * d;
+  float *Zh = ws.A, *G = ws.B, *T = ws.S, *P = ws.tmp, *Qs = ws.Q;
+  GemmDesc g{};
+  g.lda = d; g.ldb = d; g.ldc = d; g.sA = dd; g.sB = dd; g.sC = dd;
+  g.M = d; g.N = d; g.K = d; g.alpha = 1.f; g.beta = 0.f; g.batch = batch;
+  g.A = Z; g.transA = 0; g.B = ws.Winv; g.transB = 0; g.C = Zh;       // Zh = Z W_old
+  DQ_CHECK(gemm_f32(ctx, g));
+  g.A = Zh; g.transA = 1; g.B = Zh; g.transB = 0; g.C = G;            // G = Zh^T Zh
+  DQ_CHECK(gemm_f32(ctx, g));
+  int bx = (int)((dd + 255) / 256);
+  if (bx > 1024) bx = 1024;
+  const dim3 grid(bx, batch);
+  const int total = n_sweeps + 3;
+  DQ_CHECK_CUDA(cudaMemsetAsync(flags, 0, sizeof(int) * (total + 2), ctx.stream));
+  fixpoint_f32_kernel<<<grid, 256, 0, ctx.stream>>>(G, nullptr, T, d, nullptr, nullptr, 0, 1e-5f, ctx.d_status);
+  DQ_CHECK(after_launch(ctx));
+  for (int it = 1; it <= total; ++it) {   // sweep it runs while sweep it - 1 moved an entry (flags[it - 1])
+    const int* run_if = (it == 1) ? nullptr : flags + it - 1;
+    g.A = T; g.transA = 1; g.B = T; g.transB = 0; g.C = P; g.run_if = run_if;   // P = T^T T
+    DQ_CHECK(gemm_f32(ctx, g));
+    fixpoint_f32_kernel<<<grid, 256, 0, ctx.stream>>>(G, P, T, d, run_if, flags + it, it == total ? 1 : 0, 1e-5f,
+                                                      ctx.d_status);
+    DQ_CHECK(after_launch(ctx));
+  }
+  g.run_if = nullptr;
+  g.A = T; g.transA = 0; g.B = U; g.transB = 0; g.C = Qs;             // U = U_old + T U_old
+  DQ_CHECK(gemm_f32(ctx, g));
+  DQ_CHECK(accumulate(ctx, U, Qs, dd * batch));
+  DQ_CHECK(qr_diag_check(ctx, U, d, batch));
+  DQ_CHECK(tri_inverse(ctx, ws, U, d, batch));                        // uses ws.tmp as scratch
+  g.A = Z; g.transA = 0; g.B = ws.Winv; g.transB = 0; g.C = R;        // R = Z W
+  return gemm_f32(ctx, g);
+}
+
 dq_status qr_backward(Ctx& ctx, QrWorkspace& ws, const float* R, const float* U, const float* Gq,
-                      float* Gz, int d, int batch) {
+                      float* Gz, int d, int batch, bool winv_fresh) {
   const int64_t dd = (int64_t)d * d;
   GemmDesc g{};
   g.A = R; g.lda = d; g.transA = 1; g.sA = dd;       // B = R^T Gq
@@ -110,7 +171,7 @@ dq_status qr_backward(Ctx& ctx, QrWorkspace& ws, const float* R, const float* U,
   DQ_CHECK(after_launch(ctx));
   g.A = R; g.transA = 0; g.B = ws.S; g.C = ws.B;     // M = R S
   DQ_CHECK(gemm_f32(ctx, g));
-  DQ_CHECK(tri_inverse(ctx, ws, U, d, batch));
+  if (!winv_fresh) DQ_CHECK(tri_inverse(ctx, ws, U, d, batch));
   g.A = ws.B; g.transA = 0; g.B = ws.Winv; g.transB = 1; g.C = Gz;   // Gz = M U^-T
   return gemm_f32(ctx, g);
 }

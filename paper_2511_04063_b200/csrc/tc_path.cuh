@@ -132,7 +132,5 @@ dq_status qrp_panel(Ctx& ctx, float* At, __nv_bfloat16* at_hi, __nv_bfloat16* at
 dq_status qrp_wy_w2(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, const float* Tk,
                     __nv_bfloat16* w2_hi, __nv_bfloat16* w2_lo, int64_t w2_bs, int n, int batch);
 dq_status qrp_gauge_ut(Ctx& ctx, const float* At, float* U, __nv_bfloat16* hi, __nv_bfloat16* lo, int d, int batch);
-// Rank / finiteness test of diag(U) (qr_forward.cu); works on either orientation.
-dq_status qr_diag_check(Ctx& ctx, const float* A, int d, int batch);
 
 }  // namespace dq
