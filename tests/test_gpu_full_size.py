@@ -25,7 +25,7 @@ def perturbed_latent(w, Z0, seed):
     return (Z0 + np.float32(0.02 / np.sqrt(w.d)) * noise).astype(np.float32)
 
 
-@pytest.mark.parametrize("name,qr", [("c1_tiny", "householder"), ("c2_7b", "householder"), ("c2_7b", "iterative"),
+@pytest.mark.parametrize("name,qr", [("c1_tiny", "householder"), ("c1_tiny", "iterative"), ("c2_7b", "householder"), ("c2_7b", "iterative"),
                                      ("c3_heads", "householder"), ("c3_heads", "iterative"), ("c4_13b", "householder"), ("c4_13b", "iterative"),
                                      ("c5_70b", "householder"), ("c5_70b", "iterative")])
 def test_one_step_at_full_size(name, qr):
