@@ -5,13 +5,16 @@
 //   Gq_h += X_t^T G_t    (second tcgen05 product: G_t goes from the epilogue's registers into shared
 //                         memory as the K-major operand, the accumulator stays in tensor memory
 //                         for all tiles of the unit)
-// so the rotated activations and dL/dO never reach HBM; X is read once in each orientation.
+// so the rotated activations and dL/dO never reach HBM and X is read exactly once: the channel-major
+// operand of the second product (X_t^T) is made on chip, the epilogue warps transpose the token-major
+// tile in shared memory (8 x 8 blocks through registers) while the first product runs.
 // R_h^T stays resident in shared memory for a unit (head, range of token tiles); every unit writes
 // one 128 x 128 fp32 partial of Gq and four loss partials, summed afterwards in a fixed order.
 //
-// 320 threads: warp 0 TMA producers (lane 0: R_h^T and the X_t ring, lane 1: the X_t^T ring), warp 1 MMA
-// issuer, warps 2..9 epilogue (two warps per quarter of the tensor-memory lanes, 64 columns each).  Two stages per operand ring (X_t is released as soon as the first product
-// has retired, X_t^T after the second), two O accumulators, two G buffers.  Every wait is bounded
+// 320 threads: warp 0 TMA producer (R_h^T and the X_t ring), warp 1 MMA issuer, warps 2..9 transpose +
+// epilogue (two warps per quarter of the tensor-memory lanes, 64 columns each).  Two stages per operand
+// ring (X_t is released once the first product has retired and the tile has been transposed, X_t^T after
+// the second product), two O accumulators, two G buffers.  Every wait is bounded
 // (DQ_ERR_TIMEOUT on expiry).
 #pragma once
 #include "tc_gemm.cuh"
@@ -45,8 +48,7 @@ struct Params {
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __global__ void __launch_bounds__(HEADS_THREADS, 1)
-heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_constant__ CUtensorMap mapX,
-                  const __grid_constant__ CUtensorMap mapXt, const Params p) {
+heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_constant__ CUtensorMap mapX, const Params p) {
   constexpr uint32_t IDESC = make_idesc_bf16(128);
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -71,15 +73,15 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
-      mbar_init(xa_full(s), 1); mbar_init(xa_empty(s), 1);
-      mbar_init(xt_full(s), 1); mbar_init(xt_empty(s), 1);
+      mbar_init(xa_full(s), 1); mbar_init(xa_empty(s), 1 + EPI_WARPS);   // first product + the transposing warps
+      mbar_init(xt_full(s), EPI_WARPS); mbar_init(xt_empty(s), 1);
       mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EPI_WARPS);
       mbar_init(gfull_bar(s), EPI_WARPS); mbar_init(gempty_bar(s), 1);
     }
     mbar_init(rtfull_bar, 1); mbar_init(rtempty_bar, 1);
     mbar_init(qfull_bar, 1); mbar_init(qempty_bar, EPI_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    prefetch_tensormap(&mapRt); prefetch_tensormap(&mapX); prefetch_tensormap(&mapXt);
+    prefetch_tensormap(&mapRt); prefetch_tensormap(&mapX);
   }
   if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
   tc_fence_before();
@@ -97,8 +99,8 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
   };
 
   if (warp == 0) {
-    // ------------------------------------------------------------- TMA producers
-    if (lane == 0) {          // R_h^T per unit and the X_t ring
+    // ------------------------------------------------------------- TMA producer: R_h^T per unit, the X_t ring
+    if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0, rt_phase = 0;
       bool ok = true;
@@ -116,22 +118,6 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
           const uint32_t xa = stage_base + stage * STAGE_BYTES;
           tma_load_3d(xa, &mapX, xa_full(stage), 0, t * 128, b);
           tma_load_3d(xa + KB_BYTES, &mapX, xa_full(stage), BLOCK_K, t * 128, b);
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-        }
-      }
-    } else if (lane == 1) {   // the X_t^T ring
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-        int b, t0, t1;
-        unit_range(u, b, t0, t1);
-        for (int t = t0; t < t1; ++t) {
-          if (!mbar_wait(xt_empty(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
-          mbar_expect_tx(xt_full(stage), XT_BYTES);
-          const uint32_t xt = stage_base + stage * STAGE_BYTES + XA_BYTES;
-          tma_load_3d(xt, &mapXt, xt_full(stage), t * 128, 0, b);
-          tma_load_3d(xt + KB_BYTES, &mapXt, xt_full(stage), t * 128 + BLOCK_K, 0, b);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -201,23 +187,57 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
     const int half = (warp - 2) >> 2;          // which 64 of the 128 columns
     const int row = q * 32 + lane;             // output channel (O^T, G^T) / input channel (Gq)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    int acc = 0, g = 0;
-    uint32_t acc_phase = 0, g_phase = 0, q_phase = 0;
+    int acc = 0, g = 0, sx = 0;
+    uint32_t acc_phase = 0, g_phase = 0, q_phase = 0, px = 0;
+    // transpose duty: this thread moves the 8 x 8 block (channels 8 bi.., tokens 8 bt..) of every tile; the
+    // diagonal assignment of blocks to lanes keeps both the 16-byte loads and the 16-byte stores of a
+    // quarter-warp on eight different bank groups of the swizzled tiles
+    const int e = (warp - 2) * 32 + lane;
+    const int bi = (e & 7) + 8 * ((e >> 6) & 1);
+    const int bt = (((e & 7) + ((e >> 3) & 7)) & 7) + 8 * ((e >> 7) & 1);
+    uint8_t* stage_ptr = smem_raw + (stage_base - smem_u32(smem_raw));
     bool ok = true;
     for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
       int b, t0, t1;
       unit_range(u, b, t0, t1);
       float esum = 0.f;
       for (int t = t0; t < t1; ++t) {
+        // ---- X_t^T of this tile (operand of the second product)
+        if (!mbar_wait(xa_full(sx), px, p.d_status)) { ok = false; break; }
+        if (!mbar_wait(xt_empty(sx), px ^ 1u, p.d_status)) { ok = false; break; }
+        {
+          const uint8_t* src = stage_ptr + sx * STAGE_BYTES + (bi >> 3) * KB_BYTES;
+          uint8_t* dst = stage_ptr + sx * STAGE_BYTES + XA_BYTES + (bt >> 3) * KB_BYTES;
+          uint32_t in[8][4];
+#pragma unroll
+          for (int r = 0; r < 8; ++r) {      // token 8 bt + r: chunk (bi & 7) of its row sits at (bi & 7) ^ r
+            const uint4 v = *reinterpret_cast<const uint4*>(src + (8 * (bt & 15) + r) * 128 + (((bi & 7) ^ r) << 4));
+            in[r][0] = v.x; in[r][1] = v.y; in[r][2] = v.z; in[r][3] = v.w;
+          }
+#pragma unroll
+          for (int r = 0; r < 8; ++r) {      // channel 8 bi + r: its eight tokens form chunk (bt & 7) of row 8 bi + r
+            uint32_t o[4];
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+              o[w] = __byte_perm(in[2 * w][r >> 1], in[2 * w + 1][r >> 1], (r & 1) ? 0x7632 : 0x5410);
+            *reinterpret_cast<uint4*>(dst + (8 * bi + r) * 128 + (((bt & 7) ^ r) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(xt_full(sx)); mbar_arrive(xa_empty(sx)); }
+        if (++sx == STAGES) { sx = 0; px ^= 1u; }
+        // ---- Eq. 4 epilogue of O^T
         if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
         if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }
         tc_fence_after();
         uint8_t* gbuf = g_ptr + g * G_BYTES;
-#pragma unroll 1
-        for (int c = 2 * half; c < 2 * half + 2; ++c) {
-          uint32_t v[32];
-          tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * 128 + c * 32), v);
-          tmem_ld_wait();
+        // both 32-column chunks of this warp are requested before the first is used
+        uint32_t va[32], vb[32];
+        tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * 128 + (2 * half) * 32), va);
+        tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * 128 + (2 * half + 1) * 32), vb);
+        tmem_ld_wait();
+        auto process = [&](int c, const uint32_t (&v)[32]) {
           uint32_t packed[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -244,7 +264,9 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             for (int i = 0; i < 4; ++i)
               dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
           }
-        }
+        };
+        process(2 * half, va);
+        process(2 * half + 1, vb);
         tc_fence_before();
         fence_async_smem();                    // the tensor core reads G through the async proxy
         __syncwarp();

@@ -161,7 +161,7 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
     hp.Gt = tc.keep_g ? tc.Gt : nullptr; hp.d_status = ctx.d_status;
     const int units = tc.batch * tc.splits;
     const int grid = units < ctx.sm_count ? units : ctx.sm_count;
-    heads::heads_whip_kernel<<<grid, heads::HEADS_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x128, mm->xt, hp);
+    heads::heads_whip_kernel<<<grid, heads::HEADS_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x128, hp);
     tc.n_partials_live = tc.splits * heads::EPI_WARPS;
     tc.fused_valid = true;
     ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;   // the second product runs here too
