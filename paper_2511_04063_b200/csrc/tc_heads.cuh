@@ -12,9 +12,9 @@
 // one 128 x 128 fp32 partial of Gq and four loss partials, summed afterwards in a fixed order.
 //
 // 320 threads: warp 0 TMA producer (R_h^T and the X_t ring), warp 1 MMA issuer, warps 2..9 transpose +
-// epilogue (two warps per quarter of the tensor-memory lanes, 64 columns each).  Two stages per operand
-// ring (X_t is released once the first product has retired and the tile has been transposed, X_t^T after
-// the second product), two O accumulators, two G buffers.  Every wait is bounded
+// epilogue (two warps per quarter of the tensor-memory lanes, 64 columns each).  X_t is released once the
+// first product has retired and the tile has been transposed, X_t^T and G_t after the second product;
+// two O accumulators.  Every wait is bounded
 // (DQ_ERR_TIMEOUT on expiry).
 #pragma once
 #include "tc_gemm.cuh"
@@ -28,10 +28,11 @@ constexpr int KB_BYTES = 128 * BLOCK_K * 2;        // one [128 rows][64 bf16] K-
 constexpr int RT_BYTES = 2 * KB_BYTES;             // R_h^T: rows = output channel, K = input channel (128)
 constexpr int XA_BYTES = 2 * KB_BYTES;             // X_t:   rows = token, K = input channel
 constexpr int XT_BYTES = 2 * KB_BYTES;             // X_t^T: rows = input channel, K = token
-constexpr int STAGE_BYTES = XA_BYTES + XT_BYTES;
 constexpr int G_BYTES = 2 * KB_BYTES;              // G_t^T: rows = output channel, K = token
-constexpr int STAGES = 2;
-constexpr int SMEM_TOTAL = RT_BYTES + STAGES * STAGE_BYTES + 2 * G_BYTES + 1024 + 1024;
+// Ring depths (measured on the 32-head workload: two of each is fastest; a deeper X_t ring with the two
+// on-chip operands of the second product single-buffered is about 10 % slower).
+constexpr int XA_STAGES = 2, XT_STAGES = 2, G_BUFS = 2;
+constexpr int SMEM_TOTAL = RT_BYTES + XA_STAGES * XA_BYTES + XT_STAGES * XT_BYTES + G_BUFS * G_BYTES + 1024 + 1024;
 constexpr uint32_t TMEM_COLS = 512;                // O (2 x 128 columns) + Gq (128 columns)
 constexpr int HEADS_THREADS = 320;
 constexpr int EPI_WARPS = 8;
@@ -53,31 +54,34 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t rt_smem = smem_base;
-  const uint32_t stage_base = rt_smem + RT_BYTES;
-  const uint32_t g_base = stage_base + STAGES * STAGE_BYTES;
-  const uint32_t bar_base = g_base + 2 * G_BYTES;
-  auto xa_full = [&](int s) { return bar_base + 8u * s; };
-  auto xa_empty = [&](int s) { return bar_base + 8u * (2 + s); };
-  auto xt_full = [&](int s) { return bar_base + 8u * (17 + s); };
-  auto xt_empty = [&](int s) { return bar_base + 8u * (19 + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (4 + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (6 + a); };
-  auto gfull_bar = [&](int g) { return bar_base + 8u * (8 + g); };
-  auto gempty_bar = [&](int g) { return bar_base + 8u * (10 + g); };
-  const uint32_t rtfull_bar = bar_base + 8u * 12, rtempty_bar = bar_base + 8u * 13;
-  const uint32_t qfull_bar = bar_base + 8u * 14, qempty_bar = bar_base + 8u * 15;
-  const uint32_t tmem_slot = bar_base + 8u * 16;   // barriers 17..20: the X_t^T ring
+  const uint32_t xa_base = rt_smem + RT_BYTES;
+  const uint32_t xt_base = xa_base + XA_STAGES * XA_BYTES;
+  const uint32_t g_base = xt_base + XT_STAGES * XT_BYTES;
+  const uint32_t bar_base = g_base + G_BUFS * G_BYTES;
+  constexpr int B_XAF = 0, B_XAE = B_XAF + XA_STAGES, B_XTF = B_XAE + XA_STAGES, B_XTE = B_XTF + XT_STAGES,
+                B_TF = B_XTE + XT_STAGES, B_TE = B_TF + 2, B_GF = B_TE + 2, B_GE = B_GF + G_BUFS, B_MISC = B_GE + G_BUFS;
+  auto xa_full = [&](int s) { return bar_base + 8u * (B_XAF + s); };
+  auto xa_empty = [&](int s) { return bar_base + 8u * (B_XAE + s); };
+  auto xt_full = [&](int s) { return bar_base + 8u * (B_XTF + s); };
+  auto xt_empty = [&](int s) { return bar_base + 8u * (B_XTE + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (B_TF + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (B_TE + a); };
+  auto gfull_bar = [&](int g) { return bar_base + 8u * (B_GF + g); };
+  auto gempty_bar = [&](int g) { return bar_base + 8u * (B_GE + g); };
+  const uint32_t rtfull_bar = bar_base + 8u * B_MISC, rtempty_bar = bar_base + 8u * (B_MISC + 1);
+  const uint32_t qfull_bar = bar_base + 8u * (B_MISC + 2), qempty_bar = bar_base + 8u * (B_MISC + 3);
+  const uint32_t tmem_slot = bar_base + 8u * (B_MISC + 4);
   uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
   uint8_t* g_ptr = smem_raw + (g_base - smem_u32(smem_raw));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < XA_STAGES; ++s) {
       mbar_init(xa_full(s), 1); mbar_init(xa_empty(s), 1 + EPI_WARPS);   // first product + the transposing warps
-      mbar_init(xt_full(s), EPI_WARPS); mbar_init(xt_empty(s), 1);
-      mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EPI_WARPS);
-      mbar_init(gfull_bar(s), EPI_WARPS); mbar_init(gempty_bar(s), 1);
     }
+    for (int s = 0; s < XT_STAGES; ++s) { mbar_init(xt_full(s), EPI_WARPS); mbar_init(xt_empty(s), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EPI_WARPS); }
+    for (int s = 0; s < G_BUFS; ++s) { mbar_init(gfull_bar(s), EPI_WARPS); mbar_init(gempty_bar(s), 1); }
     mbar_init(rtfull_bar, 1); mbar_init(rtempty_bar, 1);
     mbar_init(qfull_bar, 1); mbar_init(qempty_bar, EPI_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -115,10 +119,10 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         for (int t = t0; t < t1; ++t) {
           if (!mbar_wait(xa_empty(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
           mbar_expect_tx(xa_full(stage), XA_BYTES);
-          const uint32_t xa = stage_base + stage * STAGE_BYTES;
+          const uint32_t xa = xa_base + stage * XA_BYTES;
           tma_load_3d(xa, &mapX, xa_full(stage), 0, t * 128, b);
           tma_load_3d(xa + KB_BYTES, &mapX, xa_full(stage), BLOCK_K, t * 128, b);
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          if (++stage == XA_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
@@ -140,7 +144,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             if (!mbar_wait(xa_full(st1), ph1, p.d_status)) { ok = false; break; }
             if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t xa = stage_base + st1 * STAGE_BYTES;
+            const uint32_t xa = xa_base + st1 * XA_BYTES;
             const uint32_t tmem_o = tmem_base + (uint32_t)(acc * 128);
 #pragma unroll
             for (int kb = 0; kb < 2; ++kb)
@@ -151,7 +155,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             umma_commit(tfull_bar(acc));
             umma_commit(xa_empty(st1));                  // X_t can be replaced once this product has retired
             if (i == nt - 1) umma_commit(rtempty_bar);   // R_h^T may be replaced once these products retire
-            if (++st1 == STAGES) { st1 = 0; ph1 ^= 1u; }
+            if (++st1 == XA_STAGES) { st1 = 0; ph1 ^= 1u; }
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
           }
           if (i > 0) {    // Gq += X_t^T G_t of tile i - 1
@@ -163,7 +167,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             if (!mbar_wait(xt_full(st2), ph2, p.d_status)) { ok = false; break; }
             if (!mbar_wait(gfull_bar(g), g_phase, p.d_status)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t xt = stage_base + st2 * STAGE_BYTES + XA_BYTES;
+            const uint32_t xt = xt_base + st2 * XT_BYTES;
             const uint32_t gb = g_base + g * G_BYTES;
 #pragma unroll
             for (int kb = 0; kb < 2; ++kb)
@@ -175,8 +179,8 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             umma_commit(xt_empty(st2));
             umma_commit(gempty_bar(g));
             if (j == nt - 1) umma_commit(qfull_bar);
-            if (++st2 == STAGES) { st2 = 0; ph2 ^= 1u; }
-            if (++g == 2) { g = 0; g_phase ^= 1u; }
+            if (++st2 == XT_STAGES) { st2 = 0; ph2 ^= 1u; }
+            if (++g == G_BUFS) { g = 0; g_phase ^= 1u; }
           }
         }
       }
@@ -187,15 +191,16 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
     const int half = (warp - 2) >> 2;          // which 64 of the 128 columns
     const int row = q * 32 + lane;             // output channel (O^T, G^T) / input channel (Gq)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    int acc = 0, g = 0, sx = 0;
-    uint32_t acc_phase = 0, g_phase = 0, q_phase = 0, px = 0;
+    int acc = 0, g = 0, sx = 0, sxt = 0;
+    uint32_t acc_phase = 0, g_phase = 0, q_phase = 0, px = 0, pxt = 0;
     // transpose duty: this thread moves the 8 x 8 block (channels 8 bi.., tokens 8 bt..) of every tile; the
     // diagonal assignment of blocks to lanes keeps both the 16-byte loads and the 16-byte stores of a
     // quarter-warp on eight different bank groups of the swizzled tiles
     const int e = (warp - 2) * 32 + lane;
     const int bi = (e & 7) + 8 * ((e >> 6) & 1);
     const int bt = (((e & 7) + ((e >> 3) & 7)) & 7) + 8 * ((e >> 7) & 1);
-    uint8_t* stage_ptr = smem_raw + (stage_base - smem_u32(smem_raw));
+    uint8_t* xa_ptr = smem_raw + (xa_base - smem_u32(smem_raw));
+    uint8_t* xt_ptr = smem_raw + (xt_base - smem_u32(smem_raw));
     bool ok = true;
     for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
       int b, t0, t1;
@@ -204,10 +209,10 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
       for (int t = t0; t < t1; ++t) {
         // ---- X_t^T of this tile (operand of the second product)
         if (!mbar_wait(xa_full(sx), px, p.d_status)) { ok = false; break; }
-        if (!mbar_wait(xt_empty(sx), px ^ 1u, p.d_status)) { ok = false; break; }
+        if (!mbar_wait(xt_empty(sxt), pxt ^ 1u, p.d_status)) { ok = false; break; }
         {
-          const uint8_t* src = stage_ptr + sx * STAGE_BYTES + (bi >> 3) * KB_BYTES;
-          uint8_t* dst = stage_ptr + sx * STAGE_BYTES + XA_BYTES + (bt >> 3) * KB_BYTES;
+          const uint8_t* src = xa_ptr + sx * XA_BYTES + (bi >> 3) * KB_BYTES;
+          uint8_t* dst = xt_ptr + sxt * XT_BYTES + (bt >> 3) * KB_BYTES;
           uint32_t in[8][4];
 #pragma unroll
           for (int r = 0; r < 8; ++r) {      // token 8 bt + r: chunk (bi & 7) of its row sits at (bi & 7) ^ r
@@ -225,8 +230,9 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) { mbar_arrive(xt_full(sx)); mbar_arrive(xa_empty(sx)); }
-        if (++sx == STAGES) { sx = 0; px ^= 1u; }
+        if (lane == 0) { mbar_arrive(xt_full(sxt)); mbar_arrive(xa_empty(sx)); }
+        if (++sx == XA_STAGES) { sx = 0; px ^= 1u; }
+        if (++sxt == XT_STAGES) { sxt = 0; pxt ^= 1u; }
         // ---- Eq. 4 epilogue of O^T
         if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
         if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }
@@ -272,7 +278,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         __syncwarp();
         if (lane == 0) { mbar_arrive(tempty_bar(acc)); mbar_arrive(gfull_bar(g)); }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-        if (++g == 2) { g = 0; g_phase ^= 1u; }
+        if (++g == G_BUFS) { g = 0; g_phase ^= 1u; }
       }
       if (!ok) break;
       // partial Gq of the unit
