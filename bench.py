@@ -355,13 +355,13 @@ def main():
                     "algorithmic_flops_per_launch": fwd_flops}
         if path == dq.DQ_PATH_BF16_TC and d == 128 and t_fwd > 0:
             # per-head rotations: both contractions and the Eq. 4 epilogue are one kernel that reads the activations
-            # twice (token-major and channel-major) and keeps everything else on chip: 64 flop per byte, HBM-bound
-            hb = 4.0 * N * d * B
+            # once and keeps everything else on chip: 128 flop per byte, below the ridge of this GPU: HBM roofline
+            hb = 2.0 * N * d * B
             roofline = {"bound": "hbm", "kernel": "heads_whip_kernel (O = X R_h, Eq. 4, Gq_h = X^T dL/dO fused)",
                         "achieved": hb / t_fwd / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": hb / t_fwd / 1e9 / peaks["hbm_gbs"],
                         "peak_source": "%s (copy bandwidth)" % peaks["_source"],
-                        "traffic": 273.4e6 if wr.name == "c3_heads" else None,   # profiles/heads_whip_fused_c3_heads.md
+                        "traffic": 139.5e6 if wr.name == "c3_heads" else None,   # profiles/heads_whip_fused_c3_heads.md
                         "algorithmic_bytes_per_launch": hb}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
