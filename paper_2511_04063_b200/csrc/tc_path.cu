@@ -36,14 +36,15 @@ __global__ void __launch_bounds__(256) transpose_f32_to_bf16_kernel(const float*
 }
 
 // out tile = sum over slices of part[slice] tile, for the tiles of `list` (mb | nb << 16; tiles
-// are bm x bn); one CTA per tile, fixed summation order.
+// are bm x bn); gridDim.y CTAs per tile (a band of rows each), fixed summation order.
 __global__ void __launch_bounds__(256) tile_reduce_kernel(const float* __restrict__ part, int slices,
                                                           int64_t slice_stride, const int* __restrict__ list, int bm,
                                                           int bn, int d, float* __restrict__ out) {
   const int code = list[blockIdx.x];
-  const int r0 = (code & 0xffff) * bm, c0 = (code >> 16) * bn;
+  const int band = bm / gridDim.y;
+  const int r0 = (code & 0xffff) * bm + blockIdx.y * band, c0 = (code >> 16) * bn;
   const int per_row = bn / 4;
-  for (int e = threadIdx.x; e < bm * per_row; e += 256) {
+  for (int e = threadIdx.x; e < band * per_row; e += 256) {
     const int64_t idx = (int64_t)(r0 + e / per_row) * d + c0 + (e % per_row) * 4;
     float4 s = *reinterpret_cast<const float4*>(part + idx);
     for (int k = 1; k < slices; ++k) {
@@ -212,7 +213,7 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
     pt.tile_list = tc.tl_tail; pt.n_list = tc.n_tail; pt.ksplit = tc.tail_split;
     pt.out = tc.tail_part; pt.batch_stride = 0; pt.split_stride = (int64_t)d * d;
     DQ_CHECK(launch(pt));
-    tile_reduce_kernel<<<tc.n_tail, 256, 0, ctx.stream>>>(tc.tail_part, tc.tail_split, (int64_t)d * d, tc.tl_tail,
+    tile_reduce_kernel<<<dim3(tc.n_tail, 8), 256, 0, ctx.stream>>>(tc.tail_part, tc.tail_split, (int64_t)d * d, tc.tl_tail,
                                                           tc.pair ? 256 : 128, bn, d, Gq);
     return after_launch(ctx);
   }
