@@ -381,8 +381,9 @@ def main():
                 "gemm_frac_of_nominal_2250": gemm_tflops / 2250.0,
                 "qr_orth_share": (phases["qr_forward"] + phases["qr_backward"]) / total_phase if total_phase else None,
                 "loss_first_last": [float(losses[0].mean()), float(losses[-1].mean())]}
-        # the optimiser update is the HBM-bound kernel of the path: 12 bytes per latent entry (SGD)
-        upd_bytes = 12.0 * d * d * B
+        # the optimiser update is the HBM-bound kernel of the path: 12 bytes per latent entry (SGD: read Z and
+        # dL/dZ, write Z) plus 4 on the tensor-core path (the split-bf16 copy of the new latent for the next QR)
+        upd_bytes = (16.0 if path == dq.DQ_PATH_BF16_TC else 12.0) * d * d * B
         if phases["update"] > 0 and d != 128:      # for d = 128 the update is fused into the backward kernel
             gbs = upd_bytes / (phases["update"] * 1e-3) / 1e9
             line["update_hbm"] = {"kernel": "sgd_kernel", "bytes_per_launch": upd_bytes, "achieved_gbs": gbs,

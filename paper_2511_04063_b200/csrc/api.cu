@@ -243,8 +243,13 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
       h->f32_winv_valid = true;
     }
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
-    if (h->optimizer == DQ_SGD) DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, n_latent));
+    if (h->optimizer == DQ_SGD) {   // the tensor-core QR-Orth reads the latent as a split-bf16 pair: written here
+      const bool split = h->fast_qr && h->qtc.ready;
+      DQ_CHECK(sgd_update(ctx, h->Z, h->Gz, c.lr, n_latent, split ? h->qtc.z_hi : nullptr, split ? h->qtc.z_lo : nullptr));
+      h->qtc.z_split_fresh = split;
+    }
   }
+  if (h->optimizer != DQ_SGD) h->qtc.z_split_fresh = false;
   if (h->optimizer == DQ_SGD_MOMENTUM)
     DQ_CHECK(momentum_update(ctx, h->Z, h->Gz, h->opt_m, c.lr, h->beta1, n_latent));
   else if (h->optimizer == DQ_ADAM)
@@ -487,6 +492,7 @@ dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z) {
   DQ_CHECK(clear_status(h));
   h->r_stale = true;
   h->qtc.t_warm = false;   // the new latent may be far from the one the iterative QR last saw
+  h->qtc.z_split_fresh = false;
   h->small_warm = false;
   h->f32_winv_valid = false;
   h->cay_started = false;  // Cayley SGD restarts from the orthogonal factor of the new latent
@@ -582,6 +588,7 @@ dq_status dq_calib_set_orth_method(dq_calib_t* h, int32_t method, float beta, fl
   }
   DQ_CHECK(clear_status(h));
   h->orth_method = method;
+  h->qtc.z_split_fresh = false;   // Cayley SGD uses the latent's operand buffers as scratch
   h->cay_started = false;
   h->r_stale = true;
   h->qtc.t_warm = false;

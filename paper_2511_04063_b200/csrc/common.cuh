@@ -125,8 +125,9 @@ dq_status gather_tokens(Ctx& ctx, const void* X, int elem_bytes, int64_t n, int 
 
 // dst += src (n elements)
 dq_status accumulate(Ctx& ctx, float* dst, const float* src, int64_t n);
-// Z <- Z - lr Gz  (n elements)
-dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n);
+// Z <- Z - lr Gz  (n elements); z_hi / z_lo (nullable): also the split-bf16 copy of the new Z
+dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n, __nv_bfloat16* z_hi = nullptr,
+                     __nv_bfloat16* z_lo = nullptr);
 // v <- mu v + Gz; Z <- Z - lr v
 dq_status momentum_update(Ctx& ctx, float* Z, const float* Gz, float* V, float lr, float mu, int64_t n);
 // Adam with bias correction; pw = device float[2] {beta1^t, beta2^t}, advanced on the device

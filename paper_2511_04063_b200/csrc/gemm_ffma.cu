@@ -194,8 +194,10 @@ __global__ void __launch_bounds__(256) loss_finalize_kernel(const float* __restr
 
 // Every update kernel leaves the parameter (and the optimiser state) untouched once the status word holds
 // an error: a step whose factorisation failed or whose loss was not finite never reaches the latent.
+// hi / lo (nullable): also write the split-bf16 copy of the new Z (hi = bf16(z), lo = bf16(z - hi)), the
+// operand form the next factorisation reads, so that it needs no separate pass over Z.
 __global__ void sgd_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz, float lr, int64_t n4,
-                           const int* __restrict__ d_status) {
+                           const int* __restrict__ d_status, uint2* __restrict__ hi, uint2* __restrict__ lo) {
   if (d_status && *d_status != 0) return;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
@@ -204,6 +206,14 @@ __global__ void sgd_kernel(float4* __restrict__ Z, const float4* __restrict__ Gz
     z.x = fmaf(-lr, g.x, z.x); z.y = fmaf(-lr, g.y, z.y);
     z.z = fmaf(-lr, g.z, z.z); z.w = fmaf(-lr, g.w, z.w);
     Z[i] = z;
+    if (hi) {
+      const __nv_bfloat162 h0 = __floats2bfloat162_rn(z.x, z.y), h1 = __floats2bfloat162_rn(z.z, z.w);
+      const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
+      const __nv_bfloat162 l0 = __floats2bfloat162_rn(z.x - f0.x, z.y - f0.y);
+      const __nv_bfloat162 l1 = __floats2bfloat162_rn(z.z - f1.x, z.w - f1.y);
+      hi[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+      lo[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+    }
   }
 }
 
@@ -284,14 +294,16 @@ dq_status accumulate(Ctx& ctx, float* dst, const float* src, int64_t n) {
 }
 
 // Algorithm 1 (update step).  n is a multiple of 4 (d is a multiple of 32).
-dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n) {
+dq_status sgd_update(Ctx& ctx, float* Z, const float* Gz, float lr, int64_t n, __nv_bfloat16* z_hi,
+                     __nv_bfloat16* z_lo) {
   const int64_t n4 = n / 4;
   int blocks = (int)((n4 + 255) / 256);
   const int cap = ctx.sm_count * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   sgd_kernel<<<blocks, 256, 0, ctx.stream>>>(reinterpret_cast<float4*>(Z),
-                                            reinterpret_cast<const float4*>(Gz), lr, n4, ctx.d_status);
+                                            reinterpret_cast<const float4*>(Gz), lr, n4, ctx.d_status,
+                                            reinterpret_cast<uint2*>(z_hi), reinterpret_cast<uint2*>(z_lo));
   return after_launch(ctx);
 }
 

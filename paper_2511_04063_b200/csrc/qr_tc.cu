@@ -378,8 +378,11 @@ dq_status qr_upper_factor_incremental(Ctx& ctx, QrWorkspace& ws, QrTcState& q, c
   bf16 *zht_hi = q.st_hi, *zht_lo = q.st_lo;   // free until the backward pass
   bf16 *uh_hi = q.gqt_hi, *uh_lo = q.gqt_lo;   // likewise
   float *Zh = ws.A, *G = ws.B, *P = ws.S, *T = ws.tmp, *scratch = ws.Q;
-  split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
-  DQ_CHECK(after_launch(ctx));
+  if (!q.z_split_fresh) {   // (the SGD update writes the split copy with the new latent)
+    split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
+    DQ_CHECK(after_launch(ctx));
+    q.z_split_fresh = true;
+  }
   {   // Zh[i][j] = sum_k Z[i][k] W_old[k][j]
     Op a{q.z_hi, q.z_lo, d, dd}, b{q.wt_hi, q.wt_lo, d, dd};
     Out o; o.f32 = Zh; o.ld = d; o.bs = dd; o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
@@ -448,9 +451,10 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
     DQ_CHECK(after_launch(ctx));
     q.t_warm = true;
   }
-  if (!incremental) {
+  if (!q.z_split_fresh) {
     split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
     DQ_CHECK(after_launch(ctx));
+    q.z_split_fresh = true;
   }
   // R[i][j] = sum_k Z[i][k] W[k][j]:  A = Z (row-major), B = W^T
   Op a{q.z_hi, q.z_lo, d, dd};

@@ -72,6 +72,7 @@ struct QrTcState {
   // near-orthogonal iterative factorisation
   __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T^T of the sweeps
   __nv_bfloat16 *uot_hi = nullptr, *uot_lo = nullptr;   // U^T of the previous step
+  bool z_split_fresh = false;                           // z_hi / z_lo are the split copy of the current latent
   bool t_warm = false;                                  // wt_* / uot_* hold the factors of the previous step's latent
   int* sweep_flags = nullptr;                           // [80] device flags: sweep k moved an entry
   // tile orders for triangular products (device arrays of mb | nb << 16)
