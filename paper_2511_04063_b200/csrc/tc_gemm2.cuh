@@ -9,11 +9,11 @@
 // peer's operands from the same shared-memory offsets.  Protocol per CTA (192 threads as in the
 // one-CTA kernel):
 //   warp 0   TMA producer: waits on its own empty barrier (armed for both CTAs by the leader's
-//            multicast commit); both CTAs' loads complete on the LEADER's full barrier
-//   warp 1   leader only: MMA issue; commits multicast to both CTAs' empty / accumulator-full barriers
+//            commit to both CTAs); both CTAs' loads complete on the LEADER's full barrier
+//   warp 1   leader only: MMA issue; its commits arrive on both CTAs' empty / accumulator-full barriers
 //   warps 2..5  epilogue from the CTA's own TMEM; both CTAs arrive on the leader's accumulator-empty
 //            barrier
-// No TMA multicast is used.  Every wait is bounded (DQ_ERR_TIMEOUT in the status word on expiry).
+// Every TMA load is a plain per-CTA copy.  Every wait is bounded (DQ_ERR_TIMEOUT in the status word on expiry).
 #pragma once
 #include "tc_gemm.cuh"
 
