@@ -52,8 +52,8 @@ enum { DQ_MEAN_TOKENS = 0, DQ_SUM_TOKENS = 1 }; /* reduction of Eq. 4 over token
 enum { DQ_SGD = 0, DQ_SGD_MOMENTUM = 1, DQ_ADAM = 2 }; /* optimiser (Algorithm 1, update step; Sec. 4.3: "SGD or Adam") */
 
 typedef struct {
-  int32_t d;         /* channels = size of the rotation; multiple of 32 (fp32 path) or 128 (tensor-core path); <= 8192 */
-  int64_t n_tokens;  /* tokens per problem; multiple of 32 (fp32 path) or 256 (tensor-core path) */
+  int32_t d;         /* channels = size of the rotation; multiple of 64 (fp32 path) or 128 (tensor-core path); <= 8192 */
+  int64_t n_tokens;  /* tokens per problem; any positive count (fp32 path) or a multiple of 256 (tensor-core path) */
   int32_t batch;     /* independent problems (e.g. attention heads); >= 1       */
   int32_t x_dtype;   /* DQ_FP32 | DQ_BF16                                       */
   int32_t path;      /* DQ_PATH_FP32: fp32 FMA contractions (needs DQ_FP32 X);
@@ -65,7 +65,7 @@ typedef struct {
 } dq_calib_config;
 
 /* Algorithm 1, hand-off before the loop: bind calibration activations and the initial
- * latent.  d_X is BORROWED (must outlive the handle, is never written).  d_Z0
+ * latent.  d_X is BORROWED (must outlive the handle; only dq_calib_run_epochs writes it).  d_Z0
  * ([batch][d][d] fp32) is COPIED.  cuda_stream is a cudaStream_t (NULL = legacy
  * default stream).  Allocates every workspace the step needs.
  * Errors: INVALID_ARG, UNSUPPORTED, ALLOC, CUDA.  *out is NULL on error. */
