@@ -25,6 +25,25 @@ constexpr int BWD_SMEM = 3 * N * LD * 4;
 using mma::warp_mm32;
 using mma::zero_acc;
 
+// 128 x 128 fp32 matrix: global memory -> registers (eight coalesced 16-byte loads per thread) and
+// registers -> shared memory (row stride LD; rows and LD are multiples of four floats).
+__device__ __forceinline__ void g2r(const float* __restrict__ g, float4 (&v)[8], int tid) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) v[k] = reinterpret_cast<const float4*>(g)[tid + k * NT];
+}
+__device__ __forceinline__ void r2s(float* s, const float4 (&v)[8], int tid) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int e = (tid + k * NT) * 4;
+    *reinterpret_cast<float4*>(s + (e >> 7) * LD + (e & 127)) = v[k];
+  }
+}
+__device__ __forceinline__ void g2s(const float* __restrict__ g, float* s, int tid) {
+  float4 v[8];
+  g2r(g, v, tid);
+  r2s(s, v, tid);
+}
+
 template <typename F>
 __device__ __forceinline__ void acc_foreach(float (&acc)[2][4][4], int r0, int c0, int lane, F f) {
   const int g = lane >> 2, t = lane & 3;
@@ -79,9 +98,12 @@ qr128_forward_inc_kernel(const float* __restrict__ Z, float* __restrict__ R, flo
   float acc[2][4][4];
 
   // ---- Zh = Z W_old (W_old upper triangular: k <= column)
-  for (int e = tid; e < N * N; e += NT) {
-    B0[(e >> 7) * LD + (e & 127)] = Z[e];
-    B1[(e >> 7) * LD + (e & 127)] = W[e];
+  {
+    float4 zv[8], wv[8];
+    g2r(Z, zv, tid);
+    g2r(W, wv, tid);
+    r2s(B0, zv, tid);
+    r2s(B1, wv, tid);
   }
   __syncthreads();
   zero_acc(acc);
@@ -137,7 +159,7 @@ qr128_forward_inc_kernel(const float* __restrict__ Z, float* __restrict__ R, flo
   if (!converged && tid == 0) set_status(d_status, DQ_ERR_NOT_CONVERGED);
   // ---- U = (I + T) U_old: both upper triangular, k in [32 wr, 32 (wc + 1))
   if (tid < N) T[tid * LD + tid] += 1.f;
-  for (int e = tid; e < N * N; e += NT) B0[(e >> 7) * LD + (e & 127)] = U[e];
+  g2s(U, B0, tid);
   __syncthreads();
   if (wr <= wc) {
     zero_acc(acc);
@@ -195,7 +217,7 @@ qr128_forward_inc_kernel(const float* __restrict__ Z, float* __restrict__ R, flo
   __syncthreads();
   smem_mm(X, LD, Tmp, TMP_LD, X + 64, LD, 64, 64, 64, -1.f, tid);
   // ---- R = Z W (Z reloaded into B0; U_old is no longer needed)
-  for (int e = tid; e < N * N; e += NT) B0[(e >> 7) * LD + (e & 127)] = Z[e];
+  g2s(Z, B0, tid);
   __syncthreads();
   zero_acc(acc);
   warp_mm32<false, false>(B0, X, LD, acc, r0, c0, 0, 32 * (wc + 1), lane);
@@ -223,9 +245,14 @@ qr128_backward_sgd_tc_kernel(const float* __restrict__ R, const float* __restric
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int wr = warp >> 2, wc = warp & 3, r0 = 32 * wr, c0 = 32 * wc;
   float acc[2][4][4];
-  for (int e = tid; e < N * N; e += NT) {
-    P0[(e >> 7) * LD + (e & 127)] = R[e];
-    P1[(e >> 7) * LD + (e & 127)] = Gq[e];
+  float4 wv[8];                      // W is fetched now and parked in registers until its buffer is free
+  {
+    float4 rv[8], gv[8];
+    g2r(R, rv, tid);
+    g2r(Gq, gv, tid);
+    g2r(W, wv, tid);
+    r2s(P0, rv, tid);
+    r2s(P1, gv, tid);
   }
   __syncthreads();
   zero_acc(acc);
@@ -241,7 +268,7 @@ qr128_backward_sgd_tc_kernel(const float* __restrict__ R, const float* __restric
   warp_mm32<false, false>(P0, P1, LD, acc, r0, c0, 32 * wc, N, lane);   // M = R S: S[k][c] = 0 for k <= c
   __syncthreads();                                                      // everyone is done reading B's buffer
   acc_foreach(acc, r0, c0, lane, [&](int r, int c, float& v) { P2[r * LD + c] = v; });
-  for (int e = tid; e < N * N; e += NT) P1[(e >> 7) * LD + (e & 127)] = W[e];
+  r2s(P1, wv, tid);
   __syncthreads();
   zero_acc(acc);
   warp_mm32<false, true>(P2, P1, LD, acc, r0, c0, 32 * wc, N, lane);    // Gz = M W^T: W[c][k] = 0 for k < c
