@@ -38,6 +38,14 @@ __device__ __forceinline__ void r2s(float* s, const float4 (&v)[8], int tid) {
     *reinterpret_cast<float4*>(s + (e >> 7) * LD + (e & 127)) = v[k];
   }
 }
+// shared memory (row stride LD) -> global, 16 bytes per store
+__device__ __forceinline__ void s2g(const float* s, float* __restrict__ g, int tid) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int e = (tid + k * NT) * 4;
+    reinterpret_cast<float4*>(g)[tid + k * NT] = *reinterpret_cast<const float4*>(s + (e >> 7) * LD + (e & 127));
+  }
+}
 __device__ __forceinline__ void g2s(const float* __restrict__ g, float* s, int tid) {
   float4 v[8];
   g2r(g, v, tid);
@@ -184,10 +192,11 @@ qr128_forward_inc_kernel(const float* __restrict__ Z, float* __restrict__ R, flo
     if (lane == 0) { sc[warp] = mn; sc[4 + warp] = mx; }
     if (!isfinite(dv)) set_status(d_status, DQ_ERR_NONFINITE);
   }
-  for (int e = tid; e < N * N; e += NT) {
-    const int r = e >> 7, c = e & 127;
-    U[e] = Us[r * LD + c];
-    X[r * LD + c] = 0.f;
+  s2g(Us, U, tid);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int e = (tid + k * NT) * 4;
+    *reinterpret_cast<float4*>(X + (e >> 7) * LD + (e & 127)) = make_float4(0.f, 0.f, 0.f, 0.f);
   }
   __syncthreads();
   if (tid == 0) {
@@ -223,11 +232,19 @@ qr128_forward_inc_kernel(const float* __restrict__ Z, float* __restrict__ R, flo
   warp_mm32<false, false>(B0, X, LD, acc, r0, c0, 0, 32 * (wc + 1), lane);
   acc_foreach(acc, r0, c0, lane, [&](int r, int c, float& v) { Us[r * LD + c] = v; });   // U is in global memory by now
   __syncthreads();
-  for (int e = tid; e < N * N; e += NT) {
-    const int r = e >> 7, c = e & 127;
-    R[e] = Us[r * LD + c];
-    W[e] = X[r * LD + c];
-    if (Rt_bf16) Rt_bf16[e] = __float2bfloat16_rn(Us[c * LD + r]);   // R^T
+  s2g(Us, R, tid);
+  s2g(X, W, tid);
+  if (Rt_bf16) {   // R^T in bf16: lane = row of R^T (consecutive columns of R in shared memory), 8 entries per store
+    for (int idx = tid; idx < N * (N / 8); idx += NT) {
+      const int c = idx & 127, rb = idx >> 7;
+      uint32_t pk[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(Us[(8 * rb + 2 * i) * LD + c], Us[(8 * rb + 2 * i + 1) * LD + c]);
+        pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      *reinterpret_cast<uint4*>(Rt_bf16 + c * N + 8 * rb) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
   }
 }
 
