@@ -1,5 +1,5 @@
 // Fused Whip step for many 128 x 128 rotations (per-head rotations): one kernel computes, per head h
-// and per tile of 128 tokens,
+// and per tile of TT = 64 tokens,
 //   O^T = R_h^T X_t^T   (tcgen05, accumulator in tensor memory)
 //   e = exp(-|o|), loss partials, G = -sign(o) e   (Eq. 4; epilogue from tensor memory)
 //   Gq_h += X_t^T G_t    (second tcgen05 product: G_t goes from the epilogue's registers into shared
@@ -12,7 +12,7 @@
 // one 128 x 128 fp32 partial of Gq and four loss partials, summed afterwards in a fixed order.
 //
 // 320 threads: warp 0 TMA producer (R_h^T and the X_t ring), warp 1 MMA issuer, warps 2..9 transpose +
-// epilogue (two warps per quarter of the tensor-memory lanes, 64 columns each).  X_t is released once the
+// epilogue (two warps per quarter of the tensor-memory lanes, 32 token columns each).  X_t is released once the
 // first product has retired and the tile has been transposed, X_t^T and G_t after the second product;
 // two O accumulators.  Every wait is bounded
 // (DQ_ERR_TIMEOUT on expiry).
@@ -24,16 +24,19 @@ namespace heads {
 
 using namespace tc;
 
+constexpr int TT = 64;                             // tokens per tile
 constexpr int KB_BYTES = 128 * BLOCK_K * 2;        // one [128 rows][64 bf16] K-major block: 16 KB
+constexpr int XKB_BYTES = TT * BLOCK_K * 2;        // one [TT rows][64 bf16] K-major block of X_t: 8 KB
 constexpr int RT_BYTES = 2 * KB_BYTES;             // R_h^T: rows = output channel, K = input channel (128)
-constexpr int XA_BYTES = 2 * KB_BYTES;             // X_t:   rows = token, K = input channel
-constexpr int XT_BYTES = 2 * KB_BYTES;             // X_t^T: rows = input channel, K = token
-constexpr int G_BYTES = 2 * KB_BYTES;              // G_t^T: rows = output channel, K = token
-// Ring depths (measured on the 32-head workload: two of each is fastest; a deeper X_t ring with the two
-// on-chip operands of the second product single-buffered is about 10 % slower).
-constexpr int XA_STAGES = 2, XT_STAGES = 2, G_BUFS = 2;
+constexpr int XA_BYTES = 2 * XKB_BYTES;            // X_t:   rows = token (TT), K = input channel (two k-blocks)
+constexpr int XT_BYTES = KB_BYTES;                 // X_t^T: rows = input channel, K = token (TT = one k-block)
+constexpr int G_BYTES = KB_BYTES;                  // G_t^T: rows = output channel, K = token
+// Two CTAs share an SM (each under half of its shared memory and half of its tensor memory): while one
+// waits for a load or runs its epilogue the other issues products.  Tiles of 64 tokens keep a CTA at
+// 96 KB: R_h^T, two X_t stages, one X_t^T and one G_t buffer.
+constexpr int XA_STAGES = 2, XT_STAGES = 1, G_BUFS = 1;
 constexpr int SMEM_TOTAL = RT_BYTES + XA_STAGES * XA_BYTES + XT_STAGES * XT_BYTES + G_BUFS * G_BYTES + 1024 + 1024;
-constexpr uint32_t TMEM_COLS = 512;                // O (2 x 128 columns) + Gq (128 columns)
+constexpr uint32_t TMEM_COLS = 256;                // O (2 x TT columns) + Gq (128 columns)
 constexpr int HEADS_THREADS = 320;
 constexpr int EPI_WARPS = 8;
 
@@ -48,9 +51,10 @@ struct Params {
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__global__ void __launch_bounds__(HEADS_THREADS, 1)
+__global__ void __launch_bounds__(HEADS_THREADS, 2)
 heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_constant__ CUtensorMap mapX, const Params p) {
-  constexpr uint32_t IDESC = make_idesc_bf16(128);
+  constexpr uint32_t IDESC_O = make_idesc_bf16(TT);     // O^T tile: 128 channels x TT tokens
+  constexpr uint32_t IDESC_Q = make_idesc_bf16(128);    // Gq: 128 x 128
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t rt_smem = smem_base;
@@ -92,7 +96,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
-  const uint32_t tmem_q = tmem_base + 256u;
+  const uint32_t tmem_q = tmem_base + 2u * TT;
 
   const int units = p.batch * p.splits;
   auto unit_range = [&](int u, int& b, int& t0, int& t1) {
@@ -120,8 +124,8 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
           if (!mbar_wait(xa_empty(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
           mbar_expect_tx(xa_full(stage), XA_BYTES);
           const uint32_t xa = xa_base + stage * XA_BYTES;
-          tma_load_3d(xa, &mapX, xa_full(stage), 0, t * 128, b);
-          tma_load_3d(xa + KB_BYTES, &mapX, xa_full(stage), BLOCK_K, t * 128, b);
+          tma_load_3d(xa, &mapX, xa_full(stage), 0, t * TT, b);
+          tma_load_3d(xa + XKB_BYTES, &mapX, xa_full(stage), BLOCK_K, t * TT, b);
           if (++stage == XA_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -145,13 +149,13 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t xa = xa_base + st1 * XA_BYTES;
-            const uint32_t tmem_o = tmem_base + (uint32_t)(acc * 128);
+            const uint32_t tmem_o = tmem_base + (uint32_t)(acc * TT);
 #pragma unroll
             for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
               for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
                 umma_bf16(tmem_o, make_kmajor_sw128_desc(rt_smem + kb * KB_BYTES + k * UMMA_K * 2),
-                          make_kmajor_sw128_desc(xa + kb * KB_BYTES + k * UMMA_K * 2), IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+                          make_kmajor_sw128_desc(xa + kb * XKB_BYTES + k * UMMA_K * 2), IDESC_O, (kb > 0 || k > 0) ? 1u : 0u);
             umma_commit(tfull_bar(acc));
             umma_commit(xa_empty(st1));                  // X_t can be replaced once this product has retired
             if (i == nt - 1) umma_commit(rtempty_bar);   // R_h^T may be replaced once these products retire
@@ -170,12 +174,9 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             const uint32_t xt = xt_base + st2 * XT_BYTES;
             const uint32_t gb = g_base + g * G_BYTES;
 #pragma unroll
-            for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-              for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                umma_bf16(tmem_q, make_kmajor_sw128_desc(xt + kb * KB_BYTES + k * UMMA_K * 2),
-                          make_kmajor_sw128_desc(gb + kb * KB_BYTES + k * UMMA_K * 2), IDESC,
-                          (j > 0 || kb > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < TT / UMMA_K; ++k)
+              umma_bf16(tmem_q, make_kmajor_sw128_desc(xt + k * UMMA_K * 2), make_kmajor_sw128_desc(gb + k * UMMA_K * 2),
+                        IDESC_Q, (j > 0 || k > 0) ? 1u : 0u);
             umma_commit(xt_empty(st2));
             umma_commit(gempty_bar(g));
             if (j == nt - 1) umma_commit(qfull_bar);
@@ -196,9 +197,10 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
     // transpose duty: this thread moves the 8 x 8 block (channels 8 bi.., tokens 8 bt..) of every tile; the
     // diagonal assignment of blocks to lanes keeps both the 16-byte loads and the 16-byte stores of a
     // quarter-warp on eight different bank groups of the swizzled tiles
-    const int e = (warp - 2) * 32 + lane;
+    const int e = (warp - 2) * 32 + lane;      // blocks: 16 (channels) x TT / 8 (tokens) = 128, threads 0..127
     const int bi = (e & 7) + 8 * ((e >> 6) & 1);
-    const int bt = (((e & 7) + ((e >> 3) & 7)) & 7) + 8 * ((e >> 7) & 1);
+    const int bt = ((e & 7) + ((e >> 3) & 7)) & 7;
+    const bool transposer = e < 16 * (TT / 8);
     uint8_t* xa_ptr = smem_raw + (xa_base - smem_u32(smem_raw));
     uint8_t* xt_ptr = smem_raw + (xt_base - smem_u32(smem_raw));
     bool ok = true;
@@ -210,13 +212,13 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         // ---- X_t^T of this tile (operand of the second product)
         if (!mbar_wait(xa_full(sx), px, p.d_status)) { ok = false; break; }
         if (!mbar_wait(xt_empty(sxt), pxt ^ 1u, p.d_status)) { ok = false; break; }
-        {
-          const uint8_t* src = xa_ptr + sx * XA_BYTES + (bi >> 3) * KB_BYTES;
-          uint8_t* dst = xt_ptr + sxt * XT_BYTES + (bt >> 3) * KB_BYTES;
+        if (transposer) {
+          const uint8_t* src = xa_ptr + sx * XA_BYTES + (bi >> 3) * XKB_BYTES;
+          uint8_t* dst = xt_ptr + sxt * XT_BYTES;
           uint32_t in[8][4];
 #pragma unroll
           for (int r = 0; r < 8; ++r) {      // token 8 bt + r: chunk (bi & 7) of its row sits at (bi & 7) ^ r
-            const uint4 v = *reinterpret_cast<const uint4*>(src + (8 * (bt & 15) + r) * 128 + (((bi & 7) ^ r) << 4));
+            const uint4 v = *reinterpret_cast<const uint4*>(src + (8 * bt + r) * 128 + (((bi & 7) ^ r) << 4));
             in[r][0] = v.x; in[r][1] = v.y; in[r][2] = v.z; in[r][3] = v.w;
           }
 #pragma unroll
@@ -225,7 +227,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
 #pragma unroll
             for (int w = 0; w < 4; ++w)
               o[w] = __byte_perm(in[2 * w][r >> 1], in[2 * w + 1][r >> 1], (r & 1) ? 0x7632 : 0x5410);
-            *reinterpret_cast<uint4*>(dst + (8 * bi + r) * 128 + (((bt & 7) ^ r) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(dst + (8 * bi + r) * 128 + ((bt ^ r) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
           }
         }
         fence_async_smem();
@@ -238,12 +240,11 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }
         tc_fence_after();
         uint8_t* gbuf = g_ptr + g * G_BYTES;
-        // both 32-column chunks of this warp are requested before the first is used
-        uint32_t va[32], vb[32];
-        tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * 128 + (2 * half) * 32), va);
-        tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * 128 + (2 * half + 1) * 32), vb);
-        tmem_ld_wait();
-        auto process = [&](int c, const uint32_t (&v)[32]) {
+        {   // this warp's 32 token columns of the TT-wide tile
+          const int c = half;
+          uint32_t v[32];
+          tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * TT + c * 32), v);
+          tmem_ld_wait();
           uint32_t packed[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -255,24 +256,22 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
             packed[i] = *reinterpret_cast<const uint32_t*>(&h);
           }
-          // tokens 32 c .. 32 c + 31 of row `row`: k-block c >> 1, 16-byte chunks 4 (c & 1) .. + 3,
-          // stored where the 128-byte swizzle of a K-major tile expects them
-          uint8_t* rowp = gbuf + (c >> 1) * KB_BYTES + row * 128;
+          // tokens 32 c .. 32 c + 31 of row `row`: 16-byte chunks 4 c .. 4 c + 3, stored where the 128-byte
+          // swizzle of a K-major tile expects them
+          uint8_t* rowp = gbuf + row * 128;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const int chunk = ((c & 1) * 4 + i) ^ (row & 7);
+            const int chunk = (c * 4 + i) ^ (row & 7);
             *reinterpret_cast<uint4*>(rowp + chunk * 16) =
                 make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
           }
           if (p.Gt) {
-            uint4* dst = reinterpret_cast<uint4*>(p.Gt + ((int64_t)b * 128 + row) * p.n_tokens + (int64_t)t * 128 + c * 32);
+            uint4* dst = reinterpret_cast<uint4*>(p.Gt + ((int64_t)b * 128 + row) * p.n_tokens + (int64_t)t * TT + c * 32);
 #pragma unroll
             for (int i = 0; i < 4; ++i)
               dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
           }
-        };
-        process(2 * half, va);
-        process(2 * half + 1, vb);
+        }
         tc_fence_before();
         fence_async_smem();                    // the tensor core reads G through the async proxy
         __syncwarp();

@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(256) tile_reduce_kernel(const float* __restric
 }
 
 struct Maps {
-  CUtensorMap rt, x, x128, xt, gt128, gt256;
+  CUtensorMap rt, x, x128, x64, xt, gt128, gt256;
 };
 
 }  // namespace
@@ -110,13 +110,14 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   DQ_CHECK(tch::make_map(&m->rt, tc.Rt, d, d, batch, d, (int64_t)d * d, tc::BLOCK_M));
   DQ_CHECK(tch::make_map(&m->x, tc.X, d, N, batch, d, N * d, 256));
   DQ_CHECK(tch::make_map(&m->x128, tc.X, d, N, batch, d, N * d, 128));
+  DQ_CHECK(tch::make_map(&m->x64, tc.X, d, N, batch, d, N * d, heads::TT));
   DQ_CHECK(tch::make_map(&m->xt, tc.Xt, N, d, batch, N, N * d, tc::BLOCK_M));
   DQ_CHECK(tch::make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
   DQ_CHECK(tch::make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
   DQ_CHECK(tc_refresh_inputs(tc, ctx));
-  if (d == 128) {   // per-head rotations: fused kernel, units = (head, range of 128-token tiles)
-    const int tiles_per_head = (int)(N / 128);
-    int sp = ctx.sm_count / batch;
+  if (d == 128) {   // per-head rotations: fused kernel, units = (head, range of token tiles), two CTAs per SM
+    const int tiles_per_head = (int)(N / heads::TT);
+    int sp = 2 * ctx.sm_count / batch;
     if (sp > tiles_per_head) sp = tiles_per_head;
     if (sp < 1) sp = 1;
     tc.splits = sp;
@@ -157,12 +158,12 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
   if (tc.fused) {
     Maps* mm = reinterpret_cast<Maps*>(tc.maps);
     heads::Params hp{};
-    hp.batch = tc.batch; hp.tiles_per_head = (int)(tc.n_tokens / 128); hp.splits = tc.splits;
+    hp.batch = tc.batch; hp.tiles_per_head = (int)(tc.n_tokens / heads::TT); hp.splits = tc.splits;
     hp.n_tokens = tc.n_tokens; hp.part = tc.heads_part; hp.partials = partials;
     hp.Gt = tc.keep_g ? tc.Gt : nullptr; hp.d_status = ctx.d_status;
     const int units = tc.batch * tc.splits;
-    const int grid = units < ctx.sm_count ? units : ctx.sm_count;
-    heads::heads_whip_kernel<<<grid, heads::HEADS_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x128, hp);
+    const int grid = units < 2 * ctx.sm_count ? units : 2 * ctx.sm_count;
+    heads::heads_whip_kernel<<<grid, heads::HEADS_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x64, hp);
     tc.n_partials_live = tc.splits * heads::EPI_WARPS;
     tc.fused_valid = true;
     ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;   // the second product runs here too
