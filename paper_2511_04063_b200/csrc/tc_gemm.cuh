@@ -86,6 +86,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* d_
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
+    __nanosleep(32);   // leave the issue slots to the warps that have work
     if ((++spins & 0xFFu) == 0u && global_timer_ns() - t0 > WAIT_LIMIT_NS) {
       set_status(d_status, DQ_ERR_TIMEOUT);
       return false;
