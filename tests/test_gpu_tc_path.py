@@ -289,3 +289,26 @@ def test_incremental_qr_takes_as_many_sweeps_as_a_large_step_needs():
     assert np.abs(R - Rr).max() <= 5e-5 * max(1.0, cond)
     assert np.abs(R.T @ R - np.eye(w.d)).max() <= 1e-4
     c.close()
+
+
+@pytest.mark.parametrize("name,d,path", [("c3_heads", 128, "tc"), ("c1_tiny", 256, "fp32")])
+def test_failed_step_freezes_the_latent_on_the_other_incremental_kernels(name, d, path):
+    """The same contract as for the large tensor-core path, on the shared-memory kernels for 128 x 128 latents
+    and on the fp32 path: after a step that moved the latent too far for the incremental factorisation, the
+    status word is set, later steps change nothing, and Householder factors the frozen latent."""
+    w = small(name, d=d, n_tokens=512, batch=2 if d == 128 else 1)
+    c = Calib(w, Z0=_near_orthogonal(d, w.batch, 0.02, 11), lr=50.0)
+    c.step(1)                                                       # Householder start, absurd step
+    assert c.status() == dq.DQ_OK
+    Z1 = c.latent()
+    c.step(3)
+    assert c.status() != dq.DQ_OK
+    assert np.array_equal(c.latent(), Z1)
+    dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_HOUSEHOLDER, 0)
+    assert c.status() == dq.DQ_OK
+    R = c.rotation()
+    for b in range(w.batch):
+        Rr, _ = orc.qr_pos_lapack(Z1[b])
+        cond = np.linalg.cond(Z1[b].astype(np.float64))
+        assert np.abs(R[b] - Rr).max() <= 5e-5 * max(1.0, cond)
+    c.close()
