@@ -30,9 +30,10 @@ sys.path.insert(0, ROOT)
 METRIC = "calibration steps/sec"
 UNIT = "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM traffic of one launch of the forward kernel on the c2_7b workload, from the ncu
-# capture summarised in profiles/ (bytes read + written); None until captured.
-NCU_TRAFFIC_BYTES = {"c2_7b": 311.0e6}   # profiles/tc_gemm_whip_forward_c2_7b.md
+# DRAM traffic (bytes read + written) of one launch of the roofline kernel, from an ncu capture of
+# that kernel on the named workload; None where no capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {"c2_7b": 311.0e6}
+NCU_TRAFFIC_BYTES_HEADS = {"c3_heads": 139.5e6}
 
 
 def load_peaks():
@@ -60,7 +61,7 @@ class ClockSampler:
     def start(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
-                                       "--format=csv,noheader,nounits", "-lms", "50"],
+                                       "--format=csv,noheader,nounits", "-lms", "10"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -98,42 +99,79 @@ class ClockSampler:
         return out
 
 
-def oracle_sample_steps_per_s(w, n_steps: int, shrink: int):
-    """Times the float64 oracle on the workload shrunk by `shrink` in both d and N.
-    Every term of a step scales with N d^2 or d^3, i.e. by shrink^3, so the full-size
-    rate is the sample's rate / shrink^3."""
-    import oracle as orc
-    from paper_2511_04063_b200 import inputs as gen
-    ws = gen.scaled(w, d=w.d // shrink, n_tokens=w.n_tokens // shrink,
-                    n_outlier_channels=max(1, w.n_outlier_channels // shrink))
-    X = gen.activations_as_f32(ws, gen.gen_activations(ws))[0].astype(np.float64)
-    Z = gen.gen_latent_init(ws)[0].astype(np.float64)
-    t0 = time.perf_counter()
-    for _ in range(n_steps):
-        Z = orc.calib_step(X, Z, ws.lr)["Z_new"]
-    dt = (time.perf_counter() - t0) / n_steps
+def oracle_thread_count() -> int:
     try:
         from threadpoolctl import threadpool_info
-        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        return max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
     except Exception:
-        cores = os.cpu_count() or 1
-    sample = ("oracle.calib_step x%d on the same recipe at d=%d, N=%d (1/%d of each dimension); "
-              "rate divided by %d^3" % (n_steps, ws.d, ws.n_tokens, shrink, shrink))
-    return 1.0 / (dt * shrink ** 3), dt, cores, sample
+        return os.cpu_count() or 1
+
+
+class OracleRun:
+    """The float64 oracle (oracle.calib_step, as it stands) on a workload's own inputs, one problem.
+
+    The QR of a step is the oracle's literal Algorithm 2 loop up to d = 512 and its library-QR form
+    (oracle.qr_pos_lapack: the same unique factors, which the oracle's tests pin the loop to) beyond, where
+    the loop's d dependent rank-one updates would take minutes per step.  A workload whose step costs more
+    than `max_flops` float64 flops is sampled: a prefix of the token rows, the rate scaled by the ratio of the
+    step's flop counts and the line marked as extrapolated."""
+
+    def __init__(self, w, max_flops: float = 4e12):
+        import oracle as orc
+        from paper_2511_04063_b200 import inputs as gen
+        self.orc, self.w = orc, w
+        d, n = w.d, w.n_tokens
+        cost = lambda nt: 4.0 * nt * d * d + 10.0 * d ** 3
+        self.n_used = n
+        while cost(self.n_used) > max_flops and self.n_used > 2048:
+            self.n_used //= 2
+        self.extrapolated = self.n_used != n
+        self.scale = cost(self.n_used) / cost(n)          # full-size steps per sampled step
+        wx = gen.scaled(w, batch=1)                       # one problem; a batch is `batch` such steps
+        X = gen.activations_as_f32(wx, gen.gen_activations(wx))[0]
+        self.X = X[:self.n_used].astype(np.float64)
+        self.Z = gen.gen_latent_init(wx)[0].astype(np.float64)
+        self.qr = orc.qr_pos if d <= 512 else orc.qr_pos_lapack
+        self.cores = oracle_thread_count()
+
+    def step(self):
+        self.Z = self.orc.calib_step(self.X, self.Z, self.w.lr, qr=self.qr)["Z_new"]
+
+    def time_steps(self, n_steps: int) -> float:
+        """Seconds per full-size step of the whole batch, from n_steps oracle steps."""
+        t0 = time.perf_counter()
+        for _ in range(n_steps):
+            self.step()
+        dt = (time.perf_counter() - t0) / n_steps
+        return dt * self.w.batch / self.scale
+
+    def sample(self, n_steps: int) -> str:
+        s = "oracle.calib_step(qr=%s) x%d at d=%d, N=%d" % (self.qr.__name__, n_steps, self.w.d, self.n_used)
+        if self.w.batch > 1:
+            s += ", one of the %d problems (time x%d)" % (self.w.batch, self.w.batch)
+        if self.extrapolated:
+            s += "; a prefix of the %d token rows, time scaled by the step's flop count (x%.2f)" % (
+                self.w.n_tokens, 1.0 / self.scale)
+        return s
 
 
 def run_reference(args, w):
+    """The reference arm: the oracle on the host cores, W untimed and K timed steps on the arm's workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    shrink = 4 if w.d >= 2048 else 1
-    total = max(1, args.steps + args.warmup)
-    v, dt, cores, sample = oracle_sample_steps_per_s(w, min(total, 3), shrink)
+    run = OracleRun(w)
+    K, W = max(1, args.steps), max(0, args.warmup)
+    if W:
+        run.time_steps(W)
+    sec = run.time_steps(K)
+    v = 1.0 / sec
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / v, "higher_is_better": True,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "d": w.d, "n_tokens": w.n_tokens, "batch": w.batch},
-            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "config": {"workload": w.name, "d": w.d, "n_tokens": w.n_tokens, "batch": w.batch, "lr": w.lr},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": run.cores, "kind": "oracle", "sample": run.sample(K),
+                             "extrapolated": run.extrapolated},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -157,27 +195,26 @@ def main():
         run_reference(args, w)
         return
 
+    from paper_2511_04063_b200 import replicas
+    if args.gpus > 1 and not replicas.launched_externally():
+        # no launcher gave this process a rank: start one process per GPU on this node and let rank 0 print
+        codes, _ = replicas.launch(args.gpus, [os.path.abspath(__file__)] + sys.argv[1:])
+        raise SystemExit(max(abs(c) for c in codes))
+
     import torch
     import paper_2511_04063_b200 as dq
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the calibration path has no CPU implementation")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    rank, local_rank, world = replicas.init_process_group("nccl")
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     # ---------------------------------------------------------------- inputs
     # every rank gets its own seeded problem (an independent rotation site)
-    from paper_2511_04063_b200 import replicas
     wr = replicas.workload_for_rank(w, rank)
     X_host = gen.gen_activations(wr)
     Z0_host = gen.gen_latent_init(wr)
@@ -361,7 +398,7 @@ def main():
                         "achieved": hb / t_fwd / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": hb / t_fwd / 1e9 / peaks["hbm_gbs"],
                         "peak_source": "%s (copy bandwidth)" % peaks["_source"],
-                        "traffic": 139.5e6 if wr.name == "c3_heads" else None,   # profiles/heads_whip_fused_c3_heads.md
+                        "traffic": NCU_TRAFFIC_BYTES_HEADS.get(wr.name),
                         "algorithmic_bytes_per_launch": hb}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -420,13 +457,14 @@ def main():
                                   "update_mma_tflops": 3 * 12.0 * d ** 3 * B / (cay["update_ms"] * 1e-3) / 1e12
                                   if cay["update_ms"] > 0 else None}
         if not args.no_cpu_baseline and world == 1:
-            shrink = 4 if d >= 2048 else 1
-            v, dt, cores, sample = oracle_sample_steps_per_s(w, 2 if shrink > 1 else 3, shrink)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+            run = OracleRun(w, max_flops=2.5e12)          # a bounded leg: about 10-30 s of host time
+            n_cpu = 3
+            sec = run.time_steps(n_cpu)
+            line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": run.cores, "kind": "oracle",
+                                    "sample": run.sample(n_cpu), "extrapolated": run.extrapolated}
         print(json.dumps(line), flush=True)
     dq.dq_calib_destroy(h)
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 if __name__ == "__main__":

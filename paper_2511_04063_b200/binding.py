@@ -247,6 +247,7 @@ def dq_rotate_apply(X, R, Y, stream=None):
     """Y = X R.  X, Y: CUDA [n, d] float32 or bfloat16 (same dtype); R: CUDA float32 [d, d]."""
     import torch
     assert X.is_cuda and R.is_cuda and Y.is_cuda and X.dtype == Y.dtype and R.dtype == torch.float32
+    assert X.stride(1) == 1 and Y.stride(1) == 1 and R.is_contiguous()
     n, d = X.shape
     _check(load_library().dq_rotate_apply(_ptr(X), DQ_FP32 if X.dtype == torch.float32 else DQ_BF16, n, d,
                                           X.stride(0), _ptr(R), _ptr(Y), Y.stride(0), _stream_ptr(stream)),
@@ -259,6 +260,7 @@ def dq_rotate_apply_static(X, R, Y, stream=None):
     import torch
     assert X.is_cuda and R.is_cuda and Y.is_cuda and R.dtype == torch.float32
     assert X.dtype == torch.bfloat16 and Y.dtype == torch.bfloat16
+    assert X.stride(1) == 1 and Y.stride(1) == 1 and R.is_contiguous()
     n, d = X.shape
     _check(load_library().dq_rotate_apply_static(_ptr(X), n, d, X.stride(0), _ptr(R), _ptr(Y), Y.stride(0),
                                                  _stream_ptr(stream)), "dq_rotate_apply_static")
@@ -280,6 +282,7 @@ def dq_eval_rotation(X, R, tau: float, bits: int, stream=None):
     X: CUDA [n, d] float32 or bfloat16; R: CUDA float32 [d, d].  Synchronises to read the result."""
     import torch
     assert X.is_cuda and R.is_cuda and R.dtype == torch.float32 and X.dim() == 2
+    assert X.stride(1) == 1 and R.is_contiguous()
     n, d = X.shape
     out = torch.zeros(2, dtype=torch.float64, device=X.device)
     _check(load_library().dq_eval_rotation(_ptr(X), DQ_FP32 if X.dtype == torch.float32 else DQ_BF16, n, d,

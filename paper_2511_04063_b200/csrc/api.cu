@@ -60,6 +60,7 @@ struct dq_calib {
   int64_t graph_launches = 0;
   double graph_flops = 0.0;
   bool graph_failed = false;
+  bool graph_needs_z_split = false;   // the captured step reads z_hi / z_lo without writing them first
   int eager_steps_done = 0;
 };
 
@@ -266,6 +267,9 @@ void try_capture(dq_calib* h) {
   const int64_t before = h->ctx.launches;
   const double flops_before = h->ctx.mma_flops;
   h->r_stale = true;
+  // With plain SGD the update kernel writes the split copy of the new latent, so a step captured while that
+  // copy is current holds no split_kernel: it may only be replayed while the copy is current.
+  h->graph_needs_z_split = h->fast_qr && h->qtc.z_split_fresh;
   if (cudaStreamBeginCapture(h->ctx.stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();
     h->graph_failed = true;
@@ -404,7 +408,8 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
     const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
     const bool use_graph = cayley ? (!h->timing && h->cay_started && h->eager_steps_done >= 1)
                                   : (!h->timing && h->r_stale && h->eager_steps_done >= 1 &&
-                                     (!iterative || warm));
+                                     (!iterative || warm) &&
+                                     (!h->graph || !h->graph_needs_z_split || h->qtc.z_split_fresh));
     if (use_graph && !h->graph && !h->graph_failed) try_capture(h);
     if (use_graph && h->graph) {
       DQ_CHECK_CUDA(cudaGraphLaunch(h->graph, ctx.stream));

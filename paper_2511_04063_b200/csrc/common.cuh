@@ -36,6 +36,20 @@ inline dq_status after_launch(Ctx& ctx) {
   return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
 }
 
+// Opt-in to more than 48 KB of dynamic shared memory.  The attribute belongs to the (function, device) pair,
+// so it is set once per device; one process may use the library on several devices.
+struct SmemOptIn { bool done[64] = {}; };
+template <typename Kernel>
+inline dq_status opt_in_dynamic_smem(Kernel kern, int bytes, SmemOptIn& table) {
+  int dev = -1;
+  DQ_CHECK_CUDA(cudaGetDevice(&dev));
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && table.done[dev]) return DQ_OK;
+  DQ_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  if (tracked) table.done[dev] = true;
+  return DQ_OK;
+}
+
 __device__ __forceinline__ void set_status(int* d_status, int code) {
   if (d_status) atomicCAS(d_status, 0, code);
 }

@@ -222,11 +222,8 @@ qr128_forward_kernel(const float* __restrict__ Z, float* __restrict__ R, float* 
 }  // namespace
 
 dq_status qr128_forward(Ctx& ctx, const float* Z, float* R, float* U, float* W, __nv_bfloat16* Rt_bf16, int batch) {
-  static bool attr = false;
-  if (!attr) {
-    DQ_CHECK_CUDA(cudaFuncSetAttribute(qr128_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM));
-    attr = true;
-  }
+  static SmemOptIn attr;
+  DQ_CHECK(opt_in_dynamic_smem(qr128_forward_kernel, FWD_SMEM, attr));
   qr128_forward_kernel<<<batch, NT, FWD_SMEM, ctx.stream>>>(Z, R, U, W, Rt_bf16, ctx.d_status);
   return after_launch(ctx);
 }

@@ -300,11 +300,8 @@ qr128_backward_sgd_tc_kernel(const float* __restrict__ R, const float* __restric
 
 dq_status qr128_forward_incremental(Ctx& ctx, const float* Z, float* R, float* U, float* W, __nv_bfloat16* Rt_bf16,
                                     int n_sweeps, int batch) {
-  static bool attr = false;
-  if (!attr) {
-    DQ_CHECK_CUDA(cudaFuncSetAttribute(qr128_forward_inc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM));
-    attr = true;
-  }
+  static SmemOptIn attr;
+  DQ_CHECK(opt_in_dynamic_smem(qr128_forward_inc_kernel, FWD_SMEM, attr));
   qr128_forward_inc_kernel<<<batch, NT, FWD_SMEM, ctx.stream>>>(Z, R, U, W, Rt_bf16, 4 * (n_sweeps < 1 ? 1 : n_sweeps), 1e-5f,
                                                                 ctx.d_status);
   return after_launch(ctx);
@@ -312,11 +309,8 @@ dq_status qr128_forward_incremental(Ctx& ctx, const float* Z, float* R, float* U
 
 dq_status qr128_backward_sgd_tc(Ctx& ctx, const float* R, const float* W, const float* Gq, float* Gz, float* Z,
                                 float lr, int batch) {
-  static bool attr = false;
-  if (!attr) {
-    DQ_CHECK_CUDA(cudaFuncSetAttribute(qr128_backward_sgd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD_SMEM));
-    attr = true;
-  }
+  static SmemOptIn attr;
+  DQ_CHECK(opt_in_dynamic_smem(qr128_backward_sgd_tc_kernel, BWD_SMEM, attr));
   qr128_backward_sgd_tc_kernel<<<batch, NT, BWD_SMEM, ctx.stream>>>(R, W, Gq, Gz, Z, lr, ctx.d_status);
   return after_launch(ctx);
 }

@@ -583,12 +583,9 @@ template <int NT>
 dq_status launch_panel(Ctx& ctx, int cs, int batch, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, bf16* y_lo,
                        float* Tk, int d, int c0) {
   using L = PanelSmem<NT / 32>;
-  static bool attr = false;
+  static SmemOptIn attr;
   auto kern = qr_panel_cm_kernel<NT>;
-  if (!attr) {
-    DQ_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES));
-    attr = true;
-  }
+  DQ_CHECK(opt_in_dynamic_smem(kern, L::BYTES, attr));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(cs, batch, 1);
   cfg.blockDim = dim3(NT, 1, 1);
@@ -615,9 +612,13 @@ dq_status qrp_panel(Ctx& ctx, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, b
   if (m <= 0 || m % OB != 0 || m > 8192) return DQ_ERR_UNSUPPORTED;
   // 512 rows per CTA (two rows per thread, 255 registers) in clusters of up to 8; beyond 4096 rows
   // either a cluster of 16 (non-portable size, if the device can co-schedule it) or 1024 rows per CTA.
-  static int can16 = -1;
-  if (m > 4096 && can16 < 0) {
-    can16 = 0;
+  static int can16_dev[64];                  // per device: 0 = not probed, 1 = no, 2 = yes
+  int dev = 0;
+  DQ_CHECK_CUDA(cudaGetDevice(&dev));
+  int can16_local = 0;
+  int& can16 = (dev >= 0 && dev < 64) ? can16_dev[dev] : can16_local;
+  if (m > 4096 && can16 == 0) {
+    can16 = 1;
     auto kern = qr_panel_cm_kernel<256>;
     using L = PanelSmem<8>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) == cudaSuccess &&
@@ -629,11 +630,11 @@ dq_status qrp_panel(Ctx& ctx, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, b
       at[0].val.clusterDim.x = 16; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
       cfg.attrs = at; cfg.numAttrs = 1;
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n >= 1) can16 = 1;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n >= 1) can16 = 2;
     }
     cudaGetLastError();
   }
-  const bool wide = m > 4096 && can16 != 1;
+  const bool wide = m > 4096 && can16 != 2;
   const int rows_per_cta = wide ? 1024 : 512;
   int cs = 1;
   while (cs * rows_per_cta < m) cs *= 2;
@@ -644,11 +645,8 @@ dq_status qrp_panel(Ctx& ctx, float* At, bf16* at_hi, bf16* at_lo, bf16* y_hi, b
 
 dq_status qrp_wy_w2(Ctx& ctx, const float* part, int ksplit, int m, int64_t part_bs, const float* Tk, bf16* w2_hi,
                     bf16* w2_lo, int64_t w2_bs, int n, int batch) {
-  static bool attr = false;
-  if (!attr) {
-    DQ_CHECK_CUDA(cudaFuncSetAttribute(wy_w2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WY_W2_SMEM));
-    attr = true;
-  }
+  static SmemOptIn attr;
+  DQ_CHECK(opt_in_dynamic_smem(wy_w2_kernel, WY_W2_SMEM, attr));
   wy_w2_kernel<<<dim3(n / W2_ROWS_PER_CTA, batch), 256, WY_W2_SMEM, ctx.stream>>>(part, ksplit, m, part_bs, Tk, w2_hi,
                                                                                  w2_lo, w2_bs);
   return after_launch(ctx);

@@ -243,11 +243,8 @@ dq_status tri_inverse_tc(Ctx& ctx, QrTcState& q, const float* U, int d, int batc
   DQ_CHECK_CUDA(cudaMemsetAsync(q.wt_hi, 0, bytes, ctx.stream));
   DQ_CHECK_CUDA(cudaMemsetAsync(q.wt_lo, 0, bytes, ctx.stream));
   const int smem = TRI_INV_SMEM;
-  static bool attr = false;
-  if (!attr) {
-    DQ_CHECK_CUDA(cudaFuncSetAttribute(tri_inv_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr = true;
-  }
+  static SmemOptIn attr;
+  DQ_CHECK(opt_in_dynamic_smem(tri_inv_diag128_kernel, smem, attr));
   tri_inv_diag128_kernel<<<dim3(d / DB, batch), TRI_INV_THREADS, smem, ctx.stream>>>(U, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, d);
   DQ_CHECK(after_launch(ctx));
   int s = DB, count = d / DB;

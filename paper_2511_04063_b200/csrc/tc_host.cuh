@@ -44,13 +44,9 @@ template <int BN, int NT, int EPI>
 dq_status launch_gemm(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& alo,
                       const CUtensorMap& blo, const tc::Params& p) {
   using L = tc::SmemLayout<BN, NT>;
-  static bool attr_set = false;
+  static SmemOptIn attr;
   auto kern = tc::tc_gemm_kernel<BN, NT, EPI>;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
-      return DQ_ERR_CUDA;
-    attr_set = true;
-  }
+  DQ_CHECK(opt_in_dynamic_smem(kern, L::TOTAL, attr));
   const int units = (p.tile_list ? p.n_list : p.m_blocks * p.n_blocks) * p.batch * p.ksplit;
   int grid = units < ctx.sm_count ? units : ctx.sm_count;
   if (grid < 1) return DQ_OK;
@@ -63,14 +59,10 @@ dq_status launch_gemm(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, cons
 template <int NT, int EPI>
 dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& alo,
                        const CUtensorMap& blo, const tc::Params& p) {
-  static bool attr_set = false;
+  static SmemOptIn attr;
   auto kern = tc2::tc_gemm2_kernel<NT, EPI>;
   constexpr int SMEM = tc2::PairSmem<NT>::TOTAL;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-      return DQ_ERR_CUDA;
-    attr_set = true;
-  }
+  DQ_CHECK(opt_in_dynamic_smem(kern, SMEM, attr));
   const int units = (p.tile_list ? p.n_list : p.m_blocks * p.n_blocks) * p.batch * p.ksplit;
   int pairs = units < ctx.sm_count / 2 ? units : ctx.sm_count / 2;
   if (pairs < 1) return DQ_OK;
@@ -111,6 +103,9 @@ inline void keep_pool_memory(int dev) {
 template <int EPI>
 inline dq_status rotate_tokens(Ctx& ctx, const void* X, int64_t n, int d, int64_t ldx, const bf16* rt, void* out,
                                int64_t ldo, int* d_status) {
+  // TMA needs 16-byte aligned bases and row strides; the epilogue stores 16 bytes at a time
+  if ((((uintptr_t)X | (uintptr_t)rt | (uintptr_t)out) & 15) || ldx % 8 != 0 || ldo % (EPI == tc::EPI_GEN ? 4 : 8) != 0)
+    return DQ_ERR_UNSUPPORTED;
   CUtensorMap ma, mb;
   tc::Params p{};
   p.batch = 1; p.ksplit = 1; p.k_blocks = d / tc::BLOCK_K;

@@ -227,6 +227,7 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
 dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t ldx, const float* d_R,
                           void* d_Y, int64_t ldy) {
   if (d % 128 != 0 || n % 128 != 0 || ldx % 8 != 0 || ldy % 8 != 0) return DQ_ERR_UNSUPPORTED;
+  if (((uintptr_t)d_X | (uintptr_t)d_Y) & 15) return DQ_ERR_UNSUPPORTED;   // 16-byte loads (TMA) and stores
   int sms = 0, dev = 0;
   DQ_CHECK_CUDA(cudaGetDevice(&dev));
   DQ_CHECK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
@@ -263,6 +264,7 @@ dq_status tc_rotate_apply_static(Ctx& ctx, const void* d_X, int64_t n, int d, in
                                  void* d_Y, int64_t ldy) {
   if (d > STATIC_MAX_D) return DQ_ERR_UNSUPPORTED;
   if (d % 128 != 0 || n % 128 != 0 || ldx % 8 != 0 || ldy % 8 != 0) return DQ_ERR_UNSUPPORTED;
+  if (((uintptr_t)d_X | (uintptr_t)d_Y) & 15) return DQ_ERR_UNSUPPORTED;   // 16-byte loads (TMA) and stores
   int dev = 0;
   DQ_CHECK_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= STATIC_MAX_DEVICES) return DQ_ERR_UNSUPPORTED;

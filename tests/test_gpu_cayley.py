@@ -9,7 +9,7 @@ import torch
 import oracle as orc
 import paper_2511_04063_b200 as dq
 from paper_2511_04063_b200 import inputs as gen
-from gpu_util import Calib, x_f64, sign_decider_from_gpu
+from gpu_util import Calib, x_f64, bf16_sign_decider
 
 pytestmark = pytest.mark.gpu
 
@@ -63,17 +63,17 @@ def test_cayley_update_every_stage(w, lr, beta, s):
             assert np.abs(R1[b] - upd["X_new"]).max() <= 2e-5
             # (ii) the whole iteration from the same rotation and momentum: loss and dL/dR carry the
             # bf16 rounding of R in the Whip contraction (see the QR-Orth parity test for the bounds)
-            row_norm = np.linalg.norm(X, axis=1)
-            dO = 8.0 * row_norm / np.sqrt(d) * 2.0 ** -9 + 1e-3
+            # the sign of dL/dO is the kernel's only where the rounding of R to bf16 moved o across the kink
+            stats = {}
             ref = orc.cayley_calib_step(X, R0[b], M0[b], lr, beta, s=s,
-                                        sign_decider=sign_decider_from_gpu(Gt[b].T, 2.0 * dO[:, None]))
+                                        sign_decider=bf16_sign_decider(X, R0[b], R0[b], Gt[b].T, stats))
             assert abs(loss[b] - ref["loss"]) <= LOSS_TOL_BF16 * ref["loss"]
             # dL/dR inherits e^-|o| dO from the bf16 rotation, with dO up to a few 1e-2 on outlier-heavy
             # tokens: up to 1e-1 relative once the rotation is no longer a Hadamard-like matrix
             rel_gq = np.linalg.norm(Gq[b] - ref["Gq"]) / np.linalg.norm(ref["Gq"])
             rel_m = np.linalg.norm(M1[b] - ref["M_new"]) / np.linalg.norm(ref["M_new"])
-            print("step %d problem %d: rel err dL/dR %.3e, M %.3e, max |dR| %.3e" %
-                  (step, b, rel_gq, rel_m, np.abs(R1[b] - ref["R_new"]).max()))
+            print("step %d problem %d: overridden %.4f%%, rel err dL/dR %.3e, M %.3e, max |dR| %.3e" %
+                  (step, b, 100 * stats["overridden"], rel_gq, rel_m, np.abs(R1[b] - ref["R_new"]).max()))
             assert rel_gq <= 1e-1 and rel_m <= 1e-1
             # the update is (to first order) alpha M_new, so its error is the relative error of M_new
             # times the step; the 1e-3 per-step bound on the rotation is meaningful for steps up to 1e-2

@@ -9,7 +9,7 @@ import oracle as orc
 from oracle import objectives as obj
 import paper_2511_04063_b200 as dq
 from paper_2511_04063_b200 import inputs as gen
-from gpu_util import Calib, x_f64
+from gpu_util import Calib, x_f64, bf16_round
 
 pytestmark = pytest.mark.gpu
 
@@ -54,17 +54,32 @@ def test_objective_step_against_oracle(w, name):
     loss_tol = 1e-4 if fp32 else 2e-2
     g_tol = {"variance": 1e-5, "kurtosis": 1e-4, "quant": 1e-3} if fp32 else \
             {"variance": 2e-2, "kurtosis": 5e-2, "quant": 1.5e-1}
-    band = 1e-4 if fp32 else 0.25     # distance (in codes) to a rounding boundary within which the kernel decides
+    R_gpu = c.buf(dq.DQ_BUF_R).cpu().numpy().astype(np.float64)
     for b in range(batch):
         X = x_f64(w, c.X_host, b)
+        # Distance (in codes) to a rounding boundary within which the kernel decides the code: what the
+        # kernel's own arithmetic moved o / scale by.  fp32 path: fp32 rounding, 1e-4 codes.  Tensor-core path:
+        # the rounding of R to bf16 moves o by dO = x (bf16(R) - R) and with it the token's min / max, i.e.
+        # the grid; the band is |(o + dO) / scale' - o / scale| per entry, from the oracle's grid of O + dO.
+        band = 1e-4
+        if not fp32 and name == "quant":
+            R_ref, _ = orc.qr_pos_lapack(Z0[b])
+            O_ref = orc.rotate(X, R_ref)
+            O_b = O_ref + orc.rotate(X, bf16_round(R_gpu[b]) - R_ref)
+            s_ref, _, _ = obj.quant_grid(O_ref, bits)
+            s_b, _, _ = obj.quant_grid(O_b, bits)
+            band = np.abs(O_b / np.where(s_b == 0.0, 1.0, s_b) - O_ref / np.where(s_ref == 0.0, 1.0, s_ref)) + 1e-3
+        stats = {}
 
-        def decider(O, scale, zero, codes, Gb=G[b]):
+        def decider(O, scale, zero, codes, Gb=G[b], band=band, stats=stats):
             # the kernel's code, recovered from its stored derivative: g = (2/d)(o - scale (q - zero))
             safe = np.where(scale == 0.0, 1.0, scale)
             q_gpu = np.clip(np.rint(zero + (O - Gb * d / 2.0) / safe), 0, 2 ** bits - 1)
             near = np.abs(np.abs(O / safe - np.rint(O / safe)) - 0.5) <= band
             assert np.array_equal(q_gpu[~near], codes[~near]), "codes differ away from a rounding boundary"
             assert np.abs(q_gpu - codes).max() <= 1.0
+            stats["overridden"] = float(near.mean())
+            stats["changed"] = float((q_gpu != codes).mean())
             return np.where(near, q_gpu, codes)
 
         ref = obj.objective_step(X, Z0[b], w.lr, name, bits=bits, qr=orc.qr_pos_lapack,
@@ -76,8 +91,14 @@ def test_objective_step_against_oracle(w, name):
         rel_gq = np.linalg.norm(Gq[b] - ref["Gq"]) / np.linalg.norm(ref["Gq"])
         R1, _ = orc.qr_pos_lapack(Z1[b])
         R1_ref, _ = orc.qr_pos_lapack(ref["Z_new"])
-        print("%s %s b%d: loss %.6g (ref %.6g) rel dL/dO %.2e dL/dR %.2e max dR %.2e" %
-              (w.name, name, b, loss[b], ref["loss"], rel_g, rel_gq, np.abs(R1 - R1_ref).max()))
+        print("%s %s b%d: loss %.6g (ref %.6g) rel dL/dO %.2e dL/dR %.2e max dR %.2e%s" %
+              (w.name, name, b, loss[b], ref["loss"], rel_g, rel_gq, np.abs(R1 - R1_ref).max(),
+               "" if not stats else ", codes overridden %.3f%% (really differ %.3f%%)" %
+               (100 * stats["overridden"], 100 * stats["changed"])))
+        if stats:
+            # at most a few percent of the entries sit that close to a rounding boundary (the band is a few
+            # hundredths of a code on the heavy-tailed rows, whose range / 15 is the grid step)
+            assert stats["overridden"] <= (1e-3 if fp32 else 8e-2), stats
         assert rel_g <= g_tol[name]
         assert rel_gq <= 2.0 * g_tol[name]
         assert np.abs(R1 - R1_ref).max() <= 1e-3

@@ -8,7 +8,8 @@ import torch
 import oracle as orc
 import paper_2511_04063_b200 as dq
 from paper_2511_04063_b200 import inputs as gen
-from gpu_util import Calib, x_f64, sign_decider_from_gpu
+from gpu_util import (Calib, x_f64, bf16_round, bf16_step_reference, check_bf16_gradients, perturbed_latent,
+                      MAX_OVERRIDDEN)
 
 pytestmark = pytest.mark.gpu
 
@@ -20,18 +21,28 @@ def small(name, **kw):
     return gen.scaled(gen.WORKLOADS[name], **kw)
 
 
+# (workload, perturbed): the random Hadamard initialisation is +-1/sqrt(d), which bf16 holds exactly when d
+# is a power of four and rounds uniformly otherwise, so no sign of dL/dO can flip from it; the perturbed
+# variants start from a latent a few SGD steps away, whose rotation bf16 really rounds.
 CASES = [
-    small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3),
-    small("c4_13b", d=640, n_tokens=512, batch=2, n_outlier_channels=4),    # 128-wide N tiles, 2 problems
-    small("c3_heads", d=128, n_tokens=2048, batch=4),                       # per-head rotations
-    small("c5_70b", d=512, n_tokens=4096, n_outlier_channels=2),            # token scales, several waves
-    small("c4_13b", d=2560, n_tokens=2048, n_outlier_channels=6),           # 200 Gq tiles on 148 SMs: split tail wave
+    (small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3), False),
+    (small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3), True),
+    (small("c4_13b", d=640, n_tokens=512, batch=2, n_outlier_channels=4), False),   # 128-wide N tiles, 2 problems
+    (small("c3_heads", d=128, n_tokens=2048, batch=4), False),                      # per-head rotations
+    (small("c3_heads", d=128, n_tokens=2048, batch=4), True),
+    (small("c5_70b", d=512, n_tokens=4096, n_outlier_channels=2), False),           # token scales, several waves
+    (small("c5_70b", d=512, n_tokens=4096, n_outlier_channels=2), True),
+    (small("c4_13b", d=2560, n_tokens=2048, n_outlier_channels=6), False),          # 200 Gq tiles on 148 SMs: split tail wave
 ]
 
 
-@pytest.mark.parametrize("w", CASES, ids=lambda w: "%s-d%d-n%d-b%d" % (w.name, w.d, w.n_tokens, w.batch))
-def test_tensor_core_step_every_stage(w):
+@pytest.mark.parametrize("w,perturbed", CASES,
+                         ids=lambda v: ("%s-d%d-n%d-b%d" % (v.name, v.d, v.n_tokens, v.batch)) if hasattr(v, "name")
+                         else ("perturbed" if v else "init"))
+def test_tensor_core_step_every_stage(w, perturbed):
     c = Calib(w)
+    if perturbed:
+        c.set_latent(perturbed_latent(w, c.Z0_host, w.seed))
     Z0 = c.latent()
     loss = c.step(1)[0]
     assert c.status() == dq.DQ_OK
@@ -43,31 +54,34 @@ def test_tensor_core_step_every_stage(w):
     Z1 = c.latent().astype(np.float64)
     for b in range(batch):
         X = x_f64(w, c.X_host, b)
-        # R is rounded to bf16 (2^-9 relative): |dO| <~ ||x_t|| 2^-9 / sqrt(d) * few.  Within that
-        # band of the kink of Eq. 4 the sign decision is the kernel's.
-        row_norm = np.linalg.norm(X, axis=1)
-        dO = 8.0 * row_norm / np.sqrt(d) * 2.0 ** -9 + 1e-3
-        ref = orc.calib_step(X, Z0[b], w.lr, sign_decider=sign_decider_from_gpu(Gt[b].T, 2.0 * dO[:, None]),
-                             qr=orc.qr_pos if d <= 1024 else orc.qr_pos_lapack)
+        # The sign of dL/dO is the kernel's only where the rounding of R to bf16 moved the rotated value
+        # across (or onto) the kink of Eq. 4; the fraction of such entries is bounded and printed.
+        st = bf16_step_reference(X, Z0[b], w.lr, R[b], Gt[b].T, qr=orc.qr_pos if d <= 1024 else orc.qr_pos_lapack)
+        ref = st["ref"]
+        tag = "%s d=%d %s[%d]" % (w.name, d, "perturbed" if perturbed else "init", b)
+        assert st["overridden"] <= MAX_OVERRIDDEN, (tag, st["overridden"])
         assert abs(loss[b] - ref["loss"]) <= LOSS_TOL_BF16 * ref["loss"]
         assert np.abs(R[b] - ref["R"]).max() <= 2e-5
-        # dL/dO (no 1/N), stored channel-major; compare where |O| is clear of the kink at 0.
+        # dL/dO (no 1/N), stored channel-major, away from the kink: the kernel's o differs from the oracle's
+        # by at most the band, so e^-|o| by the factor e^band; bf16 storage adds 2^-9 relative
         G_ref = ref["G"] * n
-        clear = np.abs(ref["O"]) > 2.0 * dO[:, None]
+        dOb = np.abs(orc.rotate(X, bf16_round(R[b]) - ref["R"])) + 4e-6 * np.linalg.norm(X, axis=1)[:, None]
+        e = np.exp(-np.abs(ref["O"]))
         err = np.abs(Gt[b].T - G_ref)
-        bound = np.exp(-np.abs(ref["O"])) * (np.exp(dO)[:, None] - 1.0) + 2.0 ** -8
-        assert (err[clear] <= bound[clear]).all()
-        assert clear.mean() > 0.5
-        # Gq inherits the relative error of dL/dO: e^-|o| dO with dO up to a few 1e-2 on the
-        # outlier-heavy tokens (bf16 R), plus 2^-9 from storing dL/dO in bf16: 5e-2 overall.
-        assert np.abs(Gq[b] - ref["Gq"]).max() <= 5e-2 * np.abs(ref["Gq"]).max()
-        rel_f = np.linalg.norm(Gq[b] - ref["Gq"]) / np.linalg.norm(ref["Gq"])
-        assert rel_f <= 5e-2
-        assert np.linalg.norm(Gz[b] - ref["Gz"]) <= 6e-2 * np.linalg.norm(ref["Gz"])
-        # one teacher-forced step: rotation of the updated latent
+        bound = e * (np.expm1(dOb) + 2.0 ** -8) + 1e-30
+        clear = ~st["near"]
+        assert (err[clear] <= bound[clear]).all(), (tag, (err[clear] / bound[clear]).max())
+        rows = check_bf16_gradients(tag, Gq[b], Gz[b], Z1[b], Z0[b].astype(np.float64), w.lr, st)
+        # one teacher-forced step: rotation of the updated latent.  Its deviation is the update's deviation
+        # (bounded above relative to the step); in the max norm it stays inside the contract's 1e-3 or, for
+        # the large steps of the small cases (few tokens, lr 1e-2), 5 % of the distance the rotation moved.
         R1, _ = orc.qr_pos_lapack(Z1[b])
         R1_ref, _ = orc.qr_pos_lapack(ref["Z_new"])
-        assert np.abs(R1 - R1_ref).max() <= R_TOL
+        R1_free, _ = orc.qr_pos_lapack(st["free"]["Z_new"])
+        moved = np.abs(R1_ref - ref["R"]).max()
+        print("%s: max|R_next - ref| hooked %.2e, hook-free %.2e, rotation moved %.2e" %
+              (tag, np.abs(R1 - R1_ref).max(), np.abs(R1 - R1_free).max(), moved))
+        assert np.abs(R1 - R1_ref).max() <= max(R_TOL, 5e-2 * moved)
     Rn = c.rotation()
     for b in range(batch):
         assert np.abs(Rn[b].T @ Rn[b] - np.eye(d)).max() <= ORTHO_TOL
@@ -261,13 +275,13 @@ def test_fused_per_head_kernel_with_and_without_stored_gradient(batch, n):
     loss0 = c.step(1)[0]
     Gq0 = c.buf(dq.DQ_BUF_GQ).cpu().numpy().astype(np.float64)
     Gt = c.buf(dq.DQ_BUF_G, dtype=torch.bfloat16, shape=(batch, 128, n)).float().cpu().numpy().astype(np.float64)
+    R0 = c.buf(dq.DQ_BUF_R).cpu().numpy().astype(np.float64)
     for b in sorted({0, batch // 2, batch - 1}):
         X = x_f64(w, c.X_host, b)
-        dO = 8.0 * np.linalg.norm(X, axis=1) / np.sqrt(128) * 2.0 ** -9 + 1e-3
-        ref = orc.calib_step(X, c.Z0_host[b], w.lr, sign_decider=sign_decider_from_gpu(Gt[b].T, 2.0 * dO[:, None]),
-                             qr=orc.qr_pos_lapack)
-        assert abs(loss0[b] - ref["loss"]) <= LOSS_TOL_BF16 * ref["loss"]
-        assert np.linalg.norm(Gq0[b] - ref["Gq"]) <= 5e-2 * np.linalg.norm(ref["Gq"])
+        st = bf16_step_reference(X, c.Z0_host[b], w.lr, R0[b], Gt[b].T, extended=False)
+        assert st["overridden"] <= MAX_OVERRIDDEN
+        assert abs(loss0[b] - st["ref"]["loss"]) <= LOSS_TOL_BF16 * st["ref"]["loss"]
+        assert np.linalg.norm(Gq0[b] - st["ref"]["Gq"]) <= 5e-2 * np.linalg.norm(st["ref"]["Gq"])
     c.close()
 
 
@@ -312,3 +326,49 @@ def test_failed_step_freezes_the_latent_on_the_other_incremental_kernels(name, d
         cond = np.linalg.cond(Z1[b].astype(np.float64))
         assert np.abs(R[b] - Rr).max() <= 5e-5 * max(1.0, cond)
     c.close()
+
+
+def test_replayed_graph_after_set_latent_factors_the_new_latent():
+    """Householder at every step, plain SGD: the captured step relies on the update kernel having written
+    the split-bf16 copy of the latent.  A latent installed by the caller has no such copy yet, so the next
+    step may not be replayed from that graph; the rotation it uses must be the factor of the NEW latent."""
+    d = 256
+    w = small("c2_7b", d=d, n_tokens=1024, n_outlier_channels=3)
+    c = Calib(w)
+    dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_HOUSEHOLDER, 0)
+    c.step(3)                                         # eager, then captured and replayed
+    assert c.status() == dq.DQ_OK
+    Zp = _near_orthogonal(d, 1, 0.05, 21)
+    c.set_latent(Zp)
+    loss = c.step(1)[0, 0]
+    assert c.status() == dq.DQ_OK
+    R = c.buf(dq.DQ_BUF_R).cpu().numpy()[0].astype(np.float64)
+    Rr, _ = orc.qr_pos_lapack(Zp[0])
+    assert np.abs(R - Rr).max() <= R_TOL
+    assert np.abs(R.T @ R - np.eye(d)).max() <= ORTHO_TOL
+    ref_loss = orc.whip_loss(orc.rotate(x_f64(w, c.X_host), Rr))
+    assert abs(loss - ref_loss) <= LOSS_TOL_BF16 * ref_loss
+    c.step(2)                                         # replayed again from here on
+    Z = c.latent()[0]
+    Rn = c.rotation()[0]
+    assert np.abs(Rn - orc.qr_pos_lapack(Z)[0]).max() <= 5e-5
+    c.close()
+
+
+def test_rotate_apply_rejects_misaligned_pointers_before_any_launch():
+    """The tensor-core rotation loads through TMA and stores 16 bytes at a time: a base address that is not
+    16-byte aligned is refused on the host (nothing is launched)."""
+    import ctypes as C
+    lib = dq.load_library()
+    n, d = 256, 256
+    X = torch.zeros((n + 1, d), dtype=torch.bfloat16, device="cuda")
+    Y = torch.zeros((n + 1, d), dtype=torch.bfloat16, device="cuda")
+    R = torch.eye(d, dtype=torch.float32, device="cuda")
+    for entry, args in (("dq_rotate_apply", lambda x, y: (x, dq.DQ_BF16, n, d, d, R.data_ptr(), y, d, None)),
+                        ("dq_rotate_apply_static", lambda x, y: (x, n, d, d, R.data_ptr(), y, d, None))):
+        f = getattr(lib, entry)
+        assert f(*args(X.data_ptr(), Y.data_ptr() + 2)) == dq.DQ_ERR_UNSUPPORTED, entry
+        assert f(*args(X.data_ptr() + 2, Y.data_ptr())) == dq.DQ_ERR_UNSUPPORTED, entry
+        assert f(*args(X.data_ptr(), Y.data_ptr())) == dq.DQ_OK, entry
+    torch.cuda.synchronize()
+    assert float(Y.float().abs().max()) == 0.0

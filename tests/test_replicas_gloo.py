@@ -39,3 +39,28 @@ def test_single_process_is_identity():
     assert replicas.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     w = gen.WORKLOADS["c1_tiny"]
     assert replicas.workload_for_rank(w, 0) == w and replicas.workload_for_rank(w, 3).seed == w.seed + 3
+
+
+def test_launch_starts_every_rank_and_rank0_prints_the_reduced_line(tmp_path):
+    """What `bench.py --gpus 2` does without an external launcher: replicas.launch starts the ranks
+    (RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* in their environment), each joins the group, and the
+    line rank 0 prints carries n_gpus = 2 and the rate over the slowest rank's time."""
+    import json
+    import sys
+    stub = os.path.join(os.path.dirname(os.path.abspath(__file__)), "replica_stub.py")
+    codes, text = replicas.launch(2, [stub, str(tmp_path)], timeout=300, capture_rank0=True)
+    assert codes == [0, 0]
+    line = json.loads(text.strip().splitlines()[-1])
+    assert line["n_gpus"] == 2 and line["scaling"] == "weak"
+    assert abs(line["value"] - 2 * 20 / 0.015) < 1e-6 and abs(line["ms_per_step"] - 0.75) < 1e-12
+    seen = [json.load(open(tmp_path / ("rank%d.json" % r))) for r in range(2)]
+    assert [s["rank"] for s in seen] == [0, 1] and [s["local_rank"] for s in seen] == [0, 1]
+    assert all(s["world"] == 2 for s in seen)
+    assert seen[0]["line"]["value"] == seen[1]["line"]["value"]      # the reduction reached both ranks
+    assert seen[0]["line"]["seed"] != seen[1]["line"]["seed"]        # independent rotation sites
+
+
+def test_launch_reports_a_failing_rank(tmp_path):
+    codes, _ = replicas.launch(2, ["-c", "import os, sys; sys.exit(3 if os.environ['RANK'] == '1' else 0)"], timeout=60)
+    assert codes == [0, 3]
+    assert not replicas.launched_externally() or "WORLD_SIZE" in os.environ

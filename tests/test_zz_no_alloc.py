@@ -1,8 +1,10 @@
 """dq_rotate_apply_static: the rotation Y = X R for callers that cannot allocate device memory
 (all of HBM already belongs to their own arena, or a cudaFree-induced device synchronisation is
 not acceptable on their path).  Its scratch is a fixed array inside the library, so the check is
-simply that it gives what dq_rotate_apply gives -- on two calls in a row with different rotations,
-because the array keeps the previous call's contents and a stale read would show up on the second.
+that it gives exactly what dq_rotate_apply gives (and what the float64 oracle gives, within bf16
+rounding) -- on calls in a row with different rotations and sizes, because the array keeps the
+previous call's contents and a stale read would show up on the later ones -- and that it takes no
+device memory.
 
 Collected last on purpose (file name): a run that stops at the first failure has then already
 run every other test."""
@@ -12,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle as orc
 import paper_2511_04063_b200 as dq
 from paper_2511_04063_b200 import inputs as gen
 
@@ -25,10 +28,12 @@ def _orthogonal(d, seed):
 
 def test_static_scratch_rotation_matches_allocating_entry_point_twice_in_a_row():
     n = 512
-    for call, (d, seed) in enumerate([(640, 11), (256, 12)]):      # second call uses a smaller part of the array
-        X = torch.from_numpy(gen.f32_to_bf16_bits(
-            np.random.default_rng(seed).standard_normal((n, d)).astype(np.float32)).view(np.int16)).cuda().view(torch.bfloat16)
-        R = torch.from_numpy(_orthogonal(d, seed)).cuda()
+    # the second call uses a smaller part of the array than the first, the third all of it (d = 2048)
+    for call, (d, seed) in enumerate([(640, 11), (256, 12), (2048, 13)]):
+        Xb = gen.f32_to_bf16_bits(np.random.default_rng(seed).standard_normal((n, d)).astype(np.float32))
+        X = torch.from_numpy(Xb.view(np.int16)).cuda().view(torch.bfloat16)
+        Rh = _orthogonal(d, seed)
+        R = torch.from_numpy(Rh).cuda()
         Y_ref = torch.empty((n, d), dtype=torch.bfloat16, device="cuda")
         Y_new = torch.full((n, d), float("nan"), dtype=torch.bfloat16, device="cuda")
         dq.dq_rotate_apply(X, R, Y_ref)
@@ -36,9 +41,30 @@ def test_static_scratch_rotation_matches_allocating_entry_point_twice_in_a_row()
         torch.cuda.synchronize()
         a, b = Y_ref.float().cpu().numpy(), Y_new.float().cpu().numpy()
         assert np.isfinite(b).all(), call
-        # same tolerance as the bf16 rotate_apply parity test (bf16 operands and output)
-        assert np.abs(a - b).max() <= 6e-2, call
-        assert np.linalg.norm(a - b) <= 1e-2 * np.linalg.norm(a), call
+        # both entry points run the same kernels on the same operands: the outputs are identical
+        assert np.array_equal(a, b), call
+        # and both are the rotation: against the float64 oracle, with the tolerance of the bf16 rotate_apply
+        # parity test (bf16 operand R and bf16 output, 2^-9 each)
+        ref = orc.rotate(gen.bf16_bits_to_f32(Xb).reshape(n, d), Rh)
+        assert np.abs(b - ref).max() <= 6e-2, call
+        assert np.linalg.norm(b - ref) <= 1e-2 * np.linalg.norm(ref), call
+
+
+def test_static_scratch_rotation_takes_no_device_memory():
+    """After one warm-up call (the first call on a device resolves the array's address and may load the
+    library's kernels), further calls leave the amount of free device memory unchanged."""
+    n, d = 256, 512
+    X = torch.zeros((n, d), dtype=torch.bfloat16, device="cuda")
+    Y = torch.empty((n, d), dtype=torch.bfloat16, device="cuda")
+    R = torch.eye(d, dtype=torch.float32, device="cuda")
+    dq.dq_rotate_apply_static(X, R, Y)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(20):
+        dq.dq_rotate_apply_static(X, R, Y)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
 
 
 def test_static_scratch_rotation_rejects_sizes_beyond_its_array():
