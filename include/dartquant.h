@@ -150,19 +150,23 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
  * give the same unique factors (diag(U) > 0).
  *   DQ_QR_ITERATIVE (default): incremental.  Blocked Householder QR (Algorithm 2 in compact-WY
  *     form) only when no factors of a nearby latent are known (first step, after
- *     dq_calib_set_latent or a change of method).  Afterwards, with the previous step's U_old,
- *     Zh = Z U_old^-1 is close to orthogonal whatever Z is, its upper factor I + T is the fixed point
- *     of T <- striu(E - T^T T) + diag(E - T^T T) / 2 with E = Zh^T Zh - I, reached from T = 0 by
- *     sweeps of triangular tensor-core GEMMs (no dependent column steps), and U = (I + T) U_old.
- *     The sweeps stop by themselves: up to n_iters sweeps with a plain bf16 product, each skipped (by
- *     a device-side flag, so the launch sequence and a captured graph stay fixed) once the sweep
- *     before it moved no entry by more than 1e-5, then up to three sweeps with the split-bf16
- *     product.  If the last of those still moved an entry, one optimiser step has moved the latent
- *     too far: the status word becomes DQ_ERR_NOT_CONVERGED and, as after every device-side error,
- *     the update kernels leave the latent and the optimiser state untouched from then on: the
- *     latent stays at the last good iterate.  Recover with
- *     dq_calib_set_qr_method(h, DQ_QR_HOUSEHOLDER, 0) (or a lower learning rate) and step again.
- *     n_iters <= 0 selects the default (12); at most 64.
+ *     dq_calib_set_latent or a change of method).  Afterwards, with the previous step's W_old = U_old^-1,
+ *     Zh = Z W_old is close to orthogonal whatever Z is, its upper factor I + T is the fixed point
+ *     of T <- striu(E - T^T T) + diag(E - T^T T) / 2 with E = Zh^T Zh - I, reached by sweeps of
+ *     triangular tensor-core GEMMs (no dependent column steps) that start from the previous step's
+ *     T^T T, and R = Zh (I + T)^-1, W = W_old (I + T)^-1 (the inverse of I + T from a few more triangular
+ *     products; U itself is not formed).  The sweeps stop by themselves: each is skipped (by a
+ *     device-side flag, so the launch sequence and a captured graph stay fixed) once the sweep before it
+ *     moved no entry by more than 1e-5; the first two use a plain bf16 product, later ones and, after
+ *     a step large enough to need them, the first-order correction products use split-bf16 operands.
+ *     At most n_iters + 3 sweeps.  If the last of those still moved an entry, one optimiser step has
+ *     moved the latent too far: the status word becomes DQ_ERR_NOT_CONVERGED and, as after every
+ *     device-side error, the update kernels leave the latent and the optimiser state untouched from
+ *     then on: the latent stays at the last good iterate.  Recover with
+ *     dq_calib_set_qr_method(h, DQ_QR_HOUSEHOLDER, 0), more sweeps or a lower learning rate, and step
+ *     again.  n_iters <= 0 selects the default (5 on this route: the paper's SGD steps need one
+ *     sweep; an optimiser that moves every entry by its learning rate, such as Adam, may need more);
+ *     at most 64.
  *   DQ_QR_HOUSEHOLDER: blocked Householder QR at every step; no assumption on the step size.
  * The call clears the status word.  For d == 128 (any path) the same two methods exist as kernels that
  * keep a whole latent in shared memory; there the sweeps stop as soon as no entry moves (one more is
@@ -192,6 +196,12 @@ dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters)
 dq_status dq_calib_run_epochs(dq_calib_t* h, const void* d_pool, int64_t n_pool, int64_t ld_pool,
                               float sample_ratio, int32_t accum, int32_t n_epochs, uint64_t seed,
                               float* d_loss_out, int64_t* h_steps_out);
+
+/* Arithmetic of the QR-Orth backward (Sec. 4.3: dL/dZ from dL/dR, Z = R U) on the tensor-core path for
+ * d >= 256.  dL/dR carries the bf16 rounding of the rotation operand and of dL/dO (a few percent), so by
+ * default (split = 0) its d x d products run on plain bf16 operands with fp32 accumulation (2^-9 relative);
+ * split != 0 runs them on split-bf16 operands (three MMAs per product, about 2^-17).  No effect elsewhere. */
+dq_status dq_calib_set_backward_precision(dq_calib_t* h, int32_t split);
 
 /* The calibration objective.  DQ_OBJ_WHIP (default) is Eq. 4.  The other three are the objectives the
  * ablation of Sec. 5.3 compares it with; the paper names them without formulas, so they are read as
@@ -239,6 +249,16 @@ dq_status dq_calib_set_latent(dq_calib_t* h, const float* d_Z);
 /* Synchronises the stream and returns the device status word
  * (DQ_OK / DQ_ERR_SINGULAR / DQ_ERR_NONFINITE / DQ_ERR_TIMEOUT / DQ_ERR_NOT_CONVERGED) or DQ_ERR_CUDA. */
 dq_status dq_calib_status(dq_calib_t* h);
+
+/* Failure detection self-test (no counterpart in the paper).  Every wait inside the tensor-core kernels (on
+ * a TMA copy, an MMA, the other CTA of a pair) is bounded: when it runs out the kernel records
+ * DQ_ERR_TIMEOUT in the status word and returns normally, and from then on the update kernels leave the
+ * latent untouched.  This call runs that same wait, with a limit of limit_ns nanoseconds (1 .. 1e8), in a
+ * one-thread kernel on a barrier that nothing ever arrives at, with no copy or MMA in flight.  Afterwards
+ * dq_calib_status returns DQ_ERR_TIMEOUT and steps leave the latent unchanged until dq_calib_set_latent (or a
+ * dq_calib_set_* call) clears the status.  d_waited_ns (nullable, device) receives the time waited.
+ * Tensor-core path only (DQ_ERR_UNSUPPORTED otherwise). */
+dq_status dq_calib_selftest_bounded_wait(dq_calib_t* h, uint64_t limit_ns, uint64_t* d_waited_ns);
 
 /* Phase times of the most recent dq_calib_step call, averaged per step, in ms
  * (synchronises).  Order: DQ_PHASE_*.  Writes min(n, DQ_PHASE_COUNT) entries

@@ -31,6 +31,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
     "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens", "dq_eval_rotation",
     "dq_calib_set_orth_method", "dq_calib_set_objective", "dq_calib_run_epochs", "dq_calib_mma_flops", "dq_calib_set_keep_gradient",
+    "dq_calib_set_backward_precision", "dq_calib_selftest_bounded_wait",
 )
 
 
@@ -88,6 +89,10 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_debug_buffer.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i64)]
     lib.dq_calib_set_keep_gradient.argtypes = [vp, i32]
     lib.dq_calib_set_keep_gradient.restype = i32
+    lib.dq_calib_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp]
+    lib.dq_calib_selftest_bounded_wait.restype = i32
+    lib.dq_calib_set_backward_precision.argtypes = [vp, i32]
+    lib.dq_calib_set_backward_precision.restype = i32
     lib.dq_calib_launch_count.argtypes = [vp]
     lib.dq_calib_mma_flops.argtypes = [vp]
     lib.dq_calib_mma_flops.restype = C.c_double
@@ -192,6 +197,20 @@ def dq_calib_run_epochs(h, pool, sample_ratio: float, accum: int, n_epochs: int,
 
 def dq_calib_set_keep_gradient(h, keep: bool = True):
     _check(load_library().dq_calib_set_keep_gradient(h, 1 if keep else 0), "dq_calib_set_keep_gradient")
+
+
+def dq_calib_set_backward_precision(h, split: bool):
+    """QR-Orth backward on split-bf16 operands (True) or plain bf16 operands (False, the default)."""
+    _check(load_library().dq_calib_set_backward_precision(h, 1 if split else 0), "dq_calib_set_backward_precision")
+
+
+def dq_calib_selftest_bounded_wait(h, limit_ns: int) -> int:
+    """Runs the library's bounded in-kernel wait on a barrier nothing arrives at; returns the nanoseconds it
+    waited before giving up (synchronises).  Leaves DQ_ERR_TIMEOUT in the handle's status word."""
+    import torch
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    _check(load_library().dq_calib_selftest_bounded_wait(h, limit_ns, waited.data_ptr()), "dq_calib_selftest_bounded_wait")
+    return int(waited.cpu()[0])
 
 
 def dq_calib_mma_flops(h) -> float:

@@ -13,6 +13,10 @@
 
 using namespace dq;
 
+// Default number of sweeps (beyond the three that always exist) of the incremental QR-Orth on the tensor-core
+// route for d >= 256, whose fixed point starts from the previous step's T^T T and so needs few.
+constexpr int DEFAULT_QR_SWEEPS_TC = 5;
+
 struct dq_calib {
   dq_calib_config cfg;
   Ctx ctx;                      // ctx.stream is the internal work stream
@@ -37,6 +41,7 @@ struct dq_calib {
   QrTcState qtc;                // tensor-core QR-Orth operand copies
   bool fast_qr = false;
   int qr_method = DQ_QR_ITERATIVE, qr_iters = 12;
+  bool qr_iters_default = true;  // n_iters was not given: the large tensor-core route then uses DEFAULT_QR_SWEEPS_TC
   int optimizer = DQ_SGD;
   float beta1 = 0.f, beta2 = 0.f, eps = 0.f;
   float* opt_m = nullptr;       // first moment / velocity
@@ -55,12 +60,16 @@ struct dq_calib {
   cudaEvent_t ev[DQ_PHASE_COUNT + 1] = {};
   double ms_acc[DQ_PHASE_COUNT] = {};
   int timed_steps = 0;
-  // one whole step (QR forward .. update) captured once and replayed
-  cudaGraphExec_t graph = nullptr;
-  int64_t graph_launches = 0;
-  double graph_flops = 0.0;
-  bool graph_failed = false;
-  bool graph_needs_z_split = false;   // the captured step reads z_hi / z_lo without writing them first
+  bool bwd_split = false;       // tensor-core QR-Orth backward with split-bf16 operands (three MMAs per product)
+  // One whole step (QR forward .. update) captured once and replayed.  The incremental QR-Orth alternates
+  // between two sets of copies of U^-1, so there is one captured step per set (index = set read by the step).
+  struct StepGraph {
+    cudaGraphExec_t exec = nullptr;
+    int64_t launches = 0;
+    double flops = 0.0;
+    bool failed = false;
+    bool needs_z_split = false;   // the captured step reads z_hi / z_lo without writing them first
+  } graph[2];
   int eager_steps_done = 0;
 };
 
@@ -75,7 +84,7 @@ dq_status dev_alloc(T** p, int64_t n) {
 
 void free_all(dq_calib* h) {
   if (!h) return;
-  if (h->graph) cudaGraphExecDestroy(h->graph);
+  for (auto& g : h->graph) if (g.exec) cudaGraphExecDestroy(g.exec);
   tc_destroy(h->tc);
   qr_tc_destroy(h->qtc);
   cayley_destroy(h->cay);
@@ -142,7 +151,8 @@ dq_status ensure_rotation(dq_calib* h) {
     }
   } else if (h->fast_qr) {
     DQ_CHECK(qr_forward_fast(h->ctx, h->ws, h->qtc, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch,
-                             h->qr_method == DQ_QR_ITERATIVE ? h->qr_iters : 0));
+                             h->qr_method == DQ_QR_ITERATIVE ? (h->qr_iters_default ? DEFAULT_QR_SWEEPS_TC : h->qr_iters) : 0,
+                             h->bwd_split || h->orth_method == DQ_ORTH_CAYLEY));
   } else if (h->qr_method == DQ_QR_ITERATIVE && h->f32_winv_valid && h->f32_flags && h->cfg.d <= 1024) {
     // fp32 path: the same incremental factorisation on fp32 FMA products (U and U^-1 of the previous step)
     DQ_CHECK(qr_forward_incremental_f32(h->ctx, h->ws, h->Z, h->R, h->U, h->cfg.d, h->cfg.batch, h->qr_iters,
@@ -213,7 +223,10 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
         DQ_CHECK(splitk_reduce(ctx, h->gq_part, h->gq_ks, (int64_t)d * d, batch, 1.f, 0.f, gq_dst));
       }
     } else {
-      DQ_CHECK(tc_grad_rotation(h->tc, ctx, gq_dst, inv_n));
+      // a single micro-batch: the contraction's epilogue also leaves bf16(Gq^T) for the QR-Orth backward
+      const bool want_t = h->fast_qr && !h->small128 && !cayley && !h->bwd_split && n_micro == 1;
+      h->qtc.gqt_fresh = false;
+      DQ_CHECK(tc_grad_rotation(h->tc, ctx, gq_dst, inv_n, want_t ? h->qtc.gqt_hi : nullptr, &h->qtc.gqt_fresh));
     }
     if (a > 0) {
       DQ_CHECK(accumulate(ctx, h->Gq, gq_dst, (int64_t)d * d * batch));
@@ -238,7 +251,7 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
     DQ_CHECK(qr128_backward_sgd_tc(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, h->optimizer == DQ_SGD ? c.lr : 0.f, batch));
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
   } else {
-    if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch));
+    if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch, h->bwd_split));
     else {
       DQ_CHECK(qr_backward(ctx, h->ws, h->R, h->U, h->Gq, h->Gz, d, batch, h->f32_winv_valid));
       h->f32_winv_valid = true;
@@ -260,44 +273,73 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
   return DQ_OK;
 }
 
+void drop_graphs(dq_calib* h) {   // the schedule or a kernel argument changed: capture again
+  for (auto& g : h->graph) {
+    if (g.exec) cudaGraphExecDestroy(g.exec);
+    g = dq_calib::StepGraph();
+  }
+}
+
+// Which captured step fits the handle's state (see dq_calib::graph).
+int graph_slot(const dq_calib* h) { return (h->fast_qr && !h->small128) ? (h->qtc.w_sel & 1) : 0; }
+
 // Capture one full step into an executable graph (after one eager step has set every
 // kernel attribute).  Failure is not an error: the handle keeps launching eagerly.
+// Host-side state that a step advances is put back: the capture enqueued nothing.
 void try_capture(dq_calib* h) {
-  if (h->graph || h->graph_failed) return;
+  dq_calib::StepGraph& sg = h->graph[graph_slot(h)];
+  if (sg.exec || sg.failed) return;
   const int64_t before = h->ctx.launches;
   const double flops_before = h->ctx.mma_flops;
+  const QrTcState q_before = h->qtc;
+  const bool f32_winv = h->f32_winv_valid, small_warm = h->small_warm, cay_started = h->cay_started;
+  auto restore = [&]() {
+    h->ctx.launches = before;
+    h->ctx.mma_flops = flops_before;
+    h->qtc = q_before;
+    h->f32_winv_valid = f32_winv; h->small_warm = small_warm; h->cay_started = cay_started;
+    h->r_stale = h->orth_method != DQ_ORTH_CAYLEY || !cay_started;
+  };
   h->r_stale = true;
   // With plain SGD the update kernel writes the split copy of the new latent, so a step captured while that
   // copy is current holds no split_kernel: it may only be replayed while the copy is current.
-  h->graph_needs_z_split = h->fast_qr && h->qtc.z_split_fresh;
+  sg.needs_z_split = h->fast_qr && h->qtc.z_split_fresh;
   if (cudaStreamBeginCapture(h->ctx.stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();
-    h->graph_failed = true;
+    sg.failed = true;
     return;
   }
   const dq_status st = enqueue_step(h, false);
   cudaGraph_t g = nullptr;
   const cudaError_t e = cudaStreamEndCapture(h->ctx.stream, &g);
+  sg.launches = h->ctx.launches - before;
+  sg.flops = h->ctx.mma_flops - flops_before;
+  restore();
   if (st != DQ_OK || e != cudaSuccess || !g) {
     cudaGetLastError();
     if (g) cudaGraphDestroy(g);
-    h->graph_failed = true;
-    h->ctx.launches = before;
-    h->ctx.mma_flops = flops_before;
-    h->r_stale = true;
+    sg.failed = true;
     return;
   }
-  if (cudaGraphInstantiate(&h->graph, g, 0) != cudaSuccess) {
+  if (cudaGraphInstantiate(&sg.exec, g, 0) != cudaSuccess) {
     cudaGetLastError();
-    h->graph = nullptr;
-    h->graph_failed = true;
+    sg.exec = nullptr;
+    sg.failed = true;
   }
   cudaGraphDestroy(g);
-  h->graph_launches = h->ctx.launches - before;
-  h->graph_flops = h->ctx.mma_flops - flops_before;
-  h->ctx.launches = before;      // capture enqueued nothing
-  h->ctx.mma_flops = flops_before;
-  h->r_stale = true;
+}
+
+// Host-side state after a replayed step (what enqueue_step would have left).
+void after_replayed_step(dq_calib* h) {
+  const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
+  h->r_stale = !cayley;
+  if (cayley) return;
+  if (h->fast_qr && !h->small128) {
+    if (h->qr_method == DQ_QR_ITERATIVE) h->qtc.w_sel ^= 1;    // the step wrote the other set of W copies
+    else h->qtc.u_fresh = true;
+    if (h->qr_method == DQ_QR_ITERATIVE) h->qtc.u_fresh = false;
+    h->qtc.z_split_fresh = h->optimizer == DQ_SGD;
+  }
 }
 
 }  // namespace
@@ -406,16 +448,17 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
     const bool iterative = h->qr_method == DQ_QR_ITERATIVE && (h->small128 || h->fast_qr || f32_inc);
     const bool warm = h->small128 ? h->small_warm : (h->fast_qr ? h->qtc.t_warm : h->f32_winv_valid);
     const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
+    dq_calib::StepGraph& sg = h->graph[graph_slot(h)];
     const bool use_graph = cayley ? (!h->timing && h->cay_started && h->eager_steps_done >= 1)
                                   : (!h->timing && h->r_stale && h->eager_steps_done >= 1 &&
                                      (!iterative || warm) &&
-                                     (!h->graph || !h->graph_needs_z_split || h->qtc.z_split_fresh));
-    if (use_graph && !h->graph && !h->graph_failed) try_capture(h);
-    if (use_graph && h->graph) {
-      DQ_CHECK_CUDA(cudaGraphLaunch(h->graph, ctx.stream));
-      ctx.launches += h->graph_launches;
-      ctx.mma_flops += h->graph_flops;
-      h->r_stale = !cayley;
+                                     (!sg.exec || !sg.needs_z_split || h->qtc.z_split_fresh));
+    if (use_graph && !sg.exec && !sg.failed) try_capture(h);
+    if (use_graph && sg.exec) {
+      DQ_CHECK_CUDA(cudaGraphLaunch(sg.exec, ctx.stream));
+      ctx.launches += sg.launches;
+      ctx.mma_flops += sg.flops;
+      after_replayed_step(h);
     } else {
       DQ_CHECK(enqueue_step(h, h->timing));
       h->eager_steps_done++;
@@ -535,25 +578,24 @@ dq_status dq_calib_set_optimizer(dq_calib_t* h, int32_t optimizer, float lr, flo
   h->optimizer = optimizer;
   h->cfg.lr = lr;
   h->beta1 = beta1; h->beta2 = beta2; h->eps = eps;
-  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
-  h->graph_failed = false;
+  drop_graphs(h);
   return DQ_OK;
 }
 
 dq_status dq_calib_set_qr_method(dq_calib_t* h, int32_t method, int32_t n_iters) {
   if (!h || (method != DQ_QR_HOUSEHOLDER && method != DQ_QR_ITERATIVE) || n_iters > 64) return DQ_ERR_INVALID_ARG;
   const int iters = n_iters <= 0 ? 12 : n_iters;
-  if (method == h->qr_method && iters == h->qr_iters) return DQ_OK;
+  if (method == h->qr_method && iters == h->qr_iters && h->qr_iters_default == (n_iters <= 0)) return DQ_OK;
   DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
   DQ_CHECK(clear_status(h));
   h->qr_method = method;
   h->qr_iters = iters;
+  h->qr_iters_default = n_iters <= 0;
   h->r_stale = true;
   h->qtc.t_warm = false;
   h->small_warm = false;
   h->f32_winv_valid = false;
-  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
-  h->graph_failed = false;
+  drop_graphs(h);
   return DQ_OK;
 }
 
@@ -567,8 +609,7 @@ dq_status dq_calib_set_objective(dq_calib_t* h, int32_t objective, int32_t bits)
   DQ_CHECK(clear_status(h));
   h->obj.objective = objective;
   h->obj.bits = bits > 0 ? bits : 4;
-  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
-  h->graph_failed = false;
+  drop_graphs(h);
   return DQ_OK;
 }
 
@@ -597,8 +638,7 @@ dq_status dq_calib_set_orth_method(dq_calib_t* h, int32_t method, float beta, fl
   h->cay_started = false;
   h->r_stale = true;
   h->qtc.t_warm = false;
-  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the schedule changed: capture again
-  h->graph_failed = false;
+  drop_graphs(h);
   return DQ_OK;
 }
 
@@ -608,9 +648,26 @@ dq_status dq_calib_set_keep_gradient(dq_calib_t* h, int32_t keep) {
   if (k == h->tc.keep_g) return DQ_OK;
   DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
   h->tc.keep_g = k;
-  if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }   // the kernel arguments changed: capture again
-  h->graph_failed = false;
+  drop_graphs(h);
   return DQ_OK;
+}
+
+dq_status dq_calib_set_backward_precision(dq_calib_t* h, int32_t split) {
+  if (!h) return DQ_ERR_INVALID_ARG;
+  const bool sp = split != 0;
+  if (sp == h->bwd_split) return DQ_OK;
+  DQ_CHECK_CUDA(cudaStreamSynchronize(h->ctx.stream));
+  h->bwd_split = sp;
+  drop_graphs(h);
+  return DQ_OK;
+}
+
+dq_status dq_calib_selftest_bounded_wait(dq_calib_t* h, uint64_t limit_ns, uint64_t* d_waited_ns) {
+  if (!h || limit_ns == 0 || limit_ns > 100000000ull) return DQ_ERR_INVALID_ARG;   // at most 0.1 s
+  if (h->cfg.path != DQ_PATH_BF16_TC) return DQ_ERR_UNSUPPORTED;
+  DQ_CHECK(fence_in(h));
+  DQ_CHECK(bounded_wait_probe(h->ctx, limit_ns, d_waited_ns));
+  return fence_out(h);
 }
 
 dq_status dq_calib_set_timing(dq_calib_t* h, int32_t enabled) {
@@ -631,7 +688,14 @@ dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int6
   const int64_t dd = (int64_t)h->cfg.d * h->cfg.d * h->cfg.batch;
   switch (which) {
     case DQ_BUF_R: *d_ptr = h->R; *n_elems = dd; break;
-    case DQ_BUF_U: *d_ptr = h->U; *n_elems = dd; break;
+    case DQ_BUF_U:
+      if (h->fast_qr && !h->small128 && !h->qtc.u_fresh && h->orth_method == DQ_ORTH_QR && h->qtc.t_warm) {
+        // the incremental factorisation carries U^-1 only: invert it for the view
+        DQ_CHECK(fence_in(h));
+        DQ_CHECK(qr_tc_materialize_u(h->ctx, h->ws, h->qtc, h->U, h->cfg.d, h->cfg.batch));
+        DQ_CHECK(fence_out(h));
+      }
+      *d_ptr = h->U; *n_elems = dd; break;
     case DQ_BUF_GQ: *d_ptr = h->Gq; *n_elems = dd; break;
     case DQ_BUF_GZ: *d_ptr = h->Gz; *n_elems = dd; break;
     case DQ_BUF_G: *d_ptr = h->G; *n_elems = h->g_elems; break;

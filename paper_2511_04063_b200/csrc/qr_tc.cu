@@ -1,14 +1,16 @@
 // QR-Orth on the tensor cores (used with the tensor-core path).
 //
-// Forward:  U of Z = R U either by the blocked Householder factorisation (qr_panel_tc.cu kernels
-//           with the compact-WY products issued here) or, from the second step on, incrementally:
-//           U = (I + T) U_old with T from fixed-point sweeps on (Z U_old^-1)^T (Z U_old^-1).
-//           Then W = U^-1 by recursive block inversion and R = Z W.  (R is the same orthogonal
-//           factor the reflectors would give; forming it as Z U^-1 costs one GEMM instead of
-//           d / 128 dependent block updates.  Its orthogonality error grows like cond(Z) * 2^-17.)
-// Backward: B = R^T Gq, S = tril(B - B^T, -1), Gz = R (S W^T).
-// All d x d products run as split-bf16 tcgen05 GEMMs (three bf16 MMAs per product, fp32
-// accumulation, ~2^-17 relative error), clipped to the non-zero blocks of triangular operands.
+// Forward:  either the blocked Householder factorisation (qr_panel_tc.cu kernels with the compact-WY
+//           products issued here), then W = U^-1 by recursive block inversion and R = Z W (the same
+//           orthogonal factor the reflectors would give; forming it as Z U^-1 costs one GEMM instead
+//           of d / 128 dependent block updates; its orthogonality error grows like cond(Z) * 2^-17);
+//           or, from the second step on, incrementally from the previous step's W:
+//           Zh = Z W_old, I + T = upper factor of Zh by fixed-point sweeps, R = Zh (I + T)^-1,
+//           W = W_old (I + T)^-1 (qr_forward_incremental_tc).
+// Backward: S = tril(R^T Gq - Gq^T R, -1), Gz = R (S W^T).
+// The d x d products run as tcgen05 GEMMs clipped to the non-zero blocks of triangular operands, on
+// split-bf16 operands (three bf16 MMAs per product, ~2^-17 relative error) where the result needs fp32
+// accuracy and on plain bf16 operands where the product is a small correction or the data is bf16-accurate.
 #include <algorithm>
 #include <vector>
 
@@ -72,61 +74,6 @@ __global__ void __launch_bounds__(256) skew_split_kernel(const float* __restrict
     const int64_t idx = (int64_t)i * d + j;
     const float v = (i > j) ? B[idx] - t[tx][r] : 0.f;
     split2(v, hi[idx], lo[idx]);
-  }
-}
-
-// One sweep of the fixed-point iteration for the Cholesky factor U = I + T of G = Z^T Z:
-//   T <- striu(G - I - P) + diag(G - I - P) / 2,   P = T^T T (nullptr on the first sweep: T = 0).
-// G and P are only valid on and above the diagonal.  Writes T (fp32, row-major, zeros below the
-// diagonal), the split-bf16 copy of T^T (operand of the next P = T^T T) and, if U is given,
-// U = I + T with its split copy.
-// run_if (nullable): the sweep is skipped when *run_if == 0 (the previous sweep moved nothing).
-// moved_out (nullable): set to 1 if an entry moved by more than tol (0 otherwise: the caller clears it).
-// fail_if_moved: that case also sets DQ_ERR_NOT_CONVERGED (last sweep the schedule allows).
-// lower_done: tiles strictly below the diagonal already hold their zeros.
-__global__ void __launch_bounds__(256) chol_fixpoint_kernel(const float* __restrict__ G, const float* __restrict__ P,
-                                                            float* __restrict__ T, bf16* __restrict__ tt_hi,
-                                                            bf16* __restrict__ tt_lo, float* __restrict__ U,
-                                                            bf16* __restrict__ u_hi, bf16* __restrict__ u_lo, int d,
-                                                            const int* __restrict__ run_if, int* __restrict__ moved_out,
-                                                            int fail_if_moved, int lower_done, float tol,
-                                                            int* d_status) {
-  __shared__ float t[32][33];
-  if (run_if && *run_if == 0) return;
-  const int64_t off = (int64_t)blockIdx.z * d * d;
-  G += off; T += off; tt_hi += off; tt_lo += off;
-  if (P) P += off;
-  if (U) { U += off; u_hi += off; u_lo += off; }
-  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const bool upper = j0 + 31 >= i0;     // tile touches the upper triangle
-  if (!upper && lower_done && !U) return;   // zeros written by an earlier sweep stay zeros
-  bool moved = false;
-  for (int r = ty; r < 32; r += 8) {
-    const int i = i0 + r, j = j0 + tx;
-    const int64_t idx = (int64_t)i * d + j;
-    float v = 0.f;
-    if (upper && j >= i) {
-      v = G[idx] - ((i == j) ? 1.f : 0.f) - (P ? P[idx] : 0.f);
-      if (i == j) v *= 0.5f;
-      if (P && !(fabsf(v - T[idx]) <= tol)) moved = true;
-    }
-    T[idx] = v;
-    t[r][tx] = v;
-    if (U) {
-      const float u = v + ((i == j) ? 1.f : 0.f);
-      U[idx] = u;
-      split2(u, u_hi[idx], u_lo[idx]);
-    }
-  }
-  if (moved) {
-    if (moved_out) *moved_out = 1;
-    if (fail_if_moved) set_status(d_status, DQ_ERR_NOT_CONVERGED);
-  }
-  __syncthreads();
-  for (int c = ty; c < 32; c += 8) {    // T^T[j][i] = T[i][j]
-    const int64_t idx = (int64_t)(j0 + c) * d + i0 + tx;
-    split2(t[tx][c], tt_hi[idx], tt_lo[idx]);
   }
 }
 
@@ -216,49 +163,66 @@ using tch::Op;
 using tch::Out;
 using tch::gemm3;
 
+// dst[b][r][c] = hi[b][r][c] + lo[b][r][c]   (fp32 value of a split pair)
+__global__ void __launch_bounds__(256) combine_kernel(const bf16* __restrict__ hi, const bf16* __restrict__ lo,
+                                                      float* __restrict__ dst, int64_t n) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] = __bfloat162float(hi[i]) + __bfloat162float(lo[i]);
+}
+
+// Operands and results of the blocked inverse of an upper-triangular matrix (all [batch][d][d]).
+struct TriInv {
+  const float* src;                 // the matrix (fp32), read for its 128 x 128 diagonal blocks
+  const bf16 *s_hi, *s_lo;          // its split copy (off-diagonal blocks)
+  bf16 *n_hi, *n_lo;                // the inverse, row-major
+  bf16 *t_hi, *t_lo;                // the inverse, transposed
+  bf16 *tmp_hi, *tmp_lo;            // scratch
+};
+
 // Block column of the inverse:  W[0:k, k:k+s] = -W[0:k,0:k] U[0:k, k:k+s] W[k:k+s, k:k+s]
 // for `count` independent diagonal positions `stride` elements apart (3rd tensor dimension).
-dq_status merge(Ctx& ctx, QrTcState& q, int d, int k, int s, int count, int64_t stride, int64_t base) {
+dq_status merge(Ctx& ctx, const TriInv& io, int d, int k, int s, int count, int64_t stride, int64_t base) {
   // T1t[j][i] = sum_l W22^T[j][l] U12[i][l]        (s x k, dense temporary)
-  Op a{q.wt_hi + base + (int64_t)k * d + k, q.wt_lo + base + (int64_t)k * d + k, d, stride};
-  Op b{q.u_hi + base + k, q.u_lo + base + k, d, stride};
-  Out t1; t1.hi = q.t1_hi; t1.lo = q.t1_lo; t1.ld_h = k; t1.bs_h = (int64_t)s * k;
+  Op a{io.t_hi + base + (int64_t)k * d + k, io.t_lo + base + (int64_t)k * d + k, d, stride};
+  Op b{io.s_hi + base + k, io.s_lo + base + k, d, stride};
+  Out t1; t1.hi = io.tmp_hi; t1.lo = io.tmp_lo; t1.ld_h = k; t1.bs_h = (int64_t)s * k;
   DQ_CHECK(gemm3(ctx, a, b, s, k, s, count, t1));
-  Op w11{q.wn_hi + base, q.wn_lo + base, d, stride};
-  Op t1o{q.t1_hi, q.t1_lo, k, (int64_t)s * k};
-  // W12[i][j] = -sum_l W11[i][l] T1t[j][l]   -> WN block (0, k)
-  Out o12; o12.hi = q.wn_hi + base + k; o12.lo = q.wn_lo + base + k; o12.ld_h = d; o12.bs_h = stride; o12.alpha = -1.f;
+  Op w11{io.n_hi + base, io.n_lo + base, d, stride};
+  Op t1o{io.tmp_hi, io.tmp_lo, k, (int64_t)s * k};
+  // W12[i][j] = -sum_l W11[i][l] T1t[j][l]   -> row-major block (0, k)
+  Out o12; o12.hi = io.n_hi + base + k; o12.lo = io.n_lo + base + k; o12.ld_h = d; o12.bs_h = stride; o12.alpha = -1.f;
   DQ_CHECK(gemm3(ctx, w11, t1o, k, s, k, count, o12));
-  // W12^T[j][i] = -sum_l T1t[j][l] W11[i][l] -> WT block (k, 0)
-  Out o21; o21.hi = q.wt_hi + base + (int64_t)k * d; o21.lo = q.wt_lo + base + (int64_t)k * d; o21.ld_h = d;
+  // W12^T[j][i] = -sum_l T1t[j][l] W11[i][l] -> transposed block (k, 0)
+  Out o21; o21.hi = io.t_hi + base + (int64_t)k * d; o21.lo = io.t_lo + base + (int64_t)k * d; o21.ld_h = d;
   o21.bs_h = stride; o21.alpha = -1.f;
   return gemm3(ctx, t1o, w11, s, k, k, count, o21);
 }
 
-dq_status tri_inverse_tc(Ctx& ctx, QrTcState& q, const float* U, int d, int batch) {
+dq_status tri_inverse_tc(Ctx& ctx, const TriInv& io, int d, int batch) {
   const int64_t dd = (int64_t)d * d;
   const size_t bytes = sizeof(bf16) * (size_t)dd * batch;
-  DQ_CHECK_CUDA(cudaMemsetAsync(q.wn_hi, 0, bytes, ctx.stream));
-  DQ_CHECK_CUDA(cudaMemsetAsync(q.wn_lo, 0, bytes, ctx.stream));
-  DQ_CHECK_CUDA(cudaMemsetAsync(q.wt_hi, 0, bytes, ctx.stream));
-  DQ_CHECK_CUDA(cudaMemsetAsync(q.wt_lo, 0, bytes, ctx.stream));
+  DQ_CHECK_CUDA(cudaMemsetAsync(io.n_hi, 0, bytes, ctx.stream));
+  DQ_CHECK_CUDA(cudaMemsetAsync(io.n_lo, 0, bytes, ctx.stream));
+  DQ_CHECK_CUDA(cudaMemsetAsync(io.t_hi, 0, bytes, ctx.stream));
+  DQ_CHECK_CUDA(cudaMemsetAsync(io.t_lo, 0, bytes, ctx.stream));
   const int smem = TRI_INV_SMEM;
   static SmemOptIn attr;
   DQ_CHECK(opt_in_dynamic_smem(tri_inv_diag128_kernel, smem, attr));
-  tri_inv_diag128_kernel<<<dim3(d / DB, batch), TRI_INV_THREADS, smem, ctx.stream>>>(U, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, d);
+  tri_inv_diag128_kernel<<<dim3(d / DB, batch), TRI_INV_THREADS, smem, ctx.stream>>>(io.src, io.n_hi, io.n_lo, io.t_hi,
+                                                                                     io.t_lo, d);
   DQ_CHECK(after_launch(ctx));
   int s = DB, count = d / DB;
   while (count > 1 && count % 2 == 0) {
     const int pairs = count / 2;
     const int64_t pair_stride = (int64_t)2 * s * (d + 1);
     if (batch == 1) {
-      DQ_CHECK(merge(ctx, q, d, s, s, pairs, pair_stride, 0));
+      DQ_CHECK(merge(ctx, io, d, s, s, pairs, pair_stride, 0));
     } else {
-      for (int pidx = 0; pidx < pairs; ++pidx) DQ_CHECK(merge(ctx, q, d, s, s, batch, dd, pidx * pair_stride));
+      for (int pidx = 0; pidx < pairs; ++pidx) DQ_CHECK(merge(ctx, io, d, s, s, batch, dd, pidx * pair_stride));
     }
     s *= 2; count = pairs;
   }
-  for (int kb = 1; kb < count; ++kb) DQ_CHECK(merge(ctx, q, d, kb * s, s, batch, dd, 0));
+  for (int kb = 1; kb < count; ++kb) DQ_CHECK(merge(ctx, io, d, kb * s, s, batch, dd, 0));
   return DQ_OK;
 }
 
@@ -276,13 +240,25 @@ int wy_ksplit(int m, int batch, int sm_count) {
   return ks < 1 ? 1 : ks;
 }
 
+// The two sets of copies of W = U^-1 (row-major and transposed, split): index 0 / 1.
+struct WSet { bf16 *n_hi, *n_lo, *t_hi, *t_lo; };
+WSet wset(const QrTcState& q, int sel) {
+  return sel == 0 ? WSet{q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo} : WSet{q.wn2_hi, q.wn2_lo, q.wt2_hi, q.wt2_lo};
+}
+
+void upper_lists(Out& o, const QrTcState& q) {
+  o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
+}
+
 }  // namespace
 
 dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   const int64_t dd = (int64_t)d * d * batch;
   bf16** all[] = {&q.z_hi, &q.z_lo, &q.u_hi, &q.u_lo, &q.wn_hi, &q.wn_lo, &q.wt_hi, &q.wt_lo, &q.r_hi, &q.r_lo,
-                  &q.rt_hi, &q.rt_lo, &q.gqt_hi, &q.gqt_lo, &q.st_hi, &q.st_lo, &q.m_hi, &q.m_lo, &q.t1_hi, &q.t1_lo};
+                  &q.rt_hi, &q.rt_lo, &q.gqt_hi, &q.gqt_lo, &q.st_hi, &q.st_lo, &q.m_hi, &q.m_lo, &q.t1_hi, &q.t1_lo,
+                  &q.wn2_hi, &q.wn2_lo, &q.wt2_hi, &q.wt2_lo, &q.yt_hi, &q.yt_lo, &q.nm1, &q.nm2};
   for (bf16** p : all) DQ_CHECK(alloc(p, dd));
+  DQ_CHECK(alloc(&q.P, dd));
   const int64_t yb = (int64_t)d * 128 * batch;
   DQ_CHECK(alloc(&q.y_hi, yb)); DQ_CHECK(alloc(&q.y_lo, yb));
   DQ_CHECK(alloc(&q.w2_hi, yb)); DQ_CHECK(alloc(&q.w2_lo, yb));
@@ -299,10 +275,11 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   for (int unit = 128; unit <= 256; unit *= 2) {   // tile orders: most expensive tiles first, dealt round-robin to the persistent CTAs
     if (d % unit != 0) break;
     const int nb = d / unit;
-    std::vector<int> upper, desc, asc;
+    std::vector<int> upper, lower, desc, asc;
     for (int j = 0; j < nb; ++j)
       for (int i = 0; i < nb; ++i) {
         if (i <= j) upper.push_back(i | (j << 16));
+        if (i >= j) lower.push_back(i | (j << 16));
         desc.push_back(i | (j << 16));
       }
     std::stable_sort(upper.begin(), upper.end(), [](int a, int b) { return (a & 0xffff) > (b & 0xffff); });
@@ -310,12 +287,15 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
     asc = desc;
     std::reverse(asc.begin(), asc.end());
     int*& tu = (unit == 128) ? q.tl_upper : q.tl2_upper;
+    int*& tlw = (unit == 128) ? q.tl_lower : q.tl2_lower;
     int*& td = (unit == 128) ? q.tl_desc_nb : q.tl2_desc_nb;
     int*& ta = (unit == 128) ? q.tl_asc_nb : q.tl2_asc_nb;
     ((unit == 128) ? q.n_upper : q.n2_upper) = (int)upper.size();
     ((unit == 128) ? q.n_all : q.n2_all) = (int)desc.size();
-    DQ_CHECK(alloc(&tu, (int64_t)upper.size())); DQ_CHECK(alloc(&td, (int64_t)desc.size())); DQ_CHECK(alloc(&ta, (int64_t)desc.size()));
+    DQ_CHECK(alloc(&tu, (int64_t)upper.size())); DQ_CHECK(alloc(&tlw, (int64_t)lower.size()));
+    DQ_CHECK(alloc(&td, (int64_t)desc.size())); DQ_CHECK(alloc(&ta, (int64_t)desc.size()));
     DQ_CHECK_CUDA(cudaMemcpy(tu, upper.data(), sizeof(int) * upper.size(), cudaMemcpyHostToDevice));
+    DQ_CHECK_CUDA(cudaMemcpy(tlw, lower.data(), sizeof(int) * lower.size(), cudaMemcpyHostToDevice));
     DQ_CHECK_CUDA(cudaMemcpy(td, desc.data(), sizeof(int) * desc.size(), cudaMemcpyHostToDevice));
     DQ_CHECK_CUDA(cudaMemcpy(ta, asc.data(), sizeof(int) * asc.size(), cudaMemcpyHostToDevice));
   }
@@ -325,11 +305,13 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
 
 void qr_tc_destroy(QrTcState& q) {
   bf16* all[] = {q.z_hi, q.z_lo, q.u_hi, q.u_lo, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, q.r_hi, q.r_lo,
-                 q.rt_hi, q.rt_lo, q.gqt_hi, q.gqt_lo, q.st_hi, q.st_lo, q.m_hi, q.m_lo, q.t1_hi, q.t1_lo};
+                 q.rt_hi, q.rt_lo, q.gqt_hi, q.gqt_lo, q.st_hi, q.st_lo, q.m_hi, q.m_lo, q.t1_hi, q.t1_lo,
+                 q.wn2_hi, q.wn2_lo, q.wt2_hi, q.wt2_lo, q.yt_hi, q.yt_lo, q.nm1, q.nm2};
   for (bf16* p : all) cudaFree(p);
+  cudaFree(q.P);
   cudaFree(q.y_hi); cudaFree(q.y_lo); cudaFree(q.w2_hi); cudaFree(q.w2_lo); cudaFree(q.part); cudaFree(q.T);
   cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.uot_hi); cudaFree(q.uot_lo); cudaFree(q.tl_upper); cudaFree(q.tl_desc_nb); cudaFree(q.tl_asc_nb);
-  cudaFree(q.tl2_upper); cudaFree(q.tl2_desc_nb); cudaFree(q.tl2_asc_nb); cudaFree(q.sweep_flags);
+  cudaFree(q.tl2_upper); cudaFree(q.tl2_desc_nb); cudaFree(q.tl2_asc_nb); cudaFree(q.tl_lower); cudaFree(q.tl2_lower); cudaFree(q.sweep_flags);
   q = QrTcState();
 }
 
@@ -362,90 +344,144 @@ dq_status qr_factor_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, 
   return qr_diag_check(ctx, At, d, batch);
 }
 
-// U of the latent one optimiser step after a latent whose factors (U_old, W_old = U_old^-1) are
-// known, without dependent column steps.  Zh = Z W_old is close to orthogonal however far Z itself
-// has drifted (Zh = R_old + (Z - Z_old) W_old), so its upper factor Uh = I + T is the fixed point of
-//   T <- Phi(Zh^T Zh - I - T^T T),  Phi(S) = striu(S) + diag(S) / 2,
-// reached from T = 0 in a few sweeps; then U = Uh U_old.  Every product is a split-bf16
-// tensor-core GEMM restricted to the non-zero blocks of its triangular operands.
-dq_status qr_upper_factor_incremental(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* U, int d,
-                                      int batch, int n_sweeps) {
+// R and W = U^-1 of the latent one optimiser step after a latent whose W_old is known, without dependent
+// column steps and without forming U.  Zh = Z W_old is close to orthogonal however far Z itself has drifted
+// (Zh = R_old + (Z - Z_old) W_old), so its upper factor I + T is the fixed point of
+//   T <- Phi(E - T^T T),  E = Zh^T Zh - I,  Phi(S) = striu(S) + diag(S) / 2.
+// The iteration starts from Phi(E - P) with P = T^T T of the previous step (consecutive steps are alike), runs
+// in the epilogues of the products T^T T (one launch per sweep), and stops by device flags: sweep k runs only
+// if sweep k - 1 moved an entry by more than 1e-5; the launch sequence is fixed, so a captured graph replays
+// it unchanged.  Then (I + T)^-1 = I + Y from the identity
+//   (I + T)^-1 = (I - T)(I + T^2)(I + T^4) (I - T^8)^-1:
+// two triangular products give (I - T)(I + T^2) (error |T|^4, enough after a small step), two more the factor
+// (I + T^4) (error |T|^8, after a large step).  R = Zh + Zh Y and W = W_old + W_old Y.  Zh and E are split-bf16 products (three MMAs); the others act on
+// terms of size |T| and use plain bf16 operands (their 2^-9 relative error is of size 2^-9 |T|) unless the
+// fixed point needed a third sweep, the sign of a large step: then the first-order ones switch to split
+// operands and the higher-order factor is added (a device flag selects which launches run).
+// need_lo: also the lo parts of the split copies of R and R^T (read only by products on split operands).
+dq_status qr_forward_incremental_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, int d,
+                                    int batch, int n_sweeps, bool need_lo) {
   const int64_t dd = (int64_t)d * d;
   const dim3 tiles(d / 32, d / 32, batch);
-  bf16 *zht_hi = q.st_hi, *zht_lo = q.st_lo;   // free until the backward pass
-  bf16 *uh_hi = q.gqt_hi, *uh_lo = q.gqt_lo;   // likewise
-  float *Zh = ws.A, *G = ws.B, *P = ws.S, *T = ws.tmp, *scratch = ws.Q;
+  const WSet wc = wset(q, q.w_sel), wn = wset(q, q.w_sel ^ 1);
+  float *Zh = ws.A, *E = ws.B, *T = ws.tmp, *T2 = ws.S, *Y3 = ws.Q, *T4 = ws.V, *Wf = ws.Winv;
+  // bf16 scratch (all free until the backward pass or owned by the Householder route)
+  bf16 *zh_hi = q.m_hi, *zh_lo = q.m_lo, *zht_hi = q.st_hi, *zht_lo = q.st_lo;
+  bf16 *twa_hi = q.tw_hi, *twa_lo = q.tw_lo, *twb_hi = q.t1_hi, *twb_lo = q.t1_lo;   // T^T, alternating between sweeps
+  bf16 *twf_hi = q.uot_hi, *twf_lo = q.uot_lo;                                       // T^T of the last sweep that ran
+  bf16 *t_hi = q.u_hi, *t_lo = q.u_lo;                                               // T row-major
+  bf16 *t2_hi = q.gqt_hi, *t2t_hi = q.gqt_lo, *y3_hi = q.nm1, *t4t_hi = q.nm2;
+  q.u_fresh = false;
   if (!q.z_split_fresh) {   // (the SGD update writes the split copy with the new latent)
     split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
     DQ_CHECK(after_launch(ctx));
     q.z_split_fresh = true;
   }
-  {   // Zh[i][j] = sum_k Z[i][k] W_old[k][j]
-    Op a{q.z_hi, q.z_lo, d, dd}, b{q.wt_hi, q.wt_lo, d, dd};
-    Out o; o.f32 = Zh; o.ld = d; o.bs = dd; o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
+  {   // Zh[i][j] = sum_k Z[i][k] W_old[k][j]  (W upper triangular: k <= j)
+    Op a{q.z_hi, q.z_lo, d, dd}, b{wc.t_hi, wc.t_lo, d, dd};
+    Out o; o.f32 = Zh; o.ld = d; o.bs = dd; o.hi = zh_hi; o.lo = zh_lo; o.ld_h = d; o.bs_h = dd;
+    o.t_hi = zht_hi; o.t_lo = zht_lo; o.ld_t = d; o.bs_t = dd;
+    o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
     DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   }
-  DQ_CHECK(qrp_transpose_split(ctx, Zh, scratch, zht_hi, zht_lo, d, batch));
-  {   // G[i][j] = sum_k Zh[k][i] Zh[k][j], tiles on and above the block diagonal
+  const int n_total = n_sweeps + 3;
+  int* flags = q.sweep_flags;      // flags[k] = 1: sweep k moved an entry
+  DQ_CHECK_CUDA(cudaMemsetAsync(flags, 0, sizeof(int) * (n_total + 2), ctx.stream));
+  {   // E = Zh^T Zh - I on the upper tiles, and the start of the fixed point T = Phi(E - P_old)
     Op a{zht_hi, zht_lo, d, dd};
-    Out o; o.f32 = G; o.ld = d; o.bs = dd; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
+    // (the first sweep always follows and reads only the hi part of T^T)
+    Out o; o.f32 = E; o.ld = d; o.bs = dd; o.add1 = q.P; o.aux = T; o.gen_mode = tc::GEN_CHOL_FIRST;
+    o.t_hi = twa_hi; o.ld_t = d; o.bs_t = dd;
+    upper_lists(o, q);
     DQ_CHECK(gemm3(ctx, a, a, d, d, d, batch, o));
   }
-  // Sweep 0 sets T = Phi(E).  Then up to n_sweeps cheap sweeps (plain bf16 product: its relative error 2^-9
-  // acts on a term of size ||T||^2 and later sweeps forgive it by a factor ||T|| each), each skipped once
-  // the sweep before it moved no entry by more than the tolerance, and finally up to three accurate sweeps
-  // (split-bf16 product), the first always taken, the others only while entries still move.  flags[k] = 1
-  // if sweep k moved something; the launch sequence is fixed, so a captured graph replays it unchanged.
-  constexpr int ACCURATE = 3;
-  int* flags = q.sweep_flags;
-  DQ_CHECK_CUDA(cudaMemsetAsync(flags, 0, sizeof(int) * (n_sweeps + ACCURATE + 2), ctx.stream));
-  chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, nullptr, T, q.tw_hi, q.tw_lo, nullptr, nullptr, nullptr, d,
-                                                      nullptr, nullptr, 0, 0, 1e-5f, ctx.d_status);
-  DQ_CHECK(after_launch(ctx));
-  for (int it = 1; it <= n_sweeps + ACCURATE; ++it) {
-    const bool accurate = it > n_sweeps;
-    const bool first_accurate = it == n_sweeps + 1;
-    const bool last = it == n_sweeps + ACCURATE;
-    // cheap sweep 1 always runs; a later cheap sweep runs if the one before moved; the first accurate sweep
-    // always runs; a later accurate sweep runs if the accurate sweep before it moved
-    const int* run_if = (it == 1 || first_accurate) ? nullptr : flags + it - 1;
-    {   // P[i][j] = sum_k T[k][i] T[k][j]; T^T is lower triangular: k < 128 (mb + 1), mb <= nb
-      Op tt{q.tw_hi, q.tw_lo, d, dd};
-      Out o; o.f32 = P; o.ld = d; o.bs = dd; o.k_mode = 2; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
-      o.nterms = accurate ? 3 : 1;
-      o.run_if = run_if;
-      DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
-    }
-    chol_fixpoint_kernel<<<tiles, 256, 0, ctx.stream>>>(G, P, T, q.tw_hi, q.tw_lo, accurate ? scratch : nullptr, uh_hi,
-                                                        uh_lo, d, run_if, flags + it, last ? 1 : 0, 1, 1e-5f,
-                                                        ctx.d_status);
-    DQ_CHECK(after_launch(ctx));
+  for (int k = 1; k <= n_total; ++k) {
+    // P[i][j] = sum_l T[l][i] T[l][j] (T^T is lower triangular: l < 128 (mb + 1), mb <= nb), then
+    // T <- Phi(E - P) in the epilogue.  The operand T^T alternates between two buffers, because the epilogue
+    // of one tile rewrites what the main loop of another still reads.
+    const bool odd = k & 1;
+    Op tt{odd ? twa_hi : twb_hi, odd ? twa_lo : twb_lo, d, dd};
+    Out o; o.f32 = q.P; o.ld = d; o.bs = dd; o.add1 = E; o.aux = T; o.gen_mode = tc::GEN_CHOL_SWEEP;
+    o.tol = 1e-5f; o.moved_out = flags + k; o.fail_if_moved = (k == n_total) ? 1 : 0;
+    o.hi = t_hi; o.lo = t_lo; o.ld_h = d; o.bs_h = dd;
+    // T^T for the next sweep (its lo part only if that sweep uses split operands), and the copies the later
+    // products read, which every sweep that runs must leave behind (which one is the last is not known here)
+    o.t_hi = odd ? twb_hi : twa_hi; o.t_lo = (k + 1 > 2) ? (odd ? twb_lo : twa_lo) : nullptr;
+    o.t2_hi = twf_hi; o.t2_lo = twf_lo;
+    o.ld_t = d; o.bs_t = dd;
+    o.k_mode = 2; upper_lists(o, q);
+    o.nterms = (k <= 2) ? 1 : 3;
+    o.run_if = (k == 1) ? nullptr : flags + k - 1;
+    DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
   }
-  {   // U[i][j] = sum_k Uh[i][k] U_old[k][j]: both upper triangular, k in [128 mb, 128 (nb + 1))
-    Op a{uh_hi, uh_lo, d, dd}, b{q.uot_hi, q.uot_lo, d, dd};
-    Out o; o.f32 = U; o.ld = d; o.bs = dd; o.hi = q.u_hi; o.lo = q.u_lo; o.ld_h = d; o.bs_h = dd;
-    o.k_mode = 1 | 4; o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
+  const int* big = flags + 2;     // a third sweep ran: a large step, first-order products with split operands
+  Op t{t_hi, t_lo, d, dd}, ttf{twf_hi, twf_lo, d, dd};
+  for (int v = 0; v < 2; ++v) {   // T2 = T T  (upper x upper: k in [128 mb, 128 (nb + 1)))
+    Out o; o.f32 = T2; o.ld = d; o.bs = dd; o.hi = t2_hi; o.ld_h = d; o.bs_h = dd; o.t_hi = t2t_hi; o.ld_t = d; o.bs_t = dd;
+    o.k_mode = 1 | 4; upper_lists(o, q);
+    o.nterms = v ? 3 : 1; (v ? o.run_if : o.run_unless) = big;
+    DQ_CHECK(gemm3(ctx, t, ttf, d, d, d, batch, o));
+  }
+  {   // Y3 = -T + T2 - T T2 = (I - T)(I + T2) - I: all of Y after a small step (error |T|^4)
+    Op b{t2t_hi, t2t_hi, d, dd};
+    Out o; o.f32 = Y3; o.ld = d; o.bs = dd; o.alpha = -1.f; o.add1 = T2; o.g1 = 1.f; o.add2 = T; o.g2 = -1.f;
+    o.hi = y3_hi; o.ld_h = d; o.bs_h = dd; o.t_hi = q.yt_hi; o.t_lo = q.yt_lo; o.ld_t = d; o.bs_t = dd;
+    o.k_mode = 1 | 4; upper_lists(o, q); o.nterms = 1;
+    DQ_CHECK(gemm3(ctx, t, b, d, d, d, batch, o));
+  }
+  {   // after a large step also the factor (I + T^4):  T4 = T2 T2
+    Op a{t2_hi, t2_hi, d, dd}, b{t2t_hi, t2t_hi, d, dd};
+    Out o; o.f32 = T4; o.ld = d; o.bs = dd; o.t_hi = t4t_hi; o.ld_t = d; o.bs_t = dd; o.k_mode = 1 | 4; upper_lists(o, q);
+    o.nterms = 1; o.run_if = big;
     DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   }
-  return qr_diag_check(ctx, U, d, batch);
+  {   // Y = Y3 + T4 + Y3 T4 = (I + Y3)(I + T4) - I; only its transposed split copy is kept
+    Op a{y3_hi, y3_hi, d, dd}, b{t4t_hi, t4t_hi, d, dd};
+    Out o; o.ld = d; o.bs = dd; o.add1 = Y3; o.add2 = T4; o.t_hi = q.yt_hi; o.t_lo = q.yt_lo; o.ld_t = d; o.bs_t = dd;
+    o.k_mode = 1 | 4; upper_lists(o, q); o.nterms = 1; o.run_if = big;
+    DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
+  }
+  Op yt{q.yt_hi, q.yt_lo, d, dd};
+  for (int v = 0; v < 2; ++v) {   // R = Zh + Zh Y  (Y upper triangular: k <= j)
+    Op a{zh_hi, zh_lo, d, dd};
+    Out o; o.f32 = R; o.ld = d; o.bs = dd; o.add1 = Zh; o.hi = q.r_hi; o.lo = need_lo ? q.r_lo : nullptr; o.ld_h = d; o.bs_h = dd;
+    o.t_hi = q.rt_hi; o.t_lo = need_lo ? q.rt_lo : nullptr; o.ld_t = d; o.bs_t = dd;
+    o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
+    o.nterms = v ? 3 : 1; (v ? o.run_if : o.run_unless) = big;
+    DQ_CHECK(gemm3(ctx, a, yt, d, d, d, batch, o));
+  }
+  for (int v = 0; v < 2; ++v) {   // W = W_old + W_old Y into the other set of copies (the fp32 W in place)
+    Op a{wc.n_hi, wc.n_lo, d, dd};
+    Out o; o.f32 = Wf; o.ld = d; o.bs = dd; o.add1 = Wf; o.hi = wn.n_hi; o.lo = wn.n_lo; o.ld_h = d; o.bs_h = dd;
+    o.t_hi = wn.t_hi; o.t_lo = wn.t_lo; o.ld_t = d; o.bs_t = dd;
+    o.k_mode = 1 | 4; upper_lists(o, q);
+    o.nterms = v ? 3 : 1; (v ? o.run_if : o.run_unless) = big;
+    DQ_CHECK(gemm3(ctx, a, yt, d, d, d, batch, o));
+  }
+  q.w_sel ^= 1;
+  // diag(W) = 1 / diag(U): the same rank and finiteness test
+  return qr_diag_check(ctx, Wf, d, batch);
 }
 
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
-                          int batch, int iterative_iters) {
+                          int batch, int iterative_iters, bool need_lo) {
   if (d % 128 != 0) return DQ_ERR_UNSUPPORTED;
   const int64_t dd = (int64_t)d * d;
   const dim3 tiles(d / 32, d / 32, batch);
-  const bool incremental = iterative_iters > 0 && q.t_warm;
-  if (incremental) {
-    DQ_CHECK(qr_upper_factor_incremental(ctx, ws, q, Z, U, d, batch, iterative_iters));
-  } else {   // no factors of a nearby latent yet (first call, latent replaced): Householder
-    DQ_CHECK(qr_factor_tc(ctx, ws, q, Z, d, batch));
-    DQ_CHECK(qrp_gauge_ut(ctx, ws.A, U, q.u_hi, q.u_lo, d, batch));
-  }
-  DQ_CHECK(tri_inverse_tc(ctx, q, U, d, batch));
-  if (iterative_iters > 0) {   // U^T for the next step's U = Uh U_old
-    split_kernel<<<tiles, 256, 0, ctx.stream>>>(U, q.uot_hi, q.uot_lo, d, 1);
+  if (iterative_iters > 0 && q.t_warm)
+    return qr_forward_incremental_tc(ctx, ws, q, Z, R, d, batch, iterative_iters, need_lo);
+  // no factors of a nearby latent yet (first call, latent replaced), or Householder at every step
+  DQ_CHECK(qr_factor_tc(ctx, ws, q, Z, d, batch));
+  DQ_CHECK(qrp_gauge_ut(ctx, ws.A, U, q.u_hi, q.u_lo, d, batch));
+  q.u_fresh = true;
+  q.w_sel = 0;
+  const WSet w = wset(q, 0);
+  const TriInv io{U, q.u_hi, q.u_lo, w.n_hi, w.n_lo, w.t_hi, w.t_lo, q.t1_hi, q.t1_lo};
+  DQ_CHECK(tri_inverse_tc(ctx, io, d, batch));
+  if (iterative_iters > 0) {   // state the incremental steps continue from: W in fp32, no T^T T yet
+    combine_kernel<<<ctx.sm_count * 8, 256, 0, ctx.stream>>>(w.n_hi, w.n_lo, ws.Winv, dd * batch);
     DQ_CHECK(after_launch(ctx));
+    DQ_CHECK_CUDA(cudaMemsetAsync(q.P, 0, sizeof(float) * (size_t)dd * batch, ctx.stream));
     q.t_warm = true;
   }
   if (!q.z_split_fresh) {
@@ -453,42 +489,71 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
     DQ_CHECK(after_launch(ctx));
     q.z_split_fresh = true;
   }
-  // R[i][j] = sum_k Z[i][k] W[k][j]:  A = Z (row-major), B = W^T
+  // R[i][j] = sum_k Z[i][k] W[k][j]:  A = Z (row-major), B = W^T; also the split copies of R and R^T
   Op a{q.z_hi, q.z_lo, d, dd};
-  Op b{q.wt_hi, q.wt_lo, d, dd};
+  Op b{w.t_hi, w.t_lo, d, dd};
   Out o; o.f32 = R; o.ld = d; o.bs = dd; o.hi = q.r_hi; o.lo = q.r_lo; o.ld_h = d; o.bs_h = dd;
+  o.t_hi = q.rt_hi; o.t_lo = q.rt_lo; o.ld_t = d; o.bs_t = dd;
   o.k_mode = 4;   // W is upper triangular: W^T[j][k] = 0 for k > j
   o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
-  DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
-  split_kernel<<<tiles, 256, 0, ctx.stream>>>(R, q.rt_hi, q.rt_lo, d, 1);
-  return after_launch(ctx);
+  return gemm3(ctx, a, b, d, d, d, batch, o);
 }
 
-dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch) {
+// U of the current factorisation for inspection: the Householder route leaves it in place; the incremental
+// route carries only W = U^-1, which is inverted here (split-bf16 accuracy, about 1e-5 relative).
+dq_status qr_tc_materialize_u(Ctx& ctx, QrWorkspace& ws, QrTcState& q, float* U, int d, int batch) {
+  if (q.u_fresh) return DQ_OK;
+  const WSet w = wset(q, q.w_sel);
+  const TriInv io{ws.Winv, w.n_hi, w.n_lo, q.u_hi, q.u_lo, q.st_hi, q.st_lo, q.t1_hi, q.t1_lo};
+  DQ_CHECK(tri_inverse_tc(ctx, io, d, batch));
+  combine_kernel<<<ctx.sm_count * 8, 256, 0, ctx.stream>>>(q.u_hi, q.u_lo, U, (int64_t)d * d * batch);
+  DQ_CHECK(after_launch(ctx));
+  q.u_fresh = true;
+  return DQ_OK;
+}
+
+// Gz = R tril(R^T Gq - Gq^T R, -1) W^T.  Gq carries the bf16 rounding of the rotation operand and of dL/dO
+// (a few percent relative), so with split == false every product runs on plain bf16 operands (2^-9):
+//   S = tril(B - B^T, -1) as ONE reduction over two operand pairs, (R^T, Gq^T) minus (Gq^T, R^T), on the tiles
+//   on and below the block diagonal;  D^T = W S^T (triangular x triangular);  Gz = R D.
+// split == true keeps three MMAs per product (B in fp32, then the skew part by an element-wise kernel).
+dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch,
+                         bool split) {
   const int64_t dd = (int64_t)d * d;
   const dim3 tiles(d / 32, d / 32, batch);
-  split_kernel<<<tiles, 256, 0, ctx.stream>>>(Gq, q.gqt_hi, q.gqt_lo, d, 1);
-  DQ_CHECK(after_launch(ctx));
-  // B[i][j] = sum_k R[k][i] Gq[k][j]:  A = R^T, B-operand = Gq^T
+  const WSet w = wset(q, q.w_sel);
+  if (split || !q.gqt_fresh) {   // (else the contraction that produced Gq already stored bf16(Gq^T))
+    split_kernel<<<tiles, 256, 0, ctx.stream>>>(Gq, q.gqt_hi, q.gqt_lo, d, 1);
+    DQ_CHECK(after_launch(ctx));
+  }
+  q.gqt_fresh = false;
   Op rt{q.rt_hi, q.rt_lo, d, dd}, gqt{q.gqt_hi, q.gqt_lo, d, dd};
-  Out ob; ob.f32 = ws.B; ob.ld = d; ob.bs = dd;
-  DQ_CHECK(gemm3(ctx, rt, gqt, d, d, d, batch, ob));
-  skew_split_kernel<<<tiles, 256, 0, ctx.stream>>>(ws.B, q.st_hi, q.st_lo, d);
-  DQ_CHECK(after_launch(ctx));
+  if (split) {
+    // B[i][j] = sum_k R[k][i] Gq[k][j]:  A = R^T, B-operand = Gq^T
+    Out ob; ob.f32 = ws.B; ob.ld = d; ob.bs = dd;
+    DQ_CHECK(gemm3(ctx, rt, gqt, d, d, d, batch, ob));
+    skew_split_kernel<<<tiles, 256, 0, ctx.stream>>>(ws.B, q.st_hi, q.st_lo, d);
+    DQ_CHECK(after_launch(ctx));
+  } else {
+    // S[i][j] = sum_k R^T[i][k] Gq^T[j][k] - sum_k Gq^T[i][k] R^T[j][k], kept for i > j
+    Out os; os.hi = q.st_hi; os.ld_h = d; os.bs_h = dd; os.gen_mode = tc::GEN_STRICT_LOWER; os.nterms = 1;
+    os.dual_a = &gqt; os.dual_b = &rt;
+    os.tile_list = q.tl_lower; os.n_list = q.n_upper; os.tile_list2 = q.tl2_lower; os.n_list2 = q.n2_upper;
+    DQ_CHECK(gemm3(ctx, rt, gqt, d, d, d, batch, os));
+  }
   // Gz = R S W^T = R D with D = S W^T lower triangular.  D^T[m][n] = sum_k W[m][k] S[n][k]: W[m][k] = 0 for
   // k < m and S[n][k] = 0 for k >= n, so only tiles mb <= nb with k in [128 mb, 128 (nb + 1)): a sixth of a
   // dense product (R S first would cost half of one).  Only the split copy of D^T is kept.
-  Op wn{q.wn_hi, q.wn_lo, d, dd}, sr{q.st_hi, q.st_lo, d, dd};
-  Out od; od.hi = q.m_hi; od.lo = q.m_lo; od.ld_h = d; od.bs_h = dd;
-  od.k_mode = 1 | 4;
-  od.tile_list = q.tl_upper; od.n_list = q.n_upper; od.tile_list2 = q.tl2_upper; od.n_list2 = q.n2_upper;
-  DQ_CHECK(gemm3(ctx, wn, sr, d, d, d, batch, od));
+  Op wnr{w.n_hi, w.n_lo, d, dd}, sr{q.st_hi, q.st_lo, d, dd};
+  Out od; od.hi = q.m_hi; od.lo = split ? q.m_lo : nullptr; od.ld_h = d; od.bs_h = dd;
+  od.k_mode = 1 | 4; upper_lists(od, q); od.nterms = split ? 3 : 1;
+  DQ_CHECK(gemm3(ctx, wnr, sr, d, d, d, batch, od));
   // (tiles below the block diagonal of D^T are neither written here nor read by the next product; the entries
   // below the diagonal inside the diagonal tiles come out as exact zeros)
   // Gz[i][j] = sum_k R[i][k] D^T[j][k]; D^T[j][k] = 0 for k < j
   Op r{q.r_hi, q.r_lo, d, dd}, dt{q.m_hi, q.m_lo, d, dd};
   Out og; og.f32 = Gz; og.ld = d; og.bs = dd;
-  og.k_mode = 8;
+  og.k_mode = 8; og.nterms = split ? 3 : 1;
   og.tile_list = q.tl_asc_nb; og.n_list = q.n_all; og.tile_list2 = q.tl2_asc_nb; og.n_list2 = q.n2_all;
   return gemm3(ctx, r, dt, d, d, d, batch, og);
 }

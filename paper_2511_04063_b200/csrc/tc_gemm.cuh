@@ -22,9 +22,14 @@ constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;          // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
-constexpr uint64_t WAIT_LIMIT_NS = 4000000000ull;
+// Limit of every in-kernel wait.  The longest legitimate wait is one output tile of the largest product
+// (256 x 256 x 65536: about half a millisecond); the limit leaves three orders of magnitude for a kernel that
+// is suspended while another context's time slice runs on a shared GPU (the timer keeps counting meanwhile).
+constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;
 
 enum { EPI_WHIP = 0, EPI_GEN = 1, EPI_BF16 = 2 };
+// What the EPI_GEN epilogue does with v = alpha * acc (see epi_gen_chunk)
+enum { GEN_LINEAR = 0, GEN_CHOL_FIRST = 1, GEN_CHOL_SWEEP = 2, GEN_STRICT_LOWER = 3, GEN_UPPER = 4 };
 
 struct Params {
   int m_blocks, n_blocks, batch, ksplit;
@@ -32,11 +37,35 @@ struct Params {
   // output addressing: out + b * batch_stride + split * split_stride + m * ld + n
   void* out;               // EPI_WHIP / EPI_BF16: bf16; EPI_GEN: fp32 (nullable)
   int64_t ld, batch_stride, split_stride;
-  // EPI_GEN only: v = alpha * acc + beta * out_old; optional split-bf16 copy (hi + lo ~ v)
+  // EPI_GEN only: v = alpha * acc + g1 * add1 + g2 * add2 (addends nullable, addressed like out; add1 may be
+  // out itself); optional split-bf16 copy (hi + lo ~ v; lo nullable) row-major (out_hi / out_lo) and transposed
+  // (element (m, n) at out_t + b * batch_stride_t + n * ld_t + m; up to two targets)
   __nv_bfloat16* out_hi;
   __nv_bfloat16* out_lo;
   int64_t ld_h, batch_stride_h;
-  float alpha, beta;
+  float alpha;
+  const float* add1; float g1;
+  const float* add2; float g2;
+  __nv_bfloat16* out_t_hi;
+  __nv_bfloat16* out_t_lo;
+  __nv_bfloat16* out_t2_hi;
+  __nv_bfloat16* out_t2_lo;
+  int64_t ld_t, batch_stride_t;
+  // gen_mode (GEN_*): GEN_LINEAR as above.  GEN_STRICT_LOWER / GEN_UPPER keep v where m > n / m <= n, 0 elsewhere.
+  // Fixed-point iteration for the upper factor I + T of a near-orthogonal matrix (T + T^T + T^T T = E), with
+  // Phi(S) = strictly upper part of S + half its diagonal:
+  //   GEN_CHOL_FIRST: acc = Zh^T Zh; e = v - I is stored to out, t = Phi(e - add1) (add1 = the previous T^T T)
+  //   GEN_CHOL_SWEEP: acc = T^T T is stored to out, t = Phi(add1 - v) (add1 = E); an entry with
+  //                   |t - aux| > tol sets *moved_out = 1 (and DQ_ERR_NOT_CONVERGED if fail_if_moved)
+  // in both t is stored to aux (fp32, addressed like out) and is the value of the bf16 copies.
+  int gen_mode;
+  float* aux;
+  float tol;
+  int* moved_out;
+  int fail_if_moved;
+  // NTERMS == 1 only: the reduction runs over two operand pairs, D = A B^T - A' B'^T with (A', B') given by
+  // the second pair of tensor maps (the MMAs of the second half negate A').
+  int k_dual;
   float* partials;         // EPI_WHIP: [unit][4] loss partial sums
   int* d_status;
   // Triangular structure (square tiles, ksplit == 1).  tri_skip: tiles below the block diagonal
@@ -49,9 +78,11 @@ struct Params {
   // most expensive tiles first so that the round-robin deal over the persistent CTAs is balanced.
   const int* tile_list;
   int n_list;
-  // Optional device flag: the kernel does nothing when *run_if == 0 (lets a fixed launch sequence, e.g. a
-  // captured graph, stop a data-dependent iteration early).  nullptr: always run.
+  // Optional device flags: the kernel does nothing when *run_if == 0 or when *run_unless != 0 (lets a fixed
+  // launch sequence, e.g. a captured graph, stop a data-dependent iteration early or choose between two
+  // variants of a product).  nullptr: no condition.
   const int* run_if;
+  const int* run_unless;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -80,14 +111,15 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: false (and DQ_ERR_TIMEOUT in the status word) after WAIT_LIMIT_NS.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* d_status) {
+// Bounded wait: false (and DQ_ERR_TIMEOUT in the status word) after limit_ns.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* d_status,
+                                          uint64_t limit_ns = WAIT_LIMIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     __nanosleep(32);   // leave the issue slots to the warps that have work
-    if ((++spins & 0xFFu) == 0u && global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+    if ((++spins & 0xFFu) == 0u && global_timer_ns() - t0 > limit_ns) {
       set_status(d_status, DQ_ERR_TIMEOUT);
       return false;
     }
@@ -159,6 +191,177 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
 }
 
+constexpr uint32_t IDESC_NEGATE_A = 1u << 13;   // kind::f16 instruction descriptor: A is negated
+
+// ----------------------------------------------------------------------------- EPI_GEN epilogue
+// The thread that owns output row `row` handles GEN_CH consecutive columns at a time.  The fp32 addends of a
+// chunk (add1, and add2 or the old aux) are fetched one chunk ahead of their use (epi_gen_fetch), so that the
+// latency of these row-per-thread loads overlaps the arithmetic and the stores of the chunk before.
+constexpr int GEN_CH = 16;
+
+struct GenAddends {
+  float4 a[GEN_CH / 4];   // add1
+  float4 b[GEN_CH / 4];   // add2 (GEN_LINEAR ...) or the old aux (GEN_CHOL_SWEEP)
+};
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+// off = offset of (row, first column of the chunk) in out / add1 / add2 / aux.
+__device__ __forceinline__ void epi_gen_fetch(const Params& p, int64_t off, GenAddends& g) {
+  const bool chol = p.gen_mode == GEN_CHOL_FIRST || p.gen_mode == GEN_CHOL_SWEEP;
+  if (p.add1) {
+    const float4* a1 = reinterpret_cast<const float4*>(p.add1 + off);
+#pragma unroll
+    for (int i = 0; i < GEN_CH / 4; ++i) g.a[i] = a1[i];
+  } else {
+#pragma unroll
+    for (int i = 0; i < GEN_CH / 4; ++i) g.a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const float* second = chol ? (p.gen_mode == GEN_CHOL_SWEEP ? p.aux : nullptr) : p.add2;
+  if (second) {
+    const float4* a2 = reinterpret_cast<const float4*>(second + off);
+#pragma unroll
+    for (int i = 0; i < GEN_CH / 4; ++i) g.b[i] = a2[i];
+  } else {
+#pragma unroll
+    for (int i = 0; i < GEN_CH / 4; ++i) g.b[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+}
+
+// v[i] = accumulator of column col0 + i of output row `row` (problem b); g = the chunk's addends.
+__device__ __forceinline__ void epi_gen_chunk(const Params& p, const uint32_t (&v)[GEN_CH], int b, int row, int col0,
+                                              int64_t off, const GenAddends& g, bool& moved) {
+  constexpr int Q = GEN_CH / 4;
+  float f[GEN_CH];
+#pragma unroll
+  for (int i = 0; i < GEN_CH; ++i) f[i] = p.alpha * __uint_as_float(v[i]);
+  float* outp = reinterpret_cast<float*>(p.out);
+  if (p.gen_mode == GEN_CHOL_FIRST || p.gen_mode == GEN_CHOL_SWEEP) {
+    const bool first = p.gen_mode == GEN_CHOL_FIRST;
+    if (first) {
+#pragma unroll
+      for (int i = 0; i < GEN_CH; ++i) f[i] -= (col0 + i == row) ? 1.f : 0.f;
+    }
+    if (outp) {   // E (first) or T^T T (sweep)
+      float4* dst = reinterpret_cast<float4*>(outp + off);
+#pragma unroll
+      for (int i = 0; i < Q; ++i) dst[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+    }
+#pragma unroll
+    for (int i = 0; i < Q; ++i) {
+      const float oo[4] = {g.a[i].x, g.a[i].y, g.a[i].z, g.a[i].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int col = col0 + 4 * i + j;
+        const float sgn = first ? f[4 * i + j] - oo[j] : oo[j] - f[4 * i + j];
+        f[4 * i + j] = (col > row) ? sgn : ((col == row) ? 0.5f * sgn : 0.f);
+      }
+      if (!first) {
+        const float od[4] = {g.b[i].x, g.b[i].y, g.b[i].z, g.b[i].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (!(fabsf(f[4 * i + j] - od[j]) <= p.tol)) moved = true;
+      }
+    }
+    float4* axw = reinterpret_cast<float4*>(p.aux + off);
+#pragma unroll
+    for (int i = 0; i < Q; ++i) axw[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+  } else {
+    if (p.add1) {
+#pragma unroll
+      for (int i = 0; i < Q; ++i) {
+        f[4 * i] = fmaf(p.g1, g.a[i].x, f[4 * i]); f[4 * i + 1] = fmaf(p.g1, g.a[i].y, f[4 * i + 1]);
+        f[4 * i + 2] = fmaf(p.g1, g.a[i].z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.g1, g.a[i].w, f[4 * i + 3]);
+      }
+    }
+    if (p.add2) {
+#pragma unroll
+      for (int i = 0; i < Q; ++i) {
+        f[4 * i] = fmaf(p.g2, g.b[i].x, f[4 * i]); f[4 * i + 1] = fmaf(p.g2, g.b[i].y, f[4 * i + 1]);
+        f[4 * i + 2] = fmaf(p.g2, g.b[i].z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.g2, g.b[i].w, f[4 * i + 3]);
+      }
+    }
+    if (p.gen_mode == GEN_STRICT_LOWER) {
+#pragma unroll
+      for (int i = 0; i < GEN_CH; ++i) f[i] = (row > col0 + i) ? f[i] : 0.f;
+    } else if (p.gen_mode == GEN_UPPER) {
+#pragma unroll
+      for (int i = 0; i < GEN_CH; ++i) f[i] = (row <= col0 + i) ? f[i] : 0.f;
+    }
+    if (outp) {
+      float4* dst = reinterpret_cast<float4*>(outp + off);
+#pragma unroll
+      for (int i = 0; i < Q; ++i) dst[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+    }
+  }
+  if (p.out_hi || p.out_t_hi || p.out_t2_hi) {
+    uint32_t ph[GEN_CH / 2], pl[GEN_CH / 2];
+#pragma unroll
+    for (int i = 0; i < GEN_CH / 2; ++i) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      const float2 hf = __bfloat1622float2(h);
+      const __nv_bfloat162 l = __floats2bfloat162_rn(f[2 * i] - hf.x, f[2 * i + 1] - hf.y);
+      ph[i] = *reinterpret_cast<const uint32_t*>(&h);
+      pl[i] = *reinterpret_cast<const uint32_t*>(&l);
+    }
+    if (p.out_hi) {
+      const int64_t off_h = (int64_t)b * p.batch_stride_h + (int64_t)row * p.ld_h + col0;
+      uint4* dh = reinterpret_cast<uint4*>(p.out_hi + off_h);
+#pragma unroll
+      for (int i = 0; i < GEN_CH / 8; ++i) dh[i] = make_uint4(ph[4 * i], ph[4 * i + 1], ph[4 * i + 2], ph[4 * i + 3]);
+      if (p.out_lo) {
+        uint4* dl = reinterpret_cast<uint4*>(p.out_lo + off_h);
+#pragma unroll
+        for (int i = 0; i < GEN_CH / 8; ++i) dl[i] = make_uint4(pl[4 * i], pl[4 * i + 1], pl[4 * i + 2], pl[4 * i + 3]);
+      }
+    }
+    if (p.out_t_hi || p.out_t2_hi) {
+      // transposed copies: for a fixed column the 32 lanes of the warp (consecutive rows) store 64 contiguous bytes
+      const int64_t off_t = (int64_t)b * p.batch_stride_t + (int64_t)col0 * p.ld_t + row;
+      unsigned short* th = reinterpret_cast<unsigned short*>(p.out_t_hi);
+      unsigned short* tl = reinterpret_cast<unsigned short*>(p.out_t_lo);
+      unsigned short* th2 = reinterpret_cast<unsigned short*>(p.out_t2_hi);
+      unsigned short* tl2 = reinterpret_cast<unsigned short*>(p.out_t2_lo);
+#pragma unroll
+      for (int i = 0; i < GEN_CH; ++i) {
+        const unsigned short hv = (unsigned short)((i & 1) ? (ph[i >> 1] >> 16) : (ph[i >> 1] & 0xffffu));
+        const unsigned short lv = (unsigned short)((i & 1) ? (pl[i >> 1] >> 16) : (pl[i >> 1] & 0xffffu));
+        const int64_t o = off_t + (int64_t)i * p.ld_t;
+        if (th) th[o] = hv;
+        if (tl) tl[o] = lv;
+        if (th2) th2[o] = hv;
+        if (tl2) tl2[o] = lv;
+      }
+    }
+  }
+}
+
+// The EPI_GEN epilogue of one accumulator (N_COLS columns at TMEM address taddr, this warp's lane quarter
+// already selected) for output row `row`; out_off = offset of (row, first column of the tile).
+template <int N_COLS>
+__device__ __forceinline__ void epi_gen_tile(const Params& p, uint32_t taddr, int b, int row, int col_base,
+                                             int64_t out_off, const GenAddends& first_chunk, bool& moved) {
+  GenAddends cur = first_chunk;
+#pragma unroll 1
+  for (int c = 0; c < N_COLS / GEN_CH; ++c) {
+    uint32_t v[GEN_CH];
+    tmem_ld16(taddr + (uint32_t)(c * GEN_CH), v);
+    GenAddends next;
+    if (c + 1 < N_COLS / GEN_CH) epi_gen_fetch(p, out_off + (c + 1) * GEN_CH, next);
+    tmem_ld_wait();
+    epi_gen_chunk(p, v, b, row, col_base + c * GEN_CH, out_off + c * GEN_CH, cur, moved);
+    cur = next;
+  }
+}
+
 __device__ __forceinline__ float fast_exp_neg_abs(float o) {
   float r;
   const float t = -fabsf(o) * 1.4426950408889634f;
@@ -183,7 +386,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapB_lo,
                const Params p) {
-  if (p.run_if && *p.run_if == 0) return;                     // uniform over the grid: nothing is allocated yet
+  if ((p.run_if && *p.run_if == 0) || (p.run_unless && *p.run_unless != 0)) return;   // uniform over the grid
   using L = SmemLayout<BLOCK_N, NTERMS>;
   constexpr int STAGES = L::STAGES;
   constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;                 // 256 or 512: power of two
@@ -207,7 +410,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tensormap(&mapA);
     prefetch_tensormap(&mapB);
-    if (NTERMS > 1) { prefetch_tensormap(&mapA_lo); prefetch_tensormap(&mapB_lo); }
+    if (NTERMS > 1 || p.k_dual) { prefetch_tensormap(&mapA_lo); prefetch_tensormap(&mapB_lo); }
   }
   if (warp == 1) tmem_alloc(tmem_slot, TMEM_COLS);
   tc_fence_before();
@@ -252,14 +455,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         if (p.tri_skip && mb > nb) continue;
         int k0, kb_per_split;
         k_range(split, mb, nb, k0, kb_per_split);
-        for (int kb = 0; kb < kb_per_split; ++kb) {
+        const int kb_total = (NTERMS == 1 && p.k_dual) ? 2 * kb_per_split : kb_per_split;
+        for (int kb = 0; kb < kb_total; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), L::STAGE_BYTES);
           const uint32_t sa = smem_base + stage * L::STAGE_BYTES;
           const uint32_t sb = sa + L::NOPS * L::A_BYTES;
-          const int kc = (k0 + kb) * BLOCK_K;
-          tma_load_3d(sa, &mapA, full_bar(stage), kc, mb * BLOCK_M, b);
-          tma_load_3d(sb, &mapB, full_bar(stage), kc, nb * BLOCK_N, b);
+          const bool second = kb >= kb_per_split;          // second operand pair of a dual reduction
+          const int kc = (k0 + (second ? kb - kb_per_split : kb)) * BLOCK_K;
+          tma_load_3d(sa, second ? &mapA_lo : &mapA, full_bar(stage), kc, mb * BLOCK_M, b);
+          tma_load_3d(sb, second ? &mapB_lo : &mapB, full_bar(stage), kc, nb * BLOCK_N, b);
           if (NTERMS > 1) {
             tma_load_3d(sa + L::A_BYTES, &mapA_lo, full_bar(stage), kc, mb * BLOCK_M, b);
             tma_load_3d(sb + L::B_BYTES, &mapB_lo, full_bar(stage), kc, nb * BLOCK_N, b);
@@ -287,16 +492,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BLOCK_N);
-        for (int kb = 0; kb < kb_per_split; ++kb) {
+        const int kb_total = (NTERMS == 1 && p.k_dual) ? 2 * kb_per_split : kb_per_split;
+        for (int kb = 0; kb < kb_total; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, p.d_status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * L::STAGE_BYTES;
           const uint32_t sb = sa + L::NOPS * L::A_BYTES;
+          const uint32_t idesc = (kb >= kb_per_split) ? (IDESC | IDESC_NEGATE_A) : IDESC;
 #pragma unroll
           for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
             const uint64_t a_hi = make_kmajor_sw128_desc(sa + k * UMMA_K * 2);
             const uint64_t b_hi = make_kmajor_sw128_desc(sb + k * UMMA_K * 2);
-            umma_bf16(tmem_d, a_hi, b_hi, IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+            umma_bf16(tmem_d, a_hi, b_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             if (NTERMS > 1) {
               const uint64_t a_lo = make_kmajor_sw128_desc(sa + L::A_BYTES + k * UMMA_K * 2);
               const uint64_t b_lo = make_kmajor_sw128_desc(sb + L::B_BYTES + k * UMMA_K * 2);
@@ -329,83 +536,41 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       const int row = mb * BLOCK_M + q * 32 + lane;
       const int64_t out_off = (int64_t)b * p.batch_stride + (int64_t)split * p.split_stride +
                               (int64_t)row * p.ld + (int64_t)nb * BLOCK_N;
-      // Accumulating epilogue (beta != 0): fetch the old output row while the MMAs of this tile
-      // are still running, so the global-load latency is not paid once per 32-column chunk.
-      constexpr bool PREFETCH = (EPI == EPI_GEN && BLOCK_N == 128);
-      float4 old[PREFETCH ? 32 : 1];
-      const bool use_old = PREFETCH && p.out != nullptr && p.beta != 0.f;
-      if (PREFETCH && use_old) {
-        const float4* src = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.out) + out_off);
-#pragma unroll
-        for (int i = 0; i < (PREFETCH ? 32 : 1); ++i) old[i] = src[i];
-      }
+      // EPI_GEN: the addends of the first chunk are fetched while the MMAs of this tile are still running
+      GenAddends g0;
+      if (EPI == EPI_GEN) epi_gen_fetch(p, out_off, g0);
+      bool moved = false;
       if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
       tc_fence_after();
       float esum = 0.f;
-#pragma unroll(PREFETCH ? 4 : 1)
-      for (int c = 0; c < BLOCK_N / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BLOCK_N + c * 32), v);
-        tmem_ld_wait();
-        if (EPI == EPI_WHIP) {
-          // Eq. 4: e = exp(-|o|); dL/do = -sign(o) e, zero at o = 0; 1/N is applied later.
+      if (EPI == EPI_GEN) {
+        epi_gen_tile<BLOCK_N>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BLOCK_N), b, row,
+                              nb * BLOCK_N, out_off, g0, moved);
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BLOCK_N / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BLOCK_N + c * 32), v);
+          tmem_ld_wait();
           uint32_t packed[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
-            const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
-            esum += e0 + e1;
-            const float g0 = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
-            const float g1 = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
-            const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
-            packed[i] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_off + c * 32);
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-        } else if (EPI == EPI_GEN) {
-          float f[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) f[i] = p.alpha * __uint_as_float(v[i]);
-          if (p.out) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_off + c * 32);
-            if (p.beta != 0.f) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const float4 o = PREFETCH ? old[PREFETCH ? c * 8 + i : 0] : dst[i];
-                f[4 * i] = fmaf(p.beta, o.x, f[4 * i]); f[4 * i + 1] = fmaf(p.beta, o.y, f[4 * i + 1]);
-                f[4 * i + 2] = fmaf(p.beta, o.z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.beta, o.w, f[4 * i + 3]);
-              }
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
-          }
-          if (p.out_hi) {
-            const int64_t off_h = (int64_t)b * p.batch_stride_h + (int64_t)row * p.ld_h + (int64_t)nb * BLOCK_N + c * 32;
-            uint32_t ph[16], pl[16];
+          if (EPI == EPI_WHIP) {
+            // Eq. 4: e = exp(-|o|); dL/do = -sign(o) e, zero at o = 0; 1/N is applied later.
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-              const float2 hf = __bfloat1622float2(h);
-              const __nv_bfloat162 l = __floats2bfloat162_rn(f[2 * i] - hf.x, f[2 * i + 1] - hf.y);
-              ph[i] = *reinterpret_cast<const uint32_t*>(&h);
-              pl[i] = *reinterpret_cast<const uint32_t*>(&l);
+              const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
+              const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
+              esum += e0 + e1;
+              const float g0v = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
+              const float g1v = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
+              const __nv_bfloat162 h = __floats2bfloat162_rn(g0v, g1v);
+              packed[i] = *reinterpret_cast<const uint32_t*>(&h);
             }
-            uint4* dh = reinterpret_cast<uint4*>(p.out_hi + off_h);
-            uint4* dl = reinterpret_cast<uint4*>(p.out_lo + off_h);
+          } else {   // EPI_BF16: plain bf16 store
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              dh[i] = make_uint4(ph[4 * i], ph[4 * i + 1], ph[4 * i + 2], ph[4 * i + 3]);
-              dl[i] = make_uint4(pl[4 * i], pl[4 * i + 1], pl[4 * i + 2], pl[4 * i + 3]);
+            for (int i = 0; i < 16; ++i) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+              packed[i] = *reinterpret_cast<const uint32_t*>(&h);
             }
-          }
-        } else {
-          uint32_t packed[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-            packed[i] = *reinterpret_cast<const uint32_t*>(&h);
           }
           uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_off + c * 32);
 #pragma unroll
@@ -416,6 +581,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));      // this warp is done with the accumulator
+      if (EPI == EPI_GEN && moved) {
+        if (p.moved_out) *p.moved_out = 1;
+        if (p.fail_if_moved) set_status(p.d_status, DQ_ERR_NOT_CONVERGED);
+      }
       if (EPI == EPI_WHIP) {
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) esum += __shfl_xor_sync(0xffffffffu, esum, off);

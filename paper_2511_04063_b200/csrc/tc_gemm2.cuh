@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapB_lo,
                 const Params p) {
-  if (p.run_if && *p.run_if == 0) return;           // uniform over the grid (both CTAs of every pair)
+  if ((p.run_if && *p.run_if == 0) || (p.run_unless && *p.run_unless != 0)) return;   // uniform over the grid (both CTAs of every pair)
   using L = PairSmem<NTERMS>;
   constexpr int STAGES = L::STAGES;
   constexpr int STAGE_BYTES = L::STAGE_BYTES;
@@ -120,7 +120,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tensormap(&mapA);
     prefetch_tensormap(&mapB);
-    if (NTERMS > 1) { prefetch_tensormap(&mapA_lo); prefetch_tensormap(&mapB_lo); }
+    if (NTERMS > 1 || p.k_dual) { prefetch_tensormap(&mapA_lo); prefetch_tensormap(&mapB_lo); }
   }
   if (warp == 1) tmem_alloc_pair(tmem_slot, TMEM_COLS);
   tc_fence_before();
@@ -165,14 +165,16 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         if (p.tri_skip && mb > nb) continue;
         int k0, kn;
         k_range(split, mb, nb, k0, kn);
-        for (int kb = 0; kb < kn; ++kb) {
+        const int kb_total = (NTERMS == 1 && p.k_dual) ? 2 * kn : kn;
+        for (int kb = 0; kb < kb_total; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
           if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + L::NOPS * A_BYTES;
-          const int kc = (k0 + kb) * BLOCK_K;
-          tma_load_3d_pair(sa, &mapA, full_bar(stage), kc, mb * PAIR_M + (int)rank * HALF, b);
-          tma_load_3d_pair(sb, &mapB, full_bar(stage), kc, nb * PAIR_N + (int)rank * HALF, b);
+          const bool second = kb >= kn;                     // second operand pair of a dual reduction
+          const int kc = (k0 + (second ? kb - kn : kb)) * BLOCK_K;
+          tma_load_3d_pair(sa, second ? &mapA_lo : &mapA, full_bar(stage), kc, mb * PAIR_M + (int)rank * HALF, b);
+          tma_load_3d_pair(sb, second ? &mapB_lo : &mapB, full_bar(stage), kc, nb * PAIR_N + (int)rank * HALF, b);
           if (NTERMS > 1) {
             tma_load_3d_pair(sa + A_BYTES, &mapA_lo, full_bar(stage), kc, mb * PAIR_M + (int)rank * HALF, b);
             tma_load_3d_pair(sb + B_BYTES, &mapB_lo, full_bar(stage), kc, nb * PAIR_N + (int)rank * HALF, b);
@@ -198,16 +200,18 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * PAIR_N);
-        for (int kb = 0; kb < kn; ++kb) {
+        const int kb_total = (NTERMS == 1 && p.k_dual) ? 2 * kn : kn;
+        for (int kb = 0; kb < kb_total; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, p.d_status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + L::NOPS * A_BYTES;
+          const uint32_t idesc = (kb >= kn) ? (IDESC | IDESC_NEGATE_A) : IDESC;
 #pragma unroll
           for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
             const uint64_t a_hi = make_kmajor_sw128_desc(sa + k * UMMA_K * 2);
             const uint64_t b_hi = make_kmajor_sw128_desc(sb + k * UMMA_K * 2);
-            umma_bf16_pair(tmem_d, a_hi, b_hi, IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+            umma_bf16_pair(tmem_d, a_hi, b_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             if (NTERMS > 1) {
               const uint64_t a_lo = make_kmajor_sw128_desc(sa + A_BYTES + k * UMMA_K * 2);
               const uint64_t b_lo = make_kmajor_sw128_desc(sb + B_BYTES + k * UMMA_K * 2);
@@ -236,86 +240,58 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       int mb, nb;
       tile_of(t % tiles_per_batch, mb, nb);
       if (p.tri_skip && mb > nb) continue;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
-      tc_fence_after();
       const int row = mb * PAIR_M + (int)rank * HALF + q * 32 + lane;
       const int64_t out_off = (int64_t)b * p.batch_stride + (int64_t)split * p.split_stride + (int64_t)row * p.ld +
                               (int64_t)nb * PAIR_N;
+      // EPI_GEN: the addends of the first chunk are fetched while the MMAs of this tile are still running
+      GenAddends g0;
+      if (EPI == EPI_GEN) epi_gen_fetch(p, out_off, g0);
+      if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
+      tc_fence_after();
       float esum = 0.f;
+      bool moved = false;
+      if (EPI == EPI_GEN) {
+        epi_gen_tile<PAIR_N>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * PAIR_N), b, row, nb * PAIR_N,
+                             out_off, g0, moved);
+      } else {
 #pragma unroll 1
-      for (int c = 0; c < PAIR_N / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * PAIR_N + c * 32), v);
-        tmem_ld_wait();
-        if (EPI == EPI_WHIP) {
-          // Eq. 4: e = exp(-|o|); dL/do = -sign(o) e, zero at o = 0; 1/N is applied later.
+        for (int c = 0; c < PAIR_N / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * PAIR_N + c * 32), v);
+          tmem_ld_wait();
           uint32_t packed[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
-            const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
-            esum += e0 + e1;
-            const float g0 = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
-            const float g1 = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
-            const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
-            packed[i] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_off + c * 32);
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-        } else if (EPI == EPI_BF16) {   // plain bf16 store
-          uint32_t packed[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-            packed[i] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_off + c * 32);
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-        } else {   // EPI_GEN: alpha * acc (+ beta * old) as fp32 and / or as a split-bf16 copy
-          float f[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) f[i] = p.alpha * __uint_as_float(v[i]);
-          if (p.out) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + out_off + c * 32);
-            if (p.beta != 0.f) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const float4 o = dst[i];
-                f[4 * i] = fmaf(p.beta, o.x, f[4 * i]); f[4 * i + 1] = fmaf(p.beta, o.y, f[4 * i + 1]);
-                f[4 * i + 2] = fmaf(p.beta, o.z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.beta, o.w, f[4 * i + 3]);
-              }
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
-          }
-          if (p.out_hi) {
-            const int64_t off_h = (int64_t)b * p.batch_stride_h + (int64_t)row * p.ld_h + (int64_t)nb * PAIR_N + c * 32;
-            uint32_t ph[16], pl[16];
+          if (EPI == EPI_WHIP) {
+            // Eq. 4: e = exp(-|o|); dL/do = -sign(o) e, zero at o = 0; 1/N is applied later.
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-              const float2 hf = __bfloat1622float2(h);
-              const __nv_bfloat162 l = __floats2bfloat162_rn(f[2 * i] - hf.x, f[2 * i + 1] - hf.y);
-              ph[i] = *reinterpret_cast<const uint32_t*>(&h);
-              pl[i] = *reinterpret_cast<const uint32_t*>(&l);
+              const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
+              const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
+              esum += e0 + e1;
+              const float g0v = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
+              const float g1v = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
+              const __nv_bfloat162 h = __floats2bfloat162_rn(g0v, g1v);
+              packed[i] = *reinterpret_cast<const uint32_t*>(&h);
             }
-            uint4* dh = reinterpret_cast<uint4*>(p.out_hi + off_h);
-            uint4* dl = reinterpret_cast<uint4*>(p.out_lo + off_h);
+          } else {   // EPI_BF16: plain bf16 store
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              dh[i] = make_uint4(ph[4 * i], ph[4 * i + 1], ph[4 * i + 2], ph[4 * i + 3]);
-              dl[i] = make_uint4(pl[4 * i], pl[4 * i + 1], pl[4 * i + 2], pl[4 * i + 3]);
+            for (int i = 0; i < 16; ++i) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+              packed[i] = *reinterpret_cast<const uint32_t*>(&h);
             }
           }
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + out_off + c * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
         }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(tempty_bar(acc));   // eight arrivals (four warps of each CTA) free the accumulator
+      if (EPI == EPI_GEN && moved) {
+        if (p.moved_out) *p.moved_out = 1;
+        if (p.fail_if_moved) set_status(p.d_status, DQ_ERR_NOT_CONVERGED);
+      }
       if (EPI == EPI_WHIP) {
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) esum += __shfl_xor_sync(0xffffffffu, esum, off);

@@ -109,7 +109,7 @@ inline dq_status rotate_tokens(Ctx& ctx, const void* X, int64_t n, int d, int64_
   CUtensorMap ma, mb;
   tc::Params p{};
   p.batch = 1; p.ksplit = 1; p.k_blocks = d / tc::BLOCK_K;
-  p.out = out; p.ld = ldo; p.alpha = 1.f; p.beta = 0.f; p.d_status = d_status;
+  p.out = out; p.ld = ldo; p.alpha = 1.f; p.d_status = d_status;
   if (d % 256 == 0 && n % 256 == 0 && ctx.sm_count >= 2) {
     DQ_CHECK(make_map(&ma, X, d, n, 1, ldx, n * ldx, tc2::HALF));
     DQ_CHECK(make_map(&mb, rt, d, d, 1, d, (int64_t)d * d, tc2::HALF));
@@ -129,16 +129,44 @@ struct Op {   // K-major operand: rows x K, split pair, leading dimension, batch
 struct Out {
   float* f32 = nullptr; int64_t ld = 0; int64_t bs = 0;
   bf16* hi = nullptr; bf16* lo = nullptr; int64_t ld_h = 0; int64_t bs_h = 0;
-  float alpha = 1.f, beta = 0.f;
-  // split-K: slice s of the reduction writes alpha * partial product (beta must be 0, no
-  // split copy) to f32 + s * split_stride; the caller reduces.
+  float alpha = 1.f, beta = 0.f;             // beta: the old contents of f32 are added (shorthand for add1 = f32)
+  // v = alpha * acc + g1 * add1 + g2 * add2: fp32 matrices addressed like f32 (same ld / bs)
+  const float* add1 = nullptr; float g1 = 1.f;
+  const float* add2 = nullptr; float g2 = 1.f;
+  // transposed split copies (element (m, n) at n * ld_t + m), up to two targets; lo parts nullable
+  bf16* t_hi = nullptr; bf16* t_lo = nullptr; bf16* t2_hi = nullptr; bf16* t2_lo = nullptr;
+  int64_t ld_t = 0; int64_t bs_t = 0;
+  int gen_mode = tc::GEN_LINEAR;             // see tc::Params
+  float* aux = nullptr; float tol = 0.f; int* moved_out = nullptr; int fail_if_moved = 0;
+  // split-K: slice s of the reduction writes alpha * partial product (no addends, no split copy) to
+  // f32 + s * split_stride; the caller reduces.
   int ksplit = 1; int64_t split_stride = 0;
   int tri_skip = 0, k_mode = 0;   // triangular structure, see tc::Params
   const int* tile_list = nullptr; int n_list = 0;   // explicit tile order (device), see tc::Params
   const int* tile_list2 = nullptr; int n_list2 = 0; // the same order in 256 x 256 tiles (two-CTA kernel)
   int nterms = 3;   // 1: plain bf16 product of the hi parts only (2^-9 relative), a third of the MMAs
-  const int* run_if = nullptr;   // device flag: skip the product when it is 0 (see tc::Params)
+  // nterms == 1 only: D = A B^T - A2 B2^T in one reduction (second operand pair, same shapes)
+  const Op* dual_a = nullptr; const Op* dual_b = nullptr;
+  const int* run_if = nullptr;       // device flag: skip the product when it is 0 (see tc::Params)
+  const int* run_unless = nullptr;   // device flag: skip the product when it is not 0
 };
+
+inline void fill_epilogue(tc::Params& p, const Out& o) {
+  p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = o.split_stride;
+  p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
+  p.alpha = o.alpha;
+  p.add1 = o.add1; p.g1 = o.g1; p.add2 = o.add2; p.g2 = o.g2;
+  if (o.beta != 0.f) {   // the output accumulates: its old contents are the (first free) addend
+    if (!p.add1) { p.add1 = o.f32; p.g1 = o.beta; } else { p.add2 = o.f32; p.g2 = o.beta; }
+  }
+  p.out_t_hi = o.t_hi; p.out_t_lo = o.t_lo; p.out_t2_hi = o.t2_hi; p.out_t2_lo = o.t2_lo;
+  p.ld_t = o.ld_t; p.batch_stride_t = o.bs_t;
+  p.gen_mode = o.gen_mode; p.aux = o.aux; p.tol = o.tol; p.moved_out = o.moved_out; p.fail_if_moved = o.fail_if_moved;
+  p.k_dual = (o.dual_a && o.dual_b) ? 1 : 0;
+  p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
+  p.run_if = o.run_if; p.run_unless = o.run_unless;
+  p.partials = nullptr;
+}
 
 // 64-wide k-blocks the kernels run for a product: the same clipping as their k_range, over all tiles or
 // (upper) over the tiles with mb <= nb.  unit = tile edge (128 or 256).
@@ -162,53 +190,48 @@ inline int64_t count_kblocks(int m_tiles, int n_tiles, int k_blocks, int k_mode,
 // product, fp32 accumulation); M, N % 128 == 0, K % 64 == 0.
 inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, int batch, const Out& o) {
   if (M % 128 || N % 128 || K % 64 || o.ksplit < 1 || o.ksplit > K / 64) return DQ_ERR_UNSUPPORTED;
+  if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
+  const bool dual = o.dual_a && o.dual_b;
+  if (dual && (o.nterms != 1 || o.k_mode || o.ksplit != 1)) return DQ_ERR_UNSUPPORTED;
+  if (o.ksplit > 1 && (o.add1 || o.add2 || o.beta != 0.f || o.hi || o.t_hi || o.gen_mode != tc::GEN_LINEAR))
+    return DQ_ERR_UNSUPPORTED;
+  // second pair of tensor maps: the lo parts of a split product, or the second operand pair of a dual one
+  const bf16* a2 = dual ? o.dual_a->hi : (o.nterms == 1 ? A.hi : A.lo);
+  const bf16* b2 = dual ? o.dual_b->hi : (o.nterms == 1 ? B.hi : B.lo);
+  const int64_t lda2 = dual ? o.dual_a->ld : A.ld, ldb2 = dual ? o.dual_b->ld : B.ld;
   CUtensorMap ma, mal, mb, mbl;
   const int64_t bsa = A.bs ? A.bs : (int64_t)M * A.ld, bsb = B.bs ? B.bs : (int64_t)N * B.ld;
+  const int64_t bsa2 = dual ? (o.dual_a->bs ? o.dual_a->bs : (int64_t)M * lda2) : bsa;
+  const int64_t bsb2 = dual ? (o.dual_b->bs ? o.dual_b->bs : (int64_t)N * ldb2) : bsb;
   // Large products run on CTA pairs (256 x 256 tiles, half the operand traffic per MMA); a caller that
   // orders its tiles must also give the order in pair tiles.
-  const bool pair_ok = M % 256 == 0 && N % 256 == 0 && (!o.tile_list || o.tile_list2) &&
+  const bool pair_ok = M % 256 == 0 && N % 256 == 0 && (!o.tile_list || o.tile_list2) && ctx.sm_count >= 2 &&
                        (int64_t)(M / 256) * (N / 256) * batch * o.ksplit >= 32;
-  if (pair_ok) {
-    if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
-    DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, tc2::HALF));
-    DQ_CHECK(make_map(&mal, A.lo, K, M, batch, A.ld, bsa, tc2::HALF));
-    DQ_CHECK(make_map(&mb, B.hi, K, N, batch, B.ld, bsb, tc2::HALF));
-    DQ_CHECK(make_map(&mbl, B.lo, K, N, batch, B.ld, bsb, tc2::HALF));
-    tc::Params p{};
-    p.m_blocks = M / 256; p.n_blocks = N / 256; p.batch = batch; p.ksplit = o.ksplit; p.k_blocks = K / tc::BLOCK_K;
-    p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = o.split_stride;
-    p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
-    p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
-    p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
-    p.tile_list = o.tile_list2; p.n_list = o.n_list2; p.run_if = o.run_if;
-    {
-      const bool upper = o.tri_skip || (o.tile_list2 && o.n_list2 < p.m_blocks * p.n_blocks);
-      if (!o.run_if)   // products that a device flag may skip are left out of the count
-        ctx.mma_flops += (double)count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode, upper, 256) *
-                         (2.0 * 256 * 256 * tc::BLOCK_K) * (o.nterms == 1 ? 1 : 3) * batch;
-    }
-    return o.nterms == 1 ? launch_gemm2<1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
-                         : launch_gemm2<3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
-  }
-  DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, tc::BLOCK_M));
-  DQ_CHECK(make_map(&mal, A.lo, K, M, batch, A.ld, bsa, tc::BLOCK_M));
-  DQ_CHECK(make_map(&mb, B.hi, K, N, batch, B.ld, bsb, 128));
-  DQ_CHECK(make_map(&mbl, B.lo, K, N, batch, B.ld, bsb, 128));
+  const int unit = pair_ok ? 256 : 128;
+  const int box = pair_ok ? tc2::HALF : 128;
+  DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, pair_ok ? tc2::HALF : tc::BLOCK_M));
+  DQ_CHECK(make_map(&mal, a2, K, M, batch, lda2, bsa2, pair_ok ? tc2::HALF : tc::BLOCK_M));
+  DQ_CHECK(make_map(&mb, B.hi, K, N, batch, B.ld, bsb, box));
+  DQ_CHECK(make_map(&mbl, b2, K, N, batch, ldb2, bsb2, box));
   tc::Params p{};
-  p.m_blocks = M / 128; p.n_blocks = N / 128; p.batch = batch; p.ksplit = o.ksplit; p.k_blocks = K / tc::BLOCK_K;
-  p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = o.split_stride;
-  p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
-  p.alpha = o.alpha; p.beta = o.beta; p.partials = nullptr; p.d_status = ctx.d_status;
-  if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
-  p.tri_skip = o.tri_skip; p.k_mode = o.k_mode;
-  p.tile_list = o.tile_list; p.n_list = o.n_list; p.run_if = o.run_if;
+  p.m_blocks = M / unit; p.n_blocks = N / unit; p.batch = batch; p.ksplit = o.ksplit; p.k_blocks = K / tc::BLOCK_K;
+  fill_epilogue(p, o);
+  p.d_status = ctx.d_status;
+  p.tile_list = pair_ok ? o.tile_list2 : o.tile_list;
+  p.n_list = pair_ok ? o.n_list2 : o.n_list;
   {
-    const bool upper = o.tri_skip || (o.tile_list && o.n_list < p.m_blocks * p.n_blocks);
-    if (!o.run_if)
-      ctx.mma_flops += (double)count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode, upper, 128) *
-                       (2.0 * 128 * 128 * tc::BLOCK_K) * (o.nterms == 1 ? 1 : 3) * batch;
+    const bool listed = p.tile_list && p.n_list < p.m_blocks * p.n_blocks;
+    if (!o.run_if && !o.run_unless) {   // products that a device flag may skip are left out of the count
+      const int64_t kb = listed && !o.k_mode ? (int64_t)p.n_list * p.k_blocks
+                                             : count_kblocks(p.m_blocks, p.n_blocks, p.k_blocks, o.k_mode,
+                                                             o.tri_skip || listed, unit);
+      ctx.mma_flops += (double)kb * (2.0 * unit * unit * tc::BLOCK_K) * (dual ? 2 : (o.nterms == 1 ? 1 : 3)) * batch;
+    }
   }
-  return o.nterms == 1 ? launch_gemm<128, 1, tc::EPI_GEN>(ctx, ma, mb, ma, mb, p)
+  if (pair_ok)
+    return o.nterms == 1 ? launch_gemm2<1, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p)
+                         : launch_gemm2<3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
+  return o.nterms == 1 ? launch_gemm<128, 1, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p)
                        : launch_gemm<128, 3, tc::EPI_GEN>(ctx, ma, mb, mal, mbl, p);
 }
 

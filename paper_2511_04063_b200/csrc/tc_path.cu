@@ -37,22 +37,44 @@ __global__ void __launch_bounds__(256) transpose_f32_to_bf16_kernel(const float*
 
 // out tile = sum over slices of part[slice] tile, for the tiles of `list` (mb | nb << 16; tiles
 // are bm x bn); gridDim.y CTAs per tile (a band of rows each), fixed summation order.
+// out_t (nullable): also the bf16 transpose, out_t[c][r] = bf16(out[r][c]).
 __global__ void __launch_bounds__(256) tile_reduce_kernel(const float* __restrict__ part, int slices,
                                                           int64_t slice_stride, const int* __restrict__ list, int bm,
-                                                          int bn, int d, float* __restrict__ out) {
+                                                          int bn, int d, float* __restrict__ out,
+                                                          __nv_bfloat16* __restrict__ out_t) {
   const int code = list[blockIdx.x];
   const int band = bm / gridDim.y;
   const int r0 = (code & 0xffff) * bm + blockIdx.y * band, c0 = (code >> 16) * bn;
   const int per_row = bn / 4;
   for (int e = threadIdx.x; e < band * per_row; e += 256) {
-    const int64_t idx = (int64_t)(r0 + e / per_row) * d + c0 + (e % per_row) * 4;
+    const int r = r0 + e / per_row, c = c0 + (e % per_row) * 4;
+    const int64_t idx = (int64_t)r * d + c;
     float4 s = *reinterpret_cast<const float4*>(part + idx);
     for (int k = 1; k < slices; ++k) {
       const float4 t = *reinterpret_cast<const float4*>(part + (int64_t)k * slice_stride + idx);
       s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
     }
     *reinterpret_cast<float4*>(out + idx) = s;
+    if (out_t) {
+      out_t[(int64_t)c * d + r] = __float2bfloat16_rn(s.x);
+      out_t[(int64_t)(c + 1) * d + r] = __float2bfloat16_rn(s.y);
+      out_t[(int64_t)(c + 2) * d + r] = __float2bfloat16_rn(s.z);
+      out_t[(int64_t)(c + 3) * d + r] = __float2bfloat16_rn(s.w);
+    }
   }
+}
+
+// One thread waits, with the bounded wait every tcgen05 kernel of the library uses, on a barrier that nothing
+// ever arrives at (no copy or MMA is in flight): the wait must give up after limit_ns, record DQ_ERR_TIMEOUT
+// and let the kernel return normally.  waited_ns receives how long it waited.
+__global__ void bounded_wait_probe_kernel(uint64_t limit_ns, int* d_status, uint64_t* waited_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  const uint32_t b = tc::smem_u32(&bar);
+  tc::mbar_init(b, 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  const uint64_t t0 = tc::global_timer_ns();
+  const bool done = tc::mbar_wait(b, 0u, d_status, limit_ns);
+  if (waited_ns) *waited_ns = done ? 0ull : tc::global_timer_ns() - t0;
 }
 
 struct Maps {
@@ -183,7 +205,10 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
 }
 
 // Gq = scale * X^T G : A = X^T [d][N], B = G^T [d][N], reduction over tokens.
-dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
+// gqt (nullable): the epilogue also stores bf16(Gq^T) there (the operand of the QR-Orth backward);
+// *gqt_written tells whether this schedule could (the split-K schedule of small shapes cannot).
+dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale, __nv_bfloat16* gqt, bool* gqt_written) {
+  if (gqt_written) *gqt_written = false;
   if (tc.fused && tc.fused_valid)   // the fused kernel left one partial per unit: sum them in a fixed order
     return splitk_reduce(ctx, tc.heads_part, tc.splits, (int64_t)tc.d * tc.d, tc.batch, scale, 0.f, Gq);
   ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;
@@ -193,7 +218,7 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
   tc::Params p{};
   p.m_blocks = d / tc::BLOCK_M; p.n_blocks = d / bn; p.batch = tc.batch; p.ksplit = tc.ksplit;
   p.k_blocks = (int)(tc.n_tokens / tc::BLOCK_K);
-  p.ld = d; p.alpha = scale; p.beta = 0.f; p.out_hi = nullptr; p.out_lo = nullptr;
+  p.ld = d; p.alpha = scale; p.out_hi = nullptr; p.out_lo = nullptr;
   p.partials = nullptr; p.d_status = ctx.d_status;
   if (tc.ksplit == 1) {
     p.out = Gq; p.batch_stride = (int64_t)d * d; p.split_stride = 0;
@@ -206,6 +231,11 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
     return (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, m->xt, m->gt256, m->xt, m->gt256, pp)
                        : tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, pp);
   };
+  const bool with_t = gqt != nullptr && tc.ksplit == 1 && tc.batch == 1;
+  if (with_t) {
+    p.out_t_hi = gqt; p.ld_t = d; p.batch_stride_t = (int64_t)d * d;
+    if (gqt_written) *gqt_written = true;
+  }
   if (tc.tail_split > 1) {
     tc::Params ph = p;      // full waves: whole reduction per tile
     ph.tile_list = tc.tl_head; ph.n_list = tc.n_head;
@@ -213,9 +243,10 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale) {
     tc::Params pt = p;      // last wave: reduction in slices, then a fixed-order sum
     pt.tile_list = tc.tl_tail; pt.n_list = tc.n_tail; pt.ksplit = tc.tail_split;
     pt.out = tc.tail_part; pt.batch_stride = 0; pt.split_stride = (int64_t)d * d;
+    pt.out_t_hi = nullptr;
     DQ_CHECK(launch(pt));
     tile_reduce_kernel<<<dim3(tc.n_tail, 8), 256, 0, ctx.stream>>>(tc.tail_part, tc.tail_split, (int64_t)d * d, tc.tl_tail,
-                                                          tc.pair ? 256 : 128, bn, d, Gq);
+                                                          tc.pair ? 256 : 128, bn, d, Gq, with_t ? gqt : nullptr);
     return after_launch(ctx);
   }
   DQ_CHECK(launch(p));
@@ -243,6 +274,11 @@ dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t l
   return st;
 }
 
+
+dq_status bounded_wait_probe(Ctx& ctx, uint64_t limit_ns, uint64_t* d_waited_ns) {
+  bounded_wait_probe_kernel<<<1, 1, 0, ctx.stream>>>(limit_ns, ctx.d_status, d_waited_ns);
+  return after_launch(ctx);
+}
 
 // ---------------------------------------------------------------------------------------------
 // Y = X R without any allocation (dq_rotate_apply_static).

@@ -39,9 +39,12 @@ void tc_destroy(TcState& tc);
 dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx);   // X changed in place: rebuild X^T
 inline __nv_bfloat16* tc_rt_operand(TcState& tc) { return tc.ready ? tc.Rt : nullptr; }
 dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials);
-dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale);
+dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale, __nv_bfloat16* gqt = nullptr,
+                           bool* gqt_written = nullptr);
 dq_status tc_rotate_apply(Ctx& ctx, const void* d_X, int64_t n, int d, int64_t ldx, const float* d_R,
                           void* d_Y, int64_t ldy);
+// Failure-detection self-test: the library's bounded in-kernel wait on a barrier nobody arrives at.
+dq_status bounded_wait_probe(Ctx& ctx, uint64_t limit_ns, uint64_t* d_waited_ns);
 // Outliers (Eq. 1) and per-token asymmetric quantisation error of O = X R (eval_metrics.cu).
 dq_status eval_rotation(Ctx& ctx, const void* d_X, int x_dtype, int64_t n, int d, int64_t ldx, const float* d_R,
                         float tau, int bits, double* d_out);
@@ -63,6 +66,14 @@ struct QrTcState {
   __nv_bfloat16 *st_hi = nullptr, *st_lo = nullptr;     // S^T
   __nv_bfloat16 *m_hi = nullptr, *m_lo = nullptr;       // R S
   __nv_bfloat16 *t1_hi = nullptr, *t1_lo = nullptr;     // scratch of the block inversion
+  // second set of copies of W: the incremental update W <- W (I + T)^-1 reads one set and writes the other
+  __nv_bfloat16 *wn2_hi = nullptr, *wn2_lo = nullptr, *wt2_hi = nullptr, *wt2_lo = nullptr;
+  int w_sel = 0;                                        // the set that holds the current W (0: wn / wt, 1: wn2 / wt2)
+  float* P = nullptr;                                   // T^T T of the last sweep: where the next step's fixed point starts
+  __nv_bfloat16 *yt_hi = nullptr, *yt_lo = nullptr;     // ((I + T)^-1 - I)^T
+  __nv_bfloat16 *nm1 = nullptr, *nm2 = nullptr;         // scratch of the products that form (I + T)^-1
+  bool u_fresh = false;                                 // U and u_hi / u_lo hold the upper factor of the current factorisation
+  bool gqt_fresh = false;                               // gqt_hi holds bf16(Gq^T) of the current step (written by the contraction)
   // blocked Householder factorisation with tensor-core trailing updates
   __nv_bfloat16 *y_hi = nullptr, *y_lo = nullptr;       // [batch][d][128] reflector block Y of the outer block
   __nv_bfloat16 *w2_hi = nullptr, *w2_lo = nullptr;     // [batch][d][128] (T^T Y^T C)^T
@@ -71,26 +82,34 @@ struct QrTcState {
   float* T = nullptr;                                   // [batch][4][32][32] compact-WY factors of the inner panels
   // near-orthogonal iterative factorisation
   __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T^T of the sweeps
-  __nv_bfloat16 *uot_hi = nullptr, *uot_lo = nullptr;   // U^T of the previous step
+  __nv_bfloat16 *uot_hi = nullptr, *uot_lo = nullptr;   // T^T of the last sweep that ran
   bool z_split_fresh = false;                           // z_hi / z_lo are the split copy of the current latent
-  bool t_warm = false;                                  // wt_* / uot_* hold the factors of the previous step's latent
+  bool t_warm = false;                                  // the current set of W copies and the fp32 W belong to the previous step's latent
   int* sweep_flags = nullptr;                           // [80] device flags: sweep k moved an entry
   // tile orders for triangular products (device arrays of mb | nb << 16)
   int* tl_upper = nullptr; int n_upper = 0;             // tiles mb <= nb, largest mb first
+  int* tl_lower = nullptr;                              // tiles mb >= nb (n_upper of them)
   int* tl_desc_nb = nullptr;                            // all tiles, largest nb first
   int* tl_asc_nb = nullptr; int n_all = 0;              // all tiles, smallest nb first
   // the same orders in 256 x 256 tiles for the two-CTA kernel (d % 256 == 0 only)
   int* tl2_upper = nullptr; int n2_upper = 0;
+  int* tl2_lower = nullptr;
   int* tl2_desc_nb = nullptr;
   int* tl2_asc_nb = nullptr; int n2_all = 0;
 };
 dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count);
 void qr_tc_destroy(QrTcState& q);
-// iterative_iters > 0 and q.t_warm: U from the previous step's factors by iterative_iters fixed-point
-// sweeps (no dependent column steps); otherwise blocked Householder.
+// iterative_iters > 0 and q.t_warm: R and W = U^-1 from the previous step's W by fixed-point sweeps (no
+// dependent column steps; U itself is not formed); otherwise blocked Householder (U is written).
+// need_lo: the incremental route also writes the lo parts of the split copies of R and R^T (the Householder
+// route always does).
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
-                          int batch, int iterative_iters);
-dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch);
+                          int batch, int iterative_iters, bool need_lo);
+// Makes U hold the upper factor of the current factorisation (inverts W after incremental steps).
+dq_status qr_tc_materialize_u(Ctx& ctx, QrWorkspace& ws, QrTcState& q, float* U, int d, int batch);
+// split: three bf16 MMAs per product (split operands) instead of one.
+dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Gq, float* Gz, int d, int batch,
+                         bool split);
 
 // Alternative objectives of the ablation in Sec. 5.3 (objectives.cu).
 struct ObjectiveState {

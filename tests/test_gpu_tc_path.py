@@ -292,6 +292,7 @@ def test_incremental_qr_takes_as_many_sweeps_as_a_large_step_needs():
     w = small("c2_7b", d=512, n_tokens=1024, n_outlier_channels=3)
     c = Calib(w)
     dq.dq_calib_set_optimizer(c.h, dq.DQ_ADAM, 5e-3, 0.9, 0.999, 1e-8)
+    dq.dq_calib_set_qr_method(c.h, dq.DQ_QR_ITERATIVE, 16)          # steps this large need more than the default
     c.step(6)
     assert c.status() == dq.DQ_OK
     Z = c.latent()[0].astype(np.float64)
@@ -372,3 +373,30 @@ def test_rotate_apply_rejects_misaligned_pointers_before_any_launch():
         assert f(*args(X.data_ptr(), Y.data_ptr())) == dq.DQ_OK, entry
     torch.cuda.synchronize()
     assert float(Y.float().abs().max()) == 0.0
+
+
+def test_a_bounded_wait_that_runs_out_sets_the_status_word_and_the_kernel_returns():
+    """Failure detection without a fault: the wait every tensor-core kernel uses, given a barrier that nothing
+    arrives at and a limit of one millisecond, gives up, records DQ_ERR_TIMEOUT and returns; the context stays
+    usable, steps leave the latent alone while the status is set, and a new latent clears it."""
+    w = small("c2_7b", d=256, n_tokens=1024, n_outlier_channels=3)
+    c = Calib(w)
+    c.step(2)
+    assert c.status() == dq.DQ_OK
+    Z = c.latent()
+    waited = dq.dq_calib_selftest_bounded_wait(c.h, 1_000_000)
+    assert c.status() == dq.DQ_ERR_TIMEOUT
+    assert 1_000_000 <= waited <= 50_000_000               # gave up after the limit, not long after
+    assert "wait" in dq.status_string(dq.DQ_ERR_TIMEOUT)
+    c.step(2)                                              # the update kernels are frozen
+    assert c.status() == dq.DQ_ERR_TIMEOUT
+    assert np.array_equal(c.latent(), Z)
+    c.set_latent(Z)                                        # acknowledges the error
+    assert c.status() == dq.DQ_OK
+    c.step(1)
+    assert c.status() == dq.DQ_OK
+    assert not np.array_equal(c.latent(), Z)
+    lib = dq.load_library()
+    assert lib.dq_calib_selftest_bounded_wait(c.h, 0, None) == dq.DQ_ERR_INVALID_ARG
+    assert lib.dq_calib_selftest_bounded_wait(c.h, 10**9, None) == dq.DQ_ERR_INVALID_ARG
+    c.close()
