@@ -61,7 +61,7 @@ typedef struct {
   int32_t reduction; /* DQ_MEAN_TOKENS (default reading of Algorithm 1's loss step) | DQ_SUM_TOKENS */
   int32_t optimizer; /* DQ_SGD here; others via dq_calib_set_optimizer          */
   float lr;          /* eta                                                     */
-  int64_t ldx;       /* row stride of X in elements (>= d); problems are n_tokens*ldx apart */
+  int64_t ldx;       /* row stride of X in elements (>= d; a multiple of 8 on the tensor-core path); problems are n_tokens*ldx apart */
 } dq_calib_config;
 
 /* Algorithm 1, hand-off before the loop: bind calibration activations and the initial

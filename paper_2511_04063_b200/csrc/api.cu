@@ -16,6 +16,9 @@ using namespace dq;
 // Default number of sweeps (beyond the three that always exist) of the incremental QR-Orth on the tensor-core
 // route for d >= 256, whose fixed point starts from the previous step's T^T T and so needs few.
 constexpr int DEFAULT_QR_SWEEPS_TC = 5;
+// |Z0^T Z0 - I|_F up to which a latent counts as orthogonal at dq_calib_init (the fixed point of the incremental
+// factorisation contracts for |E|_2 well below 1/2; the Frobenius norm bounds the spectral norm)
+constexpr float ORTHOGONAL_START_THRESHOLD = 0.05f;
 
 struct dq_calib {
   dq_calib_config cfg;
@@ -114,7 +117,7 @@ dq_status validate(const dq_calib_config* c) {
     if (c->x_dtype != DQ_FP32) return DQ_ERR_UNSUPPORTED;
   } else {
     if (c->x_dtype != DQ_BF16) return DQ_ERR_UNSUPPORTED;
-    if (c->d % 128 != 0 || c->n_tokens % 256 != 0 || c->ldx != c->d) return DQ_ERR_UNSUPPORTED;
+    if (c->d % 128 != 0 || c->n_tokens % 256 != 0 || c->ldx % 8 != 0) return DQ_ERR_UNSUPPORTED;   // (TMA: 16-byte row stride)
   }
   return DQ_OK;
 }
@@ -429,6 +432,12 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
   A(dev_alloc(&h->partials, (int64_t)batch * (h->n_partials > 0 ? h->n_partials : 1)));
   if (st == DQ_OK && cudaMemsetAsync(h->ctx.d_status, 0, sizeof(int), h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
   if (st == DQ_OK && cudaMemcpyAsync(h->Z, d_Z0, sizeof(float) * dd, cudaMemcpyDeviceToDevice, h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
+  if (st == DQ_OK && h->fast_qr && !h->small128) {
+    // The paper initialises the latent with a random Hadamard matrix, which is orthogonal: then U = I and the
+    // incremental factorisation can start at once (no Householder pass for the first step).
+    bool started = false;
+    st = qr_tc_try_orthogonal_start(h->ctx, h->ws, h->qtc, h->Z, d, batch, ORTHOGONAL_START_THRESHOLD, &started);
+  }
   if (st == DQ_OK) st = fence_out(h);
   if (st != DQ_OK) { free_all(h); return st; }
   *out = h;

@@ -170,6 +170,41 @@ __global__ void __launch_bounds__(256) combine_kernel(const bf16* __restrict__ h
     dst[i] = __bfloat162float(hi[i]) + __bfloat162float(lo[i]);
 }
 
+// W = I in every form the incremental factorisation carries: fp32, split row-major and split transposed
+// (hi = 1 on the diagonal, everything else 0).
+__global__ void __launch_bounds__(256) identity_w_kernel(float* __restrict__ Wf, bf16* __restrict__ n_hi,
+                                                         bf16* __restrict__ n_lo, bf16* __restrict__ t_hi,
+                                                         bf16* __restrict__ t_lo, int d, int64_t n) {
+  const bf16 zero = __float2bfloat16_rn(0.f), one = __float2bfloat16_rn(1.f);
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t e = i % ((int64_t)d * d);
+    const bool diag = (e / d) == (e % d);
+    Wf[i] = diag ? 1.f : 0.f;
+    n_hi[i] = diag ? one : zero; t_hi[i] = diag ? one : zero;
+    n_lo[i] = zero; t_lo[i] = zero;
+  }
+}
+
+// part[block] = sum of squares of this block's share of E on and above the diagonal (off-diagonal entries
+// count twice: E is symmetric and only its upper tiles are stored), in double precision, fixed order.
+__global__ void __launch_bounds__(256) sym_sumsq_kernel(const float* __restrict__ E, int d, int64_t n,
+                                                        double* __restrict__ part) {
+  __shared__ double sm[256];
+  double acc = 0.0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t e = i % ((int64_t)d * d);
+    const int r = (int)(e / d), c = (int)(e % d);
+    if (c >= r) { const double v = E[i]; acc += (c > r ? 2.0 : 1.0) * v * v; }
+  }
+  sm[threadIdx.x] = acc;
+  __syncthreads();
+  for (int off = 128; off >= 1; off >>= 1) {
+    if (threadIdx.x < off) sm[threadIdx.x] += sm[threadIdx.x + off];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) part[blockIdx.x] = sm[0];
+}
+
 // Operands and results of the blocked inverse of an upper-triangular matrix (all [batch][d][d]).
 struct TriInv {
   const float* src;                 // the matrix (fp32), read for its 128 x 128 diagonal blocks
@@ -497,6 +532,46 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
   o.k_mode = 4;   // W is upper triangular: W^T[j][k] = 0 for k > j
   o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
   return gemm3(ctx, a, b, d, d, d, batch, o);
+}
+
+// A latent that is orthogonal to begin with (the paper's initialisation is a random Hadamard matrix) has
+// U = I: the incremental steps can start from W = I without a Householder factorisation.  Measures
+// |Z^T Z - I|_F (one split-bf16 product on the upper tiles and a reduction; synchronises the stream) and, if
+// it is at most `threshold` for every problem, installs W = I as the previous step's factor.
+dq_status qr_tc_try_orthogonal_start(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, int d, int batch,
+                                     float threshold, bool* started) {
+  *started = false;
+  const int64_t dd = (int64_t)d * d;
+  DQ_CHECK(qrp_transpose_split(ctx, Z, ws.A, q.st_hi, q.st_lo, d, batch));
+  {   // E = Z^T Z - I on the upper tiles
+    Op a{q.st_hi, q.st_lo, d, dd};
+    Out o; o.f32 = ws.B; o.ld = d; o.bs = dd; o.gen_mode = tc::GEN_CHOL_FIRST; o.aux = ws.tmp;
+    upper_lists(o, q);
+    DQ_CHECK(gemm3(ctx, a, a, d, d, d, batch, o));
+  }
+  constexpr int BLOCKS = 256;
+  double* d_part = reinterpret_cast<double*>(ws.S);       // scratch: [batch][BLOCKS] doubles
+  for (int b = 0; b < batch; ++b) {
+    sym_sumsq_kernel<<<BLOCKS, 256, 0, ctx.stream>>>(ws.B + b * dd, d, dd, d_part + (int64_t)b * BLOCKS);
+    DQ_CHECK(after_launch(ctx));
+  }
+  std::vector<double> part((size_t)batch * BLOCKS);
+  DQ_CHECK_CUDA(cudaMemcpyAsync(part.data(), d_part, sizeof(double) * part.size(), cudaMemcpyDeviceToHost, ctx.stream));
+  DQ_CHECK_CUDA(cudaStreamSynchronize(ctx.stream));
+  for (int b = 0; b < batch; ++b) {
+    double s = 0.0;
+    for (int i = 0; i < BLOCKS; ++i) s += part[(size_t)b * BLOCKS + i];
+    if (!(s <= (double)threshold * threshold)) return DQ_OK;   // (also catches NaN)
+  }
+  q.w_sel = 0;
+  const WSet w = wset(q, 0);
+  identity_w_kernel<<<ctx.sm_count * 8, 256, 0, ctx.stream>>>(ws.Winv, w.n_hi, w.n_lo, w.t_hi, w.t_lo, d, dd * batch);
+  DQ_CHECK(after_launch(ctx));
+  DQ_CHECK_CUDA(cudaMemsetAsync(q.P, 0, sizeof(float) * (size_t)dd * batch, ctx.stream));
+  q.t_warm = true;
+  q.u_fresh = false;
+  *started = true;
+  return DQ_OK;
 }
 
 // U of the current factorisation for inspection: the Householder route leaves it in place; the incremental

@@ -200,8 +200,8 @@ constexpr uint32_t IDESC_NEGATE_A = 1u << 13;   // kind::f16 instruction descrip
 constexpr int GEN_CH = 16;
 
 struct GenAddends {
-  float4 a[GEN_CH / 4];   // add1
-  float4 b[GEN_CH / 4];   // add2 (GEN_LINEAR ...) or the old aux (GEN_CHOL_SWEEP)
+  float a[GEN_CH];   // add1
+  float b[GEN_CH];   // add2 (GEN_LINEAR ...) or the old aux (GEN_CHOL_SWEEP)
 };
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -214,32 +214,47 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "memory");
 }
 
+// 32-byte global accesses (addresses 32-byte aligned).  Every thread of the epilogue owns a row, so a warp-wide
+// access touches 32 different lines whatever its width: the wider the access, the fewer such instructions.
+__device__ __forceinline__ void ld_global_f32x8(const float* ptr, float* v) {
+  asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+               : "l"(ptr) : "memory");
+}
+__device__ __forceinline__ void st_global_f32x8(float* ptr, const float* v) {
+  asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               :: "l"(ptr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+               : "memory");
+}
+__device__ __forceinline__ void st_global_b32x8(void* ptr, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               :: "l"(ptr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+
 // off = offset of (row, first column of the chunk) in out / add1 / add2 / aux.
 __device__ __forceinline__ void epi_gen_fetch(const Params& p, int64_t off, GenAddends& g) {
   const bool chol = p.gen_mode == GEN_CHOL_FIRST || p.gen_mode == GEN_CHOL_SWEEP;
   if (p.add1) {
-    const float4* a1 = reinterpret_cast<const float4*>(p.add1 + off);
 #pragma unroll
-    for (int i = 0; i < GEN_CH / 4; ++i) g.a[i] = a1[i];
+    for (int i = 0; i < GEN_CH / 8; ++i) ld_global_f32x8(p.add1 + off + 8 * i, g.a + 8 * i);
   } else {
 #pragma unroll
-    for (int i = 0; i < GEN_CH / 4; ++i) g.a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < GEN_CH; ++i) g.a[i] = 0.f;
   }
   const float* second = chol ? (p.gen_mode == GEN_CHOL_SWEEP ? p.aux : nullptr) : p.add2;
   if (second) {
-    const float4* a2 = reinterpret_cast<const float4*>(second + off);
 #pragma unroll
-    for (int i = 0; i < GEN_CH / 4; ++i) g.b[i] = a2[i];
+    for (int i = 0; i < GEN_CH / 8; ++i) ld_global_f32x8(second + off + 8 * i, g.b + 8 * i);
   } else {
 #pragma unroll
-    for (int i = 0; i < GEN_CH / 4; ++i) g.b[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < GEN_CH; ++i) g.b[i] = 0.f;
   }
 }
 
 // v[i] = accumulator of column col0 + i of output row `row` (problem b); g = the chunk's addends.
 __device__ __forceinline__ void epi_gen_chunk(const Params& p, const uint32_t (&v)[GEN_CH], int b, int row, int col0,
                                               int64_t off, const GenAddends& g, bool& moved) {
-  constexpr int Q = GEN_CH / 4;
   float f[GEN_CH];
 #pragma unroll
   for (int i = 0; i < GEN_CH; ++i) f[i] = p.alpha * __uint_as_float(v[i]);
@@ -251,43 +266,26 @@ __device__ __forceinline__ void epi_gen_chunk(const Params& p, const uint32_t (&
       for (int i = 0; i < GEN_CH; ++i) f[i] -= (col0 + i == row) ? 1.f : 0.f;
     }
     if (outp) {   // E (first) or T^T T (sweep)
-      float4* dst = reinterpret_cast<float4*>(outp + off);
 #pragma unroll
-      for (int i = 0; i < Q; ++i) dst[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+      for (int i = 0; i < GEN_CH / 8; ++i) st_global_f32x8(outp + off + 8 * i, f + 8 * i);
     }
 #pragma unroll
-    for (int i = 0; i < Q; ++i) {
-      const float oo[4] = {g.a[i].x, g.a[i].y, g.a[i].z, g.a[i].w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int col = col0 + 4 * i + j;
-        const float sgn = first ? f[4 * i + j] - oo[j] : oo[j] - f[4 * i + j];
-        f[4 * i + j] = (col > row) ? sgn : ((col == row) ? 0.5f * sgn : 0.f);
-      }
-      if (!first) {
-        const float od[4] = {g.b[i].x, g.b[i].y, g.b[i].z, g.b[i].w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          if (!(fabsf(f[4 * i + j] - od[j]) <= p.tol)) moved = true;
-      }
+    for (int i = 0; i < GEN_CH; ++i) {
+      const int col = col0 + i;
+      const float sgn = first ? f[i] - g.a[i] : g.a[i] - f[i];
+      f[i] = (col > row) ? sgn : ((col == row) ? 0.5f * sgn : 0.f);
+      if (!first && !(fabsf(f[i] - g.b[i]) <= p.tol)) moved = true;
     }
-    float4* axw = reinterpret_cast<float4*>(p.aux + off);
 #pragma unroll
-    for (int i = 0; i < Q; ++i) axw[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+    for (int i = 0; i < GEN_CH / 8; ++i) st_global_f32x8(p.aux + off + 8 * i, f + 8 * i);
   } else {
     if (p.add1) {
 #pragma unroll
-      for (int i = 0; i < Q; ++i) {
-        f[4 * i] = fmaf(p.g1, g.a[i].x, f[4 * i]); f[4 * i + 1] = fmaf(p.g1, g.a[i].y, f[4 * i + 1]);
-        f[4 * i + 2] = fmaf(p.g1, g.a[i].z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.g1, g.a[i].w, f[4 * i + 3]);
-      }
+      for (int i = 0; i < GEN_CH; ++i) f[i] = fmaf(p.g1, g.a[i], f[i]);
     }
     if (p.add2) {
 #pragma unroll
-      for (int i = 0; i < Q; ++i) {
-        f[4 * i] = fmaf(p.g2, g.b[i].x, f[4 * i]); f[4 * i + 1] = fmaf(p.g2, g.b[i].y, f[4 * i + 1]);
-        f[4 * i + 2] = fmaf(p.g2, g.b[i].z, f[4 * i + 2]); f[4 * i + 3] = fmaf(p.g2, g.b[i].w, f[4 * i + 3]);
-      }
+      for (int i = 0; i < GEN_CH; ++i) f[i] = fmaf(p.g2, g.b[i], f[i]);
     }
     if (p.gen_mode == GEN_STRICT_LOWER) {
 #pragma unroll
@@ -297,9 +295,8 @@ __device__ __forceinline__ void epi_gen_chunk(const Params& p, const uint32_t (&
       for (int i = 0; i < GEN_CH; ++i) f[i] = (row <= col0 + i) ? f[i] : 0.f;
     }
     if (outp) {
-      float4* dst = reinterpret_cast<float4*>(outp + off);
 #pragma unroll
-      for (int i = 0; i < Q; ++i) dst[i] = make_float4(f[4 * i], f[4 * i + 1], f[4 * i + 2], f[4 * i + 3]);
+      for (int i = 0; i < GEN_CH / 8; ++i) st_global_f32x8(outp + off + 8 * i, f + 8 * i);
     }
   }
   if (p.out_hi || p.out_t_hi || p.out_t2_hi) {
@@ -314,14 +311,8 @@ __device__ __forceinline__ void epi_gen_chunk(const Params& p, const uint32_t (&
     }
     if (p.out_hi) {
       const int64_t off_h = (int64_t)b * p.batch_stride_h + (int64_t)row * p.ld_h + col0;
-      uint4* dh = reinterpret_cast<uint4*>(p.out_hi + off_h);
-#pragma unroll
-      for (int i = 0; i < GEN_CH / 8; ++i) dh[i] = make_uint4(ph[4 * i], ph[4 * i + 1], ph[4 * i + 2], ph[4 * i + 3]);
-      if (p.out_lo) {
-        uint4* dl = reinterpret_cast<uint4*>(p.out_lo + off_h);
-#pragma unroll
-        for (int i = 0; i < GEN_CH / 8; ++i) dl[i] = make_uint4(pl[4 * i], pl[4 * i + 1], pl[4 * i + 2], pl[4 * i + 3]);
-      }
+      st_global_b32x8(p.out_hi + off_h, ph);
+      if (p.out_lo) st_global_b32x8(p.out_lo + off_h, pl);
     }
     if (p.out_t_hi || p.out_t2_hi) {
       // transposed copies: for a fixed column the 32 lanes of the warp (consecutive rows) store 64 contiguous bytes

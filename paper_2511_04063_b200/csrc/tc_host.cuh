@@ -104,7 +104,8 @@ template <int EPI>
 inline dq_status rotate_tokens(Ctx& ctx, const void* X, int64_t n, int d, int64_t ldx, const bf16* rt, void* out,
                                int64_t ldo, int* d_status) {
   // TMA needs 16-byte aligned bases and row strides; the epilogue stores 16 bytes at a time
-  if ((((uintptr_t)X | (uintptr_t)rt | (uintptr_t)out) & 15) || ldx % 8 != 0 || ldo % (EPI == tc::EPI_GEN ? 4 : 8) != 0)
+  if ((((uintptr_t)X | (uintptr_t)rt | (uintptr_t)out) & 15) || ldx % 8 != 0 || ldo % 8 != 0 ||
+      (EPI == tc::EPI_GEN && ((uintptr_t)out & 31)))   // (the fp32 epilogue stores 32 bytes at a time)
     return DQ_ERR_UNSUPPORTED;
   CUtensorMap ma, mb;
   tc::Params p{};
@@ -193,6 +194,14 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
   if ((o.tri_skip || o.k_mode) && (o.ksplit != 1 || M != N)) return DQ_ERR_UNSUPPORTED;
   const bool dual = o.dual_a && o.dual_b;
   if (dual && (o.nterms != 1 || o.k_mode || o.ksplit != 1)) return DQ_ERR_UNSUPPORTED;
+  {   // the epilogue moves 32 bytes per access: bases, leading dimensions and strides must keep rows 32-byte aligned
+    auto bad = [](const void* ptr, int64_t ld, int64_t bs, int esz) {
+      return ptr && ((((uintptr_t)ptr) & 31) || (ld * esz) % 32 || (bs * esz) % 32);
+    };
+    if (bad(o.f32, o.ld, o.bs, 4) || bad(o.add1, o.ld, o.bs, 4) || bad(o.add2, o.ld, o.bs, 4) || bad(o.aux, o.ld, o.bs, 4) ||
+        bad(o.hi, o.ld_h, o.bs_h, 2) || bad(o.lo, o.ld_h, o.bs_h, 2) || (o.split_stride * 4) % 32)
+      return DQ_ERR_UNSUPPORTED;
+  }
   if (o.ksplit > 1 && (o.add1 || o.add2 || o.beta != 0.f || o.hi || o.t_hi || o.gen_mode != tc::GEN_LINEAR))
     return DQ_ERR_UNSUPPORTED;
   // second pair of tensor maps: the lo parts of a split product, or the second operand pair of a dual one

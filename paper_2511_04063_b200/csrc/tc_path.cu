@@ -130,9 +130,11 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   if (!m) return DQ_ERR_ALLOC;
   tc.maps = m;
   DQ_CHECK(tch::make_map(&m->rt, tc.Rt, d, d, batch, d, (int64_t)d * d, tc::BLOCK_M));
-  DQ_CHECK(tch::make_map(&m->x, tc.X, d, N, batch, d, N * d, 256));
-  DQ_CHECK(tch::make_map(&m->x128, tc.X, d, N, batch, d, N * d, 128));
-  DQ_CHECK(tch::make_map(&m->x64, tc.X, d, N, batch, d, N * d, heads::TT));
+  const int64_t ldx = cfg.ldx;   // row stride of the borrowed activations (>= d, a multiple of 8 elements)
+  tc.ldx = ldx;
+  DQ_CHECK(tch::make_map(&m->x, tc.X, d, N, batch, ldx, N * ldx, 256));
+  DQ_CHECK(tch::make_map(&m->x128, tc.X, d, N, batch, ldx, N * ldx, 128));
+  DQ_CHECK(tch::make_map(&m->x64, tc.X, d, N, batch, ldx, N * ldx, heads::TT));
   DQ_CHECK(tch::make_map(&m->xt, tc.Xt, N, d, batch, N, N * d, tc::BLOCK_M));
   DQ_CHECK(tch::make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
   DQ_CHECK(tch::make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
@@ -160,7 +162,7 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
 // X^T copy (channel-major) for the K-major A operand of Gq = X^T G.
 dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx) {
   transpose_bf16_kernel<<<dim3(tc.d / 64, (unsigned)(tc.n_tokens / 64), tc.batch), 256, 0, ctx.stream>>>(
-      tc.X, tc.Xt, tc.n_tokens, tc.d, tc.d);
+      tc.X, tc.Xt, tc.n_tokens, tc.d, tc.ldx);
   return after_launch(ctx);
 }
 

@@ -7,8 +7,8 @@ namespace dq {
 struct TcState {
   bool ready = false;
   int d = 0, batch = 0;
-  int64_t n_tokens = 0;
-  const __nv_bfloat16* X = nullptr;   // [batch][N][d] token-major (borrowed)
+  int64_t n_tokens = 0, ldx = 0;
+  const __nv_bfloat16* X = nullptr;   // [batch][N][ldx] token-major (borrowed)
   __nv_bfloat16* Xt = nullptr;        // [batch][d][N] channel-major copy (owned)
   __nv_bfloat16* Rt = nullptr;        // [batch][d][d] bf16(R^T) (owned unless rt_external)
   bool rt_external = false;
@@ -105,6 +105,10 @@ void qr_tc_destroy(QrTcState& q);
 // route always does).
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
                           int batch, int iterative_iters, bool need_lo);
+// If |Z^T Z - I|_F <= threshold for every problem: installs W = I so that the incremental route can factor Z
+// without a Householder start (*started = true).  Synchronises the stream.
+dq_status qr_tc_try_orthogonal_start(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, int d, int batch,
+                                     float threshold, bool* started);
 // Makes U hold the upper factor of the current factorisation (inverts W after incremental steps).
 dq_status qr_tc_materialize_u(Ctx& ctx, QrWorkspace& ws, QrTcState& q, float* U, int d, int batch);
 // split: three bf16 MMAs per product (split operands) instead of one.

@@ -142,7 +142,9 @@ def test_switching_back_to_qr_orth_restarts_from_the_latent():
     assert np.abs(c.rotation()[0] - R0).max() > 0        # the iterate moved
     assert np.array_equal(c.latent(), c.Z0_host)           # the latent is not touched by Cayley SGD
     dq.dq_calib_set_orth_method(c.h, dq.DQ_ORTH_QR)
-    assert np.array_equal(c.rotation()[0], R0)
+    # the same rotation again (the first came from the start at W = I of an orthogonal latent, this one from a
+    # Householder factorisation: the unique factor either way, to the accuracy of the split-bf16 products)
+    assert np.abs(c.rotation()[0] - R0).max() <= 5e-6
     c.close()
 
 

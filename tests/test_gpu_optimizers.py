@@ -101,3 +101,37 @@ def test_set_optimizer_rejects_bad_arguments():
     assert lib.dq_calib_set_optimizer(c.h, dq.DQ_ADAM, 0.1, 0.9, 0.999, -1.0) == dq.DQ_ERR_INVALID_ARG
     assert lib.dq_calib_set_optimizer(None, dq.DQ_SGD, 0.1, 0.0, 0.0, 0.0) == dq.DQ_ERR_INVALID_ARG
     c.close()
+
+
+@pytest.mark.parametrize("opt", ["momentum", "adam"])
+def test_tensor_core_path_optimiser_update_matches_oracle_rule_on_its_own_gradients(opt):
+    """Teacher-forced on the gradient: after every step on the tensor-core path the latent must be what the
+    oracle's update rule makes of the previous latent, the previous optimiser state and the dL/dZ the kernels
+    just produced (the gradient itself is compared with the oracle by the stage tests).  Steps after the first
+    are replayed from a CUDA graph, so Adam's step count must advance on the device."""
+    w = gen.scaled(gen.WORKLOADS["c2_7b"], d=256, n_tokens=1024, n_outlier_channels=3)
+    lr, b1, b2, eps = (1e-3, 0.9, 0.999, 1e-8) if opt == "adam" else (w.lr, 0.9, 0.0, 0.0)
+    c = Calib(w)
+    dq.dq_calib_set_optimizer(c.h, dq.DQ_ADAM if opt == "adam" else dq.DQ_SGD_MOMENTUM, lr, b1, b2, eps)
+    Z = c.latent()[0].astype(np.float64)
+    m, v = np.zeros_like(Z), np.zeros_like(Z)
+    for t in range(1, 5):
+        c.step(1)
+        assert c.status() == dq.DQ_OK
+        g = c.buf(dq.DQ_BUF_GZ).cpu().numpy()[0].astype(np.float64)
+        if opt == "adam":
+            Z_ref, m, v = orc.adam_step(Z, g, m, v, t, lr, b1, b2, eps)
+        else:
+            Z_ref, m = orc.momentum_step(Z, g, m, lr, b1)
+        Zg = c.latent()[0].astype(np.float64)
+        moved = np.abs(Z_ref - Z).max()
+        # fp32 arithmetic of the update: a few ulp of the latent plus 1e-5 of the step
+        assert np.abs(Zg - Z_ref).max() <= 4 * 6e-8 * np.abs(Z).max() + 2e-5 * moved, (opt, t)
+        assert moved > 0
+        M = c.buf(dq.DQ_BUF_OPT_M).cpu().numpy()[0].astype(np.float64)
+        assert np.abs(M - m).max() <= 1e-5 * np.abs(m).max() + 1e-12
+        Z = Zg                                                      # the next step starts from the kernel's latent
+        m = M
+        if opt == "adam":
+            v = c.buf(dq.DQ_BUF_OPT_V).cpu().numpy()[0].astype(np.float64)
+    c.close()

@@ -400,3 +400,60 @@ def test_a_bounded_wait_that_runs_out_sets_the_status_word_and_the_kernel_return
     assert lib.dq_calib_selftest_bounded_wait(c.h, 0, None) == dq.DQ_ERR_INVALID_ARG
     assert lib.dq_calib_selftest_bounded_wait(c.h, 10**9, None) == dq.DQ_ERR_INVALID_ARG
     c.close()
+
+
+@pytest.mark.parametrize("name,d,n,batch", [("c2_7b", 256, 1024, 1), ("c3_heads", 128, 512, 3)])
+def test_padded_activation_rows_give_the_same_step(name, d, n, batch):
+    """ldx > d on the tensor-core path: activations that sit in a wider buffer (row stride a multiple of 8
+    elements) are read in place; the step is bit-identical to the one on a packed copy."""
+    w = small(name, d=d, n_tokens=n, batch=batch, **({"n_outlier_channels": 3} if d != 128 else {}))
+    X = gen.gen_activations(w)
+    Z0 = torch.from_numpy(gen.gen_latent_init(w)).cuda()
+    packed = torch.from_numpy(X.view(np.int16)).cuda().view(torch.bfloat16)
+    wide = torch.full((batch, n, d + 72), float("nan"), dtype=torch.bfloat16, device="cuda")
+    wide[:, :, :d] = packed
+    outs = []
+    for Xd in (packed, wide[:, :, :d]):
+        h = dq.dq_calib_init(Xd, Z0, lr=w.lr, path=dq.DQ_PATH_BF16_TC)
+        loss = torch.empty((3, batch), dtype=torch.float32, device="cuda")
+        dq.dq_calib_step(h, 3, loss)
+        Z = torch.empty_like(Z0)
+        dq.dq_calib_get_latent(h, Z)
+        assert dq.dq_calib_status(h) == dq.DQ_OK
+        outs.append((loss.cpu().numpy(), Z.cpu().numpy()))
+        dq.dq_calib_destroy(h)
+    assert np.isfinite(outs[1][0]).all()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    lib = dq.load_library()
+    import ctypes as C
+    cfg = dq.dq_calib_config(d=d, n_tokens=n, batch=batch, x_dtype=dq.DQ_BF16, path=dq.DQ_PATH_BF16_TC, reduction=0,
+                             optimizer=0, lr=0.1, ldx=d + 4)          # 8-byte row stride: not a TMA stride
+    hh = C.c_void_p(0)
+    assert lib.dq_calib_init(C.byref(hh), C.byref(cfg), C.c_void_p(wide.data_ptr()), C.c_void_p(Z0.data_ptr()),
+                             None) == dq.DQ_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("d,amp", [(512, 0.0), (1024, 0.0), (512, 3e-4)])
+def test_orthogonal_initial_latent_starts_without_householder(d, amp):
+    """The paper's initial latent (a random Hadamard matrix) is orthogonal, so U = I: the handle starts the
+    incremental factorisation from W = I at once.  The rotation is the unique factor all the same, and the
+    first factorisation takes a few dozen launches instead of the d / 128 panel steps."""
+    w = small("c2_7b", d=d, n_tokens=512, n_outlier_channels=2)
+    Z0 = gen.gen_latent_init(w)
+    if amp:
+        Z0 = (Z0 + np.float32(amp) * np.random.default_rng(3).standard_normal(Z0.shape).astype(np.float32)).astype(np.float32)
+    c = Calib(w, Z0=Z0)
+    n0 = dq.dq_calib_launch_count(c.h)
+    R = c.rotation()[0]
+    assert c.status() == dq.DQ_OK
+    assert dq.dq_calib_launch_count(c.h) - n0 <= 40
+    Rr, Ur = orc.qr_pos_lapack(Z0[0])
+    assert np.abs(R - Rr).max() <= 2e-5
+    assert np.abs(R.T @ R - np.eye(d)).max() <= 2e-5
+    U = c.buf(dq.DQ_BUF_U).cpu().numpy()[0].astype(np.float64)
+    assert np.abs(U - Ur).max() <= 3e-5 and np.abs(np.tril(U, -1)).max() == 0.0
+    c.step(3)
+    assert c.status() == dq.DQ_OK
+    Z = c.latent()[0]
+    assert np.abs(c.rotation()[0] - orc.qr_pos_lapack(Z)[0]).max() <= 5e-5
+    c.close()
