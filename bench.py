@@ -260,6 +260,11 @@ def main():
     phases = dq.dq_calib_get_timings(h)
     dq.dq_calib_set_timing(h, False)
 
+    # ---------------------------------------------------------------- one QR-Orth product alone
+    prod_ms = None
+    if path == dq.DQ_PATH_BF16_TC and wr.d != 128:
+        prod_ms = {3: dq.dq_calib_time_product(h, 3, 10), 1: dq.dq_calib_time_product(h, 1, 10)}
+
     # ---------------------------------------------------------------- same workload, the other QR-Orth forward
     alt = None
     if path == dq.DQ_PATH_BF16_TC and wr.d != 128:
@@ -445,6 +450,24 @@ def main():
                                   "qr_orth_tflops": qr_flops / t_qr / 1e12 if t_qr > 0 else None,
                                   "qr_orth_frac_of_measured_burst": qr_flops / t_qr / 1e12 / peaks["bf16_tflops"],
                                   "note": "QR-Orth phases also hold their HBM-bound element-wise kernels"}
+        if prod_ms is not None:
+            # The kernel family QR-Orth spends its time in, timed alone: one dense d^3 product on split-bf16
+            # operands (three bf16 MMAs per product term: 6 d^3 issued MMA flops for 2 d^3 algorithmic ones) and on
+            # plain bf16 operands, against the measured burst bf16 peak; and the share of the step's event-timed
+            # phases that each family of kernels takes.
+            issued3, issued1 = 6.0 * d ** 3 * B, 2.0 * d ** 3 * B
+            line["roofline_qr_orth"] = {
+                "bound": "tensor", "kernel": "tc_gemm2_kernel<3,GEN> / <1,GEN> (d x d products of QR-Orth)",
+                "achieved": issued3 / (prod_ms[3] * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": issued3 / (prod_ms[3] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                "peak_source": "%s (burst bf16 matmul peak)" % peaks["_source"],
+                "ms_per_launch": prod_ms[3], "issued_flops_per_launch": issued3,
+                "algorithmic_flops_per_launch": 2.0 * d ** 3 * B,
+                "algorithmic_tflops": 2.0 * d ** 3 * B / (prod_ms[3] * 1e-3) / 1e12,
+                "plain_bf16": {"ms_per_launch": prod_ms[1], "achieved": issued1 / (prod_ms[1] * 1e-3) / 1e12,
+                               "frac": issued1 / (prod_ms[1] * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+                "traffic": None}
+            line["phase_share"] = {k: v / total_phase for k, v in phases.items()} if total_phase else None
         if rot is not None:
             # includes the fp32 -> bf16 transpose of R (d^2 entries) in front of the contraction
             line["rotate_apply"] = {"ms": rot, "tflops": 2.0 * N * d * d / (rot * 1e-3) / 1e12,

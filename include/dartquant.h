@@ -279,7 +279,9 @@ dq_status dq_calib_set_timing(dq_calib_t* h, int32_t enabled);
  * diagnostics.  *d_ptr is valid until the handle is destroyed. */
 enum {
   DQ_BUF_R = 0,        /* fp32 [batch][d][d]  rotation used by the last step       */
-  DQ_BUF_U = 1,        /* fp32 [batch][d][d]  upper factor, positive diagonal      */
+  DQ_BUF_U = 1,        /* fp32 [batch][d][d]  upper factor, positive diagonal (after incremental steps on the tensor-core
+                          path only U^-1 is carried: for d >= 256 it is inverted on demand, to about 1e-5; for d == 128 the
+                          view is DQ_ERR_UNSUPPORTED until the next Householder factorisation) */
   DQ_BUF_GQ = 2,       /* fp32 [batch][d][d]  dL/dR                                */
   DQ_BUF_GZ = 3,       /* fp32 [batch][d][d]  dL/dZ                                */
   DQ_BUF_G = 4,        /* dL/dO without the 1/N factor: fp32 [batch][N][d] (fp32 path)
@@ -307,6 +309,13 @@ int64_t dq_calib_launch_count(dq_calib_t* h);
  * operands exactly as the kernels clip it; counted on the host at launch).  For measurement:
  * the difference across a timed region divided by its duration is the issued MMA rate. */
 double dq_calib_mma_flops(dq_calib_t* h);
+
+/* For measurement: times (CUDA events on the handle's work stream; synchronises) `reps` launches of one
+ * dense d x d x d product of the kind QR-Orth is made of, on the handle's own operand copies, result to
+ * scratch: nterms = 3 on split-bf16 operands (three bf16 MMAs per product term, 6 d^3 MMA flops for the
+ * 2 d^3 of the product), nterms = 1 on plain bf16 operands.  *h_ms receives the mean per launch.  Tensor-core
+ * path with d >= 256 only; call it after at least one step.  Changes no state of the calibration. */
+dq_status dq_calib_time_product(dq_calib_t* h, int32_t nterms, int32_t reps, float* h_ms);
 
 const char* dq_status_string(dq_status s);
 void dq_calib_destroy(dq_calib_t* h);

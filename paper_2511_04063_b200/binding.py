@@ -31,7 +31,7 @@ EXPORTED_SYMBOLS = (
     "dq_calib_get_timings", "dq_calib_set_timing", "dq_calib_debug_buffer", "dq_calib_launch_count", "dq_status_string",
     "dq_calib_destroy", "dq_version", "dq_rotate_apply_static", "dq_calib_set_qr_method", "dq_calib_set_optimizer", "dq_gather_tokens", "dq_eval_rotation",
     "dq_calib_set_orth_method", "dq_calib_set_objective", "dq_calib_run_epochs", "dq_calib_mma_flops", "dq_calib_set_keep_gradient",
-    "dq_calib_set_backward_precision", "dq_calib_selftest_bounded_wait",
+    "dq_calib_set_backward_precision", "dq_calib_selftest_bounded_wait", "dq_calib_time_product",
 )
 
 
@@ -91,6 +91,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.dq_calib_set_keep_gradient.restype = i32
     lib.dq_calib_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp]
     lib.dq_calib_selftest_bounded_wait.restype = i32
+    lib.dq_calib_time_product.argtypes = [vp, i32, i32, C.POINTER(C.c_float)]
+    lib.dq_calib_time_product.restype = i32
     lib.dq_calib_set_backward_precision.argtypes = [vp, i32]
     lib.dq_calib_set_backward_precision.restype = i32
     lib.dq_calib_launch_count.argtypes = [vp]
@@ -211,6 +213,13 @@ def dq_calib_selftest_bounded_wait(h, limit_ns: int) -> int:
     waited = torch.zeros(1, dtype=torch.int64, device="cuda")
     _check(load_library().dq_calib_selftest_bounded_wait(h, limit_ns, waited.data_ptr()), "dq_calib_selftest_bounded_wait")
     return int(waited.cpu()[0])
+
+
+def dq_calib_time_product(h, nterms: int, reps: int = 10) -> float:
+    """Mean milliseconds of one dense d^3 QR-Orth product (nterms 3: split-bf16, 1: plain bf16); measurement."""
+    ms = C.c_float(0.0)
+    _check(load_library().dq_calib_time_product(h, nterms, reps, C.byref(ms)), "dq_calib_time_product")
+    return float(ms.value)
 
 
 def dq_calib_mma_flops(h) -> float:

@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libdartquant.so")
 OBJ_DIR = os.path.join(HERE, "_build")
-SOURCES = ["api.cu", "gemm_ffma.cu", "qr_forward.cu", "qr_backward.cu", "tc_path.cu", "qr_tc.cu", "qr_panel_tc.cu", "qr128.cu", "token_sampling.cu", "eval_metrics.cu", "cayley_tc.cu", "objectives.cu", "qr128_inc.cu"]
+SOURCES = ["api.cu", "gemm_ffma.cu", "qr_forward.cu", "qr_backward.cu", "tc_path.cu", "qr_tc.cu", "qr_panel_tc.cu", "qr128.cu", "token_sampling.cu", "eval_metrics.cu", "cayley_tc.cu", "objectives.cu", "qr128_inc.cu", "qr128_tc5.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

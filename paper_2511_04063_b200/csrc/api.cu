@@ -58,6 +58,10 @@ struct dq_calib {
   int* f32_flags = nullptr;     // fp32 path: sweep flags of the incremental factorisation
   bool small_warm = false;      // d == 128: U and U^-1 hold the factors of the previous step's latent
   bool small128 = false;        // d == 128: shared-memory-resident batched QR-Orth
+  bool tc5 = false;             // d == 128 on the tensor-core path: tcgen05 kernel for the incremental QR-Orth
+  float* p128 = nullptr;        // [batch][128][128] T^T T of the last sweep (tc5)
+  float* scratch128 = nullptr;  // [batch][4][128][128] scratch of the tc5 kernel
+  bool u128_fresh = false;      // U holds the upper factor of the current factorisation (tc5 carries only U^-1)
   bool r_stale = true;
   bool timing = false;
   cudaEvent_t ev[DQ_PHASE_COUNT + 1] = {};
@@ -93,7 +97,7 @@ void free_all(dq_calib* h) {
   cayley_destroy(h->cay);
   objective_destroy(h->obj);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
-  cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw);
+  cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw); cudaFree(h->p128); cudaFree(h->scratch128);
   cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->loss_tmp); cudaFree(h->f32_flags); cudaFree(h->ctx.d_status);
   cudaFree(h->ws.A); cudaFree(h->ws.V); cudaFree(h->ws.T); cudaFree(h->ws.W); cudaFree(h->ws.W2);
   cudaFree(h->ws.Q); cudaFree(h->ws.Winv); cudaFree(h->ws.B); cudaFree(h->ws.S); cudaFree(h->ws.tmp);
@@ -147,9 +151,18 @@ dq_status ensure_rotation(dq_calib* h) {
   if (h->small128) {
     __nv_bfloat16* rt = h->cfg.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr;
     if (h->qr_method == DQ_QR_ITERATIVE && h->small_warm) {
-      DQ_CHECK(qr128_forward_incremental(h->ctx, h->Z, h->R, h->U, h->ws.Winv, rt, h->qr_iters, h->cfg.batch));
+      if (h->tc5) {   // tcgen05 kernel: needs only W (no U), starts its fixed point from the last step's T^T T
+        DQ_CHECK(qr128_step_tc5(h->ctx, h->Z, h->ws.Winv, h->p128, h->R, rt, nullptr, nullptr, h->scratch128, 0.f,
+                                false, true, h->qr_iters + 3, h->cfg.batch));
+        h->u128_fresh = false;
+      } else {
+        DQ_CHECK(qr128_forward_incremental(h->ctx, h->Z, h->R, h->U, h->ws.Winv, rt, h->qr_iters, h->cfg.batch));
+      }
     } else {
       DQ_CHECK(qr128_forward(h->ctx, h->Z, h->R, h->U, h->ws.Winv, rt, h->cfg.batch));
+      if (h->tc5)
+        DQ_CHECK_CUDA(cudaMemsetAsync(h->p128, 0, sizeof(float) * (size_t)128 * 128 * h->cfg.batch, h->ctx.stream));
+      h->u128_fresh = true;
       h->small_warm = true;
     }
   } else if (h->fast_qr) {
@@ -251,7 +264,12 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
     return DQ_OK;
   }
   if (h->small128) {   // plain SGD is fused into the backward kernel; other optimisers follow it
-    DQ_CHECK(qr128_backward_sgd_tc(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, h->optimizer == DQ_SGD ? c.lr : 0.f, batch));
+    const float lr128 = h->optimizer == DQ_SGD ? c.lr : 0.f;
+    if (h->tc5 && h->qr_method == DQ_QR_ITERATIVE)
+      DQ_CHECK(qr128_step_tc5(ctx, h->Z, h->ws.Winv, h->p128, h->R, nullptr, h->Gq, h->Gz, h->scratch128, lr128, true,
+                              false, 0, batch));
+    else
+      DQ_CHECK(qr128_backward_sgd_tc(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, lr128, batch));
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
   } else {
     if (h->fast_qr) DQ_CHECK(qr_backward_tc(ctx, h->ws, h->qtc, h->Gq, h->Gz, d, batch, h->bwd_split));
@@ -428,6 +446,10 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
     h->fast_qr = (st == DQ_OK);
     if (st == DQ_OK)
       A(tc_init(h->tc, h->ctx, *cfg, d_X, (__nv_bfloat16*)h->G, h->qtc.rt_hi, &h->n_partials));
+  }
+  if (h->small128 && cfg->path == DQ_PATH_BF16_TC) {
+    A(dev_alloc(&h->p128, dd)); A(dev_alloc(&h->scratch128, 4 * dd));
+    h->tc5 = (st == DQ_OK);
   }
   A(dev_alloc(&h->partials, (int64_t)batch * (h->n_partials > 0 ? h->n_partials : 1)));
   if (st == DQ_OK && cudaMemsetAsync(h->ctx.d_status, 0, sizeof(int), h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
@@ -679,6 +701,25 @@ dq_status dq_calib_selftest_bounded_wait(dq_calib_t* h, uint64_t limit_ns, uint6
   return fence_out(h);
 }
 
+dq_status dq_calib_time_product(dq_calib_t* h, int32_t nterms, int32_t reps, float* h_ms) {
+  if (!h || !h_ms || (nterms != 1 && nterms != 3) || reps < 1 || reps > 1000) return DQ_ERR_INVALID_ARG;
+  if (!h->fast_qr || h->small128) return DQ_ERR_UNSUPPORTED;
+  DQ_CHECK(fence_in(h));
+  const int64_t launches = h->ctx.launches;
+  const double flops = h->ctx.mma_flops;
+  DQ_CHECK(qr_tc_bench_product(h->ctx, h->ws, h->qtc, h->cfg.d, h->cfg.batch, nterms));   // warm-up
+  DQ_CHECK_CUDA(cudaEventRecord(h->ev[0], h->ctx.stream));
+  for (int r = 0; r < reps; ++r) DQ_CHECK(qr_tc_bench_product(h->ctx, h->ws, h->qtc, h->cfg.d, h->cfg.batch, nterms));
+  DQ_CHECK_CUDA(cudaEventRecord(h->ev[1], h->ctx.stream));
+  DQ_CHECK_CUDA(cudaEventSynchronize(h->ev[1]));
+  float ms = 0.f;
+  DQ_CHECK_CUDA(cudaEventElapsedTime(&ms, h->ev[0], h->ev[1]));
+  *h_ms = ms / reps;
+  h->ctx.launches = launches;      // measurement launches are not part of the calibration's counts
+  h->ctx.mma_flops = flops;
+  return fence_out(h);
+}
+
 dq_status dq_calib_set_timing(dq_calib_t* h, int32_t enabled) {
   if (!h) return DQ_ERR_INVALID_ARG;
   h->timing = enabled != 0;
@@ -698,6 +739,7 @@ dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int6
   switch (which) {
     case DQ_BUF_R: *d_ptr = h->R; *n_elems = dd; break;
     case DQ_BUF_U:
+      if (h->tc5 && h->small_warm && !h->u128_fresh) return DQ_ERR_UNSUPPORTED;   // only U^-1 is carried there
       if (h->fast_qr && !h->small128 && !h->qtc.u_fresh && h->orth_method == DQ_ORTH_QR && h->qtc.t_warm) {
         // the incremental factorisation carries U^-1 only: invert it for the view
         DQ_CHECK(fence_in(h));

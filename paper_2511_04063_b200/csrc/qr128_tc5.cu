@@ -1,0 +1,453 @@
+// Batched QR-Orth for 128 x 128 latents on the 5th-generation tensor cores: one CTA per problem, every
+// 128^3 product as tcgen05.mma on bf16 (hi, lo) operand pairs that the CTA itself writes into shared memory
+// in the K-major 128-byte-swizzled layout, accumulator in tensor memory, one thread per accumulator row.
+//
+//   backward  S = tril(R^T Gq - Gq^T R, -1) (one reduction over two operand pairs), D^T = W S^T, Gz = R D,
+//             Z <- Z - lr Gz                                                   (plain bf16 operands)
+//   forward   incremental factorisation from the previous step's W = U^-1 (no U, no triangular inverse):
+//             Zh = Z W, E = Zh^T Zh - I, T <- Phi(E - T^T T) from Phi(E - P_old) until no entry moves,
+//             Y = (I + T)^-1 - I by the series Y <- -T - T Y until no entry moves, R = Zh + Zh Y, W <- W + W Y.
+//             Zh and E on split operands (three MMAs per term); the others on plain bf16 operands unless the
+//             fixed point needed a third sweep (a large step), then on split operands too.
+// Both halves run in one launch when the optimiser is plain SGD (the update sits between them), so a step
+// boundary is one kernel and the latent, W and the operands made from them never leave the chip in between.
+// The products are a dependent chain, so nothing overlaps: write operands, one thread issues the MMAs, all
+// wait (bounded) for their completion, every thread reads its accumulator row and prepares the next operands.
+#include "common.cuh"
+#include "tc_gemm.cuh"
+
+namespace dq {
+namespace {
+
+using namespace tc;
+
+constexpr int N5 = 128;
+constexpr int PART_BYTES = N5 * N5 * 2;          // one bf16 operand part: two [128][64] K-major blocks
+constexpr int KBLK_BYTES = N5 * BLOCK_K * 2;     // 16 KB
+constexpr int N_BUFS = 6;
+constexpr int TC5_SMEM = N_BUFS * PART_BYTES + 1024 + 1024;
+constexpr int TC5_THREADS = 128;
+constexpr uint32_t TC5_TMEM_COLS = 128;
+constexpr int MAX_SERIES = 48;
+
+struct Tc5Params {
+  float* Z;            // [batch][128][128] latent (updated when lr != 0)
+  float* W;            // [batch][128][128] U^-1 of the previous factorisation (updated by the forward half)
+  float* P;            // [batch][128][128] T^T T of the previous step's last sweep (updated)
+  float* R;            // [batch][128][128] rotation: read by the backward half, written by the forward half
+  __nv_bfloat16* Rt;   // nullable: bf16(R^T), the operand of O = X R
+  const float* Gq;     // backward: dL/dR
+  float* Gz;           // backward: dL/dZ
+  float* scratch;      // [batch][4][128][128] fp32: E, T, Zh, Y
+  float lr;
+  int do_backward, do_forward;
+  int max_sweeps;
+  float tol;
+  int* d_status;
+};
+
+__device__ __forceinline__ void fence_async_smem5() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+constexpr int CH = 16;                           // columns of the accumulator row handled at a time
+
+// CH consecutive fp32 of a row (two 32-byte accesses); a null source reads as zeros
+__device__ __forceinline__ void fetch_ch(const float* p, float* v) {
+  if (p) {
+    ld_global_f32x8(p, v);
+    ld_global_f32x8(p + 8, v + 8);
+  } else {
+#pragma unroll
+    for (int i = 0; i < CH; ++i) v[i] = 0.f;
+  }
+}
+__device__ __forceinline__ void store_ch(float* p, const float* v) {
+  st_global_f32x8(p, v);
+  st_global_f32x8(p + 8, v + 8);
+}
+
+__device__ __forceinline__ void split_ch(const float* f, uint32_t* ph, uint32_t* pl) {
+#pragma unroll
+  for (int i = 0; i < CH / 2; ++i) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    const float2 hf = __bfloat1622float2(h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(f[2 * i] - hf.x, f[2 * i + 1] - hf.y);
+    ph[i] = *reinterpret_cast<const uint32_t*>(&h);
+    pl[i] = *reinterpret_cast<const uint32_t*>(&l);
+  }
+}
+
+// Operand with rows = this matrix's rows (K = its columns): columns [CH c, CH c + CH) of row r.
+__device__ __forceinline__ void put_rowmajor(uint8_t* buf, int r, int c, const uint32_t* packed) {
+  uint8_t* rowp = buf + (c >> 2) * KBLK_BYTES + r * 128;
+#pragma unroll
+  for (int i = 0; i < CH / 8; ++i) {
+    const int chunk = ((c & 3) * 2 + i) ^ (r & 7);
+    *reinterpret_cast<uint4*>(rowp + chunk * 16) =
+        make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+  }
+}
+// Operand with rows = this matrix's columns (K = its rows): entry (r, CH c + i) goes to row CH c + i, k = r.
+__device__ __forceinline__ void put_transposed(uint8_t* buf, int r, int c, const uint32_t* packed) {
+  uint8_t* base = buf + (r >> 6) * KBLK_BYTES + (r & 7) * 2;
+  const int j = (r & 63) >> 3;
+#pragma unroll
+  for (int i = 0; i < CH; ++i) {
+    const int col = CH * c + i;
+    const unsigned short v = (unsigned short)((i & 1) ? (packed[i >> 1] >> 16) : (packed[i >> 1] & 0xffffu));
+    *reinterpret_cast<unsigned short*>(base + col * 128 + ((j ^ (col & 7)) << 4)) = v;
+  }
+}
+
+struct Tc5 {
+  uint8_t* smem;        // operand buffers (generic pointer)
+  uint32_t smem_u;      // the same, shared-window address
+  uint32_t bar;         // mbarrier the MMAs commit to
+  uint32_t parity;
+  uint32_t tmem_row;    // accumulator, this thread's lane
+  uint32_t tmem;        // accumulator base
+  int* d_status;
+  __device__ __forceinline__ uint8_t* buf(int i) const { return smem + i * PART_BYTES; }
+  // acc (+)= A B^T over the whole K = 128 (issuing thread only)
+  __device__ __forceinline__ void mma(int a, int b, bool accumulate, bool negate_a = false) const {
+    const uint32_t idesc = make_idesc_bf16(N5) | (negate_a ? IDESC_NEGATE_A : 0u);
+    const uint32_t sa = smem_u + a * PART_BYTES, sb = smem_u + b * PART_BYTES;
+#pragma unroll
+    for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+      for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+        umma_bf16(tmem, make_kmajor_sw128_desc(sa + kb * KBLK_BYTES + k * UMMA_K * 2),
+                  make_kmajor_sw128_desc(sb + kb * KBLK_BYTES + k * UMMA_K * 2), idesc,
+                  (accumulate || kb > 0 || k > 0) ? 1u : 0u);
+  }
+  // split-operand product: A = (a_hi, a_lo), B = (b_hi, b_lo): hi hi + hi lo + lo hi
+  __device__ __forceinline__ void mma3(int a_hi, int a_lo, int b_hi, int b_lo) const {
+    mma(a_hi, b_hi, false);
+    mma(a_hi, b_lo, true);
+    mma(a_lo, b_hi, true);
+  }
+};
+
+// One product of the chain: all threads have written their operand rows; thread 0 issues the MMAs (issue());
+// every thread waits (bounded) for their completion and then runs body(c, v, a0, a1) on the CH-wide chunks of
+// its accumulator row, with the fp32 rows s0 / s1 (nullable; this thread's row of some matrix) fetched one
+// chunk ahead, the first chunk while the MMAs run.  Returns false if the wait gave up (for all threads alike).
+template <typename Issue, typename Body>
+__device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* s0, const float* s1, Body body) {
+  tmem_ld_wait();
+  tc_fence_before();
+  fence_async_smem5();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    tc_fence_after();
+    issue();
+    umma_commit(k.bar);
+  }
+  float cur0[CH], cur1[CH];
+  fetch_ch(s0, cur0);
+  fetch_ch(s1, cur1);
+  const bool done = mbar_wait(k.bar, k.parity, k.d_status);
+  k.parity ^= 1u;
+  tc_fence_after();
+  if (!__syncthreads_and(done ? 1 : 0)) return false;
+#pragma unroll 1
+  for (int c = 0; c < N5 / CH; ++c) {
+    uint32_t v[CH];
+    tmem_ld16(k.tmem_row + (uint32_t)(c * CH), v);
+    float nx0[CH], nx1[CH];
+    if (c + 1 < N5 / CH) {
+      fetch_ch(s0 ? s0 + (c + 1) * CH : nullptr, nx0);
+      fetch_ch(s1 ? s1 + (c + 1) * CH : nullptr, nx1);
+    }
+    tmem_ld_wait();
+    body(c, v, cur0, cur1);
+#pragma unroll
+    for (int i = 0; i < CH; ++i) { cur0[i] = nx0[i]; cur1[i] = nx1[i]; }
+  }
+  return true;
+}
+
+// This thread's row of an fp32 matrix in global memory -> operand buffers (row-major and / or transposed forms;
+// a negative buffer index skips that form).
+__device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* row, int r, int rm_hi, int rm_lo,
+                                                     int tr_hi, int tr_lo) {
+#pragma unroll 1
+  for (int c = 0; c < N5 / CH; ++c) {
+    float f[CH];
+    fetch_ch(row + c * CH, f);
+    uint32_t ph[CH / 2], pl[CH / 2];
+    split_ch(f, ph, pl);
+    if (rm_hi >= 0) put_rowmajor(k.buf(rm_hi), r, c, ph);
+    if (rm_lo >= 0) put_rowmajor(k.buf(rm_lo), r, c, pl);
+    if (tr_hi >= 0) put_transposed(k.buf(tr_hi), r, c, ph);
+    if (tr_lo >= 0) put_transposed(k.buf(tr_lo), r, c, pl);
+  }
+}
+
+__device__ __forceinline__ float phi(float s, int row, int col) {
+  return (col > row) ? s : ((col == row) ? 0.5f * s : 0.f);
+}
+
+__global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc5Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_ptr = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar = smem_base + N_BUFS * PART_BYTES;
+  const uint32_t tmem_slot = bar + 16u;
+  uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_ptr + N_BUFS * PART_BYTES + 16);
+  float* red = reinterpret_cast<float*>(smem_ptr + N_BUFS * PART_BYTES + 64);   // [8] block reductions
+
+  const int r = threadIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t off = (int64_t)blockIdx.x * N5 * N5;
+  float lr = p.lr;
+  if (p.d_status && *p.d_status != 0) lr = 0.f;   // an earlier error freezes the latent
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) tmem_alloc(tmem_slot, TC5_TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  Tc5 k;
+  k.smem = smem_ptr; k.smem_u = smem_base; k.bar = bar; k.parity = 0u; k.d_status = p.d_status;
+  k.tmem = *tmem_slot_ptr;
+  k.tmem_row = k.tmem + ((uint32_t)(warp * 32) << 16);
+
+  float* Zrow = p.Z + off + r * N5;
+  float* Wrow = p.W + off + r * N5;
+  float* Prow = p.P + off + r * N5;
+  float* Rrow = p.R + off + r * N5;
+  float* sc = p.scratch + (int64_t)blockIdx.x * 4 * N5 * N5 + r * N5;
+  float* Erow = sc;
+  float* Trow = sc + N5 * N5;
+  float* Zhrow = sc + 2 * N5 * N5;
+  float* Yrow = sc + 3 * N5 * N5;
+  bool ok = true;
+
+  if (p.do_backward) {
+    // operands: R row-major -> 0, R^T -> 1, Gq^T -> 2, W row-major -> 3   (hi parts)
+    load_row_to_operands(k, Rrow, r, 0, -1, 1, -1);
+    load_row_to_operands(k, p.Gq + off + r * N5, r, -1, -1, 2, -1);
+    load_row_to_operands(k, Wrow, r, 3, -1, -1, -1);
+    // S = tril(R^T Gq - Gq^T R, -1), row-major -> 4
+    ok = product(k, [&]() { k.mma(1, 2, false); k.mma(2, 1, true, true); }, nullptr, nullptr,
+                 [&](int c, const uint32_t (&v)[CH], const float (&)[CH], const float (&)[CH]) {
+                   float f[CH];
+#pragma unroll
+                   for (int i = 0; i < CH; ++i) f[i] = (r > CH * c + i) ? __uint_as_float(v[i]) : 0.f;
+                   uint32_t ph[CH / 2], pl[CH / 2];
+                   split_ch(f, ph, pl);
+                   put_rowmajor(k.buf(4), r, c, ph);
+                 });
+    // D^T = W S^T, row-major -> 5
+    if (ok)
+      ok = product(k, [&]() { k.mma(3, 4, false); }, nullptr, nullptr,
+                   [&](int c, const uint32_t (&v)[CH], const float (&)[CH], const float (&)[CH]) {
+                     float f[CH];
+#pragma unroll
+                     for (int i = 0; i < CH; ++i) f[i] = __uint_as_float(v[i]);
+                     uint32_t ph[CH / 2], pl[CH / 2];
+                     split_ch(f, ph, pl);
+                     put_rowmajor(k.buf(5), r, c, ph);
+                   });
+    // Gz = R D, then Z <- Z - lr Gz; the new latent goes straight into the forward's operands (1, 2)
+    if (ok)
+      ok = product(k, [&]() { k.mma(0, 5, false); }, Zrow, nullptr,
+                   [&](int c, const uint32_t (&v)[CH], const float (&z)[CH], const float (&)[CH]) {
+                     float g[CH], zn[CH];
+#pragma unroll
+                     for (int i = 0; i < CH; ++i) {
+                       g[i] = __uint_as_float(v[i]);
+                       zn[i] = fmaf(-lr, g[i], z[i]);
+                     }
+                     store_ch(p.Gz + off + r * N5 + c * CH, g);
+                     if (lr != 0.f) store_ch(Zrow + c * CH, zn);
+                     if (p.do_forward) {
+                       uint32_t ph[CH / 2], pl[CH / 2];
+                       split_ch(zn, ph, pl);
+                       put_rowmajor(k.buf(1), r, c, ph);
+                       put_rowmajor(k.buf(2), r, c, pl);
+                     }
+                   });
+  }
+
+  if (p.do_forward && ok) {
+    if (!p.do_backward) load_row_to_operands(k, Zrow, r, 1, 2, -1, -1);     // Z row-major -> 1 (hi), 2 (lo)
+    load_row_to_operands(k, Wrow, r, -1, -1, 3, 4);                         // W^T -> 3, 4
+    // Zh = Z W (split operands): fp32 to scratch, Zh^T -> 0, 5, Zh row-major -> 1, 2
+    ok = product(k, [&]() { k.mma3(1, 2, 3, 4); }, nullptr, nullptr,
+                 [&](int c, const uint32_t (&v)[CH], const float (&)[CH], const float (&)[CH]) {
+                   float f[CH];
+#pragma unroll
+                   for (int i = 0; i < CH; ++i) f[i] = __uint_as_float(v[i]);
+                   store_ch(Zhrow + c * CH, f);
+                   uint32_t ph[CH / 2], pl[CH / 2];
+                   split_ch(f, ph, pl);
+                   put_transposed(k.buf(0), r, c, ph);
+                   put_transposed(k.buf(5), r, c, pl);
+                   put_rowmajor(k.buf(1), r, c, ph);
+                   put_rowmajor(k.buf(2), r, c, pl);
+                 });
+    // E = Zh^T Zh - I (split operands) and the start of the fixed point T = Phi(E - P_old):
+    // T^T -> 3, 4; T row-major -> 0, 5
+    if (ok)
+      ok = product(k, [&]() { k.mma3(0, 5, 0, 5); }, Prow, nullptr,
+                   [&](int c, const uint32_t (&v)[CH], const float (&pold)[CH], const float (&)[CH]) {
+                     float e[CH], t[CH];
+#pragma unroll
+                     for (int i = 0; i < CH; ++i) {
+                       const int col = CH * c + i;
+                       e[i] = __uint_as_float(v[i]) - ((col == r) ? 1.f : 0.f);
+                       t[i] = phi(e[i] - pold[i], r, col);
+                     }
+                     store_ch(Erow + c * CH, e);
+                     store_ch(Trow + c * CH, t);
+                     uint32_t ph[CH / 2], pl[CH / 2];
+                     split_ch(t, ph, pl);
+                     put_transposed(k.buf(3), r, c, ph);
+                     put_transposed(k.buf(4), r, c, pl);
+                     put_rowmajor(k.buf(0), r, c, ph);
+                     put_rowmajor(k.buf(5), r, c, pl);
+                   });
+    // sweeps T <- Phi(E - T^T T) until no entry moves (the count is data dependent: the whole problem is here)
+    int sweeps = 0;
+    bool converged = false;
+    while (ok && sweeps < p.max_sweeps && !converged) {
+      ++sweeps;
+      const bool accurate = sweeps > 2;
+      bool moved = false;
+      ok = product(k, [&]() { if (accurate) k.mma3(3, 4, 3, 4); else k.mma(3, 3, false); }, Erow, Trow,
+                   [&](int c, const uint32_t (&v)[CH], const float (&e)[CH], const float (&told)[CH]) {
+                     float pp[CH], t[CH];
+#pragma unroll
+                     for (int i = 0; i < CH; ++i) {
+                       pp[i] = __uint_as_float(v[i]);
+                       t[i] = phi(e[i] - pp[i], r, CH * c + i);
+                       if (!(fabsf(t[i] - told[i]) <= p.tol)) moved = true;
+                     }
+                     store_ch(Prow + c * CH, pp);
+                     store_ch(Trow + c * CH, t);
+                     uint32_t ph[CH / 2], pl[CH / 2];
+                     split_ch(t, ph, pl);
+                     put_transposed(k.buf(3), r, c, ph);
+                     put_transposed(k.buf(4), r, c, pl);
+                     put_rowmajor(k.buf(0), r, c, ph);
+                     put_rowmajor(k.buf(5), r, c, pl);
+                   });
+      converged = !__syncthreads_or(moved ? 1 : 0);
+    }
+    if (ok && !converged) { set_status(p.d_status, DQ_ERR_NOT_CONVERGED); }
+    const bool big = sweeps > 2;        // a large step: the first-order products on split operands as well
+    // Y = (I + T)^-1 - I by Y <- -T - T Y from Y = -T;  Y^T -> 3, 4 (T^T is no longer needed)
+    if (ok) {
+#pragma unroll 1
+      for (int c = 0; c < N5 / CH; ++c) {
+        float t[CH];
+        fetch_ch(Trow + c * CH, t);
+#pragma unroll
+        for (int i = 0; i < CH; ++i) t[i] = -t[i];
+        store_ch(Yrow + c * CH, t);
+        uint32_t ph[CH / 2], pl[CH / 2];
+        split_ch(t, ph, pl);
+        put_transposed(k.buf(3), r, c, ph);
+        put_transposed(k.buf(4), r, c, pl);
+      }
+    }
+    int terms = 0;
+    converged = false;
+    while (ok && terms < MAX_SERIES && !converged) {
+      ++terms;
+      bool moved = false;
+      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4); else k.mma(0, 3, false); }, Trow, Yrow,
+                   [&](int c, const uint32_t (&v)[CH], const float (&t)[CH], const float (&yold)[CH]) {
+                     float y[CH];
+#pragma unroll
+                     for (int i = 0; i < CH; ++i) {
+                       y[i] = -t[i] - __uint_as_float(v[i]);
+                       if (!(fabsf(y[i] - yold[i]) <= 2e-7f)) moved = true;
+                     }
+                     store_ch(Yrow + c * CH, y);
+                     uint32_t ph[CH / 2], pl[CH / 2];
+                     split_ch(y, ph, pl);
+                     put_transposed(k.buf(3), r, c, ph);
+                     put_transposed(k.buf(4), r, c, pl);
+                   });
+      converged = !__syncthreads_or(moved ? 1 : 0);
+    }
+    if (ok && !converged) { set_status(p.d_status, DQ_ERR_NOT_CONVERGED); }
+    // R = Zh + Zh Y
+    if (ok)
+      ok = product(k, [&]() { if (big) k.mma3(1, 2, 3, 4); else k.mma(1, 3, false); }, Zhrow, nullptr,
+                   [&](int c, const uint32_t (&v)[CH], const float (&zh)[CH], const float (&)[CH]) {
+                     float f[CH];
+#pragma unroll
+                     for (int i = 0; i < CH; ++i) f[i] = zh[i] + __uint_as_float(v[i]);
+                     store_ch(Rrow + c * CH, f);
+                     if (p.Rt) {   // bf16(R^T): for a fixed column the warp's 32 rows are 64 contiguous bytes
+                       __nv_bfloat16* rt = p.Rt + off + r;
+#pragma unroll
+                       for (int i = 0; i < CH; ++i) rt[(CH * c + i) * N5] = __float2bfloat16_rn(f[i]);
+                     }
+                   });
+    // W <- W + W Y  (W row-major -> 0, 5: T is no longer needed)
+    float dv = 1.f;
+    if (ok) {
+      load_row_to_operands(k, Wrow, r, 0, 5, -1, -1);
+      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4); else k.mma(0, 3, false); }, Wrow, nullptr,
+                   [&](int c, const uint32_t (&v)[CH], const float (&w)[CH], const float (&)[CH]) {
+                     float f[CH];
+#pragma unroll
+                     for (int i = 0; i < CH; ++i) {
+                       f[i] = w[i] + __uint_as_float(v[i]);
+                       if (CH * c + i == r) dv = f[i];
+                     }
+                     store_ch(Wrow + c * CH, f);
+                   });
+    }
+    if (ok) {   // rank / finiteness test on diag(W) = 1 / diag(U)
+      float mn = fabsf(dv), mx = fabsf(dv);
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+      if (lane == 0) { red[warp] = mn; red[4 + warp] = mx; }
+      if (!isfinite(dv)) set_status(p.d_status, DQ_ERR_NONFINITE);
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        const float a = fminf(fminf(red[0], red[1]), fminf(red[2], red[3]));
+        const float b = fmaxf(fmaxf(red[4], red[5]), fmaxf(red[6], red[7]));
+        if (!(a > 1e-6f * b) || !(dv > 0.f)) set_status(p.d_status, DQ_ERR_SINGULAR);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------- teardown
+  tmem_ld_wait();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(k.tmem, TC5_TMEM_COLS);
+  }
+}
+
+}  // namespace
+
+// Backward (do_backward), SGD update (lr != 0) and incremental forward (do_forward) of `batch` 128 x 128
+// problems, one CTA each.  scratch: [batch][4][128][128] fp32.  P: T^T T of the previous step (zeros after a
+// factorisation from scratch).
+dq_status qr128_step_tc5(Ctx& ctx, float* Z, float* W, float* P, float* R, __nv_bfloat16* Rt, const float* Gq, float* Gz,
+                         float* scratch, float lr, bool do_backward, bool do_forward, int max_sweeps, int batch) {
+  static SmemOptIn attr;
+  DQ_CHECK(opt_in_dynamic_smem(qr128_step_tc5_kernel, TC5_SMEM, attr));
+  Tc5Params p{};
+  p.Z = Z; p.W = W; p.P = P; p.R = R; p.Rt = Rt; p.Gq = Gq; p.Gz = Gz; p.scratch = scratch;
+  p.lr = lr; p.do_backward = do_backward ? 1 : 0; p.do_forward = do_forward ? 1 : 0;
+  p.max_sweeps = max_sweeps < 3 ? 3 : max_sweeps; p.tol = 1e-5f; p.d_status = ctx.d_status;
+  qr128_step_tc5_kernel<<<batch, TC5_THREADS, TC5_SMEM, ctx.stream>>>(p);
+  return after_launch(ctx);
+}
+
+}  // namespace dq

@@ -574,6 +574,16 @@ dq_status qr_tc_try_orthogonal_start(Ctx& ctx, QrWorkspace& ws, QrTcState& q, co
   return DQ_OK;
 }
 
+// One dense d x d x d product of the kind QR-Orth is made of (split-bf16 operands, nterms = 3, or plain bf16,
+// nterms = 1) on the handle's operand copies of Z and W^T, result to scratch: for measurement.
+dq_status qr_tc_bench_product(Ctx& ctx, QrWorkspace& ws, QrTcState& q, int d, int batch, int nterms) {
+  const int64_t dd = (int64_t)d * d;
+  const WSet w = wset(q, q.w_sel);
+  Op a{q.z_hi, q.z_lo, d, dd}, b{w.t_hi, w.t_lo, d, dd};
+  Out o; o.f32 = ws.Q; o.ld = d; o.bs = dd; o.nterms = nterms;
+  return gemm3(ctx, a, b, d, d, d, batch, o);
+}
+
 // U of the current factorisation for inspection: the Householder route leaves it in place; the incremental
 // route carries only W = U^-1, which is inverted here (split-bf16 accuracy, about 1e-5 relative).
 dq_status qr_tc_materialize_u(Ctx& ctx, QrWorkspace& ws, QrTcState& q, float* U, int d, int batch) {

@@ -109,6 +109,8 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
 // without a Householder start (*started = true).  Synchronises the stream.
 dq_status qr_tc_try_orthogonal_start(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, int d, int batch,
                                      float threshold, bool* started);
+// Measurement: one dense d^3 product on the handle's operand copies (nterms = 3: split-bf16; 1: plain bf16).
+dq_status qr_tc_bench_product(Ctx& ctx, QrWorkspace& ws, QrTcState& q, int d, int batch, int nterms);
 // Makes U hold the upper factor of the current factorisation (inverts W after incremental steps).
 dq_status qr_tc_materialize_u(Ctx& ctx, QrWorkspace& ws, QrTcState& q, float* U, int d, int batch);
 // split: three bf16 MMAs per product (split operands) instead of one.
