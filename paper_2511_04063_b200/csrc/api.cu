@@ -60,7 +60,6 @@ struct dq_calib {
   bool small128 = false;        // d == 128: shared-memory-resident batched QR-Orth
   bool tc5 = false;             // d == 128 on the tensor-core path: tcgen05 kernel for the incremental QR-Orth
   float* p128 = nullptr;        // [batch][128][128] T^T T of the last sweep (tc5)
-  float* scratch128 = nullptr;  // [batch][4][128][128] scratch of the tc5 kernel
   bool u128_fresh = false;      // U holds the upper factor of the current factorisation (tc5 carries only U^-1)
   bool r_stale = true;
   bool timing = false;
@@ -97,7 +96,7 @@ void free_all(dq_calib* h) {
   cayley_destroy(h->cay);
   objective_destroy(h->obj);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
-  cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw); cudaFree(h->p128); cudaFree(h->scratch128);
+  cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw); cudaFree(h->p128);
   cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->loss_tmp); cudaFree(h->f32_flags); cudaFree(h->ctx.d_status);
   cudaFree(h->ws.A); cudaFree(h->ws.V); cudaFree(h->ws.T); cudaFree(h->ws.W); cudaFree(h->ws.W2);
   cudaFree(h->ws.Q); cudaFree(h->ws.Winv); cudaFree(h->ws.B); cudaFree(h->ws.S); cudaFree(h->ws.tmp);
@@ -152,7 +151,7 @@ dq_status ensure_rotation(dq_calib* h) {
     __nv_bfloat16* rt = h->cfg.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr;
     if (h->qr_method == DQ_QR_ITERATIVE && h->small_warm) {
       if (h->tc5) {   // tcgen05 kernel: needs only W (no U), starts its fixed point from the last step's T^T T
-        DQ_CHECK(qr128_step_tc5(h->ctx, h->Z, h->ws.Winv, h->p128, h->R, rt, nullptr, nullptr, h->scratch128, 0.f,
+        DQ_CHECK(qr128_step_tc5(h->ctx, h->Z, h->ws.Winv, h->p128, h->R, rt, nullptr, nullptr, 0.f,
                                 false, true, h->qr_iters + 3, h->cfg.batch));
         h->u128_fresh = false;
       } else {
@@ -266,7 +265,7 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
   if (h->small128) {   // plain SGD is fused into the backward kernel; other optimisers follow it
     const float lr128 = h->optimizer == DQ_SGD ? c.lr : 0.f;
     if (h->tc5 && h->qr_method == DQ_QR_ITERATIVE)
-      DQ_CHECK(qr128_step_tc5(ctx, h->Z, h->ws.Winv, h->p128, h->R, nullptr, h->Gq, h->Gz, h->scratch128, lr128, true,
+      DQ_CHECK(qr128_step_tc5(ctx, h->Z, h->ws.Winv, h->p128, h->R, nullptr, h->Gq, h->Gz, lr128, true,
                               false, 0, batch));
     else
       DQ_CHECK(qr128_backward_sgd_tc(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, lr128, batch));
@@ -448,7 +447,7 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
       A(tc_init(h->tc, h->ctx, *cfg, d_X, (__nv_bfloat16*)h->G, h->qtc.rt_hi, &h->n_partials));
   }
   if (h->small128 && cfg->path == DQ_PATH_BF16_TC) {
-    A(dev_alloc(&h->p128, dd)); A(dev_alloc(&h->scratch128, 4 * dd));
+    A(dev_alloc(&h->p128, dd));
     h->tc5 = (st == DQ_OK);
   }
   A(dev_alloc(&h->partials, (int64_t)batch * (h->n_partials > 0 ? h->n_partials : 1)));

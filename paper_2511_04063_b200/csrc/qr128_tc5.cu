@@ -26,8 +26,10 @@ constexpr int PART_BYTES = N5 * N5 * 2;          // one bf16 operand part: two [
 constexpr int KBLK_BYTES = N5 * BLOCK_K * 2;     // 16 KB
 constexpr int N_BUFS = 6;
 constexpr int TC5_SMEM = N_BUFS * PART_BYTES + 1024 + 1024;
-constexpr int TC5_THREADS = 128;
-constexpr uint32_t TC5_TMEM_COLS = 128;
+constexpr int TC5_THREADS = 256;                // two threads per accumulator row, half of the columns each
+constexpr int CHUNKS_PER_THREAD = 4;
+constexpr uint32_t TC5_TMEM_COLS = 512;          // the accumulator and three fp32 matrices that stay on chip
+constexpr uint32_t REG_E = 128, REG_T = 256, REG_ZH = 384;   // tensor-memory columns of E (later Y), T and Zh
 constexpr int MAX_SERIES = 48;
 
 struct Tc5Params {
@@ -38,7 +40,6 @@ struct Tc5Params {
   __nv_bfloat16* Rt;   // nullable: bf16(R^T), the operand of O = X R
   const float* Gq;     // backward: dL/dR
   float* Gz;           // backward: dL/dZ
-  float* scratch;      // [batch][4][128][128] fp32: E, T, Zh, Y
   float lr;
   int do_backward, do_forward;
   int max_sweeps;
@@ -49,6 +50,24 @@ struct Tc5Params {
 __device__ __forceinline__ void fence_async_smem5() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 constexpr int CH = 16;                           // columns of the accumulator row handled at a time
+
+// This thread's lane of tensor memory also keeps its rows of the fp32 matrices the chain needs again (E, T, Zh,
+// Y): 16 columns per access, no shared or global memory traffic.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* f) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      :: "r"(taddr), "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]), "f"(f[4]), "f"(f[5]), "f"(f[6]), "f"(f[7]),
+         "f"(f[8]), "f"(f[9]), "f"(f[10]), "f"(f[11]), "f"(f[12]), "f"(f[13]), "f"(f[14]), "f"(f[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld16f(uint32_t taddr, float* f) {
+  uint32_t r[16];
+  tmem_ld16(taddr, r);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) f[i] = __uint_as_float(r[i]);
+}
 
 // CH consecutive fp32 of a row (two 32-byte accesses); a null source reads as zeros
 __device__ __forceinline__ void fetch_ch(const float* p, float* v) {
@@ -105,6 +124,7 @@ struct Tc5 {
   uint32_t parity;
   uint32_t tmem_row;    // accumulator, this thread's lane
   uint32_t tmem;        // accumulator base
+  int c_begin;          // first of this thread's CHUNKS_PER_THREAD chunks of its row
   int* d_status;
   __device__ __forceinline__ uint8_t* buf(int i) const { return smem + i * PART_BYTES; }
   // acc (+)= A B^T over the whole K = 128 (issuing thread only)
@@ -128,12 +148,14 @@ struct Tc5 {
 };
 
 // One product of the chain: all threads have written their operand rows; thread 0 issues the MMAs (issue());
-// every thread waits (bounded) for their completion and then runs body(c, v, a0, a1) on the CH-wide chunks of
-// its accumulator row, with the fp32 rows s0 / s1 (nullable; this thread's row of some matrix) fetched one
-// chunk ahead, the first chunk while the MMAs run.  Returns false if the wait gave up (for all threads alike).
+// every thread waits (bounded) for their completion and then runs body(c, v, g, x0, x1) on the CH-wide chunks of
+// its accumulator row.  g: the same chunk of the fp32 row `grow` in global memory (nullable; fetched one chunk
+// ahead, the first one while the MMAs run); x0 / x1: the same chunk of the matrices kept in tensor memory at
+// columns t0 / t1 (0: none).  Returns false if the wait gave up (for all threads alike).
 template <typename Issue, typename Body>
-__device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* s0, const float* s1, Body body) {
+__device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, uint32_t t0, uint32_t t1, Body body) {
   tmem_ld_wait();
+  tmem_st_wait();
   tc_fence_before();
   fence_async_smem5();
   __syncthreads();
@@ -142,26 +164,29 @@ __device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* s0, co
     issue();
     umma_commit(k.bar);
   }
-  float cur0[CH], cur1[CH];
-  fetch_ch(s0, cur0);
-  fetch_ch(s1, cur1);
+  const int c_begin = k.c_begin;
+  float ga[CH], gb[CH];
+  fetch_ch(grow ? grow + c_begin * CH : nullptr, ga);
   const bool done = mbar_wait(k.bar, k.parity, k.d_status);
   k.parity ^= 1u;
   tc_fence_after();
   if (!__syncthreads_and(done ? 1 : 0)) return false;
-#pragma unroll 1
-  for (int c = 0; c < N5 / CH; ++c) {
+  static_assert(CHUNKS_PER_THREAD % 2 == 0, "chunks are processed in pairs");
+  auto one = [&](int c, const float (&g)[CH]) {
     uint32_t v[CH];
+    float x0[CH], x1[CH];
     tmem_ld16(k.tmem_row + (uint32_t)(c * CH), v);
-    float nx0[CH], nx1[CH];
-    if (c + 1 < N5 / CH) {
-      fetch_ch(s0 ? s0 + (c + 1) * CH : nullptr, nx0);
-      fetch_ch(s1 ? s1 + (c + 1) * CH : nullptr, nx1);
-    }
+    if (t0) tmem_ld16f(k.tmem_row + t0 + (uint32_t)(c * CH), x0);
+    if (t1) tmem_ld16f(k.tmem_row + t1 + (uint32_t)(c * CH), x1);
     tmem_ld_wait();
-    body(c, v, cur0, cur1);
-#pragma unroll
-    for (int i = 0; i < CH; ++i) { cur0[i] = nx0[i]; cur1[i] = nx1[i]; }
+    body(c, v, g, x0, x1);
+  };
+#pragma unroll 1
+  for (int c = c_begin; c < c_begin + CHUNKS_PER_THREAD; c += 2) {
+    fetch_ch(grow ? grow + (c + 1) * CH : nullptr, gb);
+    one(c, ga);
+    if (c + 2 < c_begin + CHUNKS_PER_THREAD) fetch_ch(grow ? grow + (c + 2) * CH : nullptr, ga);
+    one(c + 1, gb);
   }
   return true;
 }
@@ -171,7 +196,7 @@ __device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* s0, co
 __device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* row, int r, int rm_hi, int rm_lo,
                                                      int tr_hi, int tr_lo) {
 #pragma unroll 1
-  for (int c = 0; c < N5 / CH; ++c) {
+  for (int c = k.c_begin; c < k.c_begin + CHUNKS_PER_THREAD; ++c) {
     float f[CH];
     fetch_ch(row + c * CH, f);
     uint32_t ph[CH / 2], pl[CH / 2];
@@ -194,9 +219,10 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
   const uint32_t bar = smem_base + N_BUFS * PART_BYTES;
   const uint32_t tmem_slot = bar + 16u;
   uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_ptr + N_BUFS * PART_BYTES + 16);
-  float* red = reinterpret_cast<float*>(smem_ptr + N_BUFS * PART_BYTES + 64);   // [8] block reductions
+  float* red = reinterpret_cast<float*>(smem_ptr + N_BUFS * PART_BYTES + 64);   // [16] block reductions
 
-  const int r = threadIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = 32 * (warp & 3) + lane;           // accumulator row (tensor-memory lane) of this thread
   const int64_t off = (int64_t)blockIdx.x * N5 * N5;
   float lr = p.lr;
   if (p.d_status && *p.d_status != 0) lr = 0.f;   // an earlier error freezes the latent
@@ -212,18 +238,16 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
   Tc5 k;
   k.smem = smem_ptr; k.smem_u = smem_base; k.bar = bar; k.parity = 0u; k.d_status = p.d_status;
   k.tmem = *tmem_slot_ptr;
-  k.tmem_row = k.tmem + ((uint32_t)(warp * 32) << 16);
+  k.tmem_row = k.tmem + ((uint32_t)((warp & 3) * 32) << 16);
+  k.c_begin = (warp >> 2) * CHUNKS_PER_THREAD;
 
   float* Zrow = p.Z + off + r * N5;
   float* Wrow = p.W + off + r * N5;
   float* Prow = p.P + off + r * N5;
   float* Rrow = p.R + off + r * N5;
-  float* sc = p.scratch + (int64_t)blockIdx.x * 4 * N5 * N5 + r * N5;
-  float* Erow = sc;
-  float* Trow = sc + N5 * N5;
-  float* Zhrow = sc + 2 * N5 * N5;
-  float* Yrow = sc + 3 * N5 * N5;
   bool ok = true;
+  using V = const uint32_t (&)[CH];
+  using F = const float (&)[CH];
 
   if (p.do_backward) {
     // operands: R row-major -> 0, R^T -> 1, Gq^T -> 2, W row-major -> 3   (hi parts)
@@ -231,8 +255,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
     load_row_to_operands(k, p.Gq + off + r * N5, r, -1, -1, 2, -1);
     load_row_to_operands(k, Wrow, r, 3, -1, -1, -1);
     // S = tril(R^T Gq - Gq^T R, -1), row-major -> 4
-    ok = product(k, [&]() { k.mma(1, 2, false); k.mma(2, 1, true, true); }, nullptr, nullptr,
-                 [&](int c, const uint32_t (&v)[CH], const float (&)[CH], const float (&)[CH]) {
+    ok = product(k, [&]() { k.mma(1, 2, false); k.mma(2, 1, true, true); }, nullptr, 0, 0,
+                 [&](int c, V v, F, F, F) {
                    float f[CH];
 #pragma unroll
                    for (int i = 0; i < CH; ++i) f[i] = (r > CH * c + i) ? __uint_as_float(v[i]) : 0.f;
@@ -242,8 +266,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                  });
     // D^T = W S^T, row-major -> 5
     if (ok)
-      ok = product(k, [&]() { k.mma(3, 4, false); }, nullptr, nullptr,
-                   [&](int c, const uint32_t (&v)[CH], const float (&)[CH], const float (&)[CH]) {
+      ok = product(k, [&]() { k.mma(3, 4, false); }, nullptr, 0, 0,
+                   [&](int c, V v, F, F, F) {
                      float f[CH];
 #pragma unroll
                      for (int i = 0; i < CH; ++i) f[i] = __uint_as_float(v[i]);
@@ -253,8 +277,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                    });
     // Gz = R D, then Z <- Z - lr Gz; the new latent goes straight into the forward's operands (1, 2)
     if (ok)
-      ok = product(k, [&]() { k.mma(0, 5, false); }, Zrow, nullptr,
-                   [&](int c, const uint32_t (&v)[CH], const float (&z)[CH], const float (&)[CH]) {
+      ok = product(k, [&]() { k.mma(0, 5, false); }, Zrow, 0, 0,
+                   [&](int c, V v, F z, F, F) {
                      float g[CH], zn[CH];
 #pragma unroll
                      for (int i = 0; i < CH; ++i) {
@@ -275,13 +299,13 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
   if (p.do_forward && ok) {
     if (!p.do_backward) load_row_to_operands(k, Zrow, r, 1, 2, -1, -1);     // Z row-major -> 1 (hi), 2 (lo)
     load_row_to_operands(k, Wrow, r, -1, -1, 3, 4);                         // W^T -> 3, 4
-    // Zh = Z W (split operands): fp32 to scratch, Zh^T -> 0, 5, Zh row-major -> 1, 2
-    ok = product(k, [&]() { k.mma3(1, 2, 3, 4); }, nullptr, nullptr,
-                 [&](int c, const uint32_t (&v)[CH], const float (&)[CH], const float (&)[CH]) {
+    // Zh = Z W (split operands): fp32 kept in tensor memory, Zh^T -> 0, 5, Zh row-major -> 1, 2
+    ok = product(k, [&]() { k.mma3(1, 2, 3, 4); }, nullptr, 0, 0,
+                 [&](int c, V v, F, F, F) {
                    float f[CH];
 #pragma unroll
                    for (int i = 0; i < CH; ++i) f[i] = __uint_as_float(v[i]);
-                   store_ch(Zhrow + c * CH, f);
+                   tmem_st16(k.tmem_row + REG_ZH + (uint32_t)(c * CH), f);
                    uint32_t ph[CH / 2], pl[CH / 2];
                    split_ch(f, ph, pl);
                    put_transposed(k.buf(0), r, c, ph);
@@ -290,10 +314,10 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                    put_rowmajor(k.buf(2), r, c, pl);
                  });
     // E = Zh^T Zh - I (split operands) and the start of the fixed point T = Phi(E - P_old):
-    // T^T -> 3, 4; T row-major -> 0, 5
+    // T^T -> 3, 4; T row-major -> 0, 5; E and T (fp32) stay in tensor memory
     if (ok)
-      ok = product(k, [&]() { k.mma3(0, 5, 0, 5); }, Prow, nullptr,
-                   [&](int c, const uint32_t (&v)[CH], const float (&pold)[CH], const float (&)[CH]) {
+      ok = product(k, [&]() { k.mma3(0, 5, 0, 5); }, Prow, 0, 0,
+                   [&](int c, V v, F pold, F, F) {
                      float e[CH], t[CH];
 #pragma unroll
                      for (int i = 0; i < CH; ++i) {
@@ -301,8 +325,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                        e[i] = __uint_as_float(v[i]) - ((col == r) ? 1.f : 0.f);
                        t[i] = phi(e[i] - pold[i], r, col);
                      }
-                     store_ch(Erow + c * CH, e);
-                     store_ch(Trow + c * CH, t);
+                     tmem_st16(k.tmem_row + REG_E + (uint32_t)(c * CH), e);
+                     tmem_st16(k.tmem_row + REG_T + (uint32_t)(c * CH), t);
                      uint32_t ph[CH / 2], pl[CH / 2];
                      split_ch(t, ph, pl);
                      put_transposed(k.buf(3), r, c, ph);
@@ -317,8 +341,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
       ++sweeps;
       const bool accurate = sweeps > 2;
       bool moved = false;
-      ok = product(k, [&]() { if (accurate) k.mma3(3, 4, 3, 4); else k.mma(3, 3, false); }, Erow, Trow,
-                   [&](int c, const uint32_t (&v)[CH], const float (&e)[CH], const float (&told)[CH]) {
+      ok = product(k, [&]() { if (accurate) k.mma3(3, 4, 3, 4); else k.mma(3, 3, false); }, nullptr, REG_E, REG_T,
+                   [&](int c, V v, F, F e, F told) {
                      float pp[CH], t[CH];
 #pragma unroll
                      for (int i = 0; i < CH; ++i) {
@@ -326,8 +350,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                        t[i] = phi(e[i] - pp[i], r, CH * c + i);
                        if (!(fabsf(t[i] - told[i]) <= p.tol)) moved = true;
                      }
-                     store_ch(Prow + c * CH, pp);
-                     store_ch(Trow + c * CH, t);
+                     store_ch(Prow + c * CH, pp);          // where the next step's fixed point starts
+                     tmem_st16(k.tmem_row + REG_T + (uint32_t)(c * CH), t);
                      uint32_t ph[CH / 2], pl[CH / 2];
                      split_ch(t, ph, pl);
                      put_transposed(k.buf(3), r, c, ph);
@@ -339,47 +363,72 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
     }
     if (ok && !converged) { set_status(p.d_status, DQ_ERR_NOT_CONVERGED); }
     const bool big = sweeps > 2;        // a large step: the first-order products on split operands as well
-    // Y = (I + T)^-1 - I by Y <- -T - T Y from Y = -T;  Y^T -> 3, 4 (T^T is no longer needed)
+    // Y = (I + T)^-1 - I by Y <- -T - T Y from Y = -T;  Y^T -> 3, 4 (T^T is no longer needed); Y (fp32) takes the
+    // place of E in tensor memory.  The terms shrink geometrically (ratio at most |T|), so the series stops as
+    // soon as the NEXT term, estimated from the last two, would change no entry by more than 2e-7: after a small
+    // step a single product.
+    constexpr float SERIES_TOL = 2e-7f;
+    uint32_t* red_u = reinterpret_cast<uint32_t*>(red);    // block-wide max of non-negative floats (as bits)
+    auto block_max = [&](float v) -> float {
+      if (threadIdx.x == 0) red_u[0] = 0u;
+      __syncthreads();
+      if (v > 0.f) atomicMax(red_u, __float_as_uint(v));
+      else if (!(v == 0.f)) atomicMax(red_u, 0x7f800000u);   // NaN: never converged
+      __syncthreads();
+      const float m = __uint_as_float(red_u[0]);
+      __syncthreads();
+      return m;
+    };
+    float prev = 0.f;
     if (ok) {
+      float tmax = 0.f;
+      tmem_st_wait();
 #pragma unroll 1
-      for (int c = 0; c < N5 / CH; ++c) {
+      for (int c = k.c_begin; c < k.c_begin + CHUNKS_PER_THREAD; ++c) {
         float t[CH];
-        fetch_ch(Trow + c * CH, t);
+        tmem_ld16f(k.tmem_row + REG_T + (uint32_t)(c * CH), t);
+        tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < CH; ++i) t[i] = -t[i];
-        store_ch(Yrow + c * CH, t);
+        for (int i = 0; i < CH; ++i) { t[i] = -t[i]; tmax = fmaxf(tmax, fabsf(t[i])); if (t[i] != t[i]) tmax = NAN; }
+        tmem_st16(k.tmem_row + REG_E + (uint32_t)(c * CH), t);
         uint32_t ph[CH / 2], pl[CH / 2];
         split_ch(t, ph, pl);
         put_transposed(k.buf(3), r, c, ph);
         put_transposed(k.buf(4), r, c, pl);
       }
+      prev = block_max(tmax);
     }
     int terms = 0;
-    converged = false;
+    converged = !(prev > 0.f);          // T = 0: Y = 0
     while (ok && terms < MAX_SERIES && !converged) {
       ++terms;
-      bool moved = false;
-      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4); else k.mma(0, 3, false); }, Trow, Yrow,
-                   [&](int c, const uint32_t (&v)[CH], const float (&t)[CH], const float (&yold)[CH]) {
+      float chg = 0.f;
+      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4); else k.mma(0, 3, false); }, nullptr, REG_T, REG_E,
+                   [&](int c, V v, F, F t, F yold) {
                      float y[CH];
 #pragma unroll
                      for (int i = 0; i < CH; ++i) {
                        y[i] = -t[i] - __uint_as_float(v[i]);
-                       if (!(fabsf(y[i] - yold[i]) <= 2e-7f)) moved = true;
+                       const float dlt = fabsf(y[i] - yold[i]);
+                       chg = (dlt == dlt) ? fmaxf(chg, dlt) : NAN;
                      }
-                     store_ch(Yrow + c * CH, y);
+                     tmem_st16(k.tmem_row + REG_E + (uint32_t)(c * CH), y);
                      uint32_t ph[CH / 2], pl[CH / 2];
                      split_ch(y, ph, pl);
                      put_transposed(k.buf(3), r, c, ph);
                      put_transposed(k.buf(4), r, c, pl);
                    });
-      converged = !__syncthreads_or(moved ? 1 : 0);
+      const float m = block_max(chg);
+      // next term ~ m * (m / prev), with the ratio capped below 1 so that a stalled series is not mistaken for done
+      const float ratio = fminf(m / prev, 0.5f);
+      converged = (m <= SERIES_TOL) || (m * ratio <= SERIES_TOL && m < prev);
+      prev = m;
     }
     if (ok && !converged) { set_status(p.d_status, DQ_ERR_NOT_CONVERGED); }
     // R = Zh + Zh Y
     if (ok)
-      ok = product(k, [&]() { if (big) k.mma3(1, 2, 3, 4); else k.mma(1, 3, false); }, Zhrow, nullptr,
-                   [&](int c, const uint32_t (&v)[CH], const float (&zh)[CH], const float (&)[CH]) {
+      ok = product(k, [&]() { if (big) k.mma3(1, 2, 3, 4); else k.mma(1, 3, false); }, nullptr, REG_ZH, 0,
+                   [&](int c, V v, F, F zh, F) {
                      float f[CH];
 #pragma unroll
                      for (int i = 0; i < CH; ++i) f[i] = zh[i] + __uint_as_float(v[i]);
@@ -391,11 +440,11 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                      }
                    });
     // W <- W + W Y  (W row-major -> 0, 5: T is no longer needed)
-    float dv = 1.f;
+    float dv = NAN;                     // the diagonal entry, in the thread whose chunks hold it
     if (ok) {
       load_row_to_operands(k, Wrow, r, 0, 5, -1, -1);
-      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4); else k.mma(0, 3, false); }, Wrow, nullptr,
-                   [&](int c, const uint32_t (&v)[CH], const float (&w)[CH], const float (&)[CH]) {
+      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4); else k.mma(0, 3, false); }, Wrow, 0, 0,
+                   [&](int c, V v, F w, F, F) {
                      float f[CH];
 #pragma unroll
                      for (int i = 0; i < CH; ++i) {
@@ -406,25 +455,28 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                    });
     }
     if (ok) {   // rank / finiteness test on diag(W) = 1 / diag(U)
-      float mn = fabsf(dv), mx = fabsf(dv);
+      const bool owner = (r / CH) >= k.c_begin && (r / CH) < k.c_begin + CHUNKS_PER_THREAD;
+      float mn = owner ? fabsf(dv) : INFINITY, mx = owner ? fabsf(dv) : 0.f;
 #pragma unroll
       for (int o = 16; o >= 1; o >>= 1) {
         mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       }
-      if (lane == 0) { red[warp] = mn; red[4 + warp] = mx; }
-      if (!isfinite(dv)) set_status(p.d_status, DQ_ERR_NONFINITE);
+      if (lane == 0) { red[warp] = mn; red[8 + warp] = mx; }
+      if (owner && !(isfinite(dv) && dv > 0.f))
+        set_status(p.d_status, isfinite(dv) ? DQ_ERR_SINGULAR : DQ_ERR_NONFINITE);
       __syncthreads();
       if (threadIdx.x == 0) {
-        const float a = fminf(fminf(red[0], red[1]), fminf(red[2], red[3]));
-        const float b = fmaxf(fmaxf(red[4], red[5]), fmaxf(red[6], red[7]));
-        if (!(a > 1e-6f * b) || !(dv > 0.f)) set_status(p.d_status, DQ_ERR_SINGULAR);
+        float a = INFINITY, b = 0.f;
+        for (int i = 0; i < 8; ++i) { a = fminf(a, red[i]); b = fmaxf(b, red[8 + i]); }
+        if (!(a > 1e-6f * b)) set_status(p.d_status, DQ_ERR_SINGULAR);
       }
     }
   }
 
   // ------------------------------------------------------------- teardown
   tmem_ld_wait();
+  tmem_st_wait();
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {
@@ -436,14 +488,13 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
 }  // namespace
 
 // Backward (do_backward), SGD update (lr != 0) and incremental forward (do_forward) of `batch` 128 x 128
-// problems, one CTA each.  scratch: [batch][4][128][128] fp32.  P: T^T T of the previous step (zeros after a
-// factorisation from scratch).
+// problems, one CTA each.  P: T^T T of the previous step (zeros after a factorisation from scratch).
 dq_status qr128_step_tc5(Ctx& ctx, float* Z, float* W, float* P, float* R, __nv_bfloat16* Rt, const float* Gq, float* Gz,
-                         float* scratch, float lr, bool do_backward, bool do_forward, int max_sweeps, int batch) {
+                         float lr, bool do_backward, bool do_forward, int max_sweeps, int batch) {
   static SmemOptIn attr;
   DQ_CHECK(opt_in_dynamic_smem(qr128_step_tc5_kernel, TC5_SMEM, attr));
   Tc5Params p{};
-  p.Z = Z; p.W = W; p.P = P; p.R = R; p.Rt = Rt; p.Gq = Gq; p.Gz = Gz; p.scratch = scratch;
+  p.Z = Z; p.W = W; p.P = P; p.R = R; p.Rt = Rt; p.Gq = Gq; p.Gz = Gz;
   p.lr = lr; p.do_backward = do_backward ? 1 : 0; p.do_forward = do_forward ? 1 : 0;
   p.max_sweeps = max_sweeps < 3 ? 3 : max_sweeps; p.tol = 1e-5f; p.d_status = ctx.d_status;
   qr128_step_tc5_kernel<<<batch, TC5_THREADS, TC5_SMEM, ctx.stream>>>(p);

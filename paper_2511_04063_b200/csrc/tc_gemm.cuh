@@ -340,16 +340,22 @@ __device__ __forceinline__ void epi_gen_chunk(const Params& p, const uint32_t (&
 template <int N_COLS>
 __device__ __forceinline__ void epi_gen_tile(const Params& p, uint32_t taddr, int b, int row, int col_base,
                                              int64_t out_off, const GenAddends& first_chunk, bool& moved) {
-  GenAddends cur = first_chunk;
+  // two sets of addends used alternately: the set fetched during chunk c is first read in chunk c + 1, and no
+  // register copy (which would wait for the loads) stands between them
+  GenAddends ga = first_chunk, gb;
+  constexpr int NCH = N_COLS / GEN_CH;
+  static_assert(NCH % 2 == 0, "chunks are processed in pairs");
 #pragma unroll 1
-  for (int c = 0; c < N_COLS / GEN_CH; ++c) {
+  for (int c = 0; c < NCH; c += 2) {
     uint32_t v[GEN_CH];
     tmem_ld16(taddr + (uint32_t)(c * GEN_CH), v);
-    GenAddends next;
-    if (c + 1 < N_COLS / GEN_CH) epi_gen_fetch(p, out_off + (c + 1) * GEN_CH, next);
+    epi_gen_fetch(p, out_off + (c + 1) * GEN_CH, gb);
     tmem_ld_wait();
-    epi_gen_chunk(p, v, b, row, col_base + c * GEN_CH, out_off + c * GEN_CH, cur, moved);
-    cur = next;
+    epi_gen_chunk(p, v, b, row, col_base + c * GEN_CH, out_off + c * GEN_CH, ga, moved);
+    tmem_ld16(taddr + (uint32_t)((c + 1) * GEN_CH), v);
+    if (c + 2 < NCH) epi_gen_fetch(p, out_off + (c + 2) * GEN_CH, ga);
+    tmem_ld_wait();
+    epi_gen_chunk(p, v, b, row, col_base + (c + 1) * GEN_CH, out_off + (c + 1) * GEN_CH, gb, moved);
   }
 }
 
