@@ -2,8 +2,8 @@
 // 128^3 product as tcgen05.mma on bf16 (hi, lo) operand pairs that the CTA itself writes into shared memory
 // in the K-major 128-byte-swizzled layout, accumulator in tensor memory, one thread per accumulator row.
 //
-//   backward  S = tril(R^T Gq - Gq^T R, -1) (one reduction over two operand pairs), D^T = W S^T, Gz = R D,
-//             Z <- Z - lr Gz                                                   (plain bf16 operands)
+//   backward  S = tril(R^T Gq - Gq^T R, -1) (one reduction over two operand pairs, split operands: the skew
+//             part is a small difference), D^T = W S^T, Gz = R D (plain bf16 operands), Z <- Z - lr Gz
 //   forward   incremental factorisation from the previous step's W = U^-1 (no U, no triangular inverse):
 //             Zh = Z W, E = Zh^T Zh - I, T <- Phi(E - T^T T) from Phi(E - P_old) until no entry moves,
 //             Y = (I + T)^-1 - I by the series Y <- -T - T Y until no entry moves, R = Zh + Zh Y, W <- W + W Y.
@@ -250,12 +250,17 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
   using F = const float (&)[CH];
 
   if (p.do_backward) {
-    // operands: R row-major -> 0, R^T -> 1, Gq^T -> 2, W row-major -> 3   (hi parts)
-    load_row_to_operands(k, Rrow, r, 0, -1, 1, -1);
-    load_row_to_operands(k, p.Gq + off + r * N5, r, -1, -1, 2, -1);
+    // operands: R row-major -> 0, R^T -> 1 (hi), 4 (lo), Gq^T -> 2 (hi), 5 (lo), W row-major -> 3
+    load_row_to_operands(k, Rrow, r, 0, -1, 1, 4);
+    load_row_to_operands(k, p.Gq + off + r * N5, r, -1, -1, 2, 5);
     load_row_to_operands(k, Wrow, r, 3, -1, -1, -1);
-    // S = tril(R^T Gq - Gq^T R, -1), row-major -> 4
-    ok = product(k, [&]() { k.mma(1, 2, false); k.mma(2, 1, true, true); }, nullptr, 0, 0,
+    // S = tril(R^T Gq - Gq^T R, -1), row-major -> 4.  The skew part is what is left of B = R^T Gq after a
+    // cancellation (B is close to symmetric near a stationary point), so this one product of the backward runs
+    // on split operands: three MMA groups per term, the second term with A negated.
+    ok = product(k, [&]() {
+                   k.mma3(1, 4, 2, 5);
+                   k.mma(2, 1, true, true); k.mma(2, 4, true, true); k.mma(5, 1, true, true);
+                 }, nullptr, 0, 0,
                  [&](int c, V v, F, F, F) {
                    float f[CH];
 #pragma unroll
