@@ -11,6 +11,8 @@
  *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.
  *   - Matrices are row-major.  X is [batch][n_tokens][ldx] (one token per row),
  *     latents / rotations are [batch][d][d] fp32.
+ *   - One process may use the library on several devices (a handle belongs to the device that was
+ *     current at dq_calib_init; per-device kernel attributes are set on first use of each device).
  *   - Every call returns a dq_status; nothing throws, aborts or traps.  Device
  *     side problems (rank-deficient latent, non-finite loss, a wait that ran
  *     out) are recorded in a device status word read by dq_calib_status().  The
@@ -101,7 +103,9 @@ dq_status dq_rotate_apply(const void* d_X, int32_t x_dtype, int64_t n, int32_t d
  *   - d <= 2048 (the size of the fixed array), d % 128 == 0, n % 128 == 0, ldx % 8 == ldy % 8 == 0;
  *     anything else returns DQ_ERR_UNSUPPORTED and launches nothing.
  *   - The first call on each device also looks up the array's device address; make that call
- *     once, with that device current, before any stream capture.
+ *     once, with that device current, before any stream capture.  It is also the call on which the
+ *     CUDA runtime may load this library's kernels (and the array itself) onto the device, which
+ *     takes device memory once: make it before the caller's arena takes the rest of HBM.
  *   - All calls share the one array.  Each call rewrites the part it uses before reading it, so
  *     calls on one stream are independent; calls that overlap on the GPU (different streams or
  *     threads without ordering between them) race on it and must be serialised by the caller. */

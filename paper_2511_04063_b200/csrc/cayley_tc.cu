@@ -21,11 +21,6 @@ using tch::Op;
 using tch::Out;
 using tch::gemm3;
 
-__device__ __forceinline__ void split2(float v, bf16& hi, bf16& lo) {
-  hi = __float2bfloat16_rn(v);
-  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-}
-
 // v = ca A + cb s B with s = alpha[b] (use_alpha) or 1; optional outputs: fp32 (may alias A),
 // split copy of v row-major, split copy of v^T.  n x n matrices, 32 x 32 tile per block.
 __global__ void __launch_bounds__(256) combine_split_kernel(const float* A, const float* __restrict__ B, float ca,

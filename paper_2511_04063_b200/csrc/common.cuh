@@ -54,6 +54,27 @@ __device__ __forceinline__ void set_status(int* d_status, int code) {
   if (d_status) atomicCAS(d_status, 0, code);
 }
 
+// v as a (hi, lo) pair of bf16 with hi + lo = v to about 2^-17 relative ("split bf16")
+__device__ __forceinline__ void split2(float v, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+  hi = __float2bfloat16_rn(v);
+  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+// Sum v[c] over the 32 lanes; lane c returns the total of column c.
+__device__ __forceinline__ float warp_transpose_reduce32(float (&v)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool up = (lane & off) != 0;
+#pragma unroll
+    for (int k = 0; k < off; ++k) {
+      const float send = up ? v[k] : v[k + off];
+      const float keep = up ? v[k + off] : v[k];
+      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+  return v[0];
+}
+
 // ---------------------------------------------------------------------------
 // fp32 FMA GEMM (gemm_ffma.cu):  C = alpha op(A) op(B) + beta C, batched/strided.
 // op(A) is M x K, op(B) is K x N; trans* = 1 means the stored matrix is the

@@ -29,21 +29,6 @@ __device__ __forceinline__ float ld_dsmem(uint32_t smem_addr, int rank) {
   return v;
 }
 
-// Sum v[c] over the 32 lanes; lane c returns the total of column c.
-__device__ __forceinline__ float warp_transpose_reduce32(float (&v)[32], int lane) {
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) {
-    const bool up = (lane & off) != 0;
-#pragma unroll
-    for (int k = 0; k < off; ++k) {
-      const float send = up ? v[k] : v[k + off];
-      const float keep = up ? v[k + off] : v[k];
-      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-    }
-  }
-  return v[0];
-}
-
 // Factor A[c0:d, c0:c0+32] (row-major, leading dimension d) in place:
 //   A  <- upper-triangular part of the panel (zeros below the diagonal)
 //   V  <- Householder vectors, unit diagonal, zeros above (same position as A)

@@ -34,10 +34,6 @@ constexpr int IB = 32;     // inner panel width
 constexpr int OB = 128;    // outer block width
 constexpr int MAX_CS = 16; // CTAs per cluster (8 is the portable limit; 16 where the device allows it)
 
-__device__ __forceinline__ void split2(float v, bf16& hi, bf16& lo) {
-  hi = __float2bfloat16_rn(v);
-  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-}
 __device__ __forceinline__ uint32_t pack2(bf16 a, bf16 b) {
   return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
 }
@@ -48,21 +44,6 @@ __device__ __forceinline__ void st_dsmem(float* local, int rank, float v) {
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(addr), "r"(rank));
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
-}
-
-// Sum v[c] over the 32 lanes; lane c returns the total of entry c.
-__device__ __forceinline__ float warp_transpose_reduce32(float (&v)[32], int lane) {
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) {
-    const bool up = (lane & off) != 0;
-#pragma unroll
-    for (int k = 0; k < off; ++k) {
-      const float send = up ? v[k] : v[k + off];
-      const float keep = up ? v[k + off] : v[k];
-      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-    }
-  }
-  return v[0];
 }
 
 // At[c][r] = Z[r][c] (fp32) plus its split-bf16 copy; 32 x 32 tiles.

@@ -22,11 +22,6 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 
-__device__ __forceinline__ void split2(float v, bf16& hi, bf16& lo) {
-  hi = __float2bfloat16_rn(v);
-  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-}
-
 // dst(hi, lo)[b][r][c] = split(src[b][r][c])             (transpose == 0)
 // dst(hi, lo)[b][c][r] = split(src[b][r][c])             (transpose == 1)
 // src is n x n fp32 row-major (n % 32 == 0); dst dense n x n.
