@@ -276,8 +276,36 @@ WSet wset(const QrTcState& q, int sel) {
   return sel == 0 ? WSet{q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo} : WSet{q.wn2_hi, q.wn2_lo, q.wt2_hi, q.wt2_lo};
 }
 
+// The upper tiles in the order made for the product's k_mode (0: all k-blocks, 2, or 1|4).
 void upper_lists(Out& o, const QrTcState& q) {
-  o.tile_list = q.tl_upper; o.n_list = q.n_upper; o.tile_list2 = q.tl2_upper; o.n_list2 = q.n2_upper;
+  o.n_list = q.n_upper; o.n_list2 = q.n2_upper;
+  if (o.k_mode == 2) { o.tile_list = q.tl_upper_k2; o.tile_list2 = q.tl2_upper_k2; }
+  else if (o.k_mode == (1 | 4)) { o.tile_list = q.tl_upper_band; o.tile_list2 = q.tl2_upper_band; }
+  else { o.tile_list = q.tl_upper; o.tile_list2 = q.tl2_upper; }
+}
+
+// Lays `tiles` out for `workers` persistent workers that take entries w, w + workers, ... : rounds of `workers`
+// tiles in ascending cost, dealt from the heaviest round down, the heaviest tile of a round to the worker with
+// the least work so far.  The last round may be partial (it falls to workers 0 .. rem - 1) and takes the heaviest
+// tiles.  A worker's first tile is its lightest: its products are the ones nothing overlaps with.
+template <class Cost>
+std::vector<int> balanced_order(std::vector<int> tiles, int workers, Cost cost) {
+  std::stable_sort(tiles.begin(), tiles.end(), [&](int a, int b) { return cost(a) > cost(b); });
+  const int n = (int)tiles.size(), full = n / workers, rem = n % workers;
+  std::vector<int> out(n);
+  std::vector<int64_t> load(workers, 0);
+  int next = 0;
+  for (int w = 0; w < rem; ++w) { out[full * workers + w] = tiles[next]; load[w] += cost(tiles[next]); ++next; }
+  std::vector<int> by_load(workers);
+  for (int r = full - 1; r >= 0; --r) {
+    for (int w = 0; w < workers; ++w) by_load[w] = w;
+    std::stable_sort(by_load.begin(), by_load.end(), [&](int a, int b) { return load[a] < load[b]; });
+    for (int j = 0; j < workers; ++j) {
+      const int w = by_load[j];
+      out[r * workers + w] = tiles[next]; load[w] += cost(tiles[next]); ++next;
+    }
+  }
+  return out;
 }
 
 }  // namespace
@@ -302,32 +330,37 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   DQ_CHECK(alloc(&q.tw_hi, dd)); DQ_CHECK(alloc(&q.tw_lo, dd));
   DQ_CHECK(alloc(&q.sweep_flags, 80));
   DQ_CHECK(alloc(&q.uot_hi, dd)); DQ_CHECK(alloc(&q.uot_lo, dd));
-  for (int unit = 128; unit <= 256; unit *= 2) {   // tile orders: most expensive tiles first, dealt round-robin to the persistent CTAs
+  for (int unit = 128; unit <= 256; unit *= 2) {   // tile orders (see QrTcState)
     if (d % unit != 0) break;
     const int nb = d / unit;
-    std::vector<int> upper, lower, desc, asc;
+    const int workers = unit == 128 ? sm_count : (sm_count / 2 > 0 ? sm_count / 2 : 1);
+    std::vector<int> upper, lower, all;
     for (int j = 0; j < nb; ++j)
       for (int i = 0; i < nb; ++i) {
         if (i <= j) upper.push_back(i | (j << 16));
         if (i >= j) lower.push_back(i | (j << 16));
-        desc.push_back(i | (j << 16));
+        all.push_back(i | (j << 16));
       }
-    std::stable_sort(upper.begin(), upper.end(), [](int a, int b) { return (a & 0xffff) > (b & 0xffff); });
-    std::stable_sort(desc.begin(), desc.end(), [](int a, int b) { return (a >> 16) > (b >> 16); });
-    asc = desc;
-    std::reverse(asc.begin(), asc.end());
-    int*& tu = (unit == 128) ? q.tl_upper : q.tl2_upper;
-    int*& tlw = (unit == 128) ? q.tl_lower : q.tl2_lower;
-    int*& td = (unit == 128) ? q.tl_desc_nb : q.tl2_desc_nb;
-    int*& ta = (unit == 128) ? q.tl_asc_nb : q.tl2_asc_nb;
-    ((unit == 128) ? q.n_upper : q.n2_upper) = (int)upper.size();
-    ((unit == 128) ? q.n_all : q.n2_all) = (int)desc.size();
-    DQ_CHECK(alloc(&tu, (int64_t)upper.size())); DQ_CHECK(alloc(&tlw, (int64_t)lower.size()));
-    DQ_CHECK(alloc(&td, (int64_t)desc.size())); DQ_CHECK(alloc(&ta, (int64_t)desc.size()));
-    DQ_CHECK_CUDA(cudaMemcpy(tu, upper.data(), sizeof(int) * upper.size(), cudaMemcpyHostToDevice));
-    DQ_CHECK_CUDA(cudaMemcpy(tlw, lower.data(), sizeof(int) * lower.size(), cudaMemcpyHostToDevice));
-    DQ_CHECK_CUDA(cudaMemcpy(td, desc.data(), sizeof(int) * desc.size(), cudaMemcpyHostToDevice));
-    DQ_CHECK_CUDA(cudaMemcpy(ta, asc.data(), sizeof(int) * asc.size(), cudaMemcpyHostToDevice));
+    auto mb_of = [](int t) { return t & 0xffff; };
+    auto nb_of = [](int t) { return t >> 16; };
+    const std::vector<int> up_k2 = balanced_order(upper, workers, [&](int t) { return mb_of(t) + 1; });
+    const std::vector<int> up_band = balanced_order(upper, workers, [&](int t) { return nb_of(t) - mb_of(t) + 1; });
+    const std::vector<int> k4 = balanced_order(all, workers, [&](int t) { return nb_of(t) + 1; });
+    const std::vector<int> k8 = balanced_order(all, workers, [&](int t) { return nb - nb_of(t); });
+    const bool one = unit == 128;
+    (one ? q.n_upper : q.n2_upper) = (int)upper.size();
+    (one ? q.n_all : q.n2_all) = (int)all.size();
+    auto upload = [&](int*& dst, const std::vector<int>& v) -> dq_status {
+      DQ_CHECK(alloc(&dst, (int64_t)v.size()));
+      DQ_CHECK_CUDA(cudaMemcpy(dst, v.data(), sizeof(int) * v.size(), cudaMemcpyHostToDevice));
+      return DQ_OK;
+    };
+    DQ_CHECK(upload(one ? q.tl_upper : q.tl2_upper, upper));
+    DQ_CHECK(upload(one ? q.tl_upper_k2 : q.tl2_upper_k2, up_k2));
+    DQ_CHECK(upload(one ? q.tl_upper_band : q.tl2_upper_band, up_band));
+    DQ_CHECK(upload(one ? q.tl_lower : q.tl2_lower, lower));
+    DQ_CHECK(upload(one ? q.tl_k4 : q.tl2_k4, k4));
+    DQ_CHECK(upload(one ? q.tl_k8 : q.tl2_k8, k8));
   }
   q.ready = true;
   return DQ_OK;
@@ -340,8 +373,8 @@ void qr_tc_destroy(QrTcState& q) {
   for (bf16* p : all) cudaFree(p);
   cudaFree(q.P);
   cudaFree(q.y_hi); cudaFree(q.y_lo); cudaFree(q.w2_hi); cudaFree(q.w2_lo); cudaFree(q.part); cudaFree(q.T);
-  cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.uot_hi); cudaFree(q.uot_lo); cudaFree(q.tl_upper); cudaFree(q.tl_desc_nb); cudaFree(q.tl_asc_nb);
-  cudaFree(q.tl2_upper); cudaFree(q.tl2_desc_nb); cudaFree(q.tl2_asc_nb); cudaFree(q.tl_lower); cudaFree(q.tl2_lower); cudaFree(q.sweep_flags);
+  cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.uot_hi); cudaFree(q.uot_lo); cudaFree(q.tl_upper); cudaFree(q.tl_k4); cudaFree(q.tl_k8); cudaFree(q.tl_upper_k2); cudaFree(q.tl_upper_band);
+  cudaFree(q.tl2_upper); cudaFree(q.tl2_k4); cudaFree(q.tl2_k8); cudaFree(q.tl2_upper_k2); cudaFree(q.tl2_upper_band); cudaFree(q.tl_lower); cudaFree(q.tl2_lower); cudaFree(q.sweep_flags);
   q = QrTcState();
 }
 
@@ -411,7 +444,7 @@ dq_status qr_forward_incremental_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, con
     Op a{q.z_hi, q.z_lo, d, dd}, b{wc.t_hi, wc.t_lo, d, dd};
     Out o; o.f32 = Zh; o.ld = d; o.bs = dd; o.hi = zh_hi; o.lo = zh_lo; o.ld_h = d; o.bs_h = dd;
     o.t_hi = zht_hi; o.t_lo = zht_lo; o.ld_t = d; o.bs_t = dd;
-    o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
+    o.k_mode = 4; o.tile_list = q.tl_k4; o.n_list = q.n_all; o.tile_list2 = q.tl2_k4; o.n_list2 = q.n2_all;
     DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   }
   const int n_total = n_sweeps + 3;
@@ -476,7 +509,7 @@ dq_status qr_forward_incremental_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, con
     Op a{zh_hi, zh_lo, d, dd};
     Out o; o.f32 = R; o.ld = d; o.bs = dd; o.add1 = Zh; o.hi = q.r_hi; o.lo = need_lo ? q.r_lo : nullptr; o.ld_h = d; o.bs_h = dd;
     o.t_hi = q.rt_hi; o.t_lo = need_lo ? q.rt_lo : nullptr; o.ld_t = d; o.bs_t = dd;
-    o.k_mode = 4; o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
+    o.k_mode = 4; o.tile_list = q.tl_k4; o.n_list = q.n_all; o.tile_list2 = q.tl2_k4; o.n_list2 = q.n2_all;
     o.nterms = v ? 3 : 1; (v ? o.run_if : o.run_unless) = big;
     DQ_CHECK(gemm3(ctx, a, yt, d, d, d, batch, o));
   }
@@ -525,7 +558,7 @@ dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* 
   Out o; o.f32 = R; o.ld = d; o.bs = dd; o.hi = q.r_hi; o.lo = q.r_lo; o.ld_h = d; o.bs_h = dd;
   o.t_hi = q.rt_hi; o.t_lo = q.rt_lo; o.ld_t = d; o.bs_t = dd;
   o.k_mode = 4;   // W is upper triangular: W^T[j][k] = 0 for k > j
-  o.tile_list = q.tl_desc_nb; o.n_list = q.n_all; o.tile_list2 = q.tl2_desc_nb; o.n_list2 = q.n2_all;
+  o.tile_list = q.tl_k4; o.n_list = q.n_all; o.tile_list2 = q.tl2_k4; o.n_list2 = q.n2_all;
   return gemm3(ctx, a, b, d, d, d, batch, o);
 }
 
@@ -634,7 +667,7 @@ dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* G
   Op r{q.r_hi, q.r_lo, d, dd}, dt{q.m_hi, q.m_lo, d, dd};
   Out og; og.f32 = Gz; og.ld = d; og.bs = dd;
   og.k_mode = 8; og.nterms = split ? 3 : 1;
-  og.tile_list = q.tl_asc_nb; og.n_list = q.n_all; og.tile_list2 = q.tl2_asc_nb; og.n_list2 = q.n2_all;
+  og.tile_list = q.tl_k8; og.n_list = q.n_all; og.tile_list2 = q.tl2_k8; og.n_list2 = q.n2_all;
   return gemm3(ctx, r, dt, d, d, d, batch, og);
 }
 

@@ -86,16 +86,23 @@ struct QrTcState {
   bool z_split_fresh = false;                           // z_hi / z_lo are the split copy of the current latent
   bool t_warm = false;                                  // the current set of W copies and the fp32 W belong to the previous step's latent
   int* sweep_flags = nullptr;                           // [80] device flags: sweep k moved an entry
-  // tile orders for triangular products (device arrays of mb | nb << 16)
-  int* tl_upper = nullptr; int n_upper = 0;             // tiles mb <= nb, largest mb first
-  int* tl_lower = nullptr;                              // tiles mb >= nb (n_upper of them)
-  int* tl_desc_nb = nullptr;                            // all tiles, largest nb first
-  int* tl_asc_nb = nullptr; int n_all = 0;              // all tiles, smallest nb first
+  // Tile orders for triangular products (device arrays of mb | nb << 16).  The persistent workers (CTAs, or CTA
+  // pairs) take list entries round-robin, so each list is laid out for its number of workers and for the cost
+  // of its tiles (the k-blocks that the product's k_mode leaves): every worker gets the same number of tiles
+  // to within one and nearly the same number of k-blocks, its lightest tile first.
+  int* tl_upper = nullptr; int n_upper = 0;             // tiles mb <= nb, all k-blocks (uniform cost)
+  int* tl_upper_k2 = nullptr;                           // the same tiles for k_mode 2 (k-blocks up to mb)
+  int* tl_upper_band = nullptr;                         // the same tiles for k_mode 1|4 (k-blocks mb .. nb)
+  int* tl_lower = nullptr;                              // tiles mb >= nb (n_upper of them), uniform cost
+  int* tl_k4 = nullptr;                                 // all tiles for k_mode 4 (k-blocks up to nb)
+  int* tl_k8 = nullptr; int n_all = 0;                  // all tiles for k_mode 8 (k-blocks from nb)
   // the same orders in 256 x 256 tiles for the two-CTA kernel (d % 256 == 0 only)
   int* tl2_upper = nullptr; int n2_upper = 0;
+  int* tl2_upper_k2 = nullptr;
+  int* tl2_upper_band = nullptr;
   int* tl2_lower = nullptr;
-  int* tl2_desc_nb = nullptr;
-  int* tl2_asc_nb = nullptr; int n2_all = 0;
+  int* tl2_k4 = nullptr;
+  int* tl2_k8 = nullptr; int n2_all = 0;
 };
 dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count);
 void qr_tc_destroy(QrTcState& q);
