@@ -20,6 +20,7 @@ import os
 import subprocess
 import sys
 import tempfile
+import threading
 import time
 
 import numpy as np
@@ -48,17 +49,55 @@ def load_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle sampling during the timed region."""
+    """SM clock and throttle reasons during the timed region: an NVML polling thread (2 ms period, so that a
+    timed region of a few tens of milliseconds still holds several samples) beside the nvidia-smi query loop
+    (whose first sample can come later than a short region lasts).  Reads only; nothing is set."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, uuid: str = None):
         self.gpu = gpu_index
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.p = None
+        self.nvml = None
+        self.handle = None
+        self.rows = []          # (sm MHz, reason bit mask) from NVML
+        self.stop_flag = threading.Event()
+        self.thread = None
+        self.sm_max = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.handle = None
+            if uuid:
+                try:
+                    self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+                except Exception:
+                    self.handle = None
+            if self.handle is None:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(gpu_index)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.nvml = pynvml
+        except Exception:
+            self.nvml = None
+
+    def _poll(self):
+        nv = self.nvml
+        while not self.stop_flag.is_set():
+            try:
+                sm = nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+                self.rows.append((float(sm), int(mask)))
+            except Exception:
+                pass
+            time.sleep(0.002)
 
     def start(self):
+        if self.nvml is not None:
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
                                        "--format=csv,noheader,nounits", "-lms", "10"],
@@ -67,32 +106,45 @@ class ClockSampler:
             self.p = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.p is None:
-            return out
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except Exception:
-            self.p.kill()
-        self.f.flush()
-        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
-        os.unlink(self.f.name)
+        out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": 0}
         sm, reasons = [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in rows:
-            if len(r) < 9:
-                continue
+        if self.thread is not None:
+            self.stop_flag.set()
+            self.thread.join(timeout=2)
+            nv = self.nvml
+            bits = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                    "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                    "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                    "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+            for clock, mask in self.rows:
+                sm.append(clock)
+                for nme, bit in bits.items():
+                    if mask & bit:
+                        reasons.add(nme)
+        if self.p is not None:
+            self.p.terminate()
             try:
-                sm.append(float(r[1]))
-                out["sm_max_mhz"] = float(r[2])
-            except ValueError:
-                continue
-            for k, nme in enumerate(names):
-                if r[5 + k].strip().lower().startswith("active"):
-                    reasons.add(nme)
+                self.p.wait(timeout=5)
+            except Exception:
+                self.p.kill()
+            self.f.flush()
+            rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+            for r in rows:
+                if len(r) < 9:
+                    continue
+                try:
+                    sm.append(float(r[1]))
+                    out["sm_max_mhz"] = float(r[2])
+                except ValueError:
+                    continue
+                for k, nme in enumerate(self.NAMES):
+                    if r[5 + k].strip().lower().startswith("active"):
+                        reasons.add(nme)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
         if sm:
-            # samples under load = upper half of the observed clocks is not meaningful; take the median
             out["sm_mhz"] = float(np.median(sm))
         out["reasons"] = sorted(reasons)
         out["samples"] = len(sm)
@@ -235,7 +287,7 @@ def main():
     dq.dq_calib_step(h, W, loss_dev)
     st = dq.dq_calib_status(h)
     assert st == dq.DQ_OK, dq.status_string(st)
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, str(getattr(torch.cuda.get_device_properties(local_rank), "uuid", "") or ""))
     launches0 = dq.dq_calib_launch_count(h)
     barrier()
     sampler.start()
