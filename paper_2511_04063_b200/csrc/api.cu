@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <utility>
 
 #include "common.cuh"
 #include "tc_path.cuh"
@@ -61,6 +62,9 @@ struct dq_calib {
   bool tc5 = false;             // d == 128 on the tensor-core path: tcgen05 kernel for the incremental QR-Orth
   float* p128 = nullptr;        // [batch][128][128] T^T T of the last sweep (tc5)
   bool u128_fresh = false;      // U holds the upper factor of the current factorisation (tc5 carries only U^-1)
+  float* R_alt = nullptr;       // tc5: second rotation buffer; a fused step reads R and leaves the next rotation here, then the two swap
+  float* R_used = nullptr;      // rotation the last step used, when that is no longer R (fused steps)
+  int r_sel = 0;                // which of the two buffers R is (captured graphs hold the pointers)
   bool r_stale = true;
   bool timing = false;
   cudaEvent_t ev[DQ_PHASE_COUNT + 1] = {};
@@ -96,7 +100,7 @@ void free_all(dq_calib* h) {
   cayley_destroy(h->cay);
   objective_destroy(h->obj);
   cudaFree(h->Z); cudaFree(h->R); cudaFree(h->U); cudaFree(h->Gq); cudaFree(h->Gz); cudaFree(h->gq_part);
-  cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw); cudaFree(h->p128);
+  cudaFree(h->opt_m); cudaFree(h->opt_v); cudaFree(h->opt_pw); cudaFree(h->p128); cudaFree(h->R_alt);
   cudaFree(h->G); cudaFree(h->partials); cudaFree(h->loss_last); cudaFree(h->loss_tmp); cudaFree(h->f32_flags); cudaFree(h->ctx.d_status);
   cudaFree(h->ws.A); cudaFree(h->ws.V); cudaFree(h->ws.T); cudaFree(h->ws.W); cudaFree(h->ws.W2);
   cudaFree(h->ws.Q); cudaFree(h->ws.Winv); cudaFree(h->ws.B); cudaFree(h->ws.S); cudaFree(h->ws.tmp);
@@ -144,14 +148,30 @@ dq_status clear_status(dq_calib* h) {
   return DQ_OK;
 }
 
+// The fused launch left the next rotation in R_alt: it becomes R, the one the step used stays readable.
+void rotation_advanced(dq_calib* h) {
+  h->R_used = h->R;
+  std::swap(h->R, h->R_alt);
+  h->r_sel ^= 1;
+  h->u128_fresh = false;
+}
+
+// 128 x 128 latents on the tensor-core path with plain SGD: the backward launch of a step also runs the
+// incremental forward of the next one, so a step begins and ends with a current rotation.
+bool fuses_forward(const dq_calib* h, bool timed) {
+  return h->tc5 && h->qr_method == DQ_QR_ITERATIVE && h->optimizer == DQ_SGD && h->orth_method != DQ_ORTH_CAYLEY &&
+         h->small_warm && !timed;
+}
+
 dq_status ensure_rotation(dq_calib* h) {
   if (h->orth_method == DQ_ORTH_CAYLEY && h->cay_started) return DQ_OK;   // R is the iterate itself
   if (!h->r_stale) return DQ_OK;
+  h->R_used = nullptr;   // R is about to hold the rotation of the current latent
   if (h->small128) {
     __nv_bfloat16* rt = h->cfg.path == DQ_PATH_BF16_TC ? h->qtc.rt_hi : nullptr;
     if (h->qr_method == DQ_QR_ITERATIVE && h->small_warm) {
       if (h->tc5) {   // tcgen05 kernel: needs only W (no U), starts its fixed point from the last step's T^T T
-        DQ_CHECK(qr128_step_tc5(h->ctx, h->Z, h->ws.Winv, h->p128, h->R, rt, nullptr, nullptr, 0.f,
+        DQ_CHECK(qr128_step_tc5(h->ctx, h->Z, h->ws.Winv, h->p128, h->R, nullptr, rt, nullptr, nullptr, 0.f,
                                 false, true, h->qr_iters + 3, h->cfg.batch));
         h->u128_fresh = false;
       } else {
@@ -252,6 +272,7 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
   // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
   // (a7) Z <- Z - lr Gz  (fused into the backward kernel for 128 x 128 latents)
   const int64_t n_latent = (int64_t)d * d * batch;
+  bool fused_forward = false;
   if (cayley) {   // Algorithm 3 updates the rotation itself; there is no latent
     DQ_CHECK(cayley_step_tc(ctx, h->ws, h->qtc, h->cay, h->R, h->Gq, c.lr, d, batch));
     h->cay_started = true;
@@ -264,10 +285,16 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
   }
   if (h->small128) {   // plain SGD is fused into the backward kernel; other optimisers follow it
     const float lr128 = h->optimizer == DQ_SGD ? c.lr : 0.f;
-    if (h->tc5 && h->qr_method == DQ_QR_ITERATIVE)
-      DQ_CHECK(qr128_step_tc5(ctx, h->Z, h->ws.Winv, h->p128, h->R, nullptr, h->Gq, h->Gz, lr128, true,
-                              false, 0, batch));
-    else
+    if (h->tc5 && h->qr_method == DQ_QR_ITERATIVE) {
+      // With plain SGD the same launch goes on to the forward pass of the NEXT step (the new latent never leaves
+      // the CTA): the step ends with the rotation of the updated latent in place.  Timed steps keep the two
+      // phases apart.
+      fused_forward = fuses_forward(h, timed);
+      DQ_CHECK(qr128_step_tc5(ctx, h->Z, h->ws.Winv, h->p128, h->R, fused_forward ? h->R_alt : nullptr,
+                              fused_forward ? h->qtc.rt_hi : nullptr, h->Gq, h->Gz, lr128, true, fused_forward,
+                              fused_forward ? h->qr_iters + 3 : 0, batch));
+      if (fused_forward) rotation_advanced(h);
+    } else
       DQ_CHECK(qr128_backward_sgd_tc(ctx, h->R, h->ws.Winv, h->Gq, h->Gz, h->Z, lr128, batch));
     if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[4], ctx.stream));
   } else {
@@ -288,7 +315,8 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
     DQ_CHECK(momentum_update(ctx, h->Z, h->Gz, h->opt_m, c.lr, h->beta1, n_latent));
   else if (h->optimizer == DQ_ADAM)
     DQ_CHECK(adam_update(ctx, h->Z, h->Gz, h->opt_m, h->opt_v, h->opt_pw, c.lr, h->beta1, h->beta2, h->eps, n_latent));
-  h->r_stale = true;
+  h->r_stale = !fused_forward;
+  if (!fused_forward) h->R_used = nullptr;
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[5], ctx.stream));
   return DQ_OK;
 }
@@ -301,7 +329,7 @@ void drop_graphs(dq_calib* h) {   // the schedule or a kernel argument changed: 
 }
 
 // Which captured step fits the handle's state (see dq_calib::graph).
-int graph_slot(const dq_calib* h) { return (h->fast_qr && !h->small128) ? (h->qtc.w_sel & 1) : 0; }
+int graph_slot(const dq_calib* h) { return (h->fast_qr && !h->small128) ? (h->qtc.w_sel & 1) : (h->tc5 ? h->r_sel : 0); }
 
 // Capture one full step into an executable graph (after one eager step has set every
 // kernel attribute).  Failure is not an error: the handle keeps launching eagerly.
@@ -312,15 +340,21 @@ void try_capture(dq_calib* h) {
   const int64_t before = h->ctx.launches;
   const double flops_before = h->ctx.mma_flops;
   const QrTcState q_before = h->qtc;
+  const bool fused = fuses_forward(h, false);
   const bool f32_winv = h->f32_winv_valid, small_warm = h->small_warm, cay_started = h->cay_started;
+  float* const r_before = h->R; float* const r_alt_before = h->R_alt; float* const r_used_before = h->R_used;
+  const int r_sel_before = h->r_sel;
+  const bool u128_before = h->u128_fresh;
   auto restore = [&]() {
+    h->R = r_before; h->R_alt = r_alt_before; h->R_used = r_used_before; h->r_sel = r_sel_before;
+    h->u128_fresh = u128_before;
     h->ctx.launches = before;
     h->ctx.mma_flops = flops_before;
     h->qtc = q_before;
     h->f32_winv_valid = f32_winv; h->small_warm = small_warm; h->cay_started = cay_started;
-    h->r_stale = h->orth_method != DQ_ORTH_CAYLEY || !cay_started;
+    h->r_stale = (h->orth_method != DQ_ORTH_CAYLEY || !cay_started) && !fused;
   };
-  h->r_stale = true;
+  h->r_stale = !fused;   // (a fused step is captured, and replayed, with the rotation current)
   // With plain SGD the update kernel writes the split copy of the new latent, so a step captured while that
   // copy is current holds no split_kernel: it may only be replayed while the copy is current.
   sg.needs_z_split = h->fast_qr && h->qtc.z_split_fresh;
@@ -352,8 +386,10 @@ void try_capture(dq_calib* h) {
 // Host-side state after a replayed step (what enqueue_step would have left).
 void after_replayed_step(dq_calib* h) {
   const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
-  h->r_stale = !cayley;
+  h->r_stale = !cayley && !fuses_forward(h, false);
   if (cayley) return;
+  if (!h->r_stale) rotation_advanced(h);
+  else h->R_used = nullptr;
   if (h->fast_qr && !h->small128) {
     if (h->qr_method == DQ_QR_ITERATIVE) h->qtc.w_sel ^= 1;    // the step wrote the other set of W copies
     else h->qtc.u_fresh = true;
@@ -448,6 +484,7 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
   }
   if (h->small128 && cfg->path == DQ_PATH_BF16_TC) {
     A(dev_alloc(&h->p128, dd));
+    A(dev_alloc(&h->R_alt, dd));
     h->tc5 = (st == DQ_OK);
   }
   A(dev_alloc(&h->partials, (int64_t)batch * (h->n_partials > 0 ? h->n_partials : 1)));
@@ -480,7 +517,7 @@ dq_status dq_calib_step(dq_calib_t* h, int32_t n_steps, float* d_loss_out) {
     const bool cayley = h->orth_method == DQ_ORTH_CAYLEY;
     dq_calib::StepGraph& sg = h->graph[graph_slot(h)];
     const bool use_graph = cayley ? (!h->timing && h->cay_started && h->eager_steps_done >= 1)
-                                  : (!h->timing && h->r_stale && h->eager_steps_done >= 1 &&
+                                  : (!h->timing && h->r_stale != fuses_forward(h, false) && h->eager_steps_done >= 1 &&
                                      (!iterative || warm) &&
                                      (!sg.exec || !sg.needs_z_split || h->qtc.z_split_fresh));
     if (use_graph && !sg.exec && !sg.failed) try_capture(h);
@@ -736,7 +773,7 @@ dq_status dq_calib_debug_buffer(dq_calib_t* h, int32_t which, void** d_ptr, int6
   if (!h || !d_ptr || !n_elems) return DQ_ERR_INVALID_ARG;
   const int64_t dd = (int64_t)h->cfg.d * h->cfg.d * h->cfg.batch;
   switch (which) {
-    case DQ_BUF_R: *d_ptr = h->R; *n_elems = dd; break;
+    case DQ_BUF_R: *d_ptr = h->R_used ? h->R_used : h->R; *n_elems = dd; break;   // the rotation the last step used
     case DQ_BUF_U:
       if (h->tc5 && h->small_warm && !h->u128_fresh) return DQ_ERR_UNSUPPORTED;   // only U^-1 is carried there
       if (h->fast_qr && !h->small128 && !h->qtc.u_fresh && h->orth_method == DQ_ORTH_QR && h->qtc.t_warm) {

@@ -155,9 +155,9 @@ dq_status qr128_backward_sgd_tc(Ctx& ctx, const float* R, const float* W, const 
 
 // tcgen05 kernel (qr128_tc5.cu): backward + SGD (do_backward; lr = 0: no update) and / or the incremental forward
 // from W = U^-1 alone (do_forward; W and P = the last sweep's T^T T are updated in place, R and bf16(R^T)
-// written).  The fp32 intermediates stay in tensor memory.
-dq_status qr128_step_tc5(Ctx& ctx, float* Z, float* W, float* P, float* R, __nv_bfloat16* Rt, const float* Gq, float* Gz,
-                         float lr, bool do_backward, bool do_forward, int max_sweeps, int batch);
+// written to R_out, or to R if that is null).  The fp32 intermediates stay in tensor memory.
+dq_status qr128_step_tc5(Ctx& ctx, float* Z, float* W, float* P, float* R, float* R_out, __nv_bfloat16* Rt, const float* Gq,
+                         float* Gz, float lr, bool do_backward, bool do_forward, int max_sweeps, int batch);
 
 // out[i] = X[pi_seed(first + i)] for i < count: seeded sampling of token rows without replacement
 // (token_sampling.cu).  elem_bytes = 2 (bf16) or 4 (fp32); rows must be multiples of 16 bytes.

@@ -36,7 +36,8 @@ struct Tc5Params {
   float* Z;            // [batch][128][128] latent (updated when lr != 0)
   float* W;            // [batch][128][128] U^-1 of the previous factorisation (updated by the forward half)
   float* P;            // [batch][128][128] T^T T of the previous step's last sweep (updated)
-  float* R;            // [batch][128][128] rotation: read by the backward half, written by the forward half
+  float* R;            // [batch][128][128] rotation read by the backward half
+  float* R_out;        // rotation written by the forward half (may be R)
   __nv_bfloat16* Rt;   // nullable: bf16(R^T), the operand of O = X R
   const float* Gq;     // backward: dL/dR
   float* Gz;           // backward: dL/dZ
@@ -437,7 +438,7 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                      float f[CH];
 #pragma unroll
                      for (int i = 0; i < CH; ++i) f[i] = zh[i] + __uint_as_float(v[i]);
-                     store_ch(Rrow + c * CH, f);
+                     store_ch(p.R_out + off + r * N5 + c * CH, f);
                      if (p.Rt) {   // bf16(R^T): for a fixed column the warp's 32 rows are 64 contiguous bytes
                        __nv_bfloat16* rt = p.Rt + off + r;
 #pragma unroll
@@ -493,13 +494,14 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
 }  // namespace
 
 // Backward (do_backward), SGD update (lr != 0) and incremental forward (do_forward) of `batch` 128 x 128
-// problems, one CTA each.  P: T^T T of the previous step (zeros after a factorisation from scratch).
-dq_status qr128_step_tc5(Ctx& ctx, float* Z, float* W, float* P, float* R, __nv_bfloat16* Rt, const float* Gq, float* Gz,
-                         float lr, bool do_backward, bool do_forward, int max_sweeps, int batch) {
+// problems, one CTA each.  P: T^T T of the previous step (zeros after a factorisation from scratch).  The forward
+// half writes the rotation to R_out (nullptr: to R, which the backward half has read by then).
+dq_status qr128_step_tc5(Ctx& ctx, float* Z, float* W, float* P, float* R, float* R_out, __nv_bfloat16* Rt, const float* Gq,
+                         float* Gz, float lr, bool do_backward, bool do_forward, int max_sweeps, int batch) {
   static SmemOptIn attr;
   DQ_CHECK(opt_in_dynamic_smem(qr128_step_tc5_kernel, TC5_SMEM, attr));
   Tc5Params p{};
-  p.Z = Z; p.W = W; p.P = P; p.R = R; p.Rt = Rt; p.Gq = Gq; p.Gz = Gz;
+  p.Z = Z; p.W = W; p.P = P; p.R = R; p.R_out = R_out ? R_out : R; p.Rt = Rt; p.Gq = Gq; p.Gz = Gz;
   p.lr = lr; p.do_backward = do_backward ? 1 : 0; p.do_forward = do_forward ? 1 : 0;
   p.max_sweeps = max_sweeps < 3 ? 3 : max_sweeps; p.tol = 1e-5f; p.d_status = ctx.d_status;
   qr128_step_tc5_kernel<<<batch, TC5_THREADS, TC5_SMEM, ctx.stream>>>(p);

@@ -186,6 +186,19 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
   return d;
 }
+// Shared-memory matrix descriptor of an MN-major operand (the M or N index is the contiguous one): rows of 128
+// bytes = 64 consecutive M (N) indices of one k, 128-byte swizzle, groups of eight k 1024 bytes apart, the
+// next 64 M (N) indices `lbo_bytes` further on.  A tile that TMA loaded as [k][64 elements] is this layout.
+__device__ __forceinline__ uint64_t make_mnmajor_sw128_desc(uint32_t smem_addr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;   // leading byte offset: between 64-element groups of M (N)
+  d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset: between groups of eight k
+  d |= (uint64_t)1 << 46;                              // descriptor version
+  d |= (uint64_t)2 << 61;                              // SWIZZLE_128B
+  return d;
+}
+constexpr uint32_t IDESC_A_MN_MAJOR = 1u << 15;   // kind::f16 instruction descriptor: A is MN-major
 // kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both K-major, M = 128.
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);

@@ -35,6 +35,12 @@ struct PairSmem {
   static constexpr int STAGES = (NTERMS == 1) ? 6 : 3;
   static constexpr int TOTAL = STAGES * STAGE_BYTES + 1024 + 1024;
 };
+// Epilogue warps per CTA: the general epilogue is a chain of dependent steps per 16-column chunk (tensor-memory
+// load, addends from global memory, stores), so it runs on eight warps, two per quarter of the tensor-memory lanes,
+// each taking half of the tile's columns; the Whip and bf16 epilogues keep four.
+template <int EPI> __host__ __device__ constexpr int epi_warps() { return EPI == EPI_GEN ? 8 : 4; }
+template <int EPI> __host__ __device__ constexpr int pair_threads() { return 64 + 32 * epi_warps<EPI>(); }
+
 constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;             // clears the bit that separates the two CTAs of a pair
 constexpr uint32_t TMEM_COLS = 512;                     // two 256-column accumulators
 
@@ -91,7 +97,7 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16_pair() {
 // are mb | nb << 16 in those units (tri_skip and k_mode refer to them too), partials get eight values
 // per tile (CTA rank, lane quarter).
 template <int NTERMS, int EPI>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(pair_threads<EPI>(), 1)
 tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapB_lo,
                 const Params p) {
@@ -100,6 +106,8 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
   constexpr int STAGES = L::STAGES;
   constexpr int STAGE_BYTES = L::STAGE_BYTES;
   constexpr uint32_t IDESC = make_idesc_bf16_pair();
+  constexpr int EPI_WARPS = epi_warps<EPI>();
+  constexpr int N_EPI = PAIR_N / (EPI_WARPS / 4);   // columns of the tile one epilogue warp handles
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
@@ -116,7 +124,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 2 * EPI_WARPS); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tensormap(&mapA);
     prefetch_tensormap(&mapB);
@@ -228,8 +236,9 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------- epilogue (warps 2..5, both CTAs)
-    const int q = warp & 3;
+    // ------------------------------------------------------------- epilogue (warps 2.., both CTAs)
+    const int q = warp & 3;                                  // quarter of the tensor-memory lanes this warp may read
+    const int col_off = ((warp - 2) >> 2) * N_EPI;           // its share of the tile's columns
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -242,7 +251,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       if (p.tri_skip && mb > nb) continue;
       const int row = mb * PAIR_M + (int)rank * HALF + q * 32 + lane;
       const int64_t out_off = (int64_t)b * p.batch_stride + (int64_t)split * p.split_stride + (int64_t)row * p.ld +
-                              (int64_t)nb * PAIR_N;
+                              (int64_t)nb * PAIR_N + col_off;
       // EPI_GEN: the addends of the first chunk are fetched while the MMAs of this tile are still running
       GenAddends g0;
       if (EPI == EPI_GEN) epi_gen_fetch(p, out_off, g0);
@@ -251,8 +260,8 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       float esum = 0.f;
       bool moved = false;
       if (EPI == EPI_GEN) {
-        epi_gen_tile<PAIR_N>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * PAIR_N), b, row, nb * PAIR_N,
-                             out_off, g0, moved);
+        epi_gen_tile<N_EPI>(p, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * PAIR_N + col_off), b, row,
+                            nb * PAIR_N + col_off, out_off, g0, moved);
       } else {
 #pragma unroll 1
         for (int c = 0; c < PAIR_N / 32; ++c) {
@@ -287,7 +296,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_leader(tempty_bar(acc));   // eight arrivals (four warps of each CTA) free the accumulator
+      if (lane == 0) mbar_arrive_leader(tempty_bar(acc));   // the arrivals of all epilogue warps of both CTAs free the accumulator
       if (EPI == EPI_GEN && moved) {
         if (p.moved_out) *p.moved_out = 1;
         if (p.fail_if_moved) set_status(p.d_status, DQ_ERR_NOT_CONVERGED);

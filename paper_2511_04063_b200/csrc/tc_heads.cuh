@@ -5,16 +5,15 @@
 //   Gq_h += X_t^T G_t    (second tcgen05 product: G_t goes from the epilogue's registers into shared
 //                         memory as the K-major operand, the accumulator stays in tensor memory
 //                         for all tiles of the unit)
-// so the rotated activations and dL/dO never reach HBM and X is read exactly once: the channel-major
-// operand of the second product (X_t^T) is made on chip, the epilogue warps transpose the token-major
-// tile in shared memory (8 x 8 blocks through registers) while the first product runs.
+// so the rotated activations and dL/dO never reach HBM and X is read exactly once: the second product
+// reads the same token-major tile of X that TMA loaded for the first one, as its MN-major A operand
+// (reduction index = token, 64 consecutive channels per 128-byte row), so no channel-major copy is made.
 // R_h^T stays resident in shared memory for a unit (head, range of token tiles); every unit writes
 // one 128 x 128 fp32 partial of Gq and four loss partials, summed afterwards in a fixed order.
 //
-// 320 threads: warp 0 TMA producer (R_h^T and the X_t ring), warp 1 MMA issuer, warps 2..9 transpose +
-// epilogue (two warps per quarter of the tensor-memory lanes, 32 token columns each).  X_t is released once the
-// first product has retired and the tile has been transposed, X_t^T and G_t after the second product;
-// two O accumulators.  Every wait is bounded
+// 320 threads: warp 0 TMA producer (R_h^T and the X_t ring), warp 1 MMA issuer, warps 2..9 epilogue (two
+// warps per quarter of the tensor-memory lanes, 32 token columns each).  X_t and G_t are released once the
+// second product of the tile has retired; two O accumulators.  Every wait is bounded
 // (DQ_ERR_TIMEOUT on expiry).
 #pragma once
 #include "tc_gemm.cuh"
@@ -29,13 +28,12 @@ constexpr int KB_BYTES = 128 * BLOCK_K * 2;        // one [128 rows][64 bf16] K-
 constexpr int XKB_BYTES = TT * BLOCK_K * 2;        // one [TT rows][64 bf16] K-major block of X_t: 8 KB
 constexpr int RT_BYTES = 2 * KB_BYTES;             // R_h^T: rows = output channel, K = input channel (128)
 constexpr int XA_BYTES = 2 * XKB_BYTES;            // X_t:   rows = token (TT), K = input channel (two k-blocks)
-constexpr int XT_BYTES = KB_BYTES;                 // X_t^T: rows = input channel, K = token (TT = one k-block)
 constexpr int G_BYTES = KB_BYTES;                  // G_t^T: rows = output channel, K = token
 // Two CTAs share an SM (each under half of its shared memory and half of its tensor memory): while one
 // waits for a load or runs its epilogue the other issues products.  Tiles of 64 tokens keep a CTA at
-// 96 KB: R_h^T, two X_t stages, one X_t^T and one G_t buffer.
-constexpr int XA_STAGES = 2, XT_STAGES = 1, G_BUFS = 1;
-constexpr int SMEM_TOTAL = RT_BYTES + XA_STAGES * XA_BYTES + XT_STAGES * XT_BYTES + G_BUFS * G_BYTES + 1024 + 1024;
+// 96 KB: R_h^T, three X_t stages (a tile stays until its second product has retired) and one G_t buffer.
+constexpr int XA_STAGES = 3, G_BUFS = 1;
+constexpr int SMEM_TOTAL = RT_BYTES + XA_STAGES * XA_BYTES + G_BUFS * G_BYTES + 1024 + 1024;
 constexpr uint32_t TMEM_COLS = 256;                // O (2 x TT columns) + Gq (128 columns)
 constexpr int HEADS_THREADS = 320;
 constexpr int EPI_WARPS = 8;
@@ -54,20 +52,16 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __global__ void __launch_bounds__(HEADS_THREADS, 2)
 heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_constant__ CUtensorMap mapX, const Params p) {
   constexpr uint32_t IDESC_O = make_idesc_bf16(TT);     // O^T tile: 128 channels x TT tokens
-  constexpr uint32_t IDESC_Q = make_idesc_bf16(128);    // Gq: 128 x 128
+  constexpr uint32_t IDESC_Q = make_idesc_bf16(128) | IDESC_A_MN_MAJOR;    // Gq: 128 x 128, A = X_t^T read from the token-major tile
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t rt_smem = smem_base;
   const uint32_t xa_base = rt_smem + RT_BYTES;
-  const uint32_t xt_base = xa_base + XA_STAGES * XA_BYTES;
-  const uint32_t g_base = xt_base + XT_STAGES * XT_BYTES;
+  const uint32_t g_base = xa_base + XA_STAGES * XA_BYTES;
   const uint32_t bar_base = g_base + G_BUFS * G_BYTES;
-  constexpr int B_XAF = 0, B_XAE = B_XAF + XA_STAGES, B_XTF = B_XAE + XA_STAGES, B_XTE = B_XTF + XT_STAGES,
-                B_TF = B_XTE + XT_STAGES, B_TE = B_TF + 2, B_GF = B_TE + 2, B_GE = B_GF + G_BUFS, B_MISC = B_GE + G_BUFS;
+  constexpr int B_XAF = 0, B_XAE = B_XAF + XA_STAGES, B_TF = B_XAE + XA_STAGES, B_TE = B_TF + 2, B_GF = B_TE + 2, B_GE = B_GF + G_BUFS, B_MISC = B_GE + G_BUFS;
   auto xa_full = [&](int s) { return bar_base + 8u * (B_XAF + s); };
   auto xa_empty = [&](int s) { return bar_base + 8u * (B_XAE + s); };
-  auto xt_full = [&](int s) { return bar_base + 8u * (B_XTF + s); };
-  auto xt_empty = [&](int s) { return bar_base + 8u * (B_XTE + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (B_TF + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (B_TE + a); };
   auto gfull_bar = [&](int g) { return bar_base + 8u * (B_GF + g); };
@@ -81,9 +75,8 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < XA_STAGES; ++s) {
-      mbar_init(xa_full(s), 1); mbar_init(xa_empty(s), 1 + EPI_WARPS);   // first product + the transposing warps
+      mbar_init(xa_full(s), 1); mbar_init(xa_empty(s), 1);
     }
-    for (int s = 0; s < XT_STAGES; ++s) { mbar_init(xt_full(s), EPI_WARPS); mbar_init(xt_empty(s), 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EPI_WARPS); }
     for (int s = 0; s < G_BUFS; ++s) { mbar_init(gfull_bar(s), EPI_WARPS); mbar_init(gempty_bar(s), 1); }
     mbar_init(rtfull_bar, 1); mbar_init(rtempty_bar, 1);
@@ -134,7 +127,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
     // ------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       int st1 = 0, st2 = 0, acc = 0, g = 0;
-      uint32_t ph1 = 0, ph2 = 0, acc_phase = 0, g_phase = 0, rt_phase = 0, q_phase = 0;
+      uint32_t ph1 = 0, acc_phase = 0, g_phase = 0, rt_phase = 0, q_phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
         int b, t0, t1;
@@ -157,7 +150,6 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
                 umma_bf16(tmem_o, make_kmajor_sw128_desc(rt_smem + kb * KB_BYTES + k * UMMA_K * 2),
                           make_kmajor_sw128_desc(xa + kb * XKB_BYTES + k * UMMA_K * 2), IDESC_O, (kb > 0 || k > 0) ? 1u : 0u);
             umma_commit(tfull_bar(acc));
-            umma_commit(xa_empty(st1));                  // X_t can be replaced once this product has retired
             if (i == nt - 1) umma_commit(rtempty_bar);   // R_h^T may be replaced once these products retire
             if (++st1 == XA_STAGES) { st1 = 0; ph1 ^= 1u; }
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -168,19 +160,20 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
               if (!mbar_wait(qempty_bar, q_phase ^ 1u, p.d_status)) { ok = false; break; }
               q_phase ^= 1u;
             }
-            if (!mbar_wait(xt_full(st2), ph2, p.d_status)) { ok = false; break; }
             if (!mbar_wait(gfull_bar(g), g_phase, p.d_status)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t xt = xt_base + st2 * XT_BYTES;
+            // A = X_t^T (128 channels x 16 tokens per instruction) straight from the token-major tile of stage st2:
+            // 16 tokens = 16 rows of 128 bytes; channels 64..127 sit in the stage's second k-block
+            const uint32_t xs = xa_base + st2 * XA_BYTES;
             const uint32_t gb = g_base + g * G_BYTES;
 #pragma unroll
             for (int k = 0; k < TT / UMMA_K; ++k)
-              umma_bf16(tmem_q, make_kmajor_sw128_desc(xt + k * UMMA_K * 2), make_kmajor_sw128_desc(gb + k * UMMA_K * 2),
-                        IDESC_Q, (j > 0 || k > 0) ? 1u : 0u);
-            umma_commit(xt_empty(st2));
+              umma_bf16(tmem_q, make_mnmajor_sw128_desc(xs + k * UMMA_K * 128, XKB_BYTES),
+                        make_kmajor_sw128_desc(gb + k * UMMA_K * 2), IDESC_Q, (j > 0 || k > 0) ? 1u : 0u);
+            umma_commit(xa_empty(st2));                  // X_t can be replaced once this product has retired
             umma_commit(gempty_bar(g));
             if (j == nt - 1) umma_commit(qfull_bar);
-            if (++st2 == XT_STAGES) { st2 = 0; ph2 ^= 1u; }
+            if (++st2 == XA_STAGES) { st2 = 0; }
             if (++g == G_BUFS) { g = 0; g_phase ^= 1u; }
           }
         }
@@ -192,49 +185,14 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
     const int half = (warp - 2) >> 2;          // which 64 of the 128 columns
     const int row = q * 32 + lane;             // output channel (O^T, G^T) / input channel (Gq)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    int acc = 0, g = 0, sx = 0, sxt = 0;
-    uint32_t acc_phase = 0, g_phase = 0, q_phase = 0, px = 0, pxt = 0;
-    // transpose duty: this thread moves the 8 x 8 block (channels 8 bi.., tokens 8 bt..) of every tile; the
-    // diagonal assignment of blocks to lanes keeps both the 16-byte loads and the 16-byte stores of a
-    // quarter-warp on eight different bank groups of the swizzled tiles
-    const int e = (warp - 2) * 32 + lane;      // blocks: 16 (channels) x TT / 8 (tokens) = 128, threads 0..127
-    const int bi = (e & 7) + 8 * ((e >> 6) & 1);
-    const int bt = ((e & 7) + ((e >> 3) & 7)) & 7;
-    const bool transposer = e < 16 * (TT / 8);
-    uint8_t* xa_ptr = smem_raw + (xa_base - smem_u32(smem_raw));
-    uint8_t* xt_ptr = smem_raw + (xt_base - smem_u32(smem_raw));
+    int acc = 0, g = 0;
+    uint32_t acc_phase = 0, g_phase = 0, q_phase = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
       int b, t0, t1;
       unit_range(u, b, t0, t1);
       float esum = 0.f;
       for (int t = t0; t < t1; ++t) {
-        // ---- X_t^T of this tile (operand of the second product)
-        if (!mbar_wait(xa_full(sx), px, p.d_status)) { ok = false; break; }
-        if (!mbar_wait(xt_empty(sxt), pxt ^ 1u, p.d_status)) { ok = false; break; }
-        if (transposer) {
-          const uint8_t* src = xa_ptr + sx * XA_BYTES + (bi >> 3) * XKB_BYTES;
-          uint8_t* dst = xt_ptr + sxt * XT_BYTES;
-          uint32_t in[8][4];
-#pragma unroll
-          for (int r = 0; r < 8; ++r) {      // token 8 bt + r: chunk (bi & 7) of its row sits at (bi & 7) ^ r
-            const uint4 v = *reinterpret_cast<const uint4*>(src + (8 * bt + r) * 128 + (((bi & 7) ^ r) << 4));
-            in[r][0] = v.x; in[r][1] = v.y; in[r][2] = v.z; in[r][3] = v.w;
-          }
-#pragma unroll
-          for (int r = 0; r < 8; ++r) {      // channel 8 bi + r: its eight tokens form chunk (bt & 7) of row 8 bi + r
-            uint32_t o[4];
-#pragma unroll
-            for (int w = 0; w < 4; ++w)
-              o[w] = __byte_perm(in[2 * w][r >> 1], in[2 * w + 1][r >> 1], (r & 1) ? 0x7632 : 0x5410);
-            *reinterpret_cast<uint4*>(dst + (8 * bi + r) * 128 + ((bt ^ r) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-          }
-        }
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) { mbar_arrive(xt_full(sxt)); mbar_arrive(xa_empty(sx)); }
-        if (++sx == XA_STAGES) { sx = 0; px ^= 1u; }
-        if (++sxt == XT_STAGES) { sxt = 0; pxt ^= 1u; }
         // ---- Eq. 4 epilogue of O^T
         if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
         if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }

@@ -68,7 +68,7 @@ dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, con
   if (pairs < 1) return DQ_OK;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
-  cfg.blockDim = dim3(tc::NUM_THREADS, 1, 1);
+  cfg.blockDim = dim3(tc2::pair_threads<EPI>(), 1, 1);
   cfg.dynamicSmemBytes = SMEM;
   cfg.stream = ctx.stream;
   cudaLaunchAttribute at[1];

@@ -179,7 +179,10 @@ def test_a_failed_step_freezes_the_latent_until_the_method_is_changed():
     w = small("c2_7b", d=d, n_tokens=256, n_outlier_channels=1)
     c = Calib(w, Z0=_near_orthogonal(d, 1, 0.02, 5), lr=20.0)
     c.step(1)                                                       # Householder start, absurd step
-    assert c.status() == dq.DQ_OK
+    # (the tcgen05 kernel for 128 x 128 latents runs the next step's forward pass in the launch that updates the
+    # latent, so there the failure is known as soon as this step ends; elsewhere the next step finds it)
+    if not (d == 128 and path == "tc"):
+        assert c.status() == dq.DQ_OK
     Z1 = c.latent()
     c.step(3)                                                       # incremental (the default): too far
     assert c.status() != dq.DQ_OK
@@ -314,7 +317,10 @@ def test_failed_step_freezes_the_latent_on_the_other_incremental_kernels(name, d
     w = small(name, d=d, n_tokens=512, batch=2 if d == 128 else 1)
     c = Calib(w, Z0=_near_orthogonal(d, w.batch, 0.02, 11), lr=50.0)
     c.step(1)                                                       # Householder start, absurd step
-    assert c.status() == dq.DQ_OK
+    # (the tcgen05 kernel for 128 x 128 latents runs the next step's forward pass in the launch that updates the
+    # latent, so there the failure is known as soon as this step ends; elsewhere the next step finds it)
+    if not (d == 128 and path == "tc"):
+        assert c.status() == dq.DQ_OK
     Z1 = c.latent()
     c.step(3)
     assert c.status() != dq.DQ_OK
