@@ -195,7 +195,6 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
       for (int t = t0; t < t1; ++t) {
         // ---- Eq. 4 epilogue of O^T
         if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
-        if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }
         tc_fence_after();
         uint8_t* gbuf = g_ptr + g * G_BYTES;
         {   // this warp's 32 token columns of the TT-wide tile
@@ -203,6 +202,9 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
           uint32_t v[32];
           tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * TT + c * 32), v);
           tmem_ld_wait();
+          tc_fence_before();                     // the accumulator is in registers: the issuer may reuse it
+          __syncwarp();
+          if (lane == 0) mbar_arrive(tempty_bar(acc));
           uint32_t packed[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -214,6 +216,8 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
             packed[i] = *reinterpret_cast<const uint32_t*>(&h);
           }
+          // (the second product of the previous tile, which reads the G buffer, ran during the arithmetic above)
+          if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }
           // tokens 32 c .. 32 c + 31 of row `row`: 16-byte chunks 4 c .. 4 c + 3, stored where the 128-byte
           // swizzle of a K-major tile expects them
           uint8_t* rowp = gbuf + row * 128;
@@ -233,7 +237,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         tc_fence_before();
         fence_async_smem();                    // the tensor core reads G through the async proxy
         __syncwarp();
-        if (lane == 0) { mbar_arrive(tempty_bar(acc)); mbar_arrive(gfull_bar(g)); }
+        if (lane == 0) mbar_arrive(gfull_bar(g));
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         if (++g == G_BUFS) { g = 0; g_phase ^= 1u; }
       }
