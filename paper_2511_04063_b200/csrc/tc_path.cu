@@ -36,19 +36,21 @@ __global__ void __launch_bounds__(256) transpose_f32_to_bf16_kernel(const float*
 }
 
 // out tile = sum over slices of part[slice] tile, for the tiles of `list` (mb | nb << 16; tiles
-// are bm x bn); gridDim.y CTAs per tile (a band of rows each), fixed summation order.
-// out_t (nullable): also the bf16 transpose, out_t[c][r] = bf16(out[r][c]).
+// are bm x bn, bn <= 256); gridDim.y CTAs per tile (a band of at most 32 rows each), fixed summation order.
+// out_t (nullable): also the bf16 transpose, out_t[c][r] = bf16(out[r][c]); the band goes through shared
+// memory so that a warp stores consecutive rows of one column (contiguous in out_t).
 __global__ void __launch_bounds__(256) tile_reduce_kernel(const float* __restrict__ part, int slices,
                                                           int64_t slice_stride, const int* __restrict__ list, int bm,
                                                           int bn, int d, float* __restrict__ out,
                                                           __nv_bfloat16* __restrict__ out_t) {
+  __shared__ __nv_bfloat16 band_t[32][256 + 2];   // [row of the band][column], padded against bank conflicts
   const int code = list[blockIdx.x];
   const int band = bm / gridDim.y;
   const int r0 = (code & 0xffff) * bm + blockIdx.y * band, c0 = (code >> 16) * bn;
   const int per_row = bn / 4;
   for (int e = threadIdx.x; e < band * per_row; e += 256) {
-    const int r = r0 + e / per_row, c = c0 + (e % per_row) * 4;
-    const int64_t idx = (int64_t)r * d + c;
+    const int rr = e / per_row, cc = (e % per_row) * 4;
+    const int64_t idx = (int64_t)(r0 + rr) * d + c0 + cc;
     float4 s = *reinterpret_cast<const float4*>(part + idx);
     for (int k = 1; k < slices; ++k) {
       const float4 t = *reinterpret_cast<const float4*>(part + (int64_t)k * slice_stride + idx);
@@ -56,12 +58,17 @@ __global__ void __launch_bounds__(256) tile_reduce_kernel(const float* __restric
     }
     *reinterpret_cast<float4*>(out + idx) = s;
     if (out_t) {
-      out_t[(int64_t)c * d + r] = __float2bfloat16_rn(s.x);
-      out_t[(int64_t)(c + 1) * d + r] = __float2bfloat16_rn(s.y);
-      out_t[(int64_t)(c + 2) * d + r] = __float2bfloat16_rn(s.z);
-      out_t[(int64_t)(c + 3) * d + r] = __float2bfloat16_rn(s.w);
+      band_t[rr][cc] = __float2bfloat16_rn(s.x);
+      band_t[rr][cc + 1] = __float2bfloat16_rn(s.y);
+      band_t[rr][cc + 2] = __float2bfloat16_rn(s.z);
+      band_t[rr][cc + 3] = __float2bfloat16_rn(s.w);
     }
   }
+  if (!out_t) return;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int c = warp; c < bn; c += 8)
+    if (lane < band) out_t[(int64_t)(c0 + c) * d + r0 + lane] = band_t[lane][c];
 }
 
 // One thread waits, with the bounded wait every tcgen05 kernel of the library uses, on a barrier that nothing
