@@ -118,8 +118,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* d_
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
-    __nanosleep(32);   // leave the issue slots to the warps that have work
-    if ((++spins & 0xFFu) == 0u && global_timer_ns() - t0 > limit_ns) {
+    // A hand-off between the warps of a CTA completes within a few polls (try_wait itself suspends the thread for a
+    // while); only a longer wait sleeps between polls and leaves the issue slots to the warps that have work.
+    if (++spins > 64u) __nanosleep(32);
+    if ((spins & 0xFFu) == 0u && global_timer_ns() - t0 > limit_ns) {
       set_status(d_status, DQ_ERR_TIMEOUT);
       return false;
     }
