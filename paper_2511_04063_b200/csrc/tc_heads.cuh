@@ -206,29 +206,16 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
           __syncwarp();
           if (lane == 0) mbar_arrive(tempty_bar(acc));
           uint32_t packed[16];
-          if (p.Gt) {   // dL/dO is materialised: exactly Eq. 4's derivative, zero at o = 0
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
-              const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
-              esum += e0 + e1;
-              const float g0 = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
-              const float g1 = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
-              const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
-              packed[i] = *reinterpret_cast<const uint32_t*>(&h);
-            }
-          } else {
-            // dL/dO only feeds Gq_h += X_t^T G_t.  An o that is exactly zero comes from a token whose activations
-            // are all zero (padding), and that token's row of X_t multiplies whatever G holds by zero: the test for
-            // o = 0 (two of nine instructions per element) changes nothing in Gq and is left out.
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
-              const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
-              esum += e0 + e1;
-              const __nv_bfloat162 h = __floats2bfloat162_rn(copysignf(e0, -o0), copysignf(e1, -o1));
-              packed[i] = *reinterpret_cast<const uint32_t*>(&h);
-            }
+          for (int i = 0; i < 16; ++i) {
+            const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
+            const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
+            esum += e0 + e1;
+            // (an exact zero is not rare: at a Hadamard start o is a signed sum of bf16 values times one constant)
+            const float g0 = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
+            const float g1 = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
+            const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
+            packed[i] = *reinterpret_cast<const uint32_t*>(&h);
           }
           // (the second product of the previous tile, which reads the G buffer, ran during the arithmetic above)
           if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }

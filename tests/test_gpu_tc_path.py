@@ -463,3 +463,40 @@ def test_orthogonal_initial_latent_starts_without_householder(d, amp):
     Z = c.latent()[0]
     assert np.abs(c.rotation()[0] - orc.qr_pos_lapack(Z)[0]).max() <= 5e-5
     c.close()
+
+
+def test_fused_128_step_matches_separate_launches_and_keeps_the_used_rotation():
+    """d = 128, plain SGD: the launch that updates the latent also runs the next step's forward pass.  Timed
+    steps keep backward and forward apart, so a timed run is the unfused reference: same losses, latents
+    and rotations bit for bit.  DQ_BUF_R names the rotation the last step used, the rotation call returns the
+    factor of the updated latent, and a latent set by the caller is factored afresh."""
+    w = small("c3_heads", d=128, n_tokens=1024, batch=3)
+    runs = []
+    for timed in (True, False):
+        c = Calib(w)
+        if timed:
+            dq.dq_calib_set_timing(c.h, True)
+        losses = c.step(4)
+        assert c.status() == dq.DQ_OK
+        R_before = c.rotation()                      # rotation of the current latent: the one step 5 will use
+        loss5 = c.step(1)
+        R_used = c.buf(dq.DQ_BUF_R).cpu().numpy().copy()
+        assert np.array_equal(R_used, R_before)
+        Z5 = c.latent()
+        R5 = c.rotation()
+        for b in range(w.batch):
+            Rr, _ = orc.qr_pos_lapack(Z5[b])
+            assert np.abs(R5[b] - Rr).max() <= 5e-5
+        runs.append((losses, loss5, Z5, R5))
+        if not timed:
+            Zp = _near_orthogonal(128, w.batch, 0.05, 5)
+            c.set_latent(Zp)
+            Rp = c.rotation()
+            for b in range(w.batch):
+                Rr, _ = orc.qr_pos_lapack(Zp[b])
+                assert np.abs(Rp[b] - Rr).max() <= 5e-5
+            c.step(2)
+            assert c.status() == dq.DQ_OK
+        c.close()
+    for a, b in zip(runs[0], runs[1]):
+        assert np.array_equal(a, b)
