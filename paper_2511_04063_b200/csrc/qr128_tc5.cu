@@ -1,6 +1,8 @@
 // Batched QR-Orth for 128 x 128 latents on the 5th-generation tensor cores: one CTA per problem, every
 // 128^3 product as tcgen05.mma on bf16 (hi, lo) operand pairs that the CTA itself writes into shared memory
-// in the K-major 128-byte-swizzled layout, accumulator in tensor memory, one thread per accumulator row.
+// row-major in the 128-byte-swizzled layout, accumulator in tensor memory, two threads per accumulator row.  A
+// product that needs a matrix transposed reads the same buffer as an MN-major operand, so every matrix is written
+// once, in 16-byte pieces.
 //
 //   backward  S = tril(R^T Gq - Gq^T R, -1) (one reduction over two operand pairs, split operands: the skew
 //             part is a small difference), D^T = W S^T, Gz = R D (plain bf16 operands), Z <- Z - lr Gz
@@ -106,18 +108,6 @@ __device__ __forceinline__ void put_rowmajor(uint8_t* buf, int r, int c, const u
         make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
   }
 }
-// Operand with rows = this matrix's columns (K = its rows): entry (r, CH c + i) goes to row CH c + i, k = r.
-__device__ __forceinline__ void put_transposed(uint8_t* buf, int r, int c, const uint32_t* packed) {
-  uint8_t* base = buf + (r >> 6) * KBLK_BYTES + (r & 7) * 2;
-  const int j = (r & 63) >> 3;
-#pragma unroll
-  for (int i = 0; i < CH; ++i) {
-    const int col = CH * c + i;
-    const unsigned short v = (unsigned short)((i & 1) ? (packed[i >> 1] >> 16) : (packed[i >> 1] & 0xffffu));
-    *reinterpret_cast<unsigned short*>(base + col * 128 + ((j ^ (col & 7)) << 4)) = v;
-  }
-}
-
 struct Tc5 {
   uint8_t* smem;        // operand buffers (generic pointer)
   uint32_t smem_u;      // the same, shared-window address
@@ -128,23 +118,29 @@ struct Tc5 {
   int c_begin;          // first of this thread's CHUNKS_PER_THREAD chunks of its row
   int* d_status;
   __device__ __forceinline__ uint8_t* buf(int i) const { return smem + i * PART_BYTES; }
-  // acc (+)= A B^T over the whole K = 128 (issuing thread only)
-  __device__ __forceinline__ void mma(int a, int b, bool accumulate, bool negate_a = false) const {
-    const uint32_t idesc = make_idesc_bf16(N5) | (negate_a ? IDESC_NEGATE_A : 0u);
+  // acc (+)= op(A) op(B)^T over the whole K = 128 (issuing thread only).  Every buffer holds a matrix row-major
+  // (row r = 128 bytes of each of its two 64-column blocks, swizzled).  Read K-major it is the operand with rows =
+  // the matrix's rows; read MN-major (at / bt: the reduction runs over the matrix's ROWS, 16 of them = 2048 bytes
+  // per instruction, the second 64 columns one block further on) it is the operand of the TRANSPOSED matrix, so no
+  // transposed copy of anything is ever written.
+  __device__ __forceinline__ void mma(int a, int b, bool accumulate, bool negate_a = false, bool at = false,
+                                      bool bt = false) const {
+    const uint32_t idesc = make_idesc_bf16(N5) | (negate_a ? IDESC_NEGATE_A : 0u) | (at ? IDESC_A_MN_MAJOR : 0u) |
+                           (bt ? IDESC_B_MN_MAJOR : 0u);
     const uint32_t sa = smem_u + a * PART_BYTES, sb = smem_u + b * PART_BYTES;
 #pragma unroll
-    for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-      for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-        umma_bf16(tmem, make_kmajor_sw128_desc(sa + kb * KBLK_BYTES + k * UMMA_K * 2),
-                  make_kmajor_sw128_desc(sb + kb * KBLK_BYTES + k * UMMA_K * 2), idesc,
-                  (accumulate || kb > 0 || k > 0) ? 1u : 0u);
+    for (int s = 0; s < N5 / UMMA_K; ++s) {
+      const uint32_t kmaj = (uint32_t)((s >> 2) * KBLK_BYTES + (s & 3) * UMMA_K * 2), mnmaj = (uint32_t)(s * UMMA_K * 128);
+      umma_bf16(tmem, at ? make_mnmajor_sw128_desc(sa + mnmaj, KBLK_BYTES) : make_kmajor_sw128_desc(sa + kmaj),
+                bt ? make_mnmajor_sw128_desc(sb + mnmaj, KBLK_BYTES) : make_kmajor_sw128_desc(sb + kmaj), idesc,
+                (accumulate || s > 0) ? 1u : 0u);
+    }
   }
   // split-operand product: A = (a_hi, a_lo), B = (b_hi, b_lo): hi hi + hi lo + lo hi
-  __device__ __forceinline__ void mma3(int a_hi, int a_lo, int b_hi, int b_lo) const {
-    mma(a_hi, b_hi, false);
-    mma(a_hi, b_lo, true);
-    mma(a_lo, b_hi, true);
+  __device__ __forceinline__ void mma3(int a_hi, int a_lo, int b_hi, int b_lo, bool at = false, bool bt = false) const {
+    mma(a_hi, b_hi, false, false, at, bt);
+    mma(a_hi, b_lo, true, false, at, bt);
+    mma(a_lo, b_hi, true, false, at, bt);
   }
 };
 
@@ -192,20 +188,16 @@ __device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, 
   return true;
 }
 
-// This thread's row of an fp32 matrix in global memory -> operand buffers (row-major and / or transposed forms;
-// a negative buffer index skips that form).
-__device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* row, int r, int rm_hi, int rm_lo,
-                                                     int tr_hi, int tr_lo) {
+// This thread's row of an fp32 matrix in global memory -> operand buffers (hi and, unless negative, lo part).
+__device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* row, int r, int rm_hi, int rm_lo) {
 #pragma unroll 1
   for (int c = k.c_begin; c < k.c_begin + CHUNKS_PER_THREAD; ++c) {
     float f[CH];
     fetch_ch(row + c * CH, f);
     uint32_t ph[CH / 2], pl[CH / 2];
     split_ch(f, ph, pl);
-    if (rm_hi >= 0) put_rowmajor(k.buf(rm_hi), r, c, ph);
+    put_rowmajor(k.buf(rm_hi), r, c, ph);
     if (rm_lo >= 0) put_rowmajor(k.buf(rm_lo), r, c, pl);
-    if (tr_hi >= 0) put_transposed(k.buf(tr_hi), r, c, ph);
-    if (tr_lo >= 0) put_transposed(k.buf(tr_lo), r, c, pl);
   }
 }
 
@@ -251,16 +243,17 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
   using F = const float (&)[CH];
 
   if (p.do_backward) {
-    // operands: R row-major -> 0, R^T -> 1 (hi), 4 (lo), Gq^T -> 2 (hi), 5 (lo), W row-major -> 3
-    load_row_to_operands(k, Rrow, r, 0, -1, 1, 4);
-    load_row_to_operands(k, p.Gq + off + r * N5, r, -1, -1, 2, 5);
-    load_row_to_operands(k, Wrow, r, 3, -1, -1, -1);
+    // operands: R -> 0 (hi), 1 (lo), Gq -> 2 (hi), 5 (lo), W -> 3
+    load_row_to_operands(k, Rrow, r, 0, 1);
+    load_row_to_operands(k, p.Gq + off + r * N5, r, 2, 5);
+    load_row_to_operands(k, Wrow, r, 3, -1);
     // S = tril(R^T Gq - Gq^T R, -1), row-major -> 4.  The skew part is what is left of B = R^T Gq after a
     // cancellation (B is close to symmetric near a stationary point), so this one product of the backward runs
     // on split operands: three MMA groups per term, the second term with A negated.
     ok = product(k, [&]() {
-                   k.mma3(1, 4, 2, 5);
-                   k.mma(2, 1, true, true); k.mma(2, 4, true, true); k.mma(5, 1, true, true);
+                   k.mma3(0, 1, 2, 5, true, true);                                  // R^T Gq
+                   k.mma(2, 0, true, true, true, true); k.mma(2, 1, true, true, true, true);   // - Gq^T R
+                   k.mma(5, 0, true, true, true, true);
                  }, nullptr, 0, 0,
                  [&](int c, V v, F, F, F) {
                    float f[CH];
@@ -303,10 +296,10 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
   }
 
   if (p.do_forward && ok) {
-    if (!p.do_backward) load_row_to_operands(k, Zrow, r, 1, 2, -1, -1);     // Z row-major -> 1 (hi), 2 (lo)
-    load_row_to_operands(k, Wrow, r, -1, -1, 3, 4);                         // W^T -> 3, 4
-    // Zh = Z W (split operands): fp32 kept in tensor memory, Zh^T -> 0, 5, Zh row-major -> 1, 2
-    ok = product(k, [&]() { k.mma3(1, 2, 3, 4); }, nullptr, 0, 0,
+    if (!p.do_backward) load_row_to_operands(k, Zrow, r, 1, 2);             // Z -> 1 (hi), 2 (lo)
+    load_row_to_operands(k, Wrow, r, 3, 4);                                 // W -> 3, 4
+    // Zh = Z W (split operands): fp32 kept in tensor memory, Zh -> 1, 2
+    ok = product(k, [&]() { k.mma3(1, 2, 3, 4, false, true); }, nullptr, 0, 0,
                  [&](int c, V v, F, F, F) {
                    float f[CH];
 #pragma unroll
@@ -314,15 +307,13 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                    tmem_st16(k.tmem_row + REG_ZH + (uint32_t)(c * CH), f);
                    uint32_t ph[CH / 2], pl[CH / 2];
                    split_ch(f, ph, pl);
-                   put_transposed(k.buf(0), r, c, ph);
-                   put_transposed(k.buf(5), r, c, pl);
                    put_rowmajor(k.buf(1), r, c, ph);
                    put_rowmajor(k.buf(2), r, c, pl);
                  });
     // E = Zh^T Zh - I (split operands) and the start of the fixed point T = Phi(E - P_old):
-    // T^T -> 3, 4; T row-major -> 0, 5; E and T (fp32) stay in tensor memory
+    // T -> 0, 5; E and T (fp32) stay in tensor memory
     if (ok)
-      ok = product(k, [&]() { k.mma3(0, 5, 0, 5); }, Prow, 0, 0,
+      ok = product(k, [&]() { k.mma3(1, 2, 1, 2, true, true); }, Prow, 0, 0,
                    [&](int c, V v, F pold, F, F) {
                      float e[CH], t[CH];
 #pragma unroll
@@ -335,8 +326,6 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                      tmem_st16(k.tmem_row + REG_T + (uint32_t)(c * CH), t);
                      uint32_t ph[CH / 2], pl[CH / 2];
                      split_ch(t, ph, pl);
-                     put_transposed(k.buf(3), r, c, ph);
-                     put_transposed(k.buf(4), r, c, pl);
                      put_rowmajor(k.buf(0), r, c, ph);
                      put_rowmajor(k.buf(5), r, c, pl);
                    });
@@ -347,7 +336,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
       ++sweeps;
       const bool accurate = sweeps > 2;
       bool moved = false;
-      ok = product(k, [&]() { if (accurate) k.mma3(3, 4, 3, 4); else k.mma(3, 3, false); }, nullptr, REG_E, REG_T,
+      ok = product(k, [&]() { if (accurate) k.mma3(0, 5, 0, 5, true, true); else k.mma(0, 0, false, false, true, true); },
+                   nullptr, REG_E, REG_T,
                    [&](int c, V v, F, F e, F told) {
                      float pp[CH], t[CH];
 #pragma unroll
@@ -360,8 +350,6 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                      tmem_st16(k.tmem_row + REG_T + (uint32_t)(c * CH), t);
                      uint32_t ph[CH / 2], pl[CH / 2];
                      split_ch(t, ph, pl);
-                     put_transposed(k.buf(3), r, c, ph);
-                     put_transposed(k.buf(4), r, c, pl);
                      put_rowmajor(k.buf(0), r, c, ph);
                      put_rowmajor(k.buf(5), r, c, pl);
                    });
@@ -369,7 +357,7 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
     }
     if (ok && !converged) { set_status(p.d_status, DQ_ERR_NOT_CONVERGED); }
     const bool big = sweeps > 2;        // a large step: the first-order products on split operands as well
-    // Y = (I + T)^-1 - I by Y <- -T - T Y from Y = -T;  Y^T -> 3, 4 (T^T is no longer needed); Y (fp32) takes the
+    // Y = (I + T)^-1 - I by Y <- -T - T Y from Y = -T;  Y -> 3, 4 (W is no longer needed there); Y (fp32) takes the
     // place of E in tensor memory.  The terms shrink geometrically (ratio at most |T|), so the series stops as
     // soon as the NEXT term, estimated from the last two, would change no entry by more than 2e-7: after a small
     // step a single product.
@@ -399,8 +387,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
         tmem_st16(k.tmem_row + REG_E + (uint32_t)(c * CH), t);
         uint32_t ph[CH / 2], pl[CH / 2];
         split_ch(t, ph, pl);
-        put_transposed(k.buf(3), r, c, ph);
-        put_transposed(k.buf(4), r, c, pl);
+        put_rowmajor(k.buf(3), r, c, ph);
+        put_rowmajor(k.buf(4), r, c, pl);
       }
       prev = block_max(tmax);
     }
@@ -409,7 +397,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
     while (ok && terms < MAX_SERIES && !converged) {
       ++terms;
       float chg = 0.f;
-      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4); else k.mma(0, 3, false); }, nullptr, REG_T, REG_E,
+      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4, false, true); else k.mma(0, 3, false, false, false, true); },
+                   nullptr, REG_T, REG_E,
                    [&](int c, V v, F, F t, F yold) {
                      float y[CH];
 #pragma unroll
@@ -421,8 +410,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                      tmem_st16(k.tmem_row + REG_E + (uint32_t)(c * CH), y);
                      uint32_t ph[CH / 2], pl[CH / 2];
                      split_ch(y, ph, pl);
-                     put_transposed(k.buf(3), r, c, ph);
-                     put_transposed(k.buf(4), r, c, pl);
+                     put_rowmajor(k.buf(3), r, c, ph);
+                     put_rowmajor(k.buf(4), r, c, pl);
                    });
       const float m = block_max(chg);
       // next term ~ m * (m / prev), with the ratio capped below 1 so that a stalled series is not mistaken for done
@@ -433,7 +422,8 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
     if (ok && !converged) { set_status(p.d_status, DQ_ERR_NOT_CONVERGED); }
     // R = Zh + Zh Y
     if (ok)
-      ok = product(k, [&]() { if (big) k.mma3(1, 2, 3, 4); else k.mma(1, 3, false); }, nullptr, REG_ZH, 0,
+      ok = product(k, [&]() { if (big) k.mma3(1, 2, 3, 4, false, true); else k.mma(1, 3, false, false, false, true); },
+                   nullptr, REG_ZH, 0,
                    [&](int c, V v, F, F zh, F) {
                      float f[CH];
 #pragma unroll
@@ -448,8 +438,9 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
     // W <- W + W Y  (W row-major -> 0, 5: T is no longer needed)
     float dv = NAN;                     // the diagonal entry, in the thread whose chunks hold it
     if (ok) {
-      load_row_to_operands(k, Wrow, r, 0, 5, -1, -1);
-      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4); else k.mma(0, 3, false); }, Wrow, 0, 0,
+      load_row_to_operands(k, Wrow, r, 0, 5);
+      ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4, false, true); else k.mma(0, 3, false, false, false, true); },
+                   Wrow, 0, 0,
                    [&](int c, V v, F w, F, F) {
                      float f[CH];
 #pragma unroll

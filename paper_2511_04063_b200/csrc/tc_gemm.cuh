@@ -201,6 +201,7 @@ __device__ __forceinline__ uint64_t make_mnmajor_sw128_desc(uint32_t smem_addr, 
   return d;
 }
 constexpr uint32_t IDESC_A_MN_MAJOR = 1u << 15;   // kind::f16 instruction descriptor: A is MN-major
+constexpr uint32_t IDESC_B_MN_MAJOR = 1u << 16;   // B is MN-major
 // kind::f16 instruction descriptor: bf16 x bf16 -> fp32, both K-major, M = 128.
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
