@@ -28,8 +28,8 @@ constexpr int PART_BYTES = N5 * N5 * 2;          // one bf16 operand part: two [
 constexpr int KBLK_BYTES = N5 * BLOCK_K * 2;     // 16 KB
 constexpr int N_BUFS = 6;
 constexpr int TC5_SMEM = N_BUFS * PART_BYTES + 1024 + 1024;
-constexpr int TC5_THREADS = 256;                // two threads per accumulator row, half of the columns each
-constexpr int CHUNKS_PER_THREAD = 4;
+constexpr int TC5_THREADS = 512;                // four threads per accumulator row, a quarter of the columns each
+constexpr int CHUNKS_PER_THREAD = 2;
 constexpr uint32_t TC5_TMEM_COLS = 512;          // the accumulator and three fp32 matrices that stay on chip
 constexpr uint32_t REG_E = 128, REG_T = 256, REG_ZH = 384;   // tensor-memory columns of E (later Y), T and Zh
 constexpr int MAX_SERIES = 48;
@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
   const uint32_t bar = smem_base + N_BUFS * PART_BYTES;
   const uint32_t tmem_slot = bar + 16u;
   uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_ptr + N_BUFS * PART_BYTES + 16);
-  float* red = reinterpret_cast<float*>(smem_ptr + N_BUFS * PART_BYTES + 64);   // [16] block reductions
+  float* red = reinterpret_cast<float*>(smem_ptr + N_BUFS * PART_BYTES + 64);   // [2 x warps] block reductions
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = 32 * (warp & 3) + lane;           // accumulator row (tensor-memory lane) of this thread
@@ -459,13 +459,14 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
         mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       }
-      if (lane == 0) { red[warp] = mn; red[8 + warp] = mx; }
+      constexpr int NW = TC5_THREADS / 32;
+      if (lane == 0) { red[warp] = mn; red[NW + warp] = mx; }
       if (owner && !(isfinite(dv) && dv > 0.f))
         set_status(p.d_status, isfinite(dv) ? DQ_ERR_SINGULAR : DQ_ERR_NONFINITE);
       __syncthreads();
       if (threadIdx.x == 0) {
         float a = INFINITY, b = 0.f;
-        for (int i = 0; i < 8; ++i) { a = fminf(a, red[i]); b = fmaxf(b, red[8 + i]); }
+        for (int i = 0; i < NW; ++i) { a = fminf(a, red[i]); b = fmaxf(b, red[NW + i]); }
         if (!(a > 1e-6f * b)) set_status(p.d_status, DQ_ERR_SINGULAR);
       }
     }
