@@ -273,7 +273,9 @@ int wy_ksplit(int m, int batch, int sm_count) {
 // The two sets of copies of W = U^-1 (row-major and transposed, split): index 0 / 1.
 struct WSet { bf16 *n_hi, *n_lo, *t_hi, *t_lo; };
 WSet wset(const QrTcState& q, int sel) {
-  return sel == 0 ? WSet{q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo} : WSet{q.wn2_hi, q.wn2_lo, q.wt2_hi, q.wt2_lo};
+  // (the transposed copies exist for set 0 only: the Householder route writes and reads them there; the
+  // incremental steps read W^T as a transposed operand)
+  return sel == 0 ? WSet{q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo} : WSet{q.wn2_hi, q.wn2_lo, nullptr, nullptr};
 }
 
 // The upper tiles in the order made for the product's k_mode (0: all k-blocks, 2, or 1|4).
@@ -314,7 +316,7 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   const int64_t dd = (int64_t)d * d * batch;
   bf16** all[] = {&q.z_hi, &q.z_lo, &q.u_hi, &q.u_lo, &q.wn_hi, &q.wn_lo, &q.wt_hi, &q.wt_lo, &q.r_hi, &q.r_lo,
                   &q.rt_hi, &q.rt_lo, &q.gqt_hi, &q.gqt_lo, &q.st_hi, &q.st_lo, &q.m_hi, &q.m_lo, &q.t1_hi, &q.t1_lo,
-                  &q.wn2_hi, &q.wn2_lo, &q.wt2_hi, &q.wt2_lo, &q.yt_hi, &q.yt_lo, &q.nm1, &q.nm2};
+                  &q.wn2_hi, &q.wn2_lo, &q.yt_hi, &q.yt_lo, &q.nm1, &q.nm2};
   for (bf16** p : all) DQ_CHECK(alloc(p, dd));
   DQ_CHECK(alloc(&q.P, dd));
   const int64_t yb = (int64_t)d * 128 * batch;
@@ -329,7 +331,6 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
   if (q.part_bs > 0) DQ_CHECK(alloc(&q.part, q.part_bs * batch));
   DQ_CHECK(alloc(&q.tw_hi, dd)); DQ_CHECK(alloc(&q.tw_lo, dd));
   DQ_CHECK(alloc(&q.sweep_flags, 80));
-  DQ_CHECK(alloc(&q.uot_hi, dd)); DQ_CHECK(alloc(&q.uot_lo, dd));
   for (int unit = 128; unit <= 256; unit *= 2) {   // tile orders (see QrTcState)
     if (d % unit != 0) break;
     const int nb = d / unit;
@@ -369,11 +370,11 @@ dq_status qr_tc_init(QrTcState& q, int d, int batch, int sm_count) {
 void qr_tc_destroy(QrTcState& q) {
   bf16* all[] = {q.z_hi, q.z_lo, q.u_hi, q.u_lo, q.wn_hi, q.wn_lo, q.wt_hi, q.wt_lo, q.r_hi, q.r_lo,
                  q.rt_hi, q.rt_lo, q.gqt_hi, q.gqt_lo, q.st_hi, q.st_lo, q.m_hi, q.m_lo, q.t1_hi, q.t1_lo,
-                 q.wn2_hi, q.wn2_lo, q.wt2_hi, q.wt2_lo, q.yt_hi, q.yt_lo, q.nm1, q.nm2};
+                 q.wn2_hi, q.wn2_lo, q.yt_hi, q.yt_lo, q.nm1, q.nm2};
   for (bf16* p : all) cudaFree(p);
   cudaFree(q.P);
   cudaFree(q.y_hi); cudaFree(q.y_lo); cudaFree(q.w2_hi); cudaFree(q.w2_lo); cudaFree(q.part); cudaFree(q.T);
-  cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.uot_hi); cudaFree(q.uot_lo); cudaFree(q.tl_upper); cudaFree(q.tl_k4); cudaFree(q.tl_k8); cudaFree(q.tl_upper_k2); cudaFree(q.tl_upper_band);
+  cudaFree(q.tw_hi); cudaFree(q.tw_lo); cudaFree(q.tl_upper); cudaFree(q.tl_k4); cudaFree(q.tl_k8); cudaFree(q.tl_upper_k2); cudaFree(q.tl_upper_band);
   cudaFree(q.tl2_upper); cudaFree(q.tl2_k4); cudaFree(q.tl2_k8); cudaFree(q.tl2_upper_k2); cudaFree(q.tl2_upper_band); cudaFree(q.tl_lower); cudaFree(q.tl2_lower); cudaFree(q.sweep_flags);
   q = QrTcState();
 }
@@ -428,22 +429,23 @@ dq_status qr_forward_incremental_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, con
   const dim3 tiles(d / 32, d / 32, batch);
   const WSet wc = wset(q, q.w_sel), wn = wset(q, q.w_sel ^ 1);
   float *Zh = ws.A, *E = ws.B, *T = ws.tmp, *T2 = ws.S, *Y3 = ws.Q, *T4 = ws.V, *Wf = ws.Winv;
-  // bf16 scratch (all free until the backward pass or owned by the Householder route)
-  bf16 *zh_hi = q.m_hi, *zh_lo = q.m_lo, *zht_hi = q.st_hi, *zht_lo = q.st_lo;
-  bf16 *twa_hi = q.tw_hi, *twa_lo = q.tw_lo, *twb_hi = q.t1_hi, *twb_lo = q.t1_lo;   // T^T, alternating between sweeps
-  bf16 *twf_hi = q.uot_hi, *twf_lo = q.uot_lo;                                       // T^T of the last sweep that ran
-  bf16 *t_hi = q.u_hi, *t_lo = q.u_lo;                                               // T row-major
-  bf16 *t2_hi = q.gqt_hi, *t2t_hi = q.gqt_lo, *y3_hi = q.nm1, *t4t_hi = q.nm2;
+  // bf16 scratch (all free until the backward pass or owned by the Householder route).  Every matrix is kept
+  // row-major only: a product that needs it transposed names it as a transposed operand (Op::t) and the tensor
+  // cores read its tiles MN-major.
+  bf16 *zh_hi = q.m_hi, *zh_lo = q.m_lo;
+  bf16 *ta_hi = q.tw_hi, *ta_lo = q.tw_lo, *tb_hi = q.t1_hi, *tb_lo = q.t1_lo;   // T, alternating between sweeps
+  bf16 *t_hi = q.u_hi, *t_lo = q.u_lo;                                           // T of the last sweep that ran
+  bf16 *t2_hi = q.gqt_hi, *y3_hi = q.nm1, *t4_hi = q.nm2;
+  bf16 *y_hi = q.yt_hi, *y_lo = q.yt_lo;                                         // Y = (I + T)^-1 - I
   q.u_fresh = false;
   if (!q.z_split_fresh) {   // (the SGD update writes the split copy with the new latent)
     split_kernel<<<tiles, 256, 0, ctx.stream>>>(Z, q.z_hi, q.z_lo, d, 0);
     DQ_CHECK(after_launch(ctx));
     q.z_split_fresh = true;
   }
-  {   // Zh[i][j] = sum_k Z[i][k] W_old[k][j]  (W upper triangular: k <= j)
-    Op a{q.z_hi, q.z_lo, d, dd}, b{wc.t_hi, wc.t_lo, d, dd};
+  {   // Zh[i][j] = sum_k Z[i][k] W_old[k][j]  (W upper triangular: k <= j); B = W^T
+    Op a{q.z_hi, q.z_lo, d, dd}, b{wc.n_hi, wc.n_lo, d, dd, true};
     Out o; o.f32 = Zh; o.ld = d; o.bs = dd; o.hi = zh_hi; o.lo = zh_lo; o.ld_h = d; o.bs_h = dd;
-    o.t_hi = zht_hi; o.t_lo = zht_lo; o.ld_t = d; o.bs_t = dd;
     o.k_mode = 4; o.tile_list = q.tl_k4; o.n_list = q.n_all; o.tile_list2 = q.tl2_k4; o.n_list2 = q.n2_all;
     DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   }
@@ -451,75 +453,73 @@ dq_status qr_forward_incremental_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, con
   int* flags = q.sweep_flags;      // flags[k] = 1: sweep k moved an entry
   DQ_CHECK_CUDA(cudaMemsetAsync(flags, 0, sizeof(int) * (n_total + 2), ctx.stream));
   {   // E = Zh^T Zh - I on the upper tiles, and the start of the fixed point T = Phi(E - P_old)
-    Op a{zht_hi, zht_lo, d, dd};
-    // (the first sweep always follows and reads only the hi part of T^T)
+    Op a{zh_hi, zh_lo, d, dd, true};   // both operands are Zh^T
+    // (the first sweep always follows and reads only the hi part of T)
     Out o; o.f32 = E; o.ld = d; o.bs = dd; o.add1 = q.P; o.aux = T; o.gen_mode = tc::GEN_CHOL_FIRST;
-    o.t_hi = twa_hi; o.ld_t = d; o.bs_t = dd;
+    o.hi = ta_hi; o.ld_h = d; o.bs_h = dd;
     upper_lists(o, q);
     DQ_CHECK(gemm3(ctx, a, a, d, d, d, batch, o));
   }
   for (int k = 1; k <= n_total; ++k) {
-    // P[i][j] = sum_l T[l][i] T[l][j] (T^T is lower triangular: l < 128 (mb + 1), mb <= nb), then
-    // T <- Phi(E - P) in the epilogue.  The operand T^T alternates between two buffers, because the epilogue
-    // of one tile rewrites what the main loop of another still reads.
+    // P[i][j] = sum_l T[l][i] T[l][j] (both operands T^T, lower triangular: l < 128 (mb + 1), mb <= nb), then
+    // T <- Phi(E - P) in the epilogue.  The bf16 copy of T that the sweeps read alternates between two buffers,
+    // because the epilogue of one tile rewrites what the main loop of another still reads.
     const bool odd = k & 1;
-    Op tt{odd ? twa_hi : twb_hi, odd ? twa_lo : twb_lo, d, dd};
+    Op tt{odd ? ta_hi : tb_hi, odd ? ta_lo : tb_lo, d, dd, true};
     Out o; o.f32 = q.P; o.ld = d; o.bs = dd; o.add1 = E; o.aux = T; o.gen_mode = tc::GEN_CHOL_SWEEP;
     o.tol = 1e-5f; o.moved_out = flags + k; o.fail_if_moved = (k == n_total) ? 1 : 0;
-    o.hi = t_hi; o.lo = t_lo; o.ld_h = d; o.bs_h = dd;
-    // T^T for the next sweep (its lo part only if that sweep uses split operands), and the copies the later
-    // products read, which every sweep that runs must leave behind (which one is the last is not known here)
-    o.t_hi = odd ? twb_hi : twa_hi; o.t_lo = (k + 1 > 2) ? (odd ? twb_lo : twa_lo) : nullptr;
-    o.t2_hi = twf_hi; o.t2_lo = twf_lo;
-    o.ld_t = d; o.bs_t = dd;
+    // T for the next sweep (its lo part only if that sweep uses split operands), and the copy the later products
+    // read, which every sweep that runs must leave behind (which one is the last is not known here)
+    o.hi = odd ? tb_hi : ta_hi; o.lo = (k + 1 > 2) ? (odd ? tb_lo : ta_lo) : nullptr;
+    o.hi2 = t_hi; o.lo2 = t_lo; o.ld_h = d; o.bs_h = dd;
     o.k_mode = 2; upper_lists(o, q);
     o.nterms = (k <= 2) ? 1 : 3;
     o.run_if = (k == 1) ? nullptr : flags + k - 1;
     DQ_CHECK(gemm3(ctx, tt, tt, d, d, d, batch, o));
   }
   const int* big = flags + 2;     // a third sweep ran: a large step, first-order products with split operands
-  Op t{t_hi, t_lo, d, dd}, ttf{twf_hi, twf_lo, d, dd};
+  Op t{t_hi, t_lo, d, dd}, t_tr{t_hi, t_lo, d, dd, true};
   for (int v = 0; v < 2; ++v) {   // T2 = T T  (upper x upper: k in [128 mb, 128 (nb + 1)))
-    Out o; o.f32 = T2; o.ld = d; o.bs = dd; o.hi = t2_hi; o.ld_h = d; o.bs_h = dd; o.t_hi = t2t_hi; o.ld_t = d; o.bs_t = dd;
+    Out o; o.f32 = T2; o.ld = d; o.bs = dd; o.hi = t2_hi; o.ld_h = d; o.bs_h = dd;
     o.k_mode = 1 | 4; upper_lists(o, q);
     o.nterms = v ? 3 : 1; (v ? o.run_if : o.run_unless) = big;
-    DQ_CHECK(gemm3(ctx, t, ttf, d, d, d, batch, o));
+    DQ_CHECK(gemm3(ctx, t, t_tr, d, d, d, batch, o));
   }
-  {   // Y3 = -T + T2 - T T2 = (I - T)(I + T2) - I: all of Y after a small step (error |T|^4)
-    Op b{t2t_hi, t2t_hi, d, dd};
+  Op t2{t2_hi, t2_hi, d, dd}, t2_tr{t2_hi, t2_hi, d, dd, true};
+  {   // Y3 = -T + T2 - T T2 = (I - T)(I + T2) - I: all of Y after a small step (error |T|^4).  Its split copy is
+      // the Y the last two products read; a second hi copy is the operand of the large-step correction below,
+      // which rewrites Y.
     Out o; o.f32 = Y3; o.ld = d; o.bs = dd; o.alpha = -1.f; o.add1 = T2; o.g1 = 1.f; o.add2 = T; o.g2 = -1.f;
-    o.hi = y3_hi; o.ld_h = d; o.bs_h = dd; o.t_hi = q.yt_hi; o.t_lo = q.yt_lo; o.ld_t = d; o.bs_t = dd;
+    o.hi = y_hi; o.lo = y_lo; o.hi2 = y3_hi; o.ld_h = d; o.bs_h = dd;
     o.k_mode = 1 | 4; upper_lists(o, q); o.nterms = 1;
-    DQ_CHECK(gemm3(ctx, t, b, d, d, d, batch, o));
+    DQ_CHECK(gemm3(ctx, t, t2_tr, d, d, d, batch, o));
   }
   {   // after a large step also the factor (I + T^4):  T4 = T2 T2
-    Op a{t2_hi, t2_hi, d, dd}, b{t2t_hi, t2t_hi, d, dd};
-    Out o; o.f32 = T4; o.ld = d; o.bs = dd; o.t_hi = t4t_hi; o.ld_t = d; o.bs_t = dd; o.k_mode = 1 | 4; upper_lists(o, q);
+    Out o; o.f32 = T4; o.ld = d; o.bs = dd; o.hi = t4_hi; o.ld_h = d; o.bs_h = dd; o.k_mode = 1 | 4; upper_lists(o, q);
     o.nterms = 1; o.run_if = big;
-    DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
+    DQ_CHECK(gemm3(ctx, t2, t2_tr, d, d, d, batch, o));
   }
-  {   // Y = Y3 + T4 + Y3 T4 = (I + Y3)(I + T4) - I; only its transposed split copy is kept
-    Op a{y3_hi, y3_hi, d, dd}, b{t4t_hi, t4t_hi, d, dd};
-    Out o; o.ld = d; o.bs = dd; o.add1 = Y3; o.add2 = T4; o.t_hi = q.yt_hi; o.t_lo = q.yt_lo; o.ld_t = d; o.bs_t = dd;
+  {   // Y = Y3 + T4 + Y3 T4 = (I + Y3)(I + T4) - I; only its split copy is kept
+    Op a{y3_hi, y3_hi, d, dd}, b{t4_hi, t4_hi, d, dd, true};
+    Out o; o.ld = d; o.bs = dd; o.add1 = Y3; o.add2 = T4; o.hi = y_hi; o.lo = y_lo; o.ld_h = d; o.bs_h = dd;
     o.k_mode = 1 | 4; upper_lists(o, q); o.nterms = 1; o.run_if = big;
     DQ_CHECK(gemm3(ctx, a, b, d, d, d, batch, o));
   }
-  Op yt{q.yt_hi, q.yt_lo, d, dd};
+  Op y_tr{y_hi, y_lo, d, dd, true};
   for (int v = 0; v < 2; ++v) {   // R = Zh + Zh Y  (Y upper triangular: k <= j)
     Op a{zh_hi, zh_lo, d, dd};
     Out o; o.f32 = R; o.ld = d; o.bs = dd; o.add1 = Zh; o.hi = q.r_hi; o.lo = need_lo ? q.r_lo : nullptr; o.ld_h = d; o.bs_h = dd;
-    o.t_hi = q.rt_hi; o.t_lo = need_lo ? q.rt_lo : nullptr; o.ld_t = d; o.bs_t = dd;
+    o.t_hi = q.rt_hi; o.t_lo = need_lo ? q.rt_lo : nullptr; o.ld_t = d; o.bs_t = dd;   // R^T: operand of O = X R
     o.k_mode = 4; o.tile_list = q.tl_k4; o.n_list = q.n_all; o.tile_list2 = q.tl2_k4; o.n_list2 = q.n2_all;
     o.nterms = v ? 3 : 1; (v ? o.run_if : o.run_unless) = big;
-    DQ_CHECK(gemm3(ctx, a, yt, d, d, d, batch, o));
+    DQ_CHECK(gemm3(ctx, a, y_tr, d, d, d, batch, o));
   }
   for (int v = 0; v < 2; ++v) {   // W = W_old + W_old Y into the other set of copies (the fp32 W in place)
     Op a{wc.n_hi, wc.n_lo, d, dd};
     Out o; o.f32 = Wf; o.ld = d; o.bs = dd; o.add1 = Wf; o.hi = wn.n_hi; o.lo = wn.n_lo; o.ld_h = d; o.bs_h = dd;
-    o.t_hi = wn.t_hi; o.t_lo = wn.t_lo; o.ld_t = d; o.bs_t = dd;
     o.k_mode = 1 | 4; upper_lists(o, q);
     o.nterms = v ? 3 : 1; (v ? o.run_if : o.run_unless) = big;
-    DQ_CHECK(gemm3(ctx, a, yt, d, d, d, batch, o));
+    DQ_CHECK(gemm3(ctx, a, y_tr, d, d, d, batch, o));
   }
   q.w_sel ^= 1;
   // diag(W) = 1 / diag(U): the same rank and finiteness test
@@ -607,7 +607,7 @@ dq_status qr_tc_try_orthogonal_start(Ctx& ctx, QrWorkspace& ws, QrTcState& q, co
 dq_status qr_tc_bench_product(Ctx& ctx, QrWorkspace& ws, QrTcState& q, int d, int batch, int nterms) {
   const int64_t dd = (int64_t)d * d;
   const WSet w = wset(q, q.w_sel);
-  Op a{q.z_hi, q.z_lo, d, dd}, b{w.t_hi, w.t_lo, d, dd};
+  Op a{q.z_hi, q.z_lo, d, dd}, b{w.n_hi, w.n_lo, d, dd, true};
   Out o; o.f32 = ws.Q; o.ld = d; o.bs = dd; o.nterms = nterms;
   return gemm3(ctx, a, b, d, d, d, batch, o);
 }

@@ -42,6 +42,8 @@ struct Params {
   // (element (m, n) at out_t + b * batch_stride_t + n * ld_t + m; up to two targets)
   __nv_bfloat16* out_hi;
   __nv_bfloat16* out_lo;
+  __nv_bfloat16* out2_hi;   // a second row-major copy (same addressing as out_hi / out_lo; nullable)
+  __nv_bfloat16* out2_lo;
   int64_t ld_h, batch_stride_h;
   float alpha;
   const float* add1; float g1;
@@ -83,6 +85,10 @@ struct Params {
   // variants of a product).  nullptr: no condition.
   const int* run_if;
   const int* run_unless;
+  // a_mn / b_mn: the operand is given TRANSPOSED, i.e. as a row-major matrix whose rows are the reduction index
+  // ([K][M] or [K][N]); its tensor maps have boxes of 64 rows (k) x 64 columns and the MMAs read the tile MN-major,
+  // so a product needs no transposed copy of a matrix that exists row-major.  Applies to all maps of the operand.
+  int a_mn, b_mn;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -135,6 +141,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_dst), "l"((uint64_t)map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
+}
+// One operand tile of a stage (ROWS rows of the operand x 64 k): one box K-major, ROWS / 64 boxes MN-major
+// (box = 64 k x 64 columns of the transposed matrix, coordinates (column, k)).
+template <int ROWS>
+__device__ __forceinline__ void load_operand(uint32_t smem_dst, const CUtensorMap* map, uint32_t bar, int kc, int row0,
+                                             int b, int mn) {
+  if (!mn) { tma_load_3d(smem_dst, map, bar, kc, row0, b); return; }
+#pragma unroll
+  for (int i = 0; i < ROWS / 64; ++i) tma_load_3d(smem_dst + i * (BLOCK_K * 128), map, bar, row0 + 64 * i, kc, b);
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)map) : "memory");
@@ -208,6 +223,14 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int n) {
 }
 
 constexpr uint32_t IDESC_NEGATE_A = 1u << 13;   // kind::f16 instruction descriptor: A is negated
+
+constexpr uint32_t MN_BOX_BYTES = BLOCK_K * 128;   // one MN-major box: 64 k x 64 columns of bf16 = 8 KB
+// Descriptor of UMMA k-step `k` (16 of the stage's 64 k) of an operand tile at `base`: K-major (rows of 128 bytes =
+// 64 k of one row) or MN-major (rows of 128 bytes = 64 columns of one k; the next 64 columns one box further on).
+__device__ __forceinline__ uint64_t operand_desc(uint32_t base, int k, int mn) {
+  return mn ? make_mnmajor_sw128_desc(base + (uint32_t)(k * UMMA_K * 128), MN_BOX_BYTES)
+            : make_kmajor_sw128_desc(base + (uint32_t)(k * UMMA_K * 2));
+}
 
 // ----------------------------------------------------------------------------- EPI_GEN epilogue
 // The thread that owns output row `row` handles GEN_CH consecutive columns at a time.  The fp32 addends of a
@@ -315,7 +338,7 @@ __device__ __forceinline__ void epi_gen_chunk(const Params& p, const uint32_t (&
       for (int i = 0; i < GEN_CH / 8; ++i) st_global_f32x8(outp + off + 8 * i, f + 8 * i);
     }
   }
-  if (p.out_hi || p.out_t_hi || p.out_t2_hi) {
+  if (p.out_hi || p.out2_hi || p.out_t_hi || p.out_t2_hi) {
     uint32_t ph[GEN_CH / 2], pl[GEN_CH / 2];
 #pragma unroll
     for (int i = 0; i < GEN_CH / 2; ++i) {
@@ -325,10 +348,12 @@ __device__ __forceinline__ void epi_gen_chunk(const Params& p, const uint32_t (&
       ph[i] = *reinterpret_cast<const uint32_t*>(&h);
       pl[i] = *reinterpret_cast<const uint32_t*>(&l);
     }
-    if (p.out_hi) {
+    if (p.out_hi || p.out2_hi) {
       const int64_t off_h = (int64_t)b * p.batch_stride_h + (int64_t)row * p.ld_h + col0;
-      st_global_b32x8(p.out_hi + off_h, ph);
+      if (p.out_hi) st_global_b32x8(p.out_hi + off_h, ph);
       if (p.out_lo) st_global_b32x8(p.out_lo + off_h, pl);
+      if (p.out2_hi) st_global_b32x8(p.out2_hi + off_h, ph);
+      if (p.out2_lo) st_global_b32x8(p.out2_lo + off_h, pl);
     }
     if (p.out_t_hi || p.out_t2_hi) {
       // transposed copies: for a fixed column the 32 lanes of the warp (consecutive rows) store 64 contiguous bytes
@@ -476,11 +501,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           const uint32_t sb = sa + L::NOPS * L::A_BYTES;
           const bool second = kb >= kb_per_split;          // second operand pair of a dual reduction
           const int kc = (k0 + (second ? kb - kb_per_split : kb)) * BLOCK_K;
-          tma_load_3d(sa, second ? &mapA_lo : &mapA, full_bar(stage), kc, mb * BLOCK_M, b);
-          tma_load_3d(sb, second ? &mapB_lo : &mapB, full_bar(stage), kc, nb * BLOCK_N, b);
+          load_operand<BLOCK_M>(sa, second ? &mapA_lo : &mapA, full_bar(stage), kc, mb * BLOCK_M, b, p.a_mn);
+          load_operand<BLOCK_N>(sb, second ? &mapB_lo : &mapB, full_bar(stage), kc, nb * BLOCK_N, b, p.b_mn);
           if (NTERMS > 1) {
-            tma_load_3d(sa + L::A_BYTES, &mapA_lo, full_bar(stage), kc, mb * BLOCK_M, b);
-            tma_load_3d(sb + L::B_BYTES, &mapB_lo, full_bar(stage), kc, nb * BLOCK_N, b);
+            load_operand<BLOCK_M>(sa + L::A_BYTES, &mapA_lo, full_bar(stage), kc, mb * BLOCK_M, b, p.a_mn);
+            load_operand<BLOCK_N>(sb + L::B_BYTES, &mapB_lo, full_bar(stage), kc, nb * BLOCK_N, b, p.b_mn);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -511,17 +536,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           tc_fence_after();
           const uint32_t sa = smem_base + stage * L::STAGE_BYTES;
           const uint32_t sb = sa + L::NOPS * L::A_BYTES;
-          const uint32_t idesc = (kb >= kb_per_split) ? (IDESC | IDESC_NEGATE_A) : IDESC;
+          const uint32_t idesc_mn = IDESC | (p.a_mn ? IDESC_A_MN_MAJOR : 0u) | (p.b_mn ? IDESC_B_MN_MAJOR : 0u);
+          const uint32_t idesc = (kb >= kb_per_split) ? (idesc_mn | IDESC_NEGATE_A) : idesc_mn;
 #pragma unroll
           for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-            const uint64_t a_hi = make_kmajor_sw128_desc(sa + k * UMMA_K * 2);
-            const uint64_t b_hi = make_kmajor_sw128_desc(sb + k * UMMA_K * 2);
+            const uint64_t a_hi = operand_desc(sa, k, p.a_mn);
+            const uint64_t b_hi = operand_desc(sb, k, p.b_mn);
             umma_bf16(tmem_d, a_hi, b_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             if (NTERMS > 1) {
-              const uint64_t a_lo = make_kmajor_sw128_desc(sa + L::A_BYTES + k * UMMA_K * 2);
-              const uint64_t b_lo = make_kmajor_sw128_desc(sb + L::B_BYTES + k * UMMA_K * 2);
-              umma_bf16(tmem_d, a_hi, b_lo, IDESC, 1u);
-              umma_bf16(tmem_d, a_lo, b_hi, IDESC, 1u);
+              const uint64_t a_lo = operand_desc(sa + L::A_BYTES, k, p.a_mn);
+              const uint64_t b_lo = operand_desc(sb + L::B_BYTES, k, p.b_mn);
+              umma_bf16(tmem_d, a_hi, b_lo, idesc_mn, 1u);
+              umma_bf16(tmem_d, a_lo, b_hi, idesc_mn, 1u);
             }
           }
           umma_commit(empty_bar(stage));       // smem slot reusable once these MMAs retire

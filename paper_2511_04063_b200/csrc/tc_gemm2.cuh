@@ -61,6 +61,13 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const CUtens
       ::"r"(smem_dst), "l"((uint64_t)map), "r"(bar & PEER_MASK), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// This CTA's half of an operand tile of a stage (128 rows of the operand x 64 k): one box K-major, two boxes MN-major.
+__device__ __forceinline__ void load_operand_pair(uint32_t smem_dst, const CUtensorMap* map, uint32_t bar, int kc,
+                                                  int row0, int b, int mn) {
+  if (!mn) { tma_load_3d_pair(smem_dst, map, bar, kc, row0, b); return; }
+  tma_load_3d_pair(smem_dst, map, bar, row0, kc, b);
+  tma_load_3d_pair(smem_dst + MN_BOX_BYTES, map, bar, row0 + 64, kc, b);
+}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -181,11 +188,12 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
           const uint32_t sb = sa + L::NOPS * A_BYTES;
           const bool second = kb >= kn;                     // second operand pair of a dual reduction
           const int kc = (k0 + (second ? kb - kn : kb)) * BLOCK_K;
-          tma_load_3d_pair(sa, second ? &mapA_lo : &mapA, full_bar(stage), kc, mb * PAIR_M + (int)rank * HALF, b);
-          tma_load_3d_pair(sb, second ? &mapB_lo : &mapB, full_bar(stage), kc, nb * PAIR_N + (int)rank * HALF, b);
+          const int ra = mb * PAIR_M + (int)rank * HALF, rb = nb * PAIR_N + (int)rank * HALF;
+          load_operand_pair(sa, second ? &mapA_lo : &mapA, full_bar(stage), kc, ra, b, p.a_mn);
+          load_operand_pair(sb, second ? &mapB_lo : &mapB, full_bar(stage), kc, rb, b, p.b_mn);
           if (NTERMS > 1) {
-            tma_load_3d_pair(sa + A_BYTES, &mapA_lo, full_bar(stage), kc, mb * PAIR_M + (int)rank * HALF, b);
-            tma_load_3d_pair(sb + B_BYTES, &mapB_lo, full_bar(stage), kc, nb * PAIR_N + (int)rank * HALF, b);
+            load_operand_pair(sa + A_BYTES, &mapA_lo, full_bar(stage), kc, ra, b, p.a_mn);
+            load_operand_pair(sb + B_BYTES, &mapB_lo, full_bar(stage), kc, rb, b, p.b_mn);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -214,17 +222,18 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + L::NOPS * A_BYTES;
-          const uint32_t idesc = (kb >= kn) ? (IDESC | IDESC_NEGATE_A) : IDESC;
+          const uint32_t idesc_mn = IDESC | (p.a_mn ? IDESC_A_MN_MAJOR : 0u) | (p.b_mn ? IDESC_B_MN_MAJOR : 0u);
+          const uint32_t idesc = (kb >= kn) ? (idesc_mn | IDESC_NEGATE_A) : idesc_mn;
 #pragma unroll
           for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-            const uint64_t a_hi = make_kmajor_sw128_desc(sa + k * UMMA_K * 2);
-            const uint64_t b_hi = make_kmajor_sw128_desc(sb + k * UMMA_K * 2);
+            const uint64_t a_hi = operand_desc(sa, k, p.a_mn);
+            const uint64_t b_hi = operand_desc(sb, k, p.b_mn);
             umma_bf16_pair(tmem_d, a_hi, b_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             if (NTERMS > 1) {
-              const uint64_t a_lo = make_kmajor_sw128_desc(sa + A_BYTES + k * UMMA_K * 2);
-              const uint64_t b_lo = make_kmajor_sw128_desc(sb + B_BYTES + k * UMMA_K * 2);
-              umma_bf16_pair(tmem_d, a_hi, b_lo, IDESC, 1u);
-              umma_bf16_pair(tmem_d, a_lo, b_hi, IDESC, 1u);
+              const uint64_t a_lo = operand_desc(sa + A_BYTES, k, p.a_mn);
+              const uint64_t b_lo = operand_desc(sb + B_BYTES, k, p.b_mn);
+              umma_bf16_pair(tmem_d, a_hi, b_lo, idesc_mn, 1u);
+              umma_bf16_pair(tmem_d, a_lo, b_hi, idesc_mn, 1u);
             }
           }
           umma_commit_pair(empty_bar(stage));      // both CTAs may refill this slot once the MMAs retire

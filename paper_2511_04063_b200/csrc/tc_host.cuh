@@ -124,12 +124,16 @@ inline dq_status rotate_tokens(Ctx& ctx, const void* X, int64_t n, int d, int64_
   return (bn == 256) ? launch_gemm<256, 1, EPI>(ctx, ma, mb, ma, mb, p) : launch_gemm<128, 1, EPI>(ctx, ma, mb, ma, mb, p);
 }
 
-struct Op {   // K-major operand: rows x K, split pair, leading dimension, batch stride (elements)
-  const bf16* hi; const bf16* lo; int64_t ld; int64_t bs;
+// Operand of a product: a row-major matrix as a split pair, leading dimension, batch stride (elements).
+// t == false: rows x K (each row of the matrix is a row of the operand).  t == true: K x rows, the operand is the
+// TRANSPOSE of the stored matrix; the MMAs read its tiles MN-major, no transposed copy is needed.
+struct Op {
+  const bf16* hi; const bf16* lo; int64_t ld; int64_t bs; bool t = false;
 };
 struct Out {
   float* f32 = nullptr; int64_t ld = 0; int64_t bs = 0;
   bf16* hi = nullptr; bf16* lo = nullptr; int64_t ld_h = 0; int64_t bs_h = 0;
+  bf16* hi2 = nullptr; bf16* lo2 = nullptr;   // a second row-major split copy (same ld_h / bs_h)
   float alpha = 1.f, beta = 0.f;             // beta: the old contents of f32 are added (shorthand for add1 = f32)
   // v = alpha * acc + g1 * add1 + g2 * add2: fp32 matrices addressed like f32 (same ld / bs)
   const float* add1 = nullptr; float g1 = 1.f;
@@ -154,7 +158,7 @@ struct Out {
 
 inline void fill_epilogue(tc::Params& p, const Out& o) {
   p.out = o.f32; p.ld = o.ld; p.batch_stride = o.bs; p.split_stride = o.split_stride;
-  p.out_hi = o.hi; p.out_lo = o.lo; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
+  p.out_hi = o.hi; p.out_lo = o.lo; p.out2_hi = o.hi2; p.out2_lo = o.lo2; p.ld_h = o.ld_h; p.batch_stride_h = o.bs_h;
   p.alpha = o.alpha;
   p.add1 = o.add1; p.g1 = o.g1; p.add2 = o.add2; p.g2 = o.g2;
   if (o.beta != 0.f) {   // the output accumulates: its old contents are the (first free) addend
@@ -199,7 +203,8 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
       return ptr && ((((uintptr_t)ptr) & 31) || (ld * esz) % 32 || (bs * esz) % 32);
     };
     if (bad(o.f32, o.ld, o.bs, 4) || bad(o.add1, o.ld, o.bs, 4) || bad(o.add2, o.ld, o.bs, 4) || bad(o.aux, o.ld, o.bs, 4) ||
-        bad(o.hi, o.ld_h, o.bs_h, 2) || bad(o.lo, o.ld_h, o.bs_h, 2) || (o.split_stride * 4) % 32)
+        bad(o.hi, o.ld_h, o.bs_h, 2) || bad(o.lo, o.ld_h, o.bs_h, 2) || bad(o.hi2, o.ld_h, o.bs_h, 2) ||
+        bad(o.lo2, o.ld_h, o.bs_h, 2) || (o.split_stride * 4) % 32)
       return DQ_ERR_UNSUPPORTED;
   }
   if (o.ksplit > 1 && (o.add1 || o.add2 || o.beta != 0.f || o.hi || o.t_hi || o.gen_mode != tc::GEN_LINEAR))
@@ -209,22 +214,35 @@ inline dq_status gemm3(Ctx& ctx, const Op& A, const Op& B, int M, int N, int K, 
   const bf16* b2 = dual ? o.dual_b->hi : (o.nterms == 1 ? B.hi : B.lo);
   const int64_t lda2 = dual ? o.dual_a->ld : A.ld, ldb2 = dual ? o.dual_b->ld : B.ld;
   CUtensorMap ma, mal, mb, mbl;
-  const int64_t bsa = A.bs ? A.bs : (int64_t)M * A.ld, bsb = B.bs ? B.bs : (int64_t)N * B.ld;
-  const int64_t bsa2 = dual ? (o.dual_a->bs ? o.dual_a->bs : (int64_t)M * lda2) : bsa;
-  const int64_t bsb2 = dual ? (o.dual_b->bs ? o.dual_b->bs : (int64_t)N * ldb2) : bsb;
+  if (dual && (o.dual_a->t != A.t || o.dual_b->t != B.t)) return DQ_ERR_UNSUPPORTED;   // one orientation per operand
+  const int64_t bsa = A.bs ? A.bs : (int64_t)(A.t ? K : M) * A.ld, bsb = B.bs ? B.bs : (int64_t)(B.t ? K : N) * B.ld;
+  const int64_t bsa2 = dual ? (o.dual_a->bs ? o.dual_a->bs : (int64_t)(A.t ? K : M) * lda2) : bsa;
+  const int64_t bsb2 = dual ? (o.dual_b->bs ? o.dual_b->bs : (int64_t)(B.t ? K : N) * ldb2) : bsb;
   // Large products run on CTA pairs (256 x 256 tiles, half the operand traffic per MMA); a caller that
   // orders its tiles must also give the order in pair tiles.
   const bool pair_ok = M % 256 == 0 && N % 256 == 0 && (!o.tile_list || o.tile_list2) && ctx.sm_count >= 2 &&
                        (int64_t)(M / 256) * (N / 256) * batch * o.ksplit >= 32;
   const int unit = pair_ok ? 256 : 128;
   const int box = pair_ok ? tc2::HALF : 128;
-  DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, pair_ok ? tc2::HALF : tc::BLOCK_M));
-  DQ_CHECK(make_map(&mal, a2, K, M, batch, lda2, bsa2, pair_ok ? tc2::HALF : tc::BLOCK_M));
-  DQ_CHECK(make_map(&mb, B.hi, K, N, batch, B.ld, bsb, box));
-  DQ_CHECK(make_map(&mbl, b2, K, N, batch, ldb2, bsb2, box));
+  // (a transposed operand: the stored matrix has K rows; boxes of 64 k x 64 columns)
+  if (A.t) {
+    DQ_CHECK(make_map(&ma, A.hi, M, K, batch, A.ld, bsa, tc::BLOCK_K));
+    DQ_CHECK(make_map(&mal, a2, M, K, batch, lda2, bsa2, tc::BLOCK_K));
+  } else {
+    DQ_CHECK(make_map(&ma, A.hi, K, M, batch, A.ld, bsa, pair_ok ? tc2::HALF : tc::BLOCK_M));
+    DQ_CHECK(make_map(&mal, a2, K, M, batch, lda2, bsa2, pair_ok ? tc2::HALF : tc::BLOCK_M));
+  }
+  if (B.t) {
+    DQ_CHECK(make_map(&mb, B.hi, N, K, batch, B.ld, bsb, tc::BLOCK_K));
+    DQ_CHECK(make_map(&mbl, b2, N, K, batch, ldb2, bsb2, tc::BLOCK_K));
+  } else {
+    DQ_CHECK(make_map(&mb, B.hi, K, N, batch, B.ld, bsb, box));
+    DQ_CHECK(make_map(&mbl, b2, K, N, batch, ldb2, bsb2, box));
+  }
   tc::Params p{};
   p.m_blocks = M / unit; p.n_blocks = N / unit; p.batch = batch; p.ksplit = o.ksplit; p.k_blocks = K / tc::BLOCK_K;
   fill_epilogue(p, o);
+  p.a_mn = A.t ? 1 : 0; p.b_mn = B.t ? 1 : 0;
   p.d_status = ctx.d_status;
   p.tile_list = pair_ok ? o.tile_list2 : o.tile_list;
   p.n_list = pair_ok ? o.n_list2 : o.n_list;

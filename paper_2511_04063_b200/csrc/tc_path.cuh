@@ -67,10 +67,10 @@ struct QrTcState {
   __nv_bfloat16 *m_hi = nullptr, *m_lo = nullptr;       // R S
   __nv_bfloat16 *t1_hi = nullptr, *t1_lo = nullptr;     // scratch of the block inversion
   // second set of copies of W: the incremental update W <- W (I + T)^-1 reads one set and writes the other
-  __nv_bfloat16 *wn2_hi = nullptr, *wn2_lo = nullptr, *wt2_hi = nullptr, *wt2_lo = nullptr;
+  __nv_bfloat16 *wn2_hi = nullptr, *wn2_lo = nullptr;
   int w_sel = 0;                                        // the set that holds the current W (0: wn / wt, 1: wn2 / wt2)
   float* P = nullptr;                                   // T^T T of the last sweep: where the next step's fixed point starts
-  __nv_bfloat16 *yt_hi = nullptr, *yt_lo = nullptr;     // ((I + T)^-1 - I)^T
+  __nv_bfloat16 *yt_hi = nullptr, *yt_lo = nullptr;     // Y = (I + T)^-1 - I (row-major split copy)
   __nv_bfloat16 *nm1 = nullptr, *nm2 = nullptr;         // scratch of the products that form (I + T)^-1
   bool u_fresh = false;                                 // U and u_hi / u_lo hold the upper factor of the current factorisation
   bool gqt_fresh = false;                               // gqt_hi holds bf16(Gq^T) of the current step (written by the contraction)
@@ -81,8 +81,7 @@ struct QrTcState {
   int64_t part_bs = 0;                                  // elements per problem
   float* T = nullptr;                                   // [batch][4][32][32] compact-WY factors of the inner panels
   // near-orthogonal iterative factorisation
-  __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T^T of the sweeps
-  __nv_bfloat16 *uot_hi = nullptr, *uot_lo = nullptr;   // T^T of the last sweep that ran
+  __nv_bfloat16 *tw_hi = nullptr, *tw_lo = nullptr;     // T of the sweeps (alternates with t1_hi / t1_lo)
   bool z_split_fresh = false;                           // z_hi / z_lo are the split copy of the current latent
   bool t_warm = false;                                  // the current set of W copies and the fp32 W belong to the previous step's latent
   int* sweep_flags = nullptr;                           // [80] device flags: sweep k moved an entry
