@@ -137,8 +137,9 @@ dq_status dq_gather_tokens(const void* d_X, int32_t x_dtype, int64_t n_total, in
 
 /* Mini-batch use (the paper feeds the loop with batches of sampled tokens): the
  * caller overwrote the borrowed activation buffer d_X in place (same shape) on
- * the handle's stream; rebuild every operand copy derived from it.  Cheap no-op on
- * the fp32 path. */
+ * the handle's stream.  Every kernel reads the activations in place (no copy of them is
+ * derived or kept), so today this call only orders the handle's internal stream after the
+ * caller's writes; call it all the same after rewriting d_X. */
 dq_status dq_calib_refresh_inputs(dq_calib_t* h);
 
 /* Optimiser of the latent (Sec. 4.3: QR-Orth works with any standard optimiser; the paper reports

@@ -8,20 +8,6 @@
 namespace dq {
 namespace {
 
-// out[b][c][r] = in[b][r][c]   (bf16; rows, cols multiples of 64)
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in,
-                                                             __nv_bfloat16* __restrict__ out, int64_t rows,
-                                                             int64_t cols, int64_t ld_in) {
-  __shared__ __nv_bfloat16 t[64][66];
-  in += (int64_t)blockIdx.z * rows * ld_in;
-  out += (int64_t)blockIdx.z * rows * cols;
-  const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
-  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-  for (int r = ty; r < 64; r += 4) t[r][tx] = in[(r0 + r) * ld_in + c0 + tx];
-  __syncthreads();
-  for (int c = ty; c < 64; c += 4) out[(c0 + c) * rows + r0 + tx] = t[tx][c];
-}
-
 // out[b][c][r] = bf16(in[b][r][c])  (fp32 in, d x d)
 __global__ void __launch_bounds__(256) transpose_f32_to_bf16_kernel(const float* __restrict__ in,
                                                                     __nv_bfloat16* __restrict__ out, int d) {
@@ -85,7 +71,7 @@ __global__ void bounded_wait_probe_kernel(uint64_t limit_ns, int* d_status, uint
 }
 
 struct Maps {
-  CUtensorMap rt, x, x128, x64, xt, gt128, gt256;
+  CUtensorMap rt, x, x128, x64, xmn, gt128, gt256;
 };
 
 }  // namespace
@@ -97,7 +83,6 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   tc.d = d; tc.batch = batch; tc.n_tokens = N;
   tc.X = reinterpret_cast<const __nv_bfloat16*>(d_X);
   tc.Gt = Gt;
-  if (cudaMalloc((void**)&tc.Xt, sizeof(__nv_bfloat16) * (size_t)batch * N * d) != cudaSuccess) return DQ_ERR_ALLOC;
   if (rt_external) {
     tc.Rt = rt_external; tc.rt_external = true;
   } else if (cudaMalloc((void**)&tc.Rt, sizeof(__nv_bfloat16) * (size_t)batch * d * d) != cudaSuccess) {
@@ -142,10 +127,10 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   DQ_CHECK(tch::make_map(&m->x, tc.X, d, N, batch, ldx, N * ldx, 256));
   DQ_CHECK(tch::make_map(&m->x128, tc.X, d, N, batch, ldx, N * ldx, 128));
   DQ_CHECK(tch::make_map(&m->x64, tc.X, d, N, batch, ldx, N * ldx, heads::TT));
-  DQ_CHECK(tch::make_map(&m->xt, tc.Xt, N, d, batch, N, N * d, tc::BLOCK_M));
+  // X again, in boxes of 64 tokens x 64 channels: the MN-major A operand (X^T) of Gq = X^T G
+  DQ_CHECK(tch::make_map(&m->xmn, tc.X, d, N, batch, ldx, N * ldx, tc::BLOCK_K));
   DQ_CHECK(tch::make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
   DQ_CHECK(tch::make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
-  DQ_CHECK(tc_refresh_inputs(tc, ctx));
   if (d == 128) {   // per-head rotations: fused kernel, units = (head, range of token tiles), two CTAs per SM
     const int tiles_per_head = (int)(N / heads::TT);
     int sp = 2 * ctx.sm_count / batch;
@@ -166,15 +151,12 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   return DQ_OK;
 }
 
-// X^T copy (channel-major) for the K-major A operand of Gq = X^T G.
-dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx) {
-  transpose_bf16_kernel<<<dim3(tc.d / 64, (unsigned)(tc.n_tokens / 64), tc.batch), 256, 0, ctx.stream>>>(
-      tc.X, tc.Xt, tc.n_tokens, tc.d, tc.ldx);
-  return after_launch(ctx);
-}
+// The activations are read in place by every kernel (the contraction over tokens takes X^T as an MN-major
+// operand straight from the token-major rows), so a caller that rewrites X has nothing to rebuild.
+dq_status tc_refresh_inputs(TcState&, Ctx&) { return DQ_OK; }
 
 void tc_destroy(TcState& tc) {
-  cudaFree(tc.Xt); if (!tc.rt_external) cudaFree(tc.Rt); cudaFree(tc.part);
+  if (!tc.rt_external) cudaFree(tc.Rt); cudaFree(tc.part);
   cudaFree(tc.tl_head); cudaFree(tc.tl_tail); cudaFree(tc.tail_part); cudaFree(tc.heads_part);
   delete reinterpret_cast<Maps*>(tc.maps);
   tc = TcState();
@@ -213,7 +195,7 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
   return tch::launch_gemm<256, 1, tc::EPI_WHIP>(ctx, m->rt, m->x, m->rt, m->x, p);
 }
 
-// Gq = scale * X^T G : A = X^T [d][N], B = G^T [d][N], reduction over tokens.
+// Gq = scale * X^T G : A = X^T taken MN-major from X [N][d], B = G^T [d][N], reduction over tokens.
 // gqt (nullable): the epilogue also stores bf16(Gq^T) there (the operand of the QR-Orth backward);
 // *gqt_written tells whether this schedule could (the split-K schedule of small shapes cannot).
 dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale, __nv_bfloat16* gqt, bool* gqt_written) {
@@ -229,6 +211,7 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale, __nv_b
   p.k_blocks = (int)(tc.n_tokens / tc::BLOCK_K);
   p.ld = d; p.alpha = scale; p.out_hi = nullptr; p.out_lo = nullptr;
   p.partials = nullptr; p.d_status = ctx.d_status;
+  p.a_mn = 1;
   if (tc.ksplit == 1) {
     p.out = Gq; p.batch_stride = (int64_t)d * d; p.split_stride = 0;
   } else {
@@ -236,9 +219,9 @@ dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale, __nv_b
   }
   if (tc.pair) p.m_blocks = d / 256;
   auto launch = [&](const tc::Params& pp) {
-    if (tc.pair) return tch::launch_gemm2<1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, pp);
-    return (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, m->xt, m->gt256, m->xt, m->gt256, pp)
-                       : tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, m->xt, m->gt128, m->xt, m->gt128, pp);
+    if (tc.pair) return tch::launch_gemm2<1, tc::EPI_GEN>(ctx, m->xmn, m->gt128, m->xmn, m->gt128, pp);
+    return (bn == 256) ? tch::launch_gemm<256, 1, tc::EPI_GEN>(ctx, m->xmn, m->gt256, m->xmn, m->gt256, pp)
+                       : tch::launch_gemm<128, 1, tc::EPI_GEN>(ctx, m->xmn, m->gt128, m->xmn, m->gt128, pp);
   };
   const bool with_t = gqt != nullptr && tc.ksplit == 1 && tc.batch == 1;
   if (with_t) {

@@ -9,7 +9,6 @@ struct TcState {
   int d = 0, batch = 0;
   int64_t n_tokens = 0, ldx = 0;
   const __nv_bfloat16* X = nullptr;   // [batch][N][ldx] token-major (borrowed)
-  __nv_bfloat16* Xt = nullptr;        // [batch][d][N] channel-major copy (owned)
   __nv_bfloat16* Rt = nullptr;        // [batch][d][d] bf16(R^T) (owned unless rt_external)
   bool rt_external = false;
   __nv_bfloat16* Gt = nullptr;        // [batch][d][N] dL/dO, channel-major (borrowed from handle)
@@ -36,7 +35,7 @@ struct TcState {
 dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void* d_X,
                   __nv_bfloat16* Gt, __nv_bfloat16* rt_external, int* n_partials);
 void tc_destroy(TcState& tc);
-dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx);   // X changed in place: rebuild X^T
+dq_status tc_refresh_inputs(TcState& tc, Ctx& ctx);   // X changed in place: nothing derived from it is kept
 inline __nv_bfloat16* tc_rt_operand(TcState& tc) { return tc.ready ? tc.Rt : nullptr; }
 dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials);
 dq_status tc_grad_rotation(TcState& tc, Ctx& ctx, float* Gq, float scale, __nv_bfloat16* gqt = nullptr,
