@@ -227,9 +227,13 @@ constexpr uint32_t IDESC_NEGATE_A = 1u << 13;   // kind::f16 instruction descrip
 constexpr uint32_t MN_BOX_BYTES = BLOCK_K * 128;   // one MN-major box: 64 k x 64 columns of bf16 = 8 KB
 // Descriptor of UMMA k-step `k` (16 of the stage's 64 k) of an operand tile at `base`: K-major (rows of 128 bytes =
 // 64 k of one row) or MN-major (rows of 128 bytes = 64 columns of one k; the next 64 columns one box further on).
-__device__ __forceinline__ uint64_t operand_desc(uint32_t base, int k, int mn) {
-  return mn ? make_mnmajor_sw128_desc(base + (uint32_t)(k * UMMA_K * 128), MN_BOX_BYTES)
-            : make_kmajor_sw128_desc(base + (uint32_t)(k * UMMA_K * 2));
+// The descriptor of k-step k is that of k-step 0 plus k times a constant in its address field (units of 16 bytes):
+// the issuing thread forms one descriptor per operand and stage and adds, whatever the orientation.
+__device__ __forceinline__ uint64_t operand_desc0(uint32_t base, int mn) {
+  return mn ? make_mnmajor_sw128_desc(base, MN_BOX_BYTES) : make_kmajor_sw128_desc(base);
+}
+__device__ __forceinline__ uint32_t operand_desc_step(int mn) {
+  return mn ? (uint32_t)(UMMA_K * 128) >> 4 : (uint32_t)(UMMA_K * 2) >> 4;
 }
 
 // ----------------------------------------------------------------------------- EPI_GEN epilogue
@@ -514,6 +518,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer
     if (lane == 0) {
+      const int a_mn = p.a_mn, b_mn = p.b_mn;
+      const uint32_t a_step = operand_desc_step(a_mn), b_step = operand_desc_step(b_mn);
+      const uint32_t idesc_mn = IDESC | (a_mn ? IDESC_A_MN_MAJOR : 0u) | (b_mn ? IDESC_B_MN_MAJOR : 0u);
+      const uint64_t a_stage0 = operand_desc0(smem_base, a_mn);                     // descriptors of stage 0
+      const uint64_t b_stage0 = operand_desc0(smem_base + L::NOPS * L::A_BYTES, b_mn);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -536,16 +545,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           tc_fence_after();
           const uint32_t sa = smem_base + stage * L::STAGE_BYTES;
           const uint32_t sb = sa + L::NOPS * L::A_BYTES;
-          const uint32_t idesc_mn = IDESC | (p.a_mn ? IDESC_A_MN_MAJOR : 0u) | (p.b_mn ? IDESC_B_MN_MAJOR : 0u);
           const uint32_t idesc = (kb >= kb_per_split) ? (idesc_mn | IDESC_NEGATE_A) : idesc_mn;
+          const uint64_t a0 = a_stage0 + (uint64_t)(stage * (L::STAGE_BYTES >> 4));
+          const uint64_t b0 = b_stage0 + (uint64_t)(stage * (L::STAGE_BYTES >> 4));
 #pragma unroll
           for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-            const uint64_t a_hi = operand_desc(sa, k, p.a_mn);
-            const uint64_t b_hi = operand_desc(sb, k, p.b_mn);
+            const uint64_t a_hi = a0 + (uint64_t)(k * a_step);
+            const uint64_t b_hi = b0 + (uint64_t)(k * b_step);
             umma_bf16(tmem_d, a_hi, b_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             if (NTERMS > 1) {
-              const uint64_t a_lo = operand_desc(sa + L::A_BYTES, k, p.a_mn);
-              const uint64_t b_lo = operand_desc(sb + L::B_BYTES, k, p.b_mn);
+              const uint64_t a_lo = a_hi + (uint64_t)(L::A_BYTES >> 4);
+              const uint64_t b_lo = b_hi + (uint64_t)(L::B_BYTES >> 4);
               umma_bf16(tmem_d, a_hi, b_lo, idesc_mn, 1u);
               umma_bf16(tmem_d, a_lo, b_hi, idesc_mn, 1u);
             }

@@ -202,6 +202,11 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer (leader CTA only)
     if (leader && lane == 0) {
+      const int a_mn = p.a_mn, b_mn = p.b_mn;
+      const uint32_t a_step = operand_desc_step(a_mn), b_step = operand_desc_step(b_mn);
+      const uint32_t idesc_mn = IDESC | (a_mn ? IDESC_A_MN_MAJOR : 0u) | (b_mn ? IDESC_B_MN_MAJOR : 0u);
+      const uint64_t a_stage0 = operand_desc0(smem_base, a_mn);                     // descriptors of stage 0
+      const uint64_t b_stage0 = operand_desc0(smem_base + L::NOPS * A_BYTES, b_mn);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -222,16 +227,18 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + L::NOPS * A_BYTES;
-          const uint32_t idesc_mn = IDESC | (p.a_mn ? IDESC_A_MN_MAJOR : 0u) | (p.b_mn ? IDESC_B_MN_MAJOR : 0u);
           const uint32_t idesc = (kb >= kn) ? (idesc_mn | IDESC_NEGATE_A) : idesc_mn;
+          // (nothing on the path from the barrier to the first MMA but one multiply-add per operand)
+          const uint64_t a0 = a_stage0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+          const uint64_t b0 = b_stage0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
 #pragma unroll
           for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-            const uint64_t a_hi = operand_desc(sa, k, p.a_mn);
-            const uint64_t b_hi = operand_desc(sb, k, p.b_mn);
+            const uint64_t a_hi = a0 + (uint64_t)(k * a_step);
+            const uint64_t b_hi = b0 + (uint64_t)(k * b_step);
             umma_bf16_pair(tmem_d, a_hi, b_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             if (NTERMS > 1) {
-              const uint64_t a_lo = operand_desc(sa + A_BYTES, k, p.a_mn);
-              const uint64_t b_lo = operand_desc(sb + B_BYTES, k, p.b_mn);
+              const uint64_t a_lo = a_hi + (uint64_t)(A_BYTES >> 4);
+              const uint64_t b_lo = b_hi + (uint64_t)(B_BYTES >> 4);
               umma_bf16_pair(tmem_d, a_hi, b_lo, idesc_mn, 1u);
               umma_bf16_pair(tmem_d, a_lo, b_hi, idesc_mn, 1u);
             }
