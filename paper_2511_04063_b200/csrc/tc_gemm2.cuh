@@ -31,8 +31,12 @@ constexpr int B_BYTES = HALF * BLOCK_K * 2;
 template <int NTERMS>
 struct PairSmem {
   static constexpr int NOPS = (NTERMS == 1) ? 1 : 2;
-  static constexpr int STAGE_BYTES = NOPS * (A_BYTES + B_BYTES);     // per CTA: 32 KB or 64 KB
-  static constexpr int STAGES = (NTERMS == 1) ? 6 : 3;
+  static constexpr int KBLOCK_BYTES = NOPS * (A_BYTES + B_BYTES);    // one k-block of 64, per CTA: 32 KB or 64 KB
+  // A stage of the plain product holds two k-blocks: half as many barrier round trips between the producer and
+  // the MMA issuer per tile (each costs the issuer some tens of the 256 cycles a k-block's MMAs take).
+  static constexpr int KPS = (NTERMS == 1) ? 2 : 1;
+  static constexpr int STAGE_BYTES = KPS * KBLOCK_BYTES;             // 64 KB
+  static constexpr int STAGES = 3;
   static constexpr int TOTAL = STAGES * STAGE_BYTES + 1024 + 1024;
 };
 // Epilogue warps per CTA: the general epilogue is a chain of dependent steps per 16-column chunk (tensor-memory
@@ -112,6 +116,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
   using L = PairSmem<NTERMS>;
   constexpr int STAGES = L::STAGES;
   constexpr int STAGE_BYTES = L::STAGE_BYTES;
+  constexpr int KPS = L::KPS, KBLOCK_BYTES = L::KBLOCK_BYTES;
   constexpr uint32_t IDESC = make_idesc_bf16_pair();
   constexpr int EPI_WARPS = epi_warps<EPI>();
   constexpr int N_EPI = PAIR_N / (EPI_WARPS / 4);   // columns of the tile one epilogue warp handles
@@ -181,19 +186,25 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         int k0, kn;
         k_range(split, mb, nb, k0, kn);
         const int kb_total = (NTERMS == 1 && p.k_dual) ? 2 * kn : kn;
-        for (int kb = 0; kb < kb_total; ++kb) {
+        const int ra = mb * PAIR_M + (int)rank * HALF, rb = nb * PAIR_N + (int)rank * HALF;
+        for (int kb0 = 0; kb0 < kb_total; kb0 += KPS) {
+          const int nk = (kb_total - kb0 < KPS) ? kb_total - kb0 : KPS;   // k-blocks in this stage
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
-          if (leader) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          const uint32_t sb = sa + L::NOPS * A_BYTES;
-          const bool second = kb >= kn;                     // second operand pair of a dual reduction
-          const int kc = (k0 + (second ? kb - kn : kb)) * BLOCK_K;
-          const int ra = mb * PAIR_M + (int)rank * HALF, rb = nb * PAIR_N + (int)rank * HALF;
-          load_operand_pair(sa, second ? &mapA_lo : &mapA, full_bar(stage), kc, ra, b, p.a_mn);
-          load_operand_pair(sb, second ? &mapB_lo : &mapB, full_bar(stage), kc, rb, b, p.b_mn);
-          if (NTERMS > 1) {
-            load_operand_pair(sa + A_BYTES, &mapA_lo, full_bar(stage), kc, ra, b, p.a_mn);
-            load_operand_pair(sb + B_BYTES, &mapB_lo, full_bar(stage), kc, rb, b, p.b_mn);
+          if (leader) mbar_expect_tx(full_bar(stage), 2 * nk * KBLOCK_BYTES);
+#pragma unroll
+          for (int j = 0; j < KPS; ++j) {
+            if (j >= nk) break;
+            const int kb = kb0 + j;
+            const uint32_t sa = smem_base + stage * STAGE_BYTES + j * KBLOCK_BYTES;
+            const uint32_t sb = sa + L::NOPS * A_BYTES;
+            const bool second = kb >= kn;                   // second operand pair of a dual reduction
+            const int kc = (k0 + (second ? kb - kn : kb)) * BLOCK_K;
+            load_operand_pair(sa, second ? &mapA_lo : &mapA, full_bar(stage), kc, ra, b, p.a_mn);
+            load_operand_pair(sb, second ? &mapB_lo : &mapB, full_bar(stage), kc, rb, b, p.b_mn);
+            if (NTERMS > 1) {
+              load_operand_pair(sa + A_BYTES, &mapA_lo, full_bar(stage), kc, ra, b, p.a_mn);
+              load_operand_pair(sb + B_BYTES, &mapB_lo, full_bar(stage), kc, rb, b, p.b_mn);
+            }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -222,25 +233,30 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * PAIR_N);
         const int kb_total = (NTERMS == 1 && p.k_dual) ? 2 * kn : kn;
-        for (int kb = 0; kb < kb_total; ++kb) {
+        for (int kb0 = 0; kb0 < kb_total; kb0 += KPS) {
+          const int nk = (kb_total - kb0 < KPS) ? kb_total - kb0 : KPS;
+          // (nothing on the path from the barrier to the first MMA but one multiply-add per operand)
+          const uint64_t a_st = a_stage0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+          const uint64_t b_st = b_stage0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
           if (!mbar_wait(full_bar(stage), phase, p.d_status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          const uint32_t sb = sa + L::NOPS * A_BYTES;
-          const uint32_t idesc = (kb >= kn) ? (idesc_mn | IDESC_NEGATE_A) : idesc_mn;
-          // (nothing on the path from the barrier to the first MMA but one multiply-add per operand)
-          const uint64_t a0 = a_stage0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
-          const uint64_t b0 = b_stage0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
 #pragma unroll
-          for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-            const uint64_t a_hi = a0 + (uint64_t)(k * a_step);
-            const uint64_t b_hi = b0 + (uint64_t)(k * b_step);
-            umma_bf16_pair(tmem_d, a_hi, b_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-            if (NTERMS > 1) {
-              const uint64_t a_lo = a_hi + (uint64_t)(A_BYTES >> 4);
-              const uint64_t b_lo = b_hi + (uint64_t)(B_BYTES >> 4);
-              umma_bf16_pair(tmem_d, a_hi, b_lo, idesc_mn, 1u);
-              umma_bf16_pair(tmem_d, a_lo, b_hi, idesc_mn, 1u);
+          for (int j = 0; j < KPS; ++j) {
+            if (j >= nk) break;
+            const int kb = kb0 + j;
+            const uint32_t idesc = (kb >= kn) ? (idesc_mn | IDESC_NEGATE_A) : idesc_mn;
+            const uint64_t a0 = a_st + (uint64_t)(j * (KBLOCK_BYTES >> 4)), b0 = b_st + (uint64_t)(j * (KBLOCK_BYTES >> 4));
+#pragma unroll
+            for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+              const uint64_t a_hi = a0 + (uint64_t)(k * a_step);
+              const uint64_t b_hi = b0 + (uint64_t)(k * b_step);
+              umma_bf16_pair(tmem_d, a_hi, b_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              if (NTERMS > 1) {
+                const uint64_t a_lo = a_hi + (uint64_t)(A_BYTES >> 4);
+                const uint64_t b_lo = b_hi + (uint64_t)(B_BYTES >> 4);
+                umma_bf16_pair(tmem_d, a_hi, b_lo, idesc_mn, 1u);
+                umma_bf16_pair(tmem_d, a_lo, b_hi, idesc_mn, 1u);
+              }
             }
           }
           umma_commit_pair(empty_bar(stage));      // both CTAs may refill this slot once the MMAs retire
