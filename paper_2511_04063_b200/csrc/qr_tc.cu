@@ -508,8 +508,9 @@ dq_status qr_forward_incremental_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, con
   Op y_tr{y_hi, y_lo, d, dd, true};
   for (int v = 0; v < 2; ++v) {   // R = Zh + Zh Y  (Y upper triangular: k <= j)
     Op a{zh_hi, zh_lo, d, dd};
-    Out o; o.f32 = R; o.ld = d; o.bs = dd; o.add1 = Zh; o.hi = q.r_hi; o.lo = need_lo ? q.r_lo : nullptr; o.ld_h = d; o.bs_h = dd;
-    o.t_hi = q.rt_hi; o.t_lo = need_lo ? q.rt_lo : nullptr; o.ld_t = d; o.bs_t = dd;   // R^T: operand of O = X R
+    // the only bf16 copy of R is R^T (operand of O = X R; the backward reads R from it as a transposed operand)
+    Out o; o.f32 = R; o.ld = d; o.bs = dd; o.add1 = Zh;
+    o.t_hi = q.rt_hi; o.t_lo = need_lo ? q.rt_lo : nullptr; o.ld_t = d; o.bs_t = dd;
     o.k_mode = 4; o.tile_list = q.tl_k4; o.n_list = q.n_all; o.tile_list2 = q.tl2_k4; o.n_list2 = q.n2_all;
     o.nterms = v ? 3 : 1; (v ? o.run_if : o.run_unless) = big;
     DQ_CHECK(gemm3(ctx, a, y_tr, d, d, d, batch, o));
@@ -664,7 +665,7 @@ dq_status qr_backward_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* G
   // (tiles below the block diagonal of D^T are neither written here nor read by the next product; the entries
   // below the diagonal inside the diagonal tiles come out as exact zeros)
   // Gz[i][j] = sum_k R[i][k] D^T[j][k]; D^T[j][k] = 0 for k < j
-  Op r{q.r_hi, q.r_lo, d, dd}, dt{q.m_hi, q.m_lo, d, dd};
+  Op r{q.rt_hi, q.rt_lo, d, dd, true}, dt{q.m_hi, q.m_lo, d, dd};   // R = (R^T)^T
   Out og; og.f32 = Gz; og.ld = d; og.bs = dd;
   og.k_mode = 8; og.nterms = split ? 3 : 1;
   og.tile_list = q.tl_k8; og.n_list = q.n_all; og.tile_list2 = q.tl2_k8; og.n_list2 = q.n2_all;
