@@ -108,6 +108,9 @@ void free_all(dq_calib* h) {
   if (h->ev_in) cudaEventDestroy(h->ev_in);
   if (h->ev_out) cudaEventDestroy(h->ev_out);
   if (h->ctx.stream) cudaStreamDestroy(h->ctx.stream);
+  if (h->ctx.side) cudaStreamDestroy(h->ctx.side);
+  if (h->ctx.ev_fork) cudaEventDestroy(h->ctx.ev_fork);
+  if (h->ctx.ev_join) cudaEventDestroy(h->ctx.ev_join);
   delete h;
 }
 
@@ -137,6 +140,7 @@ dq_status fence_in(dq_calib* h) {
   return DQ_OK;
 }
 dq_status fence_out(dq_calib* h) {
+  DQ_CHECK(join_side(h->ctx));
   DQ_CHECK_CUDA(cudaEventRecord(h->ev_out, h->ctx.stream));
   DQ_CHECK_CUDA(cudaStreamWaitEvent(h->user_stream, h->ev_out, 0));
   return DQ_OK;
@@ -239,8 +243,11 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
       } else {
         DQ_CHECK(tc_whip_forward(h->tc, ctx, h->partials));
       }
-      DQ_CHECK(loss_finalize(ctx, h->partials, c.path == DQ_PATH_BF16_TC ? h->tc.n_partials_live : h->n_partials, batch,
-                             inv_n, nullptr, loss_dst));
+      const int n_part = c.path == DQ_PATH_BF16_TC ? h->tc.n_partials_live : h->n_partials;
+      if (n_micro == 1 && !timed)   // (beside the next contraction: the loss is read after the step)
+        DQ_CHECK(on_side(ctx, [&](Ctx& cs) { return loss_finalize(cs, h->partials, n_part, batch, inv_n, nullptr, loss_dst); }));
+      else
+        DQ_CHECK(loss_finalize(ctx, h->partials, n_part, batch, inv_n, nullptr, loss_dst));
     }
     if (timed && a == n_micro - 1) DQ_CHECK_CUDA(cudaEventRecord(h->ev[2], ctx.stream));
     // (a5) Gq = (1/N) X^T G
@@ -269,6 +276,7 @@ dq_status enqueue_step(dq_calib* h, bool timed, const MiniBatch* mb = nullptr) {
     }
   }
   if (timed) DQ_CHECK_CUDA(cudaEventRecord(h->ev[3], ctx.stream));
+  DQ_CHECK(join_side(ctx));   // the checks and the loss of this step are in before the latent may change
   // (a6) Gz = R tril(R^T Gq - Gq^T R, -1) U^-T
   // (a7) Z <- Z - lr Gz  (fused into the backward kernel for 128 x 128 latents)
   const int64_t n_latent = (int64_t)d * d * batch;
@@ -443,6 +451,10 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
   dq_status st = DQ_OK;
   auto A = [&](dq_status s) { if (st == DQ_OK) st = s; };
   if (cudaStreamCreateWithFlags(&h->ctx.stream, cudaStreamNonBlocking) != cudaSuccess) st = DQ_ERR_CUDA;
+  if (st == DQ_OK && (cudaStreamCreateWithFlags(&h->ctx.side, cudaStreamNonBlocking) != cudaSuccess ||
+                      cudaEventCreateWithFlags(&h->ctx.ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                      cudaEventCreateWithFlags(&h->ctx.ev_join, cudaEventDisableTiming) != cudaSuccess))
+    st = DQ_ERR_CUDA;
   if (st == DQ_OK && cudaEventCreateWithFlags(&h->ev_in, cudaEventDisableTiming) != cudaSuccess) st = DQ_ERR_CUDA;
   if (st == DQ_OK && cudaEventCreateWithFlags(&h->ev_out, cudaEventDisableTiming) != cudaSuccess) st = DQ_ERR_CUDA;
   A(dev_alloc(&h->ctx.d_status, 1));

@@ -17,6 +17,11 @@ struct Ctx {
   int64_t launches = 0;
   double mma_flops = 0.0;   // bf16 tensor-core flops issued by the tcgen05 kernels (counted on the host)
   int sm_count = 148;
+  // Optional side branch: small checks and reductions that nothing on the main stream waits for run beside
+  // the next large kernel (on_side) and are ordered back in before their results are needed (join_side).
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  bool side_pending = false;
 };
 
 #define DQ_CHECK_CUDA(expr)                          \
@@ -34,6 +39,29 @@ struct Ctx {
 inline dq_status after_launch(Ctx& ctx) {
   ctx.launches++;
   return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
+}
+
+// Runs launch(ctx) with ctx.stream replaced by the side stream, ordered after everything enqueued on the main
+// stream so far.  Without a side stream the work stays on the main stream.
+template <typename F>
+inline dq_status on_side(Ctx& ctx, F launch) {
+  if (!ctx.side) return launch(ctx);
+  if (cudaEventRecord(ctx.ev_fork, ctx.stream) != cudaSuccess || cudaStreamWaitEvent(ctx.side, ctx.ev_fork, 0) != cudaSuccess)
+    return DQ_ERR_CUDA;
+  cudaStream_t main_stream = ctx.stream;
+  ctx.stream = ctx.side;
+  const dq_status st = launch(ctx);
+  ctx.stream = main_stream;
+  ctx.side_pending = true;
+  return st;
+}
+// Orders the main stream after the side work enqueued so far.
+inline dq_status join_side(Ctx& ctx) {
+  if (!ctx.side_pending) return DQ_OK;
+  ctx.side_pending = false;
+  if (cudaEventRecord(ctx.ev_join, ctx.side) != cudaSuccess || cudaStreamWaitEvent(ctx.stream, ctx.ev_join, 0) != cudaSuccess)
+    return DQ_ERR_CUDA;
+  return DQ_OK;
 }
 
 // Opt-in to more than 48 KB of dynamic shared memory.  The attribute belongs to the (function, device) pair,

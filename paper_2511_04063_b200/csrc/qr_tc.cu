@@ -523,8 +523,8 @@ dq_status qr_forward_incremental_tc(Ctx& ctx, QrWorkspace& ws, QrTcState& q, con
     DQ_CHECK(gemm3(ctx, a, y_tr, d, d, d, batch, o));
   }
   q.w_sel ^= 1;
-  // diag(W) = 1 / diag(U): the same rank and finiteness test
-  return qr_diag_check(ctx, Wf, d, batch);
+  // diag(W) = 1 / diag(U): the same rank and finiteness test (beside the next kernel: only the update waits for it)
+  return on_side(ctx, [&](Ctx& c) { return qr_diag_check(c, Wf, d, batch); });
 }
 
 dq_status qr_forward_fast(Ctx& ctx, QrWorkspace& ws, QrTcState& q, const float* Z, float* R, float* U, int d,
