@@ -190,12 +190,14 @@ __device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, 
 
 // This thread's row of an fp32 matrix in global memory -> operand buffers (hi and, unless negative, lo part).
 __device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* row, int r, int rm_hi, int rm_lo) {
-#pragma unroll 1
-  for (int c = k.c_begin; c < k.c_begin + CHUNKS_PER_THREAD; ++c) {
-    float f[CH];
-    fetch_ch(row + c * CH, f);
+  float f[CHUNKS_PER_THREAD][CH];   // all of the thread's loads in flight before the first is used
+#pragma unroll
+  for (int i = 0; i < CHUNKS_PER_THREAD; ++i) fetch_ch(row + (k.c_begin + i) * CH, f[i]);
+#pragma unroll
+  for (int i = 0; i < CHUNKS_PER_THREAD; ++i) {
+    const int c = k.c_begin + i;
     uint32_t ph[CH / 2], pl[CH / 2];
-    split_ch(f, ph, pl);
+    split_ch(f[i], ph, pl);
     put_rowmajor(k.buf(rm_hi), r, c, ph);
     if (rm_lo >= 0) put_rowmajor(k.buf(rm_lo), r, c, pl);
   }

@@ -1,20 +1,23 @@
 // Fused Whip step for many 128 x 128 rotations (per-head rotations): one kernel computes, per head h
 // and per tile of TT = 64 tokens,
-//   O^T = R_h^T X_t^T   (tcgen05, accumulator in tensor memory)
+//   O^T = R_h^T X_t^T     (tcgen05, accumulator in tensor memory)
 //   e = exp(-|o|), loss partials, G = -sign(o) e   (Eq. 4; epilogue from tensor memory)
-//   Gq_h += X_t^T G_t    (second tcgen05 product: G_t goes from the epilogue's registers into shared
-//                         memory as the K-major operand, the accumulator stays in tensor memory
-//                         for all tiles of the unit)
-// so the rotated activations and dL/dO never reach HBM and X is read exactly once: the second product
-// reads the same token-major tile of X that TMA loaded for the first one, as its MN-major A operand
+//   Gq_h^T += G_t^T X_t    (second tcgen05 product: the epilogue writes bf16 G_t^T back into tensor memory, over
+//                           the part of the O^T accumulator it has just read, and the product takes it from
+//                           there as its A operand; the accumulator stays in tensor memory for all tiles of
+//                           the unit)
+// so the rotated activations and dL/dO never reach HBM or shared memory and X is read exactly once: the second
+// product reads the same token-major tile of X that TMA loaded for the first one, as its MN-major B operand
 // (reduction index = token, 64 consecutive channels per 128-byte row), so no channel-major copy is made.
-// R_h^T stays resident in shared memory for a unit (head, range of token tiles); every unit writes
-// one 128 x 128 fp32 partial of Gq and four loss partials, summed afterwards in a fixed order.
+// Shared-memory bandwidth is what bounds this kernel (operands of both products, the TMA writes), which is why
+// G_t^T does not pass through it.  R_h^T stays resident in shared memory for a unit (head, range of token
+// tiles); every unit writes one 128 x 128 fp32 partial of Gq and its loss partials, summed afterwards in a
+// fixed order.
 //
 // 320 threads: warp 0 TMA producer (R_h^T and the X_t ring), warp 1 MMA issuer, warps 2..9 epilogue (two
-// warps per quarter of the tensor-memory lanes, 32 token columns each).  X_t and G_t are released once the
-// second product of the tile has retired; two O accumulators.  Every wait is bounded
-// (DQ_ERR_TIMEOUT on expiry).
+// warps per quarter of the tensor-memory lanes, 32 token columns each).  X_t and the O^T accumulator that
+// holds G_t^T are released once the second product of the tile has retired; two O^T accumulators.  Every
+// wait is bounded (DQ_ERR_TIMEOUT on expiry).
 #pragma once
 #include "tc_gemm.cuh"
 
@@ -28,13 +31,12 @@ constexpr int KB_BYTES = 128 * BLOCK_K * 2;        // one [128 rows][64 bf16] K-
 constexpr int XKB_BYTES = TT * BLOCK_K * 2;        // one [TT rows][64 bf16] K-major block of X_t: 8 KB
 constexpr int RT_BYTES = 2 * KB_BYTES;             // R_h^T: rows = output channel, K = input channel (128)
 constexpr int XA_BYTES = 2 * XKB_BYTES;            // X_t:   rows = token (TT), K = input channel (two k-blocks)
-constexpr int G_BYTES = KB_BYTES;                  // G_t^T: rows = output channel, K = token
 // Two CTAs share an SM (each under half of its shared memory and half of its tensor memory): while one
 // waits for a load or runs its epilogue the other issues products.  Tiles of 64 tokens keep a CTA at
-// 96 KB: R_h^T, three X_t stages (a tile stays until its second product has retired) and one G_t buffer.
-constexpr int XA_STAGES = 3, G_BUFS = 1;
-constexpr int SMEM_TOTAL = RT_BYTES + XA_STAGES * XA_BYTES + G_BUFS * G_BYTES + 1024 + 1024;
-constexpr uint32_t TMEM_COLS = 256;                // O (2 x TT columns) + Gq (128 columns)
+// 98 KB: R_h^T and four X_t stages (a tile stays until its second product has retired).
+constexpr int XA_STAGES = 4;
+constexpr int SMEM_TOTAL = RT_BYTES + XA_STAGES * XA_BYTES + 1024 + 1024;
+constexpr uint32_t TMEM_COLS = 256;                // O^T (2 x TT columns; G_t^T over half of each) + Gq^T (128 columns)
 constexpr int HEADS_THREADS = 320;
 constexpr int EPI_WARPS = 8;
 
@@ -47,38 +49,52 @@ struct Params {
   int* d_status;
 };
 
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// D (+)= A B^T with A taken from tensor memory: lane = row of A, two bf16 of consecutive k per 32-bit column.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns from registers: thread l writes row (lane base + l).
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __global__ void __launch_bounds__(HEADS_THREADS, 2)
 heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_constant__ CUtensorMap mapX, const Params p) {
   constexpr uint32_t IDESC_O = make_idesc_bf16(TT);     // O^T tile: 128 channels x TT tokens
-  constexpr uint32_t IDESC_Q = make_idesc_bf16(128) | IDESC_A_MN_MAJOR;    // Gq: 128 x 128, A = X_t^T read from the token-major tile
+  constexpr uint32_t IDESC_Q = make_idesc_bf16(128) | IDESC_B_MN_MAJOR;    // Gq^T: 128 x 128, B = X_t^T read from the token-major tile
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t rt_smem = smem_base;
   const uint32_t xa_base = rt_smem + RT_BYTES;
-  const uint32_t g_base = xa_base + XA_STAGES * XA_BYTES;
-  const uint32_t bar_base = g_base + G_BUFS * G_BYTES;
-  constexpr int B_XAF = 0, B_XAE = B_XAF + XA_STAGES, B_TF = B_XAE + XA_STAGES, B_TE = B_TF + 2, B_GF = B_TE + 2, B_GE = B_GF + G_BUFS, B_MISC = B_GE + G_BUFS;
+  const uint32_t bar_base = xa_base + XA_STAGES * XA_BYTES;
+  constexpr int B_XAF = 0, B_XAE = B_XAF + XA_STAGES, B_TF = B_XAE + XA_STAGES, B_TE = B_TF + 2, B_GF = B_TE + 2, B_MISC = B_GF + 2;
   auto xa_full = [&](int s) { return bar_base + 8u * (B_XAF + s); };
   auto xa_empty = [&](int s) { return bar_base + 8u * (B_XAE + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (B_TF + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (B_TE + a); };
-  auto gfull_bar = [&](int g) { return bar_base + 8u * (B_GF + g); };
-  auto gempty_bar = [&](int g) { return bar_base + 8u * (B_GE + g); };
+  auto gfull_bar = [&](int a) { return bar_base + 8u * (B_GF + a); };     // G_t^T written over accumulator a
   const uint32_t rtfull_bar = bar_base + 8u * B_MISC, rtempty_bar = bar_base + 8u * (B_MISC + 1);
   const uint32_t qfull_bar = bar_base + 8u * (B_MISC + 2), qempty_bar = bar_base + 8u * (B_MISC + 3);
   const uint32_t tmem_slot = bar_base + 8u * (B_MISC + 4);
   uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
-  uint8_t* g_ptr = smem_raw + (g_base - smem_u32(smem_raw));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < XA_STAGES; ++s) {
       mbar_init(xa_full(s), 1); mbar_init(xa_empty(s), 1);
     }
-    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), EPI_WARPS); }
-    for (int s = 0; s < G_BUFS; ++s) { mbar_init(gfull_bar(s), EPI_WARPS); mbar_init(gempty_bar(s), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(tfull_bar(s), 1); mbar_init(tempty_bar(s), 1); mbar_init(gfull_bar(s), EPI_WARPS); }
     mbar_init(rtfull_bar, 1); mbar_init(rtempty_bar, 1);
     mbar_init(qfull_bar, 1); mbar_init(qempty_bar, EPI_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -126,7 +142,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      int st1 = 0, st2 = 0, acc = 0, g = 0;
+      int st1 = 0, st2 = 0, acc = 0, g = 0;      // g: accumulator that holds G_t^T of the next second product
       uint32_t ph1 = 0, acc_phase = 0, g_phase = 0, rt_phase = 0, q_phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
@@ -154,7 +170,7 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             if (++st1 == XA_STAGES) { st1 = 0; ph1 ^= 1u; }
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
           }
-          if (i > 0) {    // Gq += X_t^T G_t of tile i - 1
+          if (i > 0) {    // Gq^T += G_t^T X_t of tile i - 1
             const int j = i - 1;
             if (j == 0) {   // the accumulator of the previous unit has been read out
               if (!mbar_wait(qempty_bar, q_phase ^ 1u, p.d_status)) { ok = false; break; }
@@ -162,19 +178,21 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             }
             if (!mbar_wait(gfull_bar(g), g_phase, p.d_status)) { ok = false; break; }
             tc_fence_after();
-            // A = X_t^T (128 channels x 16 tokens per instruction) straight from the token-major tile of stage st2:
-            // 16 tokens = 16 rows of 128 bytes; channels 64..127 sit in the stage's second k-block
+            // A = G_t^T from tensor memory: 16 tokens = 8 columns; each epilogue warp left its 32 tokens at the
+            // start of the 32 accumulator columns it read.  B = X_t^T (128 channels x 16 tokens per instruction)
+            // straight from the token-major tile of stage st2: 16 tokens = 16 rows of 128 bytes; channels 64..127
+            // sit in the stage's second k-block.
             const uint32_t xs = xa_base + st2 * XA_BYTES;
-            const uint32_t gb = g_base + g * G_BYTES;
+            const uint32_t tmem_g = tmem_base + (uint32_t)(g * TT);
 #pragma unroll
             for (int k = 0; k < TT / UMMA_K; ++k)
-              umma_bf16(tmem_q, make_mnmajor_sw128_desc(xs + k * UMMA_K * 128, XKB_BYTES),
-                        make_kmajor_sw128_desc(gb + k * UMMA_K * 2), IDESC_Q, (j > 0 || k > 0) ? 1u : 0u);
+              umma_bf16_ts(tmem_q, tmem_g + (uint32_t)((k >> 1) * 32 + (k & 1) * 8),
+                           make_mnmajor_sw128_desc(xs + k * UMMA_K * 128, XKB_BYTES), IDESC_Q, (j > 0 || k > 0) ? 1u : 0u);
             umma_commit(xa_empty(st2));                  // X_t can be replaced once this product has retired
-            umma_commit(gempty_bar(g));
+            umma_commit(tempty_bar(g));                  // and so can the accumulator that held O^T, then G_t^T
             if (j == nt - 1) umma_commit(qfull_bar);
             if (++st2 == XA_STAGES) { st2 = 0; }
-            if (++g == G_BUFS) { g = 0; g_phase ^= 1u; }
+            if (++g == 2) { g = 0; g_phase ^= 1u; }
           }
         }
       }
@@ -183,10 +201,10 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
     // ------------------------------------------------------------- epilogue (warps 2..9)
     const int q = warp & 3;                    // quarter of the tensor-memory lanes this warp may read
     const int half = (warp - 2) >> 2;          // which 64 of the 128 columns
-    const int row = q * 32 + lane;             // output channel (O^T, G^T) / input channel (Gq)
+    const int row = q * 32 + lane;             // output channel (row of O^T, G^T and Gq^T)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    int acc = 0, g = 0;
-    uint32_t acc_phase = 0, g_phase = 0, q_phase = 0;
+    int acc = 0;
+    uint32_t acc_phase = 0, q_phase = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
       int b, t0, t1;
@@ -196,15 +214,12 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         // ---- Eq. 4 epilogue of O^T
         if (!mbar_wait(tfull_bar(acc), acc_phase, p.d_status)) { ok = false; break; }
         tc_fence_after();
-        uint8_t* gbuf = g_ptr + g * G_BYTES;
         {   // this warp's 32 token columns of the TT-wide tile
           const int c = half;
+          const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(acc * TT + c * 32);
           uint32_t v[32];
-          tmem_ld32(tmem_base + lane_addr + (uint32_t)(acc * TT + c * 32), v);
+          tmem_ld32(taddr, v);
           tmem_ld_wait();
-          tc_fence_before();                     // the accumulator is in registers: the issuer may reuse it
-          __syncwarp();
-          if (lane == 0) mbar_arrive(tempty_bar(acc));
           uint32_t packed[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -217,17 +232,9 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
             const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
             packed[i] = *reinterpret_cast<const uint32_t*>(&h);
           }
-          // (the second product of the previous tile, which reads the G buffer, ran during the arithmetic above)
-          if (!mbar_wait(gempty_bar(g), g_phase ^ 1u, p.d_status)) { ok = false; break; }
-          // tokens 32 c .. 32 c + 31 of row `row`: 16-byte chunks 4 c .. 4 c + 3, stored where the 128-byte
-          // swizzle of a K-major tile expects them
-          uint8_t* rowp = gbuf + row * 128;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int chunk = (c * 4 + i) ^ (row & 7);
-            *reinterpret_cast<uint4*>(rowp + chunk * 16) =
-                make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-          }
+          // tokens 32 c .. 32 c + 31 of row `row` as 16 columns of bf16 pairs, over the first half of the 32
+          // columns this warp has just read (no other warp reads or writes them)
+          tmem_st16(taddr, packed);
           if (p.Gt) {
             uint4* dst = reinterpret_cast<uint4*>(p.Gt + ((int64_t)b * 128 + row) * p.n_tokens + (int64_t)t * TT + c * 32);
 #pragma unroll
@@ -235,29 +242,27 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
               dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
           }
         }
+        tmem_st_wait();
         tc_fence_before();
-        fence_async_smem();                    // the tensor core reads G through the async proxy
         __syncwarp();
-        if (lane == 0) mbar_arrive(gfull_bar(g));
+        if (lane == 0) mbar_arrive(gfull_bar(acc));
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-        if (++g == G_BUFS) { g = 0; g_phase ^= 1u; }
       }
       if (!ok) break;
       // partial Gq of the unit
       if (!mbar_wait(qfull_bar, q_phase, p.d_status)) { ok = false; break; }
       q_phase ^= 1u;
       tc_fence_after();
-      float* dst_row = p.part + ((int64_t)u * 128 + row) * 128;
+      // the accumulator holds Gq^T (lane = output channel, column = input channel): a warp's store of one
+      // column is 32 consecutive floats of a row of Gq
+      float* dst_col = p.part + (int64_t)u * 128 * 128 + row;
 #pragma unroll 1
       for (int c = 2 * half; c < 2 * half + 2; ++c) {
         uint32_t v[32];
         tmem_ld32(tmem_q + lane_addr + (uint32_t)(c * 32), v);
         tmem_ld_wait();
-        float4* dst = reinterpret_cast<float4*>(dst_row + c * 32);
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-          dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
-                               __uint_as_float(v[4 * i + 3]));
+        for (int i = 0; i < 32; ++i) dst_col[(c * 32 + i) * 128] = __uint_as_float(v[i]);
       }
       tc_fence_before();
       __syncwarp();
