@@ -14,8 +14,9 @@
 // tiles); every unit writes one 128 x 128 fp32 partial of Gq and its loss partials, summed afterwards in a
 // fixed order.
 //
-// 320 threads: warp 0 TMA producer (R_h^T and the X_t ring), warp 1 MMA issuer, warps 2..9 epilogue (two
-// warps per quarter of the tensor-memory lanes, 32 token columns each).  X_t and the O^T accumulator that
+// 352 threads: warp 0 TMA producer (R_h^T and the X_t ring), warp 1 issuer of the first product, warps 2..9
+// epilogue (two warps per quarter of the tensor-memory lanes, 32 token columns each), warp 10 issuer of the
+// second product.  X_t and the O^T accumulator that
 // holds G_t^T are released once the second product of the tile has retired; two O^T accumulators.  Every
 // wait is bounded (DQ_ERR_TIMEOUT on expiry).
 #pragma once
@@ -37,8 +38,9 @@ constexpr int XA_BYTES = 2 * XKB_BYTES;            // X_t:   rows = token (TT), 
 constexpr int XA_STAGES = 4;
 constexpr int SMEM_TOTAL = RT_BYTES + XA_STAGES * XA_BYTES + 1024 + 1024;
 constexpr uint32_t TMEM_COLS = 256;                // O^T (2 x TT columns; G_t^T over half of each) + Gq^T (128 columns)
-constexpr int HEADS_THREADS = 320;
 constexpr int EPI_WARPS = 8;
+constexpr int Q_WARP = 2 + EPI_WARPS;                // warp of the second product's issuer
+constexpr int HEADS_THREADS = 32 * (Q_WARP + 1);
 
 struct Params {
   int batch, tiles_per_head, splits;   // units = batch * splits; unit u = head u / splits, slice u % splits
@@ -140,10 +142,19 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------- MMA issuer
+    // ------------------------------------------------------------- issuer of the first product, O^T = R_h^T X_t^T
     if (lane == 0) {
-      int st1 = 0, st2 = 0, acc = 0, g = 0;      // g: accumulator that holds G_t^T of the next second product
-      uint32_t ph1 = 0, acc_phase = 0, g_phase = 0, rt_phase = 0, q_phase = 0;
+      // descriptors of R_h^T (fixed) and of stage 0 of the X_t ring; a later stage or k-step adds its byte
+      // offset / 16 to the address field
+      uint64_t rd[2 * (BLOCK_K / UMMA_K)];
+#pragma unroll
+      for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+          rd[kb * (BLOCK_K / UMMA_K) + k] = make_kmajor_sw128_desc(rt_smem + kb * KB_BYTES + k * UMMA_K * 2);
+      const uint64_t x0 = make_kmajor_sw128_desc(xa_base);
+      int st1 = 0, acc = 0;
+      uint32_t ph1 = 0, acc_phase = 0, rt_phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
         int b, t0, t1;
@@ -151,49 +162,61 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
         const int nt = t1 - t0;
         if (!mbar_wait(rtfull_bar, rt_phase, p.d_status)) break;
         rt_phase ^= 1u;
-        tc_fence_after();
-        for (int i = 0; i <= nt && ok; ++i) {
-          if (i < nt) {   // O^T of tile i
-            if (!mbar_wait(xa_full(st1), ph1, p.d_status)) { ok = false; break; }
-            if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t xa = xa_base + st1 * XA_BYTES;
-            const uint32_t tmem_o = tmem_base + (uint32_t)(acc * TT);
+        for (int i = 0; i < nt; ++i) {
+          if (!mbar_wait(xa_full(st1), ph1, p.d_status)) { ok = false; break; }
+          // the accumulator is free once the second product of the tile that used it last has retired
+          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, p.d_status)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t xd = x0 + (uint64_t)((st1 * XA_BYTES) >> 4);
+          const uint32_t tmem_o = tmem_base + (uint32_t)(acc * TT);
 #pragma unroll
-            for (int kb = 0; kb < 2; ++kb)
+          for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
-              for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                umma_bf16(tmem_o, make_kmajor_sw128_desc(rt_smem + kb * KB_BYTES + k * UMMA_K * 2),
-                          make_kmajor_sw128_desc(xa + kb * XKB_BYTES + k * UMMA_K * 2), IDESC_O, (kb > 0 || k > 0) ? 1u : 0u);
-            umma_commit(tfull_bar(acc));
-            if (i == nt - 1) umma_commit(rtempty_bar);   // R_h^T may be replaced once these products retire
-            if (++st1 == XA_STAGES) { st1 = 0; ph1 ^= 1u; }
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+              umma_bf16(tmem_o, rd[kb * (BLOCK_K / UMMA_K) + k], xd + (uint64_t)((kb * XKB_BYTES + k * UMMA_K * 2) >> 4), IDESC_O,
+                        (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(tfull_bar(acc));
+          if (i == nt - 1) umma_commit(rtempty_bar);   // R_h^T may be replaced once these products retire
+          if (++st1 == XA_STAGES) { st1 = 0; ph1 ^= 1u; }
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == Q_WARP) {
+    // ------------------------------------------------------------- issuer of the second product, Gq^T += G_t^T X_t
+    // (a thread of its own: one thread issues a product of this size no faster than every 60 cycles or so, and
+    // the two streams of products do not depend on each other's order)
+    if (lane == 0) {
+      const uint64_t xm0 = make_mnmajor_sw128_desc(xa_base, XKB_BYTES);
+      int st2 = 0, g = 0;                         // g: accumulator that holds G_t^T of the next product
+      uint32_t g_phase = 0, q_phase = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        int b, t0, t1;
+        unit_range(u, b, t0, t1);
+        const int nt = t1 - t0;
+        for (int j = 0; j < nt; ++j) {
+          if (j == 0) {   // the accumulator of the previous unit has been read out
+            if (!mbar_wait(qempty_bar, q_phase ^ 1u, p.d_status)) { ok = false; break; }
+            q_phase ^= 1u;
           }
-          if (i > 0) {    // Gq^T += G_t^T X_t of tile i - 1
-            const int j = i - 1;
-            if (j == 0) {   // the accumulator of the previous unit has been read out
-              if (!mbar_wait(qempty_bar, q_phase ^ 1u, p.d_status)) { ok = false; break; }
-              q_phase ^= 1u;
-            }
-            if (!mbar_wait(gfull_bar(g), g_phase, p.d_status)) { ok = false; break; }
-            tc_fence_after();
-            // A = G_t^T from tensor memory: 16 tokens = 8 columns; each epilogue warp left its 32 tokens at the
-            // start of the 32 accumulator columns it read.  B = X_t^T (128 channels x 16 tokens per instruction)
-            // straight from the token-major tile of stage st2: 16 tokens = 16 rows of 128 bytes; channels 64..127
-            // sit in the stage's second k-block.
-            const uint32_t xs = xa_base + st2 * XA_BYTES;
-            const uint32_t tmem_g = tmem_base + (uint32_t)(g * TT);
+          if (!mbar_wait(gfull_bar(g), g_phase, p.d_status)) { ok = false; break; }
+          tc_fence_after();
+          // A = G_t^T from tensor memory: 16 tokens = 8 columns; each epilogue warp left its 32 tokens at the
+          // start of the 32 accumulator columns it read.  B = X_t^T (128 channels x 16 tokens per instruction)
+          // straight from the token-major tile of stage st2: 16 tokens = 16 rows of 128 bytes; channels 64..127
+          // sit in the stage's second k-block.
+          const uint64_t xd = xm0 + (uint64_t)((st2 * XA_BYTES) >> 4);
+          const uint32_t tmem_g = tmem_base + (uint32_t)(g * TT);
 #pragma unroll
-            for (int k = 0; k < TT / UMMA_K; ++k)
-              umma_bf16_ts(tmem_q, tmem_g + (uint32_t)((k >> 1) * 32 + (k & 1) * 8),
-                           make_mnmajor_sw128_desc(xs + k * UMMA_K * 128, XKB_BYTES), IDESC_Q, (j > 0 || k > 0) ? 1u : 0u);
-            umma_commit(xa_empty(st2));                  // X_t can be replaced once this product has retired
-            umma_commit(tempty_bar(g));                  // and so can the accumulator that held O^T, then G_t^T
-            if (j == nt - 1) umma_commit(qfull_bar);
-            if (++st2 == XA_STAGES) { st2 = 0; }
-            if (++g == 2) { g = 0; g_phase ^= 1u; }
-          }
+          for (int k = 0; k < TT / UMMA_K; ++k)
+            umma_bf16_ts(tmem_q, tmem_g + (uint32_t)((k >> 1) * 32 + (k & 1) * 8), xd + (uint64_t)((k * UMMA_K * 128) >> 4), IDESC_Q,
+                         (j > 0 || k > 0) ? 1u : 0u);
+          umma_commit(xa_empty(st2));                  // X_t can be replaced once this product has retired
+          umma_commit(tempty_bar(g));                  // and so can the accumulator that held O^T, then G_t^T
+          if (j == nt - 1) umma_commit(qfull_bar);
+          if (++st2 == XA_STAGES) { st2 = 0; }
+          if (++g == 2) { g = 0; g_phase ^= 1u; }
         }
       }
     }
