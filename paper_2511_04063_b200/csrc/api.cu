@@ -500,6 +500,8 @@ dq_status dq_calib_init(dq_calib_t** out, const dq_calib_config* cfg, const void
     h->tc5 = (st == DQ_OK);
   }
   A(dev_alloc(&h->partials, (int64_t)batch * (h->n_partials > 0 ? h->n_partials : 1)));
+  // (the per-head fused kernel writes only the slots its launch shape uses and relies on the others being zero)
+  if (st == DQ_OK && cudaMemsetAsync(h->partials, 0, sizeof(float) * (size_t)batch * (h->n_partials > 0 ? h->n_partials : 1), h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
   if (st == DQ_OK && cudaMemsetAsync(h->ctx.d_status, 0, sizeof(int), h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
   if (st == DQ_OK && cudaMemcpyAsync(h->Z, d_Z0, sizeof(float) * dd, cudaMemcpyDeviceToDevice, h->ctx.stream) != cudaSuccess) st = DQ_ERR_CUDA;
   if (st == DQ_OK && h->fast_qr && !h->small128) {

@@ -71,7 +71,7 @@ __global__ void bounded_wait_probe_kernel(uint64_t limit_ns, int* d_status, uint
 }
 
 struct Maps {
-  CUtensorMap rt, x, x128, x64, xmn, gt128, gt256;
+  CUtensorMap rt, x, x128, xmn, gt128, gt256;
 };
 
 }  // namespace
@@ -126,19 +126,25 @@ dq_status tc_init(TcState& tc, Ctx& ctx, const dq_calib_config& cfg, const void*
   tc.ldx = ldx;
   DQ_CHECK(tch::make_map(&m->x, tc.X, d, N, batch, ldx, N * ldx, 256));
   DQ_CHECK(tch::make_map(&m->x128, tc.X, d, N, batch, ldx, N * ldx, 128));
-  DQ_CHECK(tch::make_map(&m->x64, tc.X, d, N, batch, ldx, N * ldx, heads::TT));
   // X again, in boxes of 64 tokens x 64 channels: the MN-major A operand (X^T) of Gq = X^T G
   DQ_CHECK(tch::make_map(&m->xmn, tc.X, d, N, batch, ldx, N * ldx, tc::BLOCK_K));
   DQ_CHECK(tch::make_map(&m->gt128, tc.Gt, N, d, batch, N, N * d, 128));
   DQ_CHECK(tch::make_map(&m->gt256, tc.Gt, N, d, batch, N, N * d, 256));
-  if (d == 128) {   // per-head rotations: fused kernel, units = (head, range of token tiles), two CTAs per SM
+  if (d == 128) {   // per-head rotations: fused kernel, one CTA per SM over equal ranges of the tile sequence
     const int tiles_per_head = (int)(N / heads::TT);
-    int sp = 2 * ctx.sm_count / batch;
-    if (sp > tiles_per_head) sp = tiles_per_head;
-    if (sp < 1) sp = 1;
+    const int64_t total = (int64_t)batch * tiles_per_head;
+    const int64_t grid = total < ctx.sm_count ? total : ctx.sm_count;
+    // partial slots per head = the most CTAs whose ranges meet any one head (its unused slots stay zero)
+    int sp = 1;
+    for (int b = 0; b < batch; ++b) {
+      const int first = heads::range_owner((int64_t)b * tiles_per_head, total, grid);
+      const int last = heads::range_owner((int64_t)(b + 1) * tiles_per_head - 1, total, grid);
+      if (last - first + 1 > sp) sp = last - first + 1;
+    }
     tc.splits = sp;
-    if (cudaMalloc((void**)&tc.heads_part, sizeof(float) * (size_t)batch * sp * 128 * 128) != cudaSuccess)
-      return DQ_ERR_ALLOC;
+    const size_t part_bytes = sizeof(float) * (size_t)batch * sp * 128 * 128;
+    if (cudaMalloc((void**)&tc.heads_part, part_bytes) != cudaSuccess) return DQ_ERR_ALLOC;
+    DQ_CHECK_CUDA(cudaMemsetAsync(tc.heads_part, 0, part_bytes, ctx.stream));
     if (cudaFuncSetAttribute(heads::heads_whip_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              heads::SMEM_TOTAL) != cudaSuccess)
       return DQ_ERR_CUDA;
@@ -171,12 +177,12 @@ dq_status tc_whip_forward(TcState& tc, Ctx& ctx, float* partials) {
   if (tc.fused) {
     Maps* mm = reinterpret_cast<Maps*>(tc.maps);
     heads::Params hp{};
-    hp.batch = tc.batch; hp.tiles_per_head = (int)(tc.n_tokens / heads::TT); hp.splits = tc.splits;
+    hp.batch = tc.batch; hp.tiles_per_head = (int)(tc.n_tokens / heads::TT); hp.slots = tc.splits;
     hp.n_tokens = tc.n_tokens; hp.part = tc.heads_part; hp.partials = partials;
     hp.Gt = tc.keep_g ? tc.Gt : nullptr; hp.d_status = ctx.d_status;
-    const int units = tc.batch * tc.splits;
-    const int grid = units < 2 * ctx.sm_count ? units : 2 * ctx.sm_count;
-    heads::heads_whip_kernel<<<grid, heads::HEADS_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x64, hp);
+    const int64_t total = (int64_t)tc.batch * hp.tiles_per_head;
+    const int grid = (int)(total < ctx.sm_count ? total : ctx.sm_count);   // (the slots were sized for this grid)
+    heads::heads_whip_kernel<<<grid, heads::HEADS_THREADS, heads::SMEM_TOTAL, ctx.stream>>>(mm->rt, mm->x128, hp);
     tc.n_partials_live = tc.splits * heads::EPI_WARPS;
     tc.fused_valid = true;
     ctx.mma_flops += 2.0 * (double)tc.n_tokens * tc.d * tc.d * tc.batch;   // the second product runs here too
