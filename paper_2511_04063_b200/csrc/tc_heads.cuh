@@ -264,16 +264,24 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
           tmem_ld32(taddr, v);
           tmem_ld_wait();
           uint32_t packed[16];
+          float amin0 = 1.f, amin1 = 1.f;       // smallest |o| of the 32: dL/do is 0, not -+1, where o is exactly 0
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float o0 = __uint_as_float(v[2 * i]), o1 = __uint_as_float(v[2 * i + 1]);
             const float e0 = fast_exp_neg_abs(o0), e1 = fast_exp_neg_abs(o1);
             esum += e0 + e1;
-            // (an exact zero is not rare: at a Hadamard start o is a signed sum of bf16 values times one constant)
-            const float g0 = (o0 == 0.f) ? 0.f : copysignf(e0, -o0);
-            const float g1 = (o1 == 0.f) ? 0.f : copysignf(e1, -o1);
-            const __nv_bfloat162 h = __floats2bfloat162_rn(g0, g1);
+            amin0 = fminf(amin0, fabsf(o0)); amin1 = fminf(amin1, fabsf(o1));
+            const __nv_bfloat162 h = __floats2bfloat162_rn(copysignf(e0, -o0), copysignf(e1, -o1));
             packed[i] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+          // (an exact zero is not rare at a Hadamard start, where o is a signed sum of bf16 values times one
+          // constant; everywhere else it is, so the per-element test stays out of the loop above)
+          if (fminf(amin0, amin1) == 0.f) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              if (__uint_as_float(v[2 * i]) == 0.f) packed[i] &= 0xFFFF0000u;
+              if (__uint_as_float(v[2 * i + 1]) == 0.f) packed[i] &= 0x0000FFFFu;
+            }
           }
           // tokens 32 cg .. 32 cg + 31 of row `row` as 16 columns of bf16 pairs, over the first half of the 32
           // columns this warp has just read (no other warp reads or writes them)
