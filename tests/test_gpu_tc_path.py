@@ -254,11 +254,12 @@ def test_rotate_apply_bf16(n, d):
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-2
 
 
-@pytest.mark.parametrize("batch,n", [(4, 2048), (160, 256), (3, 768)])
+@pytest.mark.parametrize("batch,n", [(4, 2048), (160, 256), (3, 768), (40, 4096)])
 def test_fused_per_head_kernel_with_and_without_stored_gradient(batch, n):
     """d = 128: one kernel computes O, Eq. 4, dL/dO and X^T dL/dO with dL/dO kept on chip.  Storing dL/dO
     as well (what the other tests switch on to read it) must not change any result; more heads than SMs
-    makes every CTA run several units back to back, 768 tokens gives an uneven split of the token tiles."""
+    makes every CTA run several units back to back, 768 tokens gives an uneven split of the token tiles, and
+    40 heads of 32 tiles give every CTA a range of eight or nine tiles that may end inside a head."""
     w = small("c3_heads", d=128, n_tokens=n, batch=batch)
     outs = []
     for keep in (True, False):
