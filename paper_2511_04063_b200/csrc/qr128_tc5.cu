@@ -149,8 +149,10 @@ struct Tc5 {
 // its accumulator row.  g: the same chunk of the fp32 row `grow` in global memory (nullable; fetched one chunk
 // ahead, the first one while the MMAs run); x0 / x1: the same chunk of the matrices kept in tensor memory at
 // columns t0 / t1 (0: none).  Returns false if the wait gave up (for all threads alike).
+// pre (nullable): the thread's part of that row when the caller holds it in registers already.
 template <typename Issue, typename Body>
-__device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, uint32_t t0, uint32_t t1, Body body) {
+__device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, uint32_t t0, uint32_t t1, Body body,
+                                        const float (*pre)[CH] = nullptr) {
   tmem_ld_wait();
   tmem_st_wait();
   tc_fence_before();
@@ -163,7 +165,7 @@ __device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, 
   }
   const int c_begin = k.c_begin;
   float ga[CH], gb[CH];
-  fetch_ch(grow ? grow + c_begin * CH : nullptr, ga);
+  if (!pre) fetch_ch(grow ? grow + c_begin * CH : nullptr, ga);
   const bool done = mbar_wait(k.bar, k.parity, k.d_status);
   k.parity ^= 1u;
   tc_fence_after();
@@ -180,6 +182,11 @@ __device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, 
   };
 #pragma unroll 1
   for (int c = c_begin; c < c_begin + CHUNKS_PER_THREAD; c += 2) {
+    if (pre) {
+      one(c, pre[c - c_begin]);
+      one(c + 1, pre[c + 1 - c_begin]);
+      continue;
+    }
     fetch_ch(grow ? grow + (c + 1) * CH : nullptr, gb);
     one(c, ga);
     if (c + 2 < c_begin + CHUNKS_PER_THREAD) fetch_ch(grow ? grow + (c + 2) * CH : nullptr, ga);
@@ -189,8 +196,10 @@ __device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, 
 }
 
 // This thread's row of an fp32 matrix in global memory -> operand buffers (hi and, unless negative, lo part).
-__device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* row, int r, int rm_hi, int rm_lo) {
-  float f[CHUNKS_PER_THREAD][CH];   // all of the thread's loads in flight before the first is used
+// f: the values stay with the caller.
+__device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* row, int r, int rm_hi, int rm_lo,
+                                                     float (&f)[CHUNKS_PER_THREAD][CH]) {
+  // all of the thread's loads in flight before the first is used
 #pragma unroll
   for (int i = 0; i < CHUNKS_PER_THREAD; ++i) fetch_ch(row + (k.c_begin + i) * CH, f[i]);
 #pragma unroll
@@ -201,6 +210,10 @@ __device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* 
     put_rowmajor(k.buf(rm_hi), r, c, ph);
     if (rm_lo >= 0) put_rowmajor(k.buf(rm_lo), r, c, pl);
   }
+}
+__device__ __forceinline__ void load_row_to_operands(const Tc5& k, const float* row, int r, int rm_hi, int rm_lo) {
+  float f[CHUNKS_PER_THREAD][CH];
+  load_row_to_operands(k, row, r, rm_hi, rm_lo, f);
 }
 
 __device__ __forceinline__ float phi(float s, int row, int col) {
@@ -440,9 +453,10 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
     // W <- W + W Y  (W row-major -> 0, 5: T is no longer needed)
     float dv = NAN;                     // the diagonal entry, in the thread whose chunks hold it
     if (ok) {
-      load_row_to_operands(k, Wrow, r, 0, 5);
+      float wrow[CHUNKS_PER_THREAD][CH];      // read once: the operands are made from it and the sum below starts from it
+      load_row_to_operands(k, Wrow, r, 0, 5, wrow);
       ok = product(k, [&]() { if (big) k.mma3(0, 5, 3, 4, false, true); else k.mma(0, 3, false, false, false, true); },
-                   Wrow, 0, 0,
+                   nullptr, 0, 0,
                    [&](int c, V v, F w, F, F) {
                      float f[CH];
 #pragma unroll
@@ -451,7 +465,7 @@ __global__ void __launch_bounds__(TC5_THREADS, 1) qr128_step_tc5_kernel(const Tc
                        if (CH * c + i == r) dv = f[i];
                      }
                      store_ch(Wrow + c * CH, f);
-                   });
+                   }, wrow);
     }
     if (ok) {   // rank / finiteness test on diag(W) = 1 / diag(U)
       const bool owner = (r / CH) >= k.c_begin && (r / CH) < k.c_begin + CHUNKS_PER_THREAD;
