@@ -128,7 +128,7 @@ struct Tc5 {
     const uint32_t idesc = make_idesc_bf16(N5) | (negate_a ? IDESC_NEGATE_A : 0u) | (at ? IDESC_A_MN_MAJOR : 0u) |
                            (bt ? IDESC_B_MN_MAJOR : 0u);
     const uint32_t sa = smem_u + a * PART_BYTES, sb = smem_u + b * PART_BYTES;
-#pragma unroll
+#pragma unroll 1
     for (int s = 0; s < N5 / UMMA_K; ++s) {
       const uint32_t kmaj = (uint32_t)((s >> 2) * KBLK_BYTES + (s & 3) * UMMA_K * 2), mnmaj = (uint32_t)(s * UMMA_K * 128);
       umma_bf16(tmem, at ? make_mnmajor_sw128_desc(sa + mnmaj, KBLK_BYTES) : make_kmajor_sw128_desc(sa + kmaj),
@@ -181,16 +181,16 @@ __device__ __forceinline__ bool product(Tc5& k, Issue issue, const float* grow, 
     body(c, v, g, x0, x1);
   };
 #pragma unroll 1
-  for (int c = c_begin; c < c_begin + CHUNKS_PER_THREAD; c += 2) {
+  for (int c = c_begin; c < c_begin + CHUNKS_PER_THREAD; ++c) {   // (one copy of the body: the kernel's code is fetched cold on every launch)
     if (pre) {
-      one(c, pre[c - c_begin]);
-      one(c + 1, pre[c + 1 - c_begin]);
-      continue;
+#pragma unroll
+      for (int i = 0; i < CH; ++i) ga[i] = (c == c_begin) ? pre[0][i] : pre[1][i];
+    } else if (c > c_begin) {
+#pragma unroll
+      for (int i = 0; i < CH; ++i) ga[i] = gb[i];
     }
-    fetch_ch(grow ? grow + (c + 1) * CH : nullptr, gb);
+    if (!pre && c + 1 < c_begin + CHUNKS_PER_THREAD) fetch_ch(grow ? grow + (c + 1) * CH : nullptr, gb);
     one(c, ga);
-    if (c + 2 < c_begin + CHUNKS_PER_THREAD) fetch_ch(grow ? grow + (c + 2) * CH : nullptr, ga);
-    one(c + 1, gb);
   }
   return true;
 }
