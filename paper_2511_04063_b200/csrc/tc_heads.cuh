@@ -142,6 +142,9 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
       int stage = 0;
       uint32_t phase = 0, rt_phase = 0;
       bool ok = true;
+      // X passes through once: first out of the L2, so that the latents, rotations and partial sums of the step's
+      // other kernels (and their code) stay there
+      const uint64_t x_policy = l2_evict_first_policy();
       for (int64_t g = g_begin; g < g_end && ok;) {
         int b, t0, t1, slot;
         segment(g, b, t0, t1, slot);
@@ -154,8 +157,8 @@ heads_whip_kernel(const __grid_constant__ CUtensorMap mapRt, const __grid_consta
           if (!mbar_wait(xa_empty(stage), phase ^ 1u, p.d_status)) { ok = false; break; }
           mbar_expect_tx(xa_full(stage), XA_BYTES);
           const uint32_t xa = xa_base + stage * XA_BYTES;
-          tma_load_3d(xa, &mapX, xa_full(stage), 0, t * TT, b);
-          tma_load_3d(xa + XKB_BYTES, &mapX, xa_full(stage), BLOCK_K, t * TT, b);
+          tma_load_3d_hint(xa, &mapX, xa_full(stage), 0, t * TT, b, x_policy);
+          tma_load_3d_hint(xa + XKB_BYTES, &mapX, xa_full(stage), BLOCK_K, t * TT, b, x_policy);
           if (++stage == XA_STAGES) { stage = 0; phase ^= 1u; }
         }
         g += t1 - t0;
