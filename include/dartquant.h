@@ -291,7 +291,9 @@ enum {
   DQ_BUF_GZ = 3,       /* fp32 [batch][d][d]  dL/dZ                                */
   DQ_BUF_G = 4,        /* dL/dO without the 1/N factor: fp32 [batch][N][d] (fp32 path)
                           or bf16 channel-major [batch][d][N] (tensor-core path)   */
-  DQ_BUF_PARTIALS = 5, /* fp32 per-tile loss partial sums of the last step         */
+  DQ_BUF_PARTIALS = 5, /* fp32 loss partial sums of the last step, a fixed number per problem: one set per
+                          output tile (d = 128 on the tensor-core path: per range of token tiles that one
+                          CTA covers; entries no CTA writes stay zero)             */
   DQ_BUF_Z = 6,        /* fp32 [batch][d][d]  current latent                       */
   DQ_BUF_OPT_M = 7,    /* fp32 [batch][d][d]  first moment / velocity (NULL for DQ_SGD)  */
   DQ_BUF_OPT_V = 8,    /* fp32 [batch][d][d]  second moment (DQ_ADAM only)         */
