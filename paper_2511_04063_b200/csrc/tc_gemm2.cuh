@@ -112,10 +112,7 @@ __global__ void __launch_bounds__(pair_threads<EPI>(), 1)
 tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapB_lo,
                 const Params p) {
-  if (p.run_if || p.run_unless) {   // (the flags are the previous kernels' results: see the wait below)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    if ((p.run_if && *p.run_if == 0) || (p.run_unless && *p.run_unless != 0)) return;   // uniform over the grid (both CTAs of every pair)
-  }
+  if ((p.run_if && *p.run_if == 0) || (p.run_unless && *p.run_unless != 0)) return;   // uniform over the grid (both CTAs of every pair)
   using L = PairSmem<NTERMS>;
   constexpr int STAGES = L::STAGES;
   constexpr int STAGE_BYTES = L::STAGE_BYTES;
@@ -151,12 +148,6 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
   cluster_sync_all();                               // both CTAs' barriers exist before any remote arrival
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
-
-  // The kernel is launched with programmatic stream serialisation: everything above (barriers, tensor memory, the
-  // fetch of its own code) may run while the previous kernel of the stream is finishing.  From here on that kernel's
-  // results are needed (operands, device flags) and its inputs may be overwritten; the next kernel may set itself up.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int tiles_per_batch = p.tile_list ? p.n_list : p.m_blocks * p.n_blocks;
   auto tile_of = [&](int r, int& mb, int& nb) {

@@ -71,13 +71,10 @@ dq_status launch_gemm2(Ctx& ctx, const CUtensorMap& a, const CUtensorMap& b, con
   cfg.blockDim = dim3(tc2::pair_threads<EPI>(), 1, 1);
   cfg.dynamicSmemBytes = SMEM;
   cfg.stream = ctx.stream;
-  cudaLaunchAttribute at[2];
+  cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  // the kernel may be set up while the stream's previous kernel finishes; it waits for that kernel itself
-  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at; cfg.numAttrs = 2;
+  cfg.attrs = at; cfg.numAttrs = 1;
   if (cudaLaunchKernelEx(&cfg, kern, a, b, alo, blo, p) != cudaSuccess) return DQ_ERR_CUDA;
   return after_launch(ctx);
 }
