@@ -33,7 +33,7 @@ UNIT = "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic (bytes read + written) of one launch of the roofline kernel, from an ncu capture of
 # that kernel on the named workload; None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"c2_7b": 312.0e6}
+NCU_TRAFFIC_BYTES = {"c2_7b": 307.4e6}
 NCU_TRAFFIC_BYTES_HEADS = {"c3_heads": 138.9e6}
 
 
