@@ -254,12 +254,13 @@ def test_rotate_apply_bf16(n, d):
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-2
 
 
-@pytest.mark.parametrize("batch,n", [(4, 2048), (160, 256), (3, 768), (40, 4096)])
+@pytest.mark.parametrize("batch,n", [(4, 2048), (160, 256), (3, 768), (40, 4096), (400, 256), (37, 1280)])
 def test_fused_per_head_kernel_with_and_without_stored_gradient(batch, n):
     """d = 128: one kernel computes O, Eq. 4, dL/dO and X^T dL/dO with dL/dO kept on chip.  Storing dL/dO
     as well (what the other tests switch on to read it) must not change any result; more heads than SMs
     makes every CTA run several units back to back, 768 tokens gives an uneven split of the token tiles, and
-    40 heads of 32 tiles give every CTA a range of eight or nine tiles that may end inside a head."""
+    40 heads of 32 tiles give every CTA a range of eight or nine tiles that may end inside a head; 400 heads of 2
+    tiles make a CTA's range cross three or four heads, 37 heads of 10 tiles share nothing with the grid size."""
     w = small("c3_heads", d=128, n_tokens=n, batch=batch)
     outs = []
     for keep in (True, False):
